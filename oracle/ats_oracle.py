@@ -1,0 +1,401 @@
+"""CPU oracle for the block-quantized per-tensor forward path and its placement.
+
+TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, fp64 statement of what
+the CUDA library computes.  Only the test-suite, the smoke check and the
+benchmark's CPU-baseline leg may import it; the product never does.  It shares
+no code with the CUDA path and does not import the package.
+
+What it follows
+---------------
+The paper schedules *tensors*: each weight tensor is one operator executed on
+the backend that holds (or receives) it (Section 3, Section 4.3.1); a GPU memory
+budget M and a placement b decide which tensors are resident (Section 4.3.2,
+the placement objective and Algorithm 1); the others sit in pinned host memory
+and are moved into temporary GPU buffers on a transfer stream (Section 4.2.1,
+4.2.2), and for MoE operators only the experts the current tokens selected are
+moved (Section 4.2.2, Section 4.4.1).  The paper inherits the operator
+arithmetic itself from its host framework and never states it; the formulas
+below are therefore the workload definition's ("signed 4-bit codes in blocks of
+32 along K with one fp16 scale per block, fp32 accumulation, fp16 output",
+RMSNorm, rotary embedding, grouped-query attention, SwiGLU, softmax top-k
+routing with ties to the lower index), written as their textbook definitions.
+
+Pins (tests/test_oracle_*.py): exact rational arithmetic on tiny shapes,
+one-hot / all-ones closed forms, linearity, zero-scale blocks, RoPE identities,
+attention special cases, sort-based top-k, 2^n brute force of the placement
+objective, prefill == sequential decode.  No function here is "parity unpinned".
+
+Conventions: fp64 everywhere; ``rn16`` (IEEE round-to-nearest-even to binary16,
+subnormals kept) is applied only at the edges named in ``edges`` (the numerics
+contract the library publishes), at K/V cache writes and at the layer output.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+BLOCK = 32
+
+# Edges of a decoder layer at which a value may be rounded to fp16 (bit i of the contract mask).
+EDGES = ("h", "q", "k", "v", "q_rot", "a", "o", "x1", "h2", "g", "u", "act", "d")
+EDGE_BIT = {name: 1 << i for i, name in enumerate(EDGES)}
+WEIGHT_EXACT, WEIGHT_F16 = 0, 1
+
+
+def edges_from_mask(mask: int):
+    return frozenset(n for n in EDGES if mask & EDGE_BIT[n])
+
+
+def rn16(a):
+    """Round fp64 values to the nearest fp16 (ties to even, subnormals kept); returned as fp64."""
+    with np.errstate(over="ignore"):
+        return np.asarray(a, dtype=np.float64).astype(np.float16).astype(np.float64)
+
+
+def _edge(val, name, edges):
+    return rn16(val) if name in edges else val
+
+
+# --------------------------------------------------------------------------------------
+# a1: block dequantization
+# --------------------------------------------------------------------------------------
+def unpack_codes(packed: np.ndarray) -> np.ndarray:
+    """Interchange bytes ``[..., K/2]`` -> signed codes int8 ``[..., K]``.
+
+    Byte j holds code 2j in bits 0..3 and code 2j+1 in bits 4..7, each a
+    two's-complement nibble (0..7 -> 0..7, 8..15 -> -8..-1).
+    """
+    p = np.asarray(packed, dtype=np.uint8)
+    lo = (p & 0x0F).astype(np.int8)
+    hi = (p >> 4).astype(np.int8)
+    lo = np.where(lo >= 8, lo - 16, lo).astype(np.int8)
+    hi = np.where(hi >= 8, hi - 16, hi).astype(np.int8)
+    out = np.empty(p.shape[:-1] + (p.shape[-1] * 2,), dtype=np.int8)
+    out[..., 0::2] = lo
+    out[..., 1::2] = hi
+    return out
+
+
+def dequantize(packed: np.ndarray, scales: np.ndarray, weight_mode: int = WEIGHT_EXACT) -> np.ndarray:
+    """w[n,k] = scale[n, k // 32] * code[n,k]  (exact in fp64 and in fp32: 11-bit x 4-bit).
+
+    ``WEIGHT_F16`` rounds that product once to fp16 (what a tensor-core operand holds).
+    """
+    codes = unpack_codes(packed).astype(np.float64)
+    s = np.asarray(scales, dtype=np.float16).astype(np.float64)
+    assert codes.shape[-1] == s.shape[-1] * BLOCK, "one scale per 32 consecutive k"
+    w = codes * np.repeat(s, BLOCK, axis=-1)
+    return rn16(w) if weight_mode == WEIGHT_F16 else w
+
+
+# --------------------------------------------------------------------------------------
+# a2 / a3: the per-tensor operator (GEMV for decode, GEMM for prefill)
+# --------------------------------------------------------------------------------------
+def linear(x: np.ndarray, packed: np.ndarray, scales: np.ndarray, weight_mode: int = WEIGHT_EXACT,
+           round_out: bool = False) -> np.ndarray:
+    """y[m,n] = sum_k w[n,k] x[m,k] in fp64; ``round_out`` gives the fp16 output of the standalone op."""
+    w = dequantize(packed, scales, weight_mode)
+    y = np.asarray(x, dtype=np.float64) @ w.T
+    return rn16(y) if round_out else y
+
+
+# --------------------------------------------------------------------------------------
+# a6: layer glue
+# --------------------------------------------------------------------------------------
+def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """h_i = x_i g_i / sqrt(mean_j x_j^2 + eps), per row."""
+    x = np.asarray(x, dtype=np.float64)
+    g = np.asarray(gain, dtype=np.float64)
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x * g / np.sqrt(ms + eps)
+
+
+def rope(u: np.ndarray, pos, theta: float) -> np.ndarray:
+    """Rotary embedding, half-split pairing, on the last axis (head_dim d).
+
+    For i < d/2 the pair (u_i, u_{i+d/2}) is rotated by the angle pos * theta^(-2i/d).
+    ``pos`` broadcasts against u's leading axes (scalar, or [T,1] for [T,heads,d]).
+    ``theta == 0`` disables the rotation.
+    """
+    u = np.asarray(u, dtype=np.float64)
+    if theta == 0:
+        return u.copy()
+    d = u.shape[-1]
+    half = d // 2
+    i = np.arange(half, dtype=np.float64)
+    ang = np.asarray(pos, dtype=np.float64)[..., None] * theta ** (-2.0 * i / d)
+    c, s = np.cos(ang), np.sin(ang)
+    a, b = u[..., :half], u[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def softmax(s: np.ndarray) -> np.ndarray:
+    s = np.asarray(s, dtype=np.float64)
+    e = np.exp(s - np.max(s, axis=-1, keepdims=True))
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def attention_one(q_heads: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, n_ctx: int) -> np.ndarray:
+    """Grouped-query attention of ONE token over cache positions 0..n_ctx-1.
+
+    q_heads [n_q][d]; caches [n_kv][capacity][d].  Query head hq reads kv head hq // (n_q / n_kv).
+    Scores are scaled by 1/sqrt(d); softmax is max-subtracted.
+    """
+    n_q, d = q_heads.shape
+    n_kv = k_cache.shape[0]
+    group = n_q // n_kv
+    out = np.empty((n_q, d), dtype=np.float64)
+    for hq in range(n_q):
+        kvh = hq // group
+        kk = np.asarray(k_cache[kvh, :n_ctx], dtype=np.float64)
+        vv = np.asarray(v_cache[kvh, :n_ctx], dtype=np.float64)
+        p = softmax(kk @ q_heads[hq] / np.sqrt(d))
+        out[hq] = p @ vv
+    return out
+
+
+def silu(z):
+    z = np.asarray(z, dtype=np.float64)
+    return z / (1.0 + np.exp(-z))
+
+
+def swiglu_ffn(h2, w_gate, w_up, w_down, edges, weight_mode):
+    """d = W_down (silu(W_gate h2) * (W_up h2)) with the contract's roundings."""
+    g = _edge(linear(h2, *w_gate, weight_mode), "g", edges)
+    u = _edge(linear(h2, *w_up, weight_mode), "u", edges)
+    act = _edge(silu(g) * u, "act", edges)
+    return _edge(linear(act, *w_down, weight_mode), "d", edges)
+
+
+def dense_layer(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.ndarray, pos0: int,
+                edges=frozenset(), weight_mode: int = WEIGHT_EXACT):
+    """One dense decoder layer over T = x.shape[0] tokens at positions pos0..pos0+T-1.
+
+    T == 1 is a decode step, T > 1 a prefill chunk; both are the same definition:
+    the new keys/values are written to the caches (as fp16) first, then the token at
+    position p attends to positions 0..p.  ``tensors`` maps 'wq','wk','wv','wo',
+    'w_gate','w_up','w_down' to (packed, scales) and 'attn_norm','ffn_norm' to fp16 gains.
+    The caches (fp16, [n_kv][capacity][d]) are updated in place.  Returns y as fp16.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    T = x.shape[0]
+    nq, nkv, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    h = _edge(rmsnorm(x, tensors["attn_norm"], shape.rms_eps), "h", edges)
+    q = _edge(linear(h, *tensors["wq"], weight_mode), "q", edges).reshape(T, nq, d)
+    k = _edge(linear(h, *tensors["wk"], weight_mode), "k", edges).reshape(T, nkv, d)
+    v = _edge(linear(h, *tensors["wv"], weight_mode), "v", edges).reshape(T, nkv, d)
+    pos = (pos0 + np.arange(T, dtype=np.float64)).reshape(T, 1)
+    q_rot = _edge(rope(q, pos, shape.rope_theta), "q_rot", edges)
+    k_rot = rope(k, pos, shape.rope_theta)
+    for t in range(T):
+        k_cache[:, pos0 + t, :] = k_rot[t].astype(np.float16)
+        v_cache[:, pos0 + t, :] = v[t].astype(np.float16)
+    a = np.empty((T, nq * d), dtype=np.float64)
+    for t in range(T):
+        a[t] = attention_one(q_rot[t], k_cache, v_cache, pos0 + t + 1).reshape(-1)
+    a = _edge(a, "a", edges)
+    o = _edge(linear(a, *tensors["wo"], weight_mode), "o", edges)
+    x1 = _edge(x + o, "x1", edges)
+    h2 = _edge(rmsnorm(x1, tensors["ffn_norm"], shape.rms_eps), "h2", edges)
+    dd = swiglu_ffn(h2, tensors["w_gate"], tensors["w_up"], tensors["w_down"], edges, weight_mode)
+    return (x1 + dd).astype(np.float16)
+
+
+# --------------------------------------------------------------------------------------
+# a4: router + top-k
+# --------------------------------------------------------------------------------------
+def route_topk(h: np.ndarray, router_w: np.ndarray, k: int):
+    """logits = h W_r (W_r fp16 [hidden][E]); ids = the k largest logits in descending order,
+    equal logits -> lower expert index first; gates = softmax over those k logits.
+
+    Returns (ids int32 [M,k], gates fp64 [M,k], logits fp64 [M,E]).
+    """
+    logits = np.asarray(h, dtype=np.float64) @ np.asarray(router_w, dtype=np.float16).astype(np.float64)
+    order = np.argsort(-logits, axis=-1, kind="stable")  # stable: ties keep ascending index
+    ids = order[:, :k].astype(np.int32)
+    top = np.take_along_axis(logits, ids.astype(np.int64), axis=-1)
+    return ids, softmax(top), logits
+
+
+def min_rank_gap(logits: np.ndarray, k: int) -> float:
+    """Smallest gap between adjacent sorted logits among ranks 1..k+1 (degenerate seeds have tiny gaps)."""
+    s = -np.sort(-np.asarray(logits, dtype=np.float64), axis=-1)[:, : k + 1]
+    return float(np.min(s[:, :-1] - s[:, 1:]))
+
+
+# --------------------------------------------------------------------------------------
+# a5: grouped-expert FFN (the MoE block)
+# --------------------------------------------------------------------------------------
+def moe_linear(x, ids, packed, scales, x_per_slot: bool = False, weight_mode: int = WEIGHT_EXACT,
+               round_out: bool = True):
+    """y[m,j,:] = W[ids[m,j]] x[m(,j),:] on a stacked expert tensor (packed [E][N][K/2])."""
+    x = np.asarray(x, dtype=np.float64)
+    M, k = ids.shape
+    n_out = packed.shape[1]
+    y = np.empty((M, k, n_out), dtype=np.float64)
+    for m in range(M):
+        for j in range(k):
+            e = int(ids[m, j])
+            xv = x[m, j] if x_per_slot else x[m]
+            y[m, j] = linear(xv[None, :], packed[e], scales[e], weight_mode)[0]
+    return rn16(y) if round_out else y
+
+
+def moe_block(x, tensors: dict, shape, edges=frozenset({"h2", "act"}), weight_mode: int = WEIGHT_EXACT):
+    """MoE FFN block: y = x + sum_j gate_j * FFN_{e_j}(h), h = RMSNorm(x), summed in rank order.
+
+    ``tensors``: 'ffn_norm' gain, 'router' fp16 [hidden][E], 'w_gate','w_up','w_down' stacked (packed, scales).
+    Returns (y fp16 [M,hidden], ids, gates, logits).
+    """
+    x = np.asarray(x, dtype=np.float64)
+    M = x.shape[0]
+    h = _edge(rmsnorm(x, tensors["ffn_norm"], shape.rms_eps), "h2", edges)
+    ids, gates, logits = route_topk(h, tensors["router"], shape.top_k)
+    y = np.empty_like(x)
+    for m in range(M):
+        acc = x[m].copy()
+        for j in range(shape.top_k):
+            e = int(ids[m, j])
+            wg = (tensors["w_gate"][0][e], tensors["w_gate"][1][e])
+            wu = (tensors["w_up"][0][e], tensors["w_up"][1][e])
+            wd = (tensors["w_down"][0][e], tensors["w_down"][1][e])
+            dj = swiglu_ffn(h[m][None, :], wg, wu, wd, edges, weight_mode)[0]
+            acc = acc + gates[m, j] * dj
+        y[m] = acc
+    return y.astype(np.float16), ids, gates, logits
+
+
+# --------------------------------------------------------------------------------------
+# a7: static placement (Algorithm 1 and the placement objective of Section 4.3.2)
+# --------------------------------------------------------------------------------------
+HOST, GPU = 0, 1
+_NEG = -(1 << 62)
+
+
+def placement_objective(b, r, c) -> int:
+    """sum_i r_i [b_i = GPU] - sum_{i>=2} c_i [b_i != b_{i-1}]   (Section 4.3.2)."""
+    val = 0
+    for i in range(len(b)):
+        if b[i] == GPU:
+            val += int(r[i])
+        if i > 0 and b[i] != b[i - 1]:
+            val -= int(c[i])
+    return val
+
+
+def size_units(nbytes, granule: int = 1 << 20):
+    """s_i = ceil(bytes_i / G): sizes round up so a unit-feasible placement is byte-feasible."""
+    return [-(-int(b) // granule) for b in nbytes]
+
+
+def budget_units(budget_bytes: int, granule: int = 1 << 20) -> int:
+    """M = floor(budget / G)."""
+    return int(budget_bytes) // granule
+
+
+def solve_knapsack_dp(s, r, c, M: int):
+    """The dense-model solver of Algorithm 1: knapsack over memory units with a penalty c_i
+    whenever tensors i-1 and i get different backends; placement recovered by backtracking.
+
+    State V[i][m][B] = best objective of tensors 1..i using at most m units with b_i = B.
+    Ties keep the *same-backend* predecessor; at the end a tie between the two final states
+    keeps HOST.  All integers.  Returns (b list of HOST/GPU, objective).
+    """
+    n = len(s)
+    if n == 0:
+        return [], 0
+    M = max(int(M), 0)
+    VH = np.zeros((n, M + 1), dtype=np.int64)
+    VG = np.full((n, M + 1), _NEG, dtype=np.int64)
+    predH = np.zeros((n, M + 1), dtype=np.int8)  # backend of tensor i-1 on the best path into (i, m, H)
+    predG = np.zeros((n, M + 1), dtype=np.int8)
+    for i in range(n):
+        si, ri, ci = int(s[i]), int(r[i]), int(c[i])
+        for m in range(M + 1):
+            if i == 0:
+                VH[i, m] = 0
+                if m >= si:
+                    VG[i, m] = ri
+                continue
+            same, other = VH[i - 1, m], VG[i - 1, m]
+            other = other - ci if other > _NEG // 2 else _NEG
+            if same >= other:
+                VH[i, m], predH[i, m] = same, HOST
+            else:
+                VH[i, m], predH[i, m] = other, GPU
+            if m >= si:
+                same, other = VG[i - 1, m - si], VH[i - 1, m - si] - ci
+                if same > _NEG // 2 and same >= other:
+                    VG[i, m], predG[i, m] = ri + same, GPU
+                else:
+                    VG[i, m], predG[i, m] = ri + other, HOST
+    b = [HOST] * n
+    m = M
+    cur = HOST if VH[n - 1, M] >= VG[n - 1, M] else GPU
+    best = int(max(VH[n - 1, M], VG[n - 1, M]))
+    for i in range(n - 1, -1, -1):
+        b[i] = cur
+        if cur == GPU:
+            nxt = predG[i, m]
+            m -= int(s[i])
+        else:
+            nxt = predH[i, m]
+        cur = int(nxt)
+    return b, best
+
+
+def static_placement(s, r, c, M: int, is_expert=None):
+    """Algorithm 1.  Dense model: the DP over all tensors.  MoE model (some ``is_expert``):
+    if the non-expert tensors fit, they all go to the GPU and the DP runs over the expert
+    tensors with the remaining budget; otherwise every expert tensor stays on the host and
+    the DP runs over the non-expert tensors with the whole budget."""
+    n = len(s)
+    if is_expert is None or not any(is_expert):
+        return solve_knapsack_dp(s, r, c, M)[0]
+    exp = [i for i in range(n) if is_expert[i]]
+    non = [i for i in range(n) if not is_expert[i]]
+    s_non = sum(int(s[i]) for i in non)
+    b = [HOST] * n
+    if M >= s_non:
+        for i in non:
+            b[i] = GPU
+        sub, rest = exp, M - s_non
+    else:
+        sub, rest = non, M
+    sol, _ = solve_knapsack_dp([s[i] for i in sub], [r[i] for i in sub], [c[i] for i in sub], rest)
+    for i, bi in zip(sub, sol):
+        b[i] = bi
+    return b
+
+
+# --------------------------------------------------------------------------------------
+# a8 / a9: streaming bookkeeping of one call
+# --------------------------------------------------------------------------------------
+def streamed_dense(tensor_bytes, where, chunk_bytes: int):
+    """Tensors of one call in execution order; those placed on the host are streamed whole.
+    Returns (bytes_streamed, copies, indices_streamed)."""
+    idx = [i for i, w in enumerate(where) if w == HOST]
+    nbytes = sum(int(tensor_bytes[i]) for i in idx)
+    copies = sum(-(-int(tensor_bytes[i]) // chunk_bytes) for i in idx)
+    return nbytes, copies, idx
+
+
+def streamed_moe(ids: np.ndarray, expert_where, slice_bytes, chunk_bytes: int):
+    """Only the experts selected by the current tokens move (Section 4.2.2): the distinct
+    host-placed experts over the batch, ascending, each contributing its gate, up and down slice.
+
+    ``expert_where[t][e]`` for t in (gate, up, down); ``slice_bytes[t]`` bytes of one expert slice.
+    Returns (bytes_streamed, copies, [(tensor, expert), ...] in issue order: gate_e, up_e for each
+    expert, then down_e for each expert).
+    """
+    sel = sorted(set(int(e) for e in np.asarray(ids).reshape(-1)))
+    order = []
+    for e in sel:
+        for t in (0, 1):
+            if expert_where[t][e] == HOST:
+                order.append((t, e))
+    for e in sel:
+        if expert_where[2][e] == HOST:
+            order.append((2, e))
+    nbytes = sum(int(slice_bytes[t]) for t, _ in order)
+    copies = sum(-(-int(slice_bytes[t]) // chunk_bytes) for t, _ in order)
+    return nbytes, copies, order
