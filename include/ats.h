@@ -1,0 +1,240 @@
+/*
+ * ats.h — C ABI of the tensor-granularity hybrid-placement forward library (B200, sm_100a).
+ *
+ * The library executes the per-tensor forward of 4-bit block-quantized transformer weights under
+ * a per-tensor placement: every weight tensor is one operator (paper Section 3 and 4.3.1: the unit
+ * that is placed and scheduled is a tensor with a size s_i and a value r_i); a GPU memory budget M
+ * and a placement b decide which tensors stay resident in GPU memory (Section 4.3.2, Algorithm 1);
+ * the others live in pinned host memory and are copied into temporary GPU buffers by a transfer
+ * stream while a compute stream runs the operators, ordered by events (Section 4.2.1, 4.2.2).
+ * For MoE operators only the experts the current tokens selected are moved (Section 4.2.2, 4.4.1).
+ *
+ * Conventions
+ *  - Every function returns an int32 status: ATS_OK (0) or a negative ATS_ERR_* code; the text of the
+ *    last error of a context is available from ats_last_error().  Nothing throws or aborts.
+ *  - Pointers are marked HOST or DEVICE.  Device pointers must belong to the context's device.
+ *  - Compute calls are asynchronous: they validate their arguments, enqueue work on the context's
+ *    compute / transfer streams and return.  Invalid arguments are rejected before anything is
+ *    enqueued.  An asynchronous CUDA error surfaces at a later call or at ats_sync() as ATS_ERR_CUDA.
+ *  - One host thread per context.  The caller owns every buffer it passes; the library owns the
+ *    pinned host store and lays the resident region / staging ring / workspace out inside the
+ *    caller's arena.
+ *  - Quantization format ATS_FMT_Q4B32 (the workload's "INT4"; the paper only names the bit width,
+ *    Section 5.1): signed 4-bit codes in [-8,7], blocks of 32 consecutive k of one output row, one
+ *    fp16 scale per block, w[n][k] = scale[n][k/32] * code[n][k].
+ *    Interchange layout at this ABI: codes row-major [E][N][K/2] bytes, byte j of a row holds code 2j
+ *    in bits 0..3 and code 2j+1 in bits 4..7 as two's-complement nibbles; scales row-major fp16
+ *    [E][N][K/32].  E = n_experts (1 for a dense tensor).  The library repacks internally.
+ */
+#ifndef ATS_H_
+#define ATS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ats_ctx ats_ctx;
+
+enum {
+  ATS_OK = 0,
+  ATS_ERR_INVALID = -1,     /* bad argument / unknown id / non-finite scale */
+  ATS_ERR_SHAPE = -2,       /* shape rule violated (k_in % 32 != 0, mismatching layer shapes, ...) */
+  ATS_ERR_NOMEM = -3,       /* host allocation failed, or workspace too small */
+  ATS_ERR_BUDGET = -4,      /* GPU-placed entries do not fit the arena, or a slice does not fit a ring slot */
+  ATS_ERR_STATE = -5,       /* call not legal in the current state (e.g. compute before placement) */
+  ATS_ERR_CUDA = -6,        /* a CUDA call failed; the context is poisoned */
+  ATS_ERR_TIMEOUT = -7,     /* ats_sync() gave up waiting */
+  ATS_ERR_UNSUPPORTED = -8  /* legal but not implemented configuration */
+};
+
+enum { ATS_HOST = 0, ATS_GPU = 1 };             /* placement b_i (Section 4.3.2) */
+enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1 };    /* F16: router weight [k_in][n_out], norm gain [n_out] */
+enum { ATS_OUT_F32 = 0, ATS_OUT_F16 = 1 };      /* ats_dequantize output */
+enum { ATS_MODE_DECODE = 0, ATS_MODE_PREFILL = 1 };
+
+/* ats_config.flags */
+enum {
+  ATS_FLAG_POISON_SLOTS = 1u,     /* debug: fill a ring slot with 0xFF after its consumer, so premature reuse shows */
+  ATS_FLAG_SKIP_SCALE_CHECK = 2u  /* do not scan scales for Inf/NaN at registration */
+};
+/* ats_layer_desc.flags */
+enum { ATS_LAYER_NO_TOPK_RENORM = 1u /* gates = full softmax entries instead of softmax over the top-k */ };
+
+typedef struct {
+  void* arena;             /* DEVICE, 256-byte aligned; workspace, staging ring and resident region are carved from it */
+  uint64_t arena_bytes;
+  void* compute_stream;    /* cudaStream_t on which operators run (0 = legacy default stream) */
+  void* transfer_stream;   /* cudaStream_t for host->device weight copies; must differ from compute_stream */
+  uint32_t ring_slots;     /* number of equal staging slots (temporary GPU buffers, Section 4.2.1); 0 = no streaming */
+  uint64_t slot_bytes;     /* bytes of one slot; every streamed tensor / expert slice must fit one slot */
+  uint64_t chunk_bytes;    /* a streamed slice is copied as ceil(bytes/chunk_bytes) cudaMemcpyAsync calls */
+  uint64_t workspace_bytes;/* activation scratch for ats_layer_* / ats_moe_linear; see ats_workspace_bytes() */
+  int32_t device;          /* CUDA device ordinal of the arena and streams */
+  uint32_t flags;
+} ats_config;
+
+/* Create a context.  cfg is copied.  ATS_ERR_INVALID for null/misaligned arena, equal streams, an arena
+ * smaller than workspace + ring.  The arena and streams stay owned by the caller and must outlive the context. */
+int32_t ats_init(const ats_config* cfg /*HOST*/, ats_ctx** out /*HOST*/);
+/* Synchronises both streams, frees the pinned store and every event.  The arena is not touched. */
+int32_t ats_destroy(ats_ctx* ctx);
+/* Text of the last error recorded on ctx (valid until the next failing call); "" if none. */
+const char* ats_last_error(const ats_ctx* ctx);
+
+/* A tensor record (Section 4.3.2: size s_i, value r_i, switching cost c_i). */
+typedef struct {
+  uint32_t fmt;        /* ATS_FMT_* */
+  uint32_t n_experts;  /* 1 = dense tensor; > 1 = stacked expert tensor [E][n_out][k_in] */
+  uint32_t n_out;      /* output features N */
+  uint32_t k_in;       /* input features K (Q4B32: multiple of 32) */
+  uint32_t layer;      /* informational */
+  uint32_t role;       /* informational */
+  int64_t value;       /* r_i, the benefit of residency; < 0 selects the default r_i = byte size */
+  int64_t switch_cost; /* c_i >= 0, charged when tensor i and its predecessor get different backends */
+} ats_tensor_desc;
+
+/* Register a tensor.  codes/scales are HOST pointers in the interchange layout; they are repacked into the
+ * library's pinned store before return and may be freed afterwards.  ATS_FMT_F16 tensors pass their fp16 data as
+ * `codes` (scales = NULL); they are small, always GPU-resident and take no part in placement.
+ * Tensors must be registered in execution order (that order is the sequence Algorithm 1 runs over).
+ * Registration after ats_set_placement/ats_plan_placement invalidates the placement (state: unplaced).
+ * Errors: ATS_ERR_SHAPE (k_in % 32, zero dims), ATS_ERR_INVALID (non-finite scale, null), ATS_ERR_NOMEM. */
+int32_t ats_register_tensor(ats_ctx* ctx, const ats_tensor_desc* desc /*HOST*/, const void* codes /*HOST*/,
+                            const void* scales /*HOST*/, int32_t* out_id /*HOST*/);
+
+/* Bytes one (tensor, expert) slice occupies in the library's format: N*K/2 code bytes + N*(K/32) fp16 scales. */
+int32_t ats_tensor_slice_bytes(const ats_ctx* ctx, int32_t id, uint64_t* out_bytes /*HOST*/);
+
+/* Explicit placement (the decision vector b of Section 4.3.2).  Entry i places tensor ids[i], expert slice
+ * experts[i] (-1 = the whole tensor, all slices) on where[i] (ATS_HOST / ATS_GPU).  Entries not named are ATS_HOST.
+ * Rebuilds the resident region (copies GPU-placed slices into the arena, synchronously).
+ * ATS_ERR_BUDGET if the GPU entries do not fit arena - workspace - ring, or a HOST slice exceeds slot_bytes
+ * (or ring_slots == 0 while something is placed on the host). */
+int32_t ats_set_placement(ats_ctx* ctx, const int32_t* ids /*HOST*/, const int32_t* experts /*HOST*/,
+                          const uint8_t* where /*HOST*/, uint32_t n);
+
+/* Algorithm 1 (static tensor placement): knapsack DP over the registered Q4B32 tensors in registration order with
+ * sizes s_i = ceil(bytes/granule), budget M = floor(budget_bytes/granule), values r_i and switch costs c_i;
+ * for a model with expert tensors the expert / non-expert partition rule of Algorithm 1 applies (a stacked expert
+ * tensor is one item).  granule_bytes = 0 selects 1 MiB (the paper quantizes at MB granularity).
+ * Applies the result like ats_set_placement and writes one ATS_HOST/ATS_GPU byte per Q4B32 tensor (registration
+ * order) to out_where[0..n) if non-null; n must then equal the number of Q4B32 tensors. */
+int32_t ats_plan_placement(ats_ctx* ctx, uint64_t budget_bytes, uint32_t granule_bytes, uint8_t* out_where /*HOST*/,
+                           uint32_t n);
+int32_t ats_get_placement(const ats_ctx* ctx, int32_t id, int32_t expert, uint8_t* out_where /*HOST*/);
+
+/* The per-tensor operator: y[m][n] = sum_k w[n][k] x[m][k], fp32 accumulation, fp16 output.
+ * x DEVICE fp16 row-major [M][k_in]; y DEVICE fp16 row-major [M][n_out].  M <= 8 runs the memory-bound GEMV
+ * (weights exact, CUDA cores); M > 8 runs the tensor-core GEMM (weights rounded once to fp16 operands).
+ * If the tensor is placed on the host it is streamed through the ring for this call. */
+int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /*DEVICE*/, uint32_t M);
+
+/* Router: logits = h W_r (fp16 weights [hidden][E], fp32 accumulation); ids[m][0..k) = the k largest logits in
+ * descending order, equal logits -> lower expert index first; gates = softmax over the selected logits.
+ * h DEVICE fp16 [M][hidden]; ids_dev DEVICE int32 [M][k]; gates_dev DEVICE fp32 [M][k].  k <= 32, E <= 1024. */
+int32_t ats_route_topk(ats_ctx* ctx, int32_t router_id, const void* h /*DEVICE*/, uint32_t M, uint32_t k,
+                       int32_t* ids_dev /*DEVICE*/, float* gates_dev /*DEVICE*/);
+
+/* Top-k routed expert GEMV on a stacked expert tensor: y[m][j][:] = W[ids[m][j]] x[m][:] (x_per_slot = 0, x [M][K])
+ * or W[ids[m][j]] x[m][j][:] (x_per_slot = 1, x [M][k][K]); fp16 in, fp32 accumulation, fp16 out [M][k][n_out].
+ * M*k <= 256.  If any expert slice of the tensor is host-placed the call copies ids to the host and waits for them
+ * (the one host synchronisation on the path: expert transfer cannot start before routing is known, Section 4.2.2),
+ * then streams only the selected host-placed slices (distinct over the batch, ascending expert id). */
+int32_t ats_moe_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, const int32_t* ids_dev /*DEVICE*/,
+                       void* y /*DEVICE*/, uint32_t M, uint32_t k, uint32_t x_per_slot);
+
+/* One decoder layer.  Tensor ids; -1 = absent.  Attention part runs if wq >= 0; the FFN part is dense SwiGLU if
+ * n_experts == 0, else a top-k MoE of SwiGLU experts (w_gate/w_up/w_down stacked, router F16 [hidden][E]).
+ * Math: h = RMSNorm(x; attn_norm); q,k,v = W h; rotary embedding (half-split pairs, angle pos*theta^(-2i/d)) on q,k;
+ * K/V of the new token(s) are written to the caches as fp16 first; causal grouped-query attention with scale
+ * 1/sqrt(head_dim), query head hq reading kv head hq/(n_q/n_kv); x1 = x + W_o a; h2 = RMSNorm(x1; ffn_norm);
+ * y = x1 + W_down(silu(W_gate h2) * (W_up h2))  (MoE: y = x1 + sum_j gate_j FFN_{e_j}(h2) in rank order). */
+typedef struct {
+  int32_t attn_norm, wq, wk, wv, wo, ffn_norm, w_gate, w_up, w_down, router;
+  uint32_t hidden, n_q_heads, n_kv_heads, head_dim, ffn, n_experts, top_k, kv_capacity;
+  float rms_eps;
+  float rope_theta;  /* 0 = no rotary embedding */
+  uint32_t flags;    /* ATS_LAYER_* */
+} ats_layer_desc;
+
+/* Decode: M tokens, each one step of its own sequence.  With an attention part M must be 1 (one sequence; the token
+ * sits at cache position `pos` = number of past tokens, pos < kv_capacity); an FFN-only layer (wq = -1) takes M <= 32.
+ * x_in, x_out DEVICE fp16 [M][hidden] (may alias); k_cache, v_cache DEVICE fp16 [n_kv_heads][kv_capacity][head_dim],
+ * caller-owned, updated in place (ignored when wq = -1).  Streams host-placed tensors of the layer through the ring. */
+int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, const void* x_in /*DEVICE*/,
+                         void* x_out /*DEVICE*/, void* k_cache /*DEVICE*/, void* v_cache /*DEVICE*/, uint32_t pos,
+                         uint32_t M);
+/* Prefill: T tokens of one sequence at cache positions pos0 .. pos0+T-1 (pos0+T <= kv_capacity); projections run as
+ * dequantize-fused tensor-core GEMMs.  Same buffers as decode with M = T.  Dense FFN only. */
+int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, const void* x_in /*DEVICE*/,
+                          void* x_out /*DEVICE*/, void* k_cache /*DEVICE*/, void* v_cache /*DEVICE*/, uint32_t pos0,
+                          uint32_t T);
+
+/* Workspace a layer call needs: pass the largest value over the calls you will make as ats_config.workspace_bytes. */
+uint64_t ats_workspace_bytes(const ats_layer_desc* desc /*HOST*/, uint32_t max_tokens);
+
+/* Block dequantization of one (tensor, expert) slice (expert = 0 for a dense tensor) from the library's internal
+ * format: out[n][k] = scale*code as fp32 (exact) or rounded once to fp16.  out_dev DEVICE [n_out][k_in].
+ * Reads the resident copy if the slice is GPU-placed, else streams it through the ring. */
+int32_t ats_dequantize(ats_ctx* ctx, int32_t id, int32_t expert, void* out_dev /*DEVICE*/, uint32_t out_fmt);
+
+/* The numerics contract of a mode: bit i of *fp16_edge_mask set = the layer rounds intermediate i to fp16, for
+ * i over {h, q, k, v, q_rot, a, o, x1, h2, g, u, act, d}; *weight_mode 0 = weights exact (scale*code in fp32),
+ * 1 = weights rounded once to fp16 (tensor-core operands).  Cache entries and x_out are always fp16. */
+int32_t ats_get_numerics(const ats_ctx* ctx, uint32_t mode, uint32_t* fp16_edge_mask /*HOST*/,
+                         uint32_t* weight_mode /*HOST*/);
+
+#define ATS_STATS_LIST 512
+typedef struct {
+  uint64_t resident_bytes;   /* Q4B32 slices placed on the GPU */
+  uint64_t aux_bytes;        /* F16 tensors (always resident) */
+  uint64_t host_store_bytes; /* pinned host store */
+  uint64_t streamed_bytes;   /* host->device weight bytes since the last ats_reset_stats */
+  uint64_t copies;           /* cudaMemcpyAsync calls for those bytes */
+  uint64_t kernel_launches;  /* kernels launched by the library since the last reset */
+  uint64_t ring_reuses;      /* copies that had to wait for a slot's previous consumer */
+  uint64_t host_syncs;       /* host waits for routing ids */
+  uint32_t n_streamed;       /* streamed slices since the last reset (list below holds the first ATS_STATS_LIST) */
+  uint32_t reserved;
+  int32_t streamed_ids[ATS_STATS_LIST];
+  int32_t streamed_experts[ATS_STATS_LIST];
+} ats_stats;
+int32_t ats_get_stats(const ats_ctx* ctx, ats_stats* out /*HOST*/);
+int32_t ats_reset_stats(ats_ctx* ctx);
+
+/* Wait for everything enqueued so far by polling events; ATS_ERR_TIMEOUT after timeout_ms (0 = wait without limit),
+ * ATS_ERR_CUDA if a kernel or copy failed. */
+int32_t ats_sync(ats_ctx* ctx, uint32_t timeout_ms);
+
+/* Measure host->device copy bandwidth from the library's own kind of pinned memory into the arena's ring:
+ * `bytes` (<= ring size) copied `reps` times, best time.  Synchronous.  Writes GB/s (1e9 bytes/s). */
+int32_t ats_measure_h2d(ats_ctx* ctx, uint64_t bytes, uint32_t reps, double* out_gbs /*HOST*/);
+
+/* Test hook: make the next n streaming copies fail as if cudaMemcpyAsync had returned an error (host-side fault
+ * injection; nothing faults on the device).  The failing call returns ATS_ERR_CUDA and the context is poisoned. */
+int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n);
+
+/* Debug/test hook: device address and byte size of an intermediate of the most recent ats_layer_decode call shape
+ * (which = 0 h, 1 qkv (fp32 [q|k|v]), 2 q_rot (fp32), 3 a (fp16), 4 x1 (fp32), 5 h2 (fp16), 6 act (fp16), 7 d (fp32, MoE),
+ * 8 ids (int32, MoE), 9 gates (fp32, MoE)).  The workspace is reused by every call; read it after ats_sync(). */
+int32_t ats_debug_decode_buffer(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, uint32_t M, uint32_t which,
+                                void** out_dev /*HOST*/, uint64_t* out_bytes /*HOST*/);
+
+/* ---- host-only utilities (no context, no GPU needed) ---- */
+
+/* Algorithm 1 on caller-supplied arrays (all HOST): n tensors in execution order with sizes s[i] (units), values r[i],
+ * switch costs c[i] (c[0] unused), is_expert[i] (0/1; null = dense model), budget M units.  Writes ATS_HOST/ATS_GPU to
+ * out_b[0..n) and, if non-null, the value of the placement objective of Section 4.3.2 to *out_objective. */
+int32_t ats_host_solve_placement(const int64_t* s, const int64_t* r, const int64_t* c, const uint8_t* is_expert, uint32_t n,
+                                 int64_t M, uint8_t* out_b, int64_t* out_objective);
+/* Interchange layout -> the library's internal slice layout (n_out*k_in/2 code bytes followed by n_out*k_in/32 fp16
+ * scales) and back; out_* are HOST buffers of the same sizes as the inputs.  The round trip is the identity. */
+int32_t ats_host_repack_q4(const void* codes, const void* scales, void* out_slice, uint32_t n_out, uint32_t k_in);
+int32_t ats_host_unpack_q4(const void* slice, void* out_codes, void* out_scales, uint32_t n_out, uint32_t k_in);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATS_H_ */

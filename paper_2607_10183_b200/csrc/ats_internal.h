@@ -1,0 +1,210 @@
+// Internal declarations shared by the host runtime and the CUDA kernels of the ats library.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/ats.h"
+
+namespace ats {
+
+constexpr int kBlock = 32;        // weights per quantization block
+constexpr uint64_t kAlign = 256;  // alignment of every region / slice inside the arena
+
+inline uint64_t align_up(uint64_t v, uint64_t a = kAlign) { return (v + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------------------------
+// Internal weight format "Q4B32i" of one (tensor, expert) slice:
+//   [codes: N rows x K/2 bytes][scales: N rows x K/32 fp16], the slice padded to 256 bytes.
+// Codes are stored per 32-bit word (8 consecutive k of a row): nibble position p of the word holds
+//   p = 0,1,2,3 -> k = 0,2,4,6 ;  p = 4,5,6,7 -> k = 1,3,5,7
+// as offset-binary u = code + 8.  With that order (word >> 8s) & 0x000F000F yields the fp16 pair
+// (k, k+1) after OR-ing the 1024.0 exponent, with no per-nibble shifts.
+// ---------------------------------------------------------------------------------------------
+struct Slice {
+  uint8_t where = ATS_HOST;
+  uint8_t* dev = nullptr;  // resident copy (null when host-placed)
+};
+
+struct Tensor {
+  ats_tensor_desc d{};
+  uint64_t codes_bytes = 0;   // per slice
+  uint64_t slice_bytes = 0;   // codes + scales (what streaming moves and the statistics count)
+  uint64_t slice_stride = 0;  // slice_bytes padded to 256 (distance between slices in host store / resident region)
+  uint8_t* host = nullptr;    // pinned store, n_experts * slice_stride bytes (F16: the raw fp16 data)
+  uint64_t host_bytes = 0;
+  uint8_t* f16_dev = nullptr;  // F16 tensors: device copy
+  std::vector<Slice> slices;
+  bool any_host = true;        // some slice is host-placed
+  bool contiguous_dev = false; // all slices resident, at dev0 + e * slice_stride
+};
+
+struct RingSlot {
+  cudaEvent_t ready = nullptr;  // recorded on the transfer stream after the slot's copies
+  cudaEvent_t freed = nullptr;  // recorded on the compute stream after the slot's consumer
+  bool used = false;            // freed has been recorded at least once
+  bool busy = false;            // holds a slice whose consumer has not been enqueued yet
+};
+
+// One streamed slice of the current call (an entry of the per-call execution plan).
+struct Fetch {
+  int tensor = -1;
+  int expert = 0;
+  int slot = -1;
+  bool enqueued = false;  // copy is on the transfer stream
+  bool waited = false;    // compute stream already waits on the slot's ready event
+};
+
+}  // namespace ats
+
+struct ats_ctx {
+  ats_config cfg{};
+  cudaStream_t cs = nullptr, ts = nullptr;
+  std::string err;
+  bool poisoned = false;
+  bool placed = false;
+  std::vector<ats::Tensor> tensors;
+  // arena layout
+  uint8_t* ws = nullptr;        // workspace
+  uint8_t* ring = nullptr;      // ring_slots * slot_stride
+  uint64_t slot_stride = 0;
+  uint8_t* resident = nullptr;  // start of aux + resident region
+  uint64_t resident_cap = 0;
+  std::vector<ats::RingSlot> slots;
+  // per-call streaming plan
+  std::vector<ats::Fetch> plan;
+  size_t plan_next = 0;  // next plan entry whose copy is not enqueued yet
+  uint32_t next_slot = 0;
+  // pinned scratch for routing ids (host side of the one synchronisation on the MoE path)
+  int32_t* ids_host = nullptr;
+  cudaEvent_t ids_event = nullptr;
+  cudaEvent_t sync_event = nullptr;
+  uint32_t fail_copies = 0;
+  ats_stats stats{};
+};
+
+namespace ats {
+
+int32_t fail(ats_ctx* c, int32_t code, const char* fmt, ...);
+int32_t check_cuda(ats_ctx* c, cudaError_t e, const char* what);
+
+// ----------------------------------------------------------------------------- kernel launchers
+// All launchers enqueue on `st`, return the cudaError of the launch and count launches in *n_launch.
+
+struct GemvSeg {
+  const uint8_t* base;  // slice base (codes, then scales)
+  int n_rows;
+};
+enum GemvMode {
+  GEMV_OUT_F32 = 0,        // y32[m][row] = acc
+  GEMV_OUT_F16 = 1,        // y16[m][row] = rn16(acc)
+  GEMV_RES16_OUT_F32 = 2,  // y32 = float(res16) + acc
+  GEMV_RES32_OUT_F16 = 3,  // y16 = rn16(res32 + acc)
+  GEMV_SWIGLU_F16 = 4,     // seg[0] = gate, seg[1] = up (same n_rows): y16 = rn16(silu(g) * u)
+  GEMV_RES16_OUT_F16 = 5   // y16 = rn16(float(res16) + acc)
+};
+struct GemvParams {
+  GemvSeg seg[3];
+  int n_seg;
+  int K;
+  int M;
+  const __half* x;
+  int ldx;
+  float* y32;
+  __half* y16;
+  int ldy;
+  const float* res32;
+  const __half* res16;
+  int ldres;
+  int mode;
+};
+cudaError_t launch_gemv(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
+
+// Grouped-expert GEMV: job j multiplies the slice w0[j] (and w1[j] for SwiGLU) with activation row xrow[j] and
+// writes output row j_out[j].  Implicit mode (n_jobs_explicit == 0): job p = 0..P-1 uses expert ids[p] of a
+// contiguous resident tensor.
+constexpr int kMoeJobsPerLaunch = 64;
+struct MoeJobs {
+  const uint8_t* w0[kMoeJobsPerLaunch];
+  const uint8_t* w1[kMoeJobsPerLaunch];
+  int16_t xrow[kMoeJobsPerLaunch];
+  int16_t orow[kMoeJobsPerLaunch];
+  int n;
+};
+struct MoeGemvParams {
+  // implicit addressing
+  const uint8_t* base0;
+  const uint8_t* base1;
+  uint64_t stride;
+  const int32_t* ids;  // [P]
+  int x_div;           // activation row of pair p is p / x_div (k when one x per token, 1 when one per slot)
+  int P;
+  // common
+  int n_rows, K;
+  const __half* x;
+  int ldx;
+  float* y32;
+  __half* y16;
+  int ldy;
+  int mode;  // GEMV_OUT_F32, GEMV_OUT_F16 or GEMV_SWIGLU_F16
+};
+cudaError_t launch_moe_gemv(const MoeGemvParams& p, const MoeJobs* jobs /*null = implicit*/, cudaStream_t st,
+                            uint64_t* n_launch);
+
+cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, cudaStream_t st,
+                           uint64_t* n_launch);
+cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
+                           cudaStream_t st, uint64_t* n_launch);
+// decode: rotary embedding of q (fp32 -> fp32) and k, append k/v rows to the caches at `pos`
+cudaError_t launch_rope_append_decode(const float* qkv, float* q_rot, __half* kc, __half* vc, int n_q, int n_kv, int d,
+                                      int cap, int pos, float theta, cudaStream_t st, uint64_t* n_launch);
+int attn_decode_splits(int n_ctx);
+size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx);
+cudaError_t launch_attn_decode(const float* q_rot, const __half* kc, const __half* vc, float* scratch, __half* a16,
+                               int n_q, int n_kv, int d, int cap, int n_ctx, cudaStream_t st, uint64_t* n_launch);
+cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
+                               float* gates, cudaStream_t st, uint64_t* n_launch);
+// y16[m] = rn16(res[m] + sum_j gates[m][j] * d32[m*k + j])   (res fp16 or fp32)
+cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gates, const float* d32, __half* y16,
+                               int M, int k, int H, cudaStream_t st, uint64_t* n_launch);
+cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uint64_t* n_launch);
+
+// prefill
+cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_rot16, __half* kc, __half* vc, int T,
+                                       int n_q, int n_kv, int d, int cap, int pos0, float theta, cudaStream_t st,
+                                       uint64_t* n_launch);
+cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const __half* vc, __half* a16, int T, int n_q,
+                                int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch);
+cudaError_t launch_add16(const __half* a, const __half* b, __half* out, uint64_t n, cudaStream_t st, uint64_t* n_launch);
+cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch);
+
+// Tensor-core GEMM  Y[T][n_rows] (fp16, leading dimension ldy) = X[T][K] (fp16, ld = ldx) * W^T for up to 3 weight
+// segments laid side by side in Y.  `scratch` holds split-K partials (gemm_scratch_bytes()).
+struct GemmParams {
+  GemvSeg seg[3];
+  int n_seg;
+  int K;
+  int T;
+  const __half* x;
+  int ldx;
+  __half* y;
+  int ldy;
+  void* scratch;
+  uint64_t scratch_bytes;
+};
+uint64_t gemm_scratch_bytes(int T, int n_total, int K);
+cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);
+
+// host-side pieces
+void repack_q4(const uint8_t* codes_in, const uint16_t* scales_in, uint8_t* slice_out, uint64_t n_rows, uint64_t K);
+// Algorithm 1's dense solver; returns placement bytes (ATS_HOST/ATS_GPU) and the objective.
+void solve_knapsack_dp(const std::vector<int64_t>& s, const std::vector<int64_t>& r, const std::vector<int64_t>& c,
+                       int64_t M, std::vector<uint8_t>* b, int64_t* objective);
+void static_placement(const std::vector<int64_t>& s, const std::vector<int64_t>& r, const std::vector<int64_t>& c,
+                      const std::vector<uint8_t>& is_expert, int64_t M, std::vector<uint8_t>* b);
+
+}  // namespace ats

@@ -1,0 +1,1164 @@
+// Host runtime of the ats library: context, tensor registry, placement, resident region, staging ring,
+// per-call execution plan and the C ABI entry points.  All device work goes through the launchers declared in
+// ats_internal.h; there is no CPU compute path.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <chrono>
+#include <thread>
+
+#include "ats_internal.h"
+
+namespace ats {
+
+int32_t fail(ats_ctx* c, int32_t code, const char* fmt, ...) {
+  if (c) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    c->err = buf;
+  }
+  return code;
+}
+
+int32_t check_cuda(ats_ctx* c, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return ATS_OK;
+  c->poisoned = true;
+  return fail(c, ATS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define ATS_CUDA(call)                                       \
+  do {                                                       \
+    int32_t _s = ats::check_cuda(ctx, (call), #call);        \
+    if (_s != ATS_OK) return _s;                             \
+  } while (0)
+#define ATS_TRY(expr)              \
+  do {                             \
+    int32_t _s = (expr);           \
+    if (_s != ATS_OK) return _s;   \
+  } while (0)
+
+static int32_t precheck(ats_ctx* ctx, bool need_placement) {
+  if (!ctx) return ATS_ERR_INVALID;
+  if (ctx->poisoned) return fail(ctx, ATS_ERR_CUDA, "context is poisoned by an earlier CUDA error: %s", ctx->err.c_str());
+  if (need_placement && !ctx->placed)
+    return fail(ctx, ATS_ERR_STATE, "no placement: call ats_set_placement or ats_plan_placement first");
+  return ATS_OK;
+}
+
+static Tensor* get_tensor(ats_ctx* ctx, int32_t id, uint32_t fmt) {
+  if (id < 0 || (size_t)id >= ctx->tensors.size()) return nullptr;
+  Tensor* t = &ctx->tensors[id];
+  return t->d.fmt == fmt ? t : nullptr;
+}
+
+// ------------------------------------------------------------------------------------ streaming ring
+// The per-call execution plan is the ordered list ctx->plan of slices to stream.  Copies are issued in plan order into
+// ring slots taken round-robin; a slot is reused only after the consumer of its previous content has been enqueued on
+// the compute stream (its `freed` event is then what the transfer stream waits for).
+
+static void plan_begin(ats_ctx* ctx) {
+  ctx->plan.clear();
+  ctx->plan_next = 0;
+}
+
+static int plan_add(ats_ctx* ctx, int tensor, int expert) {
+  Fetch f;
+  f.tensor = tensor;
+  f.expert = expert;
+  ctx->plan.push_back(f);
+  return (int)ctx->plan.size() - 1;
+}
+
+static int plan_find(const ats_ctx* ctx, int tensor, int expert) {
+  for (size_t i = 0; i < ctx->plan.size(); ++i)
+    if (ctx->plan[i].tensor == tensor && ctx->plan[i].expert == expert) return (int)i;
+  return -1;
+}
+
+static int32_t pump(ats_ctx* ctx) {
+  const uint32_t S = ctx->cfg.ring_slots;
+  while (ctx->plan_next < ctx->plan.size()) {
+    if (S == 0) return fail(ctx, ATS_ERR_BUDGET, "a host-placed tensor needs streaming but ring_slots is 0");
+    RingSlot& slot = ctx->slots[ctx->next_slot];
+    if (slot.busy) break;
+    Fetch& f = ctx->plan[ctx->plan_next];
+    const Tensor& t = ctx->tensors[f.tensor];
+    if (t.slice_bytes > ctx->cfg.slot_bytes)
+      return fail(ctx, ATS_ERR_BUDGET, "slice of tensor %d (%llu bytes) does not fit a ring slot (%llu bytes)", f.tensor,
+                  (unsigned long long)t.slice_bytes, (unsigned long long)ctx->cfg.slot_bytes);
+    if (slot.used) {
+      ATS_CUDA(cudaStreamWaitEvent(ctx->ts, slot.freed, 0));
+      ctx->stats.ring_reuses++;
+    }
+    uint8_t* dst = ctx->ring + (uint64_t)ctx->next_slot * ctx->slot_stride;
+    const uint8_t* src = t.host + (uint64_t)f.expert * t.slice_stride;
+    const uint64_t chunk = ctx->cfg.chunk_bytes ? ctx->cfg.chunk_bytes : t.slice_bytes;
+    for (uint64_t off = 0; off < t.slice_bytes; off += chunk) {
+      const uint64_t nb = std::min<uint64_t>(chunk, t.slice_bytes - off);
+      if (ctx->fail_copies) {
+        ctx->fail_copies--;
+        ctx->poisoned = true;
+        return fail(ctx, ATS_ERR_CUDA, "cudaMemcpyAsync failed (injected) while streaming tensor %d", f.tensor);
+      }
+      ATS_CUDA(cudaMemcpyAsync(dst + off, src + off, nb, cudaMemcpyHostToDevice, ctx->ts));
+      ctx->stats.copies++;
+    }
+    ATS_CUDA(cudaEventRecord(slot.ready, ctx->ts));
+    ctx->stats.streamed_bytes += t.slice_bytes;
+    if (ctx->stats.n_streamed < ATS_STATS_LIST) {
+      ctx->stats.streamed_ids[ctx->stats.n_streamed] = f.tensor;
+      ctx->stats.streamed_experts[ctx->stats.n_streamed] = f.expert;
+    }
+    ctx->stats.n_streamed++;
+    f.slot = (int)ctx->next_slot;
+    f.enqueued = true;
+    slot.busy = true;
+    ctx->next_slot = (ctx->next_slot + 1) % S;
+    ctx->plan_next++;
+  }
+  return ATS_OK;
+}
+
+// Make the compute stream wait for plan entry idx and return where its bytes land.
+static int32_t acquire(ats_ctx* ctx, int idx, const uint8_t** out) {
+  Fetch& f = ctx->plan[idx];
+  if (!f.enqueued) {
+    ATS_TRY(pump(ctx));
+    if (!f.enqueued)
+      return fail(ctx, ATS_ERR_BUDGET, "staging ring too small: %u slots cannot hold the slices one operator consumes together",
+                  ctx->cfg.ring_slots);
+  }
+  if (!f.waited) {
+    ATS_CUDA(cudaStreamWaitEvent(ctx->cs, ctx->slots[f.slot].ready, 0));
+    f.waited = true;
+  }
+  *out = ctx->ring + (uint64_t)f.slot * ctx->slot_stride;
+  return ATS_OK;
+}
+
+// The consumer of plan entry idx is on the compute stream: its slot may be refilled after it.
+static int32_t release(ats_ctx* ctx, int idx) {
+  Fetch& f = ctx->plan[idx];
+  RingSlot& slot = ctx->slots[f.slot];
+  if (ctx->cfg.flags & ATS_FLAG_POISON_SLOTS)
+    ATS_CUDA(launch_fill(ctx->ring + (uint64_t)f.slot * ctx->slot_stride, ctx->slot_stride, 0xFF, ctx->cs,
+                         &ctx->stats.kernel_launches));
+  ATS_CUDA(cudaEventRecord(slot.freed, ctx->cs));
+  slot.used = true;
+  slot.busy = false;
+  return pump(ctx);
+}
+
+// A dense tensor as a kernel operand: resident pointer, or a plan entry to acquire.
+struct Operand {
+  const Tensor* t = nullptr;
+  int id = -1;
+  int fetch = -1;  // plan index, -1 = resident
+  const uint8_t* ptr = nullptr;
+};
+
+static void plan_dense(ats_ctx* ctx, int id, Operand* op) {
+  op->id = id;
+  op->t = &ctx->tensors[id];
+  if (op->t->slices[0].where == ATS_GPU) {
+    op->ptr = op->t->slices[0].dev;
+    op->fetch = -1;
+  } else {
+    op->fetch = plan_add(ctx, id, 0);
+  }
+}
+
+static int32_t acquire_ops(ats_ctx* ctx, Operand* ops, int n) {
+  for (int i = 0; i < n; ++i)
+    if (ops[i].fetch >= 0) ATS_TRY(acquire(ctx, ops[i].fetch, &ops[i].ptr));
+  return ATS_OK;
+}
+static int32_t release_ops(ats_ctx* ctx, Operand* ops, int n) {
+  for (int i = 0; i < n; ++i)
+    if (ops[i].fetch >= 0) ATS_TRY(release(ctx, ops[i].fetch));
+  return ATS_OK;
+}
+static int count_streamed(const Operand* ops, int n) {
+  int c = 0;
+  for (int i = 0; i < n; ++i) c += ops[i].fetch >= 0;
+  return c;
+}
+
+// GEMV over 1..3 dense tensors whose outputs lie side by side.  When the ring cannot hold all streamed operands of
+// the group at once the segments run one by one (same per-row arithmetic, so results do not depend on it).
+static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
+  p.K = (int)ops[0].t->d.k_in;
+  if (count_streamed(ops, n) <= (int)ctx->cfg.ring_slots || n == 1) {
+    ATS_TRY(acquire_ops(ctx, ops, n));
+    p.n_seg = n;
+    for (int i = 0; i < n; ++i) p.seg[i] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
+    ATS_CUDA(launch_gemv(p, ctx->cs, &ctx->stats.kernel_launches));
+    return release_ops(ctx, ops, n);
+  }
+  if (p.mode == GEMV_SWIGLU_F16)
+    return fail(ctx, ATS_ERR_BUDGET, "fused gate/up needs 2 ring slots when both tensors are host-placed");
+  int row0 = 0;
+  for (int i = 0; i < n; ++i) {
+    ATS_TRY(acquire_ops(ctx, ops + i, 1));
+    GemvParams q = p;
+    q.n_seg = 1;
+    q.seg[0] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
+    if (q.y32) q.y32 += row0;
+    if (q.y16) q.y16 += row0;
+    if (q.res32) q.res32 += row0;
+    if (q.res16) q.res16 += row0;
+    ATS_CUDA(launch_gemv(q, ctx->cs, &ctx->stats.kernel_launches));
+    ATS_TRY(release_ops(ctx, ops + i, 1));
+    row0 += (int)ops[i].t->d.n_out;
+  }
+  return ATS_OK;
+}
+
+static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
+  p.K = (int)ops[0].t->d.k_in;
+  std::string err;
+  if (count_streamed(ops, n) <= (int)ctx->cfg.ring_slots || n == 1) {
+    ATS_TRY(acquire_ops(ctx, ops, n));
+    p.n_seg = n;
+    for (int i = 0; i < n; ++i) p.seg[i] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
+    cudaError_t e = launch_gemm(p, ctx->cs, &ctx->stats.kernel_launches, &err);
+    if (e != cudaSuccess) return check_cuda(ctx, e, err.empty() ? "launch_gemm" : err.c_str());
+    return release_ops(ctx, ops, n);
+  }
+  int row0 = 0;
+  for (int i = 0; i < n; ++i) {
+    ATS_TRY(acquire_ops(ctx, ops + i, 1));
+    GemmParams q = p;
+    q.n_seg = 1;
+    q.seg[0] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
+    q.y += row0;
+    cudaError_t e = launch_gemm(q, ctx->cs, &ctx->stats.kernel_launches, &err);
+    if (e != cudaSuccess) return check_cuda(ctx, e, err.empty() ? "launch_gemm" : err.c_str());
+    ATS_TRY(release_ops(ctx, ops + i, 1));
+    row0 += (int)ops[i].t->d.n_out;
+  }
+  return ATS_OK;
+}
+
+// ------------------------------------------------------------------------------------ workspace
+struct Bump {
+  uint8_t* base;
+  uint64_t cap, off = 0;
+  bool ok = true;
+  Bump(uint8_t* b, uint64_t c) : base(b), cap(c) {}
+  void* take(uint64_t bytes) {
+    const uint64_t o = align_up(off);
+    off = o + bytes;
+    if (off > cap) ok = false;
+    return base ? base + o : nullptr;
+  }
+};
+
+struct LayerWs {
+  // decode
+  __half* h16 = nullptr;
+  float* qkv32 = nullptr;
+  float* qrot32 = nullptr;
+  float* attn_scratch = nullptr;
+  __half* a16 = nullptr;
+  float* x1_32 = nullptr;
+  __half* h2_16 = nullptr;
+  __half* act16 = nullptr;
+  float* d32 = nullptr;
+  int32_t* ids = nullptr;
+  float* gates = nullptr;
+  // prefill
+  __half* qkv16 = nullptr;
+  __half* qrot16 = nullptr;
+  __half* o16 = nullptr;
+  __half* x1_16 = nullptr;
+  __half* gu16 = nullptr;
+  __half* d16 = nullptr;
+  void* gemm_scratch = nullptr;
+  uint64_t gemm_scratch_bytes = 0;
+  uint64_t total = 0;
+  bool ok = true;
+};
+
+static LayerWs layout_decode(const ats_layer_desc& L, uint32_t M, uint8_t* base, uint64_t cap) {
+  LayerWs w;
+  Bump b(base, cap);
+  const uint64_t H = L.hidden, qd = (uint64_t)L.n_q_heads * L.head_dim, kvd = (uint64_t)L.n_kv_heads * L.head_dim;
+  if (L.wq >= 0) {
+    w.h16 = (__half*)b.take(M * H * 2);
+    w.qkv32 = (float*)b.take(M * (qd + 2 * kvd) * 4);
+    w.qrot32 = (float*)b.take(M * qd * 4);
+    w.attn_scratch = (float*)b.take(attn_decode_scratch_floats((int)L.n_q_heads, (int)L.head_dim, (int)L.kv_capacity) * 4);
+    w.a16 = (__half*)b.take(M * qd * 2);
+    w.x1_32 = (float*)b.take(M * H * 4);
+  }
+  w.h2_16 = (__half*)b.take(M * H * 2);
+  if (L.n_experts == 0) {
+    w.act16 = (__half*)b.take((uint64_t)M * L.ffn * 2);
+  } else {
+    const uint64_t P = (uint64_t)M * L.top_k;
+    w.act16 = (__half*)b.take(P * L.ffn * 2);
+    w.d32 = (float*)b.take(P * H * 4);
+    w.ids = (int32_t*)b.take(P * 4);
+    w.gates = (float*)b.take(P * 4);
+  }
+  w.total = align_up(b.off);
+  w.ok = b.ok;
+  return w;
+}
+
+static LayerWs layout_prefill(const ats_layer_desc& L, uint32_t T, uint8_t* base, uint64_t cap) {
+  LayerWs w;
+  Bump b(base, cap);
+  const uint64_t H = L.hidden, qd = (uint64_t)L.n_q_heads * L.head_dim, kvd = (uint64_t)L.n_kv_heads * L.head_dim;
+  uint64_t scratch = 0;
+  if (L.wq >= 0) {
+    w.h16 = (__half*)b.take(T * H * 2);
+    w.qkv16 = (__half*)b.take(T * (qd + 2 * kvd) * 2);
+    w.qrot16 = (__half*)b.take(T * qd * 2);
+    w.a16 = (__half*)b.take(T * qd * 2);
+    w.o16 = (__half*)b.take(T * H * 2);
+    w.x1_16 = (__half*)b.take(T * H * 2);
+    scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)(qd + 2 * kvd), (int)H));
+    scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)H, (int)qd));
+  }
+  w.h2_16 = (__half*)b.take(T * H * 2);
+  w.gu16 = (__half*)b.take((uint64_t)T * 2 * L.ffn * 2);
+  w.act16 = (__half*)b.take((uint64_t)T * L.ffn * 2);
+  w.d16 = (__half*)b.take(T * H * 2);
+  scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)(2 * L.ffn), (int)H));
+  scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)H, (int)L.ffn));
+  w.gemm_scratch = b.take(scratch);
+  w.gemm_scratch_bytes = scratch;
+  w.total = align_up(b.off);
+  w.ok = b.ok;
+  return w;
+}
+
+// ------------------------------------------------------------------------------------ placement
+static int32_t apply_placement(ats_ctx* ctx) {
+  // everything enqueued so far may still read the old resident region
+  ATS_CUDA(cudaStreamSynchronize(ctx->cs));
+  ATS_CUDA(cudaStreamSynchronize(ctx->ts));
+  uint64_t off = 0, resident = 0, aux = 0;
+  for (Tensor& t : ctx->tensors) {
+    if (t.d.fmt == ATS_FMT_F16) {
+      off = align_up(off) + t.host_bytes;
+      aux += t.host_bytes;
+      continue;
+    }
+    for (Slice& s : t.slices)
+      if (s.where == ATS_GPU) {
+        off = align_up(off) + t.slice_stride;
+        resident += t.slice_bytes;
+      } else if (ctx->cfg.ring_slots == 0 || t.slice_bytes > ctx->cfg.slot_bytes) {
+        return fail(ctx, ATS_ERR_BUDGET, "host-placed slice of %llu bytes cannot be streamed (ring_slots %u, slot_bytes %llu)",
+                    (unsigned long long)t.slice_bytes, ctx->cfg.ring_slots, (unsigned long long)ctx->cfg.slot_bytes);
+      }
+  }
+  if (off > ctx->resident_cap)
+    return fail(ctx, ATS_ERR_BUDGET, "placement needs %llu resident bytes, arena has %llu after workspace and ring",
+                (unsigned long long)off, (unsigned long long)ctx->resident_cap);
+  off = 0;
+  for (Tensor& t : ctx->tensors) {
+    if (t.d.fmt == ATS_FMT_F16) {
+      off = align_up(off);
+      t.f16_dev = ctx->resident + off;
+      ATS_CUDA(cudaMemcpyAsync(t.f16_dev, t.host, t.host_bytes, cudaMemcpyHostToDevice, ctx->ts));
+      off += t.host_bytes;
+      continue;
+    }
+    t.any_host = false;
+    t.contiguous_dev = true;
+    uint8_t* prev = nullptr;
+    for (size_t e = 0; e < t.slices.size(); ++e) {
+      Slice& s = t.slices[e];
+      if (s.where == ATS_GPU) {
+        off = align_up(off);
+        s.dev = ctx->resident + off;
+        ATS_CUDA(cudaMemcpyAsync(s.dev, t.host + e * t.slice_stride, t.slice_bytes, cudaMemcpyHostToDevice, ctx->ts));
+        off += t.slice_stride;
+        if (prev && s.dev != prev + t.slice_stride) t.contiguous_dev = false;
+        prev = s.dev;
+      } else {
+        s.dev = nullptr;
+        t.any_host = true;
+        t.contiguous_dev = false;
+      }
+    }
+  }
+  ATS_CUDA(cudaStreamSynchronize(ctx->ts));
+  ctx->stats.resident_bytes = resident;
+  ctx->stats.aux_bytes = aux;
+  for (RingSlot& s : ctx->slots) s.busy = false;
+  ctx->placed = true;
+  return ATS_OK;
+}
+
+// ------------------------------------------------------------------------------------ MoE stages
+// One grouped GEMV stage over P = M*k (token, slot) pairs on stacked tensors t0 (and t1 for the fused SwiGLU stage).
+// ids_host == null: every slice is resident and contiguous, the kernel indexes experts from device ids.
+// Otherwise pairs on resident experts run first (overlapping the copies), then the streamed experts in ascending order
+// in groups that fit the ring.
+static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_dev, const int32_t* ids_host,
+                             MoeGemvParams p) {
+  const Tensor& t0 = ctx->tensors[id0];
+  const Tensor* t1 = id1 >= 0 ? &ctx->tensors[id1] : nullptr;
+  p.n_rows = (int)t0.d.n_out;
+  p.K = (int)t0.d.k_in;
+  p.stride = t0.slice_stride;
+  p.ids = ids_dev;
+  if (!ids_host) {
+    p.base0 = t0.slices[0].dev;
+    p.base1 = t1 ? t1->slices[0].dev : nullptr;
+    ATS_CUDA(launch_moe_gemv(p, nullptr, ctx->cs, &ctx->stats.kernel_launches));
+    return ATS_OK;
+  }
+  const int P = p.P;
+  MoeJobs jobs;
+  jobs.n = 0;
+  auto flush = [&]() -> int32_t {
+    if (jobs.n == 0) return ATS_OK;
+    ATS_CUDA(launch_moe_gemv(p, &jobs, ctx->cs, &ctx->stats.kernel_launches));
+    jobs.n = 0;
+    return ATS_OK;
+  };
+  auto add_job = [&](int pair, const uint8_t* w0, const uint8_t* w1) -> int32_t {
+    jobs.w0[jobs.n] = w0;
+    jobs.w1[jobs.n] = w1;
+    jobs.xrow[jobs.n] = (int16_t)(pair / p.x_div);
+    jobs.orow[jobs.n] = (int16_t)pair;
+    if (++jobs.n == kMoeJobsPerLaunch) return flush();
+    return ATS_OK;
+  };
+  auto is_res = [&](int e) {
+    return t0.slices[e].where == ATS_GPU && (!t1 || t1->slices[e].where == ATS_GPU);
+  };
+  // resident experts first
+  for (int pr = 0; pr < P; ++pr) {
+    const int e = ids_host[pr];
+    if (is_res(e)) ATS_TRY(add_job(pr, t0.slices[e].dev, t1 ? t1->slices[e].dev : nullptr));
+  }
+  ATS_TRY(flush());
+  // streamed experts, ascending, in groups whose slices fit the ring together
+  std::vector<int> sel;
+  for (int pr = 0; pr < P; ++pr)
+    if (!is_res(ids_host[pr])) sel.push_back(ids_host[pr]);
+  std::sort(sel.begin(), sel.end());
+  sel.erase(std::unique(sel.begin(), sel.end()), sel.end());
+  size_t i = 0;
+  while (i < sel.size()) {
+    std::vector<int> fetches;
+    size_t j = i;
+    int need = 0;
+    while (j < sel.size()) {
+      const int e = sel[j];
+      const int n_e = (t0.slices[e].where == ATS_HOST) + (t1 && t1->slices[e].where == ATS_HOST);
+      if (need + n_e > (int)ctx->cfg.ring_slots) break;
+      need += n_e;
+      ++j;
+    }
+    if (j == i) return fail(ctx, ATS_ERR_BUDGET, "staging ring too small for one expert's gate and up slices");
+    for (size_t q = i; q < j; ++q) {
+      const int e = sel[q];
+      const uint8_t *w0 = t0.slices[e].dev, *w1 = t1 ? t1->slices[e].dev : nullptr;
+      if (t0.slices[e].where == ATS_HOST) {
+        const int f = plan_find(ctx, id0, e);
+        ATS_TRY(acquire(ctx, f, &w0));
+        fetches.push_back(f);
+      }
+      if (t1 && t1->slices[e].where == ATS_HOST) {
+        const int f = plan_find(ctx, id1, e);
+        ATS_TRY(acquire(ctx, f, &w1));
+        fetches.push_back(f);
+      }
+      for (int pr = 0; pr < P; ++pr)
+        if (ids_host[pr] == e) ATS_TRY(add_job(pr, w0, w1));
+    }
+    ATS_TRY(flush());
+    for (int f : fetches) ATS_TRY(release(ctx, f));
+    i = j;
+  }
+  return ATS_OK;
+}
+
+// Bring the routing ids to the host (the single host synchronisation of the MoE path) and validate them.
+static int32_t fetch_ids(ats_ctx* ctx, const int32_t* ids_dev, int P, int E) {
+  ATS_CUDA(cudaMemcpyAsync(ctx->ids_host, ids_dev, (size_t)P * 4, cudaMemcpyDeviceToHost, ctx->cs));
+  ATS_CUDA(cudaEventRecord(ctx->ids_event, ctx->cs));
+  ATS_CUDA(cudaEventSynchronize(ctx->ids_event));
+  ctx->stats.host_syncs++;
+  for (int i = 0; i < P; ++i)
+    if (ctx->ids_host[i] < 0 || ctx->ids_host[i] >= E)
+      return fail(ctx, ATS_ERR_INVALID, "routing id %d out of range [0,%d)", ctx->ids_host[i], E);
+  return ATS_OK;
+}
+
+// Plan the streamed slices of an MoE stage set: for each selected expert (ascending) the host-placed gate and up
+// slices, then the host-placed down slices (only selected experts move, Section 4.2.2).
+static void plan_moe(ats_ctx* ctx, const int32_t* ids_host, int P, const int* tensor_ids, int n_first, int n_total) {
+  std::vector<int> sel(ids_host, ids_host + P);
+  std::sort(sel.begin(), sel.end());
+  sel.erase(std::unique(sel.begin(), sel.end()), sel.end());
+  for (int e : sel)
+    for (int t = 0; t < n_first; ++t)
+      if (ctx->tensors[tensor_ids[t]].slices[e].where == ATS_HOST) plan_add(ctx, tensor_ids[t], e);
+  for (int t = n_first; t < n_total; ++t)
+    for (int e : sel)
+      if (ctx->tensors[tensor_ids[t]].slices[e].where == ATS_HOST) plan_add(ctx, tensor_ids[t], e);
+}
+
+}  // namespace ats
+
+using namespace ats;
+
+// ====================================================================================== C ABI
+extern "C" {
+
+int32_t ats_init(const ats_config* cfg, ats_ctx** out) {
+  if (!cfg || !out) return ATS_ERR_INVALID;
+  *out = nullptr;
+  if (!cfg->arena || ((uintptr_t)cfg->arena % kAlign) != 0) return ATS_ERR_INVALID;
+  if (cfg->compute_stream == cfg->transfer_stream) return ATS_ERR_INVALID;
+  const uint64_t slot_stride = align_up(cfg->slot_bytes);
+  const uint64_t ws = align_up(cfg->workspace_bytes);
+  const uint64_t ring_bytes = (uint64_t)cfg->ring_slots * slot_stride;
+  if (ws + ring_bytes > cfg->arena_bytes) return ATS_ERR_INVALID;
+  if (cfg->ring_slots && cfg->slot_bytes == 0) return ATS_ERR_INVALID;
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return ATS_ERR_CUDA;
+  ats_ctx* ctx = new (std::nothrow) ats_ctx();
+  if (!ctx) return ATS_ERR_NOMEM;
+  ctx->cfg = *cfg;
+  ctx->cs = (cudaStream_t)cfg->compute_stream;
+  ctx->ts = (cudaStream_t)cfg->transfer_stream;
+  ctx->ws = (uint8_t*)cfg->arena;
+  ctx->ring = ctx->ws + ws;
+  ctx->slot_stride = slot_stride;
+  ctx->resident = ctx->ring + ring_bytes;
+  ctx->resident_cap = cfg->arena_bytes - ws - ring_bytes;
+  ctx->slots.resize(cfg->ring_slots);
+  bool ok = true;
+  for (RingSlot& s : ctx->slots) {
+    ok &= cudaEventCreateWithFlags(&s.ready, cudaEventDisableTiming) == cudaSuccess;
+    ok &= cudaEventCreateWithFlags(&s.freed, cudaEventDisableTiming) == cudaSuccess;
+  }
+  ok &= cudaEventCreateWithFlags(&ctx->ids_event, cudaEventDisableTiming) == cudaSuccess;
+  ok &= cudaEventCreateWithFlags(&ctx->sync_event, cudaEventDisableTiming) == cudaSuccess;
+  ok &= cudaHostAlloc((void**)&ctx->ids_host, 4096 * sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess;
+  if (!ok) {
+    ats_destroy(ctx);
+    return ATS_ERR_CUDA;
+  }
+  *out = ctx;
+  return ATS_OK;
+}
+
+int32_t ats_destroy(ats_ctx* ctx) {
+  if (!ctx) return ATS_ERR_INVALID;
+  cudaStreamSynchronize(ctx->cs);
+  cudaStreamSynchronize(ctx->ts);
+  for (Tensor& t : ctx->tensors)
+    if (t.host) cudaFreeHost(t.host);
+  for (RingSlot& s : ctx->slots) {
+    if (s.ready) cudaEventDestroy(s.ready);
+    if (s.freed) cudaEventDestroy(s.freed);
+  }
+  if (ctx->ids_event) cudaEventDestroy(ctx->ids_event);
+  if (ctx->sync_event) cudaEventDestroy(ctx->sync_event);
+  if (ctx->ids_host) cudaFreeHost(ctx->ids_host);
+  delete ctx;
+  return ATS_OK;
+}
+
+const char* ats_last_error(const ats_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int32_t ats_register_tensor(ats_ctx* ctx, const ats_tensor_desc* d, const void* codes, const void* scales,
+                            int32_t* out_id) {
+  ATS_TRY(precheck(ctx, false));
+  if (!d || !codes || !out_id) return fail(ctx, ATS_ERR_INVALID, "null argument");
+  if (d->fmt != ATS_FMT_Q4B32 && d->fmt != ATS_FMT_F16) return fail(ctx, ATS_ERR_INVALID, "unknown format %u", d->fmt);
+  if (d->n_out == 0 || d->k_in == 0 || d->n_experts == 0) return fail(ctx, ATS_ERR_SHAPE, "zero dimension");
+  if (d->switch_cost < 0) return fail(ctx, ATS_ERR_INVALID, "switch_cost must be >= 0");
+  Tensor t;
+  t.d = *d;
+  if (d->fmt == ATS_FMT_F16) {
+    if (d->n_experts != 1) return fail(ctx, ATS_ERR_SHAPE, "F16 tensors are not stacked");
+    t.host_bytes = (uint64_t)d->n_out * d->k_in * 2;
+    if (cudaHostAlloc((void**)&t.host, t.host_bytes, cudaHostAllocDefault) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, ATS_ERR_NOMEM, "pinned allocation of %llu bytes failed", (unsigned long long)t.host_bytes);
+    }
+    memcpy(t.host, codes, t.host_bytes);
+  } else {
+    if (d->k_in % kBlock) return fail(ctx, ATS_ERR_SHAPE, "k_in = %u is not a multiple of 32", d->k_in);
+    if (!scales) return fail(ctx, ATS_ERR_INVALID, "null scales");
+    const uint64_t N = d->n_out, K = d->k_in, E = d->n_experts;
+    t.codes_bytes = N * K / 2;
+    t.slice_bytes = t.codes_bytes + N * (K / kBlock) * 2;
+    t.slice_stride = align_up(t.slice_bytes);
+    t.host_bytes = E * t.slice_stride;
+    if (!(ctx->cfg.flags & ATS_FLAG_SKIP_SCALE_CHECK)) {
+      const uint16_t* s = (const uint16_t*)scales;
+      const uint64_t ns = E * N * (K / kBlock);
+      for (uint64_t i = 0; i < ns; ++i)
+        if ((s[i] & 0x7C00u) == 0x7C00u) return fail(ctx, ATS_ERR_INVALID, "scale %llu is Inf or NaN", (unsigned long long)i);
+    }
+    if (cudaHostAlloc((void**)&t.host, t.host_bytes, cudaHostAllocDefault) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, ATS_ERR_NOMEM, "pinned allocation of %llu bytes failed", (unsigned long long)t.host_bytes);
+    }
+    for (uint64_t e = 0; e < E; ++e) {
+      uint8_t* dst = t.host + e * t.slice_stride;
+      repack_q4((const uint8_t*)codes + e * t.codes_bytes, (const uint16_t*)scales + e * N * (K / kBlock), dst, N, K);
+      if (t.slice_stride > t.slice_bytes) memset(dst + t.slice_bytes, 0, t.slice_stride - t.slice_bytes);
+    }
+    t.slices.resize(E);
+    if (t.d.value < 0) t.d.value = (int64_t)(E * t.slice_bytes);
+  }
+  ctx->stats.host_store_bytes += t.host_bytes;
+  ctx->tensors.push_back(std::move(t));
+  ctx->placed = false;
+  *out_id = (int32_t)ctx->tensors.size() - 1;
+  return ATS_OK;
+}
+
+int32_t ats_tensor_slice_bytes(const ats_ctx* ctx, int32_t id, uint64_t* out_bytes) {
+  if (!ctx || !out_bytes || id < 0 || (size_t)id >= ctx->tensors.size()) return ATS_ERR_INVALID;
+  const Tensor& t = ctx->tensors[id];
+  *out_bytes = t.d.fmt == ATS_FMT_F16 ? t.host_bytes : t.slice_bytes;
+  return ATS_OK;
+}
+
+int32_t ats_set_placement(ats_ctx* ctx, const int32_t* ids, const int32_t* experts, const uint8_t* where, uint32_t n) {
+  ATS_TRY(precheck(ctx, false));
+  if (n && (!ids || !where)) return fail(ctx, ATS_ERR_INVALID, "null argument");
+  for (uint32_t i = 0; i < n; ++i) {
+    Tensor* t = get_tensor(ctx, ids[i], ATS_FMT_Q4B32);
+    if (!t) return fail(ctx, ATS_ERR_INVALID, "entry %u: id %d is not a registered Q4B32 tensor", i, ids[i]);
+    const int32_t e = experts ? experts[i] : -1;
+    if (e < -1 || e >= (int32_t)t->slices.size()) return fail(ctx, ATS_ERR_INVALID, "entry %u: expert %d out of range", i, e);
+    if (where[i] != ATS_HOST && where[i] != ATS_GPU) return fail(ctx, ATS_ERR_INVALID, "entry %u: placement %u", i, where[i]);
+  }
+  for (Tensor& t : ctx->tensors)
+    for (Slice& s : t.slices) s.where = ATS_HOST;
+  for (uint32_t i = 0; i < n; ++i) {
+    Tensor& t = ctx->tensors[ids[i]];
+    const int32_t e = experts ? experts[i] : -1;
+    if (e < 0)
+      for (Slice& s : t.slices) s.where = where[i];
+    else
+      t.slices[e].where = where[i];
+  }
+  ctx->placed = false;
+  return apply_placement(ctx);
+}
+
+int32_t ats_plan_placement(ats_ctx* ctx, uint64_t budget_bytes, uint32_t granule_bytes, uint8_t* out_where, uint32_t n) {
+  ATS_TRY(precheck(ctx, false));
+  const uint64_t G = granule_bytes ? granule_bytes : (1u << 20);
+  std::vector<int64_t> s, r, c;
+  std::vector<uint8_t> is_exp;
+  std::vector<int> idx;
+  for (size_t i = 0; i < ctx->tensors.size(); ++i) {
+    const Tensor& t = ctx->tensors[i];
+    if (t.d.fmt != ATS_FMT_Q4B32) continue;
+    const uint64_t bytes = t.slice_bytes * t.slices.size();
+    s.push_back((int64_t)((bytes + G - 1) / G));
+    r.push_back(t.d.value);
+    c.push_back(t.d.switch_cost);
+    is_exp.push_back(t.slices.size() > 1);
+    idx.push_back((int)i);
+  }
+  if (out_where && n != idx.size())
+    return fail(ctx, ATS_ERR_INVALID, "out_where holds %u entries, %zu Q4B32 tensors are registered", n, idx.size());
+  std::vector<uint8_t> b;
+  static_placement(s, r, c, is_exp, (int64_t)(budget_bytes / G), &b);
+  for (size_t j = 0; j < idx.size(); ++j)
+    for (Slice& sl : ctx->tensors[idx[j]].slices) sl.where = b[j];
+  if (out_where) memcpy(out_where, b.data(), b.size());
+  ctx->placed = false;
+  return apply_placement(ctx);
+}
+
+int32_t ats_get_placement(const ats_ctx* ctx, int32_t id, int32_t expert, uint8_t* out_where) {
+  if (!ctx || !out_where) return ATS_ERR_INVALID;
+  if (id < 0 || (size_t)id >= ctx->tensors.size()) return ATS_ERR_INVALID;
+  const Tensor& t = ctx->tensors[id];
+  if (t.d.fmt == ATS_FMT_F16) {
+    *out_where = ATS_GPU;
+    return ATS_OK;
+  }
+  if (expert < 0) expert = 0;
+  if ((size_t)expert >= t.slices.size()) return ATS_ERR_INVALID;
+  *out_where = t.slices[expert].where;
+  return ATS_OK;
+}
+
+int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M) {
+  ATS_TRY(precheck(ctx, true));
+  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", id);
+  if (!x || !y) return fail(ctx, ATS_ERR_INVALID, "null pointer");
+  if (M == 0) return ATS_OK;
+  plan_begin(ctx);
+  Operand op;
+  plan_dense(ctx, id, &op);
+  ATS_TRY(pump(ctx));
+  if (M <= 8) {
+    GemvParams p{};
+    p.M = (int)M;
+    p.x = (const __half*)x;
+    p.ldx = (int)t->d.k_in;
+    p.y16 = (__half*)y;
+    p.ldy = (int)t->d.n_out;
+    p.mode = GEMV_OUT_F16;
+    return run_gemv_group(ctx, &op, 1, p);
+  }
+  GemmParams g{};
+  g.T = (int)M;
+  g.x = (const __half*)x;
+  g.ldx = (int)t->d.k_in;
+  g.y = (__half*)y;
+  g.ldy = (int)t->d.n_out;
+  g.scratch_bytes = gemm_scratch_bytes((int)M, (int)t->d.n_out, (int)t->d.k_in);
+  if (g.scratch_bytes > align_up(ctx->cfg.workspace_bytes))
+    return fail(ctx, ATS_ERR_NOMEM, "workspace too small for the GEMM: need %llu bytes", (unsigned long long)g.scratch_bytes);
+  g.scratch = ctx->ws;
+  return run_gemm_group(ctx, &op, 1, g);
+}
+
+int32_t ats_dequantize(ats_ctx* ctx, int32_t id, int32_t expert, void* out_dev, uint32_t out_fmt) {
+  ATS_TRY(precheck(ctx, true));
+  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not a Q4B32 tensor", id);
+  if (expert < 0 || (size_t)expert >= t->slices.size()) return fail(ctx, ATS_ERR_INVALID, "expert %d out of range", expert);
+  if (!out_dev || out_fmt > ATS_OUT_F16) return fail(ctx, ATS_ERR_INVALID, "bad output argument");
+  plan_begin(ctx);
+  const uint8_t* ptr = t->slices[expert].dev;
+  int f = -1;
+  if (t->slices[expert].where == ATS_HOST) {
+    f = plan_add(ctx, id, expert);
+    ATS_TRY(pump(ctx));
+    ATS_TRY(acquire(ctx, f, &ptr));
+  }
+  ATS_CUDA(launch_dequant(ptr, (int)t->d.n_out, (int)t->d.k_in, out_dev, out_fmt == ATS_OUT_F16, ctx->cs,
+                          &ctx->stats.kernel_launches));
+  if (f >= 0) ATS_TRY(release(ctx, f));
+  return ATS_OK;
+}
+
+int32_t ats_route_topk(ats_ctx* ctx, int32_t router_id, const void* h, uint32_t M, uint32_t k, int32_t* ids_dev,
+                       float* gates_dev) {
+  ATS_TRY(precheck(ctx, true));
+  Tensor* t = get_tensor(ctx, router_id, ATS_FMT_F16);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not an F16 router tensor", router_id);
+  if (!h || !ids_dev || !gates_dev) return fail(ctx, ATS_ERR_INVALID, "null pointer");
+  const uint32_t E = t->d.n_out;
+  if (k == 0 || k > 32 || k > E || E > 1024) return fail(ctx, ATS_ERR_SHAPE, "top-k %u of %u experts unsupported", k, E);
+  if (M == 0) return ATS_OK;
+  ATS_CUDA(launch_router_topk((const __half*)h, (const __half*)t->f16_dev, (int)M, (int)t->d.k_in, (int)E, (int)k, 1,
+                              ids_dev, gates_dev, ctx->cs, &ctx->stats.kernel_launches));
+  return ATS_OK;
+}
+
+int32_t ats_moe_linear(ats_ctx* ctx, int32_t id, const void* x, const int32_t* ids_dev, void* y, uint32_t M, uint32_t k,
+                       uint32_t x_per_slot) {
+  ATS_TRY(precheck(ctx, true));
+  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not a Q4B32 tensor", id);
+  if (!x || !y || !ids_dev) return fail(ctx, ATS_ERR_INVALID, "null pointer");
+  const uint32_t P = M * k;
+  if (P == 0) return ATS_OK;
+  if (P > 256) return fail(ctx, ATS_ERR_SHAPE, "M*k = %u exceeds 256", P);
+  MoeGemvParams p{};
+  p.P = (int)P;
+  p.x_div = x_per_slot ? 1 : (int)k;
+  p.x = (const __half*)x;
+  p.ldx = (int)t->d.k_in;
+  p.y16 = (__half*)y;
+  p.ldy = (int)t->d.n_out;
+  p.mode = GEMV_OUT_F16;
+  plan_begin(ctx);
+  const int32_t* ids_host = nullptr;
+  if (t->any_host || !t->contiguous_dev) {
+    ATS_TRY(fetch_ids(ctx, ids_dev, (int)P, (int)t->slices.size()));
+    ids_host = ctx->ids_host;
+    const int tid = id;
+    plan_moe(ctx, ids_host, (int)P, &tid, 1, 1);
+    ATS_TRY(pump(ctx));
+  }
+  return run_moe_stage(ctx, id, -1, ids_dev, ids_host, p);
+}
+
+static int32_t check_q4(ats_ctx* ctx, int32_t id, uint32_t n_out, uint32_t k_in, uint32_t n_experts, const char* name) {
+  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "layer tensor %s (id %d) is not a registered Q4B32 tensor", name, id);
+  if (t->d.n_out != n_out || t->d.k_in != k_in || t->slices.size() != n_experts)
+    return fail(ctx, ATS_ERR_SHAPE, "layer tensor %s is [%zu][%u][%u], the layer needs [%u][%u][%u]", name, t->slices.size(),
+                t->d.n_out, t->d.k_in, n_experts, n_out, k_in);
+  return ATS_OK;
+}
+static int32_t check_f16(ats_ctx* ctx, int32_t id, uint32_t n_out, uint32_t k_in, const char* name) {
+  Tensor* t = get_tensor(ctx, id, ATS_FMT_F16);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "layer tensor %s (id %d) is not a registered F16 tensor", name, id);
+  if ((uint64_t)t->d.n_out * t->d.k_in != (uint64_t)n_out * k_in)
+    return fail(ctx, ATS_ERR_SHAPE, "layer tensor %s has %u x %u elements, the layer needs %u x %u", name, t->d.k_in, t->d.n_out,
+                k_in, n_out);
+  return ATS_OK;
+}
+
+static int32_t check_layer(ats_ctx* ctx, const ats_layer_desc* L, bool prefill) {
+  if (!L) return fail(ctx, ATS_ERR_INVALID, "null layer descriptor");
+  if (L->hidden == 0 || L->ffn == 0) return fail(ctx, ATS_ERR_SHAPE, "zero hidden/ffn size");
+  if (L->hidden % 32 || L->ffn % 32) return fail(ctx, ATS_ERR_SHAPE, "hidden and ffn must be multiples of 32");
+  if (L->wq >= 0) {
+    if (L->head_dim != 64 && L->head_dim != 128) return fail(ctx, ATS_ERR_UNSUPPORTED, "head_dim %u (64 or 128)", L->head_dim);
+    if (L->n_kv_heads == 0 || L->n_q_heads % L->n_kv_heads) return fail(ctx, ATS_ERR_SHAPE, "n_q_heads %% n_kv_heads != 0");
+    if (L->n_q_heads / L->n_kv_heads > 8) return fail(ctx, ATS_ERR_UNSUPPORTED, "more than 8 query heads per kv head");
+    const uint32_t qd = L->n_q_heads * L->head_dim, kvd = L->n_kv_heads * L->head_dim;
+    ATS_TRY(check_f16(ctx, L->attn_norm, L->hidden, 1, "attn_norm"));
+    ATS_TRY(check_q4(ctx, L->wq, qd, L->hidden, 1, "wq"));
+    ATS_TRY(check_q4(ctx, L->wk, kvd, L->hidden, 1, "wk"));
+    ATS_TRY(check_q4(ctx, L->wv, kvd, L->hidden, 1, "wv"));
+    ATS_TRY(check_q4(ctx, L->wo, L->hidden, qd, 1, "wo"));
+    if (L->kv_capacity == 0) return fail(ctx, ATS_ERR_SHAPE, "kv_capacity is 0");
+  }
+  ATS_TRY(check_f16(ctx, L->ffn_norm, L->hidden, 1, "ffn_norm"));
+  const uint32_t E = L->n_experts ? L->n_experts : 1;
+  if (L->n_experts) {
+    if (prefill) return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE prefill is not implemented");
+    if (L->top_k == 0 || L->top_k > 32 || L->top_k > L->n_experts || L->n_experts > 1024)
+      return fail(ctx, ATS_ERR_SHAPE, "top_k %u of %u experts unsupported", L->top_k, L->n_experts);
+    ATS_TRY(check_f16(ctx, L->router, L->n_experts, L->hidden, "router"));
+  }
+  ATS_TRY(check_q4(ctx, L->w_gate, L->ffn, L->hidden, E, "w_gate"));
+  ATS_TRY(check_q4(ctx, L->w_up, L->ffn, L->hidden, E, "w_up"));
+  ATS_TRY(check_q4(ctx, L->w_down, L->hidden, L->ffn, E, "w_down"));
+  return ATS_OK;
+}
+
+uint64_t ats_workspace_bytes(const ats_layer_desc* L, uint32_t max_tokens) {
+  if (!L || max_tokens == 0) return 0;
+  uint64_t need = layout_decode(*L, std::min<uint32_t>(max_tokens, 32), nullptr, ~0ull).total;
+  if (L->n_experts == 0) need = std::max(need, layout_prefill(*L, max_tokens, nullptr, ~0ull).total);
+  return need + kAlign;
+}
+
+int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in, void* x_out, void* k_cache,
+                         void* v_cache, uint32_t pos, uint32_t M) {
+  ATS_TRY(precheck(ctx, true));
+  ATS_TRY(check_layer(ctx, L, false));
+  if (!x_in || !x_out) return fail(ctx, ATS_ERR_INVALID, "null activation pointer");
+  const bool attn = L->wq >= 0;
+  if (M == 0) return ATS_OK;
+  if (attn && M != 1) return fail(ctx, ATS_ERR_UNSUPPORTED, "decode with attention takes M = 1 (one sequence)");
+  if (!attn && M > 32) return fail(ctx, ATS_ERR_SHAPE, "FFN-only decode takes M <= 32");
+  if (L->n_experts == 0 && M > 8) return fail(ctx, ATS_ERR_SHAPE, "dense decode takes M <= 8");
+  if (attn && (!k_cache || !v_cache)) return fail(ctx, ATS_ERR_INVALID, "null cache pointer");
+  if (attn && pos >= L->kv_capacity) return fail(ctx, ATS_ERR_SHAPE, "pos %u >= kv_capacity %u", pos, L->kv_capacity);
+  LayerWs w = layout_decode(*L, M, ctx->ws, align_up(ctx->cfg.workspace_bytes));
+  if (!w.ok) return fail(ctx, ATS_ERR_NOMEM, "workspace too small: layer needs %llu bytes", (unsigned long long)w.total);
+  uint64_t* nl = &ctx->stats.kernel_launches;
+  const int H = (int)L->hidden, d = (int)L->head_dim, nq = (int)L->n_q_heads, nkv = (int)L->n_kv_heads;
+  const int qd = nq * d, kvd = nkv * d;
+
+  // the execution plan of this call: dense host-placed tensors in execution order
+  plan_begin(ctx);
+  Operand qkv[3], wo, gu[2], wd;
+  if (attn) {
+    plan_dense(ctx, L->wq, &qkv[0]);
+    plan_dense(ctx, L->wk, &qkv[1]);
+    plan_dense(ctx, L->wv, &qkv[2]);
+    plan_dense(ctx, L->wo, &wo);
+  }
+  if (L->n_experts == 0) {
+    plan_dense(ctx, L->w_gate, &gu[0]);
+    plan_dense(ctx, L->w_up, &gu[1]);
+    plan_dense(ctx, L->w_down, &wd);
+  }
+  ATS_TRY(pump(ctx));
+
+  if (attn) {
+    ATS_CUDA(launch_rmsnorm(x_in, 0, (const __half*)ctx->tensors[L->attn_norm].f16_dev, w.h16, (int)M, H, L->rms_eps, ctx->cs, nl));
+    GemvParams p{};
+    p.M = (int)M;
+    p.x = w.h16;
+    p.ldx = H;
+    p.y32 = w.qkv32;
+    p.ldy = qd + 2 * kvd;
+    p.mode = GEMV_OUT_F32;
+    ATS_TRY(run_gemv_group(ctx, qkv, 3, p));
+    ATS_CUDA(launch_rope_append_decode(w.qkv32, w.qrot32, (__half*)k_cache, (__half*)v_cache, nq, nkv, d, (int)L->kv_capacity,
+                                       (int)pos, L->rope_theta, ctx->cs, nl));
+    ATS_CUDA(launch_attn_decode(w.qrot32, (const __half*)k_cache, (const __half*)v_cache, w.attn_scratch, w.a16, nq, nkv, d,
+                                (int)L->kv_capacity, (int)pos + 1, ctx->cs, nl));
+    GemvParams o{};
+    o.M = (int)M;
+    o.x = w.a16;
+    o.ldx = qd;
+    o.y32 = w.x1_32;
+    o.ldy = H;
+    o.res16 = (const __half*)x_in;
+    o.ldres = H;
+    o.mode = GEMV_RES16_OUT_F32;
+    ATS_TRY(run_gemv_group(ctx, &wo, 1, o));
+  }
+  ATS_CUDA(launch_rmsnorm(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev,
+                          w.h2_16, (int)M, H, L->rms_eps, ctx->cs, nl));
+  if (L->n_experts == 0) {
+    GemvParams g{};
+    g.M = (int)M;
+    g.x = w.h2_16;
+    g.ldx = H;
+    g.y16 = w.act16;
+    g.ldy = (int)L->ffn;
+    g.mode = GEMV_SWIGLU_F16;
+    if (count_streamed(gu, 2) > (int)ctx->cfg.ring_slots)
+      return fail(ctx, ATS_ERR_BUDGET, "fused gate/up needs 2 ring slots when both tensors are host-placed");
+    ATS_TRY(run_gemv_group(ctx, gu, 2, g));
+    GemvParams dn{};
+    dn.M = (int)M;
+    dn.x = w.act16;
+    dn.ldx = (int)L->ffn;
+    dn.y16 = (__half*)x_out;
+    dn.ldy = H;
+    dn.ldres = H;
+    if (attn) {
+      dn.res32 = w.x1_32;
+      dn.mode = GEMV_RES32_OUT_F16;
+    } else {
+      dn.res16 = (const __half*)x_in;
+      dn.mode = GEMV_RES16_OUT_F16;
+    }
+    return run_gemv_group(ctx, &wd, 1, dn);
+  }
+  // ---- MoE FFN
+  const int k = (int)L->top_k, P = (int)M * k, E = (int)L->n_experts;
+  ATS_CUDA(launch_router_topk(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)M, H, E, k,
+                              (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, ctx->cs, nl));
+  const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
+  const bool implicit = tg.contiguous_dev && tu.contiguous_dev && td.contiguous_dev;
+  const int32_t* ids_host = nullptr;
+  if (!implicit) {
+    ATS_TRY(fetch_ids(ctx, w.ids, P, E));
+    ids_host = ctx->ids_host;
+    const int tids[3] = {L->w_gate, L->w_up, L->w_down};
+    plan_moe(ctx, ids_host, P, tids, 2, 3);
+    ATS_TRY(pump(ctx));
+  }
+  MoeGemvParams s1{};
+  s1.P = P;
+  s1.x_div = k;
+  s1.x = w.h2_16;
+  s1.ldx = H;
+  s1.y16 = w.act16;
+  s1.ldy = (int)L->ffn;
+  s1.mode = GEMV_SWIGLU_F16;
+  ATS_TRY(run_moe_stage(ctx, L->w_gate, L->w_up, w.ids, ids_host, s1));
+  MoeGemvParams s2{};
+  s2.P = P;
+  s2.x_div = 1;
+  s2.x = w.act16;
+  s2.ldx = (int)L->ffn;
+  s2.y32 = w.d32;
+  s2.ldy = H;
+  s2.mode = GEMV_OUT_F32;
+  ATS_TRY(run_moe_stage(ctx, L->w_down, -1, w.ids, ids_host, s2));
+  ATS_CUDA(launch_moe_combine(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, w.gates, w.d32, (__half*)x_out, (int)M, k, H,
+                              ctx->cs, nl));
+  return ATS_OK;
+}
+
+int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in, void* x_out, void* k_cache,
+                          void* v_cache, uint32_t pos0, uint32_t T) {
+  ATS_TRY(precheck(ctx, true));
+  ATS_TRY(check_layer(ctx, L, true));
+  if (!x_in || !x_out) return fail(ctx, ATS_ERR_INVALID, "null activation pointer");
+  if (T == 0) return ATS_OK;
+  const bool attn = L->wq >= 0;
+  if (attn && (!k_cache || !v_cache)) return fail(ctx, ATS_ERR_INVALID, "null cache pointer");
+  if (attn && (uint64_t)pos0 + T > L->kv_capacity)
+    return fail(ctx, ATS_ERR_SHAPE, "pos0 + T = %llu exceeds kv_capacity %u", (unsigned long long)pos0 + T, L->kv_capacity);
+  LayerWs w = layout_prefill(*L, T, ctx->ws, align_up(ctx->cfg.workspace_bytes));
+  if (!w.ok) return fail(ctx, ATS_ERR_NOMEM, "workspace too small: prefill of %u tokens needs %llu bytes", T, (unsigned long long)w.total);
+  uint64_t* nl = &ctx->stats.kernel_launches;
+  const int H = (int)L->hidden, d = (int)L->head_dim, nq = (int)L->n_q_heads, nkv = (int)L->n_kv_heads;
+  const int qd = nq * d, kvd = nkv * d;
+
+  plan_begin(ctx);
+  Operand qkv[3], wo, gu[2], wd;
+  if (attn) {
+    plan_dense(ctx, L->wq, &qkv[0]);
+    plan_dense(ctx, L->wk, &qkv[1]);
+    plan_dense(ctx, L->wv, &qkv[2]);
+    plan_dense(ctx, L->wo, &wo);
+  }
+  plan_dense(ctx, L->w_gate, &gu[0]);
+  plan_dense(ctx, L->w_up, &gu[1]);
+  plan_dense(ctx, L->w_down, &wd);
+  ATS_TRY(pump(ctx));
+
+  GemmParams g{};
+  g.T = (int)T;
+  g.scratch = w.gemm_scratch;
+  g.scratch_bytes = w.gemm_scratch_bytes;
+  const __half* resid = (const __half*)x_in;
+  if (attn) {
+    ATS_CUDA(launch_rmsnorm(x_in, 0, (const __half*)ctx->tensors[L->attn_norm].f16_dev, w.h16, (int)T, H, L->rms_eps, ctx->cs, nl));
+    g.x = w.h16;
+    g.ldx = H;
+    g.y = w.qkv16;
+    g.ldy = qd + 2 * kvd;
+    ATS_TRY(run_gemm_group(ctx, qkv, 3, g));
+    ATS_CUDA(launch_rope_append_prefill(w.qkv16, qd + 2 * kvd, w.qrot16, (__half*)k_cache, (__half*)v_cache, (int)T, nq, nkv, d,
+                                        (int)L->kv_capacity, (int)pos0, L->rope_theta, ctx->cs, nl));
+    ATS_CUDA(launch_attn_prefill(w.qrot16, (const __half*)k_cache, (const __half*)v_cache, w.a16, (int)T, nq, nkv, d,
+                                 (int)L->kv_capacity, (int)pos0, ctx->cs, nl));
+    g.x = w.a16;
+    g.ldx = qd;
+    g.y = w.o16;
+    g.ldy = H;
+    ATS_TRY(run_gemm_group(ctx, &wo, 1, g));
+    ATS_CUDA(launch_add16((const __half*)x_in, w.o16, w.x1_16, (uint64_t)T * H, ctx->cs, nl));
+    resid = w.x1_16;
+  }
+  ATS_CUDA(launch_rmsnorm(resid, 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, w.h2_16, (int)T, H, L->rms_eps, ctx->cs, nl));
+  g.x = w.h2_16;
+  g.ldx = H;
+  g.y = w.gu16;
+  g.ldy = 2 * (int)L->ffn;
+  ATS_TRY(run_gemm_group(ctx, gu, 2, g));
+  ATS_CUDA(launch_swiglu16(w.gu16, 2 * (int)L->ffn, (int)L->ffn, w.act16, (int)T, ctx->cs, nl));
+  g.x = w.act16;
+  g.ldx = (int)L->ffn;
+  g.y = w.d16;
+  g.ldy = H;
+  ATS_TRY(run_gemm_group(ctx, &wd, 1, g));
+  ATS_CUDA(launch_add16(resid, w.d16, (__half*)x_out, (uint64_t)T * H, ctx->cs, nl));
+  return ATS_OK;
+}
+
+int32_t ats_get_numerics(const ats_ctx* ctx, uint32_t mode, uint32_t* fp16_edge_mask, uint32_t* weight_mode) {
+  if (!ctx || !fp16_edge_mask || !weight_mode) return ATS_ERR_INVALID;
+  // edge bits: h=0 q=1 k=2 v=3 q_rot=4 a=5 o=6 x1=7 h2=8 g=9 u=10 act=11 d=12
+  if (mode == ATS_MODE_DECODE) {
+    *fp16_edge_mask = (1u << 0) | (1u << 5) | (1u << 8) | (1u << 11);  // the GEMV inputs h, a, h2, act
+    *weight_mode = 0;
+  } else if (mode == ATS_MODE_PREFILL) {
+    *fp16_edge_mask = (1u << 13) - 1;  // every intermediate is stored as fp16
+    *weight_mode = 1;
+  } else {
+    return ATS_ERR_INVALID;
+  }
+  return ATS_OK;
+}
+
+int32_t ats_get_stats(const ats_ctx* ctx, ats_stats* out) {
+  if (!ctx || !out) return ATS_ERR_INVALID;
+  *out = ctx->stats;
+  return ATS_OK;
+}
+
+int32_t ats_reset_stats(ats_ctx* ctx) {
+  if (!ctx) return ATS_ERR_INVALID;
+  ats_stats& s = ctx->stats;
+  s.streamed_bytes = s.copies = s.kernel_launches = s.ring_reuses = s.host_syncs = 0;
+  s.n_streamed = 0;
+  return ATS_OK;
+}
+
+int32_t ats_sync(ats_ctx* ctx, uint32_t timeout_ms) {
+  if (!ctx) return ATS_ERR_INVALID;
+  if (ctx->poisoned) return fail(ctx, ATS_ERR_CUDA, "context is poisoned: %s", std::string(ctx->err).c_str());
+  const auto t0 = std::chrono::steady_clock::now();
+  cudaStream_t streams[2] = {ctx->ts, ctx->cs};
+  for (cudaStream_t st : streams) {
+    ATS_CUDA(cudaEventRecord(ctx->sync_event, st));
+    for (;;) {
+      cudaError_t e = cudaEventQuery(ctx->sync_event);
+      if (e == cudaSuccess) break;
+      if (e != cudaErrorNotReady) return check_cuda(ctx, e, "ats_sync");
+      if (timeout_ms) {
+        const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+        if (ms >= (long long)timeout_ms) return fail(ctx, ATS_ERR_TIMEOUT, "ats_sync: still running after %u ms", timeout_ms);
+      }
+      std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return check_cuda(ctx, e, "asynchronous error");
+  return ATS_OK;
+}
+
+int32_t ats_measure_h2d(ats_ctx* ctx, uint64_t bytes, uint32_t reps, double* out_gbs) {
+  ATS_TRY(precheck(ctx, false));
+  if (!out_gbs || bytes == 0 || reps == 0) return fail(ctx, ATS_ERR_INVALID, "bad argument");
+  const uint64_t ring_bytes = (uint64_t)ctx->cfg.ring_slots * ctx->slot_stride;
+  if (bytes > ring_bytes) return fail(ctx, ATS_ERR_BUDGET, "%llu bytes exceed the ring (%llu)", (unsigned long long)bytes, (unsigned long long)ring_bytes);
+  ATS_CUDA(cudaStreamSynchronize(ctx->cs));
+  ATS_CUDA(cudaStreamSynchronize(ctx->ts));
+  void* hbuf = nullptr;
+  if (cudaHostAlloc(&hbuf, bytes, cudaHostAllocDefault) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(ctx, ATS_ERR_NOMEM, "pinned allocation of %llu bytes failed", (unsigned long long)bytes);
+  }
+  memset(hbuf, 1, bytes);
+  cudaEvent_t a, b;
+  cudaEventCreate(&a);
+  cudaEventCreate(&b);
+  float best = 1e30f;
+  int32_t st = ATS_OK;
+  for (uint32_t r = 0; r < reps && st == ATS_OK; ++r) {
+    cudaEventRecord(a, ctx->ts);
+    cudaError_t e = cudaMemcpyAsync(ctx->ring, hbuf, bytes, cudaMemcpyHostToDevice, ctx->ts);
+    cudaEventRecord(b, ctx->ts);
+    if (e == cudaSuccess) e = cudaEventSynchronize(b);
+    st = check_cuda(ctx, e, "ats_measure_h2d copy");
+    float ms = 0;
+    if (st == ATS_OK && cudaEventElapsedTime(&ms, a, b) == cudaSuccess && ms > 0) best = std::min(best, ms);
+  }
+  cudaEventDestroy(a);
+  cudaEventDestroy(b);
+  cudaFreeHost(hbuf);
+  if (st != ATS_OK) return st;
+  *out_gbs = (double)bytes / (best * 1e-3) / 1e9;
+  return ATS_OK;
+}
+
+int32_t ats_debug_decode_buffer(ats_ctx* ctx, const ats_layer_desc* L, uint32_t M, uint32_t which, void** out_dev,
+                                uint64_t* out_bytes) {
+  if (!ctx || !L || !out_dev || !out_bytes || M == 0) return ATS_ERR_INVALID;
+  LayerWs w = layout_decode(*L, M, ctx->ws, align_up(ctx->cfg.workspace_bytes));
+  if (!w.ok) return fail(ctx, ATS_ERR_NOMEM, "workspace too small");
+  const uint64_t H = L->hidden, qd = (uint64_t)L->n_q_heads * L->head_dim, kvd = (uint64_t)L->n_kv_heads * L->head_dim;
+  const uint64_t P = (uint64_t)M * (L->n_experts ? L->top_k : 1);
+  switch (which) {
+    case 0: *out_dev = w.h16; *out_bytes = M * H * 2; break;
+    case 1: *out_dev = w.qkv32; *out_bytes = M * (qd + 2 * kvd) * 4; break;
+    case 2: *out_dev = w.qrot32; *out_bytes = M * qd * 4; break;
+    case 3: *out_dev = w.a16; *out_bytes = M * qd * 2; break;
+    case 4: *out_dev = w.x1_32; *out_bytes = M * H * 4; break;
+    case 5: *out_dev = w.h2_16; *out_bytes = M * H * 2; break;
+    case 6: *out_dev = w.act16; *out_bytes = P * L->ffn * 2; break;
+    case 7: *out_dev = w.d32; *out_bytes = P * H * 4; break;
+    case 8: *out_dev = w.ids; *out_bytes = P * 4; break;
+    case 9: *out_dev = w.gates; *out_bytes = P * 4; break;
+    default: return fail(ctx, ATS_ERR_INVALID, "unknown buffer %u", which);
+  }
+  if (!*out_dev) return fail(ctx, ATS_ERR_INVALID, "buffer %u is not part of this layer", which);
+  return ATS_OK;
+}
+
+int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n) {
+  if (!ctx) return ATS_ERR_INVALID;
+  ctx->fail_copies = n;
+  return ATS_OK;
+}
+
+}  // extern "C"

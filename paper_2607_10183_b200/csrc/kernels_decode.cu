@@ -1,0 +1,746 @@
+// Decode-side CUDA kernels (sm_100a): block dequantization, the dequantize-fused GEMV (dense and grouped-expert),
+// RMSNorm, rotary embedding + KV append, split attention over the KV cache, router top-k and the MoE combine.
+//
+// The GEMV is memory-bound: 4.5 bits per weight must cross HBM once.  Every lane loads one quantization block per
+// step with a single 128-bit load (32 codes) plus its fp16 scale, expands the nibbles to exact fp16 integers with
+// two logic ops and one half2 op per pair, accumulates sum_k code*x in fp32 per block, and applies the block scale
+// once: y += scale * sum.  No tensor cores, no atomics; reductions run in a fixed order so results are reproducible
+// run to run and independent of where the weight bytes live (resident region or staging slot).
+#include "ats_internal.h"
+
+namespace ats {
+
+// ------------------------------------------------------------------------------------------- helpers
+__device__ __forceinline__ __half2 u32_as_half2(uint32_t v) {
+  __half2 h;
+  *reinterpret_cast<uint32_t*>(&h) = v;
+  return h;
+}
+
+// One 32-bit word of the internal format -> 8 exact fp16 codes as the pairs (k0,k1) (k2,k3) (k4,k5) (k6,k7).
+// Nibble u = code + 8.  (w & 0x000F000F) | 0x6400 is the fp16 pair 1024 + u; the 0x00F000F0 pair is 1024 + 16u.
+__device__ __forceinline__ void unpack8(uint32_t w, __half2 (&c)[4]) {
+  const uint32_t kMagic = 0x64006400u;
+  const __half2 k1032 = u32_as_half2(0x64086408u);   // 1032
+  const __half2 k16th = u32_as_half2(0x2C002C00u);   // 1/16
+  const __half2 kM72 = u32_as_half2(0xD480D480u);    // -72 = -(1024/16 + 8)
+  const uint32_t w8 = w >> 8;
+  c[0] = __hsub2(u32_as_half2((w & 0x000F000Fu) | kMagic), k1032);
+  c[1] = __hfma2(u32_as_half2((w & 0x00F000F0u) | kMagic), k16th, kM72);
+  c[2] = __hsub2(u32_as_half2((w8 & 0x000F000Fu) | kMagic), k1032);
+  c[3] = __hfma2(u32_as_half2((w8 & 0x00F000F0u) | kMagic), k16th, kM72);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.0f + expf(-g)) * u; }
+
+// ------------------------------------------------------------------------------------------- dequantize (a1)
+template <bool F16>
+__global__ void dequant_kernel(const uint8_t* __restrict__ slice, int n_rows, int K, void* __restrict__ out) {
+  const uint64_t words = (uint64_t)n_rows * K / 8;
+  const uint32_t* codes = reinterpret_cast<const uint32_t*>(slice);
+  const __half* scales = reinterpret_cast<const __half*>(slice + (uint64_t)n_rows * K / 2);
+  for (uint64_t w = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; w < words; w += (uint64_t)gridDim.x * blockDim.x) {
+    __half2 c[4];
+    unpack8(codes[w], c);
+    const __half s = scales[w / 4];  // 4 words per block of 32
+    if (F16) {
+      const __half2 s2 = __half2half2(s);
+      uint4 o;
+      __half2 r0 = __hmul2(c[0], s2), r1 = __hmul2(c[1], s2), r2 = __hmul2(c[2], s2), r3 = __hmul2(c[3], s2);
+      o.x = *reinterpret_cast<uint32_t*>(&r0);
+      o.y = *reinterpret_cast<uint32_t*>(&r1);
+      o.z = *reinterpret_cast<uint32_t*>(&r2);
+      o.w = *reinterpret_cast<uint32_t*>(&r3);
+      reinterpret_cast<uint4*>(out)[w] = o;
+    } else {
+      const float sf = __half2float(s);
+      float4 a, b;
+      float2 f;
+      f = __half22float2(c[0]); a.x = sf * f.x; a.y = sf * f.y;
+      f = __half22float2(c[1]); a.z = sf * f.x; a.w = sf * f.y;
+      f = __half22float2(c[2]); b.x = sf * f.x; b.y = sf * f.y;
+      f = __half22float2(c[3]); b.z = sf * f.x; b.w = sf * f.y;
+      reinterpret_cast<float4*>(out)[2 * w] = a;
+      reinterpret_cast<float4*>(out)[2 * w + 1] = b;
+    }
+  }
+}
+
+cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, cudaStream_t st,
+                           uint64_t* n_launch) {
+  const uint64_t words = (uint64_t)n_rows * K / 8;
+  const int block = 256;
+  const int grid = (int)std::min<uint64_t>((words + block - 1) / block, 148 * 16);
+  if (out_f16)
+    dequant_kernel<true><<<grid, block, 0, st>>>(slice, n_rows, K, out);
+  else
+    dequant_kernel<false><<<grid, block, 0, st>>>(slice, n_rows, K, out);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------- GEMV core (a2, a5)
+constexpr int kGemvMaxWarps = 8;
+constexpr int kWR = 4;  // weight rows a CTA works on at once
+
+// Accumulate WR weight rows against M activation rows over the blocks this thread owns.
+// cptr[i]: row i's codes as uint4 (one per block of 32); sptr[i]: row i's scales.
+template <int M>
+__device__ __forceinline__ void gemv_accumulate(const uint4* const (&cptr)[kWR], const __half* const (&sptr)[kWR],
+                                                const bool (&valid)[kWR], const __half* __restrict__ x, int ldx, int nblk,
+                                                float (&acc)[kWR][M]) {
+  const int nthreads = blockDim.x;
+  for (int blk = threadIdx.x; blk < nblk; blk += nthreads) {
+    uint4 q[kWR];
+    float s[kWR];
+#pragma unroll
+    for (int i = 0; i < kWR; ++i) {
+      if (valid[i]) {
+        q[i] = __ldg(cptr[i] + blk);
+        s[i] = __half2float(sptr[i][blk]);
+      } else {
+        q[i] = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);
+        s[i] = 0.f;
+      }
+    }
+    float part[kWR][M];
+#pragma unroll
+    for (int i = 0; i < kWR; ++i)
+#pragma unroll
+      for (int m = 0; m < M; ++m) part[i][m] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float xf[M][8];
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * ldx + (size_t)blk * 32 + j * 8));
+        float2 f;
+        f = __half22float2(u32_as_half2(xv.x)); xf[m][0] = f.x; xf[m][1] = f.y;
+        f = __half22float2(u32_as_half2(xv.y)); xf[m][2] = f.x; xf[m][3] = f.y;
+        f = __half22float2(u32_as_half2(xv.z)); xf[m][4] = f.x; xf[m][5] = f.y;
+        f = __half22float2(u32_as_half2(xv.w)); xf[m][6] = f.x; xf[m][7] = f.y;
+      }
+#pragma unroll
+      for (int i = 0; i < kWR; ++i) {
+        const uint32_t word = j == 0 ? q[i].x : j == 1 ? q[i].y : j == 2 ? q[i].z : q[i].w;
+        __half2 c[4];
+        unpack8(word, c);
+        float cf[8];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const float2 f = __half22float2(c[t]);
+          cf[2 * t] = f.x;
+          cf[2 * t + 1] = f.y;
+        }
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+#pragma unroll
+          for (int t = 0; t < 8; ++t) part[i][m] = fmaf(cf[t], xf[m][t], part[i][m]);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kWR; ++i)
+#pragma unroll
+      for (int m = 0; m < M; ++m) acc[i][m] = fmaf(s[i], part[i][m], acc[i][m]);
+  }
+}
+
+// Sum acc over the CTA in a fixed order (lanes by butterfly, warps ascending); the totals land in tot[] (shared).
+template <int M>
+__device__ __forceinline__ void gemv_reduce(float (&acc)[kWR][M], float* red /*[kGemvMaxWarps][kWR*M]*/, float* tot /*[kWR*M]*/) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+#pragma unroll
+  for (int i = 0; i < kWR; ++i)
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const float v = warp_sum(acc[i][m]);
+      if (lane == 0) red[warp * (kWR * M) + i * M + m] = v;
+    }
+  __syncthreads();
+  if (threadIdx.x < kWR * M) {
+    float t = 0.f;
+    for (int w = 0; w < nwarps; ++w) t += red[w * (kWR * M) + threadIdx.x];
+    tot[threadIdx.x] = t;
+  }
+  __syncthreads();
+}
+
+template <int M, bool SW>
+__global__ void __launch_bounds__(kGemvMaxWarps * 32) gemv_kernel(const GemvParams p) {
+  __shared__ float red[kGemvMaxWarps * kWR * M];
+  __shared__ float tot[kWR * M];
+  const int K = p.K, nblk = K / 32;
+  const uint4* cptr[kWR];
+  const __half* sptr[kWR];
+  bool valid[kWR];
+  int orow[kWR];  // output row (global, across segments)
+#pragma unroll
+  for (int i = 0; i < kWR; ++i) {
+    int s, r;
+    if (SW) {
+      s = i & 1;
+      r = blockIdx.x * (kWR / 2) + (i >> 1);
+      valid[i] = r < p.seg[0].n_rows;
+      orow[i] = r;
+    } else {
+      r = blockIdx.x * kWR + i;
+      orow[i] = r;
+      s = 0;
+      while (s < p.n_seg - 1 && r >= p.seg[s].n_rows) {
+        r -= p.seg[s].n_rows;
+        ++s;
+      }
+      valid[i] = r < p.seg[s].n_rows;
+    }
+    const uint8_t* base = p.seg[s].base;
+    cptr[i] = reinterpret_cast<const uint4*>(base + (size_t)r * (K / 2));
+    sptr[i] = reinterpret_cast<const __half*>(base + (size_t)p.seg[s].n_rows * (K / 2)) + (size_t)r * nblk;
+  }
+  float acc[kWR][M];
+#pragma unroll
+  for (int i = 0; i < kWR; ++i)
+#pragma unroll
+    for (int m = 0; m < M; ++m) acc[i][m] = 0.f;
+  gemv_accumulate<M>(cptr, sptr, valid, p.x, p.ldx, nblk, acc);
+  gemv_reduce<M>(acc, red, tot);
+
+  if (SW) {
+    if (threadIdx.x < (kWR / 2) * M) {
+      const int i2 = threadIdx.x / M, m = threadIdx.x % M;
+      const int row = blockIdx.x * (kWR / 2) + i2;
+      if (row < p.seg[0].n_rows) {
+        const float g = tot[(2 * i2) * M + m], u = tot[(2 * i2 + 1) * M + m];
+        p.y16[(size_t)m * p.ldy + row] = __float2half_rn(silu_mul(g, u));
+      }
+    }
+    return;
+  }
+  if (threadIdx.x < kWR * M) {
+    const int i = threadIdx.x / M, m = threadIdx.x % M;
+    // valid[]/orow[] are per-thread copies of the same values; recompute validity for row i
+    int r = blockIdx.x * kWR + i, total = 0;
+    for (int s = 0; s < p.n_seg; ++s) total += p.seg[s].n_rows;
+    if (r < total) {
+      const float v = tot[i * M + m];
+      const size_t o = (size_t)m * p.ldy + r;
+      switch (p.mode) {
+        case GEMV_OUT_F32: p.y32[o] = v; break;
+        case GEMV_OUT_F16: p.y16[o] = __float2half_rn(v); break;
+        case GEMV_RES16_OUT_F32: p.y32[o] = __half2float(p.res16[(size_t)m * p.ldres + r]) + v; break;
+        case GEMV_RES32_OUT_F16: p.y16[o] = __float2half_rn(p.res32[(size_t)m * p.ldres + r] + v); break;
+        case GEMV_RES16_OUT_F16: p.y16[o] = __float2half_rn(__half2float(p.res16[(size_t)m * p.ldres + r]) + v); break;
+        default: break;
+      }
+    }
+  }
+}
+
+static int gemv_threads(int K) {
+  const int nblk = K / 32;
+  int warps = (nblk + 31) / 32;
+  warps = std::max(1, std::min(warps, kGemvMaxWarps));
+  return warps * 32;
+}
+
+template <int M>
+static void launch_gemv_m(const GemvParams& p, int grid, int block, cudaStream_t st) {
+  if (p.mode == GEMV_SWIGLU_F16)
+    gemv_kernel<M, true><<<grid, block, 0, st>>>(p);
+  else
+    gemv_kernel<M, false><<<grid, block, 0, st>>>(p);
+}
+
+cudaError_t launch_gemv(const GemvParams& p, cudaStream_t st, uint64_t* n_launch) {
+  int total = 0;
+  for (int s = 0; s < p.n_seg; ++s) total += p.seg[s].n_rows;
+  const bool sw = p.mode == GEMV_SWIGLU_F16;
+  const int rows_per_cta = sw ? kWR / 2 : kWR;
+  const int out_rows = sw ? p.seg[0].n_rows : total;
+  const int grid = (out_rows + rows_per_cta - 1) / rows_per_cta;
+  const int block = gemv_threads(p.K);
+  switch (p.M) {
+    case 1: launch_gemv_m<1>(p, grid, block, st); break;
+    case 2: launch_gemv_m<2>(p, grid, block, st); break;
+    case 3: launch_gemv_m<3>(p, grid, block, st); break;
+    case 4: launch_gemv_m<4>(p, grid, block, st); break;
+    case 5: launch_gemv_m<5>(p, grid, block, st); break;
+    case 6: launch_gemv_m<6>(p, grid, block, st); break;
+    case 7: launch_gemv_m<7>(p, grid, block, st); break;
+    case 8: launch_gemv_m<8>(p, grid, block, st); break;
+    default: return cudaErrorInvalidValue;
+  }
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+// Grouped-expert GEMV: blockIdx.y = job (one (token, slot) pair), blockIdx.x = row group of that expert's matrix.
+template <bool SW, bool EXPLICIT>
+__global__ void __launch_bounds__(kGemvMaxWarps * 32)
+    moe_gemv_kernel(const MoeGemvParams p, const __grid_constant__ MoeJobs jobs) {
+  __shared__ float red[kGemvMaxWarps * kWR];
+  __shared__ float tot[kWR];
+  const int job = blockIdx.y;
+  const uint8_t *b0, *b1;
+  int xrow, out_row;
+  if (EXPLICIT) {
+    b0 = jobs.w0[job];
+    b1 = jobs.w1[job];
+    xrow = jobs.xrow[job];
+    out_row = jobs.orow[job];
+  } else {
+    const int e = p.ids[job];
+    b0 = p.base0 + (size_t)e * p.stride;
+    b1 = SW ? p.base1 + (size_t)e * p.stride : nullptr;
+    xrow = job / p.x_div;
+    out_row = job;
+  }
+  const int K = p.K, nblk = K / 32, N = p.n_rows;
+  const uint4* cptr[kWR];
+  const __half* sptr[kWR];
+  bool valid[kWR];
+#pragma unroll
+  for (int i = 0; i < kWR; ++i) {
+    const int r = SW ? blockIdx.x * (kWR / 2) + (i >> 1) : blockIdx.x * kWR + i;
+    const uint8_t* base = (SW && (i & 1)) ? b1 : b0;
+    valid[i] = r < N;
+    cptr[i] = reinterpret_cast<const uint4*>(base + (size_t)r * (K / 2));
+    sptr[i] = reinterpret_cast<const __half*>(base + (size_t)N * (K / 2)) + (size_t)r * nblk;
+  }
+  float acc[kWR][1];
+#pragma unroll
+  for (int i = 0; i < kWR; ++i) acc[i][0] = 0.f;
+  gemv_accumulate<1>(cptr, sptr, valid, p.x + (size_t)xrow * p.ldx, p.ldx, nblk, acc);
+  gemv_reduce<1>(acc, red, tot);
+  if (SW) {
+    if (threadIdx.x < kWR / 2) {
+      const int row = blockIdx.x * (kWR / 2) + threadIdx.x;
+      if (row < N)
+        p.y16[(size_t)out_row * p.ldy + row] = __float2half_rn(silu_mul(tot[2 * threadIdx.x], tot[2 * threadIdx.x + 1]));
+    }
+  } else if (threadIdx.x < kWR) {
+    const int row = blockIdx.x * kWR + threadIdx.x;
+    if (row < N) {
+      if (p.mode == GEMV_OUT_F32)
+        p.y32[(size_t)out_row * p.ldy + row] = tot[threadIdx.x];
+      else
+        p.y16[(size_t)out_row * p.ldy + row] = __float2half_rn(tot[threadIdx.x]);
+    }
+  }
+}
+
+cudaError_t launch_moe_gemv(const MoeGemvParams& p, const MoeJobs* jobs, cudaStream_t st, uint64_t* n_launch) {
+  const bool sw = p.mode == GEMV_SWIGLU_F16;
+  const int rows_per_cta = sw ? kWR / 2 : kWR;
+  const int gx = (p.n_rows + rows_per_cta - 1) / rows_per_cta;
+  const int block = gemv_threads(p.K);
+  if (jobs) {
+    dim3 grid(gx, jobs->n);
+    if (sw)
+      moe_gemv_kernel<true, true><<<grid, block, 0, st>>>(p, *jobs);
+    else
+      moe_gemv_kernel<false, true><<<grid, block, 0, st>>>(p, *jobs);
+  } else {
+    static const MoeJobs none{};
+    dim3 grid(gx, p.P);
+    if (sw)
+      moe_gemv_kernel<true, false><<<grid, block, 0, st>>>(p, none);
+    else
+      moe_gemv_kernel<false, false><<<grid, block, 0, st>>>(p, none);
+  }
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------- RMSNorm (a6)
+template <typename TIn>
+__device__ __forceinline__ float load_f(const TIn* p, size_t i);
+template <>
+__device__ __forceinline__ float load_f<float>(const float* p, size_t i) { return p[i]; }
+template <>
+__device__ __forceinline__ float load_f<__half>(const __half* p, size_t i) { return __half2float(p[i]); }
+
+template <typename TIn>
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const TIn* __restrict__ x, const __half* __restrict__ gain,
+                                                      __half* __restrict__ out, int H, float eps) {
+  __shared__ float red[8];
+  __shared__ float inv_s;
+  const TIn* xr = x + (size_t)blockIdx.x * H;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    const float v = load_f<TIn>(xr, i);
+    ss = fmaf(v, v, ss);
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+    inv_s = 1.0f / sqrtf(t / (float)H + eps);
+  }
+  __syncthreads();
+  const float inv = inv_s;
+  for (int i = threadIdx.x; i < H; i += blockDim.x)
+    out[(size_t)blockIdx.x * H + i] = __float2half_rn(load_f<TIn>(xr, i) * __half2float(gain[i]) * inv);
+}
+
+cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
+                           cudaStream_t st, uint64_t* n_launch) {
+  if (x_is_f32)
+    rmsnorm_kernel<float><<<M, 256, 0, st>>>((const float*)x, gain, out, H, eps);
+  else
+    rmsnorm_kernel<__half><<<M, 256, 0, st>>>((const __half*)x, gain, out, H, eps);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------- RoPE + KV append (decode)
+// Half-split pairing: (u_i, u_{i+d/2}) rotated by pos * theta^(-2i/d); the angle is formed in fp64.
+__device__ __forceinline__ void rope_cs(int i, int d, int pos, float theta, float* c, float* s) {
+  if (theta == 0.f) {
+    *c = 1.f;
+    *s = 0.f;
+    return;
+  }
+  const double inv = pow((double)theta, -2.0 * (double)i / (double)d);
+  double sd, cd;
+  sincos((double)pos * inv, &sd, &cd);
+  *c = (float)cd;
+  *s = (float)sd;
+}
+
+__global__ void rope_append_decode_kernel(const float* __restrict__ qkv, float* __restrict__ q_rot, __half* __restrict__ kc,
+                                          __half* __restrict__ vc, int n_q, int n_kv, int d, int cap, int pos, float theta) {
+  const int half = d / 2;
+  const int n_pairs = (n_q + n_kv) * half;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int qd = n_q * d, kvd = n_kv * d;
+  if (idx < n_pairs) {
+    const int hh = idx / half, i = idx % half;
+    float c, s;
+    rope_cs(i, d, pos, theta, &c, &s);
+    if (hh < n_q) {
+      const float a = qkv[hh * d + i], b = qkv[hh * d + i + half];
+      q_rot[hh * d + i] = a * c - b * s;
+      q_rot[hh * d + i + half] = b * c + a * s;
+    } else {
+      const int kvh = hh - n_q;
+      const float a = qkv[qd + kvh * d + i], b = qkv[qd + kvh * d + i + half];
+      __half* dst = kc + ((size_t)kvh * cap + pos) * d;
+      dst[i] = __float2half_rn(a * c - b * s);
+      dst[i + half] = __float2half_rn(b * c + a * s);
+    }
+  } else if (idx < n_pairs + kvd) {
+    const int j = idx - n_pairs;
+    const int kvh = j / d, e = j % d;
+    vc[((size_t)kvh * cap + pos) * d + e] = __float2half_rn(qkv[qd + kvd + j]);
+  }
+}
+
+cudaError_t launch_rope_append_decode(const float* qkv, float* q_rot, __half* kc, __half* vc, int n_q, int n_kv, int d,
+                                      int cap, int pos, float theta, cudaStream_t st, uint64_t* n_launch) {
+  const int total = (n_q + n_kv) * (d / 2) + n_kv * d;
+  rope_append_decode_kernel<<<(total + 127) / 128, 128, 0, st>>>(qkv, q_rot, kc, vc, n_q, n_kv, d, cap, pos, theta);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------- decode attention
+// Split over cache positions: CTA (split, kv head) covers 128 positions, one per lane of its 4 warps, for all query
+// heads of the group.  Partials (running max, sum, unnormalised output) go to scratch; a second kernel merges the
+// splits in ascending order.
+constexpr int kAttnPosPerCta = 128;
+constexpr int kAttnMaxGroup = 8;
+
+int attn_decode_splits(int n_ctx) { return (n_ctx + kAttnPosPerCta - 1) / kAttnPosPerCta; }
+size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) {
+  return (size_t)n_q * attn_decode_splits(n_ctx) * (d + 2);
+}
+
+template <int D>
+__global__ void __launch_bounds__(128) attn_decode_partial_kernel(const float* __restrict__ q_rot, const __half* __restrict__ kc,
+                                                                  const __half* __restrict__ vc, float* __restrict__ part,
+                                                                  int group, int cap, int n_ctx, int n_splits, float scale) {
+  constexpr int V = D / 32;  // output dims per lane
+  __shared__ float q_s[kAttnMaxGroup * D];
+  __shared__ float w_m[4][kAttnMaxGroup], w_l[4][kAttnMaxGroup];
+  __shared__ float w_acc[4][kAttnMaxGroup][D];
+  const int split = blockIdx.x, kvh = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int i = threadIdx.x; i < group * D; i += blockDim.x) q_s[i] = q_rot[(size_t)kvh * group * D + i];
+  __syncthreads();
+  const int t0 = split * kAttnPosPerCta + warp * 32;
+  const int t = t0 + lane;
+  const bool ok = t < n_ctx;
+  float sc[kAttnMaxGroup];
+#pragma unroll
+  for (int g = 0; g < kAttnMaxGroup; ++g) sc[g] = 0.f;
+  if (ok) {
+    const uint4* kr = reinterpret_cast<const uint4*>(kc + ((size_t)kvh * cap + t) * D);
+#pragma unroll 4
+    for (int c = 0; c < D / 8; ++c) {
+      const uint4 kv = __ldg(kr + c);
+      float kf[8];
+      float2 f;
+      f = __half22float2(u32_as_half2(kv.x)); kf[0] = f.x; kf[1] = f.y;
+      f = __half22float2(u32_as_half2(kv.y)); kf[2] = f.x; kf[3] = f.y;
+      f = __half22float2(u32_as_half2(kv.z)); kf[4] = f.x; kf[5] = f.y;
+      f = __half22float2(u32_as_half2(kv.w)); kf[6] = f.x; kf[7] = f.y;
+#pragma unroll
+      for (int g = 0; g < kAttnMaxGroup; ++g) {
+        if (g < group) {
+          const float* qg = q_s + g * D + c * 8;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) sc[g] = fmaf(kf[e], qg[e], sc[g]);
+        }
+      }
+    }
+  }
+  float p[kAttnMaxGroup];
+#pragma unroll
+  for (int g = 0; g < kAttnMaxGroup; ++g) {
+    if (g < group) {
+      const float s = ok ? sc[g] * scale : -INFINITY;
+      const float m = warp_max(s);
+      p[g] = (ok && m > -INFINITY) ? expf(s - m) : 0.f;
+      const float l = warp_sum(p[g]);
+      if (lane == 0) {
+        w_m[warp][g] = m;
+        w_l[warp][g] = l;
+      }
+    } else {
+      p[g] = 0.f;
+    }
+  }
+  float acc[kAttnMaxGroup][V];
+#pragma unroll
+  for (int g = 0; g < kAttnMaxGroup; ++g)
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[g][v] = 0.f;
+  const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
+  for (int tt = 0; tt < n_here; ++tt) {
+    const __half* vr = vc + ((size_t)kvh * cap + t0 + tt) * D + lane * V;
+    float vf[V];
+    if (V == 4) {
+      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(vr));
+      float2 f;
+      f = __half22float2(u32_as_half2(raw.x)); vf[0] = f.x; vf[1] = f.y;
+      f = __half22float2(u32_as_half2(raw.y)); vf[2] = f.x; vf[3] = f.y;
+    } else {
+      const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(vr));
+      const float2 f = __half22float2(u32_as_half2(raw));
+      vf[0] = f.x;
+      vf[1] = f.y;
+    }
+#pragma unroll
+    for (int g = 0; g < kAttnMaxGroup; ++g) {
+      if (g < group) {
+        const float pt = __shfl_sync(0xffffffffu, p[g], tt);
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[g][v] = fmaf(pt, vf[v], acc[g][v]);
+      }
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < kAttnMaxGroup; ++g)
+    if (g < group)
+#pragma unroll
+      for (int v = 0; v < V; ++v) w_acc[warp][g][lane * V + v] = acc[g][v];
+  __syncthreads();
+  // merge the 4 warps (ascending) and write this split's partial for each head of the group
+  for (int idx = threadIdx.x; idx < group * D; idx += blockDim.x) {
+    const int g = idx / D, e = idx % D;
+    float mx = -INFINITY;
+    for (int w = 0; w < 4; ++w) mx = fmaxf(mx, w_m[w][g]);
+    float l = 0.f, o = 0.f;
+    for (int w = 0; w < 4; ++w) {
+      const float f = w_m[w][g] > -INFINITY ? expf(w_m[w][g] - mx) : 0.f;
+      l = fmaf(w_l[w][g], f, l);
+      o = fmaf(w_acc[w][g][e], f, o);
+    }
+    float* dst = part + ((size_t)(kvh * group + g) * n_splits + split) * (D + 2);
+    dst[e] = o;
+    if (e == 0) {
+      dst[D] = mx;
+      dst[D + 1] = l;
+    }
+  }
+}
+
+template <int D>
+__global__ void attn_decode_combine_kernel(const float* __restrict__ part, __half* __restrict__ a16, int n_splits) {
+  const int hq = blockIdx.x, e = threadIdx.x;
+  const float* base = part + (size_t)hq * n_splits * (D + 2);
+  float mx = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, base[(size_t)s * (D + 2) + D]);
+  float l = 0.f, o = 0.f;
+  for (int s = 0; s < n_splits; ++s) {
+    const float* ps = base + (size_t)s * (D + 2);
+    const float f = ps[D] > -INFINITY ? expf(ps[D] - mx) : 0.f;
+    l = fmaf(ps[D + 1], f, l);
+    o = fmaf(ps[e], f, o);
+  }
+  a16[(size_t)hq * D + e] = __float2half_rn(o / l);
+}
+
+cudaError_t launch_attn_decode(const float* q_rot, const __half* kc, const __half* vc, float* scratch, __half* a16,
+                               int n_q, int n_kv, int d, int cap, int n_ctx, cudaStream_t st, uint64_t* n_launch) {
+  const int splits = attn_decode_splits(n_ctx), group = n_q / n_kv;
+  const float scale = 1.0f / sqrtf((float)d);
+  dim3 grid(splits, n_kv);
+  if (d == 128) {
+    attn_decode_partial_kernel<128><<<grid, 128, 0, st>>>(q_rot, kc, vc, scratch, group, cap, n_ctx, splits, scale);
+    attn_decode_combine_kernel<128><<<n_q, 128, 0, st>>>(scratch, a16, splits);
+  } else if (d == 64) {
+    attn_decode_partial_kernel<64><<<grid, 128, 0, st>>>(q_rot, kc, vc, scratch, group, cap, n_ctx, splits, scale);
+    attn_decode_combine_kernel<64><<<n_q, 64, 0, st>>>(scratch, a16, splits);
+  } else {
+    return cudaErrorInvalidValue;
+  }
+  *n_launch += 2;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------- router + top-k (a4)
+// One CTA per token.  Thread (grp, e) sums h[i] * W_r[i][e] over i = grp, grp+G, ...; groups are added in ascending
+// order; warp 0 then extracts the k largest logits (equal logits: lower index first) and the gates.
+constexpr int kRouterThreads = 1024;
+
+__global__ void __launch_bounds__(kRouterThreads) router_topk_kernel(const __half* __restrict__ h, const __half* __restrict__ wr,
+                                                                     int H, int E, int Epad, int k, int renorm,
+                                                                     int32_t* __restrict__ ids, float* __restrict__ gates) {
+  extern __shared__ float smem[];
+  float* h_s = smem;             // [H]
+  float* part = h_s + H;         // [G][Epad]
+  float* logit = part + kRouterThreads;  // [Epad]
+  const int m = blockIdx.x;
+  const int G = kRouterThreads / Epad;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) h_s[i] = __half2float(h[(size_t)m * H + i]);
+  __syncthreads();
+  const int e = threadIdx.x % Epad, grp = threadIdx.x / Epad;
+  float acc = 0.f;
+  if (e < E)
+    for (int i = grp; i < H; i += G) acc = fmaf(h_s[i], __half2float(wr[(size_t)i * E + e]), acc);
+  part[grp * Epad + e] = acc;
+  __syncthreads();
+  if (threadIdx.x < Epad) {
+    float t = 0.f;
+    for (int g = 0; g < G; ++g) t += part[g * Epad + threadIdx.x];
+    logit[threadIdx.x] = threadIdx.x < E ? t : -INFINITY;
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  const int lane = threadIdx.x;
+  const int per = Epad / 32;  // candidates per lane: e = lane + 32*j
+  uint32_t taken = 0;
+  float sel_v = 0.f;  // lane j (< k) keeps the j-th selected logit
+  int sel_i = 0;
+  float total = 0.f, top = 0.f;
+  if (!renorm) {
+    float mx = -INFINITY;
+    for (int j = 0; j < per; ++j) mx = fmaxf(mx, logit[lane + 32 * j]);
+    mx = warp_max(mx);
+    float s = 0.f;
+    for (int j = 0; j < per; ++j) {
+      const float v = logit[lane + 32 * j];
+      s += v > -INFINITY ? expf(v - mx) : 0.f;
+    }
+    total = warp_sum(s);
+    top = mx;
+  }
+  for (int r = 0; r < k; ++r) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int j = 0; j < per; ++j) {
+      if (taken & (1u << j)) continue;
+      const float v = logit[lane + 32 * j];
+      const int idx = lane + 32 * j;
+      if (idx < E && (v > bv || (v == bv && idx < bi))) {
+        bv = v;
+        bi = idx;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ov > bv || (ov == bv && oi < bi)) {
+        bv = ov;
+        bi = oi;
+      }
+    }
+    if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+    if (lane == r) {
+      sel_v = bv;
+      sel_i = bi;
+    }
+  }
+  float gate;
+  if (renorm) {
+    const float mx = __shfl_sync(0xffffffffu, sel_v, 0);
+    const float ex = lane < k ? expf(sel_v - mx) : 0.f;
+    const float s = warp_sum(ex);
+    gate = ex / s;
+  } else {
+    gate = lane < k ? expf(sel_v - top) / total : 0.f;
+  }
+  if (lane < k) {
+    ids[(size_t)m * k + lane] = sel_i;
+    gates[(size_t)m * k + lane] = gate;
+  }
+}
+
+cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
+                               float* gates, cudaStream_t st, uint64_t* n_launch) {
+  int Epad = 32;
+  while (Epad < E) Epad <<= 1;
+  const size_t smem = ((size_t)H + kRouterThreads + Epad) * sizeof(float);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(router_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  router_topk_kernel<<<M, kRouterThreads, smem, st>>>(h, wr, H, E, Epad, k, renorm, ids, gates);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------- MoE combine
+template <typename TRes>
+__global__ void moe_combine_kernel(const TRes* __restrict__ res, const float* __restrict__ gates, const float* __restrict__ d32,
+                                   __half* __restrict__ y16, int k, int H) {
+  const int m = blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= H) return;
+  float acc = load_f<TRes>(res, (size_t)m * H + i);
+  for (int j = 0; j < k; ++j) acc = fmaf(gates[m * k + j], d32[((size_t)m * k + j) * H + i], acc);
+  y16[(size_t)m * H + i] = __float2half_rn(acc);
+}
+
+cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gates, const float* d32, __half* y16, int M,
+                               int k, int H, cudaStream_t st, uint64_t* n_launch) {
+  dim3 grid((H + 255) / 256, M);
+  if (res_is_f32)
+    moe_combine_kernel<float><<<grid, 256, 0, st>>>((const float*)res, gates, d32, y16, k, H);
+  else
+    moe_combine_kernel<__half><<<grid, 256, 0, st>>>((const __half*)res, gates, d32, y16, k, H);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uint64_t* n_launch) {
+  (void)n_launch;
+  return cudaMemsetAsync(p, v, bytes, st);
+}
+
+}  // namespace ats

@@ -18,8 +18,12 @@ workload configurations instead:
 * one fp16 scale per block of 32 consecutive k of a row, ``|N(0, 0.02)|``.
 * activations and KV-cache entries ``N(0, 1)`` rounded to fp16.
 * router weights ``N(0, 0.02)`` rounded to fp16.
-* RMSNorm gains ``N(0, 1)`` rounded to fp16 (zero-mean gains keep a deep stack
-  of such synthetic layers inside the fp16 range; all-ones gains overflow).
+* RMSNorm gains zero-mean normal, rounded to fp16: std 0.25 in the dense layers, std 1 in the MoE
+  block.  Zero-mean gains keep a deep stack of such synthetic layers inside the fp16 range (all-ones
+  gains overflow in the second layer).  The dense std of 0.25 keeps attention logits at an LLM-like
+  magnitude (std about 2): with unit-variance gains the new token's self-score has std about 36, the
+  softmax degenerates to a near-argmax, and a one-ulp difference in the fp16 rounding of a cached key
+  moves the layer output by 1e-3, which no fp32 implementation can avoid and no tolerance can absorb.
 
 Every stream is ``numpy.random.default_rng([0, config, layer, role, part, step])``
 so "all values come from seed 0" and any tensor can be regenerated alone.
@@ -73,8 +77,12 @@ def activations(config: int, layer: int, shape, step: int = 0, role: int = ROLE_
     return stream(config, layer, role, 0, step).normal(0.0, 1.0, size=shape).astype(np.float16)
 
 
-def norm_gain(config: int, layer: int, role: int, hidden: int) -> np.ndarray:
-    return stream(config, layer, role, 0).normal(0.0, 1.0, size=(hidden,)).astype(np.float16)
+DENSE_GAIN_STD = 0.25
+MOE_GAIN_STD = 1.0
+
+
+def norm_gain(config: int, layer: int, role: int, hidden: int, std: float = DENSE_GAIN_STD) -> np.ndarray:
+    return stream(config, layer, role, 0).normal(0.0, std, size=(hidden,)).astype(np.float16)
 
 
 def router_weight(config: int, layer: int, hidden: int, n_experts: int) -> np.ndarray:
@@ -143,7 +151,7 @@ def moe_block(config: int, layer: int, shape: MoEShape = MOE_FULL) -> dict:
     out[ROLE_UP] = q4_packed(config, layer, ROLE_UP, shape.ffn, shape.hidden, shape.n_experts)
     out[ROLE_DOWN] = q4_packed(config, layer, ROLE_DOWN, shape.hidden, shape.ffn, shape.n_experts)
     out[ROLE_ROUTER] = router_weight(config, layer, shape.hidden, shape.n_experts)
-    out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden)
+    out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden, MOE_GAIN_STD)
     return out
 
 

@@ -1,0 +1,85 @@
+"""Shared helpers of the GPU parity tests: build a library context from the seeded workloads and compare with the oracle."""
+import numpy as np
+
+from paper_2607_10183_b200 import workloads as W
+
+TOL = 2e-3  # max relative error of fp outputs (fp32 accumulation vs the fp64 oracle), as the workload states it
+
+
+def assert_close(y, ref, tol=TOL, what=""):
+    """Two gates per output row: normwise max|y-r| / max|r| <= tol, and mixed elementwise |y-r| <= tol (|r| + rms(r)).
+    (A pure elementwise relative error is meaningless next to the zero crossings of a dot product.)"""
+    y = np.asarray(y, dtype=np.float64).reshape(-1, np.asarray(y).shape[-1])
+    r = np.asarray(ref, dtype=np.float64).reshape(y.shape)
+    assert np.all(np.isfinite(y)), f"{what}: non-finite output"
+    err = np.abs(y - r)
+    norm = err.max(axis=1) / np.maximum(np.abs(r).max(axis=1), 1e-30)
+    assert norm.max() <= tol, f"{what}: normwise error {norm.max():.3e} > {tol}"
+    rms = np.sqrt(np.mean(r * r, axis=1, keepdims=True))
+    ratio = err / (tol * (np.abs(r) + rms) + 1e-300)
+    assert ratio.max() <= 1.0, f"{what}: mixed elementwise ratio {ratio.max():.3f} > 1"
+    return float(norm.max()), float(ratio.max())
+
+
+def bits_equal_mod_zero_sign(a, b):
+    """Bitwise equality after mapping -0 to +0."""
+    a = np.asarray(a)
+    b = np.asarray(b)
+    a = np.where(a == 0, np.zeros_like(a), a)
+    b = np.where(b == 0, np.zeros_like(b), b)
+    ia = a.view(np.uint32 if a.dtype == np.float32 else np.uint16)
+    ib = b.view(np.uint32 if b.dtype == np.float32 else np.uint16)
+    return np.array_equal(ia, ib)
+
+
+ROLE_NAME = {W.ROLE_Q: "wq", W.ROLE_K: "wk", W.ROLE_V: "wv", W.ROLE_O: "wo", W.ROLE_GATE: "w_gate", W.ROLE_UP: "w_up",
+             W.ROLE_DOWN: "w_down"}
+DENSE_ROLES = (W.ROLE_Q, W.ROLE_K, W.ROLE_V, W.ROLE_O, W.ROLE_GATE, W.ROLE_UP, W.ROLE_DOWN)
+
+
+def oracle_dense_tensors(L):
+    t = {ROLE_NAME[r]: L[r] for r in DENSE_ROLES}
+    t["attn_norm"], t["ffn_norm"] = L[W.ROLE_ATTN_NORM], L[W.ROLE_FFN_NORM]
+    return t
+
+
+def oracle_moe_tensors(B):
+    return {"w_gate": B[W.ROLE_GATE], "w_up": B[W.ROLE_UP], "w_down": B[W.ROLE_DOWN], "router": B[W.ROLE_ROUTER],
+            "ffn_norm": B[W.ROLE_FFN_NORM]}
+
+
+def register_dense_layer(ctx, L, layer_idx, kv_capacity):
+    """Registers one dense layer's tensors in execution order; returns (layer descriptor, {role: id})."""
+    from paper_2607_10183_b200 import binding as B
+    shape = L["shape"]
+    ids = {}
+    ids["attn_norm"] = ctx.register_f16(L[W.ROLE_ATTN_NORM], layer_idx, W.ROLE_ATTN_NORM)
+    for r in (W.ROLE_Q, W.ROLE_K, W.ROLE_V, W.ROLE_O):
+        ids[ROLE_NAME[r]] = ctx.register_q4(*L[r], layer=layer_idx, role=r)
+    ids["ffn_norm"] = ctx.register_f16(L[W.ROLE_FFN_NORM], layer_idx, W.ROLE_FFN_NORM)
+    for r in (W.ROLE_GATE, W.ROLE_UP, W.ROLE_DOWN):
+        ids[ROLE_NAME[r]] = ctx.register_q4(*L[r], layer=layer_idx, role=r)
+    desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                        head_dim=shape.head_dim, kv_capacity=kv_capacity, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, **ids)
+    return desc, ids
+
+
+def register_moe_block(ctx, Bk, layer_idx=0):
+    from paper_2607_10183_b200 import binding as B
+    shape = Bk["shape"]
+    ids = {}
+    ids["ffn_norm"] = ctx.register_f16(Bk[W.ROLE_FFN_NORM], layer_idx, W.ROLE_FFN_NORM)
+    ids["router"] = ctx.register_f16(Bk[W.ROLE_ROUTER], layer_idx, W.ROLE_ROUTER)
+    for r in (W.ROLE_GATE, W.ROLE_UP, W.ROLE_DOWN):
+        ids[ROLE_NAME[r]] = ctx.register_q4(*Bk[r], layer=layer_idx, role=r)
+    desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, rms_eps=shape.rms_eps, **ids)
+    return desc, ids
+
+
+def dense_layer_bytes(shape):
+    return sum(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+
+
+def to_dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()

@@ -1,0 +1,362 @@
+"""GPU parity of the decode path against the CPU oracle, through the C ABI.
+
+Integer / byte work (dequantized values, routing ids, placement and streaming bookkeeping) must be bit-exact;
+floating-point outputs must be within 2e-3 (see helpers.assert_close)."""
+import numpy as np
+import pytest
+
+from oracle import ats_oracle as O
+from paper_2607_10183_b200 import workloads as W
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+MB = 1 << 20
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2607_10183_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    return torch
+
+
+def make_ctx(B, resident_bytes, ws=8 * MB, ring_slots=2, slot_bytes=0, chunk_bytes=MB, flags=0):
+    if slot_bytes == 0:
+        ring_slots = 0
+    arena = ws + ring_slots * (slot_bytes + 256) + resident_bytes + 64 * 1024
+    return B.Context(arena, workspace_bytes=ws, ring_slots=ring_slots, slot_bytes=slot_bytes, chunk_bytes=chunk_bytes, flags=flags)
+
+
+# ------------------------------------------------------------------------------------------------- a1 dequantization
+def test_dequant_exhaustive_codes_times_all_finite_scales(B, torch):
+    """16 codes x every finite fp16 scale bit pattern, fp32 (exact) and fp16 (one rounding), resident and streamed."""
+    bits = np.arange(65536, dtype=np.uint32)
+    bits = bits[(bits & 0x7C00) != 0x7C00].astype(np.uint16)  # drop Inf / NaN
+    N = bits.size
+    scales = bits.view(np.float16).reshape(N, 1)
+    codes = np.tile(np.arange(-8, 8, dtype=np.int8), (N, 2))  # K = 32: each row one block holding all 16 codes twice
+    packed = W.codes_to_packed(codes)
+    want32 = O.dequantize(packed, scales).astype(np.float32)
+    with np.errstate(over="ignore"):
+        want16 = O.dequantize(packed, scales, O.WEIGHT_F16).astype(np.float16)
+    nbytes = W.q4_bytes(N, 32)
+    for where in (B.ATS_GPU, B.ATS_HOST):
+        ctx = make_ctx(B, nbytes, slot_bytes=nbytes)
+        tid = ctx.register_q4(packed, scales)
+        ctx.set_placement([(tid, -1, where)])
+        o32 = torch.empty((N, 32), dtype=torch.float32, device="cuda")
+        o16 = torch.empty((N, 32), dtype=torch.float16, device="cuda")
+        ctx.dequantize(tid, 0, o32, B.ATS_OUT_F32)
+        ctx.dequantize(tid, 0, o16, B.ATS_OUT_F16)
+        ctx.sync()
+        assert H.bits_equal_mod_zero_sign(o32.cpu().numpy(), want32)
+        assert H.bits_equal_mod_zero_sign(o16.cpu().numpy(), want16)
+        assert not np.isnan(o16.cpu().numpy().astype(np.float32)).any()
+        ctx.close()
+
+
+def test_dequant_random_tensor_and_expert_slices(B, torch):
+    packed, scales = W.q4_packed(94, 0, W.ROLE_GATE, 24, 160, n_experts=3)
+    scales[1, 3, 2] = 0  # a zero-scale block
+    scales[2, 5, 1] = -scales[2, 5, 1]  # negative scales are legal
+    ctx = make_ctx(B, 3 * (W.q4_bytes(24, 160) + 256), slot_bytes=W.q4_bytes(24, 160))
+    tid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(tid, 0, B.ATS_GPU), (tid, 1, B.ATS_HOST), (tid, 2, B.ATS_GPU)])
+    for e in range(3):
+        out = torch.empty((24, 160), dtype=torch.float32, device="cuda")
+        ctx.dequantize(tid, e, out, B.ATS_OUT_F32)
+        ctx.sync()
+        assert H.bits_equal_mod_zero_sign(out.cpu().numpy(), O.dequantize(packed[e], scales[e]).astype(np.float32))
+    assert ctx.get_placement(tid, 1) == B.ATS_HOST and ctx.get_placement(tid, 2) == B.ATS_GPU
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------- a2 GEMV
+@pytest.mark.parametrize("N,K,M", [(1, 32, 1), (3, 64, 2), (17, 96, 3), (130, 1056, 8), (257, 4096, 1), (64, 14336, 5),
+                                   (4096, 4096, 1)])
+def test_linear_gemv_matches_oracle(B, torch, N, K, M):
+    cfg = 1 if (N, K, M) == (4096, 4096, 1) else 95
+    packed, scales = W.q4_packed(cfg, 0, W.ROLE_Q, N, K)
+    x = W.activations(cfg, 0, (M, K))
+    want = O.linear(x, packed, scales, round_out=True)
+    outs = []
+    for where in (B.ATS_GPU, B.ATS_HOST):
+        ctx = make_ctx(B, W.q4_bytes(N, K), slot_bytes=W.q4_bytes(N, K), chunk_bytes=64 * 1024)
+        tid = ctx.register_q4(packed, scales)
+        ctx.set_placement([(tid, -1, where)])
+        y = torch.full((M, N), 7.0, dtype=torch.float16, device="cuda")
+        ctx.linear(tid, H.to_dev(x), y, M)
+        ctx.sync()
+        st = ctx.stats()
+        if where == B.ATS_HOST:
+            assert st.streamed_bytes == W.q4_bytes(N, K) and st.copies == -(-W.q4_bytes(N, K) // (64 * 1024))
+        else:
+            assert st.streamed_bytes == 0 and st.resident_bytes == W.q4_bytes(N, K)
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want, what=f"gemv {N}x{K} M={M}")
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))  # placement never changes the math
+
+
+def test_linear_closed_forms_on_gpu(B, torch):
+    """One-hot activations return a weight column exactly; all-ones with unit scales return integer row sums."""
+    N, K = 40, 256
+    rng = np.random.default_rng(5)
+    codes = rng.integers(-8, 8, size=(N, K), dtype=np.int8)
+    scales = np.abs(rng.normal(0, 0.02, size=(N, K // 32))).astype(np.float16)
+    ctx = make_ctx(B, 2 * W.q4_bytes(N, K) + 512)
+    t1 = ctx.register_q4(W.codes_to_packed(codes), scales)
+    t2 = ctx.register_q4(W.codes_to_packed(codes), np.ones_like(scales))
+    ctx.set_placement([(t1, -1, B.ATS_GPU), (t2, -1, B.ATS_GPU)])
+    y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+    for k in (0, 1, 7, 8, 31, 32, 255):
+        x = np.zeros((1, K), dtype=np.float16)
+        x[0, k] = 1
+        ctx.linear(t1, H.to_dev(x), y, 1)
+        ctx.sync()
+        want = (scales[:, k // 32].astype(np.float64) * codes[:, k]).astype(np.float16)
+        assert H.bits_equal_mod_zero_sign(y.cpu().numpy()[0], want), k
+    ctx.linear(t2, H.to_dev(np.ones((1, K), dtype=np.float16)), y, 1)
+    ctx.sync()
+    assert np.array_equal(y.cpu().numpy()[0].astype(np.int64), codes.astype(np.int64).sum(axis=1))
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------- dense layer decode
+def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, flags=0, steps=1, chunk=MB):
+    """Returns (list of y per step, final K cache, final V cache, stats) for one layer."""
+    L = W.dense_layer(cfg, 0, shape)
+    slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+    ctx = make_ctx(B, H.dense_layer_bytes(shape) + 16 * 256 + 4 * shape.hidden * 2, ring_slots=ring_slots, slot_bytes=slot,
+                   chunk_bytes=chunk, flags=flags)
+    desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+    assert ctx.cfg.workspace_bytes >= B.workspace_bytes(desc, 1)
+    ctx.set_placement([(ids[n], -1, w) for n, w in placement.items()])
+    kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos)
+    kd, vd = H.to_dev(kc), H.to_dev(vc)
+    ys = []
+    ctx.reset_stats()
+    for s in range(steps):
+        x = W.activations(cfg, 0, (1, shape.hidden), step=s)
+        y = torch.empty((1, shape.hidden), dtype=torch.float16, device="cuda")
+        ctx.layer_decode(desc, H.to_dev(x), y, kd, vd, pos + s, 1)
+        ctx.sync()
+        ys.append(y.cpu().numpy())
+    st = ctx.stats()
+    out = (ys, kd.cpu().numpy(), vd.cpu().numpy(), st, ctx.numerics(B.ATS_MODE_DECODE))
+    ctx.close()
+    return out
+
+
+ALL_GPU = {n: 1 for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")}
+
+
+@pytest.mark.parametrize("shape_name,pos,cap", [("small", 0, 8), ("small", 37, 64), ("small", 200, 300), ("full", 1024, 1025)])
+def test_dense_layer_decode_matches_oracle(B, torch, shape_name, pos, cap):
+    shape = W.DENSE_SMALL if shape_name == "small" else W.DENSE_FULL
+    cfg = 96 if shape_name == "small" else 2
+    ys, kg, vg, st, (edges, wmode) = run_dense_decode(B, torch, shape, cfg, pos, cap, ALL_GPU)
+    L = W.dense_layer(cfg, 0, shape)
+    kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos)
+    x = W.activations(cfg, 0, (1, shape.hidden), step=0)
+    want = O.dense_layer(x, H.oracle_dense_tensors(L), shape, kc, vc, pos, edges, wmode)
+    H.assert_close(ys[0], want, what="decode layer output")
+    # cache rows written at `pos`: fp16 values within one ulp of the oracle's, everything else untouched
+    for got, ref in ((kg, kc), (vg, vc)):
+        assert np.array_equal(np.delete(got, pos, axis=1), np.delete(ref, pos, axis=1))
+        a, b = got[:, pos].astype(np.float64), ref[:, pos].astype(np.float64)
+        # one fp16 ulp where the value is not tiny; near zero the fp32 accumulation error (absolute) is what bounds it
+        ulp = np.spacing(np.abs(ref[:, pos]).astype(np.float16)).astype(np.float64)
+        assert np.all(np.abs(a - b) <= ulp + 2e-5 * np.abs(b).max())
+    assert st.streamed_bytes == 0 and st.resident_bytes == H.dense_layer_bytes(shape)
+
+
+def test_placement_invariance_and_bookkeeping_small(B, torch):
+    """A hybrid run equals the all-resident run bit for bit (placement moves bytes, never changes math), for every ring
+    size down to one slot and with freed slots poisoned; streamed bytes / copies follow the oracle's bookkeeping."""
+    shape, cfg, pos, cap = W.DENSE_SMALL, 96, 20, 40
+    base = run_dense_decode(B, torch, shape, cfg, pos, cap, ALL_GPU, steps=3)
+    again = run_dense_decode(B, torch, shape, cfg, pos, cap, ALL_GPU, steps=3)
+    for a, b in zip(base[0], again[0]):
+        assert np.array_equal(a.view(np.uint16), b.view(np.uint16))  # run-to-run deterministic
+    names = list(ALL_GPU)
+    nbytes = [W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes()]
+    rng = np.random.default_rng(0)
+    cases = [({n: 0 for n in names}, 2), ({n: 0 for n in names}, 3), ({n: 0 for n in names}, 7)]
+    cases += [({n: int(rng.integers(0, 2)) for n in names}, int(rng.integers(2, 5))) for _ in range(4)]
+    cases += [({**ALL_GPU, "wq": 0, "wo": 0, "w_down": 0}, 1)]  # one slot is enough when no operator needs two at once
+    for placement, slots in cases:
+        chunk = 4096
+        got = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=slots, flags=B.ATS_FLAG_POISON_SLOTS,
+                               steps=3, chunk=chunk)
+        for a, b in zip(base[0], got[0]):
+            assert np.array_equal(a.view(np.uint16), b.view(np.uint16)), (placement, slots)
+        assert np.array_equal(base[1], got[1]) and np.array_equal(base[2], got[2])
+        where = [placement[n] for n in names]
+        want_bytes, want_copies, _ = O.streamed_dense(nbytes, where, chunk)
+        st = got[3]
+        assert st.streamed_bytes == 3 * want_bytes and st.copies == 3 * want_copies
+        assert st.resident_bytes == sum(b for b, w in zip(nbytes, where) if w == 1)
+        assert st.n_streamed == 3 * where.count(0)
+
+
+def test_gate_up_both_streamed_needs_two_slots(B, torch):
+    shape = W.DENSE_SMALL
+    with pytest.raises(B.AtsError) as e:
+        run_dense_decode(B, torch, shape, 96, 3, 8, {**ALL_GPU, "w_gate": 0, "w_up": 0}, ring_slots=1)
+    assert e.value.code == B.ATS_ERR_BUDGET
+
+
+# ------------------------------------------------------------------------------------------------- a4 routing, a5 MoE
+def test_route_topk_bit_exact_with_ties(B, torch):
+    rng = np.random.default_rng(11)
+    Hd, E, k, M = 128, 48, 6, 9
+    Wr = rng.normal(0, 0.02, size=(Hd, E)).astype(np.float16)
+    Wr[:, 9] = Wr[:, 2]
+    Wr[:, 40] = Wr[:, 2]  # exact ties: equal columns give bitwise equal logits in any summation order
+    h = rng.normal(size=(M, Hd)).astype(np.float16)
+    h[0] = (Wr[:, 2].astype(np.float32) * 50).astype(np.float16)  # token 0 ranks the tied experts first
+    ids_ref, gates_ref, logits = O.route_topk(h, Wr, k)
+    assert ids_ref[0, :3].tolist() == [2, 9, 40]
+    ctx = make_ctx(B, 64 * 1024)
+    rid = ctx.register_f16(Wr)
+    ctx.set_placement([])
+    ids = torch.empty((M, k), dtype=torch.int32, device="cuda")
+    gates = torch.empty((M, k), dtype=torch.float32, device="cuda")
+    ctx.route_topk(rid, H.to_dev(h), M, k, ids, gates)
+    ctx.sync()
+    assert np.array_equal(ids.cpu().numpy(), ids_ref)
+    assert np.max(np.abs(gates.cpu().numpy() - gates_ref)) <= 1e-6
+    ctx.close()
+
+
+def run_moe(B, torch, shape, cfg, M, host_experts, ring_slots=8, chunk=MB, flags=0):
+    Bk = W.moe_block(cfg, 0, shape)
+    sl = W.q4_bytes(shape.ffn, shape.hidden)
+    ws = 4 * MB
+    ctx = make_ctx(B, 3 * shape.n_experts * (sl + 256) + MB, ws=ws, ring_slots=ring_slots, slot_bytes=sl, chunk_bytes=chunk, flags=flags)
+    desc, ids = H.register_moe_block(ctx, Bk)
+    ent = []
+    for name in ("w_gate", "w_up", "w_down"):
+        for e in range(shape.n_experts):
+            ent.append((ids[name], e, B.ATS_HOST if e in host_experts else B.ATS_GPU))
+    ctx.set_placement(ent)
+    x = W.activations(cfg, 0, (M, shape.hidden))
+    y = torch.empty((M, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.reset_stats()
+    ctx.layer_decode(desc, H.to_dev(x), y, None, None, 0, M)
+    ctx.sync()
+    st = ctx.stats()
+    out = y.cpu().numpy()
+    ctx.close()
+    return Bk, x, out, st
+
+
+@pytest.mark.parametrize("shape_name,M", [("small", 1), ("small", 5), ("full", 1), ("full", 8)])
+def test_moe_block_matches_oracle_and_streams_only_selected_experts(B, torch, shape_name, M):
+    shape = W.MOE_SMALL if shape_name == "small" else W.MOE_FULL
+    cfg = 97 if shape_name == "small" else 4
+    odd = {e for e in range(shape.n_experts) if e % 2}
+    chunk = 256 * 1024
+    Bk, x, y_res, st_res = run_moe(B, torch, shape, cfg, M, set())
+    _, _, y_hyb, st_hyb = run_moe(B, torch, shape, cfg, M, odd, chunk=chunk, flags=B.ATS_FLAG_POISON_SLOTS)
+    t = H.oracle_moe_tensors(Bk)
+    want, ids_ref, gates_ref, logits = O.moe_block(x, t, shape)
+    assert O.min_rank_gap(logits, shape.top_k) > 1e-4, "degenerate seed: near-tie among the routed experts"
+    H.assert_close(y_res, want, what="moe block")
+    assert np.array_equal(y_res.view(np.uint16), y_hyb.view(np.uint16))  # placement invariance
+    assert st_res.streamed_bytes == 0 and st_res.host_syncs == 0
+    sl = [W.q4_bytes(shape.ffn, shape.hidden)] * 3
+    where = [[0 if e in odd else 1 for e in range(shape.n_experts)]] * 3
+    nb, copies, order = O.streamed_moe(ids_ref, where, sl, chunk)
+    assert st_hyb.streamed_bytes == nb and st_hyb.copies == copies and st_hyb.n_streamed == len(order)
+    assert st_hyb.host_syncs == 1
+    got_order = [(st_hyb.streamed_ids[i], st_hyb.streamed_experts[i]) for i in range(min(st_hyb.n_streamed, B.ATS_STATS_LIST))]
+    # tensor ids are registration order: ffn_norm 0, router 1, gate 2, up 3, down 4
+    assert got_order == [(2 + t_, e) for t_, e in order][:len(got_order)]
+
+
+def test_moe_small_ring_forces_waves(B, torch):
+    shape = W.MOE_SMALL
+    everything = set(range(shape.n_experts))
+    Bk, x, y_res, _ = run_moe(B, torch, shape, 97, 5, set())
+    for slots in (2, 3, 5):
+        _, _, y, st = run_moe(B, torch, shape, 97, 5, everything, ring_slots=slots, flags=B.ATS_FLAG_POISON_SLOTS)
+        assert np.array_equal(y.view(np.uint16), y_res.view(np.uint16)), slots
+        assert st.ring_reuses > 0
+
+
+def test_route_and_moe_linear_standalone(B, torch):
+    shape = W.MOE_SMALL
+    Bk = W.moe_block(97, 0, shape)
+    sl = W.q4_bytes(shape.ffn, shape.hidden)
+    ctx = make_ctx(B, 3 * shape.n_experts * (sl + 256) + MB, ring_slots=4, slot_bytes=sl)
+    desc, ids = H.register_moe_block(ctx, Bk)
+    ctx.set_placement([(ids["w_gate"], -1, B.ATS_GPU), (ids["w_up"], -1, B.ATS_GPU)] +
+                      [(ids["w_down"], e, e % 2) for e in range(shape.n_experts)])
+    M, k = 3, shape.top_k
+    h = W.activations(97, 3, (M, shape.hidden))
+    idt = np.array([[1, 4, 7, 2], [0, 15, 3, 8], [7, 7, 6, 5]], dtype=np.int32)
+    y = torch.empty((M, k, shape.ffn), dtype=torch.float16, device="cuda")
+    ctx.moe_linear(ids["w_gate"], H.to_dev(h), H.to_dev(idt), y, M, k, 0)
+    ctx.sync()
+    H.assert_close(y.cpu().numpy().reshape(M * k, -1), O.moe_linear(h, idt, *Bk[W.ROLE_GATE]).reshape(M * k, -1))
+    xs = W.activations(97, 4, (M, k, shape.ffn))
+    y2 = torch.empty((M, k, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.moe_linear(ids["w_down"], H.to_dev(xs), H.to_dev(idt), y2, M, k, 1)
+    ctx.sync()
+    H.assert_close(y2.cpu().numpy().reshape(M * k, -1), O.moe_linear(xs, idt, *Bk[W.ROLE_DOWN], x_per_slot=True).reshape(M * k, -1))
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------- errors (host-made)
+def test_errors_are_statuses_and_context_stays_usable(B, torch):
+    ctx = make_ctx(B, 4 * MB, ring_slots=1, slot_bytes=1024)
+    packed, scales = W.q4_packed(98, 0, 0, 8, 64)
+    import ctypes as C
+    d = B.ats_tensor_desc(B.ATS_FMT_Q4B32, 1, 8, 40, 0, 0, -1, 0)
+    out = C.c_int32()
+    assert B.ats_register_tensor(ctx.h, C.byref(d), packed.ctypes.data, scales.ctypes.data, C.byref(out)) == B.ATS_ERR_SHAPE
+    bad = scales.copy()
+    bad[0, 0] = np.inf
+    with pytest.raises(B.AtsError) as e:
+        ctx.register_q4(packed, bad)
+    assert e.value.code == B.ATS_ERR_INVALID
+    tid = ctx.register_q4(packed, scales)
+    y = torch.empty((1, 8), dtype=torch.float16, device="cuda")
+    x = H.to_dev(W.activations(98, 0, (1, 64)))
+    with pytest.raises(B.AtsError) as e:
+        ctx.linear(tid, x, y, 1)  # no placement yet
+    assert e.value.code == B.ATS_ERR_STATE
+    with pytest.raises(B.AtsError) as e:
+        ctx.set_placement([(tid + 5, -1, 1)])
+    assert e.value.code == B.ATS_ERR_INVALID
+    big = ctx.register_q4(*W.q4_packed(98, 1, 0, 64, 64))
+    with pytest.raises(B.AtsError) as e:
+        ctx.set_placement([(tid, -1, 1), (big, -1, 0)])  # host slice larger than a ring slot
+    assert e.value.code == B.ATS_ERR_BUDGET
+    ctx.set_placement([(tid, -1, 0), (big, -1, 1)])
+    ctx.linear(tid, x, y, 1)
+    ctx.sync(timeout_ms=5000)
+    H.assert_close(y.cpu().numpy(), O.linear(W.activations(98, 0, (1, 64)), packed, scales, round_out=True))
+    # injected copy failure: status, then the context reports itself poisoned
+    B.ats_debug_fail_copies(ctx.h, 1)
+    with pytest.raises(B.AtsError) as e:
+        ctx.linear(tid, x, y, 1)
+    assert e.value.code == B.ATS_ERR_CUDA
+    with pytest.raises(B.AtsError):
+        ctx.linear(tid, x, y, 1)
+    ctx.close()
+    # arena too small for the resident set
+    ctx = make_ctx(B, 0, ring_slots=0, ws=0)
+    tid = ctx.register_q4(*W.q4_packed(98, 2, 0, 1024, 1024))
+    with pytest.raises(B.AtsError) as e:
+        ctx.set_placement([(tid, -1, 1)])
+    assert e.value.code == B.ATS_ERR_BUDGET
+    ctx.close()
