@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Benchmark of the per-tensor block-quantized forward path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
+
+One *step* is one decode step of one dense decoder layer (hidden 4096, 32/8 heads of 128, SwiGLU 14336, 4-bit block-32
+weights, 1024 cached tokens, batch 1) with every tensor resident in HBM: RMSNorm, fused QKV GEMV, RoPE + KV append,
+attention over 1025 positions, O GEMV + residual, RMSNorm, fused gate/up GEMV + SwiGLU, down GEMV + residual.
+Steps rotate over `--replicas` distinct layers (weights > L2) so every weight byte comes from HBM.
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an independent replica of the same job: the path
+does not shard ("replicas only"), there is no data-path collective, and `value` sums the ranks.
+
+The line also carries `roofline` (the GEMV kernel family against the measured HBM copy bandwidth), `e2e` (the same step
+driven from pinned host buffers, copies inside the timed region), `cpu_baseline` (the fp64 oracle timed on this machine's host
+cores on a bounded sample) and `extra` (single-GEMV GB/s, MoE, prefill and PCIe streaming figures of the other configs).
+`--impl reference` times the oracle instead (the reference arm).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi (SM clock, throttle reasons) every 100 ms in a child process while the benchmark runs."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.lines = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0, t1):
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for _, l in self.lines]
+        sm, smax, reasons = [], [], set()
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- oracle legs
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_layer_decode_step(cfg=2):
+    """Builds the inputs of one dense-layer decode step and returns a closure that runs the oracle on them."""
+    from oracle import ats_oracle as O
+    from paper_2607_10183_b200 import workloads as W
+    shape = W.DENSE_FULL
+    L = W.dense_layer(cfg, 0, shape)
+    names = {W.ROLE_Q: "wq", W.ROLE_K: "wk", W.ROLE_V: "wv", W.ROLE_O: "wo", W.ROLE_GATE: "w_gate", W.ROLE_UP: "w_up", W.ROLE_DOWN: "w_down"}
+    t = {names[r]: L[r] for r in names}
+    t["attn_norm"], t["ffn_norm"] = L[W.ROLE_ATTN_NORM], L[W.ROLE_FFN_NORM]
+    x = W.activations(cfg, 0, (1, shape.hidden))
+    kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, 1025, shape.head_dim, 1024)
+    edges = frozenset({"h", "a", "h2", "act"})
+
+    def step():
+        return O.dense_layer(x, t, shape, kc, vc, 1024, edges, O.WEIGHT_EXACT)
+    return step
+
+
+def time_oracle(budget_s=15.0, max_reps=5):
+    step = oracle_layer_decode_step()
+    t0 = time.time()
+    step()
+    t1 = time.time() - t0
+    reps = int(min(max_reps, max(1, round(budget_s / max(t1, 1e-3)))))
+    t0 = time.time()
+    for _ in range(reps):
+        step()
+    dt = (time.time() - t0) / reps
+    return {"value": 1.0 / dt, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"{reps} decode steps of one dense layer (fp64 numpy oracle, {dt:.2f} s per step)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    step = oracle_layer_decode_step()
+    for _ in range(min(args.warmup, 1)):
+        step()
+    k = max(1, min(args.steps, 3))
+    t0 = time.time()
+    for _ in range(k):
+        step()
+    dt = (time.time() - t0) / k
+    val = 1.0 / dt
+    line = {"impl": "reference", "metric": "decode_tokens_per_s", "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": k, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "dense decoder layer decode step, all tensors resident (config 2); oracle on host cores"},
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+                             "sample": f"{k} decode steps of one dense layer"},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------- our arm
+def build_dense_replicas(B, W, n_layers, cfg, kv_cap, ring_slots=0, slot_bytes=0, chunk_bytes=0, extra_ws=0, flags=0):
+    """A context holding n_layers distinct dense layers of the config-2 shape."""
+    shape = W.DENSE_FULL
+    layer_bytes = sum(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=kv_cap)
+    ws = max(B.workspace_bytes(probe, 1), extra_ws) + (1 << 20)
+    arena = ws + ring_slots * (slot_bytes + 256) + n_layers * (layer_bytes + 16 * 1024 + 4 * shape.hidden) + (1 << 20)
+    ctx = B.Context(arena, workspace_bytes=ws, ring_slots=ring_slots, slot_bytes=slot_bytes, chunk_bytes=chunk_bytes, flags=flags)
+    names = {W.ROLE_Q: "wq", W.ROLE_K: "wk", W.ROLE_V: "wv", W.ROLE_O: "wo", W.ROLE_GATE: "w_gate", W.ROLE_UP: "w_up", W.ROLE_DOWN: "w_down"}
+    descs, q4_ids = [], []
+    for l in range(n_layers):
+        L = W.dense_layer(cfg, l, shape)
+        ids = {"attn_norm": ctx.register_f16(L[W.ROLE_ATTN_NORM], l, W.ROLE_ATTN_NORM)}
+        for r in (W.ROLE_Q, W.ROLE_K, W.ROLE_V, W.ROLE_O):
+            ids[names[r]] = ctx.register_q4(*L[r], layer=l, role=r)
+        ids["ffn_norm"] = ctx.register_f16(L[W.ROLE_FFN_NORM], l, W.ROLE_FFN_NORM)
+        for r in (W.ROLE_GATE, W.ROLE_UP, W.ROLE_DOWN):
+            ids[names[r]] = ctx.register_q4(*L[r], layer=l, role=r)
+        q4_ids += [ids[names[r]] for r in names]
+        descs.append(B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                                  head_dim=shape.head_dim, kv_capacity=kv_cap, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, **ids))
+        del L
+    return ctx, descs, q4_ids, layer_bytes
+
+
+def event_time_ms(torch, stream, fn):
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    fn()
+    b.record(stream)
+    torch.cuda.synchronize()
+    return a.elapsed_time(b)
+
+
+def extra_gemv(torch, B, W, peaks, quick):
+    """Config 1: single 4096x4096 GEMV (9,453,568 algorithmic bytes), rotating over 64 distinct weight replicas (> L2)."""
+    N = K = 4096
+    reps = 64
+    nb = W.q4_bytes(N, K)
+    ctx = B.Context(reps * (nb + 256) + (4 << 20), workspace_bytes=1 << 20)
+    packed, scales = W.q4_packed(1, 0, W.ROLE_Q, N, K)
+    ids = []
+    for r in range(reps):
+        ids.append(ctx.register_q4(np.roll(packed, r, axis=0), scales))
+    ctx.set_placement([(i, -1, B.ATS_GPU) for i in ids])
+    x = torch.from_numpy(W.activations(1, 0, (1, K))).cuda()
+    y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+    n = 64 * (10 if quick else 50)
+
+    def go(k):
+        for i in range(k):
+            ctx.linear(ids[i % reps], x, y, 1)
+    go(128)
+    ms = event_time_ms(torch, ctx.compute, lambda: go(n))
+    ctx.set_flags(B.ATS_FLAG_TIME_KERNELS)
+    ctx.reset_stats()
+    go(640)
+    ctx.sync()
+    st = ctx.stats()
+    ctx.close()
+    alg = nb + K * 2 + N * 2
+    back_to_back = alg * n / (ms * 1e-3) / 1e9
+    kernel = st.timed_work[0] / (st.timed_ms[0] * 1e-3) / 1e9
+    return {"workload": "config 1: GEMV 4096x4096, batch 1, resident, 64 replicas rotated", "algorithmic_bytes": alg,
+            "us_per_call_back_to_back": ms * 1e3 / n, "gbs_back_to_back": back_to_back, "kernel_us": st.timed_ms[0] * 1e3 / st.timed_launches[0],
+            "gbs_kernel": kernel, "frac_of_measured_hbm": kernel / peaks["hbm_gbs"], "frac_of_nominal_8TBs": kernel / 8000.0}
+
+
+EXTRAS = {"cfg1_gemv": extra_gemv}
+
+
+def run_ours(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2607_10183_b200 import binding as B, workloads as W
+    peaks = load_peaks()
+    shape = W.DENSE_FULL
+    R, pos, cap = args.replicas, 1024, 1025
+    sampler = ClockSampler(local)
+
+    ctx, descs, q4_ids, layer_bytes = build_dense_replicas(B, W, R, 2, cap)
+    ctx.set_placement([(i, -1, B.ATS_GPU) for i in q4_ids])
+    caches = []
+    for l in range(R):
+        kc, vc = W.kv_cache(2, l, shape.n_kv_heads, cap, shape.head_dim, pos)
+        caches.append((torch.from_numpy(kc).cuda(local), torch.from_numpy(vc).cuda(local)))
+    x_host = torch.from_numpy(W.activations(2, 0, (1, shape.hidden))).pin_memory()
+    y_host = torch.empty((1, shape.hidden), dtype=torch.float16).pin_memory()
+    x_dev = x_host.cuda(local)
+    y_dev = torch.empty_like(x_dev)
+    cs = ctx.compute
+
+    def steps(n, start=0):
+        for s in range(start, start + n):
+            r = s % R
+            ctx.layer_decode(descs[r], x_dev, y_dev, caches[r][0], caches[r][1], pos, 1)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing (the headline value)
+    steps(args.warmup)
+    barrier()
+    ctx.reset_stats()
+    t_wall0 = time.time()
+    ms = event_time_ms(torch, cs, lambda: steps(args.steps, args.warmup))
+    t_wall1 = time.time()
+    barrier()
+    launches = ctx.stats().kernel_launches
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    clocks = sampler.summary(t_wall0, t_wall1)
+    tok_s = world * args.steps / (ms * 1e-3)
+
+    # ---- profiling pass: the same steps with every GEMV launch bracketed by events -> roofline of the dominant kernel
+    ctx.set_flags(B.ATS_FLAG_TIME_KERNELS)
+    ctx.reset_stats()
+    n_prof = min(args.steps, 2000)
+    steps(n_prof, args.warmup)
+    ctx.sync()
+    st = ctx.stats()
+    ctx.set_flags(0)
+    gemv_ms, gemv_n, gemv_bytes = st.timed_ms[0], st.timed_launches[0], st.timed_work[0]
+    achieved = gemv_bytes / (gemv_ms * 1e-3) / 1e9 if gemv_ms > 0 else None
+    roofline = {"bound": "hbm", "kernel": "gemv_kernel (4 launches per step: fused QKV, O, fused gate/up+SwiGLU, down)",
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"] + " HBM copy bandwidth",
+                "unit": "GB/s", "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
+                "frac_of_nominal_8TBs": (achieved / 8000.0) if achieved else None,
+                "bytes_per_launch": gemv_bytes / max(gemv_n, 1), "avg_launch_us": gemv_ms * 1e3 / max(gemv_n, 1),
+                "launches_timed": int(gemv_n), "traffic": args.traffic}
+
+    # ---- end to end: the same step driven from pinned host buffers (H2D of x and D2H of y inside the timed region)
+    def e2e_steps(n, start=0):
+        with torch.cuda.stream(cs):
+            for s in range(start, start + n):
+                r = s % R
+                x_dev.copy_(x_host, non_blocking=True)
+                ctx.layer_decode(descs[r], x_dev, y_dev, caches[r][0], caches[r][1], pos, 1)
+                y_host.copy_(y_dev, non_blocking=True)
+                cs.synchronize()  # the caller reads the result of every step
+    e2e_steps(min(args.warmup, 50))
+    barrier()
+    n_e2e = min(args.steps, 5000)
+    t0 = time.perf_counter()
+    e2e_steps(n_e2e, 50)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": int(x_host.numel() * 2),
+           "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": n_e2e}
+    ctx.close()
+    del ctx, caches
+    torch.cuda.empty_cache()
+
+    extra, cpu = {}, None
+    if rank == 0:
+        if not args.no_extra:
+            for name, fn in EXTRAS.items():
+                try:
+                    extra[name] = fn(torch, B, W, peaks, args.quick)
+                except Exception as e:  # an extra must never take the headline line down
+                    extra[name] = {"error": f"{type(e).__name__}: {e}"}
+                torch.cuda.empty_cache()
+        if world == 1 and not args.no_cpu:
+            cpu = time_oracle()
+    sampler.stop()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    line = {"metric": "decode_tokens_per_s", "value": tok_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "config 2: one dense decoder layer (hidden 4096, 32 q / 8 kv heads x 128, SwiGLU 14336, 4-bit "
+                                   "block-32 weights), decode step at position 1024, batch 1, all tensors resident",
+                       "replicas_rotated": R, "weight_bytes_per_step": layer_bytes,
+                       "l2_policy": f"steps rotate over {R} distinct layers ({R * layer_bytes / 1e6:.0f} MB of weights > 126 MB L2)",
+                       "multi_gpu": "replicas only (no data-path collective)"},
+            "step_bytes_gbs": (layer_bytes + 2 * shape.n_kv_heads * cap * shape.head_dim * 2) / (ms / args.steps * 1e-3) / 1e9,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "extra": extra}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--replicas", type=int, default=8)
+    ap.add_argument("--no-extra", action="store_true", help="skip the figures of the other configs")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
+    ap.add_argument("--quick", action="store_true", help="smaller extras")
+    ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -57,7 +57,9 @@ enum { ATS_MODE_DECODE = 0, ATS_MODE_PREFILL = 1 };
 /* ats_config.flags */
 enum {
   ATS_FLAG_POISON_SLOTS = 1u,     /* debug: fill a ring slot with 0xFF after its consumer, so premature reuse shows */
-  ATS_FLAG_SKIP_SCALE_CHECK = 2u  /* do not scan scales for Inf/NaN at registration */
+  ATS_FLAG_SKIP_SCALE_CHECK = 2u, /* do not scan scales for Inf/NaN at registration */
+  ATS_FLAG_TIME_KERNELS = 4u,     /* bracket every GEMV / grouped GEMV / GEMM launch with CUDA events (see ats_stats.timed_*) */
+  ATS_FLAG_NO_PDL = 8u            /* launch every kernel fully serialized (no programmatic dependent launch overlap) */
 };
 /* ats_layer_desc.flags */
 enum { ATS_LAYER_NO_TOPK_RENORM = 1u /* gates = full softmax entries instead of softmax over the top-k */ };
@@ -70,7 +72,7 @@ typedef struct {
   uint32_t ring_slots;     /* number of equal staging slots (temporary GPU buffers, Section 4.2.1); 0 = no streaming */
   uint64_t slot_bytes;     /* bytes of one slot; every streamed tensor / expert slice must fit one slot */
   uint64_t chunk_bytes;    /* a streamed slice is copied as ceil(bytes/chunk_bytes) cudaMemcpyAsync calls */
-  uint64_t workspace_bytes;/* activation scratch for ats_layer_* / ats_moe_linear; see ats_workspace_bytes() */
+  uint64_t workspace_bytes;/* activation scratch (>= 1024; for ats_layer_* pass ats_workspace_bytes()) */
   int32_t device;          /* CUDA device ordinal of the arena and streams */
   uint32_t flags;
 } ats_config;
@@ -196,12 +198,21 @@ typedef struct {
   uint64_t kernel_launches;  /* kernels launched by the library since the last reset */
   uint64_t ring_reuses;      /* copies that had to wait for a slot's previous consumer */
   uint64_t host_syncs;       /* host waits for routing ids */
+  /* With ATS_FLAG_TIME_KERNELS: per kernel family (0 GEMV, 1 grouped-expert GEMV, 2 tensor-core GEMM) since the last
+   * reset: launches, summed device time of the completed launches (CUDA events on the compute stream) and the
+   * algorithmic work they did (families 0,1: bytes = weights + activations in + out; family 2: flops = 2*T*N*K). */
+  uint64_t timed_launches[3];
+  uint64_t timed_work[3];
+  double timed_ms[3];
   uint32_t n_streamed;       /* streamed slices since the last reset (list below holds the first ATS_STATS_LIST) */
   uint32_t reserved;
   int32_t streamed_ids[ATS_STATS_LIST];
   int32_t streamed_experts[ATS_STATS_LIST];
 } ats_stats;
-int32_t ats_get_stats(const ats_ctx* ctx, ats_stats* out /*HOST*/);
+/* Kernel times are read from events here: call after ats_sync() so that every timed launch has completed. */
+int32_t ats_get_stats(ats_ctx* ctx, ats_stats* out /*HOST*/);
+/* Replace the context's flags (ATS_FLAG_*) at run time, e.g. to switch kernel timing on for a profiling pass. */
+int32_t ats_set_flags(ats_ctx* ctx, uint32_t flags);
 int32_t ats_reset_stats(ats_ctx* ctx);
 
 /* Wait for everything enqueued so far by polling events; ATS_ERR_TIMEOUT after timeout_ms (0 = wait without limit),

@@ -21,7 +21,7 @@ ATS_HOST, ATS_GPU = 0, 1
 ATS_FMT_Q4B32, ATS_FMT_F16 = 0, 1
 ATS_OUT_F32, ATS_OUT_F16 = 0, 1
 ATS_MODE_DECODE, ATS_MODE_PREFILL = 0, 1
-ATS_FLAG_POISON_SLOTS, ATS_FLAG_SKIP_SCALE_CHECK = 1, 2
+ATS_FLAG_POISON_SLOTS, ATS_FLAG_SKIP_SCALE_CHECK, ATS_FLAG_TIME_KERNELS, ATS_FLAG_NO_PDL = 1, 2, 4, 8
 ATS_LAYER_NO_TOPK_RENORM = 1
 ATS_STATS_LIST = 512
 EDGES = ("h", "q", "k", "v", "q_rot", "a", "o", "x1", "h2", "g", "u", "act", "d")
@@ -29,7 +29,7 @@ EDGES = ("h", "q", "k", "v", "q_rot", "a", "o", "x1", "h2", "g", "u", "act", "d"
 EXPORTS = (
     "ats_init", "ats_destroy", "ats_last_error", "ats_register_tensor", "ats_tensor_slice_bytes", "ats_set_placement",
     "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_route_topk", "ats_moe_linear", "ats_layer_decode",
-    "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_reset_stats",
+    "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
     "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
     "ats_host_unpack_q4",
 )
@@ -55,7 +55,8 @@ class ats_layer_desc(C.Structure):
 class ats_stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("resident_bytes", "aux_bytes", "host_store_bytes", "streamed_bytes", "copies",
                                           "kernel_launches", "ring_reuses", "host_syncs")] + \
-               [("n_streamed", C.c_uint32), ("reserved", C.c_uint32),
+               [("timed_launches", C.c_uint64 * 3), ("timed_work", C.c_uint64 * 3), ("timed_ms", C.c_double * 3),
+                ("n_streamed", C.c_uint32), ("reserved", C.c_uint32),
                 ("streamed_ids", C.c_int32 * ATS_STATS_LIST), ("streamed_experts", C.c_int32 * ATS_STATS_LIST)]
 
 
@@ -85,6 +86,7 @@ def _load():
         "ats_get_numerics": (i32, [vp, u32, P(u32), P(u32)]),
         "ats_get_stats": (i32, [vp, P(ats_stats)]),
         "ats_reset_stats": (i32, [vp]),
+        "ats_set_flags": (i32, [vp, u32]),
         "ats_sync": (i32, [vp, u32]),
         "ats_measure_h2d": (i32, [vp, u64, u32, P(C.c_double)]),
         "ats_debug_fail_copies": (i32, [vp, u32]),
@@ -238,6 +240,9 @@ class Context:
         s = ats_stats()
         self.check(lib.ats_get_stats(self.h, C.byref(s)))
         return s
+
+    def set_flags(self, flags):
+        return self.check(lib.ats_set_flags(self.h, flags))
 
     def reset_stats(self):
         return self.check(lib.ats_reset_stats(self.h))

@@ -84,7 +84,17 @@ struct ats_ctx {
   cudaEvent_t ids_event = nullptr;
   cudaEvent_t sync_event = nullptr;
   uint32_t fail_copies = 0;
+  int* dev_status = nullptr;  // device word kernels raise when a bounded wait expires (first bytes of the workspace)
+  int* host_status = nullptr; // pinned copy read by ats_sync
+  int sm_count = 148;
+  std::vector<double> rope_inv;  // cached theta^(-2i/d)
+  float rope_theta = -1.f;
+  int rope_d = 0;
   ats_stats stats{};
+  // kernel timing (ATS_FLAG_TIME_KERNELS): event pairs in launch order, family per pair
+  std::vector<cudaEvent_t> tev;
+  std::vector<uint8_t> tev_family;
+  size_t tev_used = 0;  // events handed out (2 per timed launch)
 };
 
 namespace ats {
@@ -121,8 +131,19 @@ struct GemvParams {
   const __half* res16;
   int ldres;
   int mode;
+  // optional RMSNorm prologue (M = 1): x = rn16(norm_x * norm_gain / sqrt(mean(norm_x^2) + norm_eps)); exactly one of
+  // norm_x16 / norm_x32 is set when norm_gain is; norm_out (optional) receives the normalised operand
+  const __half* norm_x16;
+  const float* norm_x32;
+  const __half* norm_gain;
+  float norm_eps;
+  __half* norm_out;
+  int pdl;  // allow the launch to overlap the tail of the preceding kernel (programmatic dependent launch)
 };
 cudaError_t launch_gemv(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
+// the streaming single-token kernel (kernels_gemv_stream.cu): shapes it accepts, and its launcher
+bool gemv_stream_eligible(const GemvParams& p);
+cudaError_t launch_gemv_stream(const GemvParams& p, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch);
 
 // Grouped-expert GEMV: job j multiplies the slice w0[j] (and w1[j] for SwiGLU) with activation row xrow[j] and
 // writes output row j_out[j].  Implicit mode (n_jobs_explicit == 0): job p = 0..P-1 uses expert ids[p] of a
@@ -159,13 +180,22 @@ cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, i
                            uint64_t* n_launch);
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
                            cudaStream_t st, uint64_t* n_launch);
-// decode: rotary embedding of q (fp32 -> fp32) and k, append k/v rows to the caches at `pos`
-cudaError_t launch_rope_append_decode(const float* qkv, float* q_rot, __half* kc, __half* vc, int n_q, int n_kv, int d,
-                                      int cap, int pos, float theta, cudaStream_t st, uint64_t* n_launch);
+// decode attention, fused with the rotary embedding and the KV append (kernels_decode.cu)
+struct AttnDecodeParams {
+  const float* qkv;   // [q | k | v] fp32 of the new token
+  float* q_rot_out;   // optional copy of the rotated query (debug / tests)
+  __half* kc;
+  __half* vc;
+  float* part;        // [n_q][splits][d + 2] scratch
+  int* counters;      // [n_kv] zero between launches
+  __half* a16;        // [n_q * d]
+  int n_q, n_kv, group, cap, pos;
+  float scale;
+  float cs[128];      // (cos, sin) of pos * theta^(-2i/d), i < d/2
+};
 int attn_decode_splits(int n_ctx);
 size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx);
-cudaError_t launch_attn_decode(const float* q_rot, const __half* kc, const __half* vc, float* scratch, __half* a16,
-                               int n_q, int n_kv, int d, int cap, int n_ctx, cudaStream_t st, uint64_t* n_launch);
+cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch);
 cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
                                float* gates, cudaStream_t st, uint64_t* n_launch);
 // y16[m] = rn16(res[m] + sum_j gates[m][j] * d32[m*k + j])   (res fp16 or fp32)

@@ -43,11 +43,50 @@ int32_t check_cuda(ats_ctx* c, cudaError_t e, const char* what) {
     if (_s != ATS_OK) return _s;   \
   } while (0)
 
+constexpr uint64_t kWsReserved = 1024;  // status word + attention counters at the start of the workspace
+
+// Kernel timing: a pair of events around one launch on the compute stream.
+constexpr size_t kMaxTimedLaunches = 1 << 16;
+struct TimedLaunch {
+  ats_ctx* ctx;
+  cudaEvent_t stop = nullptr;
+  TimedLaunch(ats_ctx* c, int family, uint64_t work) : ctx(c) {
+    if (!(c->cfg.flags & ATS_FLAG_TIME_KERNELS) || c->tev_used / 2 >= kMaxTimedLaunches) return;
+    while (c->tev.size() < c->tev_used + 2) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->tev.push_back(e);
+    }
+    cudaEvent_t start = c->tev[c->tev_used];
+    stop = c->tev[c->tev_used + 1];
+    if (c->tev_family.size() < c->tev_used / 2 + 1) c->tev_family.resize(c->tev_used / 2 + 1);
+    c->tev_family[c->tev_used / 2] = (uint8_t)family;
+    c->tev_used += 2;
+    c->stats.timed_launches[family]++;
+    c->stats.timed_work[family] += work;
+    cudaEventRecord(start, c->cs);
+  }
+  ~TimedLaunch() {
+    if (stop) cudaEventRecord(stop, ctx->cs);
+  }
+};
+
+static uint64_t gemv_work_bytes(const GemvParams& p) {
+  uint64_t rows = 0;
+  for (int i = 0; i < p.n_seg; ++i) rows += (uint64_t)p.seg[i].n_rows;
+  const uint64_t K = (uint64_t)p.K, M = (uint64_t)p.M;
+  const uint64_t out_rows = p.mode == GEMV_SWIGLU_F16 ? rows / 2 : rows;
+  const uint64_t out_b = (p.mode == GEMV_OUT_F32 || p.mode == GEMV_RES16_OUT_F32) ? 4 : 2;
+  return rows * K / 2 + rows * (K / 32) * 2 + M * K * 2 + M * out_rows * out_b;
+}
+
 static int32_t precheck(ats_ctx* ctx, bool need_placement) {
   if (!ctx) return ATS_ERR_INVALID;
   if (ctx->poisoned) return fail(ctx, ATS_ERR_CUDA, "context is poisoned by an earlier CUDA error: %s", ctx->err.c_str());
   if (need_placement && !ctx->placed)
     return fail(ctx, ATS_ERR_STATE, "no placement: call ats_set_placement or ats_plan_placement first");
+  if (need_placement && !ctx->dev_status)
+    return fail(ctx, ATS_ERR_NOMEM, "workspace_bytes must be at least %llu", (unsigned long long)kWsReserved);
   return ATS_OK;
 }
 
@@ -190,6 +229,27 @@ static int count_streamed(const Operand* ops, int n) {
   return c;
 }
 
+// One GEMV launch: the streaming kernel where the shapes allow it, else the generic kernel (preceded by a separate
+// RMSNorm launch when a norm prologue was asked for).  Which kernel runs depends on shapes only, never on placement.
+static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
+  p.pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
+  if (gemv_stream_eligible(p)) {
+    TimedLaunch tl(ctx, 0, gemv_work_bytes(p));
+    ATS_CUDA(launch_gemv_stream(p, ctx->dev_status, ctx->sm_count, ctx->cs, &ctx->stats.kernel_launches));
+    return ATS_OK;
+  }
+  if (p.norm_gain) {
+    if (!p.norm_out) return fail(ctx, ATS_ERR_INVALID, "internal: norm prologue without an output buffer");
+    ATS_CUDA(launch_rmsnorm(p.norm_x32 ? (const void*)p.norm_x32 : (const void*)p.norm_x16, p.norm_x32 != nullptr, p.norm_gain,
+                            p.norm_out, p.M, p.K, p.norm_eps, ctx->cs, &ctx->stats.kernel_launches));
+    p.x = p.norm_out;
+    p.norm_gain = nullptr;
+  }
+  TimedLaunch tl(ctx, 0, gemv_work_bytes(p));
+  ATS_CUDA(launch_gemv(p, ctx->cs, &ctx->stats.kernel_launches));
+  return ATS_OK;
+}
+
 // GEMV over 1..3 dense tensors whose outputs lie side by side.  When the ring cannot hold all streamed operands of
 // the group at once the segments run one by one (same per-row arithmetic, so results do not depend on it).
 static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
@@ -198,7 +258,7 @@ static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
     ATS_TRY(acquire_ops(ctx, ops, n));
     p.n_seg = n;
     for (int i = 0; i < n; ++i) p.seg[i] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
-    ATS_CUDA(launch_gemv(p, ctx->cs, &ctx->stats.kernel_launches));
+    ATS_TRY(launch_gemv_any(ctx, p));
     return release_ops(ctx, ops, n);
   }
   if (p.mode == GEMV_SWIGLU_F16)
@@ -213,7 +273,7 @@ static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
     if (q.y16) q.y16 += row0;
     if (q.res32) q.res32 += row0;
     if (q.res16) q.res16 += row0;
-    ATS_CUDA(launch_gemv(q, ctx->cs, &ctx->stats.kernel_launches));
+    ATS_TRY(launch_gemv_any(ctx, q));
     ATS_TRY(release_ops(ctx, ops + i, 1));
     row0 += (int)ops[i].t->d.n_out;
   }
@@ -226,8 +286,16 @@ static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
   if (count_streamed(ops, n) <= (int)ctx->cfg.ring_slots || n == 1) {
     ATS_TRY(acquire_ops(ctx, ops, n));
     p.n_seg = n;
-    for (int i = 0; i < n; ++i) p.seg[i] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
-    cudaError_t e = launch_gemm(p, ctx->cs, &ctx->stats.kernel_launches, &err);
+    uint64_t rows = 0;
+    for (int i = 0; i < n; ++i) {
+      p.seg[i] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
+      rows += ops[i].t->d.n_out;
+    }
+    cudaError_t e;
+    {
+      TimedLaunch tl(ctx, 2, 2ull * (uint64_t)p.T * rows * (uint64_t)p.K);
+      e = launch_gemm(p, ctx->cs, &ctx->stats.kernel_launches, &err);
+    }
     if (e != cudaSuccess) return check_cuda(ctx, e, err.empty() ? "launch_gemm" : err.c_str());
     return release_ops(ctx, ops, n);
   }
@@ -238,7 +306,11 @@ static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
     q.n_seg = 1;
     q.seg[0] = GemvSeg{ops[i].ptr, (int)ops[i].t->d.n_out};
     q.y += row0;
-    cudaError_t e = launch_gemm(q, ctx->cs, &ctx->stats.kernel_launches, &err);
+    cudaError_t e;
+    {
+      TimedLaunch tl(ctx, 2, 2ull * (uint64_t)q.T * (uint64_t)q.seg[0].n_rows * (uint64_t)q.K);
+      e = launch_gemm(q, ctx->cs, &ctx->stats.kernel_launches, &err);
+    }
     if (e != cudaSuccess) return check_cuda(ctx, e, err.empty() ? "launch_gemm" : err.c_str());
     ATS_TRY(release_ops(ctx, ops + i, 1));
     row0 += (int)ops[i].t->d.n_out;
@@ -289,6 +361,7 @@ struct LayerWs {
 static LayerWs layout_decode(const ats_layer_desc& L, uint32_t M, uint8_t* base, uint64_t cap) {
   LayerWs w;
   Bump b(base, cap);
+  b.take(kWsReserved);
   const uint64_t H = L.hidden, qd = (uint64_t)L.n_q_heads * L.head_dim, kvd = (uint64_t)L.n_kv_heads * L.head_dim;
   if (L.wq >= 0) {
     w.h16 = (__half*)b.take(M * H * 2);
@@ -316,6 +389,7 @@ static LayerWs layout_decode(const ats_layer_desc& L, uint32_t M, uint8_t* base,
 static LayerWs layout_prefill(const ats_layer_desc& L, uint32_t T, uint8_t* base, uint64_t cap) {
   LayerWs w;
   Bump b(base, cap);
+  b.take(kWsReserved);
   const uint64_t H = L.hidden, qd = (uint64_t)L.n_q_heads * L.head_dim, kvd = (uint64_t)L.n_kv_heads * L.head_dim;
   uint64_t scratch = 0;
   if (L.wq >= 0) {
@@ -417,6 +491,7 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
   if (!ids_host) {
     p.base0 = t0.slices[0].dev;
     p.base1 = t1 ? t1->slices[0].dev : nullptr;
+    TimedLaunch tl(ctx, 1, (uint64_t)p.P * ((t1 ? 2 : 1) * t0.slice_bytes + (uint64_t)p.K * 2 + (uint64_t)p.n_rows * 2));
     ATS_CUDA(launch_moe_gemv(p, nullptr, ctx->cs, &ctx->stats.kernel_launches));
     return ATS_OK;
   }
@@ -425,6 +500,7 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
   jobs.n = 0;
   auto flush = [&]() -> int32_t {
     if (jobs.n == 0) return ATS_OK;
+    TimedLaunch tl(ctx, 1, (uint64_t)jobs.n * ((t1 ? 2 : 1) * t0.slice_bytes + (uint64_t)p.K * 2 + (uint64_t)p.n_rows * 2));
     ATS_CUDA(launch_moe_gemv(p, &jobs, ctx->cs, &ctx->stats.kernel_launches));
     jobs.n = 0;
     return ATS_OK;
@@ -514,6 +590,30 @@ static void plan_moe(ats_ctx* ctx, const int32_t* ids_host, int P, const int* te
       if (ctx->tensors[tensor_ids[t]].slices[e].where == ATS_HOST) plan_add(ctx, tensor_ids[t], e);
 }
 
+// (cos, sin) of pos * theta^(-2i/d) for i < d/2, formed in fp64 on the host and rounded to fp32.  The inverse
+// frequencies are cached per (theta, d).
+static void rope_table(ats_ctx* ctx, float theta, int d, int pos, float* cs) {
+  const int half = d / 2;
+  if (theta == 0.f) {
+    for (int i = 0; i < half; ++i) {
+      cs[2 * i] = 1.f;
+      cs[2 * i + 1] = 0.f;
+    }
+    return;
+  }
+  if (ctx->rope_theta != theta || ctx->rope_d != d) {
+    ctx->rope_inv.resize(half);
+    for (int i = 0; i < half; ++i) ctx->rope_inv[i] = pow((double)theta, -2.0 * (double)i / (double)d);
+    ctx->rope_theta = theta;
+    ctx->rope_d = d;
+  }
+  for (int i = 0; i < half; ++i) {
+    const double a = (double)pos * ctx->rope_inv[i];
+    cs[2 * i] = (float)cos(a);
+    cs[2 * i + 1] = (float)sin(a);
+  }
+}
+
 }  // namespace ats
 
 using namespace ats;
@@ -551,6 +651,14 @@ int32_t ats_init(const ats_config* cfg, ats_ctx** out) {
   ok &= cudaEventCreateWithFlags(&ctx->ids_event, cudaEventDisableTiming) == cudaSuccess;
   ok &= cudaEventCreateWithFlags(&ctx->sync_event, cudaEventDisableTiming) == cudaSuccess;
   ok &= cudaHostAlloc((void**)&ctx->ids_host, 4096 * sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess;
+  ok &= cudaHostAlloc((void**)&ctx->host_status, 64, cudaHostAllocDefault) == cudaSuccess;
+  if (ws >= kWsReserved) {
+    ctx->dev_status = (int*)ctx->ws;
+    ok &= cudaMemsetAsync(ctx->ws, 0, kWsReserved, ctx->cs) == cudaSuccess;
+    ok &= cudaStreamSynchronize(ctx->cs) == cudaSuccess;
+  }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0) ctx->sm_count = sms;
   if (!ok) {
     ats_destroy(ctx);
     return ATS_ERR_CUDA;
@@ -569,9 +677,11 @@ int32_t ats_destroy(ats_ctx* ctx) {
     if (s.ready) cudaEventDestroy(s.ready);
     if (s.freed) cudaEventDestroy(s.freed);
   }
+  for (cudaEvent_t e : ctx->tev) cudaEventDestroy(e);
   if (ctx->ids_event) cudaEventDestroy(ctx->ids_event);
   if (ctx->sync_event) cudaEventDestroy(ctx->sync_event);
   if (ctx->ids_host) cudaFreeHost(ctx->ids_host);
+  if (ctx->host_status) cudaFreeHost(ctx->host_status);
   delete ctx;
   return ATS_OK;
 }
@@ -884,20 +994,34 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   }
   ATS_TRY(pump(ctx));
 
+  const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
   if (attn) {
-    ATS_CUDA(launch_rmsnorm(x_in, 0, (const __half*)ctx->tensors[L->attn_norm].f16_dev, w.h16, (int)M, H, L->rms_eps, ctx->cs, nl));
     GemvParams p{};
     p.M = (int)M;
-    p.x = w.h16;
+    p.norm_x16 = (const __half*)x_in;
+    p.norm_gain = (const __half*)ctx->tensors[L->attn_norm].f16_dev;
+    p.norm_eps = L->rms_eps;
+    p.norm_out = w.h16;
     p.ldx = H;
     p.y32 = w.qkv32;
     p.ldy = qd + 2 * kvd;
     p.mode = GEMV_OUT_F32;
     ATS_TRY(run_gemv_group(ctx, qkv, 3, p));
-    ATS_CUDA(launch_rope_append_decode(w.qkv32, w.qrot32, (__half*)k_cache, (__half*)v_cache, nq, nkv, d, (int)L->kv_capacity,
-                                       (int)pos, L->rope_theta, ctx->cs, nl));
-    ATS_CUDA(launch_attn_decode(w.qrot32, (const __half*)k_cache, (const __half*)v_cache, w.attn_scratch, w.a16, nq, nkv, d,
-                                (int)L->kv_capacity, (int)pos + 1, ctx->cs, nl));
+    AttnDecodeParams ap{};
+    ap.qkv = w.qkv32;
+    ap.q_rot_out = w.qrot32;
+    ap.kc = (__half*)k_cache;
+    ap.vc = (__half*)v_cache;
+    ap.part = w.attn_scratch;
+    ap.counters = ctx->dev_status + 64;
+    ap.a16 = w.a16;
+    ap.n_q = nq;
+    ap.n_kv = nkv;
+    ap.group = nq / nkv;
+    ap.cap = (int)L->kv_capacity;
+    ap.pos = (int)pos;
+    rope_table(ctx, L->rope_theta, d, (int)pos, ap.cs);
+    ATS_CUDA(launch_attn_decode_fused(ap, d, pdl, ctx->cs, nl));
     GemvParams o{};
     o.M = (int)M;
     o.x = w.a16;
@@ -909,12 +1033,16 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     o.mode = GEMV_RES16_OUT_F32;
     ATS_TRY(run_gemv_group(ctx, &wo, 1, o));
   }
-  ATS_CUDA(launch_rmsnorm(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev,
-                          w.h2_16, (int)M, H, L->rms_eps, ctx->cs, nl));
+  if (L->n_experts != 0)  // the MoE path needs the normalised row in memory (router and grouped GEMV read it)
+    ATS_CUDA(launch_rmsnorm(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev,
+                            w.h2_16, (int)M, H, L->rms_eps, ctx->cs, nl));
   if (L->n_experts == 0) {
     GemvParams g{};
     g.M = (int)M;
-    g.x = w.h2_16;
+    if (attn) g.norm_x32 = w.x1_32; else g.norm_x16 = (const __half*)x_in;
+    g.norm_gain = (const __half*)ctx->tensors[L->ffn_norm].f16_dev;
+    g.norm_eps = L->rms_eps;
+    g.norm_out = w.h2_16;
     g.ldx = H;
     g.y16 = w.act16;
     g.ldy = (int)L->ffn;
@@ -1059,9 +1187,23 @@ int32_t ats_get_numerics(const ats_ctx* ctx, uint32_t mode, uint32_t* fp16_edge_
   return ATS_OK;
 }
 
-int32_t ats_get_stats(const ats_ctx* ctx, ats_stats* out) {
+int32_t ats_get_stats(ats_ctx* ctx, ats_stats* out) {
   if (!ctx || !out) return ATS_ERR_INVALID;
+  for (int f = 0; f < 3; ++f) ctx->stats.timed_ms[f] = 0.0;
+  for (size_t i = 0; i + 1 < ctx->tev_used; i += 2) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->tev[i], ctx->tev[i + 1]) == cudaSuccess)
+      ctx->stats.timed_ms[ctx->tev_family[i / 2]] += ms;
+    else
+      cudaGetLastError();  // launch not finished yet: not counted
+  }
   *out = ctx->stats;
+  return ATS_OK;
+}
+
+int32_t ats_set_flags(ats_ctx* ctx, uint32_t flags) {
+  if (!ctx) return ATS_ERR_INVALID;
+  ctx->cfg.flags = flags;
   return ATS_OK;
 }
 
@@ -1070,6 +1212,11 @@ int32_t ats_reset_stats(ats_ctx* ctx) {
   ats_stats& s = ctx->stats;
   s.streamed_bytes = s.copies = s.kernel_launches = s.ring_reuses = s.host_syncs = 0;
   s.n_streamed = 0;
+  for (int f = 0; f < 3; ++f) {
+    s.timed_launches[f] = s.timed_work[f] = 0;
+    s.timed_ms[f] = 0.0;
+  }
+  ctx->tev_used = 0;
   return ATS_OK;
 }
 
@@ -1093,6 +1240,14 @@ int32_t ats_sync(ats_ctx* ctx, uint32_t timeout_ms) {
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return check_cuda(ctx, e, "asynchronous error");
+  if (ctx->dev_status) {
+    ATS_CUDA(cudaMemcpyAsync(ctx->host_status, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->cs));
+    ATS_CUDA(cudaStreamSynchronize(ctx->cs));
+    if (*ctx->host_status != 0) {
+      ctx->poisoned = true;
+      return fail(ctx, ATS_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d); results are invalid", *ctx->host_status);
+    }
+  }
   return ATS_OK;
 }
 

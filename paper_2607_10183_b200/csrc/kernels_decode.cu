@@ -405,122 +405,106 @@ cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __ha
   return cudaGetLastError();
 }
 
-// ------------------------------------------------------------------------------------------- RoPE + KV append (decode)
-// Half-split pairing: (u_i, u_{i+d/2}) rotated by pos * theta^(-2i/d); the angle is formed in fp64.
-__device__ __forceinline__ void rope_cs(int i, int d, int pos, float theta, float* c, float* s) {
-  if (theta == 0.f) {
-    *c = 1.f;
-    *s = 0.f;
-    return;
-  }
-  const double inv = pow((double)theta, -2.0 * (double)i / (double)d);
-  double sd, cd;
-  sincos((double)pos * inv, &sd, &cd);
-  *c = (float)cd;
-  *s = (float)sd;
-}
+// ------------------------------------------------------------------------------------------- fused decode attention
+// One launch does the rotary embedding of q and of the new key (half-split pairs, angle pos * theta^(-2i/d), the
+// cos/sin table for `pos` computed on the host in fp64 and passed by value), appends the new K/V row to the caches as
+// fp16, attends over positions 0..pos split across CTAs, and merges the splits: the last CTA to finish a kv head
+// (a counter in global memory, reset for the next launch) sums the partials in ascending split order, so the result
+// does not depend on which CTA arrives last.  CTA (split, kv head) covers 64 positions, one per lane of its 2 warps,
+// for all query heads of the group.
+constexpr int kAttnPos = 64;
+constexpr int kAttnMaxGroup = 8;
 
-__global__ void rope_append_decode_kernel(const float* __restrict__ qkv, float* __restrict__ q_rot, __half* __restrict__ kc,
-                                          __half* __restrict__ vc, int n_q, int n_kv, int d, int cap, int pos, float theta) {
-  const int half = d / 2;
-  const int n_pairs = (n_q + n_kv) * half;
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  const int qd = n_q * d, kvd = n_kv * d;
-  if (idx < n_pairs) {
-    const int hh = idx / half, i = idx % half;
-    float c, s;
-    rope_cs(i, d, pos, theta, &c, &s);
-    if (hh < n_q) {
-      const float a = qkv[hh * d + i], b = qkv[hh * d + i + half];
-      q_rot[hh * d + i] = a * c - b * s;
-      q_rot[hh * d + i + half] = b * c + a * s;
-    } else {
-      const int kvh = hh - n_q;
-      const float a = qkv[qd + kvh * d + i], b = qkv[qd + kvh * d + i + half];
-      __half* dst = kc + ((size_t)kvh * cap + pos) * d;
+int attn_decode_splits(int n_ctx) { return (n_ctx + kAttnPos - 1) / kAttnPos; }
+size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) { return (size_t)n_q * attn_decode_splits(n_ctx) * (d + 2); }
+
+template <int D>
+__global__ void __launch_bounds__(kAttnPos) attn_decode_fused_kernel(const AttnDecodeParams p) {
+  constexpr int V = D / 32;  // output dims per lane
+  constexpr int NW = kAttnPos / 32;
+  __shared__ float q_s[kAttnMaxGroup * D];
+  __shared__ float w_m[NW][kAttnMaxGroup], w_l[NW][kAttnMaxGroup];
+  __shared__ float w_acc[NW][kAttnMaxGroup][D];
+  __shared__ int is_last;
+  const int split = blockIdx.x, kvh = blockIdx.y, n_splits = gridDim.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int group = p.group, half = D / 2, n_ctx = p.pos + 1;
+  const int qd = p.n_q * D, kvd = p.n_kv * D;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // rotary embedding of the group's query heads into shared memory
+  for (int idx = threadIdx.x; idx < group * half; idx += blockDim.x) {
+    const int g = idx / half, i = idx % half;
+    const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
+    const float* q = p.qkv + (size_t)(kvh * group + g) * D;
+    const float a = q[i], b = q[i + half];
+    const float ra = a * c - b * s, rb = b * c + a * s;
+    q_s[g * D + i] = ra;
+    q_s[g * D + i + half] = rb;
+    if (p.q_rot_out && split == 0) {
+      p.q_rot_out[(size_t)(kvh * group + g) * D + i] = ra;
+      p.q_rot_out[(size_t)(kvh * group + g) * D + i + half] = rb;
+    }
+  }
+  // the CTA that owns position `pos` appends the new key (rotated) and value rows first
+  if (split == p.pos / kAttnPos) {
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+      const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
+      const float* k = p.qkv + qd + (size_t)kvh * D;
+      const float a = k[i], b = k[i + half];
+      __half* dst = p.kc + ((size_t)kvh * p.cap + p.pos) * D;
       dst[i] = __float2half_rn(a * c - b * s);
       dst[i + half] = __float2half_rn(b * c + a * s);
     }
-  } else if (idx < n_pairs + kvd) {
-    const int j = idx - n_pairs;
-    const int kvh = j / d, e = j % d;
-    vc[((size_t)kvh * cap + pos) * d + e] = __float2half_rn(qkv[qd + kvd + j]);
+    for (int e = threadIdx.x; e < D; e += blockDim.x)
+      p.vc[((size_t)kvh * p.cap + p.pos) * D + e] = __float2half_rn(p.qkv[qd + kvd + (size_t)kvh * D + e]);
   }
-}
-
-cudaError_t launch_rope_append_decode(const float* qkv, float* q_rot, __half* kc, __half* vc, int n_q, int n_kv, int d,
-                                      int cap, int pos, float theta, cudaStream_t st, uint64_t* n_launch) {
-  const int total = (n_q + n_kv) * (d / 2) + n_kv * d;
-  rope_append_decode_kernel<<<(total + 127) / 128, 128, 0, st>>>(qkv, q_rot, kc, vc, n_q, n_kv, d, cap, pos, theta);
-  ++*n_launch;
-  return cudaGetLastError();
-}
-
-// ------------------------------------------------------------------------------------------- decode attention
-// Split over cache positions: CTA (split, kv head) covers 128 positions, one per lane of its 4 warps, for all query
-// heads of the group.  Partials (running max, sum, unnormalised output) go to scratch; a second kernel merges the
-// splits in ascending order.
-constexpr int kAttnPosPerCta = 128;
-constexpr int kAttnMaxGroup = 8;
-
-int attn_decode_splits(int n_ctx) { return (n_ctx + kAttnPosPerCta - 1) / kAttnPosPerCta; }
-size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) {
-  return (size_t)n_q * attn_decode_splits(n_ctx) * (d + 2);
-}
-
-template <int D>
-__global__ void __launch_bounds__(128) attn_decode_partial_kernel(const float* __restrict__ q_rot, const __half* __restrict__ kc,
-                                                                  const __half* __restrict__ vc, float* __restrict__ part,
-                                                                  int group, int cap, int n_ctx, int n_splits, float scale) {
-  constexpr int V = D / 32;  // output dims per lane
-  __shared__ float q_s[kAttnMaxGroup * D];
-  __shared__ float w_m[4][kAttnMaxGroup], w_l[4][kAttnMaxGroup];
-  __shared__ float w_acc[4][kAttnMaxGroup][D];
-  const int split = blockIdx.x, kvh = blockIdx.y;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int i = threadIdx.x; i < group * D; i += blockDim.x) q_s[i] = q_rot[(size_t)kvh * group * D + i];
   __syncthreads();
-  const int t0 = split * kAttnPosPerCta + warp * 32;
+  const int t0 = split * kAttnPos + warp * 32;
   const int t = t0 + lane;
   const bool ok = t < n_ctx;
   float sc[kAttnMaxGroup];
 #pragma unroll
   for (int g = 0; g < kAttnMaxGroup; ++g) sc[g] = 0.f;
   if (ok) {
-    const uint4* kr = reinterpret_cast<const uint4*>(kc + ((size_t)kvh * cap + t) * D);
-#pragma unroll 4
+    const uint4* kr = reinterpret_cast<const uint4*>(p.kc + ((size_t)kvh * p.cap + t) * D);
+    uint4 kv[D / 8];
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) kv[c] = kr[c];  // plain loads: the row at `pos` was written by this CTA
+#pragma unroll
     for (int c = 0; c < D / 8; ++c) {
-      const uint4 kv = __ldg(kr + c);
       float kf[8];
       float2 f;
-      f = __half22float2(u32_as_half2(kv.x)); kf[0] = f.x; kf[1] = f.y;
-      f = __half22float2(u32_as_half2(kv.y)); kf[2] = f.x; kf[3] = f.y;
-      f = __half22float2(u32_as_half2(kv.z)); kf[4] = f.x; kf[5] = f.y;
-      f = __half22float2(u32_as_half2(kv.w)); kf[6] = f.x; kf[7] = f.y;
+      f = __half22float2(u32_as_half2(kv[c].x)); kf[0] = f.x; kf[1] = f.y;
+      f = __half22float2(u32_as_half2(kv[c].y)); kf[2] = f.x; kf[3] = f.y;
+      f = __half22float2(u32_as_half2(kv[c].z)); kf[4] = f.x; kf[5] = f.y;
+      f = __half22float2(u32_as_half2(kv[c].w)); kf[6] = f.x; kf[7] = f.y;
 #pragma unroll
       for (int g = 0; g < kAttnMaxGroup; ++g) {
         if (g < group) {
-          const float* qg = q_s + g * D + c * 8;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) sc[g] = fmaf(kf[e], qg[e], sc[g]);
+          const float4 q0 = *reinterpret_cast<const float4*>(q_s + g * D + c * 8);
+          const float4 q1 = *reinterpret_cast<const float4*>(q_s + g * D + c * 8 + 4);
+          sc[g] = fmaf(kf[0], q0.x, sc[g]); sc[g] = fmaf(kf[1], q0.y, sc[g]);
+          sc[g] = fmaf(kf[2], q0.z, sc[g]); sc[g] = fmaf(kf[3], q0.w, sc[g]);
+          sc[g] = fmaf(kf[4], q1.x, sc[g]); sc[g] = fmaf(kf[5], q1.y, sc[g]);
+          sc[g] = fmaf(kf[6], q1.z, sc[g]); sc[g] = fmaf(kf[7], q1.w, sc[g]);
         }
       }
     }
   }
-  float p[kAttnMaxGroup];
+  float pr[kAttnMaxGroup];
 #pragma unroll
   for (int g = 0; g < kAttnMaxGroup; ++g) {
+    pr[g] = 0.f;
     if (g < group) {
-      const float s = ok ? sc[g] * scale : -INFINITY;
+      const float s = ok ? sc[g] * p.scale : -INFINITY;
       const float m = warp_max(s);
-      p[g] = (ok && m > -INFINITY) ? expf(s - m) : 0.f;
-      const float l = warp_sum(p[g]);
+      pr[g] = (ok && m > -INFINITY) ? expf(s - m) : 0.f;
+      const float l = warp_sum(pr[g]);
       if (lane == 0) {
         w_m[warp][g] = m;
         w_l[warp][g] = l;
       }
-    } else {
-      p[g] = 0.f;
     }
   }
   float acc[kAttnMaxGroup][V];
@@ -529,24 +513,24 @@ __global__ void __launch_bounds__(128) attn_decode_partial_kernel(const float* _
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[g][v] = 0.f;
   const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
+#pragma unroll 8
   for (int tt = 0; tt < n_here; ++tt) {
-    const __half* vr = vc + ((size_t)kvh * cap + t0 + tt) * D + lane * V;
+    const __half* vr = p.vc + ((size_t)kvh * p.cap + t0 + tt) * D + lane * V;
     float vf[V];
     if (V == 4) {
-      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(vr));
+      const uint2 raw = *reinterpret_cast<const uint2*>(vr);
       float2 f;
       f = __half22float2(u32_as_half2(raw.x)); vf[0] = f.x; vf[1] = f.y;
       f = __half22float2(u32_as_half2(raw.y)); vf[2] = f.x; vf[3] = f.y;
     } else {
-      const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(vr));
-      const float2 f = __half22float2(u32_as_half2(raw));
+      const float2 f = __half22float2(u32_as_half2(*reinterpret_cast<const uint32_t*>(vr)));
       vf[0] = f.x;
       vf[1] = f.y;
     }
 #pragma unroll
     for (int g = 0; g < kAttnMaxGroup; ++g) {
       if (g < group) {
-        const float pt = __shfl_sync(0xffffffffu, p[g], tt);
+        const float pt = __shfl_sync(0xffffffffu, pr[g], tt);
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[g][v] = fmaf(pt, vf[v], acc[g][v]);
       }
@@ -558,58 +542,69 @@ __global__ void __launch_bounds__(128) attn_decode_partial_kernel(const float* _
 #pragma unroll
       for (int v = 0; v < V; ++v) w_acc[warp][g][lane * V + v] = acc[g][v];
   __syncthreads();
-  // merge the 4 warps (ascending) and write this split's partial for each head of the group
+  // merge the warps (ascending) into this split's partial for each head of the group
   for (int idx = threadIdx.x; idx < group * D; idx += blockDim.x) {
     const int g = idx / D, e = idx % D;
     float mx = -INFINITY;
-    for (int w = 0; w < 4; ++w) mx = fmaxf(mx, w_m[w][g]);
+    for (int w = 0; w < NW; ++w) mx = fmaxf(mx, w_m[w][g]);
     float l = 0.f, o = 0.f;
-    for (int w = 0; w < 4; ++w) {
+    for (int w = 0; w < NW; ++w) {
       const float f = w_m[w][g] > -INFINITY ? expf(w_m[w][g] - mx) : 0.f;
       l = fmaf(w_l[w][g], f, l);
       o = fmaf(w_acc[w][g][e], f, o);
     }
-    float* dst = part + ((size_t)(kvh * group + g) * n_splits + split) * (D + 2);
+    float* dst = p.part + ((size_t)(kvh * group + g) * n_splits + split) * (D + 2);
     dst[e] = o;
     if (e == 0) {
       dst[D] = mx;
       dst[D + 1] = l;
     }
   }
+  // last CTA of this kv head merges the splits
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int prev = atomicAdd(p.counters + kvh, 1);
+    is_last = prev == n_splits - 1;
+    if (is_last) p.counters[kvh] = 0;  // ready for the next launch
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int idx = threadIdx.x; idx < group * D; idx += blockDim.x) {
+    const int g = idx / D, e = idx % D;
+    const float* base = p.part + (size_t)(kvh * group + g) * n_splits * (D + 2);
+    float mx = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldcg(base + (size_t)s * (D + 2) + D));
+    float l = 0.f, o = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+      const float* ps = base + (size_t)s * (D + 2);
+      const float m = __ldcg(ps + D);
+      const float f = m > -INFINITY ? expf(m - mx) : 0.f;
+      l = fmaf(__ldcg(ps + D + 1), f, l);
+      o = fmaf(__ldcg(ps + e), f, o);
+    }
+    p.a16[(size_t)(kvh * group + g) * D + e] = __float2half_rn(o / l);
+  }
 }
 
-template <int D>
-__global__ void attn_decode_combine_kernel(const float* __restrict__ part, __half* __restrict__ a16, int n_splits) {
-  const int hq = blockIdx.x, e = threadIdx.x;
-  const float* base = part + (size_t)hq * n_splits * (D + 2);
-  float mx = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, base[(size_t)s * (D + 2) + D]);
-  float l = 0.f, o = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float* ps = base + (size_t)s * (D + 2);
-    const float f = ps[D] > -INFINITY ? expf(ps[D] - mx) : 0.f;
-    l = fmaf(ps[D + 1], f, l);
-    o = fmaf(ps[e], f, o);
-  }
-  a16[(size_t)hq * D + e] = __float2half_rn(o / l);
-}
-
-cudaError_t launch_attn_decode(const float* q_rot, const __half* kc, const __half* vc, float* scratch, __half* a16,
-                               int n_q, int n_kv, int d, int cap, int n_ctx, cudaStream_t st, uint64_t* n_launch) {
-  const int splits = attn_decode_splits(n_ctx), group = n_q / n_kv;
-  const float scale = 1.0f / sqrtf((float)d);
-  dim3 grid(splits, n_kv);
-  if (d == 128) {
-    attn_decode_partial_kernel<128><<<grid, 128, 0, st>>>(q_rot, kc, vc, scratch, group, cap, n_ctx, splits, scale);
-    attn_decode_combine_kernel<128><<<n_q, 128, 0, st>>>(scratch, a16, splits);
-  } else if (d == 64) {
-    attn_decode_partial_kernel<64><<<grid, 128, 0, st>>>(q_rot, kc, vc, scratch, group, cap, n_ctx, splits, scale);
-    attn_decode_combine_kernel<64><<<n_q, 64, 0, st>>>(scratch, a16, splits);
-  } else {
-    return cudaErrorInvalidValue;
-  }
-  *n_launch += 2;
-  return cudaGetLastError();
+cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch) {
+  const int splits = attn_decode_splits(p.pos + 1);
+  p.scale = 1.0f / sqrtf((float)d);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(splits, p.n_kv);
+  cfg.blockDim = dim3(kAttnPos);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ++*n_launch;
+  if (d == 128) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<128>, p);
+  if (d == 64) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<64>, p);
+  return cudaErrorInvalidValue;
 }
 
 // ------------------------------------------------------------------------------------------- router + top-k (a4)

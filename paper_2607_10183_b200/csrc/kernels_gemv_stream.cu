@@ -1,0 +1,443 @@
+// Streaming decode GEMV for one token (sm_100a): the memory-bound hot kernel of the decode path.
+//
+// Structure: persistent CTAs (2 per SM) of 8 consumer warps + 1 producer warp.  The producer streams row tiles of the
+// packed weights (codes and scales, contiguous byte ranges) into a ring of shared-memory stages with 1-D bulk-async
+// copies (TMA) that complete on mbarriers; consumers never touch global memory for weights.  Every lane owns up to two
+// quantization blocks (32 k each) of a k-part of the row and keeps the activation for them in registers for the whole
+// kernel, so a weight byte is read once from shared memory and an activation never again.
+//
+// Arithmetic: the activation block is re-expressed once per CTA as 24-bit block fixed point, x_k = xi_k * 2^-sh with
+// sh chosen from the block's largest exponent (exact for every element within 2^-12 of the block maximum, rounded at
+// 2^-24 of it otherwise, i.e. at the level of one fp32 rounding).  The three byte planes of xi are multiplied with the
+// masked 4-bit codes by dp4a: block dot products are exact integers; one fp32 multiply-add per block applies the
+// scale, and blocks are accumulated in fp32.  sum_k (u_k - 8) x_k = sum_k u_k x_k - 8 sum_k x_k with the second term
+// precomputed per block.  Lane partials are reduced by warp shuffles, k-parts through shared memory, both in fixed order.
+//
+// Optional prologue: RMSNorm of the input row (fp16 or fp32) with an fp16 gain, rounded to fp16 (the operand edge of
+// the numerics contract), computed redundantly by every CTA while its first weight tiles are in flight.
+// All waits on mbarriers are bounded; on expiry the kernel raises a status word and returns.
+#include "ats_internal.h"
+
+namespace ats {
+
+namespace {
+
+constexpr int kStages = 4;
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kRPW = 2;      // rows per consumer warp per tile
+constexpr int kJ = 2;        // quantization blocks per lane per row
+constexpr int kMaxIt = 48;   // tiles whose partial sums are buffered before a flush
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after about a second of SM clocks (the caller then raises the status word and returns).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > 2000000000ll) return false;
+  }
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {
+  int d;
+  asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {
+  int d;
+  asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+__device__ __forceinline__ float silu_mul_f(float g, float u) { return g / (1.0f + expf(-g)) * u; }
+
+// 32 fp16 activations (16 registers of half2, k ascending) -> three byte planes laid out to meet the masked code words.
+// Code word w of a block holds codes k = 8w..8w+7 at nibble positions (0,2,4,6,1,3,5,7); (word & 0x0F0F0F0F) therefore
+// carries k = 8w + {0,4,1,5} in its bytes and ((word >> 4) & 0x0F0F0F0F) carries k = 8w + {2,6,3,7}.
+// planes[p*8 + 2w + h] holds byte p of xi for those four k (h = 0 / 1).  mul = 2^-sh, corr = -8 * sum(xi) * mul.
+__device__ __forceinline__ void quantize_block(const uint32_t (&xh)[16], uint32_t (&planes)[24], float& mul, float& corr) {
+  uint32_t m = 0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) m = __vmaxu2(m, xh[i] & 0x7C007C00u);
+  int E = (int)(max(m & 0xFFFFu, m >> 16) >> 10);
+  E = max(E, 1);
+  const int sh = 37 - E;
+  const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
+  mul = __uint_as_float((uint32_t)(127 - sh) << 23);
+  int xi[32];
+  int sx = 0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    __half2 h;
+    *reinterpret_cast<uint32_t*>(&h) = xh[i];
+    const float2 f = __half22float2(h);
+    xi[2 * i] = __float2int_rn(f.x * up);
+    xi[2 * i + 1] = __float2int_rn(f.y * up);
+    sx += xi[2 * i] + xi[2 * i + 1];
+  }
+  corr = -8.0f * (float)sx * mul;
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    const int* v = xi + 8 * w;
+    // a-side: k = 0,4,1,5 ; b-side: k = 2,6,3,7
+#pragma unroll
+    for (int p = 0; p < 3; ++p) {
+      const uint32_t sel_lo = 0x0040u + 0x0011u * p;  // bytes p of (x, y) -> result bytes 0,1
+      const uint32_t a01 = __byte_perm((uint32_t)v[0], (uint32_t)v[4], sel_lo);
+      const uint32_t a23 = __byte_perm((uint32_t)v[1], (uint32_t)v[5], sel_lo);
+      const uint32_t b01 = __byte_perm((uint32_t)v[2], (uint32_t)v[6], sel_lo);
+      const uint32_t b23 = __byte_perm((uint32_t)v[3], (uint32_t)v[7], sel_lo);
+      planes[p * 8 + 2 * w] = __byte_perm(a01, a23, 0x5410u);
+      planes[p * 8 + 2 * w + 1] = __byte_perm(b01, b23, 0x5410u);
+    }
+  }
+}
+
+struct StreamSeg {
+  const uint8_t* base;
+  int n_rows;
+  int tile0;  // first tile index of the segment
+};
+
+struct StreamParams {
+  StreamSeg seg[3];
+  int n_seg;
+  int n_tiles;
+  int K;
+  int mode;
+  // activation source: x16 (already the operand), or a row to RMS-normalise first
+  const __half* x16;
+  const __half* norm_in16;
+  const float* norm_in32;
+  const __half* gain;
+  float eps;
+  __half* h_out;  // optional copy of the normalised operand (written by CTA 0)
+  float* y32;
+  __half* y16;
+  const float* res32;
+  const __half* res16;
+  int* status;
+};
+
+template <int PARTS, bool SW>
+__global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ uint64_t full[kStages], empty[kStages];
+  __shared__ float part_s[kMaxIt * kConsumerWarps * kRPW];
+  __shared__ float red_s[kConsumerWarps];
+  __shared__ int fail_s;
+  constexpr int ROWS = kConsumerWarps / PARTS * kRPW;  // weight rows per tile
+  constexpr int OUT_ROWS = SW ? ROWS / 2 : ROWS;       // output rows per tile
+  const int K = p.K, nblk = K / 32;
+  const int row_codes = K / 2, row_scales = K / 16;
+  const int stage_bytes = ROWS * (row_codes + row_scales);
+  uint8_t* stages = smem;
+  __half* hs = reinterpret_cast<__half*>(smem + (size_t)kStages * stage_bytes);  // normalised operand (norm prologue only)
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) {
+    fail_s = 0;
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], kConsumerWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const int first = blockIdx.x;
+  const int n_it = first < p.n_tiles ? (p.n_tiles - first + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------------------------ producer: weights do not depend on the
+    // preceding kernel, so their copies start before the grid dependency is resolved.
+    if (lane == 0) {
+      for (int it = 0; it < n_it; ++it) {
+        const int s = it % kStages;
+        if (it >= kStages && !mbar_wait(&empty[s], ((it / kStages) - 1) & 1)) {
+          atomicExch(p.status, 2);
+          break;
+        }
+        if (it == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        const int tile = first + it * gridDim.x;
+        uint8_t* dst = stages + (size_t)s * stage_bytes;
+        mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+        if (SW) {
+          // gate rows land in stage rows [0, ROWS/2), up rows in [ROWS/2, ROWS)
+          const size_t r0 = (size_t)tile * OUT_ROWS;
+          const uint8_t *g = p.seg[0].base, *u = p.seg[1].base;
+          const size_t n = (size_t)p.seg[0].n_rows;
+          bulk_g2s(dst, g + r0 * row_codes, OUT_ROWS * row_codes, &full[s]);
+          bulk_g2s(dst + OUT_ROWS * row_codes, u + r0 * row_codes, OUT_ROWS * row_codes, &full[s]);
+          uint8_t* sd = dst + ROWS * row_codes;
+          bulk_g2s(sd, g + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s]);
+          bulk_g2s(sd + OUT_ROWS * row_scales, u + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s]);
+        } else {
+          int sg = 0;
+          while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
+          const size_t r0 = (size_t)(tile - p.seg[sg].tile0) * ROWS;
+          const uint8_t* b = p.seg[sg].base;
+          bulk_g2s(dst, b + r0 * row_codes, ROWS * row_codes, &full[s]);
+          bulk_g2s(dst + ROWS * row_codes, b + (size_t)p.seg[sg].n_rows * row_codes + r0 * row_scales, ROWS * row_scales, &full[s]);
+        }
+      }
+    }
+    return;
+  }
+
+  // ------------------------------------------------------------------ consumers
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the activation comes from the preceding kernel
+  const int tid = threadIdx.x;                        // 0..255
+  const __half* xsrc = p.x16;
+  if (p.gain) {
+    // RMSNorm prologue: h = rn16(x * g / sqrt(mean(x^2) + eps)), K = hidden
+    float ss = 0.f;
+    for (int i = tid; i < K; i += 256) {
+      const float v = p.norm_in32 ? p.norm_in32[i] : __half2float(p.norm_in16[i]);
+      ss = fmaf(v, v, ss);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) red_s[warp] = ss;
+    consumer_sync();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; ++w) tot += red_s[w];
+    const float inv = 1.0f / sqrtf(tot / (float)K + p.eps);
+    for (int i = tid; i < K; i += 256) {
+      const float v = p.norm_in32 ? p.norm_in32[i] : __half2float(p.norm_in16[i]);
+      const __half h = __float2half_rn(v * __half2float(p.gain[i]) * inv);
+      hs[i] = h;
+      if (p.h_out && blockIdx.x == 0) p.h_out[i] = h;
+    }
+    consumer_sync();
+    xsrc = hs;
+  }
+  const int part = warp % PARTS, rsub = warp / PARTS;
+  const int pblk = (nblk + PARTS - 1) / PARTS;
+  const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
+  uint32_t xr[kJ][24];
+  float xm[kJ], xc[kJ];
+#pragma unroll
+  for (int j = 0; j < kJ; ++j) {
+    const int b = b0 + lane + 32 * j;
+    if (b < b1) {
+      uint32_t xh[16];
+      const uint4* src = reinterpret_cast<const uint4*>(xsrc + (size_t)b * 32);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 v = src[q];
+        xh[4 * q] = v.x;
+        xh[4 * q + 1] = v.y;
+        xh[4 * q + 2] = v.z;
+        xh[4 * q + 3] = v.w;
+      }
+      quantize_block(xh, xr[j], xm[j], xc[j]);
+    } else {
+#pragma unroll
+      for (int q = 0; q < 24; ++q) xr[j][q] = 0;
+      xm[j] = 0.f;
+      xc[j] = 0.f;
+    }
+  }
+
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  bool failed = false;
+  for (int it0 = 0; it0 < n_it; it0 += kMaxIt) {
+    const int it1 = min(n_it, it0 + kMaxIt);
+    for (int it = it0; it < it1; ++it) {
+      const int s = it % kStages;
+      if (!mbar_wait(&full[s], (it / kStages) & 1)) {
+        failed = true;
+        break;
+      }
+      const uint8_t* st = stages + (size_t)s * stage_bytes;
+      float acc[kRPW];
+#pragma unroll
+      for (int r = 0; r < kRPW; ++r) {
+        const int row = r * (ROWS / kRPW) + rsub;  // stage row of this warp's r-th row
+        const uint4* codes = reinterpret_cast<const uint4*>(st + (size_t)row * row_codes);
+        const __half* sc = reinterpret_cast<const __half*>(st + (size_t)ROWS * row_codes + (size_t)row * row_scales);
+        acc[r] = 0.f;
+#pragma unroll
+        for (int j = 0; j < kJ; ++j) {
+          const int b = b0 + lane + 32 * j;
+          if (b < b1) {
+            const uint4 q = codes[b];
+            const float scale = __half2float(sc[b]);
+            const uint32_t ws[4] = {q.x, q.y, q.z, q.w};
+            int d0 = 0, d1 = 0, d2 = 0;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+              const uint32_t lo = ws[w] & 0x0F0F0F0Fu, hi = (ws[w] >> 4) & 0x0F0F0F0Fu;
+              d0 = dp4a_uu(lo, xr[j][2 * w], d0);
+              d0 = dp4a_uu(hi, xr[j][2 * w + 1], d0);
+              d1 = dp4a_uu(lo, xr[j][8 + 2 * w], d1);
+              d1 = dp4a_uu(hi, xr[j][8 + 2 * w + 1], d1);
+              d2 = dp4a_us(lo, xr[j][16 + 2 * w], d2);
+              d2 = dp4a_us(hi, xr[j][16 + 2 * w + 1], d2);
+            }
+            const float dot = fmaf((float)d2, 65536.f, (float)(d1 * 256 + d0));
+            acc[r] = fmaf(scale, fmaf(dot, xm[j], xc[j]), acc[r]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);  // this warp is done reading stage s
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int r = 0; r < kRPW; ++r) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
+      if (lane == 0) {
+#pragma unroll
+        for (int r = 0; r < kRPW; ++r) part_s[((it - it0) * ROWS + r * (ROWS / kRPW) + rsub) * PARTS + part] = acc[r];
+      }
+    }
+    if (failed) fail_s = 1;
+    consumer_sync();
+    if (fail_s) {  // uniform over the consumers: nobody waits at a barrier for a warp that gave up
+      if (tid == 0) atomicExch(p.status, 1);
+      return;
+    }
+    // flush: sum the k-parts (ascending) and run the epilogue
+    const int n_out = (it1 - it0) * OUT_ROWS;
+    for (int i = tid; i < n_out; i += 256) {
+      const int itl = i / OUT_ROWS, j = i % OUT_ROWS;
+      const int tile = first + (it0 + itl) * gridDim.x;
+      float v[2];
+#pragma unroll
+      for (int h = 0; h < (SW ? 2 : 1); ++h) {
+        const float* ps = part_s + ((size_t)itl * ROWS + j + h * OUT_ROWS) * PARTS;
+        float t = 0.f;
+#pragma unroll
+        for (int q = 0; q < PARTS; ++q) t += ps[q];
+        v[h] = t;
+      }
+      if (SW) {
+        p.y16[(size_t)tile * OUT_ROWS + j] = __float2half_rn(silu_mul_f(v[0], v[1]));
+      } else {
+        // output index: rows of the segments lie side by side
+        int sg = 0;
+        while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
+        int row = (tile - p.seg[sg].tile0) * ROWS + j;
+        for (int q = 0; q < sg; ++q) row += p.seg[q].n_rows;
+        switch (p.mode) {
+          case GEMV_OUT_F32: p.y32[row] = v[0]; break;
+          case GEMV_OUT_F16: p.y16[row] = __float2half_rn(v[0]); break;
+          case GEMV_RES16_OUT_F32: p.y32[row] = __half2float(p.res16[row]) + v[0]; break;
+          case GEMV_RES32_OUT_F16: p.y16[row] = __float2half_rn(p.res32[row] + v[0]); break;
+          case GEMV_RES16_OUT_F16: p.y16[row] = __float2half_rn(__half2float(p.res16[row]) + v[0]); break;
+          default: break;
+        }
+      }
+    }
+    consumer_sync();
+  }
+}
+
+int parts_for(int K) { return K <= 2048 ? 1 : K <= 4096 ? 2 : K <= 8192 ? 4 : 8; }
+
+}  // namespace
+
+bool gemv_stream_eligible(const GemvParams& p) {
+  if (p.M != 1 || p.K % 256 != 0 || p.K > 16384) return false;
+  const int parts = parts_for(p.K);
+  const int rows = kConsumerWarps / parts * kRPW;
+  if (p.mode == GEMV_SWIGLU_F16) {
+    if (p.n_seg != 2 || p.seg[0].n_rows != p.seg[1].n_rows || p.seg[0].n_rows % (rows / 2)) return false;
+  } else {
+    for (int s = 0; s < p.n_seg; ++s)
+      if (p.seg[s].n_rows % rows) return false;
+  }
+  if (p.norm_gain && p.K > 8192) return false;
+  return true;
+}
+
+cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch) {
+  const int parts = parts_for(g.K);
+  const int rows = kConsumerWarps / parts * kRPW;
+  const bool sw = g.mode == GEMV_SWIGLU_F16;
+  StreamParams p{};
+  p.n_seg = g.n_seg;
+  int tiles = 0;
+  if (sw) {
+    p.seg[0] = StreamSeg{g.seg[0].base, g.seg[0].n_rows, 0};
+    p.seg[1] = StreamSeg{g.seg[1].base, g.seg[1].n_rows, 0};
+    tiles = g.seg[0].n_rows / (rows / 2);
+  } else {
+    for (int s = 0; s < g.n_seg; ++s) {
+      p.seg[s] = StreamSeg{g.seg[s].base, g.seg[s].n_rows, tiles};
+      tiles += g.seg[s].n_rows / rows;
+    }
+  }
+  p.n_tiles = tiles;
+  p.K = g.K;
+  p.mode = g.mode;
+  p.x16 = g.x;
+  p.norm_in16 = g.norm_x16;
+  p.norm_in32 = g.norm_x32;
+  p.gain = g.norm_gain;
+  p.eps = g.norm_eps;
+  p.h_out = g.norm_out;
+  p.y32 = g.y32;
+  p.y16 = g.y16;
+  p.res32 = g.res32;
+  p.res16 = g.res16;
+  p.status = status;
+  const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
+  const size_t smem = kStages * stage_bytes + (g.norm_gain ? (size_t)g.K * 2 : 0);
+  const int grid = std::max(1, std::min(tiles, 2 * sm_count));
+  void (*kern)(const StreamParams) = nullptr;
+  switch (parts) {
+    case 1: kern = sw ? gemv_stream_kernel<1, true> : gemv_stream_kernel<1, false>; break;
+    case 2: kern = sw ? gemv_stream_kernel<2, true> : gemv_stream_kernel<2, false>; break;
+    case 4: kern = sw ? gemv_stream_kernel<4, true> : gemv_stream_kernel<4, false>; break;
+    default: kern = sw ? gemv_stream_kernel<8, true> : gemv_stream_kernel<8, false>; break;
+  }
+  static bool attr_set[8] = {};
+  const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
+  if (!attr_set[ki]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set[ki] = true;
+  }
+  if (smem > 100 * 1024) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = g.pdl ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ++*n_launch;
+  return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+}  // namespace ats

@@ -36,7 +36,7 @@ def test_struct_layouts_match_header_sizes():
     assert C.sizeof(B.ats_config) == 72
     assert C.sizeof(B.ats_tensor_desc) == 40
     assert C.sizeof(B.ats_layer_desc) == 10 * 4 + 8 * 4 + 12
-    assert C.sizeof(B.ats_stats) == 8 * 8 + 8 + 2 * 4 * B.ATS_STATS_LIST
+    assert C.sizeof(B.ats_stats) == 8 * 8 + 9 * 8 + 8 + 2 * 4 * B.ATS_STATS_LIST
 
 
 def test_host_placement_matches_oracle_vector():
