@@ -233,6 +233,11 @@ int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n);
 int32_t ats_debug_decode_buffer(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, uint32_t M, uint32_t which,
                                 void** out_dev /*HOST*/, uint64_t* out_bytes /*HOST*/);
 
+/* Same for ats_layer_prefill with T tokens: which = 0 h, 1 qkv (fp16 [T][q|k|v]), 2 q_rot, 3 a, 4 o, 5 x1, 6 h2,
+ * 7 gate|up (fp16 [T][2*ffn]), 8 act, 9 d; all fp16. */
+int32_t ats_debug_prefill_buffer(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, uint32_t T, uint32_t which,
+                                 void** out_dev /*HOST*/, uint64_t* out_bytes /*HOST*/);
+
 /* ---- host-only utilities (no context, no GPU needed) ---- */
 
 /* Algorithm 1 on caller-supplied arrays (all HOST): n tensors in execution order with sizes s[i] (units), values r[i],

@@ -30,7 +30,7 @@ EXPORTS = (
     "ats_init", "ats_destroy", "ats_last_error", "ats_register_tensor", "ats_tensor_slice_bytes", "ats_set_placement",
     "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_route_topk", "ats_moe_linear", "ats_layer_decode",
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
-    "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
+    "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
     "ats_host_unpack_q4",
 )
 
@@ -91,6 +91,7 @@ def _load():
         "ats_measure_h2d": (i32, [vp, u64, u32, P(C.c_double)]),
         "ats_debug_fail_copies": (i32, [vp, u32]),
         "ats_debug_decode_buffer": (i32, [vp, P(ats_layer_desc), u32, u32, P(vp), P(u64)]),
+        "ats_debug_prefill_buffer": (i32, [vp, P(ats_layer_desc), u32, u32, P(vp), P(u64)]),
         "ats_host_solve_placement": (i32, [vp, vp, vp, vp, u32, C.c_int64, vp, P(C.c_int64)]),
         "ats_host_repack_q4": (i32, [vp, vp, vp, u32, u32]),
         "ats_host_unpack_q4": (i32, [vp, vp, vp, u32, u32]),
@@ -257,6 +258,13 @@ class Context:
         off = ptr.value - self.arena.data_ptr()
         raw = self.arena[off:off + nb.value].cpu().numpy()
         return raw.view(dtype)
+
+    def debug_prefill_buffer(self, desc, T, which):
+        """fp16 copy of an intermediate of the last ats_layer_prefill call (see ats_debug_prefill_buffer)."""
+        ptr, nb = C.c_void_p(), C.c_uint64()
+        self.check(lib.ats_debug_prefill_buffer(self.h, C.byref(desc), T, which, C.byref(ptr), C.byref(nb)))
+        off = ptr.value - self.arena.data_ptr()
+        return self.arena[off:off + nb.value].cpu().numpy().view(np.float16).reshape(T, -1)
 
     def measure_h2d(self, nbytes, reps=10) -> float:
         v = C.c_double()

@@ -225,6 +225,7 @@ struct GemmParams {
   int ldy;
   void* scratch;
   uint64_t scratch_bytes;
+  int* status;  // device word raised when a bounded wait expires
 };
 uint64_t gemm_scratch_bytes(int T, int n_total, int K);
 cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);

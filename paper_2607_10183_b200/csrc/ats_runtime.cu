@@ -282,6 +282,7 @@ static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
 
 static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
   p.K = (int)ops[0].t->d.k_in;
+  p.status = ctx->dev_status;
   std::string err;
   if (count_streamed(ops, n) <= (int)ctx->cfg.ring_slots || n == 1) {
     ATS_TRY(acquire_ops(ctx, ops, n));
@@ -837,9 +838,10 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M)
   g.y = (__half*)y;
   g.ldy = (int)t->d.n_out;
   g.scratch_bytes = gemm_scratch_bytes((int)M, (int)t->d.n_out, (int)t->d.k_in);
-  if (g.scratch_bytes > align_up(ctx->cfg.workspace_bytes))
-    return fail(ctx, ATS_ERR_NOMEM, "workspace too small for the GEMM: need %llu bytes", (unsigned long long)g.scratch_bytes);
-  g.scratch = ctx->ws;
+  if (g.scratch_bytes + kWsReserved > align_up(ctx->cfg.workspace_bytes))
+    return fail(ctx, ATS_ERR_NOMEM, "workspace too small for the GEMM: need %llu bytes",
+                (unsigned long long)(g.scratch_bytes + kWsReserved));
+  g.scratch = ctx->ws + kWsReserved;
   return run_gemm_group(ctx, &op, 1, g);
 }
 
@@ -1304,6 +1306,29 @@ int32_t ats_debug_decode_buffer(ats_ctx* ctx, const ats_layer_desc* L, uint32_t 
     case 7: *out_dev = w.d32; *out_bytes = P * H * 4; break;
     case 8: *out_dev = w.ids; *out_bytes = P * 4; break;
     case 9: *out_dev = w.gates; *out_bytes = P * 4; break;
+    default: return fail(ctx, ATS_ERR_INVALID, "unknown buffer %u", which);
+  }
+  if (!*out_dev) return fail(ctx, ATS_ERR_INVALID, "buffer %u is not part of this layer", which);
+  return ATS_OK;
+}
+
+int32_t ats_debug_prefill_buffer(ats_ctx* ctx, const ats_layer_desc* L, uint32_t T, uint32_t which, void** out_dev,
+                                 uint64_t* out_bytes) {
+  if (!ctx || !L || !out_dev || !out_bytes || T == 0) return ATS_ERR_INVALID;
+  LayerWs w = layout_prefill(*L, T, ctx->ws, align_up(ctx->cfg.workspace_bytes));
+  if (!w.ok) return fail(ctx, ATS_ERR_NOMEM, "workspace too small");
+  const uint64_t H = L->hidden, qd = (uint64_t)L->n_q_heads * L->head_dim, kvd = (uint64_t)L->n_kv_heads * L->head_dim;
+  switch (which) {
+    case 0: *out_dev = w.h16; *out_bytes = T * H * 2; break;
+    case 1: *out_dev = w.qkv16; *out_bytes = T * (qd + 2 * kvd) * 2; break;
+    case 2: *out_dev = w.qrot16; *out_bytes = T * qd * 2; break;
+    case 3: *out_dev = w.a16; *out_bytes = T * qd * 2; break;
+    case 4: *out_dev = w.o16; *out_bytes = T * H * 2; break;
+    case 5: *out_dev = w.x1_16; *out_bytes = T * H * 2; break;
+    case 6: *out_dev = w.h2_16; *out_bytes = T * H * 2; break;
+    case 7: *out_dev = w.gu16; *out_bytes = (uint64_t)T * 2 * L->ffn * 2; break;
+    case 8: *out_dev = w.act16; *out_bytes = (uint64_t)T * L->ffn * 2; break;
+    case 9: *out_dev = w.d16; *out_bytes = T * H * 2; break;
     default: return fail(ctx, ATS_ERR_INVALID, "unknown buffer %u", which);
   }
   if (!*out_dev) return fail(ctx, ATS_ERR_INVALID, "buffer %u is not part of this layer", which);

@@ -1,9 +1,448 @@
-// placeholder until the tensor-core GEMM lands
+// Dequantize-fused prefill GEMM on the 5th-generation tensor cores (sm_100a): Y[T][N] = X[T][K] * W^T, fp16 operands,
+// fp32 accumulation in tensor memory, fp16 output.
+//
+// One CTA computes a tile of 128 output features x up to 512 tokens over a K range (split-K when the feature tiles do not
+// fill the GPU).  The weight tile is the MMA A operand: four warps read the packed 4-bit codes and fp16 scales straight
+// from global memory (each thread one weight row), expand them to fp16 (w = rn16(scale * code), a single rounding) and
+// store them into shared memory in the canonical K-major 128-byte-swizzle layout the tensor core reads.  The activation
+// tile is the B operand, loaded by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-range rows zero-filled).  A single
+// thread issues tcgen05.mma (M = 128, N = tokens, K = 16 per instruction) into up to two 256-column accumulators in TMEM;
+// tcgen05.commit releases the stage to the producers through an mbarrier.  The four dequantization warps then become the
+// epilogue: tcgen05.ld brings the accumulator rows back (lane = feature, columns = tokens) and writes Y (or an fp32
+// split-K partial that a second kernel sums in split order).
+//
+// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 = weight dequantization, then epilogue.
+// No cluster launch and no multicast.  Every mbarrier wait is bounded; on expiry the CTA raises the status word, skips
+// the rest of its work, frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "ats_internal.h"
+
 namespace ats {
-uint64_t gemm_scratch_bytes(int, int, int) { return 0; }
-cudaError_t launch_gemm(const GemmParams&, cudaStream_t, uint64_t*, std::string* err) {
-  if (err) *err = "prefill GEMM not built";
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr int BM = 128;         // features per tile (MMA M)
+constexpr int BK = 64;          // k per stage: 64 fp16 = one 128-byte swizzle row
+constexpr int TACC = 256;       // tokens per accumulator (MMA N <= 256)
+constexpr int TTILE = 512;      // tokens per CTA (two accumulators = all 512 TMEM columns)
+constexpr int BOXR = 64;        // activation rows per TMA box
+constexpr int kGemmThreads = 192;
+constexpr int A_BYTES = BM * BK * 2;      // 16 KB
+constexpr int B_ACC_BYTES = TACC * BK * 2;  // 32 KB per accumulator
+constexpr int kMaxStages = 4;
+
+struct GemmSeg {
+  const uint8_t* base;
+  int n_rows;
+  int tile0;  // first feature tile of the segment
+  int col0;   // first output column of the segment
+};
+struct GemmKParams {
+  GemmSeg seg[3];
+  int n_seg;
+  int K, T;
+  int total_ksteps, ksteps_per_split, splits;
+  __half* y;
+  int ldy;
+  float* partial;  // [splits][T][ldy] when splits > 1
+  int stages;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait (about a second of SM clocks)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > 2000000000ll) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+// K-major operand tile with 128-byte rows in the 128-byte swizzle: rows at 128 B, groups of 8 rows at 1024 B.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                    // leading byte offset (not used by swizzled K-major layouts)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+  return d;
+}
+// kind::f16, fp16 x fp16 -> fp32, both operands K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, "
+      "%18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+        "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+        "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ __half2 u2h2(uint32_t v) {
+  __half2 h;
+  *reinterpret_cast<uint32_t*>(&h) = v;
+  return h;
+}
+// One code word (8 codes, internal nibble order) times the block scale -> 8 fp16 weights (k ascending) as one 16-byte chunk.
+__device__ __forceinline__ uint4 dequant8(uint32_t w, __half2 s2) {
+  const uint32_t kMagic = 0x64006400u;
+  const __half2 k1032 = u2h2(0x64086408u), k16th = u2h2(0x2C002C00u), kM72 = u2h2(0xD480D480u);
+  const uint32_t w8 = w >> 8;
+  const __half2 c0 = __hmul2(__hsub2(u2h2((w & 0x000F000Fu) | kMagic), k1032), s2);
+  const __half2 c1 = __hmul2(__hfma2(u2h2((w & 0x00F000F0u) | kMagic), k16th, kM72), s2);
+  const __half2 c2 = __hmul2(__hsub2(u2h2((w8 & 0x000F000Fu) | kMagic), k1032), s2);
+  const __half2 c3 = __hmul2(__hfma2(u2h2((w8 & 0x00F000F0u) | kMagic), k16th, kM72), s2);
+  uint4 o;
+  o.x = *reinterpret_cast<const uint32_t*>(&c0);
+  o.y = *reinterpret_cast<const uint32_t*>(&c1);
+  o.z = *reinterpret_cast<const uint32_t*>(&c2);
+  o.w = *reinterpret_cast<const uint32_t*>(&c3);
+  return o;
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const GemmKParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t full_a[kMaxStages], full_b[kMaxStages], empty[kMaxStages], acc_full;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int fail_s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int S = p.stages;
+  // ---- which tile
+  const int tile = blockIdx.x;
+  int sg = 0;
+  while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
+  const int row0 = (tile - p.seg[sg].tile0) * BM;
+  const int n_rows = p.seg[sg].n_rows;
+  const int t0 = blockIdx.y * TTILE;
+  const int Tt = min(TTILE, p.T - t0);
+  const int n_acc = (Tt + TACC - 1) / TACC;
+  const int split = blockIdx.z;
+  const int ks0 = split * p.ksteps_per_split;
+  const int nks = min(p.ksteps_per_split, p.total_ksteps - ks0);
+  const int stage_bytes = A_BYTES + n_acc * B_ACC_BYTES;
+  int nj[2], nmma[2], boxes[2];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    nj[j] = max(0, min(TACC, Tt - TACC * j));
+    nmma[j] = (nj[j] + 15) / 16 * 16;
+    boxes[j] = (nj[j] + BOXR - 1) / BOXR;
+  }
+  if (threadIdx.x == 0) {
+    fail_s = 0;
+    for (int s = 0; s < kMaxStages; ++s) {
+      mbar_init(&full_a[s], 128);
+      mbar_init(&full_b[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(&acc_full, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_s;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations come from the preceding kernel
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (activation tile)
+    if (lane == 0) {
+      uint32_t tx = 0;
+      for (int j = 0; j < n_acc; ++j) tx += (uint32_t)boxes[j] * BOXR * BK * 2;
+      for (int i = 0; i < nks; ++i) {
+        const int s = i % S;
+        if (i >= S && !mbar_wait(&empty[s], ((i / S) - 1) & 1)) {
+          fail_s = 1;
+          break;
+        }
+        uint8_t* bdst = smem + (size_t)s * stage_bytes + A_BYTES;
+        mbar_expect_tx(&full_b[s], tx);
+        for (int j = 0; j < n_acc; ++j)
+          for (int b = 0; b < boxes[j]; ++b)
+            tma_load_2d(bdst + (size_t)j * B_ACC_BYTES + (size_t)b * BOXR * BK * 2, &xmap, (ks0 + i) * BK, t0 + j * TACC + b * BOXR,
+                        &full_b[s]);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issue
+    if (lane == 0) {
+      bool ok = true;
+      for (int i = 0; i < nks && ok; ++i) {
+        const int s = i % S;
+        const uint32_t par = (i / S) & 1;
+        if (!mbar_wait(&full_a[s], par) || !mbar_wait(&full_b[s], par)) {
+          fail_s = 1;
+          ok = false;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint64_t adesc = umma_desc(a_addr);
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk) {
+          for (int j = 0; j < n_acc; ++j) {
+            const uint64_t bdesc = umma_desc(a_addr + A_BYTES + j * B_ACC_BYTES);
+            umma_f16(tmem_base + (uint32_t)(j * TACC), adesc + 2 * kk, bdesc + 2 * kk, umma_idesc(nmma[j]), (i > 0 || kk > 0) ? 1u : 0u);
+          }
+        }
+        umma_commit(&empty[s]);  // arrives when the MMAs reading stage s are done
+      }
+      if (ok) umma_commit(&acc_full);
+    }
+  } else {
+    // ------------------------------------------------------------ weight dequantization (A tile), one row per thread
+    const int r = (warp - 2) * 32 + lane;
+    const int grow = row0 + r;
+    const bool valid = grow < n_rows;
+    const int K = p.K, nblk = K / 32;
+    const uint8_t* crow = p.seg[sg].base + (size_t)(valid ? grow : 0) * (K / 2);
+    const __half* srow = reinterpret_cast<const __half*>(p.seg[sg].base + (size_t)n_rows * (K / 2)) + (size_t)(valid ? grow : 0) * nblk;
+    uint4 q0, q1;
+    uint32_t sc;
+    auto fetch = [&](int ks) {
+      const int kb = ks * 2;  // first block of the k-step
+      q0 = make_uint4(0, 0, 0, 0);
+      q1 = q0;
+      sc = 0;
+      if (valid && kb < nblk) {
+        q0 = __ldg(reinterpret_cast<const uint4*>(crow + (size_t)kb * 16));
+        sc = (uint32_t)__half_as_ushort(srow[kb]);
+        if (kb + 1 < nblk) {
+          q1 = __ldg(reinterpret_cast<const uint4*>(crow + (size_t)(kb + 1) * 16));
+          sc |= (uint32_t)__half_as_ushort(srow[kb + 1]) << 16;
+        }
+      }
+    };
+    if (nks > 0) fetch(ks0);
+    bool ok = true;
+    for (int i = 0; i < nks; ++i) {
+      const int s = i % S;
+      const uint4 c0 = q0, c1 = q1;
+      const uint32_t scw = sc;
+      if (i + 1 < nks) fetch(ks0 + i + 1);  // next k-step's packed weights are in flight while this one is expanded
+      if (i >= S && !mbar_wait(&empty[s], ((i / S) - 1) & 1)) {
+        fail_s = 1;
+        ok = false;
+        break;
+      }
+      uint8_t* arow = smem + (size_t)s * stage_bytes + (size_t)r * 128;
+      const __half2 s0 = __half2half2(__ushort_as_half((unsigned short)(scw & 0xFFFF)));
+      const __half2 s1 = __half2half2(__ushort_as_half((unsigned short)(scw >> 16)));
+      const int sw = r & 7;
+      *reinterpret_cast<uint4*>(arow + ((0 ^ sw) << 4)) = dequant8(c0.x, s0);
+      *reinterpret_cast<uint4*>(arow + ((1 ^ sw) << 4)) = dequant8(c0.y, s0);
+      *reinterpret_cast<uint4*>(arow + ((2 ^ sw) << 4)) = dequant8(c0.z, s0);
+      *reinterpret_cast<uint4*>(arow + ((3 ^ sw) << 4)) = dequant8(c0.w, s0);
+      *reinterpret_cast<uint4*>(arow + ((4 ^ sw) << 4)) = dequant8(c1.x, s1);
+      *reinterpret_cast<uint4*>(arow + ((5 ^ sw) << 4)) = dequant8(c1.y, s1);
+      *reinterpret_cast<uint4*>(arow + ((6 ^ sw) << 4)) = dequant8(c1.z, s1);
+      *reinterpret_cast<uint4*>(arow + ((7 ^ sw) << 4)) = dequant8(c1.w, s1);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core's reads
+      mbar_arrive(&full_a[s]);
+    }
+    // ------------------------------------------------------------ epilogue: accumulator rows -> Y (transposed)
+    if (ok && nks > 0 && mbar_wait(&acc_full, 0)) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int q = warp & 3;               // TMEM lane quarter this warp may read
+      const int f = q * 32 + lane;          // feature row within the tile
+      const bool fvalid = row0 + f < n_rows;
+      const int col = p.seg[sg].col0 + row0 + f;
+      for (int j = 0; j < n_acc; ++j) {
+        for (int c0 = 0; c0 < nmma[j]; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * TACC + c0), v);
+          if (fvalid) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int t = t0 + j * TACC + c0 + e;
+              if (t < p.T) {
+                if (p.splits > 1)
+                  p.partial[((size_t)split * p.T + t) * p.ldy + col] = __uint_as_float(v[e]);
+                else
+                  p.y[(size_t)t * p.ldy + col] = __float2half_rn(__uint_as_float(v[e]));
+              }
+            }
+          }
+        }
+      }
+    } else if (nks > 0) {
+      fail_s = 1;
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (fail_s && threadIdx.x == 0) atomicExch(p.status, 3);
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// y[t][c] = rn16(sum_s partial[s][t][c]) for c < n_cols, splits summed in ascending order
+__global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, __half* __restrict__ y, int T, int n_cols, int ldy,
+                                          int splits) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const size_t total = (size_t)T * n_cols;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t t = i / n_cols, c = i % n_cols;
+    float acc = 0.f;
+    for (int s = 0; s < splits; ++s) acc += partial[((size_t)s * T + t) * ldy + c];
+    y[t * ldy + c] = __float2half_rn(acc);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+int pick_splits(int tiles, int total_ksteps, int sm_count) {
+  int s = 1;
+  while (tiles * s < sm_count && s < 8 && total_ksteps % (s * 2) == 0 && total_ksteps / (s * 2) >= 8) s *= 2;
+  return s;
+}
+
+int feature_tiles(const GemmParams& p) {
+  int tiles = 0;
+  for (int i = 0; i < p.n_seg; ++i) tiles += (p.seg[i].n_rows + BM - 1) / BM;
+  return tiles;
+}
+
+}  // namespace
+
+uint64_t gemm_scratch_bytes(int T, int n_total, int K) {
+  // fp32 partials of the split choice for this shape (fewer tiles can only mean more splits, so the tile count of the
+  // concatenated rows bounds it from above); the launcher falls back to one split if the buffer it gets is smaller
+  const int total_ksteps = (K + BK - 1) / BK;
+  const int tiles = ((n_total + BM - 1) / BM) * ((T + TTILE - 1) / TTILE);
+  const int s = pick_splits(tiles, total_ksteps, 148);
+  return s > 1 ? (uint64_t)s * T * n_total * 4 + 256 : 256;
+}
+
+cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch, std::string* err) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) {
+    if (err) *err = "cuTensorMapEncodeTiled is not available from the driver";
+    return cudaErrorNotSupported;
+  }
+  if (((uintptr_t)g.x & 15) || (g.ldx % 8)) {
+    if (err) *err = "GEMM activations must be 16-byte aligned with a leading dimension that is a multiple of 8";
+    return cudaErrorInvalidValue;
+  }
+  CUtensorMap xmap;
+  const cuuint64_t dims[2] = {(cuuint64_t)g.K, (cuuint64_t)g.T};
+  const cuuint64_t strides[1] = {(cuuint64_t)g.ldx * 2};
+  const cuuint32_t box[2] = {BK, BOXR};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half*>(g.x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+    if (err) *err = "cuTensorMapEncodeTiled failed for the activation tile";
+    return cudaErrorInvalidValue;
+  }
+  GemmKParams p{};
+  p.n_seg = g.n_seg;
+  int tiles = 0, col = 0;
+  for (int i = 0; i < g.n_seg; ++i) {
+    p.seg[i] = GemmSeg{g.seg[i].base, g.seg[i].n_rows, tiles, col};
+    tiles += (g.seg[i].n_rows + BM - 1) / BM;
+    col += g.seg[i].n_rows;
+  }
+  const int tchunks = (g.T + TTILE - 1) / TTILE;
+  p.K = g.K;
+  p.T = g.T;
+  p.total_ksteps = (g.K + BK - 1) / BK;
+  int sm_count = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  p.splits = pick_splits(tiles * tchunks, p.total_ksteps, sm_count);
+  if (p.splits > 1 && (uint64_t)p.splits * g.T * g.ldy * 4 > g.scratch_bytes) p.splits = 1;
+  p.ksteps_per_split = (p.total_ksteps + p.splits - 1) / p.splits;
+  p.y = g.y;
+  p.ldy = g.ldy;
+  p.partial = (float*)g.scratch;
+  p.status = g.status;
+  const int n_acc = std::min(g.T, TTILE) > TACC ? 2 : 1;
+  p.stages = n_acc == 2 ? 2 : 4;
+  const size_t smem = (size_t)p.stages * (A_BYTES + n_acc * B_ACC_BYTES) + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_q4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  dim3 grid(tiles, tchunks, p.splits);
+  gemm_q4_kernel<<<grid, kGemmThreads, smem, st>>>(xmap, p);
+  ++*n_launch;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (p.splits > 1) {
+    const size_t total = (size_t)g.T * col;
+    const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)sm_count * 8);
+    gemm_splitk_reduce_kernel<<<blocks, 256, 0, st>>>(p.partial, g.y, g.T, col, g.ldy, p.splits);
+    ++*n_launch;
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
 }  // namespace ats

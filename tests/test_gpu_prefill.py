@@ -1,0 +1,205 @@
+"""GPU parity of the prefill path (dequantize-fused tensor-core GEMM, causal attention, layer) against the CPU oracle."""
+import numpy as np
+import pytest
+
+from oracle import ats_oracle as O
+from paper_2607_10183_b200 import workloads as W
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+MB = 1 << 20
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2607_10183_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    return torch
+
+
+def gemm_ctx(B, N, K, T, where, extra=0):
+    nb = W.q4_bytes(N, K)
+    ws = 8 * T * N * 4 + 2 * MB
+    arena = ws + 2 * (nb + 256) + nb + MB + extra
+    ctx = B.Context(arena, workspace_bytes=ws, ring_slots=2, slot_bytes=nb, chunk_bytes=MB)
+    return ctx
+
+
+@pytest.mark.parametrize("N,K,T", [(128, 64, 16), (128, 256, 9), (136, 320, 127), (256, 512, 128), (384, 1024, 129), (130, 96, 300),
+                                   (512, 2048, 512), (256, 4096, 600), (1024, 14336, 33)])
+def test_linear_gemm_matches_oracle(B, torch, N, K, T):
+    """M > 8 takes the tensor-core GEMM: fp16 operands (weights rounded once), fp32 accumulation, fp16 output.
+    Shapes cover ragged feature tiles, ragged token tiles, split-K and K that is not a multiple of the 64-wide stage."""
+    packed, scales = W.q4_packed(99, 0, W.ROLE_Q, N, K)
+    x = W.activations(99, 0, (T, K))
+    want16 = O.linear(x, packed, scales, O.WEIGHT_F16, round_out=True)
+    want_exact = O.linear(x, packed, scales, O.WEIGHT_EXACT, round_out=True)
+    outs = []
+    for where in (B.ATS_GPU, B.ATS_HOST):
+        ctx = gemm_ctx(B, N, K, T, where)
+        tid = ctx.register_q4(packed, scales)
+        ctx.set_placement([(tid, -1, where)])
+        y = torch.full((T, N), 7.0, dtype=torch.float16, device="cuda")
+        ctx.linear(tid, H.to_dev(x), y, T)
+        ctx.sync()
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want16, what=f"gemm {N}x{K} T={T} vs fp16-weight oracle")
+        H.assert_close(outs[-1], want_exact, what=f"gemm {N}x{K} T={T} vs exact-weight oracle")
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+
+
+def test_gemm_rows_equal_gemv_within_tolerance_and_one_hot(B, torch):
+    """Row m of the GEMM agrees with the GEMV of row m; one-hot activations return the fp16-rounded weight column."""
+    N, K, T = 256, 512, 64
+    packed, scales = W.q4_packed(99, 1, W.ROLE_Q, N, K)
+    ctx = gemm_ctx(B, N, K, T, 1)
+    tid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(tid, -1, B.ATS_GPU)])
+    x = W.activations(99, 1, (T, K))
+    yg = torch.empty((T, N), dtype=torch.float16, device="cuda")
+    ctx.linear(tid, H.to_dev(x), yg, T)
+    yv = torch.empty((4, N), dtype=torch.float16, device="cuda")
+    ctx.linear(tid, H.to_dev(x[10:14]), yv, 4)
+    ctx.sync()
+    H.assert_close(yg.cpu().numpy()[10:14], yv.cpu().numpy().astype(np.float64), what="gemm row vs gemv")
+    eye = np.zeros((T, K), dtype=np.float16)
+    ks = [0, 1, 7, 8, 31, 32, 63, 64, 65, 255, 256, 511]
+    for i, k in enumerate(ks):
+        eye[i, k] = 1
+    ctx.linear(tid, H.to_dev(eye), yg, T)
+    ctx.sync()
+    w16 = O.dequantize(packed, scales, O.WEIGHT_F16).astype(np.float16)
+    got = yg.cpu().numpy()
+    for i, k in enumerate(ks):
+        assert H.bits_equal_mod_zero_sign(got[i], w16[:, k]), k
+    assert not got[len(ks):].any()
+    ctx.close()
+
+
+def prefill_ctx(B, shape, cap, T, placement, ring_slots=2):
+    L = None
+    slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=cap)
+    ws = B.workspace_bytes(probe, T) + MB
+    arena = ws + ring_slots * (slot + 256) + H.dense_layer_bytes(shape) + MB
+    return B.Context(arena, workspace_bytes=ws, ring_slots=ring_slots, slot_bytes=slot, chunk_bytes=4 * MB)
+
+
+def run_prefill(B, torch, shape, cfg, pos0, T, cap, placement):
+    L = W.dense_layer(cfg, 0, shape)
+    ctx = prefill_ctx(B, shape, cap, T, placement)
+    desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+    ctx.set_placement([(ids[n], -1, w) for n, w in placement.items()])
+    kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos0)
+    kd, vd = H.to_dev(kc), H.to_dev(vc)
+    x = W.activations(cfg, 0, (T, shape.hidden))
+    y = torch.empty((T, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.reset_stats()
+    ctx.layer_prefill(desc, H.to_dev(x), y, kd, vd, pos0, T)
+    ctx.sync()
+    out = (y.cpu().numpy(), kd.cpu().numpy(), vd.cpu().numpy(), ctx.stats(), ctx.numerics(B.ATS_MODE_PREFILL), L, x, kc, vc)
+    ctx.close()
+    return out
+
+
+ALL_GPU = {n: 1 for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")}
+
+
+@pytest.mark.parametrize("shape_name,pos0,T,cap", [("small", 0, 7, 16), ("small", 5, 40, 64), ("small", 0, 130, 130), ("full", 0, 512, 512)])
+def test_dense_layer_prefill_matches_oracle(B, torch, shape_name, pos0, T, cap):
+    shape = W.DENSE_SMALL if shape_name == "small" else W.DENSE_FULL
+    cfg = 96 if shape_name == "small" else 3
+    y, kg, vg, st, (edges, wmode), L, x, kc, vc = run_prefill(B, torch, shape, cfg, pos0, T, cap, ALL_GPU)
+    assert wmode == O.WEIGHT_F16 and edges == frozenset(O.EDGES)
+    want = O.dense_layer(x, H.oracle_dense_tensors(L), shape, kc, vc, pos0, edges, wmode)
+    H.assert_close(y, want, what="prefill layer output", elementwise=(shape_name == "small"))
+    for got, ref in ((kg, kc), (vg, vc)):
+        a = got[:, pos0:pos0 + T].astype(np.float64)
+        b = ref[:, pos0:pos0 + T].astype(np.float64)
+        assert np.array_equal(got[:, :pos0], ref[:, :pos0]) and np.array_equal(got[:, pos0 + T:], ref[:, pos0 + T:])
+        # written rows: fp16 values of an fp16 GEMM output, so at most a few ulps off the oracle's
+        assert np.max(np.abs(a - b)) <= 4e-3 * np.max(np.abs(b))
+
+
+def test_prefill_placement_invariance(B, torch):
+    shape, cfg = W.DENSE_SMALL, 96
+    base = run_prefill(B, torch, shape, cfg, 3, 40, 64, ALL_GPU)
+    hyb = run_prefill(B, torch, shape, cfg, 3, 40, 64, {**ALL_GPU, "wk": 0, "wo": 0, "w_gate": 0, "w_up": 0})
+    assert np.array_equal(base[0].view(np.uint16), hyb[0].view(np.uint16))
+    assert np.array_equal(base[1], hyb[1]) and np.array_equal(base[2], hyb[2])
+    nbytes = {n: W.q4_bytes(r, k) for (role, r, k), n in zip(shape.tensor_shapes(), ALL_GPU)}
+    assert hyb[3].streamed_bytes == sum(nbytes[n] for n in ("wk", "wo", "w_gate", "w_up"))
+
+
+def test_prefill_then_decode_continues_the_cache(B, torch):
+    """A prefill of T tokens followed by a decode step equals (within tolerance) the oracle doing the same, which pins
+    that both calls agree on cache layout and positions."""
+    shape, cfg, T, cap = W.DENSE_SMALL, 96, 24, 32
+    L = W.dense_layer(cfg, 0, shape)
+    ctx = prefill_ctx(B, shape, cap, T, ALL_GPU)
+    desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+    ctx.set_placement([(ids[n], -1, 1) for n in ALL_GPU])
+    kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, 0)
+    kd, vd = H.to_dev(kc), H.to_dev(vc)
+    x = W.activations(cfg, 0, (T, shape.hidden))
+    y = torch.empty((T, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.layer_prefill(desc, H.to_dev(x), y, kd, vd, 0, T)
+    x1 = W.activations(cfg, 0, (1, shape.hidden), step=7)
+    y1 = torch.empty((1, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.layer_decode(desc, H.to_dev(x1), y1, kd, vd, T, 1)
+    ctx.sync()
+    t = H.oracle_dense_tensors(L)
+    O.dense_layer(x, t, shape, kc, vc, 0, frozenset(O.EDGES), O.WEIGHT_F16)
+    e, w = ctx.numerics(B.ATS_MODE_DECODE)
+    want = O.dense_layer(x1, t, shape, kc, vc, T, e, w)
+    H.assert_close(y1.cpu().numpy(), want, what="decode after prefill")
+    ctx.close()
+
+
+def test_prefill_layer_stage_by_stage_full_size(B, torch):
+    """Config 3 (512 tokens through the full-size layer), every kernel on its own: each stage's output is compared with the
+    oracle's definition of that stage applied to the inputs the stage actually consumed, under both error gates."""
+    shape, cfg, T, cap = W.DENSE_FULL, 3, 512, 512
+    L = W.dense_layer(cfg, 0, shape)
+    t = H.oracle_dense_tensors(L)
+    ctx = prefill_ctx(B, shape, cap, T, ALL_GPU)
+    desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+    ctx.set_placement([(ids[n], -1, 1) for n in ALL_GPU])
+    kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, 0)
+    kd, vd = H.to_dev(kc), H.to_dev(vc)
+    x = W.activations(cfg, 0, (T, shape.hidden))
+    y = torch.empty((T, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.layer_prefill(desc, H.to_dev(x), y, kd, vd, 0, T)
+    ctx.sync()
+    g = {n: ctx.debug_prefill_buffer(desc, T, i).astype(np.float64)
+         for i, n in enumerate(("h", "qkv", "q_rot", "a", "o", "x1", "h2", "gu", "act", "d"))}
+    yg, kg, vg = y.cpu().numpy(), kd.cpu().numpy(), vd.cpu().numpy()
+    ctx.close()
+    nq, nkv, d, ffn = shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn
+    qd, kvd = nq * d, nkv * d
+    F16 = O.WEIGHT_F16
+    H.assert_close(g["h"], O.rn16(O.rmsnorm(x, t["attn_norm"], shape.rms_eps)), what="h")
+    for name, lo, hi in (("wq", 0, qd), ("wk", qd, qd + kvd), ("wv", qd + kvd, qd + 2 * kvd)):
+        H.assert_close(g["qkv"][:, lo:hi], O.linear(g["h"], *t[name], F16, round_out=True), what=name)
+    pos = np.arange(T, dtype=np.float64).reshape(T, 1)
+    H.assert_close(g["q_rot"], O.rn16(O.rope(g["qkv"][:, :qd].reshape(T, nq, d), pos, shape.rope_theta)).reshape(T, -1), what="q_rot")
+    k_rot = O.rn16(O.rope(g["qkv"][:, qd:qd + kvd].reshape(T, nkv, d), pos, shape.rope_theta))
+    H.assert_close(kg.transpose(1, 0, 2).reshape(T, -1), k_rot.reshape(T, -1), what="k cache")
+    assert np.array_equal(vg.transpose(1, 0, 2).reshape(T, -1).astype(np.float64), g["qkv"][:, qd + kvd:])
+    a = np.stack([O.attention_one(g["q_rot"][i].reshape(nq, d), kg, vg, i + 1).reshape(-1) for i in range(T)])
+    H.assert_close(g["a"], O.rn16(a), what="attention")
+    H.assert_close(g["o"], O.linear(g["a"], *t["wo"], F16, round_out=True), what="wo")
+    assert np.array_equal(g["x1"], O.rn16(x.astype(np.float64) + g["o"]))
+    H.assert_close(g["h2"], O.rn16(O.rmsnorm(g["x1"], t["ffn_norm"], shape.rms_eps)), what="h2")
+    H.assert_close(g["gu"][:, :ffn], O.linear(g["h2"], *t["w_gate"], F16, round_out=True), what="w_gate")
+    H.assert_close(g["gu"][:, ffn:], O.linear(g["h2"], *t["w_up"], F16, round_out=True), what="w_up")
+    H.assert_close(g["act"], O.rn16(O.silu(g["gu"][:, :ffn]) * g["gu"][:, ffn:]), what="swiglu")
+    H.assert_close(g["d"], O.linear(g["act"], *t["w_down"], F16, round_out=True), what="w_down")
+    assert np.array_equal(yg.astype(np.float64), O.rn16(g["x1"] + g["d"]))
