@@ -230,7 +230,126 @@ def extra_gemv(torch, B, W, peaks, quick):
             "gbs_kernel": kernel, "frac_of_measured_hbm": kernel / peaks["hbm_gbs"], "frac_of_nominal_8TBs": kernel / 8000.0}
 
 
-EXTRAS = {"cfg1_gemv": extra_gemv}
+def extra_prefill(torch, B, W, peaks, quick):
+    """Config 3: 512 prompt tokens through one dense layer (seven projections as dequantize-fused tcgen05 GEMMs)."""
+    shape, T, cap = W.DENSE_FULL, 512, 512
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=cap)
+    R = 2
+    ctx, descs, q4_ids, layer_bytes = build_dense_replicas(B, W, R, 3, cap, extra_ws=B.workspace_bytes(probe, T))
+    ctx.set_placement([(i, -1, B.ATS_GPU) for i in q4_ids])
+    x = torch.from_numpy(W.activations(3, 0, (T, shape.hidden))).cuda()
+    y = torch.empty_like(x)
+    kc = torch.zeros((shape.n_kv_heads, cap, shape.head_dim), dtype=torch.float16, device="cuda")
+    vc = torch.zeros_like(kc)
+    n = 6 if quick else 20
+
+    def go(k):
+        for i in range(k):
+            ctx.layer_prefill(descs[i % R], x, y, kc, vc, 0, T)
+    go(3)
+    ms = event_time_ms(torch, ctx.compute, lambda: go(n)) / n
+    ctx.set_flags(B.ATS_FLAG_TIME_KERNELS)
+    ctx.reset_stats()
+    go(4)
+    ctx.sync()
+    st = ctx.stats()
+    ctx.close()
+    flops = sum(2.0 * T * nn * kk for _, nn, kk in shape.tensor_shapes())
+    gemm_ms = st.timed_ms[2] / 4
+    tf = st.timed_work[2] / (st.timed_ms[2] * 1e-3) / 1e12
+    return {"workload": "config 3: dense layer prefill, 512 tokens, all resident", "layer_ms": ms, "prefill_tokens_per_s": T / (ms * 1e-3),
+            "gemm_flop_per_layer": flops, "gemm_ms_per_layer": gemm_ms, "gemm_tflops": tf,
+            "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"], "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": tf / 2250.0, "non_gemm_ms_per_layer": ms - gemm_ms}
+
+
+def extra_moe(torch, B, W, peaks, quick):
+    """Config 4: MoE FFN block (hidden 2048, 128 experts x SwiGLU 768, top-8), batch 1 and 8; all resident, and with the
+    odd experts in pinned host memory and streamed when selected."""
+    shape = W.MOE_FULL
+    Bk = W.moe_block(4, 0, shape)
+    sl = W.q4_bytes(shape.ffn, shape.hidden)
+    out = {"workload": "config 4: MoE block decode; hybrid = odd experts host-placed", "expert_slice_bytes": sl}
+    for hybrid in (False, True):
+        ctx = B.Context(3 * shape.n_experts * (sl + 256) + 64 * (sl + 256) + (16 << 20), workspace_bytes=8 << 20, ring_slots=64,
+                        slot_bytes=sl, chunk_bytes=sl)
+        ids = {"ffn_norm": ctx.register_f16(Bk[W.ROLE_FFN_NORM]), "router": ctx.register_f16(Bk[W.ROLE_ROUTER])}
+        for name, r in (("w_gate", W.ROLE_GATE), ("w_up", W.ROLE_UP), ("w_down", W.ROLE_DOWN)):
+            ids[name] = ctx.register_q4(*Bk[r], role=r)
+        desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, rms_eps=shape.rms_eps, **ids)
+        ctx.set_placement([(ids[n], e, B.ATS_HOST if (hybrid and e % 2) else B.ATS_GPU) for n in ("w_gate", "w_up", "w_down")
+                           for e in range(shape.n_experts)])
+        if hybrid:
+            out["pcie_h2d_measured_gbs"] = ctx.measure_h2d(64 * sl, 10)
+        for M in (1, 8):
+            xs = [torch.from_numpy(W.activations(4, 0, (M, shape.hidden), step=s)).cuda() for s in range(16)]
+            y = torch.empty((M, shape.hidden), dtype=torch.float16, device="cuda")
+            n = 64 if quick else 256
+
+            def go(k):
+                for i in range(k):
+                    ctx.layer_decode(desc, xs[i % 16], y, None, None, 0, M)
+            go(16)
+            ctx.sync()
+            ctx.reset_stats()
+            t0 = time.perf_counter()
+            go(n)
+            ctx.sync()
+            dt = (time.perf_counter() - t0) / n
+            st = ctx.stats()
+            key = f"{'hybrid' if hybrid else 'resident'}_M{M}"
+            out[key] = {"us_per_call": dt * 1e6, "tokens_per_s": M / dt, "streamed_bytes_per_call": st.streamed_bytes / n,
+                        "launches_per_call": st.kernel_launches / n}
+            if hybrid and st.streamed_bytes:
+                out[key]["pcie_gbs_over_call_time"] = st.streamed_bytes / n / dt / 1e9
+        ctx.close()
+    return out
+
+
+def extra_stream(torch, B, W, peaks, quick, n_layers=None):
+    """Config 5: a stack of dense layers under a 60 % byte budget chosen by the library's placement DP (Algorithm 1);
+    the rest sits in pinned host memory and is streamed every decode step, overlapped with compute."""
+    shape = W.DENSE_FULL
+    L = n_layers or (4 if quick else 8)
+    cap, pos0 = 640, 512
+    slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+    ctx, descs, q4_ids, layer_bytes = build_dense_replicas(B, W, L, 5, cap, ring_slots=8, slot_bytes=slot, chunk_bytes=8 << 20)
+    total = L * layer_bytes
+    where = ctx.plan_placement(int(0.60 * total), len(q4_ids))
+    pcie = ctx.measure_h2d(8 * slot, 5)
+    st0 = ctx.stats()
+    caches = [(torch.zeros((shape.n_kv_heads, cap, shape.head_dim), dtype=torch.float16, device="cuda"),
+               torch.zeros((shape.n_kv_heads, cap, shape.head_dim), dtype=torch.float16, device="cuda")) for _ in range(L)]
+    xa = torch.from_numpy(W.activations(5, 0, (1, shape.hidden))).cuda()
+    xb = torch.empty_like(xa)
+
+    def step(pos):
+        src, dst = xa, xb
+        for l in range(L):
+            ctx.layer_decode(descs[l], src, dst, caches[l][0], caches[l][1], pos, 1)
+            src, dst = dst, src
+    for s in range(3):
+        step(pos0 + s)
+    ctx.sync()
+    ctx.reset_stats()
+    n = 8 if quick else 24
+    t0 = time.perf_counter()
+    for s in range(n):
+        step(pos0 + 3 + s)
+    ctx.sync()
+    dt = (time.perf_counter() - t0) / n
+    st = ctx.stats()
+    streamed = st.streamed_bytes / n
+    ctx.close()
+    return {"workload": f"config 5 shape: {L}-layer dense stack, 60 % byte budget via ats_plan_placement, decode steps at positions {pos0 + 3}+",
+            "layers": L, "total_weight_bytes": total, "resident_bytes": int(st0.resident_bytes), "resident_frac": st0.resident_bytes / total,
+            "gpu_tensors": int(where.sum()), "host_tensors": int(len(where) - where.sum()), "streamed_bytes_per_step": streamed,
+            "ms_per_step": dt * 1e3, "decode_tokens_per_s": 1.0 / dt, "pcie_gbs_streamed": streamed / dt / 1e9, "pcie_h2d_measured_gbs": pcie,
+            "frac_of_measured_pcie": streamed / dt / 1e9 / pcie, "fully_overlapped_at_80pct": bool(dt <= streamed / (0.8 * pcie * 1e9))}
+
+
+EXTRAS = {"cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
 
 
 def run_ours(args):
@@ -371,9 +490,17 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the figures of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--quick", action="store_true", help="smaller extras")
+    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream"],
+                    help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.only_extra:
+        import torch
+        from paper_2607_10183_b200 import binding as B, workloads as W
+        torch.cuda.set_device(0)
+        print(json.dumps({args.only_extra: EXTRAS[args.only_extra](torch, B, W, load_peaks(), True)}))
+        return
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

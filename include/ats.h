@@ -59,7 +59,10 @@ enum {
   ATS_FLAG_POISON_SLOTS = 1u,     /* debug: fill a ring slot with 0xFF after its consumer, so premature reuse shows */
   ATS_FLAG_SKIP_SCALE_CHECK = 2u, /* do not scan scales for Inf/NaN at registration */
   ATS_FLAG_TIME_KERNELS = 4u,     /* bracket every GEMV / grouped GEMV / GEMM launch with CUDA events (see ats_stats.timed_*) */
-  ATS_FLAG_NO_PDL = 8u            /* launch every kernel fully serialized (no programmatic dependent launch overlap) */
+  ATS_FLAG_NO_PDL = 8u,           /* launch every kernel fully serialized (no programmatic dependent launch overlap) */
+  /* timing experiments only: do not launch a stage of ats_layer_decode (its outputs are then stale); bit 24 = QKV GEMV,
+   * 25 = attention, 26 = O GEMV, 27 = gate/up GEMV, 28 = down GEMV */
+  ATS_FLAG_DEBUG_SKIP_SHIFT = 24
 };
 /* ats_layer_desc.flags */
 enum { ATS_LAYER_NO_TOPK_RENORM = 1u /* gates = full softmax entries instead of softmax over the top-k */ };

@@ -940,6 +940,8 @@ static int32_t check_layer(ats_ctx* ctx, const ats_layer_desc* L, bool prefill) 
     ATS_TRY(check_q4(ctx, L->wv, kvd, L->hidden, 1, "wv"));
     ATS_TRY(check_q4(ctx, L->wo, L->hidden, qd, 1, "wo"));
     if (L->kv_capacity == 0) return fail(ctx, ATS_ERR_SHAPE, "kv_capacity is 0");
+    if (!prefill && (L->kv_capacity > 131072 || L->n_q_heads > 192))
+      return fail(ctx, ATS_ERR_UNSUPPORTED, "decode attention supports kv_capacity <= 131072 and <= 192 query heads");
   }
   ATS_TRY(check_f16(ctx, L->ffn_norm, L->hidden, 1, "ffn_norm"));
   const uint32_t E = L->n_experts ? L->n_experts : 1;
@@ -1008,7 +1010,8 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     p.y32 = w.qkv32;
     p.ldy = qd + 2 * kvd;
     p.mode = GEMV_OUT_F32;
-    ATS_TRY(run_gemv_group(ctx, qkv, 3, p));
+    const uint32_t skip = ctx->cfg.flags >> ATS_FLAG_DEBUG_SKIP_SHIFT;
+    if (!(skip & 1)) ATS_TRY(run_gemv_group(ctx, qkv, 3, p));
     AttnDecodeParams ap{};
     ap.qkv = w.qkv32;
     ap.q_rot_out = w.qrot32;
@@ -1023,7 +1026,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     ap.cap = (int)L->kv_capacity;
     ap.pos = (int)pos;
     rope_table(ctx, L->rope_theta, d, (int)pos, ap.cs);
-    ATS_CUDA(launch_attn_decode_fused(ap, d, pdl, ctx->cs, nl));
+    if (!(skip & 2)) ATS_CUDA(launch_attn_decode_fused(ap, d, pdl, ctx->cs, nl));
     GemvParams o{};
     o.M = (int)M;
     o.x = w.a16;
@@ -1033,7 +1036,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     o.res16 = (const __half*)x_in;
     o.ldres = H;
     o.mode = GEMV_RES16_OUT_F32;
-    ATS_TRY(run_gemv_group(ctx, &wo, 1, o));
+    if (!(skip & 4)) ATS_TRY(run_gemv_group(ctx, &wo, 1, o));
   }
   if (L->n_experts != 0)  // the MoE path needs the normalised row in memory (router and grouped GEMV read it)
     ATS_CUDA(launch_rmsnorm(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev,
@@ -1051,7 +1054,8 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     g.mode = GEMV_SWIGLU_F16;
     if (count_streamed(gu, 2) > (int)ctx->cfg.ring_slots)
       return fail(ctx, ATS_ERR_BUDGET, "fused gate/up needs 2 ring slots when both tensors are host-placed");
-    ATS_TRY(run_gemv_group(ctx, gu, 2, g));
+    const uint32_t skip2 = ctx->cfg.flags >> ATS_FLAG_DEBUG_SKIP_SHIFT;
+    if (!(skip2 & 8)) ATS_TRY(run_gemv_group(ctx, gu, 2, g));
     GemvParams dn{};
     dn.M = (int)M;
     dn.x = w.act16;
@@ -1066,6 +1070,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
       dn.res16 = (const __half*)x_in;
       dn.mode = GEMV_RES16_OUT_F16;
     }
+    if (skip2 & 16) return ATS_OK;
     return run_gemv_group(ctx, &wd, 1, dn);
   }
   // ---- MoE FFN

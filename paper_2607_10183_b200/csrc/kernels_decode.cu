@@ -410,191 +410,246 @@ cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __ha
 // cos/sin table for `pos` computed on the host in fp64 and passed by value), appends the new K/V row to the caches as
 // fp16, attends over positions 0..pos split across CTAs, and merges the splits: the last CTA to finish a kv head
 // (a counter in global memory, reset for the next launch) sums the partials in ascending split order, so the result
-// does not depend on which CTA arrives last.  CTA (split, kv head) covers 64 positions, one per lane of its 2 warps,
-// for all query heads of the group.
-constexpr int kAttnPos = 64;
+// does not depend on which CTA arrives last.  CTA (split, kv head) covers 256 positions, one per lane of its 8 warps,
+// for all query heads of the group.  The kernel is a short chain of memory round trips, so every phase issues all of
+// its loads before it uses any of them.
+constexpr int kAttnPos = 256;
 constexpr int kAttnMaxGroup = 8;
+constexpr int kAttnMaxSplits = 512;  // 131072 cached positions
 
 int attn_decode_splits(int n_ctx) { return (n_ctx + kAttnPos - 1) / kAttnPos; }
 size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) { return (size_t)n_q * attn_decode_splits(n_ctx) * (d + 2); }
 
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+
 template <int D>
 __global__ void __launch_bounds__(kAttnPos) attn_decode_fused_kernel(const AttnDecodeParams p) {
-  constexpr int V = D / 32;  // output dims per lane
+  constexpr int V = D / 32;            // output dims per lane
   constexpr int NW = kAttnPos / 32;
-  __shared__ float q_s[kAttnMaxGroup * D];
-  __shared__ float w_m[NW][kAttnMaxGroup], w_l[NW][kAttnMaxGroup];
-  __shared__ float w_acc[NW][kAttnMaxGroup][D];
+  constexpr int CH = D * 2 / 16;       // 16-byte chunks per key row
+  constexpr int KROW = D * 2 + 16;     // key row pitch in shared memory: the 16-byte pad makes lane-per-row reads conflict-free
+  extern __shared__ __align__(16) uint8_t k_s[];  // [kAttnPos][KROW]
+  __shared__ __align__(16) float q_s[D];
+  __shared__ float w_m[NW], w_l[NW];
+  __shared__ float w_acc[NW][D];
+  __shared__ float f_s[2 * kAttnMaxSplits + 1];
   __shared__ int is_last;
-  const int split = blockIdx.x, kvh = blockIdx.y, n_splits = gridDim.x;
+  const int split = blockIdx.x, hq = blockIdx.y, n_splits = gridDim.x;
+  const int kvh = hq / p.group;
+  const bool writer = hq % p.group == 0;  // one CTA per kv head writes the new cache rows
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int group = p.group, half = D / 2, n_ctx = p.pos + 1;
+  const int half = D / 2, n_ctx = p.pos + 1;
   const int qd = p.n_q * D, kvd = p.n_kv * D;
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v come from the preceding kernel
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // rotary embedding of the group's query heads into shared memory
-  for (int idx = threadIdx.x; idx < group * half; idx += blockDim.x) {
-    const int g = idx / half, i = idx % half;
-    const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
-    const float* q = p.qkv + (size_t)(kvh * group + g) * D;
-    const float a = q[i], b = q[i + half];
-    const float ra = a * c - b * s, rb = b * c + a * s;
-    q_s[g * D + i] = ra;
-    q_s[g * D + i + half] = rb;
-    if (p.q_rot_out && split == 0) {
-      p.q_rot_out[(size_t)(kvh * group + g) * D + i] = ra;
-      p.q_rot_out[(size_t)(kvh * group + g) * D + i + half] = rb;
+  const int tc0 = split * kAttnPos;                     // first position of the CTA
+  const int rows_here = min(kAttnPos, n_ctx - tc0);     // >= 1
+  const bool own = split == p.pos / kAttnPos;           // this CTA holds the new token's position
+  const int r_new = p.pos - tc0;
+  // The cache rows of past tokens do not depend on the preceding kernel: stage the keys (coalesced 16-byte async copies
+  // into padded rows) and fetch this lane's value slices before waiting for it.
+  for (int c = threadIdx.x; c < rows_here * CH; c += kAttnPos) {
+    const int row = c / CH, ch = c % CH;
+    if (!(own && row == r_new))
+      cp_async16(k_s + (size_t)row * KROW + ch * 16, p.kc + ((size_t)kvh * p.cap + tc0 + row) * D + ch * 8);
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  const int t0 = tc0 + warp * 32;
+  const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
+  uint2 vraw[32];
+#pragma unroll
+  for (int tt = 0; tt < 32; ++tt) {
+    vraw[tt] = make_uint2(0u, 0u);
+    if (tt < n_here && t0 + tt != p.pos) {
+      const __half* vr = p.vc + ((size_t)kvh * p.cap + t0 + tt) * D + lane * V;
+      if (V == 4)
+        vraw[tt] = __ldg(reinterpret_cast<const uint2*>(vr));
+      else
+        vraw[tt].x = __ldg(reinterpret_cast<const uint32_t*>(vr));
     }
   }
-  // the CTA that owns position `pos` appends the new key (rotated) and value rows first
-  if (split == p.pos / kAttnPos) {
-    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v of the new token come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // rotary embedding of this query head into shared memory
+  if (threadIdx.x < half) {
+    const int i = threadIdx.x;
+    const float* q = p.qkv + (size_t)hq * D;
+    const float a = q[i], b = q[i + half];
+    const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
+    const float ra = a * c - b * s, rb = b * c + a * s;
+    q_s[i] = ra;
+    q_s[i + half] = rb;
+    if (p.q_rot_out && split == 0) {
+      p.q_rot_out[(size_t)hq * D + i] = ra;
+      p.q_rot_out[(size_t)hq * D + i + half] = rb;
+    }
+  }
+  // the CTAs that cover position `pos` rotate the new key and put its fp16 value into their staged tile; one of them
+  // per kv head also appends key and value rows to the caches
+  if (own) {
+    if (threadIdx.x >= kAttnPos - half) {
+      const int i = threadIdx.x - (kAttnPos - half);
       const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
       const float* k = p.qkv + qd + (size_t)kvh * D;
       const float a = k[i], b = k[i + half];
-      __half* dst = p.kc + ((size_t)kvh * p.cap + p.pos) * D;
-      dst[i] = __float2half_rn(a * c - b * s);
-      dst[i + half] = __float2half_rn(b * c + a * s);
+      const __half ka = __float2half_rn(a * c - b * s), kb = __float2half_rn(b * c + a * s);
+      __half* srow = reinterpret_cast<__half*>(k_s + (size_t)r_new * KROW);
+      srow[i] = ka;
+      srow[i + half] = kb;
+      if (writer) {
+        __half* dst = p.kc + ((size_t)kvh * p.cap + p.pos) * D;
+        dst[i] = ka;
+        dst[i + half] = kb;
+      }
     }
-    for (int e = threadIdx.x; e < D; e += blockDim.x)
-      p.vc[((size_t)kvh * p.cap + p.pos) * D + e] = __float2half_rn(p.qkv[qd + kvd + (size_t)kvh * D + e]);
+    if (writer && threadIdx.x < D)
+      p.vc[((size_t)kvh * p.cap + p.pos) * D + threadIdx.x] = __float2half_rn(p.qkv[qd + kvd + (size_t)kvh * D + threadIdx.x]);
+    if (p.pos >= t0 && p.pos < t0 + 32) {  // the warp whose lanes cover `pos`: its value slice, rounded as the cache holds it
+      const float* vn = p.qkv + qd + kvd + (size_t)kvh * D + lane * V;
+      __half2 h01 = __floats2half2_rn(vn[0], vn[1]);
+      uint2 r = make_uint2(*reinterpret_cast<uint32_t*>(&h01), 0u);
+      if (V == 4) {
+        __half2 h23 = __floats2half2_rn(vn[2], vn[3]);
+        r.y = *reinterpret_cast<uint32_t*>(&h23);
+      }
+#pragma unroll
+      for (int tt = 0; tt < 32; ++tt)
+        if (t0 + tt == p.pos) vraw[tt] = r;
+    }
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
-  const int t0 = split * kAttnPos + warp * 32;
   const int t = t0 + lane;
   const bool ok = t < n_ctx;
-  float sc[kAttnMaxGroup];
-#pragma unroll
-  for (int g = 0; g < kAttnMaxGroup; ++g) sc[g] = 0.f;
+  float sc = 0.f;
   if (ok) {
-    const uint4* kr = reinterpret_cast<const uint4*>(p.kc + ((size_t)kvh * p.cap + t) * D);
-    uint4 kv[D / 8];
+    const uint4* kr = reinterpret_cast<const uint4*>(k_s + (size_t)(warp * 32 + lane) * KROW);
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int c = 0; c < D / 8; ++c) kv[c] = kr[c];  // plain loads: the row at `pos` was written by this CTA
-#pragma unroll
-    for (int c = 0; c < D / 8; ++c) {
-      float kf[8];
+    for (int c = 0; c < CH; ++c) {
+      const uint4 kv = kr[c];
+      const float4 q0 = *reinterpret_cast<const float4*>(q_s + c * 8);
+      const float4 q1 = *reinterpret_cast<const float4*>(q_s + c * 8 + 4);
       float2 f;
-      f = __half22float2(u32_as_half2(kv[c].x)); kf[0] = f.x; kf[1] = f.y;
-      f = __half22float2(u32_as_half2(kv[c].y)); kf[2] = f.x; kf[3] = f.y;
-      f = __half22float2(u32_as_half2(kv[c].z)); kf[4] = f.x; kf[5] = f.y;
-      f = __half22float2(u32_as_half2(kv[c].w)); kf[6] = f.x; kf[7] = f.y;
-#pragma unroll
-      for (int g = 0; g < kAttnMaxGroup; ++g) {
-        if (g < group) {
-          const float4 q0 = *reinterpret_cast<const float4*>(q_s + g * D + c * 8);
-          const float4 q1 = *reinterpret_cast<const float4*>(q_s + g * D + c * 8 + 4);
-          sc[g] = fmaf(kf[0], q0.x, sc[g]); sc[g] = fmaf(kf[1], q0.y, sc[g]);
-          sc[g] = fmaf(kf[2], q0.z, sc[g]); sc[g] = fmaf(kf[3], q0.w, sc[g]);
-          sc[g] = fmaf(kf[4], q1.x, sc[g]); sc[g] = fmaf(kf[5], q1.y, sc[g]);
-          sc[g] = fmaf(kf[6], q1.z, sc[g]); sc[g] = fmaf(kf[7], q1.w, sc[g]);
-        }
-      }
+      f = __half22float2(u32_as_half2(kv.x)); s0 = fmaf(f.x, q0.x, s0); s1 = fmaf(f.y, q0.y, s1);
+      f = __half22float2(u32_as_half2(kv.y)); s0 = fmaf(f.x, q0.z, s0); s1 = fmaf(f.y, q0.w, s1);
+      f = __half22float2(u32_as_half2(kv.z)); s0 = fmaf(f.x, q1.x, s0); s1 = fmaf(f.y, q1.y, s1);
+      f = __half22float2(u32_as_half2(kv.w)); s0 = fmaf(f.x, q1.z, s0); s1 = fmaf(f.y, q1.w, s1);
     }
+    sc = s0 + s1;
   }
-  float pr[kAttnMaxGroup];
-#pragma unroll
-  for (int g = 0; g < kAttnMaxGroup; ++g) {
-    pr[g] = 0.f;
-    if (g < group) {
-      const float s = ok ? sc[g] * p.scale : -INFINITY;
-      const float m = warp_max(s);
-      pr[g] = (ok && m > -INFINITY) ? expf(s - m) : 0.f;
-      const float l = warp_sum(pr[g]);
-      if (lane == 0) {
-        w_m[warp][g] = m;
-        w_l[warp][g] = l;
-      }
-    }
+  const float sv = ok ? sc * p.scale : -INFINITY;
+  const float mw = warp_max(sv);
+  const float pr = (ok && mw > -INFINITY) ? expf(sv - mw) : 0.f;
+  const float lw = warp_sum(pr);
+  if (lane == 0) {
+    w_m[warp] = mw;
+    w_l[warp] = lw;
   }
-  float acc[kAttnMaxGroup][V];
+  float acc[V];
 #pragma unroll
-  for (int g = 0; g < kAttnMaxGroup; ++g)
+  for (int v = 0; v < V; ++v) acc[v] = 0.f;
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[g][v] = 0.f;
-  const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
-#pragma unroll 8
-  for (int tt = 0; tt < n_here; ++tt) {
-    const __half* vr = p.vc + ((size_t)kvh * p.cap + t0 + tt) * D + lane * V;
-    float vf[V];
+  for (int tt = 0; tt < 32; ++tt) {
+    const float pt = __shfl_sync(0xffffffffu, pr, tt);  // zero for positions beyond n_ctx
+    float2 f;
+    f = __half22float2(u32_as_half2(vraw[tt].x));
+    acc[0] = fmaf(pt, f.x, acc[0]);
+    acc[1] = fmaf(pt, f.y, acc[1]);
     if (V == 4) {
-      const uint2 raw = *reinterpret_cast<const uint2*>(vr);
-      float2 f;
-      f = __half22float2(u32_as_half2(raw.x)); vf[0] = f.x; vf[1] = f.y;
-      f = __half22float2(u32_as_half2(raw.y)); vf[2] = f.x; vf[3] = f.y;
-    } else {
-      const float2 f = __half22float2(u32_as_half2(*reinterpret_cast<const uint32_t*>(vr)));
-      vf[0] = f.x;
-      vf[1] = f.y;
-    }
-#pragma unroll
-    for (int g = 0; g < kAttnMaxGroup; ++g) {
-      if (g < group) {
-        const float pt = __shfl_sync(0xffffffffu, pr[g], tt);
-#pragma unroll
-        for (int v = 0; v < V; ++v) acc[g][v] = fmaf(pt, vf[v], acc[g][v]);
-      }
+      f = __half22float2(u32_as_half2(vraw[tt].y));
+      acc[2] = fmaf(pt, f.x, acc[2]);
+      acc[3] = fmaf(pt, f.y, acc[3]);
     }
   }
 #pragma unroll
-  for (int g = 0; g < kAttnMaxGroup; ++g)
-    if (g < group)
-#pragma unroll
-      for (int v = 0; v < V; ++v) w_acc[warp][g][lane * V + v] = acc[g][v];
+  for (int v = 0; v < V; ++v) w_acc[warp][lane * V + v] = acc[v];
   __syncthreads();
-  // merge the warps (ascending) into this split's partial for each head of the group
-  for (int idx = threadIdx.x; idx < group * D; idx += blockDim.x) {
-    const int g = idx / D, e = idx % D;
+  // merge the warps (ascending) into this split's partial
+  float* part = p.part + ((size_t)hq * n_splits + split) * (D + 2);
+  if (threadIdx.x < D) {
+    const int e = threadIdx.x;
     float mx = -INFINITY;
-    for (int w = 0; w < NW; ++w) mx = fmaxf(mx, w_m[w][g]);
+#pragma unroll
+    for (int w = 0; w < NW; ++w) mx = fmaxf(mx, w_m[w]);
     float l = 0.f, o = 0.f;
+#pragma unroll
     for (int w = 0; w < NW; ++w) {
-      const float f = w_m[w][g] > -INFINITY ? expf(w_m[w][g] - mx) : 0.f;
-      l = fmaf(w_l[w][g], f, l);
-      o = fmaf(w_acc[w][g][e], f, o);
+      const float f = w_m[w] > -INFINITY ? expf(w_m[w] - mx) : 0.f;
+      l = fmaf(w_l[w], f, l);
+      o = fmaf(w_acc[w][e], f, o);
     }
-    float* dst = p.part + ((size_t)(kvh * group + g) * n_splits + split) * (D + 2);
-    dst[e] = o;
+    part[e] = o;
     if (e == 0) {
-      dst[D] = mx;
-      dst[D + 1] = l;
+      part[D] = mx;
+      part[D + 1] = l;
     }
   }
-  // last CTA of this kv head merges the splits
+  // the last CTA of this head merges the splits
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int prev = atomicAdd(p.counters + kvh, 1);
+    const int prev = atomicAdd(p.counters + hq, 1);
     is_last = prev == n_splits - 1;
-    if (is_last) p.counters[kvh] = 0;  // ready for the next launch
+    if (is_last) p.counters[hq] = 0;  // ready for the next launch
   }
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  for (int idx = threadIdx.x; idx < group * D; idx += blockDim.x) {
-    const int g = idx / D, e = idx % D;
-    const float* base = p.part + (size_t)(kvh * group + g) * n_splits * (D + 2);
+  const float* base = p.part + (size_t)hq * n_splits * (D + 2);
+  for (int i = threadIdx.x; i < 2 * n_splits; i += kAttnPos)  // all maxima and sums at once: one round trip
+    f_s[i] = __ldcg(base + (size_t)(i >> 1) * (D + 2) + D + (i & 1));
+  // this thread's output element for every split, in flight before the weights are known
+  float pv[kAttnMaxSplits / (kAttnPos / D) > 0 ? 1 : 1];
+  (void)pv;
+  const int e = threadIdx.x % D, sub = threadIdx.x / D;  // kAttnPos / D threads share an element and take alternate splits
+  constexpr int SUBS = kAttnPos / D;
+  float o = 0.f;
+  __syncthreads();
+  if (threadIdx.x == 0) {
     float mx = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, __ldcg(base + (size_t)s * (D + 2) + D));
-    float l = 0.f, o = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-      const float* ps = base + (size_t)s * (D + 2);
-      const float m = __ldcg(ps + D);
+    for (int s2 = 0; s2 < n_splits; ++s2) mx = fmaxf(mx, f_s[2 * s2]);
+    float l = 0.f;
+    for (int s2 = 0; s2 < n_splits; ++s2) {
+      const float m = f_s[2 * s2];
       const float f = m > -INFINITY ? expf(m - mx) : 0.f;
-      l = fmaf(__ldcg(ps + D + 1), f, l);
-      o = fmaf(__ldcg(ps + e), f, o);
+      l = fmaf(f_s[2 * s2 + 1], f, l);
+      f_s[2 * s2] = f;
     }
-    p.a16[(size_t)(kvh * group + g) * D + e] = __float2half_rn(o / l);
+    f_s[2 * n_splits] = 1.0f / l;
+  }
+  __syncthreads();
+  (void)sub;
+  (void)SUBS;
+  if (threadIdx.x < D) {
+    for (int s0 = 0; s0 < n_splits; s0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = (s0 + u < n_splits) ? __ldcg(base + (size_t)(s0 + u) * (D + 2) + e) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (s0 + u < n_splits) o = fmaf(v[u], f_s[2 * (s0 + u)], o);
+    }
+    p.a16[(size_t)hq * D + e] = __float2half_rn(o * f_s[2 * n_splits]);
   }
 }
 
 cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch) {
   const int splits = attn_decode_splits(p.pos + 1);
+  if (splits > kAttnMaxSplits) return cudaErrorInvalidValue;
   p.scale = 1.0f / sqrtf((float)d);
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(splits, p.n_kv);
+  cfg.gridDim = dim3(splits, p.n_q);
   cfg.blockDim = dim3(kAttnPos);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = (size_t)kAttnPos * (d * 2 + 16);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e1 = cudaFuncSetAttribute(attn_decode_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnPos * (128 * 2 + 16));
+    cudaError_t e2 = cudaFuncSetAttribute(attn_decode_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnPos * (64 * 2 + 16));
+    if (e1 != cudaSuccess) return e1;
+    if (e2 != cudaSuccess) return e2;
+    attr_set = true;
+  }
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

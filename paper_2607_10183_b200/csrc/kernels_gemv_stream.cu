@@ -182,7 +182,12 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
           atomicExch(p.status, 2);
           break;
         }
-        if (it == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        if (it == kStages) {
+          // The first stages are in flight.  Dependents may only be released once this grid's own dependency is
+          // resolved, so that a dependent's prologue never overlaps anything older than this kernel.
+          asm volatile("griddepcontrol.wait;" ::: "memory");
+          asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        }
         const int tile = first + it * gridDim.x;
         uint8_t* dst = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
@@ -214,11 +219,45 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
   const int tid = threadIdx.x;                        // 0..255
   const __half* xsrc = p.x16;
   if (p.gain) {
-    // RMSNorm prologue: h = rn16(x * g / sqrt(mean(x^2) + eps)), K = hidden
+    // RMSNorm prologue: h = rn16(x * g / sqrt(mean(x^2) + eps)), K = hidden.  Each thread owns runs of 8 consecutive
+    // elements (run r = tid + 256 j), loaded once with 128-bit loads and kept in registers for the second pass.
+    constexpr int kRuns = 4;  // K <= 8192
+    float xv[kRuns][8], gv[kRuns][8];
     float ss = 0.f;
-    for (int i = tid; i < K; i += 256) {
-      const float v = p.norm_in32 ? p.norm_in32[i] : __half2float(p.norm_in16[i]);
-      ss = fmaf(v, v, ss);
+#pragma unroll
+    for (int j = 0; j < kRuns; ++j) {
+      const int i0 = (tid + 256 * j) * 8;
+      if (i0 < K) {
+        if (p.norm_in32) {
+          const float4 a = *reinterpret_cast<const float4*>(p.norm_in32 + i0);
+          const float4 b = *reinterpret_cast<const float4*>(p.norm_in32 + i0 + 4);
+          xv[j][0] = a.x; xv[j][1] = a.y; xv[j][2] = a.z; xv[j][3] = a.w;
+          xv[j][4] = b.x; xv[j][5] = b.y; xv[j][6] = b.z; xv[j][7] = b.w;
+        } else {
+          const uint4 a = *reinterpret_cast<const uint4*>(p.norm_in16 + i0);
+          const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            __half2 h2;
+            *reinterpret_cast<uint32_t*>(&h2) = w[q];
+            const float2 f = __half22float2(h2);
+            xv[j][2 * q] = f.x;
+            xv[j][2 * q + 1] = f.y;
+          }
+        }
+        const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(p.gain + i0));
+        const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          __half2 h2;
+          *reinterpret_cast<uint32_t*>(&h2) = gw[q];
+          const float2 f = __half22float2(h2);
+          gv[j][2 * q] = f.x;
+          gv[j][2 * q + 1] = f.y;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) ss = fmaf(xv[j][q], xv[j][q], ss);
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -228,11 +267,20 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
 #pragma unroll
     for (int w = 0; w < kConsumerWarps; ++w) tot += red_s[w];
     const float inv = 1.0f / sqrtf(tot / (float)K + p.eps);
-    for (int i = tid; i < K; i += 256) {
-      const float v = p.norm_in32 ? p.norm_in32[i] : __half2float(p.norm_in16[i]);
-      const __half h = __float2half_rn(v * __half2float(p.gain[i]) * inv);
-      hs[i] = h;
-      if (p.h_out && blockIdx.x == 0) p.h_out[i] = h;
+#pragma unroll
+    for (int j = 0; j < kRuns; ++j) {
+      const int i0 = (tid + 256 * j) * 8;
+      if (i0 < K) {
+        uint32_t o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const __half2 h2 = __floats2half2_rn(xv[j][2 * q] * gv[j][2 * q] * inv, xv[j][2 * q + 1] * gv[j][2 * q + 1] * inv);
+          o[q] = *reinterpret_cast<const uint32_t*>(&h2);
+        }
+        const uint4 ov = make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(hs + i0) = ov;
+        if (p.h_out && blockIdx.x == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = ov;
+      }
     }
     consumer_sync();
     xsrc = hs;
@@ -242,11 +290,13 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
   const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
   uint32_t xr[kJ][24];
   float xm[kJ], xc[kJ];
-#pragma unroll
-  for (int j = 0; j < kJ; ++j) {
-    const int b = b0 + lane + 32 * j;
-    if (b < b1) {
-      uint32_t xh[16];
+  if (PARTS <= 2) {
+    // Warps that share a k-part need the same activation blocks: quantize every block once per CTA into shared memory
+    // (28 words per block: 24 plane words, mul, corr; the 112-byte pitch keeps the 128-bit reads conflict-free).
+    uint32_t* xq_s = reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes + (p.gain ? (size_t)K * 2 : 0));
+    for (int b = tid; b < nblk; b += 256) {
+      uint32_t xh[16], pl[24];
+      float mul, corr;
       const uint4* src = reinterpret_cast<const uint4*>(xsrc + (size_t)b * 32);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -256,12 +306,58 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
         xh[4 * q + 2] = v.z;
         xh[4 * q + 3] = v.w;
       }
-      quantize_block(xh, xr[j], xm[j], xc[j]);
-    } else {
+      quantize_block(xh, pl, mul, corr);
+      uint4* dst = reinterpret_cast<uint4*>(xq_s + (size_t)b * 28);
 #pragma unroll
-      for (int q = 0; q < 24; ++q) xr[j][q] = 0;
-      xm[j] = 0.f;
-      xc[j] = 0.f;
+      for (int q = 0; q < 6; ++q) dst[q] = make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
+      *reinterpret_cast<float2*>(xq_s + (size_t)b * 28 + 24) = make_float2(mul, corr);
+    }
+    consumer_sync();
+#pragma unroll
+    for (int j = 0; j < kJ; ++j) {
+      const int b = b0 + lane + 32 * j;
+      if (b < b1) {
+        const uint4* src = reinterpret_cast<const uint4*>(xq_s + (size_t)b * 28);
+#pragma unroll
+        for (int q = 0; q < 6; ++q) {
+          const uint4 v = src[q];
+          xr[j][4 * q] = v.x;
+          xr[j][4 * q + 1] = v.y;
+          xr[j][4 * q + 2] = v.z;
+          xr[j][4 * q + 3] = v.w;
+        }
+        const float2 mc = *reinterpret_cast<const float2*>(xq_s + (size_t)b * 28 + 24);
+        xm[j] = mc.x;
+        xc[j] = mc.y;
+      } else {
+#pragma unroll
+        for (int q = 0; q < 24; ++q) xr[j][q] = 0;
+        xm[j] = 0.f;
+        xc[j] = 0.f;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < kJ; ++j) {
+      const int b = b0 + lane + 32 * j;
+      if (b < b1) {
+        uint32_t xh[16];
+        const uint4* src = reinterpret_cast<const uint4*>(xsrc + (size_t)b * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint4 v = src[q];
+          xh[4 * q] = v.x;
+          xh[4 * q + 1] = v.y;
+          xh[4 * q + 2] = v.z;
+          xh[4 * q + 3] = v.w;
+        }
+        quantize_block(xh, xr[j], xm[j], xc[j]);
+      } else {
+#pragma unroll
+        for (int q = 0; q < 24; ++q) xr[j][q] = 0;
+        xm[j] = 0.f;
+        xc[j] = 0.f;
+      }
     }
   }
 
@@ -409,7 +505,7 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   p.res16 = g.res16;
   p.status = status;
   const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (g.norm_gain ? (size_t)g.K * 2 : 0);
+  const size_t smem = kStages * stage_bytes + (g.norm_gain ? (size_t)g.K * 2 : 0) + (parts <= 2 ? (size_t)(g.K / 32) * 112 : 0);
   const int grid = std::max(1, std::min(tiles, 2 * sm_count));
   void (*kern)(const StreamParams) = nullptr;
   switch (parts) {
