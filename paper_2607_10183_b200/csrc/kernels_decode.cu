@@ -410,9 +410,10 @@ cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __ha
 // cos/sin table for `pos` computed on the host in fp64 and passed by value), appends the new K/V row to the caches as
 // fp16, attends over positions 0..pos split across CTAs, and merges the splits: the last CTA to finish a kv head
 // (a counter in global memory, reset for the next launch) sums the partials in ascending split order, so the result
-// does not depend on which CTA arrives last.  CTA (split, kv head) covers 256 positions, one per lane of its 8 warps,
-// for all query heads of the group.  The kernel is a short chain of memory round trips, so every phase issues all of
-// its loads before it uses any of them.
+// does not depend on which CTA arrives last.  CTA (split, query head) covers 256 positions, one per lane of its 8
+// warps (the heads of a group re-read the same K/V rows from L2).  The kernel is a short chain of memory round trips,
+// so every phase issues all of its loads before it uses any of them: key rows are staged with 16-byte async copies
+// into padded shared-memory rows and the value slices are fetched into registers before the grid dependency resolves.
 constexpr int kAttnPos = 256;
 constexpr int kAttnMaxGroup = 8;
 constexpr int kAttnMaxSplits = 512;  // 131072 cached positions
@@ -599,11 +600,7 @@ __global__ void __launch_bounds__(kAttnPos) attn_decode_fused_kernel(const AttnD
   const float* base = p.part + (size_t)hq * n_splits * (D + 2);
   for (int i = threadIdx.x; i < 2 * n_splits; i += kAttnPos)  // all maxima and sums at once: one round trip
     f_s[i] = __ldcg(base + (size_t)(i >> 1) * (D + 2) + D + (i & 1));
-  // this thread's output element for every split, in flight before the weights are known
-  float pv[kAttnMaxSplits / (kAttnPos / D) > 0 ? 1 : 1];
-  (void)pv;
-  const int e = threadIdx.x % D, sub = threadIdx.x / D;  // kAttnPos / D threads share an element and take alternate splits
-  constexpr int SUBS = kAttnPos / D;
+  const int e = threadIdx.x % D;
   float o = 0.f;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -619,8 +616,6 @@ __global__ void __launch_bounds__(kAttnPos) attn_decode_fused_kernel(const AttnD
     f_s[2 * n_splits] = 1.0f / l;
   }
   __syncthreads();
-  (void)sub;
-  (void)SUBS;
   if (threadIdx.x < D) {
     for (int s0 = 0; s0 < n_splits; s0 += 8) {
       float v[8];

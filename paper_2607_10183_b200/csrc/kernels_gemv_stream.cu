@@ -119,6 +119,41 @@ __device__ __forceinline__ void quantize_block(const uint32_t (&xh)[16], uint32_
   }
 }
 
+// The same quantization done by four adjacent lanes, each holding one run of 8 consecutive elements (one code word's
+// worth) of a 32-element block: exponent maximum and integer sum are shared by two butterfly shuffles.  Lane w of the
+// group writes plane words 2w, 2w+1 of every plane into blk[28] (24 plane words, then mul, corr).
+__device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32_t* blk) {
+  uint32_t m = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m = max(m, (__float_as_uint(x[i]) >> 23) & 0xFFu);  // fp32 exponent field of an fp16-valued number
+  m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
+  // fp16 exponent field E = fp32 field - 112 (normals); subnormal fp16 values have fp32 fields <= 112 -> E = 1
+  const int E = max((int)m - 112, 1);
+  const int sh = 37 - E;
+  const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
+  const float mul = __uint_as_float((uint32_t)(127 - sh) << 23);
+  int xi[8];
+  int sx = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    xi[i] = __float2int_rn(x[i] * up);
+    sx += xi[i];
+  }
+  sx += __shfl_xor_sync(0xffffffffu, sx, 1);
+  sx += __shfl_xor_sync(0xffffffffu, sx, 2);
+#pragma unroll
+  for (int p = 0; p < 3; ++p) {
+    const uint32_t sel_lo = 0x0040u + 0x0011u * p;
+    const uint32_t a01 = __byte_perm((uint32_t)xi[0], (uint32_t)xi[4], sel_lo);
+    const uint32_t a23 = __byte_perm((uint32_t)xi[1], (uint32_t)xi[5], sel_lo);
+    const uint32_t b01 = __byte_perm((uint32_t)xi[2], (uint32_t)xi[6], sel_lo);
+    const uint32_t b23 = __byte_perm((uint32_t)xi[3], (uint32_t)xi[7], sel_lo);
+    *reinterpret_cast<uint2*>(blk + p * 8 + 2 * w) = make_uint2(__byte_perm(a01, a23, 0x5410u), __byte_perm(b01, b23, 0x5410u));
+  }
+  if (w == 0) *reinterpret_cast<float2*>(blk + 24) = make_float2(mul, -8.0f * (float)sx * mul);
+}
+
 struct StreamSeg {
   const uint8_t* base;
   int n_rows;
@@ -158,7 +193,6 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
   const int row_codes = K / 2, row_scales = K / 16;
   const int stage_bytes = ROWS * (row_codes + row_scales);
   uint8_t* stages = smem;
-  __half* hs = reinterpret_cast<__half*>(smem + (size_t)kStages * stage_bytes);  // normalised operand (norm prologue only)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) {
     fail_s = 0;
@@ -217,100 +251,94 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
   // ------------------------------------------------------------------ consumers
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the activation comes from the preceding kernel
   const int tid = threadIdx.x;                        // 0..255
-  const __half* xsrc = p.x16;
-  if (p.gain) {
-    // RMSNorm prologue: h = rn16(x * g / sqrt(mean(x^2) + eps)), K = hidden.  Each thread owns runs of 8 consecutive
-    // elements (run r = tid + 256 j), loaded once with 128-bit loads and kept in registers for the second pass.
-    constexpr int kRuns = 4;  // K <= 8192
-    float xv[kRuns][8], gv[kRuns][8];
-    float ss = 0.f;
-#pragma unroll
-    for (int j = 0; j < kRuns; ++j) {
-      const int i0 = (tid + 256 * j) * 8;
-      if (i0 < K) {
-        if (p.norm_in32) {
-          const float4 a = *reinterpret_cast<const float4*>(p.norm_in32 + i0);
-          const float4 b = *reinterpret_cast<const float4*>(p.norm_in32 + i0 + 4);
-          xv[j][0] = a.x; xv[j][1] = a.y; xv[j][2] = a.z; xv[j][3] = a.w;
-          xv[j][4] = b.x; xv[j][5] = b.y; xv[j][6] = b.z; xv[j][7] = b.w;
-        } else {
-          const uint4 a = *reinterpret_cast<const uint4*>(p.norm_in16 + i0);
-          const uint32_t w[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            __half2 h2;
-            *reinterpret_cast<uint32_t*>(&h2) = w[q];
-            const float2 f = __half22float2(h2);
-            xv[j][2 * q] = f.x;
-            xv[j][2 * q + 1] = f.y;
-          }
-        }
-        const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(p.gain + i0));
-        const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          __half2 h2;
-          *reinterpret_cast<uint32_t*>(&h2) = gw[q];
-          const float2 f = __half22float2(h2);
-          gv[j][2 * q] = f.x;
-          gv[j][2 * q + 1] = f.y;
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) ss = fmaf(xv[j][q], xv[j][q], ss);
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    if (lane == 0) red_s[warp] = ss;
-    consumer_sync();
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < kConsumerWarps; ++w) tot += red_s[w];
-    const float inv = 1.0f / sqrtf(tot / (float)K + p.eps);
-#pragma unroll
-    for (int j = 0; j < kRuns; ++j) {
-      const int i0 = (tid + 256 * j) * 8;
-      if (i0 < K) {
-        uint32_t o[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const __half2 h2 = __floats2half2_rn(xv[j][2 * q] * gv[j][2 * q] * inv, xv[j][2 * q + 1] * gv[j][2 * q + 1] * inv);
-          o[q] = *reinterpret_cast<const uint32_t*>(&h2);
-        }
-        const uint4 ov = make_uint4(o[0], o[1], o[2], o[3]);
-        *reinterpret_cast<uint4*>(hs + i0) = ov;
-        if (p.h_out && blockIdx.x == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = ov;
-      }
-    }
-    consumer_sync();
-    xsrc = hs;
-  }
   const int part = warp % PARTS, rsub = warp / PARTS;
   const int pblk = (nblk + PARTS - 1) / PARTS;
   const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
   uint32_t xr[kJ][24];
   float xm[kJ], xc[kJ];
   if (PARTS <= 2) {
-    // Warps that share a k-part need the same activation blocks: quantize every block once per CTA into shared memory
-    // (28 words per block: 24 plane words, mul, corr; the 112-byte pitch keeps the 128-bit reads conflict-free).
-    uint32_t* xq_s = reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes + (p.gain ? (size_t)K * 2 : 0));
-    for (int b = tid; b < nblk; b += 256) {
-      uint32_t xh[16], pl[24];
-      float mul, corr;
-      const uint4* src = reinterpret_cast<const uint4*>(xsrc + (size_t)b * 32);
+    // K <= 4096.  Thread t owns the runs of 8 consecutive elements r = t + 256 j; four adjacent lanes hold one block.
+    // Optional RMSNorm (h = rn16(x * g / sqrt(mean(x^2) + eps))) and the block quantization both work on those
+    // registers; the quantized blocks go to shared memory once per CTA (28 words per block; the 112-byte pitch keeps
+    // the 128-bit reads conflict-free) and every lane then fetches the blocks of its k-part.
+    constexpr int kRuns = 2;
+    uint32_t* xq_s = reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes);
+    float xv[kRuns][8];
+    float ss = 0.f;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint4 v = src[q];
-        xh[4 * q] = v.x;
-        xh[4 * q + 1] = v.y;
-        xh[4 * q + 2] = v.z;
-        xh[4 * q + 3] = v.w;
+    for (int j = 0; j < kRuns; ++j) {
+      const int i0 = (tid + 256 * j) * 8;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) xv[j][q] = 0.f;
+      if (i0 < K) {
+        if (p.gain && p.norm_in32) {
+          const float4 a = *reinterpret_cast<const float4*>(p.norm_in32 + i0);
+          const float4 b = *reinterpret_cast<const float4*>(p.norm_in32 + i0 + 4);
+          xv[j][0] = a.x; xv[j][1] = a.y; xv[j][2] = a.z; xv[j][3] = a.w;
+          xv[j][4] = b.x; xv[j][5] = b.y; xv[j][6] = b.z; xv[j][7] = b.w;
+        } else {
+          const uint4 a = *reinterpret_cast<const uint4*>((p.gain ? p.norm_in16 : p.x16) + i0);
+          const uint32_t w4[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            __half2 h2;
+            *reinterpret_cast<uint32_t*>(&h2) = w4[q];
+            const float2 f = __half22float2(h2);
+            xv[j][2 * q] = f.x;
+            xv[j][2 * q + 1] = f.y;
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) ss = fmaf(xv[j][q], xv[j][q], ss);
       }
-      quantize_block(xh, pl, mul, corr);
-      uint4* dst = reinterpret_cast<uint4*>(xq_s + (size_t)b * 28);
+    }
+    if (p.gain) {
+      float gv[kRuns][8];
 #pragma unroll
-      for (int q = 0; q < 6; ++q) dst[q] = make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
-      *reinterpret_cast<float2*>(xq_s + (size_t)b * 28 + 24) = make_float2(mul, corr);
+      for (int j = 0; j < kRuns; ++j) {
+        const int i0 = (tid + 256 * j) * 8;
+        if (i0 < K) {
+          const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(p.gain + i0));
+          const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            __half2 h2;
+            *reinterpret_cast<uint32_t*>(&h2) = gw[q];
+            const float2 f = __half22float2(h2);
+            gv[j][2 * q] = f.x;
+            gv[j][2 * q + 1] = f.y;
+          }
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      if (lane == 0) red_s[warp] = ss;
+      consumer_sync();
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) tot += red_s[w];
+      const float inv = 1.0f / sqrtf(tot / (float)K + p.eps);
+#pragma unroll
+      for (int j = 0; j < kRuns; ++j) {
+        const int i0 = (tid + 256 * j) * 8;
+        if (i0 < K) {
+          uint32_t o4[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const __half2 h2 = __floats2half2_rn(xv[j][2 * q] * gv[j][2 * q] * inv, xv[j][2 * q + 1] * gv[j][2 * q + 1] * inv);
+            o4[q] = *reinterpret_cast<const uint32_t*>(&h2);
+            const float2 f = __half22float2(h2);  // the operand is the fp16-rounded value
+            xv[j][2 * q] = f.x;
+            xv[j][2 * q + 1] = f.y;
+          }
+          if (p.h_out && blockIdx.x == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kRuns; ++j) {
+      const int r = tid + 256 * j;  // run index; block r / 4, word r % 4.  All four lanes of a group are in range together.
+      if (r * 8 < K) quantize_run4(xv[j], r & 3, xq_s + (size_t)(r >> 2) * 28);
     }
     consumer_sync();
 #pragma unroll
@@ -342,7 +370,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
       const int b = b0 + lane + 32 * j;
       if (b < b1) {
         uint32_t xh[16];
-        const uint4* src = reinterpret_cast<const uint4*>(xsrc + (size_t)b * 32);
+        const uint4* src = reinterpret_cast<const uint4*>(p.x16 + (size_t)b * 32);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const uint4 v = src[q];
@@ -469,7 +497,7 @@ bool gemv_stream_eligible(const GemvParams& p) {
     for (int s = 0; s < p.n_seg; ++s)
       if (p.seg[s].n_rows % rows) return false;
   }
-  if (p.norm_gain && p.K > 8192) return false;
+  if (p.norm_gain && p.K > 4096) return false;  // the fused norm prologue covers hidden sizes up to 4096
   return true;
 }
 
@@ -505,7 +533,7 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   p.res16 = g.res16;
   p.status = status;
   const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (g.norm_gain ? (size_t)g.K * 2 : 0) + (parts <= 2 ? (size_t)(g.K / 32) * 112 : 0);
+  const size_t smem = kStages * stage_bytes + (parts <= 2 ? (size_t)(g.K / 32) * 112 : 0);
   const int grid = std::max(1, std::min(tiles, 2 * sm_count));
   void (*kern)(const StreamParams) = nullptr;
   switch (parts) {
