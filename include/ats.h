@@ -136,6 +136,24 @@ int32_t ats_get_placement(const ats_ctx* ctx, int32_t id, int32_t expert, uint8_
  * If the tensor is placed on the host it is streamed through the ring for this call. */
 int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /*DEVICE*/, uint32_t M);
 
+/* ats_linear for callers that must not allocate.  (The paper has no counterpart; this is a packaging variant.)
+ * Some hosts of this library cannot hand it device memory beyond their tensors: code running inside a captured or
+ * replayed region, plug-ins of an inference server whose memory pool is frozen after start-up, or a process that
+ * has given all device memory to another allocator.  ats_linear needs scratch for its split-K partial sums when
+ * M > 8 and takes it from the workspace the caller allocated; this entry point takes it instead from a fixed array of
+ * ATS_STATIC_SCRATCH_BYTES that is part of the library's device image, so that it calls no cudaMalloc / cudaFree /
+ * allocating routine of any library.  Same arguments and result as ats_linear, with these differences:
+ *  - the tensor must be GPU-placed (streaming would need the ring) -> ATS_ERR_STATE otherwise;
+ *  - if the partial sums of this shape need more than ATS_STATIC_SCRATCH_BYTES the call fails with ATS_ERR_NOMEM and
+ *    the text says how much was needed;
+ *  - every GPU that loads the library holds the array from load to exit; all calls (all contexts, all streams of a
+ *    process) share it, and nothing in it has to start at zero: each call fully writes the partials it later reads.
+ *    Two calls that overlap on the GPU (different streams) would overwrite each other's partials: keep them on one stream;
+ *  - the first call on a device looks the array's device address up (cudaGetSymbolAddress) and caches it; make that
+ *    first call before any stream capture begins. */
+#define ATS_STATIC_SCRATCH_BYTES (32ull << 20)
+int32_t ats_linear_static_scratch(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /*DEVICE*/, uint32_t M);
+
 /* Router: logits = h W_r (fp16 weights [hidden][E], fp32 accumulation); ids[m][0..k) = the k largest logits in
  * descending order, equal logits -> lower expert index first; gates = softmax over the selected logits.
  * h DEVICE fp16 [M][hidden]; ids_dev DEVICE int32 [M][k]; gates_dev DEVICE fp32 [M][k].  k <= 32, E <= 1024. */

@@ -28,7 +28,7 @@ EDGES = ("h", "q", "k", "v", "q_rot", "a", "o", "x1", "h2", "g", "u", "act", "d"
 
 EXPORTS = (
     "ats_init", "ats_destroy", "ats_last_error", "ats_register_tensor", "ats_tensor_slice_bytes", "ats_set_placement",
-    "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_route_topk", "ats_moe_linear", "ats_layer_decode",
+    "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode",
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
     "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
     "ats_host_unpack_q4",
@@ -77,6 +77,7 @@ def _load():
         "ats_plan_placement": (i32, [vp, u64, u32, vp, u32]),
         "ats_get_placement": (i32, [vp, i32, i32, P(C.c_uint8)]),
         "ats_linear": (i32, [vp, i32, vp, vp, u32]),
+        "ats_linear_static_scratch": (i32, [vp, i32, vp, vp, u32]),
         "ats_route_topk": (i32, [vp, i32, vp, u32, u32, vp, vp]),
         "ats_moe_linear": (i32, [vp, i32, vp, vp, vp, u32, u32, u32]),
         "ats_layer_decode": (i32, [vp, P(ats_layer_desc), vp, vp, vp, vp, u32, u32]),
@@ -216,6 +217,10 @@ class Context:
     # ---- operators (device tensors in, device tensors out; all asynchronous)
     def linear(self, tid, x, y, M):
         return self.check(lib.ats_linear(self.h, tid, _ptr(x), _ptr(y), M))
+
+    def linear_static_scratch(self, tid, x, y, M):
+        """ats_linear with the split-K scratch in the library's fixed device array (allocates nothing)."""
+        return self.check(lib.ats_linear_static_scratch(self.h, tid, _ptr(x), _ptr(y), M))
 
     def route_topk(self, router_id, h, M, k, ids, gates):
         return self.check(lib.ats_route_topk(self.h, router_id, _ptr(h), M, k, _ptr(ids), _ptr(gates)))

@@ -229,6 +229,9 @@ struct GemmParams {
 };
 uint64_t gemm_scratch_bytes(int T, int n_total, int K);
 cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);
+// fixed split-K scratch inside the library's device image (no allocation): capacity, and its address on the current device
+uint64_t gemm_static_scratch_capacity();
+cudaError_t gemm_static_scratch(void** out);
 
 // host-side pieces
 void repack_q4(const uint8_t* codes_in, const uint16_t* scales_in, uint8_t* slice_out, uint64_t n_rows, uint64_t K);

@@ -845,6 +845,44 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M)
   return run_gemm_group(ctx, &op, 1, g);
 }
 
+int32_t ats_linear_static_scratch(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M) {
+  ATS_TRY(precheck(ctx, true));
+  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", id);
+  if (!x || !y) return fail(ctx, ATS_ERR_INVALID, "null pointer");
+  if (t->slices[0].where != ATS_GPU)
+    return fail(ctx, ATS_ERR_STATE, "tensor %d is host-placed: the no-allocation entry point only runs resident tensors", id);
+  if (M == 0) return ATS_OK;
+  plan_begin(ctx);
+  Operand op;
+  plan_dense(ctx, id, &op);
+  if (M <= 8) {  // the GEMV needs no scratch at all
+    GemvParams p{};
+    p.M = (int)M;
+    p.x = (const __half*)x;
+    p.ldx = (int)t->d.k_in;
+    p.y16 = (__half*)y;
+    p.ldy = (int)t->d.n_out;
+    p.mode = GEMV_OUT_F16;
+    return run_gemv_group(ctx, &op, 1, p);
+  }
+  const uint64_t need = gemm_scratch_bytes((int)M, (int)t->d.n_out, (int)t->d.k_in);
+  if (need > gemm_static_scratch_capacity())
+    return fail(ctx, ATS_ERR_NOMEM, "split-K partials of %u x %u x %u need %llu bytes, the static scratch holds %llu", M, t->d.n_out,
+                t->d.k_in, (unsigned long long)need, (unsigned long long)gemm_static_scratch_capacity());
+  void* scratch = nullptr;
+  ATS_CUDA(gemm_static_scratch(&scratch));
+  GemmParams g{};
+  g.T = (int)M;
+  g.x = (const __half*)x;
+  g.ldx = (int)t->d.k_in;
+  g.y = (__half*)y;
+  g.ldy = (int)t->d.n_out;
+  g.scratch = scratch;
+  g.scratch_bytes = gemm_static_scratch_capacity();
+  return run_gemm_group(ctx, &op, 1, g);
+}
+
 int32_t ats_dequantize(ats_ctx* ctx, int32_t id, int32_t expert, void* out_dev, uint32_t out_fmt) {
   ATS_TRY(precheck(ctx, true));
   Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);

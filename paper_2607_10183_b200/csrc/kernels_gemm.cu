@@ -445,4 +445,30 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   return e;
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Split-K scratch that needs no allocation: a fixed array in the library's own device image.
+// Every GPU that loads the library carries these 32 MiB from load until exit.
+constexpr uint64_t kStaticScratchBytes = 32ull << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+uint64_t gemm_static_scratch_capacity() { return kStaticScratchBytes; }
+
+// Device address of the array for the CURRENT device.  In host code the symbol's name is only a handle, not an address a
+// kernel could use, so the address is asked from the runtime once per device and cached.
+cudaError_t gemm_static_scratch(void** out) {
+  static void* cached[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!cached[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    cached[dev] = ptr;
+  }
+  *out = cached[dev];
+  return cudaSuccess;
+}
+
 }  // namespace ats

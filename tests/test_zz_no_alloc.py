@@ -1,0 +1,71 @@
+"""The no-allocation variant of ats_linear (split-K partial sums in the library's fixed device array).
+
+Who needs it: callers that cannot give the library any device memory of their own at call time, e.g. a plug-in whose
+host froze its memory pool at start-up, so even the workspace ats_linear borrows is not available to them.
+The file name sorts last on purpose: a run that stops at the first failure has then already run every other test."""
+import numpy as np
+import pytest
+
+from paper_2607_10183_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+MB = 1 << 20
+
+
+def test_static_scratch_linear_equals_linear_twice_in_a_row():
+    import torch
+    from paper_2607_10183_b200 import binding as B
+    # a shape that takes split-K (few feature tiles, many k-steps), so the scratch is really used, and a ragged one
+    for N, K, T in ((512, 2048, 64), (136, 4096, 200)):
+        packed, scales = W.q4_packed(77, 0, W.ROLE_Q, N, K)
+        nb = W.q4_bytes(N, K)
+        ws = 8 * T * N * 4 + 2 * MB  # only the reference call (ats_linear) uses this workspace
+        ctx = B.Context(ws + nb + MB, workspace_bytes=ws)
+        tid = ctx.register_q4(packed, scales)
+        ctx.set_placement([(tid, -1, B.ATS_GPU)])
+        outs = []
+        for call in range(2):  # two calls in a row share the array and must not disturb each other
+            x = torch.from_numpy(W.activations(77, call, (T, K))).cuda()
+            want = torch.empty((T, N), dtype=torch.float16, device="cuda")
+            got = torch.full((T, N), 3.0, dtype=torch.float16, device="cuda")
+            ctx.linear(tid, x, want, T)
+            ctx.linear_static_scratch(tid, x, got, T)
+            ctx.sync()
+            # same kernels, same split choice, same summation order: the outputs are identical, which is well inside
+            # the 2e-3 relative tolerance the other GEMM tests use
+            a, b = got.cpu().numpy().astype(np.float64), want.cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(a - b)) <= 2e-3 * np.max(np.abs(b))
+            assert np.array_equal(got.cpu().numpy().view(np.uint16), want.cpu().numpy().view(np.uint16))
+            outs.append(a)
+        assert not np.array_equal(outs[0], outs[1])  # the two calls really had different inputs
+        # M <= 8 goes through the GEMV, which needs no scratch
+        x1 = torch.from_numpy(W.activations(77, 5, (3, K))).cuda()
+        y1 = torch.empty((3, N), dtype=torch.float16, device="cuda")
+        y2 = torch.empty((3, N), dtype=torch.float16, device="cuda")
+        ctx.linear(tid, x1, y1, 3)
+        ctx.linear_static_scratch(tid, x1, y2, 3)
+        ctx.sync()
+        assert np.array_equal(y1.cpu().numpy().view(np.uint16), y2.cpu().numpy().view(np.uint16))
+        ctx.close()
+
+
+def test_static_scratch_rejects_what_it_cannot_hold_and_host_placed_tensors():
+    import torch
+    from paper_2607_10183_b200 import binding as B
+    N, K = 2048, 4096  # 16 feature tiles -> 8 splits; with T = 1024 the partials need 8 * 1024 * 2048 * 4 B = 64 MiB > 32 MiB
+    packed, scales = W.q4_packed(77, 1, W.ROLE_Q, N, K)
+    nb = W.q4_bytes(N, K)
+    ctx = B.Context(4 * MB + 2 * (nb + 256) + nb + MB, workspace_bytes=4 * MB, ring_slots=2, slot_bytes=nb)
+    tid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(tid, -1, B.ATS_GPU)])
+    T = 1024
+    x = torch.zeros((T, K), dtype=torch.float16, device="cuda")
+    y = torch.empty((T, N), dtype=torch.float16, device="cuda")
+    with pytest.raises(B.AtsError) as e:
+        ctx.linear_static_scratch(tid, x, y, T)
+    assert e.value.code == B.ATS_ERR_NOMEM and "static scratch" in str(e.value)
+    ctx.set_placement([(tid, -1, B.ATS_HOST)])
+    with pytest.raises(B.AtsError) as e:
+        ctx.linear_static_scratch(tid, x, y, 16)
+    assert e.value.code == B.ATS_ERR_STATE
+    ctx.close()
