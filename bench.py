@@ -407,22 +407,35 @@ def run_ours(args):
     clocks = sampler.summary(t_wall0, t_wall1)
     tok_s = world * args.steps / (ms * 1e-3)
 
-    # ---- profiling pass: the same steps with every GEMV launch bracketed by events -> roofline of the dominant kernel
+    # ---- roofline of the dominant kernel family (the GEMV: 4 of the 5 launches of a step, 81 % of its time).
+    # Its average launch duration is measured live with CUDA events over a timed region of the same steps in which the
+    # one other launch (attention) is switched off, so the GEMV launches run back to back exactly as in the step
+    # (programmatic dependent launch included) and nothing but them is inside the events.  Bracketing every launch
+    # with its own event pair instead (ATS_FLAG_TIME_KERNELS) serialises the launches and adds ~3 us to each; that
+    # figure is reported as `achieved_event_bracketed`.
+    skip_attn = 2 << 24
+    ctx.set_flags(skip_attn)
+    steps(args.warmup)
+    barrier()
+    n_prof = min(args.steps, 5000)
+    gemv_only_ms = event_time_ms(torch, cs, lambda: steps(n_prof, args.warmup))
     ctx.set_flags(B.ATS_FLAG_TIME_KERNELS)
     ctx.reset_stats()
-    n_prof = min(args.steps, 2000)
-    steps(n_prof, args.warmup)
+    steps(min(n_prof, 2000), args.warmup)
     ctx.sync()
     st = ctx.stats()
     ctx.set_flags(0)
-    gemv_ms, gemv_n, gemv_bytes = st.timed_ms[0], st.timed_launches[0], st.timed_work[0]
-    achieved = gemv_bytes / (gemv_ms * 1e-3) / 1e9 if gemv_ms > 0 else None
-    roofline = {"bound": "hbm", "kernel": "gemv_kernel (4 launches per step: fused QKV, O, fused gate/up+SwiGLU, down)",
+    gemv_n, gemv_bytes = st.timed_launches[0], st.timed_work[0]
+    bytes_per_launch = gemv_bytes / max(gemv_n, 1)
+    avg_launch_us = gemv_only_ms * 1e3 / (4 * n_prof)
+    achieved = bytes_per_launch / (avg_launch_us * 1e-6) / 1e9
+    bracketed = gemv_bytes / (st.timed_ms[0] * 1e-3) / 1e9 if st.timed_ms[0] > 0 else None
+    roofline = {"bound": "hbm", "kernel": "gemv_stream_kernel (4 launches per step: fused QKV, O, fused gate/up+SwiGLU, down)",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"] + " HBM copy bandwidth",
-                "unit": "GB/s", "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
-                "frac_of_nominal_8TBs": (achieved / 8000.0) if achieved else None,
-                "bytes_per_launch": gemv_bytes / max(gemv_n, 1), "avg_launch_us": gemv_ms * 1e3 / max(gemv_n, 1),
-                "launches_timed": int(gemv_n), "traffic": args.traffic}
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBs": achieved / 8000.0,
+                "bytes_per_launch": bytes_per_launch, "avg_launch_us": avg_launch_us, "launches_timed": 4 * n_prof,
+                "achieved_event_bracketed": bracketed, "traffic": args.traffic if args.traffic else 30.73e6,
+                "traffic_note": "ncu dram__bytes_read+write per launch, mean of the four launches of a step (123 MB / 4); equals the algorithmic bytes"}
 
     # ---- end to end: the same step driven from pinned host buffers (H2D of x and D2H of y inside the timed region)
     def e2e_steps(n, start=0):
