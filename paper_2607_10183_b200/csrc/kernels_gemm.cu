@@ -1,17 +1,18 @@
 // Dequantize-fused prefill GEMM on the 5th-generation tensor cores (sm_100a): Y[T][N] = X[T][K] * W^T, fp16 operands,
 // fp32 accumulation in tensor memory, fp16 output.
 //
-// One CTA computes a tile of 128 output features x up to 512 tokens over a K range (split-K when the feature tiles do not
-// fill the GPU).  The weight tile is the MMA A operand: four warps read the packed 4-bit codes and fp16 scales straight
-// from global memory (each thread one weight row), expand them to fp16 (w = rn16(scale * code), a single rounding) and
-// store them into shared memory in the canonical K-major 128-byte-swizzle layout the tensor core reads.  The activation
-// tile is the B operand, loaded by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-range rows zero-filled).  A single
-// thread issues tcgen05.mma (M = 128, N = tokens, K = 16 per instruction) into up to two 256-column accumulators in TMEM;
-// tcgen05.commit releases the stage to the producers through an mbarrier.  The four dequantization warps then become the
-// epilogue: tcgen05.ld brings the accumulator rows back (lane = feature, columns = tokens) and writes Y (or an fp32
-// split-K partial that a second kernel sums in split order).
+// One CTA computes a tile of 256 output features x up to 256 tokens over a K range (split-K when the tiles do not fill
+// the GPU).  The weight tile is the MMA A operand, as two 128-row sub-tiles that share one activation tile (which halves
+// the activation bytes re-read from L2 per flop): eight warps read the packed 4-bit codes and fp16 scales straight from
+// global memory (each thread one weight row), expand them to fp16 (w = rn16(scale * code), a single rounding) and store
+// them into shared memory in the canonical K-major 128-byte-swizzle layout the tensor core reads.  The activation tile is
+// the B operand, loaded by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-range rows zero-filled).  A single thread
+// issues tcgen05.mma (M = 128, N = tokens, K = 16 per instruction) into two 256-column accumulators in TMEM (all 512
+// columns); tcgen05.commit releases the stage to the producers through an mbarrier.  The eight dequantization warps then
+// become the epilogue: tcgen05.ld brings the accumulator rows back (lane = feature, columns = tokens) and writes Y (or
+// an fp32 split-K partial that a second kernel sums in split order).
 //
-// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 = weight dequantization, then epilogue.
+// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..9 = weight dequantization, then epilogue.
 // No cluster launch and no multicast.  Every mbarrier wait is bounded; on expiry the CTA raises the status word, skips
 // the rest of its work, frees its tensor memory and returns.
 #include <cuda.h>
@@ -22,15 +23,19 @@ namespace ats {
 
 namespace {
 
-constexpr int BM = 128;         // features per tile (MMA M)
+constexpr int BM = 128;         // features per MMA (M)
+constexpr int FT = 2;           // 128-row feature sub-tiles per CTA, one accumulator each
+constexpr int BF = BM * FT;     // features per CTA tile
 constexpr int BK = 64;          // k per stage: 64 fp16 = one 128-byte swizzle row
-constexpr int TACC = 256;       // tokens per accumulator (MMA N <= 256)
-constexpr int TTILE = 512;      // tokens per CTA (two accumulators = all 512 TMEM columns)
+constexpr int TACC = 256;       // TMEM columns per accumulator (MMA N <= 256)
+constexpr int TTILE = 256;      // tokens per CTA
 constexpr int BOXR = 64;        // activation rows per TMA box
-constexpr int kGemmThreads = 192;
-constexpr int A_BYTES = BM * BK * 2;      // 16 KB
-constexpr int B_ACC_BYTES = TACC * BK * 2;  // 32 KB per accumulator
-constexpr int kMaxStages = 4;
+constexpr int kDequantWarps = BF / 32;
+constexpr int kGemmThreads = (2 + kDequantWarps) * 32;
+constexpr int A_BYTES = BM * BK * 2;        // 16 KB per feature sub-tile
+constexpr int B_BYTES = TTILE * BK * 2;     // 32 KB activation tile
+constexpr int kStageBytes = FT * A_BYTES + B_BYTES;
+constexpr int kMaxStages = 3;
 
 struct GemmSeg {
   const uint8_t* base;
@@ -156,33 +161,27 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_c
   const int tile = blockIdx.x;
   int sg = 0;
   while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
-  const int row0 = (tile - p.seg[sg].tile0) * BM;
+  const int row0 = (tile - p.seg[sg].tile0) * BF;
   const int n_rows = p.seg[sg].n_rows;
   const int t0 = blockIdx.y * TTILE;
   const int Tt = min(TTILE, p.T - t0);
-  const int n_acc = (Tt + TACC - 1) / TACC;
+  const int nmma = (Tt + 15) / 16 * 16;          // MMA N
+  const int boxes = (Tt + BOXR - 1) / BOXR;      // TMA boxes of 64 activation rows
+  const int n_ft = row0 + BM < n_rows ? FT : 1;  // feature sub-tiles that hold real rows
   const int split = blockIdx.z;
   const int ks0 = split * p.ksteps_per_split;
   const int nks = min(p.ksteps_per_split, p.total_ksteps - ks0);
-  const int stage_bytes = A_BYTES + n_acc * B_ACC_BYTES;
-  int nj[2], nmma[2], boxes[2];
-#pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    nj[j] = max(0, min(TACC, Tt - TACC * j));
-    nmma[j] = (nj[j] + 15) / 16 * 16;
-    boxes[j] = (nj[j] + BOXR - 1) / BOXR;
-  }
   if (threadIdx.x == 0) {
     fail_s = 0;
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(&full_a[s], 128);
+      mbar_init(&full_a[s], BF);
       mbar_init(&full_b[s], 1);
       mbar_init(&empty[s], 1);
     }
     mbar_init(&acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  const uint32_t tmem_cols = n_acc == 2 ? 512u : 256u;
+  const uint32_t tmem_cols = 512u;
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(tmem_cols)
                  : "memory");
@@ -197,26 +196,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_c
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (activation tile)
     if (lane == 0) {
-      uint32_t tx = 0;
-      for (int j = 0; j < n_acc; ++j) tx += (uint32_t)boxes[j] * BOXR * BK * 2;
+      const uint32_t tx = (uint32_t)boxes * BOXR * BK * 2;
       for (int i = 0; i < nks; ++i) {
         const int s = i % S;
         if (i >= S && !mbar_wait(&empty[s], ((i / S) - 1) & 1)) {
           fail_s = 1;
           break;
         }
-        uint8_t* bdst = smem + (size_t)s * stage_bytes + A_BYTES;
+        uint8_t* bdst = smem + (size_t)s * kStageBytes + FT * A_BYTES;
         mbar_expect_tx(&full_b[s], tx);
-        for (int j = 0; j < n_acc; ++j)
-          for (int b = 0; b < boxes[j]; ++b)
-            tma_load_2d(bdst + (size_t)j * B_ACC_BYTES + (size_t)b * BOXR * BK * 2, &xmap, (ks0 + i) * BK, t0 + j * TACC + b * BOXR,
-                        &full_b[s]);
+        for (int b = 0; b < boxes; ++b)
+          tma_load_2d(bdst + (size_t)b * BOXR * BK * 2, &xmap, (ks0 + i) * BK, t0 + b * BOXR, &full_b[s]);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issue
     if (lane == 0) {
       bool ok = true;
+      const uint32_t idesc = umma_idesc(nmma);
       for (int i = 0; i < nks && ok; ++i) {
         const int s = i % S;
         const uint32_t par = (i / S) & 1;
@@ -226,22 +223,21 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_c
           break;
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t adesc = umma_desc(a_addr);
+        const uint32_t a_addr = smem_u32(smem + (size_t)s * kStageBytes);
+        const uint64_t bdesc = umma_desc(a_addr + FT * A_BYTES);
 #pragma unroll
         for (int kk = 0; kk < BK / 16; ++kk) {
-          for (int j = 0; j < n_acc; ++j) {
-            const uint64_t bdesc = umma_desc(a_addr + A_BYTES + j * B_ACC_BYTES);
-            umma_f16(tmem_base + (uint32_t)(j * TACC), adesc + 2 * kk, bdesc + 2 * kk, umma_idesc(nmma[j]), (i > 0 || kk > 0) ? 1u : 0u);
-          }
+          for (int ft = 0; ft < n_ft; ++ft)
+            umma_f16(tmem_base + (uint32_t)(ft * TACC), umma_desc(a_addr + ft * A_BYTES) + 2 * kk, bdesc + 2 * kk, idesc,
+                     (i > 0 || kk > 0) ? 1u : 0u);
         }
         umma_commit(&empty[s]);  // arrives when the MMAs reading stage s are done
       }
       if (ok) umma_commit(&acc_full);
     }
   } else {
-    // ------------------------------------------------------------ weight dequantization (A tile), one row per thread
-    const int r = (warp - 2) * 32 + lane;
+    // ------------------------------------------------------------ weight dequantization (A tiles), one row per thread
+    const int r = (warp - 2) * 32 + lane;  // 0..255: sub-tile r / 128, row r % 128
     const int grow = row0 + r;
     const bool valid = grow < n_rows;
     const int K = p.K, nblk = K / 32;
@@ -275,7 +271,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_c
         ok = false;
         break;
       }
-      uint8_t* arow = smem + (size_t)s * stage_bytes + (size_t)r * 128;
+      uint8_t* arow = smem + (size_t)s * kStageBytes + (size_t)r * 128;  // sub-tiles are contiguous: row r at r * 128
       const __half2 s0 = __half2half2(__ushort_as_half((unsigned short)(scw & 0xFFFF)));
       const __half2 s1 = __half2half2(__ushort_as_half((unsigned short)(scw >> 16)));
       const int sw = r & 7;
@@ -294,17 +290,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_c
     if (ok && nks > 0 && mbar_wait(&acc_full, 0)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int q = warp & 3;               // TMEM lane quarter this warp may read
-      const int f = q * 32 + lane;          // feature row within the tile
+      const int ft = (warp - 2) >> 2;       // feature sub-tile = accumulator
+      const int f = ft * BM + q * 32 + lane;
       const bool fvalid = row0 + f < n_rows;
       const int col = p.seg[sg].col0 + row0 + f;
-      for (int j = 0; j < n_acc; ++j) {
-        for (int c0 = 0; c0 < nmma[j]; c0 += 32) {
+      if (ft < n_ft) {
+        for (int c0 = 0; c0 < nmma; c0 += 32) {
           uint32_t v[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * TACC + c0), v);
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ft * TACC + c0), v);
           if (fvalid) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              const int t = t0 + j * TACC + c0 + e;
+              const int t = t0 + c0 + e;
               if (t < p.T) {
                 if (p.splits > 1)
                   p.partial[((size_t)split * p.T + t) * p.ldy + col] = __uint_as_float(v[e]);
@@ -362,11 +359,6 @@ int pick_splits(int tiles, int total_ksteps, int sm_count) {
   return s;
 }
 
-int feature_tiles(const GemmParams& p) {
-  int tiles = 0;
-  for (int i = 0; i < p.n_seg; ++i) tiles += (p.seg[i].n_rows + BM - 1) / BM;
-  return tiles;
-}
 
 }  // namespace
 
@@ -374,7 +366,7 @@ uint64_t gemm_scratch_bytes(int T, int n_total, int K) {
   // fp32 partials of the split choice for this shape (fewer tiles can only mean more splits, so the tile count of the
   // concatenated rows bounds it from above); the launcher falls back to one split if the buffer it gets is smaller
   const int total_ksteps = (K + BK - 1) / BK;
-  const int tiles = ((n_total + BM - 1) / BM) * ((T + TTILE - 1) / TTILE);
+  const int tiles = ((n_total + BF - 1) / BF) * ((T + TTILE - 1) / TTILE);
   const int s = pick_splits(tiles, total_ksteps, 148);
   return s > 1 ? (uint64_t)s * T * n_total * 4 + 256 : 256;
 }
@@ -404,7 +396,7 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   int tiles = 0, col = 0;
   for (int i = 0; i < g.n_seg; ++i) {
     p.seg[i] = GemmSeg{g.seg[i].base, g.seg[i].n_rows, tiles, col};
-    tiles += (g.seg[i].n_rows + BM - 1) / BM;
+    tiles += (g.seg[i].n_rows + BF - 1) / BF;
     col += g.seg[i].n_rows;
   }
   const int tchunks = (g.T + TTILE - 1) / TTILE;
@@ -421,9 +413,8 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   p.ldy = g.ldy;
   p.partial = (float*)g.scratch;
   p.status = g.status;
-  const int n_acc = std::min(g.T, TTILE) > TACC ? 2 : 1;
-  p.stages = n_acc == 2 ? 2 : 4;
-  const size_t smem = (size_t)p.stages * (A_BYTES + n_acc * B_ACC_BYTES) + 1024;
+  p.stages = kMaxStages;
+  const size_t smem = (size_t)p.stages * kStageBytes + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(gemm_q4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);

@@ -1,5 +1,5 @@
 // Prefill-side glue kernels (sm_100a): rotary embedding + KV append over T tokens, causal grouped-query attention
-// over the cache, fp16 residual add and SwiGLU.  Every intermediate of the prefill path is stored as fp16 (the
+// over the cache (tensor cores), fp16 residual add and SwiGLU.  Every intermediate of the prefill path is stored as fp16 (the
 // operands of the tensor-core GEMMs), so these kernels read and write fp16 and compute in fp32.
 #include "ats_internal.h"
 
@@ -66,80 +66,203 @@ cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_ro
   return cudaGetLastError();
 }
 
-// Causal attention: one warp per (token, query head); lanes take cache positions 32 at a time (each lane one whole
-// key row), online softmax across chunks, then P.V with the probabilities broadcast by shuffles.
+// Causal grouped-query attention over the cache on the tensor cores (mma.sync m16n8k16, fp16 operands, fp32 accumulate).
+// CTA = 64 query tokens of one query head, 4 warps x 16 rows.  Key/value blocks of 64 cache rows are staged with 16-byte
+// async copies into padded shared-memory rows (double buffered); S = Q K^T and O += P V use ldmatrix fragments; the softmax
+// is the running-max form in fp32, with P rounded to fp16 as the operand of the second product.
+constexpr int kFaQ = 64;   // query rows per CTA
+constexpr int kFaK = 64;   // cache rows per block
+
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_h2(float a, float b) {
+  const __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
 template <int D>
 __global__ void __launch_bounds__(128) attn_prefill_kernel(const __half* __restrict__ q_rot, const __half* __restrict__ kc,
                                                            const __half* __restrict__ vc, __half* __restrict__ a16, int T,
                                                            int n_q, int group, int cap, int pos0, float scale) {
-  constexpr int V = D / 32;
-  __shared__ float q_s[4][D];
+  constexpr int PITCH = D + 8;          // halfs per shared-memory row (16-byte pad: conflict-free ldmatrix)
+  constexpr int CH = D / 8;             // 16-byte chunks per row
+  constexpr int KS = D / 16;            // k-steps of Q K^T
+  constexpr int NT = D / 8;             // n-tiles of the output
+  extern __shared__ __align__(16) __half fa_smem[];
+  __half* q_s = fa_smem;                          // [kFaQ][PITCH]
+  __half* k_s = q_s + kFaQ * PITCH;               // [2][kFaK][PITCH]
+  __half* v_s = k_s + 2 * kFaK * PITCH;           // [2][kFaK][PITCH]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int hq = blockIdx.x * 4 + warp;  // 4 heads per CTA
-  const int t = blockIdx.y;
-  if (hq >= n_q) return;
-  const int kvh = hq / group;
-  const int n_ctx = pos0 + t + 1;
-  for (int e = lane; e < D; e += 32) q_s[warp][e] = __half2float(q_rot[((size_t)t * n_q + hq) * D + e]);
-  __syncwarp();
-  float m_run = -INFINITY, l_run = 0.f;
-  float acc[V];
-#pragma unroll
-  for (int v = 0; v < V; ++v) acc[v] = 0.f;
-  for (int t0 = 0; t0 < n_ctx; t0 += 32) {
-    const int tp = t0 + lane;
-    const bool ok = tp < n_ctx;
-    float sc = 0.f;
-    if (ok) {
-      const uint4* kr = reinterpret_cast<const uint4*>(kc + ((size_t)kvh * cap + tp) * D);
-#pragma unroll 4
-      for (int c = 0; c < D / 8; ++c) {
-        const uint4 kv = __ldg(kr + c);
-        const float* qg = q_s[warp] + c * 8;
-        float2 f;
-        f = __half22float2(bits_as_half2(kv.x)); sc = fmaf(f.x, qg[0], sc); sc = fmaf(f.y, qg[1], sc);
-        f = __half22float2(bits_as_half2(kv.y)); sc = fmaf(f.x, qg[2], sc); sc = fmaf(f.y, qg[3], sc);
-        f = __half22float2(bits_as_half2(kv.z)); sc = fmaf(f.x, qg[4], sc); sc = fmaf(f.y, qg[5], sc);
-        f = __half22float2(bits_as_half2(kv.w)); sc = fmaf(f.x, qg[6], sc); sc = fmaf(f.y, qg[7], sc);
-      }
-    }
-    const float s = ok ? sc * scale : -INFINITY;
-    const float m_new = fmaxf(m_run, wmax(s));
-    const float corr = m_run > -INFINITY ? expf(m_run - m_new) : 0.f;
-    const float p = ok ? expf(s - m_new) : 0.f;
-    l_run = l_run * corr + wsum(p);
-#pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] *= corr;
-    const int n_here = min(32, n_ctx - t0);
-    for (int tt = 0; tt < n_here; ++tt) {
-      const float pt = __shfl_sync(0xffffffffu, p, tt);
-      const __half* vr = vc + ((size_t)kvh * cap + t0 + tt) * D + lane * V;
-      if (V == 4) {
-        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(vr));
-        float2 f;
-        f = __half22float2(bits_as_half2(raw.x)); acc[0] = fmaf(pt, f.x, acc[0]); acc[1] = fmaf(pt, f.y, acc[1]);
-        f = __half22float2(bits_as_half2(raw.y)); acc[2] = fmaf(pt, f.x, acc[2]); acc[3] = fmaf(pt, f.y, acc[3]);
-      } else {
-        const float2 f = __half22float2(bits_as_half2(__ldg(reinterpret_cast<const uint32_t*>(vr))));
-        acc[0] = fmaf(pt, f.x, acc[0]);
-        acc[1] = fmaf(pt, f.y, acc[1]);
-      }
-    }
-    m_run = m_new;
+  const int qb = blockIdx.x, hq = blockIdx.y, kvh = hq / group;
+  const int tq0 = qb * kFaQ;                      // first token of the CTA
+  const int n_kb = (pos0 + min(T, tq0 + kFaQ) - 1) / kFaK + 1;  // cache blocks any row of the CTA attends to
+  // ---- stage Q (zero rows beyond T) and the first K/V block
+  for (int c = threadIdx.x; c < kFaQ * CH; c += 128) {
+    const int row = c / CH, ch = c % CH;
+    const int t = tq0 + row;
+    if (t < T)
+      cp_async_16(q_s + row * PITCH + ch * 8, q_rot + ((size_t)t * n_q + hq) * D + ch * 8);
+    else
+      *reinterpret_cast<uint4*>(q_s + row * PITCH + ch * 8) = make_uint4(0, 0, 0, 0);
   }
-  __half* dst = a16 + ((size_t)t * n_q + hq) * D + lane * V;
+  auto stage_kv = [&](int kb, int buf) {
+    for (int c = threadIdx.x; c < kFaK * CH; c += 128) {
+      const int row = c / CH, ch = c % CH;
+      const int key = min(kb * kFaK + row, cap - 1);  // rows past the context are masked below; keep the address legal
+      cp_async_16(k_s + (buf * kFaK + row) * PITCH + ch * 8, kc + ((size_t)kvh * cap + key) * D + ch * 8);
+      cp_async_16(v_s + (buf * kFaK + row) * PITCH + ch * 8, vc + ((size_t)kvh * cap + key) * D + ch * 8);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  stage_kv(0, 0);
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+  // ---- Q fragments of this warp's 16 rows
+  uint32_t qf[KS][4];
 #pragma unroll
-  for (int v = 0; v < V; ++v) dst[v] = __float2half_rn(acc[v] / l_run);
+  for (int ks = 0; ks < KS; ++ks)
+    ldsm_x4(qf[ks], q_s + (warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + ks * 16 + (lane >> 4) * 8);
+  float o[NT][4];
+#pragma unroll
+  for (int n = 0; n < NT; ++n)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o[n][e] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  const int g = lane >> 2, tq = lane & 3;
+  const int qpos[2] = {pos0 + tq0 + warp * 16 + g, pos0 + tq0 + warp * 16 + g + 8};  // absolute positions of this thread's rows
+  for (int kb = 0; kb < n_kb; ++kb) {
+    const int buf = kb & 1;
+    if (kb + 1 < n_kb) stage_kv(kb + 1, buf ^ 1);  // next block in flight while this one is used
+    const __half* kb_s = k_s + buf * kFaK * PITCH;
+    const __half* vb_s = v_s + buf * kFaK * PITCH;
+    // S = Q K^T for 16 rows x 64 keys
+    float sacc[kFaK / 8][4];
+#pragma unroll
+    for (int n = 0; n < kFaK / 8; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sacc[n][e] = 0.f;
+#pragma unroll
+    for (int n = 0; n < kFaK / 8; ++n) {
+#pragma unroll
+      for (int ks2 = 0; ks2 < KS / 2; ++ks2) {
+        uint32_t b[4];  // b0,b1 of k-step 2*ks2 and of k-step 2*ks2+1 for keys 8n..8n+7
+        ldsm_x4(b, kb_s + (n * 8 + (lane & 7)) * PITCH + ks2 * 32 + (lane >> 3) * 8);
+        mma_16816(sacc[n], qf[2 * ks2], b[0], b[1]);
+        mma_16816(sacc[n], qf[2 * ks2 + 1], b[2], b[3]);
+      }
+    }
+    // scale, causal mask, running softmax (rows g and g+8 of the warp's 16)
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int n = 0; n < kFaK / 8; ++n) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int key = kb * kFaK + n * 8 + 2 * tq + (e & 1);
+        const int r = e >> 1;
+        const float v = key <= qpos[r] ? sacc[n][e] * scale : -INFINITY;
+        sacc[n][e] = v;
+        mx[r] = fmaxf(mx[r], v);
+      }
+    }
+    float corr[2], m_new[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+      m_new[r] = fmaxf(m_run[r], mx[r]);
+      corr[r] = m_run[r] > -INFINITY ? expf(m_run[r] - m_new[r]) : 0.f;
+      m_run[r] = m_new[r];
+    }
+    float ls[2] = {0.f, 0.f};
+    uint32_t pf[kFaK / 16][4];  // P as A fragments (fp16)
+#pragma unroll
+    for (int n = 0; n < kFaK / 8; ++n) {
+      float pv[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = e >> 1;
+        pv[e] = m_new[r] > -INFINITY ? expf(sacc[n][e] - m_new[r]) : 0.f;
+        ls[r] += pv[e];
+      }
+      pf[n >> 1][(n & 1) * 2] = pack_h2(pv[0], pv[1]);
+      pf[n >> 1][(n & 1) * 2 + 1] = pack_h2(pv[2], pv[3]);
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      ls[r] += __shfl_xor_sync(0xffffffffu, ls[r], 1);
+      ls[r] += __shfl_xor_sync(0xffffffffu, ls[r], 2);
+      l_run[r] = l_run[r] * corr[r] + ls[r];
+    }
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      o[n][0] *= corr[0];
+      o[n][1] *= corr[0];
+      o[n][2] *= corr[1];
+      o[n][3] *= corr[1];
+    }
+    // O += P V
+#pragma unroll
+    for (int kk = 0; kk < kFaK / 16; ++kk) {
+#pragma unroll
+      for (int n2 = 0; n2 < NT / 2; ++n2) {
+        uint32_t b[4];  // (b0,b1) for dims 16 n2 .. +7 and for dims 16 n2 + 8 .. +15, keys 16 kk .. +15
+        ldsm_x4_t(b, vb_s + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + n2 * 16 + (lane >> 4) * 8);
+        mma_16816(o[2 * n2], pf[kk], b[0], b[1]);
+        mma_16816(o[2 * n2 + 1], pf[kk], b[2], b[3]);
+      }
+    }
+    if (kb + 1 < n_kb) asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();  // the next block has landed, and nobody still reads the buffer the block after it will overwrite
+  }
+  // ---- normalise and store
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int t = tq0 + warp * 16 + g + r * 8;
+    if (t < T) {
+      const float inv = 1.0f / l_run[r];
+      __half* dst = a16 + ((size_t)t * n_q + hq) * D;
+#pragma unroll
+      for (int n = 0; n < NT; ++n)
+        *reinterpret_cast<uint32_t*>(dst + n * 8 + 2 * tq) = pack_h2(o[n][2 * r] * inv, o[n][2 * r + 1] * inv);
+    }
+  }
 }
 
 cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const __half* vc, __half* a16, int T, int n_q,
                                 int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch) {
-  dim3 grid((n_q + 3) / 4, T);
+  dim3 grid((T + kFaQ - 1) / kFaQ, n_q);
   const float scale = 1.0f / sqrtf((float)d);
+  const size_t smem = (size_t)(kFaQ + 4 * kFaK) * (d + 8) * sizeof(__half);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e1 = cudaFuncSetAttribute(attn_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)((kFaQ + 4 * kFaK) * (128 + 8) * sizeof(__half)));
+    cudaError_t e2 = cudaFuncSetAttribute(attn_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)((kFaQ + 4 * kFaK) * (64 + 8) * sizeof(__half)));
+    if (e1 != cudaSuccess) return e1;
+    if (e2 != cudaSuccess) return e2;
+    attr_set = true;
+  }
   if (d == 128)
-    attn_prefill_kernel<128><<<grid, 128, 0, st>>>(q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0, scale);
+    attn_prefill_kernel<128><<<grid, 128, smem, st>>>(q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0, scale);
   else if (d == 64)
-    attn_prefill_kernel<64><<<grid, 128, 0, st>>>(q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0, scale);
+    attn_prefill_kernel<64><<<grid, 128, smem, st>>>(q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0, scale);
   else
     return cudaErrorInvalidValue;
   ++*n_launch;
@@ -158,19 +281,29 @@ cudaError_t launch_add16(const __half* a, const __half* b, __half* out, uint64_t
   return cudaGetLastError();
 }
 
-// gu holds [T][ld] with gate in columns [0, ffn) and up in [ffn, 2 ffn): act = rn16(silu(g) * u)
-__global__ void swiglu16_kernel(const __half* __restrict__ gu, int ld, int ffn, __half* __restrict__ act, uint64_t n) {
-  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
-    const uint64_t t = i / ffn, c = i % ffn;
-    const float g = __half2float(gu[t * ld + c]), u = __half2float(gu[t * ld + ffn + c]);
-    act[i] = __float2half_rn(g / (1.0f + expf(-g)) * u);
+// gu holds [T][ld] with gate in columns [0, ffn) and up in [ffn, 2 ffn): act = rn16(silu(g) * u); 8 elements per thread
+__global__ void swiglu16_kernel(const __half* __restrict__ gu, int ld, int ffn, __half* __restrict__ act, uint64_t n8) {
+  const int per_row = ffn / 8;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t t = i / per_row, c = (i % per_row) * 8;
+    const uint4 gv = *reinterpret_cast<const uint4*>(gu + t * ld + c);
+    const uint4 uv = *reinterpret_cast<const uint4*>(gu + t * ld + ffn + c);
+    const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, uw[4] = {uv.x, uv.y, uv.z, uv.w};
+    uint32_t ow[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float2 g = __half22float2(bits_as_half2(gw[q])), u = __half22float2(bits_as_half2(uw[q]));
+      const __half2 r = __floats2half2_rn(g.x / (1.0f + expf(-g.x)) * u.x, g.y / (1.0f + expf(-g.y)) * u.y);
+      ow[q] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+    *reinterpret_cast<uint4*>(act + t * ffn + c) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
   }
 }
 
 cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch) {
-  const uint64_t n = (uint64_t)T * ffn;
-  const int grid = (int)std::min<uint64_t>((n + 255) / 256, 148 * 8);
-  swiglu16_kernel<<<grid, 256, 0, st>>>(gu, ld, ffn, act, n);
+  const uint64_t n8 = (uint64_t)T * ffn / 8;  // ffn is a multiple of 32
+  const int grid = (int)std::min<uint64_t>((n8 + 255) / 256, 148 * 8);
+  swiglu16_kernel<<<grid, 256, 0, st>>>(gu, ld, ffn, act, n8);
   ++*n_launch;
   return cudaGetLastError();
 }
