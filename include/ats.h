@@ -151,7 +151,7 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /
  *    Two calls that overlap on the GPU (different streams) would overwrite each other's partials: keep them on one stream;
  *  - the first call on a device looks the array's device address up (cudaGetSymbolAddress) and caches it; make that
  *    first call before any stream capture begins. */
-#define ATS_STATIC_SCRATCH_BYTES (32ull << 20)
+#define ATS_STATIC_SCRATCH_BYTES (8ull << 20)
 int32_t ats_linear_static_scratch(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /*DEVICE*/, uint32_t M);
 
 /* Router: logits = h W_r (fp16 weights [hidden][E], fp32 accumulation); ids[m][0..k) = the k largest logits in

@@ -3,16 +3,16 @@
 //
 // One CTA computes a tile of 256 output features x up to 256 tokens over a K range (split-K when the tiles do not fill
 // the GPU).  The weight tile is the MMA A operand, as two 128-row sub-tiles that share one activation tile (which halves
-// the activation bytes re-read from L2 per flop): eight warps read the packed 4-bit codes and fp16 scales straight from
-// global memory (each thread one weight row), expand them to fp16 (w = rn16(scale * code), a single rounding) and store
+// the activation bytes re-read from L2 per flop): sixteen warps read the packed 4-bit codes and fp16 scales straight from
+// global memory (two threads per weight row, one 32-k block each per stage), expand them to fp16 (w = rn16(scale * code), a single rounding) and store
 // them into shared memory in the canonical K-major 128-byte-swizzle layout the tensor core reads.  The activation tile is
 // the B operand, loaded by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-range rows zero-filled).  A single thread
 // issues tcgen05.mma (M = 128, N = tokens, K = 16 per instruction) into two 256-column accumulators in TMEM (all 512
-// columns); tcgen05.commit releases the stage to the producers through an mbarrier.  The eight dequantization warps then
+// columns); tcgen05.commit releases the stage to the producers through an mbarrier.  The sixteen dequantization warps then
 // become the epilogue: tcgen05.ld brings the accumulator rows back (lane = feature, columns = tokens) and writes Y (or
 // an fp32 split-K partial that a second kernel sums in split order).
 //
-// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..9 = weight dequantization, then epilogue.
+// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..17 = weight dequantization, then epilogue.
 // No cluster launch and no multicast.  Every mbarrier wait is bounded; on expiry the CTA raises the status word, skips
 // the rest of its work, frees its tensor memory and returns.
 #include <cuda.h>
@@ -24,18 +24,24 @@ namespace ats {
 namespace {
 
 constexpr int BM = 128;         // features per MMA (M)
-constexpr int FT = 2;           // 128-row feature sub-tiles per CTA, one accumulator each
-constexpr int BF = BM * FT;     // features per CTA tile
 constexpr int BK = 64;          // k per stage: 64 fp16 = one 128-byte swizzle row
-constexpr int TACC = 256;       // TMEM columns per accumulator (MMA N <= 256)
-constexpr int TTILE = 256;      // tokens per CTA
 constexpr int BOXR = 64;        // activation rows per TMA box
-constexpr int kDequantWarps = BF / 32;
-constexpr int kGemmThreads = (2 + kDequantWarps) * 32;
-constexpr int A_BYTES = BM * BK * 2;        // 16 KB per feature sub-tile
-constexpr int B_BYTES = TTILE * BK * 2;     // 32 KB activation tile
-constexpr int kStageBytes = FT * A_BYTES + B_BYTES;
-constexpr int kMaxStages = 3;
+constexpr int A_BYTES = BM * BK * 2;        // 16 KB per 128-row feature sub-tile
+constexpr int kMaxStages = 6;
+// Two tile configurations <FT, TT>: FT 128-row feature sub-tiles (one accumulator each) x TT tokens per CTA.
+//   <2, 256>: 256 x 256, 3 stages of 64 KB, all 512 TMEM columns - for operators with enough feature tiles to fill the GPU
+//   <1, 128>: 128 x 128, 6 stages of 32 KB, 128 TMEM columns    - four times the CTAs for the narrow operators, which
+//             would otherwise need split-K and its fp32 partial traffic
+template <int FT, int TT>
+struct TileCfg {
+  static constexpr int BF = BM * FT;                      // features per CTA
+  static constexpr int kDequantWarps = 2 * BF / 32;       // two threads per weight row: one 32-k block each per k-step
+  static constexpr int kThreads = (2 + kDequantWarps) * 32;
+  static constexpr int B_BYTES = TT * BK * 2;
+  static constexpr int kStageBytes = FT * A_BYTES + B_BYTES;
+  static constexpr int kStages = (FT == 2 ? 3 : 6);
+  static constexpr int kTmemCols = FT * TT;               // 512 or 128: powers of two >= 32
+};
 
 struct GemmSeg {
   const uint8_t* base;
@@ -65,22 +71,24 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// Non-blocking poll.  (try_wait may put the thread to sleep, and waking it after the phase completes costs on the order
+// of a microsecond: far more than a k-step of this pipeline.)
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok)
       : "r"(smem_u32(bar)), "r"(parity)
       : "memory");
   return ok != 0;
 }
-// bounded wait (about a second of SM clocks)
+// bounded spin (about a second of SM clocks)
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_test_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
-    for (int i = 0; i < 64; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
+    for (int i = 0; i < 256; ++i)
+      if (mbar_test_wait(bar, parity)) return true;
     if (clock64() - t0 > 2000000000ll) return false;
   }
 }
@@ -149,7 +157,10 @@ __device__ __forceinline__ uint4 dequant8(uint32_t w, __half2 s2) {
   return o;
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const GemmKParams p) {
+template <int FT, int TT>
+__global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const GemmKParams p) {
+  using Cfg = TileCfg<FT, TT>;
+  constexpr int BF = Cfg::BF, TTILE = TT, TACC = TT, kDequantWarps = Cfg::kDequantWarps, kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_a[kMaxStages], full_b[kMaxStages], empty[kMaxStages], acc_full;
@@ -174,14 +185,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_c
   if (threadIdx.x == 0) {
     fail_s = 0;
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(&full_a[s], BF);
+      mbar_init(&full_a[s], kDequantWarps);  // one arrival per dequantization warp
       mbar_init(&full_b[s], 1);
       mbar_init(&empty[s], 1);
     }
     mbar_init(&acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  const uint32_t tmem_cols = 512u;
+  const uint32_t tmem_cols = (uint32_t)Cfg::kTmemCols;
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(tmem_cols)
                  : "memory");
@@ -236,66 +247,84 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_q4_kernel(const __grid_c
       if (ok) umma_commit(&acc_full);
     }
   } else {
-    // ------------------------------------------------------------ weight dequantization (A tiles), one row per thread
-    const int r = (warp - 2) * 32 + lane;  // 0..255: sub-tile r / 128, row r % 128
+    // ------------------------------------------------------------ weight dequantization (A tiles): thread = (row, block)
+    const int w2 = warp - 2;                         // 0 .. kDequantWarps-1
+    const int r = (w2 % (FT * 4)) * 32 + lane;       // row of the CTA tile: sub-tile r / 128, row r % 128
+    const int hb = w2 / (FT * 4);                    // which of the two 32-k blocks of a k-step
     const int grow = row0 + r;
     const bool valid = grow < n_rows;
     const int K = p.K, nblk = K / 32;
     const uint8_t* crow = p.seg[sg].base + (size_t)(valid ? grow : 0) * (K / 2);
     const __half* srow = reinterpret_cast<const __half*>(p.seg[sg].base + (size_t)n_rows * (K / 2)) + (size_t)(valid ? grow : 0) * nblk;
-    uint4 q0, q1;
-    uint32_t sc;
-    auto fetch = [&](int ks) {
-      const int kb = ks * 2;  // first block of the k-step
-      q0 = make_uint4(0, 0, 0, 0);
-      q1 = q0;
+    // Packed weights are fetched kPD k-steps ahead into registers: a k-step lasts about a thousand cycles, less than
+    // the latency of a first-touch DRAM read under load.
+    constexpr int kPD = 4;
+    uint4 qbuf[kPD];
+    uint32_t sbuf[kPD];
+    auto fetch = [&](int ks, uint4& q, uint32_t& sc) {
+      const int kb = ks * 2 + hb;
+      q = make_uint4(0, 0, 0, 0);
       sc = 0;
       if (valid && kb < nblk) {
-        q0 = __ldg(reinterpret_cast<const uint4*>(crow + (size_t)kb * 16));
+        q = __ldg(reinterpret_cast<const uint4*>(crow + (size_t)kb * 16));
         sc = (uint32_t)__half_as_ushort(srow[kb]);
-        if (kb + 1 < nblk) {
-          q1 = __ldg(reinterpret_cast<const uint4*>(crow + (size_t)(kb + 1) * 16));
-          sc |= (uint32_t)__half_as_ushort(srow[kb + 1]) << 16;
-        }
       }
     };
-    if (nks > 0) fetch(ks0);
+#pragma unroll
+    for (int d = 0; d < kPD; ++d) {
+      qbuf[d] = make_uint4(0, 0, 0, 0);
+      sbuf[d] = 0;
+      if (d < nks) fetch(ks0 + d, qbuf[d], sbuf[d]);
+    }
     bool ok = true;
-    for (int i = 0; i < nks; ++i) {
-      const int s = i % S;
-      const uint4 c0 = q0, c1 = q1;
-      const uint32_t scw = sc;
-      if (i + 1 < nks) fetch(ks0 + i + 1);  // next k-step's packed weights are in flight while this one is expanded
-      if (i >= S && !mbar_wait(&empty[s], ((i / S) - 1) & 1)) {
-        fail_s = 1;
-        ok = false;
-        break;
+    for (int i0 = 0; i0 < nks && ok; i0 += kPD) {
+#pragma unroll
+      for (int d = 0; d < kPD; ++d) {
+        const int i = i0 + d;
+        if (i >= nks || !ok) break;
+        const int s = i % S;
+        const uint4 c0 = qbuf[d];
+        const uint32_t scw = sbuf[d];
+        if (i + kPD < nks) fetch(ks0 + i + kPD, qbuf[d], sbuf[d]);
+        if (i >= S) {
+          // one lane polls for the warp: hundreds of threads hammering the same mbarrier word slow its arrivals down
+          int got = 1;
+          if (lane == 0) got = mbar_wait(&empty[s], ((i / S) - 1) & 1) ? 1 : 0;
+          got = __shfl_sync(0xffffffffu, got, 0);
+          if (!got) {
+            fail_s = 1;
+            ok = false;
+            break;
+          }
+        }
+        uint8_t* arow = smem + (size_t)s * kStageBytes + (size_t)r * 128;  // sub-tiles are contiguous: row r at r * 128
+        const __half2 s0 = __half2half2(__ushort_as_half((unsigned short)(scw & 0xFFFF)));
+        const int sw = r & 7, cb = hb * 4;
+        *reinterpret_cast<uint4*>(arow + (((cb + 0) ^ sw) << 4)) = dequant8(c0.x, s0);
+        *reinterpret_cast<uint4*>(arow + (((cb + 1) ^ sw) << 4)) = dequant8(c0.y, s0);
+        *reinterpret_cast<uint4*>(arow + (((cb + 2) ^ sw) << 4)) = dequant8(c0.z, s0);
+        *reinterpret_cast<uint4*>(arow + (((cb + 3) ^ sw) << 4)) = dequant8(c0.w, s0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core's reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full_a[s]);  // one arrival per warp: an mbarrier retires only a few arrivals per cycle
       }
-      uint8_t* arow = smem + (size_t)s * kStageBytes + (size_t)r * 128;  // sub-tiles are contiguous: row r at r * 128
-      const __half2 s0 = __half2half2(__ushort_as_half((unsigned short)(scw & 0xFFFF)));
-      const __half2 s1 = __half2half2(__ushort_as_half((unsigned short)(scw >> 16)));
-      const int sw = r & 7;
-      *reinterpret_cast<uint4*>(arow + ((0 ^ sw) << 4)) = dequant8(c0.x, s0);
-      *reinterpret_cast<uint4*>(arow + ((1 ^ sw) << 4)) = dequant8(c0.y, s0);
-      *reinterpret_cast<uint4*>(arow + ((2 ^ sw) << 4)) = dequant8(c0.z, s0);
-      *reinterpret_cast<uint4*>(arow + ((3 ^ sw) << 4)) = dequant8(c0.w, s0);
-      *reinterpret_cast<uint4*>(arow + ((4 ^ sw) << 4)) = dequant8(c1.x, s1);
-      *reinterpret_cast<uint4*>(arow + ((5 ^ sw) << 4)) = dequant8(c1.y, s1);
-      *reinterpret_cast<uint4*>(arow + ((6 ^ sw) << 4)) = dequant8(c1.z, s1);
-      *reinterpret_cast<uint4*>(arow + ((7 ^ sw) << 4)) = dequant8(c1.w, s1);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core's reads
-      mbar_arrive(&full_a[s]);
     }
     // ------------------------------------------------------------ epilogue: accumulator rows -> Y (transposed)
-    if (ok && nks > 0 && mbar_wait(&acc_full, 0)) {
+    int acc_ready = 0;
+    if (ok && nks > 0) {
+      if (lane == 0) acc_ready = mbar_wait(&acc_full, 0) ? 1 : 0;
+      acc_ready = __shfl_sync(0xffffffffu, acc_ready, 0);
+    }
+    if (acc_ready) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int q = warp & 3;               // TMEM lane quarter this warp may read
-      const int ft = (warp - 2) >> 2;       // feature sub-tile = accumulator
+      const int ft = (w2 >> 2) % FT;        // feature sub-tile = accumulator
+      const int ch = w2 / (FT * 4);         // which half of the token columns
       const int f = ft * BM + q * 32 + lane;
       const bool fvalid = row0 + f < n_rows;
       const int col = p.seg[sg].col0 + row0 + f;
       if (ft < n_ft) {
-        for (int c0 = 0; c0 < nmma; c0 += 32) {
+        for (int c0 = ch * (TACC / 2); c0 < min(nmma, (ch + 1) * (TACC / 2)); c0 += 32) {
           uint32_t v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ft * TACC + c0), v);
           if (fvalid) {
@@ -353,6 +382,12 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+// The wide configuration when its tiles alone fill most of the GPU, else the narrow one.
+bool use_wide_tiles(int n_total, int T, int sm_count) {
+  const int wide = ((n_total + 255) / 256) * ((T + 255) / 256);
+  return wide * 10 >= sm_count * 9;
+}
+
 int pick_splits(int tiles, int total_ksteps, int sm_count) {
   int s = 1;
   while (tiles * s < sm_count && s < 8 && total_ksteps % (s * 2) == 0 && total_ksteps / (s * 2) >= 8) s *= 2;
@@ -366,7 +401,9 @@ uint64_t gemm_scratch_bytes(int T, int n_total, int K) {
   // fp32 partials of the split choice for this shape (fewer tiles can only mean more splits, so the tile count of the
   // concatenated rows bounds it from above); the launcher falls back to one split if the buffer it gets is smaller
   const int total_ksteps = (K + BK - 1) / BK;
-  const int tiles = ((n_total + BF - 1) / BF) * ((T + TTILE - 1) / TTILE);
+  const bool wide = use_wide_tiles(n_total, T, 148);
+  const int bf = wide ? 256 : 128, tt = wide ? 256 : 128;
+  const int tiles = ((n_total + bf - 1) / bf) * ((T + tt - 1) / tt);
   const int s = pick_splits(tiles, total_ksteps, 148);
   return s > 1 ? (uint64_t)s * T * n_total * 4 + 256 : 256;
 }
@@ -391,21 +428,25 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
     if (err) *err = "cuTensorMapEncodeTiled failed for the activation tile";
     return cudaErrorInvalidValue;
   }
+  int sm_count = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  int n_total = 0;
+  for (int i = 0; i < g.n_seg; ++i) n_total += g.seg[i].n_rows;
+  const bool wide = use_wide_tiles(n_total, g.T, sm_count);
+  const int bf = wide ? 256 : 128, tt = wide ? 256 : 128;
   GemmKParams p{};
   p.n_seg = g.n_seg;
   int tiles = 0, col = 0;
   for (int i = 0; i < g.n_seg; ++i) {
     p.seg[i] = GemmSeg{g.seg[i].base, g.seg[i].n_rows, tiles, col};
-    tiles += (g.seg[i].n_rows + BF - 1) / BF;
+    tiles += (g.seg[i].n_rows + bf - 1) / bf;
     col += g.seg[i].n_rows;
   }
-  const int tchunks = (g.T + TTILE - 1) / TTILE;
+  const int tchunks = (g.T + tt - 1) / tt;
   p.K = g.K;
   p.T = g.T;
   p.total_ksteps = (g.K + BK - 1) / BK;
-  int sm_count = 148;
-  int dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   p.splits = pick_splits(tiles * tchunks, p.total_ksteps, sm_count);
   if (p.splits > 1 && (uint64_t)p.splits * g.T * g.ldy * 4 > g.scratch_bytes) p.splits = 1;
   p.ksteps_per_split = (p.total_ksteps + p.splits - 1) / p.splits;
@@ -413,16 +454,24 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   p.ldy = g.ldy;
   p.partial = (float*)g.scratch;
   p.status = g.status;
-  p.stages = kMaxStages;
-  const size_t smem = (size_t)p.stages * kStageBytes + 1024;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_q4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
+    cudaError_t e1 = cudaFuncSetAttribute(gemm_q4_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e2 = cudaFuncSetAttribute(gemm_q4_kernel<1, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e1 != cudaSuccess) return e1;
+    if (e2 != cudaSuccess) return e2;
     attr_set = true;
   }
   dim3 grid(tiles, tchunks, p.splits);
-  gemm_q4_kernel<<<grid, kGemmThreads, smem, st>>>(xmap, p);
+  if (wide) {
+    using Cfg = TileCfg<2, 256>;
+    p.stages = Cfg::kStages;
+    gemm_q4_kernel<2, 256><<<grid, Cfg::kThreads, (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st>>>(xmap, p);
+  } else {
+    using Cfg = TileCfg<1, 128>;
+    p.stages = Cfg::kStages;
+    gemm_q4_kernel<1, 128><<<grid, Cfg::kThreads, (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st>>>(xmap, p);
+  }
   ++*n_launch;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -438,8 +487,8 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
 
 // ---------------------------------------------------------------------------------------------------------------
 // Split-K scratch that needs no allocation: a fixed array in the library's own device image.
-// Every GPU that loads the library carries these 32 MiB from load until exit.
-constexpr uint64_t kStaticScratchBytes = 32ull << 20;
+// Every GPU that loads the library carries these 8 MiB from load until exit.
+constexpr uint64_t kStaticScratchBytes = 8ull << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 uint64_t gemm_static_scratch_capacity() { return kStaticScratchBytes; }

@@ -52,10 +52,11 @@ def test_static_scratch_linear_equals_linear_twice_in_a_row():
 def test_static_scratch_rejects_what_it_cannot_hold_and_host_placed_tensors():
     import torch
     from paper_2607_10183_b200 import binding as B
-    N, K = 2048, 4096  # 16 feature tiles -> 8 splits; with T = 1024 the partials need 8 * 1024 * 2048 * 4 B = 64 MiB > 32 MiB
+    N, K = 1024, 4096  # 8 x 8 tiles of 128 x 128 -> 4 splits; the partials need 4 * 1024 * 1024 * 4 B = 16 MiB > 8 MiB
     packed, scales = W.q4_packed(77, 1, W.ROLE_Q, N, K)
     nb = W.q4_bytes(N, K)
     ctx = B.Context(4 * MB + 2 * (nb + 256) + nb + MB, workspace_bytes=4 * MB, ring_slots=2, slot_bytes=nb)
+    assert B.lib.ats_linear_static_scratch is not None
     tid = ctx.register_q4(packed, scales)
     ctx.set_placement([(tid, -1, B.ATS_GPU)])
     T = 1024
