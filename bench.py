@@ -186,6 +186,21 @@ def build_dense_replicas(B, W, n_layers, cfg, kv_cap, ring_slots=0, slot_bytes=0
     return ctx, descs, q4_ids, layer_bytes
 
 
+def max_over_ranks(dist, value, device="cpu"):
+    """The slowest rank's time: every multi-rank number is the max over ranks (no-op without a process group)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(world, units_per_rank, seconds):
+    """Whole-job throughput of `world` independent replicas (weak scaling): all ranks' units over the slowest rank's time."""
+    return world * units_per_rank / seconds
+
+
 def event_time_ms(torch, stream, fn):
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -311,7 +326,7 @@ def extra_stream(torch, B, W, peaks, quick, n_layers=None):
     """Config 5: a stack of dense layers under a 60 % byte budget chosen by the library's placement DP (Algorithm 1);
     the rest sits in pinned host memory and is streamed every decode step, overlapped with compute."""
     shape = W.DENSE_FULL
-    L = n_layers or (4 if quick else 8)
+    L = n_layers or STACK_LAYERS[0] or (4 if quick else 8)
     cap, pos0 = 640, 512
     slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
     ctx, descs, q4_ids, layer_bytes = build_dense_replicas(B, W, L, 5, cap, ring_slots=8, slot_bytes=slot, chunk_bytes=8 << 20)
@@ -349,6 +364,7 @@ def extra_stream(torch, B, W, peaks, quick, n_layers=None):
             "frac_of_measured_pcie": streamed / dt / 1e9 / pcie, "fully_overlapped_at_80pct": bool(dt <= streamed / (0.8 * pcie * 1e9))}
 
 
+STACK_LAYERS = [0]
 EXTRAS = {"cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
 
 
@@ -400,12 +416,9 @@ def run_ours(args):
     t_wall1 = time.time()
     barrier()
     launches = ctx.stats().kernel_launches
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(dist, ms, "cuda")
     clocks = sampler.summary(t_wall0, t_wall1)
-    tok_s = world * args.steps / (ms * 1e-3)
+    tok_s = aggregate_throughput(world, args.steps, ms * 1e-3)
 
     # ---- roofline of the dominant kernel family (the GEMV: 4 of the 5 launches of a step, 81 % of its time).
     # Its average launch duration is measured live with CUDA events over a timed region of the same steps in which the
@@ -453,11 +466,8 @@ def run_ours(args):
     e2e_steps(n_e2e, 50)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * n_e2e / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": int(x_host.numel() * 2),
+    e2e_s = max_over_ranks(dist, e2e_s, "cuda")
+    e2e = {"value": aggregate_throughput(world, n_e2e, e2e_s), "unit": "tokens/s", "h2d_bytes_per_step": int(x_host.numel() * 2),
            "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": n_e2e}
     ctx.close()
     del ctx, caches
@@ -505,9 +515,11 @@ def main():
     ap.add_argument("--quick", action="store_true", help="smaller extras")
     ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream"],
                     help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
+    ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = 8, or 4 with --quick; 32 = the full configuration)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    STACK_LAYERS[0] = args.stack_layers
     if args.only_extra:
         import torch
         from paper_2607_10183_b200 import binding as B, workloads as W
