@@ -225,71 +225,114 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
     if (lane == 0) {
       bool ok = true;
       const uint32_t idesc = umma_idesc(nmma);
-      for (int i = 0; i < nks && ok; ++i) {
-        const int s = i % S;
-        const uint32_t par = (i / S) & 1;
+      // Descriptors differ from stage to stage and from MMA to MMA only in the 14-bit start-address field, so each is
+      // one 32-bit add on the low word: the loop stays a handful of instructions per MMA and the issuing thread keeps
+      // the tensor pipe fed even when the other warps of its scheduler are busy.
+      const uint64_t desc0 = umma_desc(smem_u32(smem));
+      uint32_t accum = 0;
+      int s = 0;
+      uint32_t par = 0;
+      for (int i = 0; i < nks; ++i) {
         if (!mbar_wait(&full_a[s], par) || !mbar_wait(&full_b[s], par)) {
           fail_s = 1;
           ok = false;
           break;
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_addr = smem_u32(smem + (size_t)s * kStageBytes);
-        const uint64_t bdesc = umma_desc(a_addr + FT * A_BYTES);
+        const uint64_t adesc = desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kStageBytes >> 4));
+        const uint64_t bdesc = adesc + (uint64_t)((FT * A_BYTES) >> 4);
+        if (n_ft == FT) {
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk) {
-          for (int ft = 0; ft < n_ft; ++ft)
-            umma_f16(tmem_base + (uint32_t)(ft * TACC), umma_desc(a_addr + ft * A_BYTES) + 2 * kk, bdesc + 2 * kk, idesc,
-                     (i > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < BK / 16; ++kk) {
+#pragma unroll
+            for (int ft = 0; ft < FT; ++ft) {
+              umma_f16(tmem_base + (uint32_t)(ft * TACC), adesc + (uint64_t)(ft * (A_BYTES >> 4) + 2 * kk), bdesc + (uint64_t)(2 * kk), idesc,
+                       kk > 0 ? 1u : accum);
+            }
+          }
+          accum = 1;
+        } else {
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            umma_f16(tmem_base, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), idesc, kk > 0 ? 1u : accum);
+          }
+          accum = 1;
         }
         umma_commit(&empty[s]);  // arrives when the MMAs reading stage s are done
+        if (++s == S) {
+          s = 0;
+          par ^= 1;
+        }
       }
       if (ok) umma_commit(&acc_full);
     }
   } else {
     // ------------------------------------------------------------ weight dequantization (A tiles): thread = (row, block)
+    // Two adjacent lanes share a weight row (one 32-k block of the k-step each), so a warp's 16-byte loads touch 16
+    // cache lines instead of 32: the L1 tag stage, which takes a cycle per distinct line, is the busiest unit here.
     const int w2 = warp - 2;                         // 0 .. kDequantWarps-1
-    const int r = (w2 % (FT * 4)) * 32 + lane;       // row of the CTA tile: sub-tile r / 128, row r % 128
-    const int hb = w2 / (FT * 4);                    // which of the two 32-k blocks of a k-step
+    const int r = w2 * 16 + (lane >> 1);             // row of the CTA tile: sub-tile r / 128, row r % 128
+    const int hb = lane & 1;                         // which of the two 32-k blocks of a k-step
     const int grow = row0 + r;
     const bool valid = grow < n_rows;
     const int K = p.K, nblk = K / 32;
     const uint8_t* crow = p.seg[sg].base + (size_t)(valid ? grow : 0) * (K / 2);
     const __half* srow = reinterpret_cast<const __half*>(p.seg[sg].base + (size_t)n_rows * (K / 2)) + (size_t)(valid ? grow : 0) * nblk;
     // Packed weights are fetched kPD k-steps ahead into registers: a k-step lasts about a thousand cycles, less than
-    // the latency of a first-touch DRAM read under load.
+    // the latency of a first-touch DRAM read under load.  Scales come as one 16-byte load per row for four k-steps
+    // (eight blocks) when the row's scale array is 16-byte aligned, else one fp16 at a time.
     constexpr int kPD = 4;
+    const bool vec_sc = (K % 256 == 0) && (ks0 % kPD == 0);
     uint4 qbuf[kPD];
     uint32_t sbuf[kPD];
-    auto fetch = [&](int ks, uint4& q, uint32_t& sc) {
+    uint4 snext = make_uint4(0, 0, 0, 0);
+    auto fetch_codes = [&](int ks, uint4& q) {
       const int kb = ks * 2 + hb;
       q = make_uint4(0, 0, 0, 0);
-      sc = 0;
-      if (valid && kb < nblk) {
-        q = __ldg(reinterpret_cast<const uint4*>(crow + (size_t)kb * 16));
-        sc = (uint32_t)__half_as_ushort(srow[kb]);
-      }
+      if (valid && kb < nblk) q = __ldg(reinterpret_cast<const uint4*>(crow + (size_t)kb * 16));
     };
+    auto fetch_scale1 = [&](int ks) -> uint32_t {
+      const int kb = ks * 2 + hb;
+      return (valid && kb < nblk) ? (uint32_t)__half_as_ushort(srow[kb]) : 0u;
+    };
+    auto fetch_scale8 = [&](int ks) -> uint4 {  // ks a multiple of kPD: blocks 2 ks .. 2 ks + 7
+      return (valid && ks * 2 < nblk) ? __ldg(reinterpret_cast<const uint4*>(srow + ks * 2)) : make_uint4(0, 0, 0, 0);
+    };
+    auto pick = [&](const uint4& v, int d) -> uint32_t {  // the scale of block 2 d + hb of the eight
+      const uint32_t w = d == 0 ? v.x : d == 1 ? v.y : d == 2 ? v.z : v.w;
+      return (w >> (16 * hb)) & 0xFFFFu;
+    };
+    if (vec_sc) snext = fetch_scale8(ks0);
 #pragma unroll
     for (int d = 0; d < kPD; ++d) {
       qbuf[d] = make_uint4(0, 0, 0, 0);
       sbuf[d] = 0;
-      if (d < nks) fetch(ks0 + d, qbuf[d], sbuf[d]);
+      if (d < nks) {
+        fetch_codes(ks0 + d, qbuf[d]);
+        sbuf[d] = vec_sc ? pick(snext, d) : fetch_scale1(ks0 + d);
+      }
     }
     bool ok = true;
+    int s = 0, round = 0;
+    const int sw = r & 7, cb = hb * 4;
     for (int i0 = 0; i0 < nks && ok; i0 += kPD) {
+      if (vec_sc && i0 + kPD < nks) snext = fetch_scale8(ks0 + i0 + kPD);
 #pragma unroll
       for (int d = 0; d < kPD; ++d) {
         const int i = i0 + d;
         if (i >= nks || !ok) break;
-        const int s = i % S;
         const uint4 c0 = qbuf[d];
-        const uint32_t scw = sbuf[d];
-        if (i + kPD < nks) fetch(ks0 + i + kPD, qbuf[d], sbuf[d]);
-        if (i >= S) {
+        const __half2 s0 = __half2half2(__ushort_as_half((unsigned short)sbuf[d]));
+        if (i + kPD < nks) {
+          fetch_codes(ks0 + i + kPD, qbuf[d]);
+          if (!vec_sc) sbuf[d] = fetch_scale1(ks0 + i + kPD);
+        }
+        // the arithmetic needs no shared memory: do it before waiting for the stage to drain
+        const uint4 o0 = dequant8(c0.x, s0), o1 = dequant8(c0.y, s0), o2 = dequant8(c0.z, s0), o3 = dequant8(c0.w, s0);
+        if (round > 0) {
           // one lane polls for the warp: hundreds of threads hammering the same mbarrier word slow its arrivals down
           int got = 1;
-          if (lane == 0) got = mbar_wait(&empty[s], ((i / S) - 1) & 1) ? 1 : 0;
+          if (lane == 0) got = mbar_wait(&empty[s], (uint32_t)(round - 1) & 1u) ? 1 : 0;
           got = __shfl_sync(0xffffffffu, got, 0);
           if (!got) {
             fail_s = 1;
@@ -298,15 +341,21 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
           }
         }
         uint8_t* arow = smem + (size_t)s * kStageBytes + (size_t)r * 128;  // sub-tiles are contiguous: row r at r * 128
-        const __half2 s0 = __half2half2(__ushort_as_half((unsigned short)(scw & 0xFFFF)));
-        const int sw = r & 7, cb = hb * 4;
-        *reinterpret_cast<uint4*>(arow + (((cb + 0) ^ sw) << 4)) = dequant8(c0.x, s0);
-        *reinterpret_cast<uint4*>(arow + (((cb + 1) ^ sw) << 4)) = dequant8(c0.y, s0);
-        *reinterpret_cast<uint4*>(arow + (((cb + 2) ^ sw) << 4)) = dequant8(c0.z, s0);
-        *reinterpret_cast<uint4*>(arow + (((cb + 3) ^ sw) << 4)) = dequant8(c0.w, s0);
+        *reinterpret_cast<uint4*>(arow + (((cb + 0) ^ sw) << 4)) = o0;
+        *reinterpret_cast<uint4*>(arow + (((cb + 1) ^ sw) << 4)) = o1;
+        *reinterpret_cast<uint4*>(arow + (((cb + 2) ^ sw) << 4)) = o2;
+        *reinterpret_cast<uint4*>(arow + (((cb + 3) ^ sw) << 4)) = o3;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core's reads
         __syncwarp();
         if (lane == 0) mbar_arrive(&full_a[s]);  // one arrival per warp: an mbarrier retires only a few arrivals per cycle
+        if (++s == S) {
+          s = 0;
+          ++round;
+        }
+      }
+      if (vec_sc) {
+#pragma unroll
+        for (int d = 0; d < kPD; ++d) sbuf[d] = pick(snext, d);
       }
     }
     // ------------------------------------------------------------ epilogue: accumulator rows -> Y (transposed)
