@@ -1,18 +1,19 @@
 // Dequantize-fused prefill GEMM on the 5th-generation tensor cores (sm_100a): Y[T][N] = X[T][K] * W^T, fp16 operands,
 // fp32 accumulation in tensor memory, fp16 output.
 //
-// One CTA computes a tile of 256 output features x up to 256 tokens over a K range (split-K when the tiles do not fill
-// the GPU).  The weight tile is the MMA A operand, as two 128-row sub-tiles that share one activation tile (which halves
-// the activation bytes re-read from L2 per flop): sixteen warps read the packed 4-bit codes and fp16 scales straight from
-// global memory (two threads per weight row, one 32-k block each per stage), expand them to fp16 (w = rn16(scale * code), a single rounding) and store
-// them into shared memory in the canonical K-major 128-byte-swizzle layout the tensor core reads.  The activation tile is
-// the B operand, loaded by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-range rows zero-filled).  A single thread
-// issues tcgen05.mma (M = 128, N = tokens, K = 16 per instruction) into two 256-column accumulators in TMEM (all 512
-// columns); tcgen05.commit releases the stage to the producers through an mbarrier.  The sixteen dequantization warps then
-// become the epilogue: tcgen05.ld brings the accumulator rows back (lane = feature, columns = tokens) and writes Y (or
-// an fp32 split-K partial that a second kernel sums in split order).
+// One CTA computes a tile of 256 tokens x 256 output features (or 128 x 128) over a K range (split-K when the tiles do
+// not fill the GPU).  The activation tile is the MMA A operand (M = 128 tokens per instruction, two token blocks share
+// one weight tile), loaded by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-range rows zero-filled).  The weight
+// tile is the B operand (N = features): sixteen warps read the packed 4-bit codes and fp16 scales straight from global
+// memory (two threads per weight row, one 32-k block each per stage), expand them to fp16 (w = rn16(scale * code), a
+// single rounding) and store them into shared memory in the canonical K-major 128-byte-swizzle layout the tensor core
+// reads.  A single thread issues tcgen05.mma (K = 16 per instruction) into one accumulator per token block in TMEM;
+// tcgen05.commit releases the stage to the producers through an mbarrier.  The dequantization warps then become the
+// epilogue: tcgen05.ld brings the accumulator back with lane = token and columns = features, so each thread holds runs
+// of consecutive features of one output row and writes Y (or an fp32 split-K partial that a second kernel sums in split
+// order) in 16-byte pieces.
 //
-// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..17 = weight dequantization, then epilogue.
+// Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2.. = weight dequantization, then epilogue.
 // No cluster launch and no multicast.  Every mbarrier wait is bounded; on expiry the CTA raises the status word, skips
 // the rest of its work, frees its tensor memory and returns.
 #include <cuda.h>
@@ -23,15 +24,14 @@ namespace ats {
 
 namespace {
 
-constexpr int BM = 128;         // features per MMA (M)
+constexpr int BM = 128;         // tokens per MMA (M); also the granule of the feature tile
 constexpr int BK = 64;          // k per stage: 64 fp16 = one 128-byte swizzle row
 constexpr int BOXR = 64;        // activation rows per TMA box
 constexpr int A_BYTES = BM * BK * 2;        // 16 KB per 128-row feature sub-tile
 constexpr int kMaxStages = 6;
-// Two tile configurations <FT, TT>: FT 128-row feature sub-tiles (one accumulator each) x TT tokens per CTA.
-//   <2, 256>: 256 x 256, 3 stages of 64 KB, all 512 TMEM columns - for operators with enough feature tiles to fill the GPU
-//   <1, 128>: 128 x 128, 6 stages of 32 KB, 128 TMEM columns    - four times the CTAs for the narrow operators, which
-//             would otherwise need split-K and its fp32 partial traffic
+// Two tile configurations <FT, TT>: FT * 128 features x TT tokens per CTA (TT / 128 accumulators of FT * 128 columns).
+//   <2, 256>: 256 x 256, 3 stages of 64 KB, all 512 TMEM columns
+//   <1, 128>: 128 x 128, 6 stages of 32 KB, 128 TMEM columns
 template <int FT, int TT>
 struct TileCfg {
   static constexpr int BF = BM * FT;                      // features per CTA
@@ -160,7 +160,7 @@ __device__ __forceinline__ uint4 dequant8(uint32_t w, __half2 s2) {
 template <int FT, int TT>
 __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const GemmKParams p) {
   using Cfg = TileCfg<FT, TT>;
-  constexpr int BF = Cfg::BF, TTILE = TT, TACC = TT, kDequantWarps = Cfg::kDequantWarps, kStageBytes = Cfg::kStageBytes;
+  constexpr int BF = Cfg::BF, TTILE = TT, MB = TT / BM, kDequantWarps = Cfg::kDequantWarps, kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_a[kMaxStages], full_b[kMaxStages], empty[kMaxStages], acc_full;
@@ -176,9 +176,9 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
   const int n_rows = p.seg[sg].n_rows;
   const int t0 = blockIdx.y * TTILE;
   const int Tt = min(TTILE, p.T - t0);
-  const int nmma = (Tt + 15) / 16 * 16;          // MMA N
-  const int boxes = (Tt + BOXR - 1) / BOXR;      // TMA boxes of 64 activation rows
-  const int n_ft = row0 + BM < n_rows ? FT : 1;  // feature sub-tiles that hold real rows
+  const int nmma = min(BF, (n_rows - row0 + 15) / 16 * 16);  // MMA N: the features of this tile that hold real rows
+  const int boxes = (Tt + BOXR - 1) / BOXR;                  // TMA boxes of 64 activation rows
+  const int n_mb = (Tt + BM - 1) / BM;                       // 128-token blocks (MMA M) that hold real tokens
   const int split = blockIdx.z;
   const int ks0 = split * p.ksteps_per_split;
   const int nks = min(p.ksteps_per_split, p.total_ksteps - ks0);
@@ -239,25 +239,22 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
           break;
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t adesc = desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kStageBytes >> 4));
-        const uint64_t bdesc = adesc + (uint64_t)((FT * A_BYTES) >> 4);
-        if (n_ft == FT) {
+        const uint64_t wdesc = desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kStageBytes >> 4));  // weight tile: the B operand
+        const uint64_t xdesc = wdesc + (uint64_t)((FT * A_BYTES) >> 4);                         // activation tile: the A operand
+        if (n_mb == MB) {
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk) {
 #pragma unroll
-            for (int ft = 0; ft < FT; ++ft) {
-              umma_f16(tmem_base + (uint32_t)(ft * TACC), adesc + (uint64_t)(ft * (A_BYTES >> 4) + 2 * kk), bdesc + (uint64_t)(2 * kk), idesc,
+            for (int mb = 0; mb < MB; ++mb)
+              umma_f16(tmem_base + (uint32_t)(mb * BF), xdesc + (uint64_t)(mb * (A_BYTES >> 4) + 2 * kk), wdesc + (uint64_t)(2 * kk), idesc,
                        kk > 0 ? 1u : accum);
-            }
           }
-          accum = 1;
         } else {
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            umma_f16(tmem_base, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), idesc, kk > 0 ? 1u : accum);
-          }
-          accum = 1;
+          for (int kk = 0; kk < BK / 16; ++kk)
+            umma_f16(tmem_base, xdesc + (uint64_t)(2 * kk), wdesc + (uint64_t)(2 * kk), idesc, kk > 0 ? 1u : accum);
         }
+        accum = 1;
         umma_commit(&empty[s]);  // arrives when the MMAs reading stage s are done
         if (++s == S) {
           s = 0;
@@ -366,26 +363,48 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
     }
     if (acc_ready) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      // accumulator mb: lane = token of the 128-token block, columns = features, so a thread holds 32 consecutive
+      // features of one token and writes them as 16-byte pieces
       const int q = warp & 3;               // TMEM lane quarter this warp may read
-      const int ft = (w2 >> 2) % FT;        // feature sub-tile = accumulator
-      const int ch = w2 / (FT * 4);         // which half of the token columns
-      const int f = ft * BM + q * 32 + lane;
-      const bool fvalid = row0 + f < n_rows;
-      const int col = p.seg[sg].col0 + row0 + f;
-      if (ft < n_ft) {
-        for (int c0 = ch * (TACC / 2); c0 < min(nmma, (ch + 1) * (TACC / 2)); c0 += 32) {
+      const int mb = (w2 >> 2) % MB;        // token block = accumulator
+      const int ch = w2 / (MB * 4);         // which half of the feature columns
+      const int t = t0 + mb * BM + q * 32 + lane;
+      const bool tvalid = t < p.T;
+      const int colbase = p.seg[sg].col0 + row0;
+      const bool vec = (p.ldy % 8 == 0) && (colbase % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+      if (mb < n_mb) {
+        for (int c0 = ch * (BF / 2); c0 < min(nmma, (ch + 1) * (BF / 2)); c0 += 32) {
           uint32_t v[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ft * TACC + c0), v);
-          if (fvalid) {
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mb * BF + c0), v);
+          if (!tvalid) continue;
+          const int nf = min(32, n_rows - row0 - c0);  // features of this chunk that exist
+          if (p.splits > 1) {
+            float* dst = p.partial + ((size_t)split * p.T + t) * p.ldy + colbase + c0;
+            if (vec && nf == 32) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const int t = t0 + c0 + e;
-              if (t < p.T) {
-                if (p.splits > 1)
-                  p.partial[((size_t)split * p.T + t) * p.ldy + col] = __uint_as_float(v[e]);
-                else
-                  p.y[(size_t)t * p.ldy + col] = __float2half_rn(__uint_as_float(v[e]));
+              for (int e = 0; e < 32; e += 4) *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (e < nf) dst[e] = __uint_as_float(v[e]);
+            }
+          } else {
+            __half* dst = p.y + (size_t)t * p.ldy + colbase + c0;
+            if (vec && nf == 32) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 8) {
+                uint32_t o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const __half2 h = __floats2half2_rn(__uint_as_float(v[e + 2 * j]), __uint_as_float(v[e + 2 * j + 1]));
+                  o[j] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                *reinterpret_cast<uint4*>(dst + e) = make_uint4(o[0], o[1], o[2], o[3]);
               }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (e < nf) dst[e] = __float2half_rn(__uint_as_float(v[e]));
             }
           }
         }
@@ -402,15 +421,40 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
   }
 }
 
-// y[t][c] = rn16(sum_s partial[s][t][c]) for c < n_cols, splits summed in ascending order
+// y[t][c] = rn16(sum_s partial[s][t][c]) for c < n_cols, splits summed in ascending order; eight columns per thread when
+// the row length allows 16-byte accesses
 __global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, __half* __restrict__ y, int T, int n_cols, int ldy,
                                           int splits) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  const size_t plane = (size_t)T * ldy;
+  if (n_cols % 8 == 0 && ldy % 8 == 0) {
+    const int cg = n_cols / 8;
+    const size_t total = (size_t)T * cg;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+      const size_t t = i / cg, c = (i % cg) * 8;
+      const float* src = partial + t * ldy + c;
+      float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
+      for (int s = 1; s < splits; ++s) {
+        const float4 a2 = *reinterpret_cast<const float4*>(src + s * plane), b2 = *reinterpret_cast<const float4*>(src + s * plane + 4);
+        a.x += a2.x; a.y += a2.y; a.z += a2.z; a.w += a2.w;
+        b.x += b2.x; b.y += b2.y; b.z += b2.z; b.w += b2.w;
+      }
+      const __half2 h0 = __floats2half2_rn(a.x, a.y), h1 = __floats2half2_rn(a.z, a.w), h2 = __floats2half2_rn(b.x, b.y),
+                    h3 = __floats2half2_rn(b.z, b.w);
+      uint4 o;
+      o.x = *reinterpret_cast<const uint32_t*>(&h0);
+      o.y = *reinterpret_cast<const uint32_t*>(&h1);
+      o.z = *reinterpret_cast<const uint32_t*>(&h2);
+      o.w = *reinterpret_cast<const uint32_t*>(&h3);
+      *reinterpret_cast<uint4*>(y + t * ldy + c) = o;
+    }
+    return;
+  }
   const size_t total = (size_t)T * n_cols;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t t = i / n_cols, c = i % n_cols;
     float acc = 0.f;
-    for (int s = 0; s < splits; ++s) acc += partial[((size_t)s * T + t) * ldy + c];
+    for (int s = 0; s < splits; ++s) acc += partial[(size_t)s * plane + t * ldy + c];
     y[t * ldy + c] = __float2half_rn(acc);
   }
 }
@@ -431,30 +475,44 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// The wide configuration when its tiles alone fill most of the GPU, else the narrow one.
-bool use_wide_tiles(int n_total, int T, int sm_count) {
-  const int wide = ((n_total + 255) / 256) * ((T + 255) / 256);
-  return wide * 10 >= sm_count * 9;
+// Tile configuration and split-K factor for one launch, picked by a small cost model (SM cycles): the CTAs run in
+// waves of sm_count; a wide k-step (256 x 256 x 64) costs about 1250 cycles and a narrow one (128 x 128 x 64) about 750,
+// both bound by the L2 traffic of the activation tile rather than by the tensor pipe, which is why few wide CTAs with
+// split-K beat many narrow ones; split-K adds the fp32 partial traffic and a second launch.
+struct GemmPlan {
+  bool wide;
+  int splits;
+};
+GemmPlan choose_plan(int tiles_wide, int tiles_narrow, int T, int n_cols, int total_ksteps, int sm_count, uint64_t scratch_bytes) {
+  GemmPlan best{false, 1};
+  double best_cost = 1e30;
+  for (int w = 0; w < 2; ++w) {
+    const int tt = w ? 256 : 128;
+    const int ctas = (w ? tiles_wide : tiles_narrow) * ((T + tt - 1) / tt);
+    const double kstep = w ? 1250.0 : 750.0;
+    for (int s = 1; s <= 8; ++s) {
+      if (s > 1 && (total_ksteps / s < 8 || (uint64_t)s * T * n_cols * 4 > scratch_bytes)) break;
+      const int per = (total_ksteps + s - 1) / s;
+      if ((s - 1) * per >= total_ksteps) continue;  // the last split would be empty
+      const int waves = (ctas * s + sm_count - 1) / sm_count;
+      double cost = (double)waves * (per * kstep + 9000.0);
+      if (s > 1) cost += 8000.0 + (double)(s + 1) * T * n_cols * 4.0 / 2000.0;  // second launch + partials at ~2 KB per cycle
+      if (cost < best_cost) {
+        best_cost = cost;
+        best = GemmPlan{w != 0, s};
+      }
+    }
+  }
+  return best;
 }
-
-int pick_splits(int tiles, int total_ksteps, int sm_count) {
-  int s = 1;
-  while (tiles * s < sm_count && s < 8 && total_ksteps % (s * 2) == 0 && total_ksteps / (s * 2) >= 8) s *= 2;
-  return s;
-}
-
 
 }  // namespace
 
 uint64_t gemm_scratch_bytes(int T, int n_total, int K) {
-  // fp32 partials of the split choice for this shape (fewer tiles can only mean more splits, so the tile count of the
-  // concatenated rows bounds it from above); the launcher falls back to one split if the buffer it gets is smaller
+  // fp32 partials of the plan this shape gets with unlimited scratch (the launcher re-plans within the buffer it is given)
   const int total_ksteps = (K + BK - 1) / BK;
-  const bool wide = use_wide_tiles(n_total, T, 148);
-  const int bf = wide ? 256 : 128, tt = wide ? 256 : 128;
-  const int tiles = ((n_total + bf - 1) / bf) * ((T + tt - 1) / tt);
-  const int s = pick_splits(tiles, total_ksteps, 148);
-  return s > 1 ? (uint64_t)s * T * n_total * 4 + 256 : 256;
+  const GemmPlan pl = choose_plan((n_total + 255) / 256, (n_total + 127) / 128, T, n_total, total_ksteps, 148, ~0ull);
+  return pl.splits > 1 ? (uint64_t)pl.splits * T * n_total * 4 + 256 : 256;
 }
 
 cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch, std::string* err) {
@@ -482,7 +540,14 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   int n_total = 0;
   for (int i = 0; i < g.n_seg; ++i) n_total += g.seg[i].n_rows;
-  const bool wide = use_wide_tiles(n_total, g.T, sm_count);
+  int tiles_w = 0, tiles_n = 0;
+  for (int i = 0; i < g.n_seg; ++i) {
+    tiles_w += (g.seg[i].n_rows + 255) / 256;
+    tiles_n += (g.seg[i].n_rows + 127) / 128;
+  }
+  const int total_ksteps = (g.K + BK - 1) / BK;
+  const GemmPlan pl = choose_plan(tiles_w, tiles_n, g.T, g.ldy, total_ksteps, sm_count, g.scratch ? g.scratch_bytes : 0);
+  const bool wide = pl.wide;
   const int bf = wide ? 256 : 128, tt = wide ? 256 : 128;
   GemmKParams p{};
   p.n_seg = g.n_seg;
@@ -495,9 +560,8 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   const int tchunks = (g.T + tt - 1) / tt;
   p.K = g.K;
   p.T = g.T;
-  p.total_ksteps = (g.K + BK - 1) / BK;
-  p.splits = pick_splits(tiles * tchunks, p.total_ksteps, sm_count);
-  if (p.splits > 1 && (uint64_t)p.splits * g.T * g.ldy * 4 > g.scratch_bytes) p.splits = 1;
+  p.total_ksteps = total_ksteps;
+  p.splits = pl.splits;
   p.ksteps_per_split = (p.total_ksteps + p.splits - 1) / p.splits;
   p.y = g.y;
   p.ldy = g.ldy;
