@@ -209,7 +209,6 @@ cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_ro
                                        uint64_t* n_launch);
 cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const __half* vc, __half* a16, int T, int n_q,
                                 int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch);
-cudaError_t launch_add16(const __half* a, const __half* b, __half* out, uint64_t n, cudaStream_t st, uint64_t* n_launch);
 cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch);
 
 // Tensor-core GEMM  Y[T][n_rows] (fp16, leading dimension ldy) = X[T][K] (fp16, ld = ldx) * W^T for up to 3 weight
@@ -226,6 +225,9 @@ struct GemmParams {
   void* scratch;
   uint64_t scratch_bytes;
   int* status;  // device word raised when a bounded wait expires
+  // optional fused residual: y2[t][c] = rn16(res[t][c] + y[t][c]) with y the fp16-rounded product (both ld = ldy)
+  const __half* res;
+  __half* y2;
 };
 uint64_t gemm_scratch_bytes(int T, int n_total, int K);
 cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);

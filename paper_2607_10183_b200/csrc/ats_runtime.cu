@@ -1197,8 +1197,11 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     g.ldx = qd;
     g.y = w.o16;
     g.ldy = H;
+    g.res = (const __half*)x_in;  // x1 = rn16(x + o) in the GEMM's own epilogue (or its split-K reduction)
+    g.y2 = w.x1_16;
     ATS_TRY(run_gemm_group(ctx, &wo, 1, g));
-    ATS_CUDA(launch_add16((const __half*)x_in, w.o16, w.x1_16, (uint64_t)T * H, ctx->cs, nl));
+    g.res = nullptr;
+    g.y2 = nullptr;
     resid = w.x1_16;
   }
   ATS_CUDA(launch_rmsnorm(resid, 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, w.h2_16, (int)T, H, L->rms_eps, ctx->cs, nl));
@@ -1212,8 +1215,9 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
   g.ldx = (int)L->ffn;
   g.y = w.d16;
   g.ldy = H;
+  g.res = resid;  // y = rn16(x1 + d)
+  g.y2 = (__half*)x_out;
   ATS_TRY(run_gemm_group(ctx, &wd, 1, g));
-  ATS_CUDA(launch_add16(resid, w.d16, (__half*)x_out, (uint64_t)T * H, ctx->cs, nl));
   return ATS_OK;
 }
 

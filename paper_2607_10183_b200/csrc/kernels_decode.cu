@@ -395,9 +395,62 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const TIn* __restrict__ x,
     out[(size_t)blockIdx.x * H + i] = __float2half_rn(load_f<TIn>(xr, i) * __half2float(gain[i]) * inv);
 }
 
+// fp16 rows of up to 8192 elements, eight per 16-byte access, held in registers between the two passes
+__global__ void __launch_bounds__(256) rmsnorm16_vec_kernel(const __half* __restrict__ x, const __half* __restrict__ gain,
+                                                            __half* __restrict__ out, int H, float eps) {
+  __shared__ float red[8];
+  const int n8 = H / 8;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)blockIdx.x * H);
+  uint4 xv[4], gv[4];
+  float ss = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = threadIdx.x + 256 * j;
+    xv[j] = make_uint4(0, 0, 0, 0);
+    gv[j] = make_uint4(0, 0, 0, 0);
+    if (c < n8) {
+      xv[j] = xr[c];
+      gv[j] = __ldg(reinterpret_cast<const uint4*>(gain) + c);
+    }
+    const uint32_t w[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float2 f = __half22float2(u32_as_half2(w[q]));
+      ss = fmaf(f.x, f.x, ss);
+      ss = fmaf(f.y, f.y, ss);
+    }
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) t += red[w];
+  const float inv = 1.0f / sqrtf(t / (float)H + eps);
+  uint4* orow = reinterpret_cast<uint4*>(out + (size_t)blockIdx.x * H);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = threadIdx.x + 256 * j;
+    if (c < n8) {
+      const uint32_t w[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w}, g[4] = {gv[j].x, gv[j].y, gv[j].z, gv[j].w};
+      uint32_t o[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 f = __half22float2(u32_as_half2(w[q])), gg = __half22float2(u32_as_half2(g[q]));
+        const __half2 h = __floats2half2_rn(f.x * gg.x * inv, f.y * gg.y * inv);
+        o[q] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      orow[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+}
+
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
                            cudaStream_t st, uint64_t* n_launch) {
-  if (x_is_f32)
+  if (!x_is_f32 && H % 8 == 0 && H <= 8192 &&
+      (((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(out)) & 15) == 0))
+    rmsnorm16_vec_kernel<<<M, 256, 0, st>>>((const __half*)x, gain, out, H, eps);
+  else if (x_is_f32)
     rmsnorm_kernel<float><<<M, 256, 0, st>>>((const float*)x, gain, out, H, eps);
   else
     rmsnorm_kernel<__half><<<M, 256, 0, st>>>((const __half*)x, gain, out, H, eps);

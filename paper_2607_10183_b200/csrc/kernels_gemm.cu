@@ -59,6 +59,8 @@ struct GemmKParams {
   float* partial;  // [splits][T][ldy] when splits > 1
   int stages;
   int* status;
+  const __half* res;  // optional residual: y2 = rn16(res + y)
+  __half* y2;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -371,7 +373,8 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
       const int t = t0 + mb * BM + q * 32 + lane;
       const bool tvalid = t < p.T;
       const int colbase = p.seg[sg].col0 + row0;
-      const bool vec = (p.ldy % 8 == 0) && (colbase % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+      const bool vec = (p.ldy % 8 == 0) && (colbase % 8 == 0) &&
+                       (((reinterpret_cast<uintptr_t>(p.y) | reinterpret_cast<uintptr_t>(p.res) | reinterpret_cast<uintptr_t>(p.y2)) & 15) == 0);
       if (mb < n_mb) {
         for (int c0 = ch * (BF / 2); c0 < min(nmma, (ch + 1) * (BF / 2)); c0 += 32) {
           uint32_t v[32];
@@ -400,11 +403,31 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
                   o[j] = *reinterpret_cast<const uint32_t*>(&h);
                 }
                 *reinterpret_cast<uint4*>(dst + e) = make_uint4(o[0], o[1], o[2], o[3]);
+                if (p.res) {
+                  const size_t off = (size_t)t * p.ldy + colbase + c0 + e;
+                  const uint4 r4 = *reinterpret_cast<const uint4*>(p.res + off);
+                  const uint32_t rr[4] = {r4.x, r4.y, r4.z, r4.w};
+                  uint32_t z[4];
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    const float2 a = __half22float2(u2h2(o[j])), b = __half22float2(u2h2(rr[j]));
+                    const __half2 h = __floats2half2_rn(b.x + a.x, b.y + a.y);
+                    z[j] = *reinterpret_cast<const uint32_t*>(&h);
+                  }
+                  *reinterpret_cast<uint4*>(p.y2 + off) = make_uint4(z[0], z[1], z[2], z[3]);
+                }
               }
             } else {
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (e < nf) dst[e] = __float2half_rn(__uint_as_float(v[e]));
+                if (e < nf) {
+                  const __half h = __float2half_rn(__uint_as_float(v[e]));
+                  dst[e] = h;
+                  if (p.res) {
+                    const size_t off = (size_t)t * p.ldy + colbase + c0 + e;
+                    p.y2[off] = __float2half_rn(__half2float(p.res[off]) + __half2float(h));
+                  }
+                }
             }
           }
         }
@@ -424,10 +447,11 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
 // y[t][c] = rn16(sum_s partial[s][t][c]) for c < n_cols, splits summed in ascending order; eight columns per thread when
 // the row length allows 16-byte accesses
 __global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, __half* __restrict__ y, int T, int n_cols, int ldy,
-                                          int splits) {
+                                          int splits, const __half* __restrict__ res, __half* __restrict__ y2) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const size_t plane = (size_t)T * ldy;
-  if (n_cols % 8 == 0 && ldy % 8 == 0) {
+  if (n_cols % 8 == 0 && ldy % 8 == 0 &&
+      (((reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(res) | reinterpret_cast<uintptr_t>(y2)) & 15) == 0)) {
     const int cg = n_cols / 8;
     const size_t total = (size_t)T * cg;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -447,6 +471,18 @@ __global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, __h
       o.z = *reinterpret_cast<const uint32_t*>(&h2);
       o.w = *reinterpret_cast<const uint32_t*>(&h3);
       *reinterpret_cast<uint4*>(y + t * ldy + c) = o;
+      if (res) {
+        const uint4 r4 = *reinterpret_cast<const uint4*>(res + t * ldy + c);
+        const uint32_t oo[4] = {o.x, o.y, o.z, o.w}, rr[4] = {r4.x, r4.y, r4.z, r4.w};
+        uint32_t z[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 p0 = __half22float2(u2h2(oo[j])), p1 = __half22float2(u2h2(rr[j]));
+          const __half2 h = __floats2half2_rn(p1.x + p0.x, p1.y + p0.y);
+          z[j] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(y2 + t * ldy + c) = make_uint4(z[0], z[1], z[2], z[3]);
+      }
     }
     return;
   }
@@ -455,7 +491,9 @@ __global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, __h
     const size_t t = i / n_cols, c = i % n_cols;
     float acc = 0.f;
     for (int s = 0; s < splits; ++s) acc += partial[(size_t)s * plane + t * ldy + c];
-    y[t * ldy + c] = __float2half_rn(acc);
+    const __half h = __float2half_rn(acc);
+    y[t * ldy + c] = h;
+    if (res) y2[t * ldy + c] = __float2half_rn(__half2float(res[t * ldy + c]) + __half2float(h));
   }
 }
 
@@ -567,6 +605,8 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   p.ldy = g.ldy;
   p.partial = (float*)g.scratch;
   p.status = g.status;
+  p.res = g.res;
+  p.y2 = g.y2;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e1 = cudaFuncSetAttribute(gemm_q4_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -591,7 +631,7 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   if (p.splits > 1) {
     const size_t total = (size_t)g.T * col;
     const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)sm_count * 8);
-    gemm_splitk_reduce_kernel<<<blocks, 256, 0, st>>>(p.partial, g.y, g.T, col, g.ldy, p.splits);
+    gemm_splitk_reduce_kernel<<<blocks, 256, 0, st>>>(p.partial, g.y, g.T, col, g.ldy, p.splits, g.res, g.y2);
     ++*n_launch;
     e = cudaGetLastError();
   }

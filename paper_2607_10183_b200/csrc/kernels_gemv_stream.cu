@@ -249,8 +249,18 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
   }
 
   // ------------------------------------------------------------------ consumers
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // the activation comes from the preceding kernel
   const int tid = threadIdx.x;                        // 0..255
+  // The norm gains are parameters, not products of the preceding kernel: fetch them before waiting for it.  (Every CTA
+  // reads the same few kilobytes, and such a broadcast read takes far longer than an ordinary L2 hit.)
+  uint4 graw[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+  if (PARTS <= 2 && p.gain) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int i0 = (tid + 256 * j) * 8;
+      if (i0 < K) graw[j] = __ldg(reinterpret_cast<const uint4*>(p.gain + i0));
+    }
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the activation comes from the preceding kernel
   const int part = warp % PARTS, rsub = warp / PARTS;
   const int pblk = (nblk + PARTS - 1) / PARTS;
   const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
@@ -298,7 +308,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
       for (int j = 0; j < kRuns; ++j) {
         const int i0 = (tid + 256 * j) * 8;
         if (i0 < K) {
-          const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(p.gain + i0));
+          const uint4 g4 = graw[j];
           const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
 #pragma unroll
           for (int q = 0; q < 4; ++q) {

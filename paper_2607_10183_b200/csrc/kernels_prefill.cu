@@ -269,18 +269,6 @@ cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const _
   return cudaGetLastError();
 }
 
-__global__ void add16_kernel(const __half* __restrict__ a, const __half* __restrict__ b, __half* __restrict__ out, uint64_t n) {
-  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
-    out[i] = __float2half_rn(__half2float(a[i]) + __half2float(b[i]));
-}
-
-cudaError_t launch_add16(const __half* a, const __half* b, __half* out, uint64_t n, cudaStream_t st, uint64_t* n_launch) {
-  const int grid = (int)std::min<uint64_t>((n + 255) / 256, 148 * 8);
-  add16_kernel<<<grid, 256, 0, st>>>(a, b, out, n);
-  ++*n_launch;
-  return cudaGetLastError();
-}
-
 // gu holds [T][ld] with gate in columns [0, ffn) and up in [ffn, 2 ffn): act = rn16(silu(g) * u); 8 elements per thread
 __global__ void swiglu16_kernel(const __half* __restrict__ gu, int ld, int ffn, __half* __restrict__ act, uint64_t n8) {
   const int per_row = ffn / 8;
