@@ -463,86 +463,87 @@ cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __ha
 // cos/sin table for `pos` computed on the host in fp64 and passed by value), appends the new K/V row to the caches as
 // fp16, attends over positions 0..pos split across CTAs, and merges the splits: the last CTA to finish a kv head
 // (a counter in global memory, reset for the next launch) sums the partials in ascending split order, so the result
-// does not depend on which CTA arrives last.  CTA (split, query head) covers 256 positions, one per lane of its 8
-// warps (the heads of a group re-read the same K/V rows from L2).  The kernel is a short chain of memory round trips,
-// so every phase issues all of its loads before it uses any of them: key rows are staged with 16-byte async copies
-// into padded shared-memory rows and the value slices are fetched into registers before the grid dependency resolves.
-constexpr int kAttnPos = 256;
+// does not depend on which CTA arrives last.
+// CTA (split, kv head) covers 64 positions for ALL query heads of the group: the K and V rows are staged once in shared
+// memory (16-byte async copies, issued before the grid dependency resolves) and every head's warps read them from
+// there, so the cache crosses the L2-to-SM fabric once instead of once per query head; that traffic, not DRAM, bounds
+// this kernel.  Warp (head, sub-block) owns 32 positions, one per lane.
 constexpr int kAttnMaxGroup = 8;
-constexpr int kAttnMaxSplits = 512;  // 131072 cached positions
-
-int attn_decode_splits(int n_ctx) { return (n_ctx + kAttnPos - 1) / kAttnPos; }
-size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) { return (size_t)n_q * attn_decode_splits(n_ctx) * (d + 2); }
+// Positions per CTA: 64, or 128 for contexts beyond 1024 so that the final merge still reads all splits of a head in
+// one round trip (16 splits) up to 2048 positions.
+int attn_decode_pos_per_cta(int n_ctx) { return n_ctx <= 1024 ? 64 : 128; }
+int attn_decode_splits(int n_ctx) {
+  const int pc = attn_decode_pos_per_cta(n_ctx);
+  return (n_ctx + pc - 1) / pc;
+}
+size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) {
+  return (size_t)n_q * ((n_ctx + 63) / 64 + 1) * (d + 2);  // enough for 64 positions per CTA at any context up to n_ctx
+}
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
 }
 
-template <int D>
-__global__ void __launch_bounds__(kAttnPos) attn_decode_fused_kernel(const AttnDecodeParams p) {
+template <int D, int SUB>
+__global__ void __launch_bounds__(512) attn_decode_fused_kernel(const AttnDecodeParams p) {
+  constexpr int POS = 32 * SUB;        // positions per CTA
   constexpr int V = D / 32;            // output dims per lane
-  constexpr int NW = kAttnPos / 32;
-  constexpr int CH = D * 2 / 16;       // 16-byte chunks per key row
+  constexpr int CH = D * 2 / 16;       // 16-byte chunks per cache row
   constexpr int KROW = D * 2 + 16;     // key row pitch in shared memory: the 16-byte pad makes lane-per-row reads conflict-free
-  extern __shared__ __align__(16) uint8_t k_s[];  // [kAttnPos][KROW]
-  __shared__ __align__(16) float q_s[D];
-  __shared__ float w_m[NW], w_l[NW];
-  __shared__ float w_acc[NW][D];
-  __shared__ float f_s[2 * kAttnMaxSplits + 1];
+  constexpr int VROW = D * 2;
+  constexpr int EPT = D / 64;          // output elements per thread in the merges (64 threads per head)
+  constexpr int MAXW = 16;             // warps per CTA at most (group * SUB)
+  extern __shared__ __align__(16) uint8_t dyn_s[];
+  uint8_t* k_s = dyn_s;                              // [POS][KROW]
+  uint8_t* v_s = dyn_s + (size_t)POS * KROW;    // [POS][VROW]
+  __shared__ __align__(16) float q_s[kAttnMaxGroup][D];
+  __shared__ float w_m[MAXW], w_l[MAXW];
+  __shared__ float w_acc[MAXW][D];
   __shared__ int is_last;
-  const int split = blockIdx.x, hq = blockIdx.y, n_splits = gridDim.x;
-  const int kvh = hq / p.group;
-  const bool writer = hq % p.group == 0;  // one CTA per kv head writes the new cache rows
+  const int split = blockIdx.x, kvh = blockIdx.y, n_splits = gridDim.x;
+  const int G = p.group, nthr = blockDim.x;  // nthr = G * POS
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = warp / SUB, sub = warp % SUB;
   const int half = D / 2, n_ctx = p.pos + 1;
   const int qd = p.n_q * D, kvd = p.n_kv * D;
-  const int tc0 = split * kAttnPos;                     // first position of the CTA
-  const int rows_here = min(kAttnPos, n_ctx - tc0);     // >= 1
-  const bool own = split == p.pos / kAttnPos;           // this CTA holds the new token's position
+  const int tc0 = split * POS;                     // first position of the CTA
+  const int rows_here = min(POS, n_ctx - tc0);     // >= 1
+  const bool own = split == p.pos / POS;           // this CTA holds the new token's position
   const int r_new = p.pos - tc0;
-  // The cache rows of past tokens do not depend on the preceding kernel: stage the keys (coalesced 16-byte async copies
-  // into padded rows) and fetch this lane's value slices before waiting for it.
-  for (int c = threadIdx.x; c < rows_here * CH; c += kAttnPos) {
+  // The cache rows of past tokens do not depend on the preceding kernel.
+  for (int c = threadIdx.x; c < rows_here * CH; c += nthr) {
     const int row = c / CH, ch = c % CH;
-    if (!(own && row == r_new))
-      cp_async16(k_s + (size_t)row * KROW + ch * 16, p.kc + ((size_t)kvh * p.cap + tc0 + row) * D + ch * 8);
-  }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-  const int t0 = tc0 + warp * 32;
-  const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
-  uint2 vraw[32];
-#pragma unroll
-  for (int tt = 0; tt < 32; ++tt) {
-    vraw[tt] = make_uint2(0u, 0u);
-    if (tt < n_here && t0 + tt != p.pos) {
-      const __half* vr = p.vc + ((size_t)kvh * p.cap + t0 + tt) * D + lane * V;
-      if (V == 4)
-        vraw[tt] = __ldg(reinterpret_cast<const uint2*>(vr));
-      else
-        vraw[tt].x = __ldg(reinterpret_cast<const uint32_t*>(vr));
+    if (!(own && row == r_new)) {
+      const size_t off = ((size_t)kvh * p.cap + tc0 + row) * D + ch * 8;
+      cp_async16(k_s + (size_t)row * KROW + ch * 16, p.kc + off);
+      cp_async16(v_s + (size_t)row * VROW + ch * 16, p.vc + off);
     }
   }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  // value rows beyond the context are read by the PV loop with weight zero: they must hold finite numbers
+  for (int c = threadIdx.x + rows_here * CH; c < POS * CH; c += nthr)
+    *reinterpret_cast<uint4*>(v_s + (size_t)(c / CH) * VROW + (c % CH) * 16) = make_uint4(0, 0, 0, 0);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v of the new token come from the preceding kernel
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // rotary embedding of this query head into shared memory
-  if (threadIdx.x < half) {
-    const int i = threadIdx.x;
-    const float* q = p.qkv + (size_t)hq * D;
+  // rotary embedding of the group's query heads into shared memory
+  for (int idx = threadIdx.x; idx < G * half; idx += nthr) {
+    const int g2 = idx / half, i = idx % half;
+    const int hq2 = kvh * G + g2;
+    const float* q = p.qkv + (size_t)hq2 * D;
     const float a = q[i], b = q[i + half];
     const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
     const float ra = a * c - b * s, rb = b * c + a * s;
-    q_s[i] = ra;
-    q_s[i + half] = rb;
+    q_s[g2][i] = ra;
+    q_s[g2][i + half] = rb;
     if (p.q_rot_out && split == 0) {
-      p.q_rot_out[(size_t)hq * D + i] = ra;
-      p.q_rot_out[(size_t)hq * D + i + half] = rb;
+      p.q_rot_out[(size_t)hq2 * D + i] = ra;
+      p.q_rot_out[(size_t)hq2 * D + i + half] = rb;
     }
   }
-  // the CTAs that cover position `pos` rotate the new key and put its fp16 value into their staged tile; one of them
-  // per kv head also appends key and value rows to the caches
+  // the CTA that covers position `pos` rotates the new key, rounds key and value to fp16 as the cache holds them, puts
+  // them into its staged tiles and appends them to the caches
   if (own) {
-    if (threadIdx.x >= kAttnPos - half) {
-      const int i = threadIdx.x - (kAttnPos - half);
+    for (int i = threadIdx.x; i < half; i += nthr) {
       const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
       const float* k = p.qkv + qd + (size_t)kvh * D;
       const float a = k[i], b = k[i + half];
@@ -550,40 +551,31 @@ __global__ void __launch_bounds__(kAttnPos) attn_decode_fused_kernel(const AttnD
       __half* srow = reinterpret_cast<__half*>(k_s + (size_t)r_new * KROW);
       srow[i] = ka;
       srow[i + half] = kb;
-      if (writer) {
-        __half* dst = p.kc + ((size_t)kvh * p.cap + p.pos) * D;
-        dst[i] = ka;
-        dst[i + half] = kb;
-      }
+      __half* dst = p.kc + ((size_t)kvh * p.cap + p.pos) * D;
+      dst[i] = ka;
+      dst[i + half] = kb;
     }
-    if (writer && threadIdx.x < D)
-      p.vc[((size_t)kvh * p.cap + p.pos) * D + threadIdx.x] = __float2half_rn(p.qkv[qd + kvd + (size_t)kvh * D + threadIdx.x]);
-    if (p.pos >= t0 && p.pos < t0 + 32) {  // the warp whose lanes cover `pos`: its value slice, rounded as the cache holds it
-      const float* vn = p.qkv + qd + kvd + (size_t)kvh * D + lane * V;
-      __half2 h01 = __floats2half2_rn(vn[0], vn[1]);
-      uint2 r = make_uint2(*reinterpret_cast<uint32_t*>(&h01), 0u);
-      if (V == 4) {
-        __half2 h23 = __floats2half2_rn(vn[2], vn[3]);
-        r.y = *reinterpret_cast<uint32_t*>(&h23);
-      }
-#pragma unroll
-      for (int tt = 0; tt < 32; ++tt)
-        if (t0 + tt == p.pos) vraw[tt] = r;
+    for (int i = threadIdx.x; i < D; i += nthr) {
+      const __half vv = __float2half_rn(p.qkv[qd + kvd + (size_t)kvh * D + i]);
+      reinterpret_cast<__half*>(v_s + (size_t)r_new * VROW)[i] = vv;
+      p.vc[((size_t)kvh * p.cap + p.pos) * D + i] = vv;
     }
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
-  const int t = t0 + lane;
-  const bool ok = t < n_ctx;
+  const int t0 = tc0 + sub * 32;
+  const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
+  const bool ok = lane < n_here;
   float sc = 0.f;
   if (ok) {
-    const uint4* kr = reinterpret_cast<const uint4*>(k_s + (size_t)(warp * 32 + lane) * KROW);
+    const uint4* kr = reinterpret_cast<const uint4*>(k_s + (size_t)(sub * 32 + lane) * KROW);
+    const float* qh = q_s[g];
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int c = 0; c < CH; ++c) {
       const uint4 kv = kr[c];
-      const float4 q0 = *reinterpret_cast<const float4*>(q_s + c * 8);
-      const float4 q1 = *reinterpret_cast<const float4*>(q_s + c * 8 + 4);
+      const float4 q0 = *reinterpret_cast<const float4*>(qh + c * 8);
+      const float4 q1 = *reinterpret_cast<const float4*>(qh + c * 8 + 4);
       float2 f;
       f = __half22float2(u32_as_half2(kv.x)); s0 = fmaf(f.x, q0.x, s0); s1 = fmaf(f.y, q0.y, s1);
       f = __half22float2(u32_as_half2(kv.y)); s0 = fmaf(f.x, q0.z, s0); s1 = fmaf(f.y, q0.w, s1);
@@ -605,97 +597,121 @@ __global__ void __launch_bounds__(kAttnPos) attn_decode_fused_kernel(const AttnD
   for (int v = 0; v < V; ++v) acc[v] = 0.f;
 #pragma unroll
   for (int tt = 0; tt < 32; ++tt) {
-    const float pt = __shfl_sync(0xffffffffu, pr, tt);  // zero for positions beyond n_ctx
-    float2 f;
-    f = __half22float2(u32_as_half2(vraw[tt].x));
-    acc[0] = fmaf(pt, f.x, acc[0]);
-    acc[1] = fmaf(pt, f.y, acc[1]);
-    if (V == 4) {
-      f = __half22float2(u32_as_half2(vraw[tt].y));
-      acc[2] = fmaf(pt, f.x, acc[2]);
-      acc[3] = fmaf(pt, f.y, acc[3]);
+    const float pt = __shfl_sync(0xffffffffu, pr, tt);
+    {
+      const uint8_t* vr = v_s + (size_t)(sub * 32 + tt) * VROW + lane * (V * 2);
+      float2 f;
+      if (V == 4) {
+        const uint2 raw = *reinterpret_cast<const uint2*>(vr);
+        f = __half22float2(u32_as_half2(raw.x));
+        acc[0] = fmaf(pt, f.x, acc[0]);
+        acc[1] = fmaf(pt, f.y, acc[1]);
+        f = __half22float2(u32_as_half2(raw.y));
+        acc[2] = fmaf(pt, f.x, acc[2]);
+        acc[3] = fmaf(pt, f.y, acc[3]);
+      } else {
+        f = __half22float2(u32_as_half2(*reinterpret_cast<const uint32_t*>(vr)));
+        acc[0] = fmaf(pt, f.x, acc[0]);
+        acc[1] = fmaf(pt, f.y, acc[1]);
+      }
     }
   }
 #pragma unroll
   for (int v = 0; v < V; ++v) w_acc[warp][lane * V + v] = acc[v];
   __syncthreads();
-  // merge the warps (ascending) into this split's partial
-  float* part = p.part + ((size_t)hq * n_splits + split) * (D + 2);
-  if (threadIdx.x < D) {
-    const int e = threadIdx.x;
+  // merge each head's warps (ascending) into this split's partial: 64 threads per head
+  const int g2 = threadIdx.x / 64, j = threadIdx.x % 64;
+  const int hq2 = kvh * G + g2;
+  if (g2 < G) {
+    float* part = p.part + ((size_t)hq2 * n_splits + split) * (D + 2);
     float mx = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) mx = fmaxf(mx, w_m[w]);
-    float l = 0.f, o = 0.f;
+    for (int w = 0; w < SUB; ++w) mx = fmaxf(mx, w_m[g2 * SUB + w]);
+    float l = 0.f, o[EPT];
 #pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      const float f = w_m[w] > -INFINITY ? expf(w_m[w] - mx) : 0.f;
-      l = fmaf(w_l[w], f, l);
-      o = fmaf(w_acc[w][e], f, o);
+    for (int q = 0; q < EPT; ++q) o[q] = 0.f;
+#pragma unroll
+    for (int w = 0; w < SUB; ++w) {
+      const float m = w_m[g2 * SUB + w];
+      const float f = m > -INFINITY ? expf(m - mx) : 0.f;
+      l = fmaf(w_l[g2 * SUB + w], f, l);
+#pragma unroll
+      for (int q = 0; q < EPT; ++q) o[q] = fmaf(w_acc[g2 * SUB + w][j + 64 * q], f, o[q]);
     }
-    part[e] = o;
-    if (e == 0) {
+#pragma unroll
+    for (int q = 0; q < EPT; ++q) part[j + 64 * q] = o[q];
+    if (j == 0) {
       part[D] = mx;
       part[D + 1] = l;
     }
   }
-  // the last CTA of this head merges the splits
+  // the last CTA of this kv head merges the splits of its query heads
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int prev = atomicAdd(p.counters + hq, 1);
+    const int prev = atomicAdd(p.counters + kvh, 1);
     is_last = prev == n_splits - 1;
-    if (is_last) p.counters[hq] = 0;  // ready for the next launch
+    if (is_last) p.counters[kvh] = 0;  // ready for the next launch
   }
   __syncthreads();
-  if (!is_last) return;
+  if (!is_last || g2 >= G) return;
   __threadfence();
-  const float* base = p.part + (size_t)hq * n_splits * (D + 2);
-  for (int i = threadIdx.x; i < 2 * n_splits; i += kAttnPos)  // all maxima and sums at once: one round trip
-    f_s[i] = __ldcg(base + (size_t)(i >> 1) * (D + 2) + D + (i & 1));
-  const int e = threadIdx.x % D;
-  float o = 0.f;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float mx = -INFINITY;
-    for (int s2 = 0; s2 < n_splits; ++s2) mx = fmaxf(mx, f_s[2 * s2]);
-    float l = 0.f;
-    for (int s2 = 0; s2 < n_splits; ++s2) {
-      const float m = f_s[2 * s2];
-      const float f = m > -INFINITY ? expf(m - mx) : 0.f;
-      l = fmaf(f_s[2 * s2 + 1], f, l);
-      f_s[2 * s2] = f;
-    }
-    f_s[2 * n_splits] = 1.0f / l;
-  }
-  __syncthreads();
-  if (threadIdx.x < D) {
-    for (int s0 = 0; s0 < n_splits; s0 += 8) {
-      float v[8];
+  const float* base = p.part + (size_t)hq2 * n_splits * (D + 2);
+  float mx = -INFINITY, l = 0.f, o[EPT];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = (s0 + u < n_splits) ? __ldcg(base + (size_t)(s0 + u) * (D + 2) + e) : 0.f;
+  for (int q = 0; q < EPT; ++q) o[q] = 0.f;
+  constexpr int NB = 16;  // splits per round trip: all of a batch's loads are issued before any is used
+  for (int s0 = 0; s0 < n_splits; s0 += NB) {
+    float m[NB], ls[NB], v[NB][EPT];
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if (s0 + u < n_splits) o = fmaf(v[u], f_s[2 * (s0 + u)], o);
+    for (int u = 0; u < NB; ++u) {
+      const bool in = s0 + u < n_splits;
+      const float* ps = base + (size_t)(s0 + u) * (D + 2);
+      m[u] = in ? __ldcg(ps + D) : -INFINITY;
+      ls[u] = in ? __ldcg(ps + D + 1) : 0.f;
+#pragma unroll
+      for (int q = 0; q < EPT; ++q) v[u][q] = in ? __ldcg(ps + j + 64 * q) : 0.f;
     }
-    p.a16[(size_t)hq * D + e] = __float2half_rn(o * f_s[2 * n_splits]);
+    float bm = mx;
+#pragma unroll
+    for (int u = 0; u < NB; ++u) bm = fmaxf(bm, m[u]);
+    const float rs = mx > -INFINITY ? expf(mx - bm) : 0.f;  // rescale what earlier batches accumulated
+    l *= rs;
+#pragma unroll
+    for (int q = 0; q < EPT; ++q) o[q] *= rs;
+#pragma unroll
+    for (int u = 0; u < NB; ++u) {
+      const float f = m[u] > -INFINITY ? expf(m[u] - bm) : 0.f;
+      l = fmaf(ls[u], f, l);
+#pragma unroll
+      for (int q = 0; q < EPT; ++q) o[q] = fmaf(v[u][q], f, o[q]);
+    }
+    mx = bm;
   }
+  const float inv = 1.0f / l;
+#pragma unroll
+  for (int q = 0; q < EPT; ++q) p.a16[(size_t)hq2 * D + j + 64 * q] = __float2half_rn(o[q] * inv);
 }
 
 cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch) {
-  const int splits = attn_decode_splits(p.pos + 1);
-  if (splits > kAttnMaxSplits) return cudaErrorInvalidValue;
+  if (p.group < 1 || p.group > kAttnMaxGroup || p.n_q != p.n_kv * p.group) return cudaErrorInvalidValue;
+  int pc = attn_decode_pos_per_cta(p.pos + 1);
+  if (p.group * pc > 512) pc = 64;  // large groups: 64 positions keep the CTA within 512 threads
+  const int splits = (p.pos + 1 + pc - 1) / pc;
   p.scale = 1.0f / sqrtf((float)d);
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(splits, p.n_q);
-  cfg.blockDim = dim3(kAttnPos);
-  cfg.dynamicSmemBytes = (size_t)kAttnPos * (d * 2 + 16);
+  cfg.gridDim = dim3(splits, p.n_kv);
+  cfg.blockDim = dim3(p.group * pc);
+  cfg.dynamicSmemBytes = (size_t)pc * (d * 4 + 16);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e1 = cudaFuncSetAttribute(attn_decode_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnPos * (128 * 2 + 16));
-    cudaError_t e2 = cudaFuncSetAttribute(attn_decode_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnPos * (64 * 2 + 16));
-    if (e1 != cudaSuccess) return e1;
-    if (e2 != cudaSuccess) return e2;
+    cudaError_t e[4] = {
+        cudaFuncSetAttribute(attn_decode_fused_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * (128 * 4 + 16)),
+        cudaFuncSetAttribute(attn_decode_fused_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (128 * 4 + 16)),
+        cudaFuncSetAttribute(attn_decode_fused_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * (64 * 4 + 16)),
+        cudaFuncSetAttribute(attn_decode_fused_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (64 * 4 + 16))};
+    for (cudaError_t x : e)
+      if (x != cudaSuccess) return x;
     attr_set = true;
   }
   cfg.stream = st;
@@ -705,8 +721,10 @@ cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStr
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   ++*n_launch;
-  if (d == 128) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<128>, p);
-  if (d == 64) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<64>, p);
+  if (d == 128 && pc == 64) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<128, 2>, p);
+  if (d == 128) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<128, 4>, p);
+  if (d == 64 && pc == 64) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<64, 2>, p);
+  if (d == 64) return cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<64, 4>, p);
   return cudaErrorInvalidValue;
 }
 

@@ -58,9 +58,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     if (clock64() - t0 > 2000000000ll) return false;
   }
 }
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+// Weights are read once per call: the copies carry an evict-first L2 policy so that a step's 100+ MB of weights do not
+// push the activations, the KV cache and the kernels' own instructions out of the L2.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
                : "memory");
 }
 __device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {
@@ -210,6 +218,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
     // ------------------------------------------------------------------ producer: weights do not depend on the
     // preceding kernel, so their copies start before the grid dependency is resolved.
     if (lane == 0) {
+      const uint64_t pol = l2_evict_first_policy();
       for (int it = 0; it < n_it; ++it) {
         const int s = it % kStages;
         if (it >= kStages && !mbar_wait(&empty[s], ((it / kStages) - 1) & 1)) {
@@ -230,18 +239,18 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
           const size_t r0 = (size_t)tile * OUT_ROWS;
           const uint8_t *g = p.seg[0].base, *u = p.seg[1].base;
           const size_t n = (size_t)p.seg[0].n_rows;
-          bulk_g2s(dst, g + r0 * row_codes, OUT_ROWS * row_codes, &full[s]);
-          bulk_g2s(dst + OUT_ROWS * row_codes, u + r0 * row_codes, OUT_ROWS * row_codes, &full[s]);
+          bulk_g2s(dst, g + r0 * row_codes, OUT_ROWS * row_codes, &full[s], pol);
+          bulk_g2s(dst + OUT_ROWS * row_codes, u + r0 * row_codes, OUT_ROWS * row_codes, &full[s], pol);
           uint8_t* sd = dst + ROWS * row_codes;
-          bulk_g2s(sd, g + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s]);
-          bulk_g2s(sd + OUT_ROWS * row_scales, u + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s]);
+          bulk_g2s(sd, g + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s], pol);
+          bulk_g2s(sd + OUT_ROWS * row_scales, u + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s], pol);
         } else {
           int sg = 0;
           while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
           const size_t r0 = (size_t)(tile - p.seg[sg].tile0) * ROWS;
           const uint8_t* b = p.seg[sg].base;
-          bulk_g2s(dst, b + r0 * row_codes, ROWS * row_codes, &full[s]);
-          bulk_g2s(dst + ROWS * row_codes, b + (size_t)p.seg[sg].n_rows * row_codes + r0 * row_scales, ROWS * row_scales, &full[s]);
+          bulk_g2s(dst, b + r0 * row_codes, ROWS * row_codes, &full[s], pol);
+          bulk_g2s(dst + ROWS * row_codes, b + (size_t)p.seg[sg].n_rows * row_codes + r0 * row_scales, ROWS * row_scales, &full[s], pol);
         }
       }
     }

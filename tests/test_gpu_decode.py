@@ -157,7 +157,11 @@ def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, fl
 ALL_GPU = {n: 1 for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")}
 
 
-@pytest.mark.parametrize("shape_name,pos,cap", [("small", 0, 8), ("small", 37, 64), ("small", 200, 300), ("full", 1024, 1025)])
+# positions around the attention kernel's tiling: 64 or 128 positions per CTA (contexts up to / beyond 1024), the final
+# merge reads 16 splits per round trip (context 2101 at 128 per CTA needs a second one)
+@pytest.mark.parametrize("shape_name,pos,cap", [("small", 0, 8), ("small", 37, 64), ("small", 63, 64), ("small", 64, 80),
+                                                ("small", 200, 300), ("small", 1023, 1024), ("small", 1100, 1101),
+                                                ("small", 2100, 2200), ("full", 1024, 1025)])
 def test_dense_layer_decode_matches_oracle(B, torch, shape_name, pos, cap):
     shape = W.DENSE_SMALL if shape_name == "small" else W.DENSE_FULL
     cfg = 96 if shape_name == "small" else 2
