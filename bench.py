@@ -315,7 +315,14 @@ def extra_moe(torch, B, W, peaks, quick):
             st = ctx.stats()
             key = f"{'hybrid' if hybrid else 'resident'}_M{M}"
             out[key] = {"us_per_call": dt * 1e6, "tokens_per_s": M / dt, "streamed_bytes_per_call": st.streamed_bytes / n,
-                        "launches_per_call": st.kernel_launches / n}
+                        "launches_per_call": st.kernel_launches / n, "timing": "wall clock around back-to-back calls (host included)"}
+            if not hybrid:
+                # all resident: no host synchronisation inside a call, so the device time of a queue of calls can be
+                # read with CUDA events (the wall-clock figure above is bound by the host's launch rate)
+                dev_ms = event_time_ms(torch, ctx.compute, lambda: go(n))
+                out[key]["device_us_per_call"] = dev_ms * 1e3 / n
+                moe_bytes = shape.top_k * min(M, shape.n_experts) * 3 * sl  # upper bound: all selected experts distinct
+                out[key]["expert_bytes_per_call_upper"] = moe_bytes
             if hybrid and st.streamed_bytes:
                 out[key]["pcie_gbs_over_call_time"] = st.streamed_bytes / n / dt / 1e9
         ctx.close()

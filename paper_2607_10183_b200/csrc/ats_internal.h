@@ -175,11 +175,15 @@ struct MoeGemvParams {
 };
 cudaError_t launch_moe_gemv(const MoeGemvParams& p, const MoeJobs* jobs /*null = implicit*/, cudaStream_t st,
                             uint64_t* n_launch);
+// the streaming kernel's grouped-expert form (kernels_gemv_stream.cu): shapes it accepts, and its launcher
+bool moe_gemv_stream_eligible(const MoeGemvParams& p);
+cudaError_t launch_moe_gemv_stream(const MoeGemvParams& p, const MoeJobs* jobs /*null = implicit*/, int* status, int sm_count,
+                                   int pdl, cudaStream_t st, uint64_t* n_launch);
 
 cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, cudaStream_t st,
                            uint64_t* n_launch);
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
-                           cudaStream_t st, uint64_t* n_launch);
+                           cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 // decode attention, fused with the rotary embedding and the KV append (kernels_decode.cu)
 struct AttnDecodeParams {
   const float* qkv;   // [q | k | v] fp32 of the new token
@@ -197,10 +201,10 @@ int attn_decode_splits(int n_ctx);
 size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx);
 cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch);
 cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
-                               float* gates, cudaStream_t st, uint64_t* n_launch);
+                               float* gates, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 // y16[m] = rn16(res[m] + sum_j gates[m][j] * d32[m*k + j])   (res fp16 or fp32)
 cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gates, const float* d32, __half* y16,
-                               int M, int k, int H, cudaStream_t st, uint64_t* n_launch);
+                               int M, int k, int H, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uint64_t* n_launch);
 
 // prefill

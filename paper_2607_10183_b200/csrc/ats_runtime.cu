@@ -481,6 +481,14 @@ static int32_t apply_placement(ats_ctx* ctx) {
 // ids_host == null: every slice is resident and contiguous, the kernel indexes experts from device ids.
 // Otherwise pairs on resident experts run first (overlapping the copies), then the streamed experts in ascending order
 // in groups that fit the ring.
+// One grouped-expert GEMV launch: the streaming kernel where the shapes allow it, else the generic one.
+static cudaError_t launch_moe_gemv_any(ats_ctx* ctx, const MoeGemvParams& p, const MoeJobs* jobs) {
+  if (moe_gemv_stream_eligible(p))
+    return launch_moe_gemv_stream(p, jobs, ctx->dev_status, ctx->sm_count, (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1, ctx->cs,
+                                  &ctx->stats.kernel_launches);
+  return launch_moe_gemv(p, jobs, ctx->cs, &ctx->stats.kernel_launches);
+}
+
 static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_dev, const int32_t* ids_host,
                              MoeGemvParams p) {
   const Tensor& t0 = ctx->tensors[id0];
@@ -493,7 +501,7 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
     p.base0 = t0.slices[0].dev;
     p.base1 = t1 ? t1->slices[0].dev : nullptr;
     TimedLaunch tl(ctx, 1, (uint64_t)p.P * ((t1 ? 2 : 1) * t0.slice_bytes + (uint64_t)p.K * 2 + (uint64_t)p.n_rows * 2));
-    ATS_CUDA(launch_moe_gemv(p, nullptr, ctx->cs, &ctx->stats.kernel_launches));
+    ATS_CUDA(launch_moe_gemv_any(ctx, p, nullptr));
     return ATS_OK;
   }
   const int P = p.P;
@@ -502,7 +510,7 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
   auto flush = [&]() -> int32_t {
     if (jobs.n == 0) return ATS_OK;
     TimedLaunch tl(ctx, 1, (uint64_t)jobs.n * ((t1 ? 2 : 1) * t0.slice_bytes + (uint64_t)p.K * 2 + (uint64_t)p.n_rows * 2));
-    ATS_CUDA(launch_moe_gemv(p, &jobs, ctx->cs, &ctx->stats.kernel_launches));
+    ATS_CUDA(launch_moe_gemv_any(ctx, p, &jobs));
     jobs.n = 0;
     return ATS_OK;
   };
@@ -1078,7 +1086,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   }
   if (L->n_experts != 0)  // the MoE path needs the normalised row in memory (router and grouped GEMV read it)
     ATS_CUDA(launch_rmsnorm(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev,
-                            w.h2_16, (int)M, H, L->rms_eps, ctx->cs, nl));
+                            w.h2_16, (int)M, H, L->rms_eps, ctx->cs, nl, pdl));
   if (L->n_experts == 0) {
     GemvParams g{};
     g.M = (int)M;
@@ -1114,7 +1122,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   // ---- MoE FFN
   const int k = (int)L->top_k, P = (int)M * k, E = (int)L->n_experts;
   ATS_CUDA(launch_router_topk(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)M, H, E, k,
-                              (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, ctx->cs, nl));
+                              (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, ctx->cs, nl, pdl));
   const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
   const bool implicit = tg.contiguous_dev && tu.contiguous_dev && td.contiguous_dev;
   const int32_t* ids_host = nullptr;
@@ -1144,7 +1152,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   s2.mode = GEMV_OUT_F32;
   ATS_TRY(run_moe_stage(ctx, L->w_down, -1, w.ids, ids_host, s2));
   ATS_CUDA(launch_moe_combine(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, w.gates, w.d32, (__half*)x_out, (int)M, k, H,
-                              ctx->cs, nl));
+                              ctx->cs, nl, pdl));
   return ATS_OK;
 }
 

@@ -370,11 +370,41 @@ __device__ __forceinline__ float load_f<float>(const float* p, size_t i) { retur
 template <>
 __device__ __forceinline__ float load_f<__half>(const __half* p, size_t i) { return __half2float(p[i]); }
 
+// Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the stream is
+// still finishing; every kernel launched this way executes griddepcontrol.wait before it touches the predecessor's data.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_dep(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int pdl, int cluster_x,
+                              Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[na].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+  ++na;
+  if (cluster_x > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = cluster_x;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 template <typename TIn>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const TIn* __restrict__ x, const __half* __restrict__ gain,
                                                       __half* __restrict__ out, int H, float eps) {
   __shared__ float red[8];
   __shared__ float inv_s;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   const TIn* xr = x + (size_t)blockIdx.x * H;
   float ss = 0.f;
   for (int i = threadIdx.x; i < H; i += blockDim.x) {
@@ -399,6 +429,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const TIn* __restrict__ x,
 __global__ void __launch_bounds__(256) rmsnorm16_vec_kernel(const __half* __restrict__ x, const __half* __restrict__ gain,
                                                             __half* __restrict__ out, int H, float eps) {
   __shared__ float red[8];
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n8 = H / 8;
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)blockIdx.x * H);
   uint4 xv[4], gv[4];
@@ -446,16 +478,13 @@ __global__ void __launch_bounds__(256) rmsnorm16_vec_kernel(const __half* __rest
 }
 
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
-                           cudaStream_t st, uint64_t* n_launch) {
+                           cudaStream_t st, uint64_t* n_launch, int pdl) {
+  ++*n_launch;
   if (!x_is_f32 && H % 8 == 0 && H <= 8192 &&
       (((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(out)) & 15) == 0))
-    rmsnorm16_vec_kernel<<<M, 256, 0, st>>>((const __half*)x, gain, out, H, eps);
-  else if (x_is_f32)
-    rmsnorm_kernel<float><<<M, 256, 0, st>>>((const float*)x, gain, out, H, eps);
-  else
-    rmsnorm_kernel<__half><<<M, 256, 0, st>>>((const __half*)x, gain, out, H, eps);
-  ++*n_launch;
-  return cudaGetLastError();
+    return launch_dep(rmsnorm16_vec_kernel, dim3(M), dim3(256), 0, st, pdl, 1, (const __half*)x, gain, out, H, eps);
+  if (x_is_f32) return launch_dep(rmsnorm_kernel<float>, dim3(M), dim3(256), 0, st, pdl, 1, (const float*)x, gain, out, H, eps);
+  return launch_dep(rmsnorm_kernel<__half>, dim3(M), dim3(256), 0, st, pdl, 1, (const __half*)x, gain, out, H, eps);
 }
 
 // ------------------------------------------------------------------------------------------- fused decode attention
@@ -731,32 +760,9 @@ cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStr
 // ------------------------------------------------------------------------------------------- router + top-k (a4)
 // One CTA per token.  Thread (grp, e) sums h[i] * W_r[i][e] over i = grp, grp+G, ...; groups are added in ascending
 // order; warp 0 then extracts the k largest logits (equal logits: lower index first) and the gates.
-constexpr int kRouterThreads = 1024;
-
-__global__ void __launch_bounds__(kRouterThreads) router_topk_kernel(const __half* __restrict__ h, const __half* __restrict__ wr,
-                                                                     int H, int E, int Epad, int k, int renorm,
-                                                                     int32_t* __restrict__ ids, float* __restrict__ gates) {
-  extern __shared__ float smem[];
-  float* h_s = smem;             // [H]
-  float* part = h_s + H;         // [G][Epad]
-  float* logit = part + kRouterThreads;  // [Epad]
-  const int m = blockIdx.x;
-  const int G = kRouterThreads / Epad;
-  for (int i = threadIdx.x; i < H; i += blockDim.x) h_s[i] = __half2float(h[(size_t)m * H + i]);
-  __syncthreads();
-  const int e = threadIdx.x % Epad, grp = threadIdx.x / Epad;
-  float acc = 0.f;
-  if (e < E)
-    for (int i = grp; i < H; i += G) acc = fmaf(h_s[i], __half2float(wr[(size_t)i * E + e]), acc);
-  part[grp * Epad + e] = acc;
-  __syncthreads();
-  if (threadIdx.x < Epad) {
-    float t = 0.f;
-    for (int g = 0; g < G; ++g) t += part[g * Epad + threadIdx.x];
-    logit[threadIdx.x] = threadIdx.x < E ? t : -INFINITY;
-  }
-  __syncthreads();
-  if (threadIdx.x >= 32) return;
+// Warp 0 extracts the k largest logits (equal logits: lower index first) and their gates from logit[Epad] in shared memory.
+__device__ __forceinline__ void router_select(const float* logit, int m, int E, int Epad, int k, int renorm,
+                                              int32_t* __restrict__ ids, float* __restrict__ gates) {
   const int lane = threadIdx.x;
   const int per = Epad / 32;  // candidates per lane: e = lane + 32*j
   uint32_t taken = 0;
@@ -817,24 +823,153 @@ __global__ void __launch_bounds__(kRouterThreads) router_topk_kernel(const __hal
   }
 }
 
+constexpr int kRouterThreads = 1024;
+
+__global__ void __launch_bounds__(kRouterThreads) router_topk_kernel(const __half* __restrict__ h, const __half* __restrict__ wr,
+                                                                     int H, int E, int Epad, int k, int renorm,
+                                                                     int32_t* __restrict__ ids, float* __restrict__ gates) {
+  extern __shared__ float smem[];
+  float* h_s = smem;             // [H]
+  float* part = h_s + H;         // [G][Epad]
+  float* logit = part + kRouterThreads;  // [Epad]
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int m = blockIdx.x;
+  const int G = kRouterThreads / Epad;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) h_s[i] = __half2float(h[(size_t)m * H + i]);
+  __syncthreads();
+  const int e = threadIdx.x % Epad, grp = threadIdx.x / Epad;
+  float acc = 0.f;
+  if (e < E)
+    for (int i = grp; i < H; i += G) acc = fmaf(h_s[i], __half2float(wr[(size_t)i * E + e]), acc);
+  part[grp * Epad + e] = acc;
+  __syncthreads();
+  if (threadIdx.x < Epad) {
+    float t = 0.f;
+    for (int g = 0; g < G; ++g) t += part[g * Epad + threadIdx.x];
+    logit[threadIdx.x] = threadIdx.x < E ? t : -INFINITY;
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  router_select(logit, m, E, Epad, k, renorm, ids, gates);
+}
+
+// The same routing for hidden sizes and expert counts that are multiples of 8, spread over a cluster of 8 CTAs per
+// token: CTA r of the cluster sums rows [r H/8, (r+1) H/8) of W_r (16-byte loads: a thread owns 8 consecutive experts of
+// the rows i = row group, row group + R, ...), adds its row groups in ascending order, and writes its partial logits
+// into CTA 0's shared memory (distributed shared memory); after the cluster barrier CTA 0 adds the 8 partials in rank
+// order and selects.  A single token's router matrix then streams through 8 SMs instead of one.
+constexpr int kRouterCluster = 8;
+constexpr int kRouterClThreads = 256;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f32(const float* local_smem_ptr, uint32_t rank, float v) {
+  uint32_t la = (uint32_t)__cvta_generic_to_shared(local_smem_ptr), ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
+}
+
+__global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(const __half* __restrict__ h,
+                                                                               const __half* __restrict__ wr, int H, int E, int Epad,
+                                                                               int k, int renorm, int32_t* __restrict__ ids,
+                                                                               float* __restrict__ gates) {
+  extern __shared__ __align__(16) float smem[];
+  const int Hc = H / kRouterCluster;          // rows of this CTA
+  const int L = E / 8;                        // threads per row
+  const int R = kRouterClThreads / L;         // row groups (L <= 128, so R >= 2)
+  float* h_s = smem;                          // [Hc]
+  float* part = h_s + Hc;                     // [R][E]
+  float* cl = part + (size_t)R * E;           // [kRouterCluster][Epad]   (used in CTA 0)
+  float* logit = cl + (size_t)kRouterCluster * Epad;  // [Epad]
+  const int m = blockIdx.y;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const uint32_t rank = cluster_ctarank();
+  const int row0 = (int)rank * Hc;
+  for (int i = threadIdx.x; i < Hc; i += kRouterClThreads) h_s[i] = __half2float(h[(size_t)m * H + row0 + i]);
+  __syncthreads();
+  const int grp = threadIdx.x / L, e0 = (threadIdx.x % L) * 8;
+  float acc[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+  if (grp < R) {
+#pragma unroll 4
+    for (int i = grp; i < Hc; i += R) {
+      const uint4 w = __ldg(reinterpret_cast<const uint4*>(wr + (size_t)(row0 + i) * E + e0));
+      const float x = h_s[i];
+      const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 f = __half22float2(u32_as_half2(ws[q]));
+        acc[2 * q] = fmaf(x, f.x, acc[2 * q]);
+        acc[2 * q + 1] = fmaf(x, f.y, acc[2 * q + 1]);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) part[(size_t)grp * E + e0 + q] = acc[q];
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < Epad; e += kRouterClThreads) {
+    float t = 0.f;
+    if (e < E)
+      for (int g = 0; g < R; ++g) t += part[(size_t)g * E + e];
+    st_cluster_f32(cl + (size_t)rank * Epad + e, 0, t);  // into CTA 0's copy of cl
+  }
+  cluster_sync_all();
+  if (rank != 0) return;
+  for (int e = threadIdx.x; e < Epad; e += kRouterClThreads) {
+    float t = 0.f;
+#pragma unroll
+    for (int r = 0; r < kRouterCluster; ++r) t += cl[(size_t)r * Epad + e];
+    logit[e] = e < E ? t : -INFINITY;
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  router_select(logit, m, E, Epad, k, renorm, ids, gates);
+}
+
 cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
-                               float* gates, cudaStream_t st, uint64_t* n_launch) {
+                               float* gates, cudaStream_t st, uint64_t* n_launch, int pdl) {
   int Epad = 32;
   while (Epad < E) Epad <<= 1;
+  if (E % 8 == 0 && H % (8 * kRouterCluster) == 0 && (((uintptr_t)wr | (uintptr_t)h) & 15) == 0) {
+    const int L = E / 8, R = kRouterClThreads / L;
+    const size_t smem_cl = ((size_t)H / kRouterCluster + (size_t)R * E + (size_t)(kRouterCluster + 1) * Epad) * sizeof(float);
+    if (smem_cl <= 160 * 1024) {
+      static size_t attr_bytes = 0;
+      if (smem_cl > 48 * 1024 && smem_cl > attr_bytes) {
+        cudaError_t e = cudaFuncSetAttribute(router_topk_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_cl);
+        if (e != cudaSuccess) return e;
+        attr_bytes = smem_cl;
+      }
+      ++*n_launch;
+      return launch_dep(router_topk_cluster_kernel, dim3(kRouterCluster, M), dim3(kRouterClThreads), smem_cl, st, pdl, kRouterCluster,
+                        h, wr, H, E, Epad, k, renorm, ids, gates);
+    }
+  }
   const size_t smem = ((size_t)H + kRouterThreads + Epad) * sizeof(float);
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(router_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  router_topk_kernel<<<M, kRouterThreads, smem, st>>>(h, wr, H, E, Epad, k, renorm, ids, gates);
   ++*n_launch;
-  return cudaGetLastError();
+  return launch_dep(router_topk_kernel, dim3(M), dim3(kRouterThreads), smem, st, pdl, 1, h, wr, H, E, Epad, k, renorm, ids, gates);
 }
 
 // ------------------------------------------------------------------------------------------- MoE combine
 template <typename TRes>
 __global__ void moe_combine_kernel(const TRes* __restrict__ res, const float* __restrict__ gates, const float* __restrict__ d32,
                                    __half* __restrict__ y16, int k, int H) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int m = blockIdx.y;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= H) return;
@@ -844,14 +979,12 @@ __global__ void moe_combine_kernel(const TRes* __restrict__ res, const float* __
 }
 
 cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gates, const float* d32, __half* y16, int M,
-                               int k, int H, cudaStream_t st, uint64_t* n_launch) {
+                               int k, int H, cudaStream_t st, uint64_t* n_launch, int pdl) {
   dim3 grid((H + 255) / 256, M);
-  if (res_is_f32)
-    moe_combine_kernel<float><<<grid, 256, 0, st>>>((const float*)res, gates, d32, y16, k, H);
-  else
-    moe_combine_kernel<__half><<<grid, 256, 0, st>>>((const __half*)res, gates, d32, y16, k, H);
   ++*n_launch;
-  return cudaGetLastError();
+  if (res_is_f32)
+    return launch_dep(moe_combine_kernel<float>, grid, dim3(256), 0, st, pdl, 1, (const float*)res, gates, d32, y16, k, H);
+  return launch_dep(moe_combine_kernel<__half>, grid, dim3(256), 0, st, pdl, 1, (const __half*)res, gates, d32, y16, k, H);
 }
 
 cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uint64_t* n_launch) {

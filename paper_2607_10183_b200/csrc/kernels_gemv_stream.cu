@@ -195,8 +195,11 @@ struct StreamParams {
   int* status;
 };
 
+// bx / gx: index of this CTA among the gx CTAs that share the work described by p (a whole launch for the dense GEMV, one
+// (token, slot) job of a grouped-expert launch).  wait_first: the weight addresses themselves come from the preceding
+// kernel (expert ids), so nothing may be fetched before the grid dependency resolves.
 template <int PARTS, bool SW>
-__global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamParams p) {
+__device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool wait_first) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t full[kStages], empty[kStages];
   __shared__ float part_s[kMaxIt * kConsumerWarps * kRPW];
@@ -218,14 +221,15 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  const int first = blockIdx.x;
-  const int n_it = first < p.n_tiles ? (p.n_tiles - first + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int first = bx;
+  const int n_it = first < p.n_tiles ? (p.n_tiles - first + gx - 1) / gx : 0;
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer: weights do not depend on the
     // preceding kernel, so their copies start before the grid dependency is resolved.
     if (lane == 0) {
       const uint64_t pol = l2_evict_first_policy();
+      if (wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int it = 0; it < n_it; ++it) {
         const int s = it % kStages;
         if (it >= kStages && !mbar_wait(&empty[s], ((it / kStages) - 1) & 1)) {
@@ -238,7 +242,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
           asm volatile("griddepcontrol.wait;" ::: "memory");
           asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         }
-        const int tile = first + it * gridDim.x;
+        const int tile = first + it * gx;
         uint8_t* dst = stages + (size_t)s * stage_bytes;
         mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
         if (SW) {
@@ -357,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
             xv[j][2 * q] = f.x;
             xv[j][2 * q + 1] = f.y;
           }
-          if (p.h_out && blockIdx.x == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+          if (p.h_out && bx == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
         }
       }
     }
@@ -477,7 +481,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
     const int n_out = (it1 - it0) * OUT_ROWS;
     for (int i = tid; i < n_out; i += 256) {
       const int itl = i / OUT_ROWS, j = i % OUT_ROWS;
-      const int tile = first + (it0 + itl) * gridDim.x;
+      const int tile = first + (it0 + itl) * gx;
       float v[2];
 #pragma unroll
       for (int h = 0; h < (SW ? 2 : 1); ++h) {
@@ -507,6 +511,46 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamPa
     }
     consumer_sync();
   }
+}
+
+template <int PARTS, bool SW>
+__global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamParams p) {
+  gemv_stream_body<PARTS, SW>(p, (int)blockIdx.x, (int)gridDim.x, false);
+}
+
+// Grouped-expert variant: blockIdx.y selects the job (a (token, slot) pair), whose expert slices, activation row and
+// output row come from the expert ids on the device (all experts resident and contiguous) or from a job table passed
+// by value (resident and streamed experts mixed); the gridDim.x CTAs of a job then run the same body.
+struct MoeSel {
+  const uint8_t* base0;
+  const uint8_t* base1;
+  unsigned long long stride;
+  const int32_t* ids;  // null: use the job table
+  int x_div;
+  int ldx, ldy;
+};
+template <int PARTS, bool SW>
+__global__ void __launch_bounds__(kThreads, 2) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
+  StreamParams p = p0;
+  const int job = blockIdx.y;
+  int xrow, orow;
+  if (m.ids) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the ids come from the router kernel
+    const size_t e = (size_t)m.ids[job];
+    p.seg[0].base = m.base0 + e * m.stride;
+    if (SW) p.seg[1].base = m.base1 + e * m.stride;
+    xrow = job / m.x_div;
+    orow = job;
+  } else {
+    p.seg[0].base = jobs.w0[job];
+    if (SW) p.seg[1].base = jobs.w1[job];
+    xrow = jobs.xrow[job];
+    orow = jobs.orow[job];
+  }
+  p.x16 = p0.x16 + (size_t)xrow * m.ldx;
+  if (p0.y32) p.y32 = p0.y32 + (size_t)orow * m.ldy;
+  if (p0.y16) p.y16 = p0.y16 + (size_t)orow * m.ldy;
+  gemv_stream_body<PARTS, SW>(p, (int)blockIdx.x, (int)gridDim.x, m.ids != nullptr);
 }
 
 int parts_for(int K) { return K <= 2048 ? 1 : K <= 4096 ? 2 : K <= 8192 ? 4 : 8; }
@@ -588,6 +632,73 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   cfg.numAttrs = 1;
   ++*n_launch;
   return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+bool moe_gemv_stream_eligible(const MoeGemvParams& p) {
+  if (p.K % 256 != 0 || p.K > 16384) return false;
+  const int rows = kConsumerWarps / parts_for(p.K) * kRPW;
+  if (p.mode == GEMV_SWIGLU_F16) return p.n_rows % (rows / 2) == 0;
+  return (p.mode == GEMV_OUT_F32 || p.mode == GEMV_OUT_F16) && p.n_rows % rows == 0;
+}
+
+cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, int* status, int sm_count, int pdl, cudaStream_t st,
+                                   uint64_t* n_launch) {
+  const int parts = parts_for(g.K);
+  const int rows = kConsumerWarps / parts * kRPW;
+  const bool sw = g.mode == GEMV_SWIGLU_F16;
+  const int n_jobs = jobs ? jobs->n : g.P;
+  if (n_jobs <= 0) return cudaSuccess;
+  StreamParams p{};
+  p.n_seg = sw ? 2 : 1;
+  p.seg[0] = StreamSeg{nullptr, g.n_rows, 0};
+  p.seg[1] = StreamSeg{nullptr, g.n_rows, 0};
+  p.n_tiles = sw ? g.n_rows / (rows / 2) : g.n_rows / rows;
+  p.K = g.K;
+  p.mode = g.mode;
+  p.x16 = g.x;
+  p.y32 = g.y32;
+  p.y16 = g.y16;
+  p.status = status;
+  MoeSel m{};
+  m.base0 = g.base0;
+  m.base1 = g.base1;
+  m.stride = g.stride;
+  m.ids = jobs ? nullptr : g.ids;
+  m.x_div = g.x_div;
+  m.ldx = g.ldx;
+  m.ldy = g.ldy;
+  MoeJobs none;
+  none.n = 0;
+  const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
+  const size_t smem = kStages * stage_bytes + (parts <= 2 ? (size_t)(g.K / 32) * 112 : 0);
+  if (smem > 100 * 1024) return cudaErrorInvalidValue;
+  const int per_job = std::max(1, std::min(p.n_tiles, (2 * sm_count + n_jobs - 1) / n_jobs));
+  void (*kern)(const StreamParams, const MoeSel, const MoeJobs) = nullptr;
+  switch (parts) {
+    case 1: kern = sw ? gemv_stream_moe_kernel<1, true> : gemv_stream_moe_kernel<1, false>; break;
+    case 2: kern = sw ? gemv_stream_moe_kernel<2, true> : gemv_stream_moe_kernel<2, false>; break;
+    case 4: kern = sw ? gemv_stream_moe_kernel<4, true> : gemv_stream_moe_kernel<4, false>; break;
+    default: kern = sw ? gemv_stream_moe_kernel<8, true> : gemv_stream_moe_kernel<8, false>; break;
+  }
+  static bool attr_set[8] = {};
+  const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
+  if (!attr_set[ki]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set[ki] = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(per_job, n_jobs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ++*n_launch;
+  return cudaLaunchKernelEx(&cfg, kern, p, m, jobs ? *jobs : none);
 }
 
 }  // namespace ats
