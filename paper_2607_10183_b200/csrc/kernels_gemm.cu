@@ -375,24 +375,37 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
       const int colbase = p.seg[sg].col0 + row0;
       const bool vec = (p.ldy % 8 == 0) && (colbase % 8 == 0) &&
                        (((reinterpret_cast<uintptr_t>(p.y) | reinterpret_cast<uintptr_t>(p.res) | reinterpret_cast<uintptr_t>(p.y2)) & 15) == 0);
+      // Full rows of a 32 x 32 block are regrouped through shared memory (the pipeline stages are idle once the
+      // accumulator is complete; each warp uses a private 4.5 KB piece) so that a store instruction writes whole 128-byte
+      // lines (fp32 partials: 4 rows x 128 B; fp16 output: 8 rows x 64 B) instead of 32 scattered 16-byte pieces.
+      uint8_t* stg = smem + (size_t)w2 * (32 * 144);
+      const int tbase = t0 + mb * BM + q * 32;  // first token of this warp's rows
       if (mb < n_mb) {
         for (int c0 = ch * (BF / 2); c0 < min(nmma, (ch + 1) * (BF / 2)); c0 += 32) {
           uint32_t v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mb * BF + c0), v);
-          if (!tvalid) continue;
           const int nf = min(32, n_rows - row0 - c0);  // features of this chunk that exist
           if (p.splits > 1) {
-            float* dst = p.partial + ((size_t)split * p.T + t) * p.ldy + colbase + c0;
             if (vec && nf == 32) {
 #pragma unroll
-              for (int e = 0; e < 32; e += 4) *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
-            } else {
+              for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<uint4*>(stg + lane * 144 + e * 4) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const int r = 4 * j + (lane >> 3), cq = lane & 7;
+                const uint4 val = *reinterpret_cast<const uint4*>(stg + r * 144 + cq * 16);
+                const int tt = tbase + r;
+                if (tt < p.T) *reinterpret_cast<uint4*>(p.partial + ((size_t)split * p.T + tt) * p.ldy + colbase + c0 + cq * 4) = val;
+              }
+              __syncwarp();
+            } else if (tvalid) {
+              float* dst = p.partial + ((size_t)split * p.T + t) * p.ldy + colbase + c0;
 #pragma unroll
               for (int e = 0; e < 32; ++e)
                 if (e < nf) dst[e] = __uint_as_float(v[e]);
             }
           } else {
-            __half* dst = p.y + (size_t)t * p.ldy + colbase + c0;
             if (vec && nf == 32) {
 #pragma unroll
               for (int e = 0; e < 32; e += 8) {
@@ -402,22 +415,34 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
                   const __half2 h = __floats2half2_rn(__uint_as_float(v[e + 2 * j]), __uint_as_float(v[e + 2 * j + 1]));
                   o[j] = *reinterpret_cast<const uint32_t*>(&h);
                 }
-                *reinterpret_cast<uint4*>(dst + e) = make_uint4(o[0], o[1], o[2], o[3]);
-                if (p.res) {
-                  const size_t off = (size_t)t * p.ldy + colbase + c0 + e;
-                  const uint4 r4 = *reinterpret_cast<const uint4*>(p.res + off);
-                  const uint32_t rr[4] = {r4.x, r4.y, r4.z, r4.w};
-                  uint32_t z[4];
+                *reinterpret_cast<uint4*>(stg + lane * 80 + e * 2) = make_uint4(o[0], o[1], o[2], o[3]);
+              }
+              __syncwarp();
 #pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    const float2 a = __half22float2(u2h2(o[j])), b = __half22float2(u2h2(rr[j]));
-                    const __half2 h = __floats2half2_rn(b.x + a.x, b.y + a.y);
-                    z[j] = *reinterpret_cast<const uint32_t*>(&h);
+              for (int j = 0; j < 4; ++j) {
+                const int r = 8 * j + (lane >> 2), cq = lane & 3;
+                const uint4 o4 = *reinterpret_cast<const uint4*>(stg + r * 80 + cq * 16);
+                const int tt = tbase + r;
+                if (tt < p.T) {
+                  const size_t off = (size_t)tt * p.ldy + colbase + c0 + cq * 8;
+                  *reinterpret_cast<uint4*>(p.y + off) = o4;
+                  if (p.res) {
+                    const uint4 r4 = *reinterpret_cast<const uint4*>(p.res + off);
+                    const uint32_t oo[4] = {o4.x, o4.y, o4.z, o4.w}, rr[4] = {r4.x, r4.y, r4.z, r4.w};
+                    uint32_t z[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                      const float2 a = __half22float2(u2h2(oo[u])), b = __half22float2(u2h2(rr[u]));
+                      const __half2 h = __floats2half2_rn(b.x + a.x, b.y + a.y);
+                      z[u] = *reinterpret_cast<const uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(p.y2 + off) = make_uint4(z[0], z[1], z[2], z[3]);
                   }
-                  *reinterpret_cast<uint4*>(p.y2 + off) = make_uint4(z[0], z[1], z[2], z[3]);
                 }
               }
-            } else {
+              __syncwarp();
+            } else if (tvalid) {
+              __half* dst = p.y + (size_t)t * p.ldy + colbase + c0;
 #pragma unroll
               for (int e = 0; e < 32; ++e)
                 if (e < nf) {
@@ -514,7 +539,7 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 // Tile configuration and split-K factor for one launch, picked by a small cost model (SM cycles): the CTAs run in
-// waves of sm_count; a wide k-step (256 x 256 x 64) costs about 1250 cycles and a narrow one (128 x 128 x 64) about 750,
+// waves of sm_count; a wide k-step (256 x 256 x 64) costs about 1250 cycles and a narrow one (128 x 128 x 64) about 1150,
 // both bound by the L2 traffic of the activation tile rather than by the tensor pipe, which is why few wide CTAs with
 // split-K beat many narrow ones; split-K adds the fp32 partial traffic and a second launch.
 struct GemmPlan {
@@ -527,7 +552,7 @@ GemmPlan choose_plan(int tiles_wide, int tiles_narrow, int T, int n_cols, int to
   for (int w = 0; w < 2; ++w) {
     const int tt = w ? 256 : 128;
     const int ctas = (w ? tiles_wide : tiles_narrow) * ((T + tt - 1) / tt);
-    const double kstep = w ? 1250.0 : 750.0;
+    const double kstep = w ? 1250.0 : 1150.0;
     for (int s = 1; s <= 8; ++s) {
       if (s > 1 && (total_ksteps / s < 8 || (uint64_t)s * T * n_cols * 4 > scratch_bytes)) break;
       const int per = (total_ksteps + s - 1) / s;

@@ -22,46 +22,67 @@ __device__ __forceinline__ float wmax(float v) {
   return v;
 }
 
-// thread <-> (token, pair index i): one fp64 sincos per (token, i), reused over all heads.
-__global__ void rope_append_prefill_kernel(const __half* __restrict__ qkv, int ld, __half* __restrict__ q_rot,
-                                           __half* __restrict__ kc, __half* __restrict__ vc, int T, int n_q, int n_kv, int d,
-                                           int cap, int pos0, float theta) {
-  const int half = d / 2;
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= T * half) return;
-  const int t = idx / half, i = idx % half;
-  const int pos = pos0 + t;
-  float c = 1.f, s = 0.f;
-  if (theta != 0.f) {
-    const double inv = pow((double)theta, -2.0 * (double)i / (double)d);
-    double sd, cd;
-    sincos((double)pos * inv, &sd, &cd);
-    c = (float)cd;
-    s = (float)sd;
+// One CTA per token.  The cos/sin table of the token's position (one fp64 sincos per pair index i) goes to shared memory;
+// the threads then take (head, run of 8 pair indices) tasks with 16-byte loads and stores: rotate q into q_rot, rotate k
+// into the key cache, copy v into the value cache.
+__global__ void __launch_bounds__(256) rope_append_prefill_kernel(const __half* __restrict__ qkv, int ld, __half* __restrict__ q_rot,
+                                                                  __half* __restrict__ kc, __half* __restrict__ vc, int n_q, int n_kv,
+                                                                  int d, int cap, int pos0, float theta) {
+  __shared__ float2 cs_s[128];  // d <= 256
+  const int half = d / 2, t = blockIdx.x, pos = pos0 + t;
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    float c = 1.f, s = 0.f;
+    if (theta != 0.f) {
+      const double inv = pow((double)theta, -2.0 * (double)i / (double)d);
+      double sd, cd;
+      sincos((double)pos * inv, &sd, &cd);
+      c = (float)cd;
+      s = (float)sd;
+    }
+    cs_s[i] = make_float2(c, s);
   }
+  __syncthreads();
   const __half* row = qkv + (size_t)t * ld;
   const int qd = n_q * d, kvd = n_kv * d;
-  for (int hq = 0; hq < n_q; ++hq) {
-    const float a = __half2float(row[hq * d + i]), b = __half2float(row[hq * d + i + half]);
-    q_rot[(size_t)t * qd + hq * d + i] = __float2half_rn(a * c - b * s);
-    q_rot[(size_t)t * qd + hq * d + i + half] = __float2half_rn(b * c + a * s);
+  const int segs = half / 8;  // runs of 8 pair indices per head
+  for (int task = threadIdx.x; task < (n_q + n_kv) * segs; task += blockDim.x) {
+    const int head = task / segs, i0 = (task % segs) * 8;
+    const bool is_q = head < n_q;
+    const __half* src = row + (is_q ? head * d : qd + (head - n_q) * d);
+    __half* dst = is_q ? q_rot + (size_t)t * qd + head * d : kc + ((size_t)(head - n_q) * cap + pos) * d;
+    const uint4 a4 = *reinterpret_cast<const uint4*>(src + i0), b4 = *reinterpret_cast<const uint4*>(src + half + i0);
+    const uint32_t aw[4] = {a4.x, a4.y, a4.z, a4.w}, bw[4] = {b4.x, b4.y, b4.z, b4.w};
+    uint32_t ra[4], rb[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      __half2 ah, bh;
+      *reinterpret_cast<uint32_t*>(&ah) = aw[q];
+      *reinterpret_cast<uint32_t*>(&bh) = bw[q];
+      const float2 a = __half22float2(ah), b = __half22float2(bh);
+      const float2 cs0 = cs_s[i0 + 2 * q], cs1 = cs_s[i0 + 2 * q + 1];
+      const __half2 oa = __floats2half2_rn(a.x * cs0.x - b.x * cs0.y, a.y * cs1.x - b.y * cs1.y);
+      const __half2 ob = __floats2half2_rn(b.x * cs0.x + a.x * cs0.y, b.y * cs1.x + a.y * cs1.y);
+      ra[q] = *reinterpret_cast<const uint32_t*>(&oa);
+      rb[q] = *reinterpret_cast<const uint32_t*>(&ob);
+    }
+    *reinterpret_cast<uint4*>(dst + i0) = make_uint4(ra[0], ra[1], ra[2], ra[3]);
+    *reinterpret_cast<uint4*>(dst + half + i0) = make_uint4(rb[0], rb[1], rb[2], rb[3]);
   }
-  for (int kvh = 0; kvh < n_kv; ++kvh) {
-    const float a = __half2float(row[qd + kvh * d + i]), b = __half2float(row[qd + kvh * d + i + half]);
-    __half* dst = kc + ((size_t)kvh * cap + pos) * d;
-    dst[i] = __float2half_rn(a * c - b * s);
-    dst[i + half] = __float2half_rn(b * c + a * s);
-    __half* vd = vc + ((size_t)kvh * cap + pos) * d;
-    vd[i] = row[qd + kvd + kvh * d + i];
-    vd[i + half] = row[qd + kvd + kvh * d + i + half];
+  for (int task = threadIdx.x; task < n_kv * (d / 8); task += blockDim.x) {
+    const int kvh = task / (d / 8), c = (task % (d / 8)) * 8;
+    *reinterpret_cast<uint4*>(vc + ((size_t)kvh * cap + pos) * d + c) = *reinterpret_cast<const uint4*>(row + qd + kvd + kvh * d + c);
   }
 }
 
 cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_rot16, __half* kc, __half* vc, int T,
                                        int n_q, int n_kv, int d, int cap, int pos0, float theta, cudaStream_t st,
                                        uint64_t* n_launch) {
-  const int total = T * (d / 2);
-  rope_append_prefill_kernel<<<(total + 127) / 128, 128, 0, st>>>(qkv16, ld, q_rot16, kc, vc, T, n_q, n_kv, d, cap, pos0, theta);
+  // 16-byte accesses: head_dim a multiple of 16, rows and caches 16-byte aligned
+  if (d % 16 != 0 || d > 256 || ld % 8 != 0 ||
+      (((reinterpret_cast<uintptr_t>(qkv16) | reinterpret_cast<uintptr_t>(q_rot16) | reinterpret_cast<uintptr_t>(kc) |
+         reinterpret_cast<uintptr_t>(vc)) & 15) != 0))
+    return cudaErrorInvalidValue;
+  rope_append_prefill_kernel<<<T, 256, 0, st>>>(qkv16, ld, q_rot16, kc, vc, n_q, n_kv, d, cap, pos0, theta);
   ++*n_launch;
   return cudaGetLastError();
 }
