@@ -148,6 +148,33 @@ cudaError_t launch_gemv_stream(const GemvParams& p, int* status, int sm_count, c
 // Grouped-expert GEMV: job j multiplies the slice w0[j] (and w1[j] for SwiGLU) with activation row xrow[j] and
 // writes output row j_out[j].  Implicit mode (n_jobs_explicit == 0): job p = 0..P-1 uses expert ids[p] of a
 // contiguous resident tensor.
+// Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the stream is
+// still finishing; every kernel launched this way executes griddepcontrol.wait before it touches the predecessor's data.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dep(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int pdl, int cluster_x,
+                              Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[na].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+  ++na;
+  if (cluster_x > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = cluster_x;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 constexpr int kMoeJobsPerLaunch = 64;
 struct MoeJobs {
   const uint8_t* w0[kMoeJobsPerLaunch];
@@ -210,10 +237,11 @@ cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uin
 // prefill
 cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_rot16, __half* kc, __half* vc, int T,
                                        int n_q, int n_kv, int d, int cap, int pos0, float theta, cudaStream_t st,
-                                       uint64_t* n_launch);
+                                       uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const __half* vc, __half* a16, int T, int n_q,
-                                int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch);
-cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch);
+                                int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
+cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch,
+                            int pdl = 0);
 
 // Tensor-core GEMM  Y[T][n_rows] (fp16, leading dimension ldy) = X[T][K] (fp16, ld = ldx) * W^T for up to 3 weight
 // segments laid side by side in Y.  `scratch` holds split-K partials (gemm_scratch_bytes()).
@@ -232,6 +260,7 @@ struct GemmParams {
   // optional fused residual: y2[t][c] = rn16(res[t][c] + y[t][c]) with y the fp16-rounded product (both ld = ldy)
   const __half* res;
   __half* y2;
+  int pdl;  // programmatic dependent launch allowed (see launch_dep)
 };
 uint64_t gemm_scratch_bytes(int T, int n_total, int K);
 cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);

@@ -1185,22 +1185,24 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
   plan_dense(ctx, L->w_down, &wd);
   ATS_TRY(pump(ctx));
 
+  const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
   GemmParams g{};
   g.T = (int)T;
   g.scratch = w.gemm_scratch;
   g.scratch_bytes = w.gemm_scratch_bytes;
+  g.pdl = pdl;
   const __half* resid = (const __half*)x_in;
   if (attn) {
-    ATS_CUDA(launch_rmsnorm(x_in, 0, (const __half*)ctx->tensors[L->attn_norm].f16_dev, w.h16, (int)T, H, L->rms_eps, ctx->cs, nl));
+    ATS_CUDA(launch_rmsnorm(x_in, 0, (const __half*)ctx->tensors[L->attn_norm].f16_dev, w.h16, (int)T, H, L->rms_eps, ctx->cs, nl, pdl));
     g.x = w.h16;
     g.ldx = H;
     g.y = w.qkv16;
     g.ldy = qd + 2 * kvd;
     ATS_TRY(run_gemm_group(ctx, qkv, 3, g));
     ATS_CUDA(launch_rope_append_prefill(w.qkv16, qd + 2 * kvd, w.qrot16, (__half*)k_cache, (__half*)v_cache, (int)T, nq, nkv, d,
-                                        (int)L->kv_capacity, (int)pos0, L->rope_theta, ctx->cs, nl));
+                                        (int)L->kv_capacity, (int)pos0, L->rope_theta, ctx->cs, nl, pdl));
     ATS_CUDA(launch_attn_prefill(w.qrot16, (const __half*)k_cache, (const __half*)v_cache, w.a16, (int)T, nq, nkv, d,
-                                 (int)L->kv_capacity, (int)pos0, ctx->cs, nl));
+                                 (int)L->kv_capacity, (int)pos0, ctx->cs, nl, pdl));
     g.x = w.a16;
     g.ldx = qd;
     g.y = w.o16;
@@ -1212,13 +1214,13 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     g.y2 = nullptr;
     resid = w.x1_16;
   }
-  ATS_CUDA(launch_rmsnorm(resid, 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, w.h2_16, (int)T, H, L->rms_eps, ctx->cs, nl));
+  ATS_CUDA(launch_rmsnorm(resid, 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, w.h2_16, (int)T, H, L->rms_eps, ctx->cs, nl, pdl));
   g.x = w.h2_16;
   g.ldx = H;
   g.y = w.gu16;
   g.ldy = 2 * (int)L->ffn;
   ATS_TRY(run_gemm_group(ctx, gu, 2, g));
-  ATS_CUDA(launch_swiglu16(w.gu16, 2 * (int)L->ffn, (int)L->ffn, w.act16, (int)T, ctx->cs, nl));
+  ATS_CUDA(launch_swiglu16(w.gu16, 2 * (int)L->ffn, (int)L->ffn, w.act16, (int)T, ctx->cs, nl, pdl));
   g.x = w.act16;
   g.ldx = (int)L->ffn;
   g.y = w.d16;

@@ -370,33 +370,6 @@ __device__ __forceinline__ float load_f<float>(const float* p, size_t i) { retur
 template <>
 __device__ __forceinline__ float load_f<__half>(const __half* p, size_t i) { return __half2float(p[i]); }
 
-// Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the stream is
-// still finishing; every kernel launched this way executes griddepcontrol.wait before it touches the predecessor's data.
-template <typename... KArgs, typename... Args>
-static cudaError_t launch_dep(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int pdl, int cluster_x,
-                              Args... args) {
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[2];
-  int na = 0;
-  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[na].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
-  ++na;
-  if (cluster_x > 1) {
-    attr[na].id = cudaLaunchAttributeClusterDimension;
-    attr[na].val.clusterDim.x = cluster_x;
-    attr[na].val.clusterDim.y = 1;
-    attr[na].val.clusterDim.z = 1;
-    ++na;
-  }
-  cfg.attrs = attr;
-  cfg.numAttrs = na;
-  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
-}
-
 template <typename TIn>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const TIn* __restrict__ x, const __half* __restrict__ gain,
                                                       __half* __restrict__ out, int H, float eps) {

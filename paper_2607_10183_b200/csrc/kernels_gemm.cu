@@ -205,6 +205,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_s;
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (activation tile)
@@ -474,6 +475,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
 __global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, __half* __restrict__ y, int T, int n_cols, int ldy,
                                           int splits, const __half* __restrict__ res, __half* __restrict__ y2) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const size_t plane = (size_t)T * ldy;
   if (n_cols % 8 == 0 && ldy % 8 == 0 &&
       (((reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(res) | reinterpret_cast<uintptr_t>(y2)) & 15) == 0)) {
@@ -641,24 +643,24 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
     attr_set = true;
   }
   dim3 grid(tiles, tchunks, p.splits);
+  ++*n_launch;
+  cudaError_t e;
   if (wide) {
     using Cfg = TileCfg<2, 256>;
     p.stages = Cfg::kStages;
-    gemm_q4_kernel<2, 256><<<grid, Cfg::kThreads, (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st>>>(xmap, p);
+    e = launch_dep(gemm_q4_kernel<2, 256>, grid, dim3(Cfg::kThreads), (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, p);
   } else {
     using Cfg = TileCfg<1, 128>;
     p.stages = Cfg::kStages;
-    gemm_q4_kernel<1, 128><<<grid, Cfg::kThreads, (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st>>>(xmap, p);
+    e = launch_dep(gemm_q4_kernel<1, 128>, grid, dim3(Cfg::kThreads), (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, p);
   }
-  ++*n_launch;
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (p.splits > 1) {
     const size_t total = (size_t)g.T * col;
-    const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)sm_count * 8);
-    gemm_splitk_reduce_kernel<<<blocks, 256, 0, st>>>(p.partial, g.y, g.T, col, g.ldy, p.splits, g.res, g.y2);
+    const int blocks = (int)std::min<size_t>((total / 8 + 255) / 256 + 1, (size_t)sm_count * 8);
     ++*n_launch;
-    e = cudaGetLastError();
+    e = launch_dep(gemm_splitk_reduce_kernel, dim3(blocks), dim3(256), 0, st, g.pdl, 1, (const float*)p.partial, g.y, g.T, col, g.ldy,
+                   p.splits, g.res, g.y2);
   }
   return e;
 }

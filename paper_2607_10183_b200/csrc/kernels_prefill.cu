@@ -29,6 +29,8 @@ __global__ void __launch_bounds__(256) rope_append_prefill_kernel(const __half* 
                                                                   __half* __restrict__ kc, __half* __restrict__ vc, int n_q, int n_kv,
                                                                   int d, int cap, int pos0, float theta) {
   __shared__ float2 cs_s[128];  // d <= 256
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int half = d / 2, t = blockIdx.x, pos = pos0 + t;
   for (int i = threadIdx.x; i < half; i += blockDim.x) {
     float c = 1.f, s = 0.f;
@@ -76,15 +78,15 @@ __global__ void __launch_bounds__(256) rope_append_prefill_kernel(const __half* 
 
 cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_rot16, __half* kc, __half* vc, int T,
                                        int n_q, int n_kv, int d, int cap, int pos0, float theta, cudaStream_t st,
-                                       uint64_t* n_launch) {
+                                       uint64_t* n_launch, int pdl) {
   // 16-byte accesses: head_dim a multiple of 16, rows and caches 16-byte aligned
   if (d % 16 != 0 || d > 256 || ld % 8 != 0 ||
       (((reinterpret_cast<uintptr_t>(qkv16) | reinterpret_cast<uintptr_t>(q_rot16) | reinterpret_cast<uintptr_t>(kc) |
          reinterpret_cast<uintptr_t>(vc)) & 15) != 0))
     return cudaErrorInvalidValue;
-  rope_append_prefill_kernel<<<T, 256, 0, st>>>(qkv16, ld, q_rot16, kc, vc, n_q, n_kv, d, cap, pos0, theta);
   ++*n_launch;
-  return cudaGetLastError();
+  return launch_dep(rope_append_prefill_kernel, dim3(T), dim3(256), 0, st, pdl, 1, qkv16, ld, q_rot16, kc, vc, n_q, n_kv, d, cap, pos0,
+                    theta);
 }
 
 // Causal grouped-query attention over the cache on the tensor cores (mma.sync m16n8k16, fp16 operands, fp32 accumulate).
@@ -130,6 +132,8 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(const __half* __restr
   __half* k_s = q_s + kFaQ * PITCH;               // [2][kFaK][PITCH]
   __half* v_s = k_s + 2 * kFaK * PITCH;           // [2][kFaK][PITCH]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int qb = blockIdx.x, hq = blockIdx.y, kvh = hq / group;
   const int tq0 = qb * kFaQ;                      // first token of the CTA
   const int n_kb = (pos0 + min(T, tq0 + kFaQ) - 1) / kFaK + 1;  // cache blocks any row of the CTA attends to
@@ -266,7 +270,7 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(const __half* __restr
 }
 
 cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const __half* vc, __half* a16, int T, int n_q,
-                                int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch) {
+                                int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch, int pdl) {
   dim3 grid((T + kFaQ - 1) / kFaQ, n_q);
   const float scale = 1.0f / sqrtf((float)d);
   const size_t smem = (size_t)(kFaQ + 4 * kFaK) * (d + 8) * sizeof(__half);
@@ -280,18 +284,20 @@ cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const _
     if (e2 != cudaSuccess) return e2;
     attr_set = true;
   }
-  if (d == 128)
-    attn_prefill_kernel<128><<<grid, 128, smem, st>>>(q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0, scale);
-  else if (d == 64)
-    attn_prefill_kernel<64><<<grid, 128, smem, st>>>(q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0, scale);
-  else
-    return cudaErrorInvalidValue;
   ++*n_launch;
-  return cudaGetLastError();
+  if (d == 128)
+    return launch_dep(attn_prefill_kernel<128>, grid, dim3(128), smem, st, pdl, 1, q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0,
+                      scale);
+  if (d == 64)
+    return launch_dep(attn_prefill_kernel<64>, grid, dim3(128), smem, st, pdl, 1, q_rot16, kc, vc, a16, T, n_q, n_q / n_kv, cap, pos0,
+                      scale);
+  return cudaErrorInvalidValue;
 }
 
 // gu holds [T][ld] with gate in columns [0, ffn) and up in [ffn, 2 ffn): act = rn16(silu(g) * u); 8 elements per thread
 __global__ void swiglu16_kernel(const __half* __restrict__ gu, int ld, int ffn, __half* __restrict__ act, uint64_t n8) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int per_row = ffn / 8;
   for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * blockDim.x) {
     const uint64_t t = i / per_row, c = (i % per_row) * 8;
@@ -309,12 +315,11 @@ __global__ void swiglu16_kernel(const __half* __restrict__ gu, int ld, int ffn, 
   }
 }
 
-cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch) {
+cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch, int pdl) {
   const uint64_t n8 = (uint64_t)T * ffn / 8;  // ffn is a multiple of 32
   const int grid = (int)std::min<uint64_t>((n8 + 255) / 256, 148 * 8);
-  swiglu16_kernel<<<grid, 256, 0, st>>>(gu, ld, ffn, act, n8);
   ++*n_launch;
-  return cudaGetLastError();
+  return launch_dep(swiglu16_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, gu, ld, ffn, act, n8);
 }
 
 }  // namespace ats
