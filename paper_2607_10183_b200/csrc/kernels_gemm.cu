@@ -204,7 +204,10 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_s;
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations come from the preceding kernel
+  // Only the activations come from the preceding kernel: the TMA producer waits for it, the weight path (parameters)
+  // starts at once, and everything that touches other kernels' data (epilogue stores, the residual read) is ordered
+  // behind the producer's wait through the pipeline's barriers.  Dependents are released after that wait, never before.
+  if (warp == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
