@@ -28,7 +28,7 @@ EDGES = ("h", "q", "k", "v", "q_rot", "a", "o", "x1", "h2", "g", "u", "act", "d"
 
 EXPORTS = (
     "ats_init", "ats_destroy", "ats_last_error", "ats_register_tensor", "ats_tensor_slice_bytes", "ats_set_placement",
-    "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode",
+    "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode", "ats_layer_decode_host",
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
     "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
     "ats_host_unpack_q4",
@@ -81,6 +81,7 @@ def _load():
         "ats_route_topk": (i32, [vp, i32, vp, u32, u32, vp, vp]),
         "ats_moe_linear": (i32, [vp, i32, vp, vp, vp, u32, u32, u32]),
         "ats_layer_decode": (i32, [vp, P(ats_layer_desc), vp, vp, vp, vp, u32, u32]),
+        "ats_layer_decode_host": (i32, [vp, P(ats_layer_desc), vp, vp, vp, vp, u32, u32]),
         "ats_layer_prefill": (i32, [vp, P(ats_layer_desc), vp, vp, vp, vp, u32, u32]),
         "ats_workspace_bytes": (u64, [P(ats_layer_desc), u32]),
         "ats_dequantize": (i32, [vp, i32, i32, vp, u32]),
@@ -230,6 +231,10 @@ class Context:
 
     def layer_decode(self, desc, x_in, x_out, k_cache, v_cache, pos, M=1):
         return self.check(lib.ats_layer_decode(self.h, C.byref(desc), _ptr(x_in), _ptr(x_out), _ptr(k_cache), _ptr(v_cache), pos, M))
+
+    def layer_decode_host(self, desc, x_in_host, x_out_host, k_cache, v_cache, pos, M=1):
+        return self.check(lib.ats_layer_decode_host(self.h, C.byref(desc), _ptr(x_in_host), _ptr(x_out_host), _ptr(k_cache),
+                                                    _ptr(v_cache), pos, M))
 
     def layer_prefill(self, desc, x_in, x_out, k_cache, v_cache, pos0, T):
         return self.check(lib.ats_layer_prefill(self.h, C.byref(desc), _ptr(x_in), _ptr(x_out), _ptr(k_cache), _ptr(v_cache), pos0, T))

@@ -1007,6 +1007,8 @@ uint64_t ats_workspace_bytes(const ats_layer_desc* L, uint32_t max_tokens) {
   if (!L || max_tokens == 0) return 0;
   uint64_t need = layout_decode(*L, std::min<uint32_t>(max_tokens, 32), nullptr, ~0ull).total;
   if (L->n_experts == 0) need = std::max(need, layout_prefill(*L, max_tokens, nullptr, ~0ull).total);
+  // staging rows of ats_layer_decode_host (input and output), each padded to the arena alignment
+  need += 2 * align_up((uint64_t)std::min<uint32_t>(max_tokens, 32) * L->hidden * 2);
   return need + kAlign;
 }
 
@@ -1153,6 +1155,28 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   ATS_TRY(run_moe_stage(ctx, L->w_down, -1, w.ids, ids_host, s2));
   ATS_CUDA(launch_moe_combine(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, w.gates, w.d32, (__half*)x_out, (int)M, k, H,
                               ctx->cs, nl, pdl));
+  return ATS_OK;
+}
+
+int32_t ats_layer_decode_host(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in, void* x_out, void* k_cache,
+                              void* v_cache, uint32_t pos, uint32_t M) {
+  ATS_TRY(precheck(ctx, true));
+  ATS_TRY(check_layer(ctx, L, false));
+  if (!x_in || !x_out) return fail(ctx, ATS_ERR_INVALID, "null activation pointer");
+  if (M == 0) return ATS_OK;
+  if (M > 32) return fail(ctx, ATS_ERR_SHAPE, "decode takes M <= 32");
+  // the staging rows sit behind everything the device call lays out in the workspace
+  const LayerWs w = layout_decode(*L, M, nullptr, ~0ull);
+  const uint64_t row_bytes = (uint64_t)M * L->hidden * 2, stage = align_up(row_bytes);
+  const uint64_t need = w.total + 2 * stage;
+  if (need > align_up(ctx->cfg.workspace_bytes))
+    return fail(ctx, ATS_ERR_NOMEM, "workspace too small: host-driven decode needs %llu bytes", (unsigned long long)need);
+  uint8_t* xin_dev = ctx->ws + w.total;
+  uint8_t* xout_dev = xin_dev + stage;
+  ATS_CUDA(cudaMemcpyAsync(xin_dev, x_in, row_bytes, cudaMemcpyHostToDevice, ctx->cs));
+  ATS_TRY(ats_layer_decode(ctx, L, xin_dev, xout_dev, k_cache, v_cache, pos, M));
+  ATS_CUDA(cudaMemcpyAsync(x_out, xout_dev, row_bytes, cudaMemcpyDeviceToHost, ctx->cs));
+  ATS_CUDA(cudaStreamSynchronize(ctx->cs));
   return ATS_OK;
 }
 

@@ -129,8 +129,9 @@ def test_linear_closed_forms_on_gpu(B, torch):
 
 
 # ------------------------------------------------------------------------------------------------- dense layer decode
-def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, flags=0, steps=1, chunk=MB):
-    """Returns (list of y per step, final K cache, final V cache, stats) for one layer."""
+def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, flags=0, steps=1, chunk=MB, host_io=False):
+    """Returns (list of y per step, final K cache, final V cache, stats) for one layer.  host_io: drive the step through
+    ats_layer_decode_host from pinned host buffers instead of device buffers."""
     L = W.dense_layer(cfg, 0, shape)
     slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
     ctx = make_ctx(B, H.dense_layer_bytes(shape) + 16 * 256 + 4 * shape.hidden * 2, ring_slots=ring_slots, slot_bytes=slot,
@@ -144,6 +145,12 @@ def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, fl
     ctx.reset_stats()
     for s in range(steps):
         x = W.activations(cfg, 0, (1, shape.hidden), step=s)
+        if host_io:
+            xh = torch.from_numpy(x).pin_memory()
+            yh = torch.zeros((1, shape.hidden), dtype=torch.float16).pin_memory()
+            ctx.layer_decode_host(desc, xh, yh, kd, vd, pos + s, 1)  # returns with yh valid: no sync here
+            ys.append(yh.numpy().copy())
+            continue
         y = torch.empty((1, shape.hidden), dtype=torch.float16, device="cuda")
         ctx.layer_decode(desc, H.to_dev(x), y, kd, vd, pos + s, 1)
         ctx.sync()
@@ -179,6 +186,18 @@ def test_dense_layer_decode_matches_oracle(B, torch, shape_name, pos, cap):
         ulp = np.spacing(np.abs(ref[:, pos]).astype(np.float16)).astype(np.float64)
         assert np.all(np.abs(a - b) <= ulp + 2e-5 * np.abs(b).max())
     assert st.streamed_bytes == 0 and st.resident_bytes == H.dense_layer_bytes(shape)
+
+
+def test_host_driven_decode_equals_device_driven(B, torch):
+    """ats_layer_decode_host (H2D, step, D2H, wait) returns bit for bit what ats_layer_decode leaves on the device, with
+    resident and with streamed tensors, over consecutive steps that extend the same caches."""
+    shape, cfg, pos, cap = W.DENSE_SMALL, 96, 20, 40
+    for placement in (ALL_GPU, {**ALL_GPU, "wk": 0, "w_up": 0, "w_down": 0}):
+        dev = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, steps=3)
+        host = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, steps=3, host_io=True)
+        for a, b in zip(dev[0], host[0]):
+            assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+        assert np.array_equal(dev[1], host[1]) and np.array_equal(dev[2], host[2])
 
 
 def test_placement_invariance_and_bookkeeping_small(B, torch):
