@@ -229,6 +229,56 @@ def test_placement_invariance_and_bookkeeping_small(B, torch):
         assert st.n_streamed == 3 * where.count(0)
 
 
+def test_stack_under_planned_budget_full_size(B, torch):
+    """Config-5 shape: a stack of full-size layers under a 60 % byte budget placed by ats_plan_placement (Algorithm 1).
+    Decode steps through the stack equal the all-resident run bit for bit; the bytes and copies that moved are the
+    oracle's bookkeeping for the planned placement; the planned placement equals the oracle's DP on the same records."""
+    shape, cfg, n_layers, cap, pos = W.DENSE_FULL, 5, 2, 48, 32
+    layer_bytes = H.dense_layer_bytes(shape)
+    slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+    chunk = 8 * MB
+    nbytes = [W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes()]
+
+    def run(budget_frac):
+        ctx = make_ctx(B, n_layers * (layer_bytes + 16 * 256) + 8 * shape.hidden * 2, ws=16 * MB, ring_slots=4, slot_bytes=slot,
+                       chunk_bytes=chunk)
+        descs, q4 = [], []
+        for l in range(n_layers):
+            desc, ids = H.register_dense_layer(ctx, W.dense_layer(cfg, l, shape), l, cap)
+            descs.append(desc)
+            q4 += [ids[n] for n in ALL_GPU]
+        if budget_frac is None:
+            ctx.set_placement([(i, -1, 1) for i in q4])
+            where = np.ones(len(q4), dtype=np.uint8)
+        else:
+            where = ctx.plan_placement(int(budget_frac * n_layers * layer_bytes), len(q4))
+        caches = [tuple(H.to_dev(c) for c in W.kv_cache(cfg, l, shape.n_kv_heads, cap, shape.head_dim, pos)) for l in range(n_layers)]
+        ctx.reset_stats()
+        outs = []
+        for s in range(2):
+            a = H.to_dev(W.activations(cfg, 0, (1, shape.hidden), step=s))
+            b = torch.empty_like(a)
+            for l in range(n_layers):
+                ctx.layer_decode(descs[l], a, b, caches[l][0], caches[l][1], pos + s, 1)
+                a, b = b, a
+            ctx.sync()
+            outs.append(a.cpu().numpy().copy())
+        st = ctx.stats()
+        ctx.close()
+        return outs, where, st
+
+    res, _, st_res = run(None)
+    hyb, where, st = run(0.60)
+    assert 0 < int(where.sum()) < len(where)
+    for a, b in zip(res, hyb):
+        assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    assert st_res.streamed_bytes == 0
+    per_step_bytes, per_step_copies, _ = O.streamed_dense(nbytes * n_layers, [int(w) for w in where], chunk)
+    assert st.streamed_bytes == 2 * per_step_bytes and st.copies == 2 * per_step_copies
+    assert st.resident_bytes == sum(b for b, w in zip(nbytes * n_layers, where) if w)
+    assert st.resident_bytes <= int(0.60 * n_layers * layer_bytes)
+
+
 def test_gate_up_both_streamed_needs_two_slots(B, torch):
     shape = W.DENSE_SMALL
     with pytest.raises(B.AtsError) as e:
