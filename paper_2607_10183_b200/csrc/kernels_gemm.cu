@@ -54,6 +54,7 @@ struct GemmKParams {
   int n_seg;
   int K, T;
   int total_ksteps, ksteps_per_split, splits;
+  int bf;  // feature rows per CTA tile: a multiple of 32, at most the configuration's width (narrower tiles even out the waves)
   __half* y;
   int ldy;
   float* partial;  // [splits][T][ldy] when splits > 1
@@ -174,11 +175,12 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
   const int tile = blockIdx.x;
   int sg = 0;
   while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
-  const int row0 = (tile - p.seg[sg].tile0) * BF;
+  const int row0 = (tile - p.seg[sg].tile0) * p.bf;
   const int n_rows = p.seg[sg].n_rows;
   const int t0 = blockIdx.y * TTILE;
   const int Tt = min(TTILE, p.T - t0);
-  const int nmma = min(BF, (n_rows - row0 + 15) / 16 * 16);  // MMA N: the features of this tile that hold real rows
+  const int nmma = min(p.bf, (n_rows - row0 + 15) / 16 * 16);  // MMA N: the features of this tile that hold real rows
+  const int n_dq = (p.bf + 15) / 16;                           // dequantization warps with rows to fill (16 rows each)
   const int boxes = (Tt + BOXR - 1) / BOXR;                  // TMA boxes of 64 activation rows
   const int n_mb = (Tt + BM - 1) / BM;                       // 128-token blocks (MMA M) that hold real tokens
   const int split = blockIdx.z;
@@ -187,7 +189,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
   if (threadIdx.x == 0) {
     fail_s = 0;
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(&full_a[s], kDequantWarps);  // one arrival per dequantization warp
+      mbar_init(&full_a[s], n_dq);  // one arrival per dequantization warp that has rows
       mbar_init(&full_b[s], 1);
       mbar_init(&empty[s], 1);
     }
@@ -305,12 +307,13 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
       const uint32_t w = d == 0 ? v.x : d == 1 ? v.y : d == 2 ? v.z : v.w;
       return (w >> (16 * hb)) & 0xFFFFu;
     };
-    if (vec_sc) snext = fetch_scale8(ks0);
+    const int nks_dq = w2 < n_dq ? nks : 0;  // warps beyond the tile's width have no rows: they only take part in the epilogue
+    if (vec_sc && nks_dq > 0) snext = fetch_scale8(ks0);
 #pragma unroll
     for (int d = 0; d < kPD; ++d) {
       qbuf[d] = make_uint4(0, 0, 0, 0);
       sbuf[d] = 0;
-      if (d < nks) {
+      if (d < nks_dq) {
         fetch_codes(ks0 + d, qbuf[d]);
         sbuf[d] = vec_sc ? pick(snext, d) : fetch_scale1(ks0 + d);
       }
@@ -318,7 +321,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
     bool ok = true;
     int s = 0, round = 0;
     const int sw = r & 7, cb = hb * 4;
-    for (int i0 = 0; i0 < nks && ok; i0 += kPD) {
+    for (int i0 = 0; i0 < nks_dq && ok; i0 += kPD) {
       if (vec_sc && i0 + kPD < nks) snext = fetch_scale8(ks0 + i0 + kPD);
 #pragma unroll
       for (int d = 0; d < kPD; ++d) {
@@ -388,7 +391,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
         for (int c0 = ch * (BF / 2); c0 < min(nmma, (ch + 1) * (BF / 2)); c0 += 32) {
           uint32_t v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mb * BF + c0), v);
-          const int nf = min(32, n_rows - row0 - c0);  // features of this chunk that exist
+          const int nf = min(32, min(p.bf, n_rows - row0) - c0);  // features of this chunk that exist and belong to this tile
           if (p.splits > 1) {
             if (vec && nf == 32) {
 #pragma unroll
@@ -550,24 +553,36 @@ EncodeTiledFn encode_tiled_fn() {
 struct GemmPlan {
   bool wide;
   int splits;
+  int bf;  // feature rows per tile
 };
-GemmPlan choose_plan(int tiles_wide, int tiles_narrow, int T, int n_cols, int total_ksteps, int sm_count, uint64_t scratch_bytes) {
-  GemmPlan best{false, 1};
+// Cost model in SM cycles.  CTAs run in waves of sm_count.  A k-step (64 k) of a 256-token x w-feature tile is bound by
+// shared-memory traffic: about 1250 cycles at w = 256, of which the part that scales with w (weight-tile stores and the
+// tensor core's reads of them) is 60 %; a 128 x 128 k-step costs about 1150.  Narrower tiles than the configuration's
+// full width are considered because they can even out the waves (28672 features at 512 tokens: 224 tiles of 256 take
+// two waves of which the second is half empty; 276 tiles of 208 fill both).  Split-K adds the fp32 partial traffic and
+// a second launch.
+GemmPlan choose_plan(const int* seg_rows, int n_seg, int T, int n_cols, int total_ksteps, int sm_count, uint64_t scratch_bytes) {
+  GemmPlan best{false, 1, 128};
   double best_cost = 1e30;
   for (int w = 0; w < 2; ++w) {
-    const int tt = w ? 256 : 128;
-    const int ctas = (w ? tiles_wide : tiles_narrow) * ((T + tt - 1) / tt);
-    const double kstep = w ? 1250.0 : 1150.0;
-    for (int s = 1; s <= 8; ++s) {
-      if (s > 1 && (total_ksteps / s < 8 || (uint64_t)s * T * n_cols * 4 > scratch_bytes)) break;
-      const int per = (total_ksteps + s - 1) / s;
-      if ((s - 1) * per >= total_ksteps) continue;  // the last split would be empty
-      const int waves = (ctas * s + sm_count - 1) / sm_count;
-      double cost = (double)waves * (per * kstep + 9000.0);
-      if (s > 1) cost += 8000.0 + (double)(s + 1) * T * n_cols * 4.0 / 2000.0;  // second launch + partials at ~2 KB per cycle
-      if (cost < best_cost) {
-        best_cost = cost;
-        best = GemmPlan{w != 0, s};
+    const int tt = w ? 256 : 128, full = w ? 256 : 128;
+    const int tchunks = (T + tt - 1) / tt;
+    for (int bf = full; bf >= (w ? 160 : 128); bf -= 32) {  // multiples of 32: whole 32-column epilogue chunks
+      int tiles = 0;
+      for (int i = 0; i < n_seg; ++i) tiles += (seg_rows[i] + bf - 1) / bf;
+      const int ctas = tiles * tchunks;
+      const double kstep = w ? 1250.0 * (0.4 + 0.6 * bf / 256.0) : 1150.0;
+      for (int s = 1; s <= 8; ++s) {
+        if (s > 1 && (total_ksteps / s < 8 || (uint64_t)s * T * n_cols * 4 > scratch_bytes)) break;
+        const int per = (total_ksteps + s - 1) / s;
+        if ((s - 1) * per >= total_ksteps) continue;  // the last split would be empty
+        const int waves = (ctas * s + sm_count - 1) / sm_count;
+        double cost = (double)waves * (per * kstep + 9000.0);
+        if (s > 1) cost += 8000.0 + (double)(s + 1) * T * n_cols * 4.0 / 2000.0;  // second launch + partials at ~2 KB per cycle
+        if (cost < best_cost * 0.97 || (cost < best_cost && bf == full)) {  // a narrower tile has to pay for itself
+          if (cost < best_cost) best_cost = cost;
+          best = GemmPlan{w != 0, s, bf};
+        }
       }
     }
   }
@@ -579,7 +594,7 @@ GemmPlan choose_plan(int tiles_wide, int tiles_narrow, int T, int n_cols, int to
 uint64_t gemm_scratch_bytes(int T, int n_total, int K) {
   // fp32 partials of the plan this shape gets with unlimited scratch (the launcher re-plans within the buffer it is given)
   const int total_ksteps = (K + BK - 1) / BK;
-  const GemmPlan pl = choose_plan((n_total + 255) / 256, (n_total + 127) / 128, T, n_total, total_ksteps, 148, ~0ull);
+  const GemmPlan pl = choose_plan(&n_total, 1, T, n_total, total_ksteps, 148, ~0ull);
   return pl.splits > 1 ? (uint64_t)pl.splits * T * n_total * 4 + 256 : 256;
 }
 
@@ -608,17 +623,15 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
   int n_total = 0;
   for (int i = 0; i < g.n_seg; ++i) n_total += g.seg[i].n_rows;
-  int tiles_w = 0, tiles_n = 0;
-  for (int i = 0; i < g.n_seg; ++i) {
-    tiles_w += (g.seg[i].n_rows + 255) / 256;
-    tiles_n += (g.seg[i].n_rows + 127) / 128;
-  }
+  int seg_rows[3] = {0, 0, 0};
+  for (int i = 0; i < g.n_seg; ++i) seg_rows[i] = g.seg[i].n_rows;
   const int total_ksteps = (g.K + BK - 1) / BK;
-  const GemmPlan pl = choose_plan(tiles_w, tiles_n, g.T, g.ldy, total_ksteps, sm_count, g.scratch ? g.scratch_bytes : 0);
+  const GemmPlan pl = choose_plan(seg_rows, g.n_seg, g.T, g.ldy, total_ksteps, sm_count, g.scratch ? g.scratch_bytes : 0);
   const bool wide = pl.wide;
-  const int bf = wide ? 256 : 128, tt = wide ? 256 : 128;
+  const int bf = pl.bf, tt = wide ? 256 : 128;
   GemmKParams p{};
   p.n_seg = g.n_seg;
+  p.bf = bf;
   int tiles = 0, col = 0;
   for (int i = 0; i < g.n_seg; ++i) {
     p.seg[i] = GemmSeg{g.seg[i].base, g.seg[i].n_rows, tiles, col};
