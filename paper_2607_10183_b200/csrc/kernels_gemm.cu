@@ -14,7 +14,7 @@
 // order) in 16-byte pieces.
 //
 // Warp roles: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2.. = weight dequantization, then epilogue.
-// No cluster launch and no multicast.  Every mbarrier wait is bounded; on expiry the CTA raises the status word, skips
+// One CTA per tile, no cluster launch.  Every mbarrier wait is bounded; on expiry the CTA raises the status word, skips
 // the rest of its work, frees its tensor memory and returns.
 #include <cuda.h>
 
