@@ -148,6 +148,16 @@ cudaError_t launch_gemv_stream(const GemvParams& p, int* status, int sm_count, c
 // Grouped-expert GEMV: job j multiplies the slice w0[j] (and w1[j] for SwiGLU) with activation row xrow[j] and
 // writes output row j_out[j].  Implicit mode (n_jobs_explicit == 0): job p = 0..P-1 uses expert ids[p] of a
 // contiguous resident tensor.
+// Function attributes (the dynamic shared-memory limit) are per device: a launcher sets them the first time it runs on
+// each device.  `done` holds one bit per device ordinal; setting an attribute twice is harmless, so no lock is needed.
+inline bool first_use_on_device(uint64_t* done) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+  if ((*done >> dev) & 1ull) return false;
+  *done |= 1ull << dev;
+  return true;
+}
+
 // Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the stream is
 // still finishing; every kernel launched this way executes griddepcontrol.wait before it touches the predecessor's data.
 template <typename... KArgs, typename... Args>

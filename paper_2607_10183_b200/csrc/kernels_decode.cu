@@ -498,8 +498,8 @@ cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStr
   cfg.gridDim = dim3(splits, p.n_kv);
   cfg.blockDim = dim3(p.group * pc);
   cfg.dynamicSmemBytes = (size_t)pc * (d * 4 + 16);
-  static bool attr_set = false;
-  if (!attr_set) {
+  static uint64_t attr_done = 0;
+  if (first_use_on_device(&attr_done)) {
     cudaError_t e[4] = {
         cudaFuncSetAttribute(attn_decode_fused_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * (128 * 4 + 16)),
         cudaFuncSetAttribute(attn_decode_fused_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (128 * 4 + 16)),
@@ -507,7 +507,6 @@ cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStr
         cudaFuncSetAttribute(attn_decode_fused_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (64 * 4 + 16))};
     for (cudaError_t x : e)
       if (x != cudaSuccess) return x;
-    attr_set = true;
   }
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -710,11 +709,9 @@ cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, 
     const int L = E / 8, R = kRouterClThreads / L;
     const size_t smem_cl = ((size_t)H / kRouterCluster + (size_t)R * E + (size_t)(kRouterCluster + 1) * Epad) * sizeof(float);
     if (smem_cl <= 160 * 1024) {
-      static size_t attr_bytes = 0;
-      if (smem_cl > 48 * 1024 && smem_cl > attr_bytes) {
+      if (smem_cl > 48 * 1024) {  // (cheap; set on every call because the size depends on the shape)
         cudaError_t e = cudaFuncSetAttribute(router_topk_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_cl);
         if (e != cudaSuccess) return e;
-        attr_bytes = smem_cl;
       }
       ++*n_launch;
       return launch_dep(router_topk_cluster_kernel, dim3(kRouterCluster, M), dim3(kRouterClThreads), smem_cl, st, pdl, kRouterCluster,

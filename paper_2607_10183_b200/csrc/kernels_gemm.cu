@@ -650,13 +650,12 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   p.status = g.status;
   p.res = g.res;
   p.y2 = g.y2;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static uint64_t attr_done = 0;
+  if (first_use_on_device(&attr_done)) {
     cudaError_t e1 = cudaFuncSetAttribute(gemm_q4_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     cudaError_t e2 = cudaFuncSetAttribute(gemm_q4_kernel<1, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e1 != cudaSuccess) return e1;
     if (e2 != cudaSuccess) return e2;
-    attr_set = true;
   }
   dim3 grid(tiles, tchunks, p.splits);
   ++*n_launch;

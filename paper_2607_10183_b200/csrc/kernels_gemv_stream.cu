@@ -612,12 +612,11 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
     case 4: kern = sw ? gemv_stream_kernel<4, true> : gemv_stream_kernel<4, false>; break;
     default: kern = sw ? gemv_stream_kernel<8, true> : gemv_stream_kernel<8, false>; break;
   }
-  static bool attr_set[8] = {};
+  static uint64_t attr_done[8] = {};
   const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
-  if (!attr_set[ki]) {
+  if (first_use_on_device(&attr_done[ki])) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (e != cudaSuccess) return e;
-    attr_set[ki] = true;
   }
   if (smem > 100 * 1024) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
@@ -680,12 +679,11 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
     case 4: kern = sw ? gemv_stream_moe_kernel<4, true> : gemv_stream_moe_kernel<4, false>; break;
     default: kern = sw ? gemv_stream_moe_kernel<8, true> : gemv_stream_moe_kernel<8, false>; break;
   }
-  static bool attr_set[8] = {};
+  static uint64_t attr_done[8] = {};
   const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
-  if (!attr_set[ki]) {
+  if (first_use_on_device(&attr_done[ki])) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (e != cudaSuccess) return e;
-    attr_set[ki] = true;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(per_job, n_jobs);

@@ -274,15 +274,14 @@ cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const _
   dim3 grid((T + kFaQ - 1) / kFaQ, n_q);
   const float scale = 1.0f / sqrtf((float)d);
   const size_t smem = (size_t)(kFaQ + 4 * kFaK) * (d + 8) * sizeof(__half);
-  static bool attr_set = false;
-  if (!attr_set) {
+  static uint64_t attr_done = 0;
+  if (first_use_on_device(&attr_done)) {
     cudaError_t e1 = cudaFuncSetAttribute(attn_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)((kFaQ + 4 * kFaK) * (128 + 8) * sizeof(__half)));
     cudaError_t e2 = cudaFuncSetAttribute(attn_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)((kFaQ + 4 * kFaK) * (64 + 8) * sizeof(__half)));
     if (e1 != cudaSuccess) return e1;
     if (e2 != cudaSuccess) return e2;
-    attr_set = true;
   }
   ++*n_launch;
   if (d == 128)
