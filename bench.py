@@ -286,7 +286,7 @@ def extra_moe(torch, B, W, peaks, quick):
     Bk = W.moe_block(4, 0, shape)
     sl = W.q4_bytes(shape.ffn, shape.hidden)
     out = {"workload": "config 4: MoE block decode; hybrid = odd experts host-placed", "expert_slice_bytes": sl}
-    for hybrid in (False, True):
+    for hybrid in (False, True, "gather"):
         ctx = B.Context(3 * shape.n_experts * (sl + 256) + 64 * (sl + 256) + (16 << 20), workspace_bytes=8 << 20, ring_slots=64,
                         slot_bytes=sl, chunk_bytes=sl)
         ids = {"ffn_norm": ctx.register_f16(Bk[W.ROLE_FFN_NORM]), "router": ctx.register_f16(Bk[W.ROLE_ROUTER])}
@@ -295,9 +295,11 @@ def extra_moe(torch, B, W, peaks, quick):
         desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, rms_eps=shape.rms_eps, **ids)
         ctx.set_placement([(ids[n], e, B.ATS_HOST if (hybrid and e % 2) else B.ATS_GPU) for n in ("w_gate", "w_up", "w_down")
                            for e in range(shape.n_experts)])
-        if hybrid:
+        if hybrid == "gather":
+            ctx.set_flags(B.ATS_FLAG_MOE_DEVICE_GATHER)  # host-placed experts read in place over PCIe, ids stay on the device
+        elif hybrid:
             out["pcie_h2d_measured_gbs"] = ctx.measure_h2d(64 * sl, 10)
-        for M in (1, 8):
+        for M in ((1,) if hybrid == "gather" else (1, 8)):  # the gather path takes single-token calls
             xs = [torch.from_numpy(W.activations(4, 0, (M, shape.hidden), step=s)).cuda() for s in range(16)]
             y = torch.empty((M, shape.hidden), dtype=torch.float16, device="cuda")
             n = 64 if quick else 256
@@ -313,7 +315,7 @@ def extra_moe(torch, B, W, peaks, quick):
             ctx.sync()
             dt = (time.perf_counter() - t0) / n
             st = ctx.stats()
-            key = f"{'hybrid' if hybrid else 'resident'}_M{M}"
+            key = f"{'hybrid_device_gather' if hybrid == 'gather' else 'hybrid' if hybrid else 'resident'}_M{M}"
             out[key] = {"us_per_call": dt * 1e6, "tokens_per_s": M / dt, "streamed_bytes_per_call": st.streamed_bytes / n,
                         "launches_per_call": st.kernel_launches / n, "timing": "wall clock around back-to-back calls (host included)"}
             if not hybrid:
@@ -323,7 +325,14 @@ def extra_moe(torch, B, W, peaks, quick):
                 out[key]["device_us_per_call"] = dev_ms * 1e3 / n
                 moe_bytes = shape.top_k * min(M, shape.n_experts) * 3 * sl  # upper bound: all selected experts distinct
                 out[key]["expert_bytes_per_call_upper"] = moe_bytes
-            if hybrid and st.streamed_bytes:
+            if hybrid == "gather":
+                # the same inputs select the same experts as in the ring run: its byte count applies
+                moved = out[f"hybrid_M{M}"]["streamed_bytes_per_call"]
+                out[key]["host_bytes_read_per_call"] = moved
+                out[key]["pcie_gbs_over_call_time"] = moved / dt / 1e9
+                dev_ms = event_time_ms(torch, ctx.compute, lambda: go(n))
+                out[key]["device_us_per_call"] = dev_ms * 1e3 / n
+            elif hybrid and st.streamed_bytes:
                 out[key]["pcie_gbs_over_call_time"] = st.streamed_bytes / n / dt / 1e9
         ctx.close()
     return out

@@ -60,6 +60,13 @@ enum {
   ATS_FLAG_SKIP_SCALE_CHECK = 2u, /* do not scan scales for Inf/NaN at registration */
   ATS_FLAG_TIME_KERNELS = 4u,     /* bracket every GEMV / grouped GEMV / GEMM launch with CUDA events (see ats_stats.timed_*) */
   ATS_FLAG_NO_PDL = 8u,           /* launch every kernel fully serialized (no programmatic dependent launch overlap) */
+  ATS_FLAG_MOE_DEVICE_GATHER = 16u, /* single-token MoE stages with host-placed experts: no staging ring and no host round trip for the
+                                     routing ids: the grouped-expert kernel reads the selected host-placed slices straight
+                                     from the pinned host store over PCIe (the store is mapped into the device's address
+                                     space), picking each slice's address from a per-tensor table on the device by the
+                                     expert id (the zero-copy path of Sections 4.1 / 4.2.1).  Same arithmetic, same results;
+                                     ats_stats.streamed_bytes / copies / host_syncs do not count these reads.  Calls with
+                                     more than one token keep the ring path (it moves every distinct expert once). */
   /* timing experiments only: do not launch a stage of ats_layer_decode (its outputs are then stale); bit 24 = QKV GEMV,
    * 25 = attention, 26 = O GEMV, 27 = gate/up GEMV, 28 = down GEMV */
   ATS_FLAG_DEBUG_SKIP_SHIFT = 24

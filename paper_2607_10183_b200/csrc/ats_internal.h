@@ -41,6 +41,9 @@ struct Tensor {
   std::vector<Slice> slices;
   bool any_host = true;        // some slice is host-placed
   bool contiguous_dev = false; // all slices resident, at dev0 + e * slice_stride
+  // expert-stacked tensors: device array of one address per slice, the resident copy or the slice's place in the pinned
+  // host store as the device sees it (mapped memory); null for single-slice tensors
+  const uint8_t** slice_tab_dev = nullptr;
 };
 
 struct RingSlot {
@@ -199,6 +202,8 @@ struct MoeGemvParams {
   const uint8_t* base1;
   uint64_t stride;
   const int32_t* ids;  // [P]
+  const uint8_t* const* tab0;  // optional per-expert slice addresses (device array); when set they replace base + id * stride
+  const uint8_t* const* tab1;
   int x_div;           // activation row of pair p is p / x_div (k when one x per token, 1 when one per slot)
   int P;
   // common

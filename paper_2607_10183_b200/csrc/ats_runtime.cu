@@ -428,6 +428,7 @@ static int32_t apply_placement(ats_ctx* ctx) {
       aux += t.host_bytes;
       continue;
     }
+    if (t.slices.size() > 1) off = align_up(off) + t.slices.size() * sizeof(uint8_t*);  // the slice address table
     for (Slice& s : t.slices)
       if (s.where == ATS_GPU) {
         off = align_up(off) + t.slice_stride;
@@ -451,6 +452,12 @@ static int32_t apply_placement(ats_ctx* ctx) {
     }
     t.any_host = false;
     t.contiguous_dev = true;
+    t.slice_tab_dev = nullptr;
+    if (t.slices.size() > 1) {
+      off = align_up(off);
+      t.slice_tab_dev = reinterpret_cast<const uint8_t**>(ctx->resident + off);
+      off += t.slices.size() * sizeof(uint8_t*);
+    }
     uint8_t* prev = nullptr;
     for (size_t e = 0; e < t.slices.size(); ++e) {
       Slice& s = t.slices[e];
@@ -467,6 +474,22 @@ static int32_t apply_placement(ats_ctx* ctx) {
         t.contiguous_dev = false;
       }
     }
+  }
+  // slice address tables: the resident copy, or the slice inside the pinned host store at the address the device sees
+  for (Tensor& t : ctx->tensors) {
+    if (!t.slice_tab_dev) continue;
+    void* host_dev = nullptr;
+    if (cudaHostGetDevicePointer(&host_dev, t.host, 0) != cudaSuccess) {
+      cudaGetLastError();
+      t.slice_tab_dev = nullptr;  // the store is not mapped on this system: the ring path remains
+      continue;
+    }
+    std::vector<const uint8_t*> tab(t.slices.size());
+    for (size_t e = 0; e < t.slices.size(); ++e)
+      tab[e] = t.slices[e].where == ATS_GPU ? t.slices[e].dev : static_cast<const uint8_t*>(host_dev) + e * t.slice_stride;
+    ATS_CUDA(cudaMemcpyAsync(const_cast<uint8_t**>(t.slice_tab_dev), tab.data(), tab.size() * sizeof(uint8_t*), cudaMemcpyHostToDevice,
+                             ctx->ts));
+    ATS_CUDA(cudaStreamSynchronize(ctx->ts));  // `tab` is pageable and goes out of scope
   }
   ATS_CUDA(cudaStreamSynchronize(ctx->ts));
   ctx->stats.resident_bytes = resident;
@@ -498,8 +521,13 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
   p.stride = t0.slice_stride;
   p.ids = ids_dev;
   if (!ids_host) {
-    p.base0 = t0.slices[0].dev;
-    p.base1 = t1 ? t1->slices[0].dev : nullptr;
+    if (t0.contiguous_dev && (!t1 || t1->contiguous_dev)) {
+      p.base0 = t0.slices[0].dev;
+      p.base1 = t1 ? t1->slices[0].dev : nullptr;
+    } else {  // device-initiated gather: addresses from the per-tensor tables
+      p.tab0 = t0.slice_tab_dev;
+      p.tab1 = t1 ? t1->slice_tab_dev : nullptr;
+    }
     TimedLaunch tl(ctx, 1, (uint64_t)p.P * ((t1 ? 2 : 1) * t0.slice_bytes + (uint64_t)p.K * 2 + (uint64_t)p.n_rows * 2));
     ATS_CUDA(launch_moe_gemv_any(ctx, p, nullptr));
     return ATS_OK;
@@ -1126,7 +1154,17 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   ATS_CUDA(launch_router_topk(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)M, H, E, k,
                               (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, ctx->cs, nl, pdl));
   const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
-  const bool implicit = tg.contiguous_dev && tu.contiguous_dev && td.contiguous_dev;
+  bool implicit = tg.contiguous_dev && tu.contiguous_dev && td.contiguous_dev;
+  if (!implicit && M == 1 && (ctx->cfg.flags & ATS_FLAG_MOE_DEVICE_GATHER) && tg.slice_tab_dev && tu.slice_tab_dev && td.slice_tab_dev) {
+    // the kernels find every selected slice themselves, in device memory or in the mapped host store: no ids on the
+    // host, no ring (shapes the streaming kernel does not take keep the ring path).  One token only: its k experts are
+    // distinct, so every host-placed slice crosses PCIe once; with several tokens, pairs that share an expert would each
+    // read it again, and the ring path, which moves every distinct expert once, is the better one.
+    MoeGemvParams probe1{}, probe2{};
+    probe1.K = H; probe1.n_rows = (int)L->ffn; probe1.mode = GEMV_SWIGLU_F16;
+    probe2.K = (int)L->ffn; probe2.n_rows = H; probe2.mode = GEMV_OUT_F32;
+    if (moe_gemv_stream_eligible(probe1) && moe_gemv_stream_eligible(probe2)) implicit = true;
+  }
   const int32_t* ids_host = nullptr;
   if (!implicit) {
     ATS_TRY(fetch_ids(ctx, w.ids, P, E));

@@ -526,6 +526,8 @@ struct MoeSel {
   const uint8_t* base1;
   unsigned long long stride;
   const int32_t* ids;  // null: use the job table
+  const uint8_t* const* tab0;  // with ids: per-expert slice addresses (device memory or mapped pinned host memory)
+  const uint8_t* const* tab1;
   int x_div;
   int ldx, ldy;
 };
@@ -537,8 +539,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_stream_moe_kernel(const Stre
   if (m.ids) {
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the ids come from the router kernel
     const size_t e = (size_t)m.ids[job];
-    p.seg[0].base = m.base0 + e * m.stride;
-    if (SW) p.seg[1].base = m.base1 + e * m.stride;
+    p.seg[0].base = m.tab0 ? m.tab0[e] : m.base0 + e * m.stride;
+    if (SW) p.seg[1].base = m.tab1 ? m.tab1[e] : m.base1 + e * m.stride;
     xrow = job / m.x_div;
     orow = job;
   } else {
@@ -663,6 +665,8 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   m.base1 = g.base1;
   m.stride = g.stride;
   m.ids = jobs ? nullptr : g.ids;
+  m.tab0 = g.tab0;
+  m.tab1 = g.tab1;
   m.x_div = g.x_div;
   m.ldx = g.ldx;
   m.ldy = g.ldy;

@@ -355,6 +355,26 @@ def test_moe_block_matches_oracle_and_streams_only_selected_experts(B, torch, sh
     assert got_order == [(2 + t_, e) for t_, e in order][:len(got_order)]
 
 
+@pytest.mark.parametrize("M", [1, 8])
+def test_moe_device_gather_equals_resident_without_host_round_trip(B, torch, M):
+    """ATS_FLAG_MOE_DEVICE_GATHER: the grouped-expert kernels read the selected host-placed experts straight from the mapped
+    pinned store, addressed through the per-tensor slice table by the ids on the device.  Same bits as the all-resident
+    run, no host synchronisation, nothing through the staging ring."""
+    shape, cfg = W.MOE_FULL, 4
+    odd = {e for e in range(shape.n_experts) if e % 2}
+    _, _, y_res, _ = run_moe(B, torch, shape, cfg, M, set())
+    _, _, y_dg, st = run_moe(B, torch, shape, cfg, M, odd, flags=B.ATS_FLAG_MOE_DEVICE_GATHER)
+    assert np.array_equal(y_res.view(np.uint16), y_dg.view(np.uint16))
+    # every expert on the host
+    _, _, y_all, st_all = run_moe(B, torch, shape, cfg, M, set(range(shape.n_experts)), flags=B.ATS_FLAG_MOE_DEVICE_GATHER)
+    assert np.array_equal(y_res.view(np.uint16), y_all.view(np.uint16))
+    if M == 1:  # the gather path: nothing through the ring, no ids on the host
+        assert st.host_syncs == 0 and st.streamed_bytes == 0 and st.copies == 0
+        assert st_all.host_syncs == 0 and st_all.streamed_bytes == 0
+    else:       # several tokens keep the ring path (every distinct expert moves once)
+        assert st.host_syncs == 1 and st.streamed_bytes > 0
+
+
 def test_moe_small_ring_forces_waves(B, torch):
     shape = W.MOE_SMALL
     everything = set(range(shape.n_experts))
