@@ -380,8 +380,77 @@ def extra_stream(torch, B, W, peaks, quick, n_layers=None):
             "frac_of_measured_pcie": streamed / dt / 1e9 / pcie, "fully_overlapped_at_80pct": bool(dt <= streamed / (0.8 * pcie * 1e9))}
 
 
+def extra_model_loop(torch, B, W, peaks, quick):
+    """Whole-model loop on the config-2 layer shape: a stack of dense layers, all resident; a 2048-token prompt prefilled in
+    512-token chunks (the chunks attend to the cache the earlier ones wrote), then 128 decode steps, each through every
+    layer and a 128256-row LM head GEMV.  Synthetic embeddings stand in for the token lookup; no final norm."""
+    shape = W.DENSE_FULL
+    L = 8 if quick else 32
+    prompt, chunk, gen, vocab = 2048, 512, 32 if quick else 128, 128256
+    cap = prompt + gen
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=cap)
+    head_bytes = W.q4_bytes(vocab, shape.hidden)
+    ws = max(B.workspace_bytes(probe, chunk), B.workspace_bytes(probe, 1)) + (1 << 20)
+    layer_bytes = sum(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+    arena = ws + L * (layer_bytes + 16 * 1024 + 4 * shape.hidden) + head_bytes + (2 << 20)
+    ctx = B.Context(arena, workspace_bytes=ws)
+    names = {W.ROLE_Q: "wq", W.ROLE_K: "wk", W.ROLE_V: "wv", W.ROLE_O: "wo", W.ROLE_GATE: "w_gate", W.ROLE_UP: "w_up", W.ROLE_DOWN: "w_down"}
+    descs, q4 = [], []
+    for l in range(L):
+        Lw = W.dense_layer(6, l % 4, shape)  # four distinct weight sets, registered L times (distinct copies in HBM)
+        # random layers amplify the residual stream from layer to layer; small norm gains keep 32 of them inside fp16
+        damp = np.float16(0.1)
+        ids = {"attn_norm": ctx.register_f16(Lw[W.ROLE_ATTN_NORM] * damp, l, W.ROLE_ATTN_NORM)}
+        for r in (W.ROLE_Q, W.ROLE_K, W.ROLE_V, W.ROLE_O):
+            ids[names[r]] = ctx.register_q4(*Lw[r], layer=l, role=r)
+        ids["ffn_norm"] = ctx.register_f16(Lw[W.ROLE_FFN_NORM] * damp, l, W.ROLE_FFN_NORM)
+        for r in (W.ROLE_GATE, W.ROLE_UP, W.ROLE_DOWN):
+            ids[names[r]] = ctx.register_q4(*Lw[r], layer=l, role=r)
+        q4 += [ids[names[r]] for r in names]
+        descs.append(B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                                  head_dim=shape.head_dim, kv_capacity=cap, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, **ids))
+    head = ctx.register_q4(*W.q4_packed(6, 0, W.ROLE_Q, vocab, shape.hidden), layer=L, role=W.ROLE_Q)
+    ctx.set_placement([(i, -1, B.ATS_GPU) for i in q4 + [head]])
+    caches = [(torch.zeros((shape.n_kv_heads, cap, shape.head_dim), dtype=torch.float16, device="cuda"),
+               torch.zeros((shape.n_kv_heads, cap, shape.head_dim), dtype=torch.float16, device="cuda")) for _ in range(L)]
+    xs = [torch.from_numpy(W.activations(6, 0, (chunk, shape.hidden), step=c) * 0.25).cuda() for c in range(prompt // chunk)]
+    pa, pb = torch.empty_like(xs[0]), torch.empty_like(xs[0])
+    d0 = torch.from_numpy(W.activations(6, 1, (1, shape.hidden)) * 0.25).cuda()  # the (synthetic) embedding of every step's token
+    da, db = torch.empty_like(d0), torch.empty_like(d0)
+    logits = torch.empty((1, vocab), dtype=torch.float16, device="cuda")
+
+    def prefill():
+        for c, x in enumerate(xs):
+            src, dst = x, pa
+            for l in range(L):
+                ctx.layer_prefill(descs[l], src, dst, caches[l][0], caches[l][1], c * chunk, chunk)
+                src, dst = dst, (pb if dst is pa else pa)
+
+    def decode(n):
+        for s in range(n):
+            src, dst = d0, da
+            for l in range(L):
+                ctx.layer_decode(descs[l], src, dst, caches[l][0], caches[l][1], prompt + s, 1)
+                src, dst = dst, (db if dst is da else da)
+            ctx.linear(head, src, logits, 1)
+    prefill()
+    decode(2)
+    ctx.sync()
+    pre_ms = event_time_ms(torch, ctx.compute, prefill)
+    dec_ms = event_time_ms(torch, ctx.compute, lambda: decode(gen))
+    finite = bool(torch.isfinite(logits.float()).all().item())
+    ctx.close()
+    weight_bytes = L * layer_bytes + head_bytes
+    return {"workload": f"{L}-layer dense stack + LM head ({vocab} rows), all resident: prompt {prompt} in chunks of {chunk}, then {gen} decode steps",
+            "layers": L, "weight_bytes": weight_bytes, "prefill_ms": pre_ms, "prefill_tokens_per_s": prompt / (pre_ms * 1e-3),
+            "decode_ms_per_token": dec_ms / gen, "decode_tokens_per_s": gen / (dec_ms * 1e-3),
+            "decode_weight_gbs": weight_bytes / (dec_ms / gen * 1e-3) / 1e9,
+            "decode_frac_of_measured_hbm": weight_bytes / (dec_ms / gen * 1e-3) / 1e9 / peaks["hbm_gbs"], "logits_finite": finite}
+
+
 STACK_LAYERS = [0]
-EXTRAS = {"cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
+EXTRAS = {"model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
 
 
 def run_ours(args):
@@ -527,7 +596,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the figures of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--quick", action="store_true", help="smaller extras")
-    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream"],
+    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop"],
                     help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
     ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = 8, or 4 with --quick; 32 = the full configuration)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")
@@ -538,7 +607,7 @@ def main():
         import torch
         from paper_2607_10183_b200 import binding as B, workloads as W
         torch.cuda.set_device(0)
-        print(json.dumps({args.only_extra: EXTRAS[args.only_extra](torch, B, W, load_peaks(), True)}))
+        print(json.dumps({args.only_extra: EXTRAS[args.only_extra](torch, B, W, load_peaks(), args.quick or args.only_extra != "model_loop")}))
         return
     if args.impl == "reference":
         return run_reference(args)

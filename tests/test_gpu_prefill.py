@@ -163,6 +163,67 @@ def test_prefill_then_decode_continues_the_cache(B, torch):
     ctx.close()
 
 
+def test_model_loop_chunked_prefill_then_decode_three_layers(B, torch):
+    """The whole-model loop on a small stack: a 40-token prompt prefilled in chunks of 16, 16 and 8 through three layers
+    with distinct weights (later chunks attend to the cache the earlier ones wrote), then two decode steps through the
+    same layers.  Every layer call is held against the oracle run on exactly what the library was given (its input rows
+    and its cache state before the call), so rounding differences do not compound from layer to layer."""
+    shape, cfg, cap, n_layers = W.DENSE_SMALL, 98, 48, 3
+    layers = [W.dense_layer(cfg, l, shape) for l in range(n_layers)]
+    ctx = make_stack_ctx(B, shape, cap, 16, n_layers)
+    descs, place = [], []
+    for l, Lw in enumerate(layers):
+        desc, ids = H.register_dense_layer(ctx, Lw, l, cap)
+        descs.append(desc)
+        place += [(ids[n], -1, 1) for n in ALL_GPU]
+    ctx.set_placement(place)
+    caches = [tuple(H.to_dev(c) for c in W.kv_cache(cfg, l, shape.n_kv_heads, cap, shape.head_dim, 0)) for l in range(n_layers)]
+    e_pre, w_pre = ctx.numerics(B.ATS_MODE_PREFILL)
+    e_dec, w_dec = ctx.numerics(B.ATS_MODE_DECODE)
+
+    def run_layer(l, x_host, pos, T, prefill):
+        kc0, vc0 = caches[l][0].cpu().numpy().copy(), caches[l][1].cpu().numpy().copy()
+        y = torch.empty((T, shape.hidden), dtype=torch.float16, device="cuda")
+        if prefill:
+            ctx.layer_prefill(descs[l], H.to_dev(x_host), y, caches[l][0], caches[l][1], pos, T)
+        else:
+            ctx.layer_decode(descs[l], H.to_dev(x_host), y, caches[l][0], caches[l][1], pos, T)
+        ctx.sync()
+        got = y.cpu().numpy()
+        want = O.dense_layer(x_host, H.oracle_dense_tensors(layers[l]), shape, kc0, vc0, pos,
+                             e_pre if prefill else e_dec, w_pre if prefill else w_dec)
+        H.assert_close(got, want, what=f"layer {l} pos {pos} T {T} {'prefill' if prefill else 'decode'}")
+        # the oracle appended the rows the library did (fp16 values of rounded projections: a few ulps apart at most),
+        # and neither touched any other row
+        for dev_c, ref_c in ((caches[l][0], kc0), (caches[l][1], vc0)):
+            got_c = dev_c.cpu().numpy()
+            a, b = got_c[:, pos:pos + T].astype(np.float64), ref_c[:, pos:pos + T].astype(np.float64)
+            assert np.max(np.abs(a - b)) <= 4e-3 * np.max(np.abs(b))
+            assert np.array_equal(got_c[:, :pos], ref_c[:, :pos]) and np.array_equal(got_c[:, pos + T:], ref_c[:, pos + T:])
+        return got
+
+    pos = 0
+    for c, T in enumerate((16, 16, 8)):
+        x = W.activations(cfg, 0, (T, shape.hidden), step=c)
+        for l in range(n_layers):
+            x = run_layer(l, x, pos, T, True)
+        pos += T
+    for s in range(2):
+        x = W.activations(cfg, 1, (1, shape.hidden), step=s)
+        for l in range(n_layers):
+            x = run_layer(l, x, pos, 1, False)
+        pos += 1
+    ctx.close()
+
+
+def make_stack_ctx(B, shape, cap, T, n_layers):
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=cap)
+    ws = max(B.workspace_bytes(probe, T), B.workspace_bytes(probe, 1)) + MB
+    arena = ws + n_layers * (H.dense_layer_bytes(shape) + 32 * 256 + 8 * shape.hidden) + MB
+    return B.Context(arena, workspace_bytes=ws)
+
+
 def test_prefill_layer_stage_by_stage_full_size(B, torch):
     """Config 3 (512 tokens through the full-size layer), every kernel on its own: each stage's output is compared with the
     oracle's definition of that stage applied to the inputs the stage actually consumed, under both error gates."""
