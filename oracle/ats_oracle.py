@@ -166,15 +166,15 @@ def swiglu_ffn(h2, w_gate, w_up, w_down, edges, weight_mode):
     return _edge(linear(act, *w_down, weight_mode), "d", edges)
 
 
-def dense_layer(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.ndarray, pos0: int,
-                edges=frozenset(), weight_mode: int = WEIGHT_EXACT):
-    """One dense decoder layer over T = x.shape[0] tokens at positions pos0..pos0+T-1.
+def attention_block(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.ndarray, pos0: int,
+                    edges=frozenset(), weight_mode: int = WEIGHT_EXACT):
+    """The attention half of a decoder layer over T = x.shape[0] tokens at positions pos0..pos0+T-1:
+    x1 = x + W_o attention(RoPE(W_q h), cache), h = RMSNorm(x).
 
-    T == 1 is a decode step, T > 1 a prefill chunk; both are the same definition:
-    the new keys/values are written to the caches (as fp16) first, then the token at
-    position p attends to positions 0..p.  ``tensors`` maps 'wq','wk','wv','wo',
-    'w_gate','w_up','w_down' to (packed, scales) and 'attn_norm','ffn_norm' to fp16 gains.
-    The caches (fp16, [n_kv][capacity][d]) are updated in place.  Returns y as fp16.
+    The new keys/values are written to the caches (as fp16) first, then the token at position p
+    attends to positions 0..p.  ``tensors`` maps 'wq','wk','wv','wo' to (packed, scales) and
+    'attn_norm' to an fp16 gain.  The caches (fp16, [n_kv][capacity][d]) are updated in place.
+    Returns x1 (fp64 values, rounded to fp16 when 'x1' is an edge).
     """
     x = np.asarray(x, dtype=np.float64)
     T = x.shape[0]
@@ -194,10 +194,30 @@ def dense_layer(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.ndarra
         a[t] = attention_one(q_rot[t], k_cache, v_cache, pos0 + t + 1).reshape(-1)
     a = _edge(a, "a", edges)
     o = _edge(linear(a, *tensors["wo"], weight_mode), "o", edges)
-    x1 = _edge(x + o, "x1", edges)
+    return _edge(x + o, "x1", edges)
+
+
+def dense_layer(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.ndarray, pos0: int,
+                edges=frozenset(), weight_mode: int = WEIGHT_EXACT):
+    """One dense decoder layer over T = x.shape[0] tokens at positions pos0..pos0+T-1: the attention
+    block, then y = x1 + W_down(silu(W_gate h2) * (W_up h2)), h2 = RMSNorm(x1).
+
+    T == 1 is a decode step, T > 1 a prefill chunk; both are the same definition.  ``tensors`` maps
+    'wq','wk','wv','wo','w_gate','w_up','w_down' to (packed, scales) and 'attn_norm','ffn_norm' to
+    fp16 gains.  The caches are updated in place.  Returns y as fp16.
+    """
+    x1 = attention_block(x, tensors, shape, k_cache, v_cache, pos0, edges, weight_mode)
     h2 = _edge(rmsnorm(x1, tensors["ffn_norm"], shape.rms_eps), "h2", edges)
     dd = swiglu_ffn(h2, tensors["w_gate"], tensors["w_up"], tensors["w_down"], edges, weight_mode)
     return (x1 + dd).astype(np.float16)
+
+
+def moe_layer(x, attn_tensors: dict, attn_shape, moe_tensors: dict, moe_shape, k_cache: np.ndarray, v_cache: np.ndarray,
+              pos0: int, edges=frozenset(), weight_mode: int = WEIGHT_EXACT):
+    """A decoder layer whose FFN is the MoE block: the attention block, then moe_block on x1.
+    Returns (y fp16, ids, gates, logits)."""
+    x1 = attention_block(x, attn_tensors, attn_shape, k_cache, v_cache, pos0, edges, weight_mode)
+    return moe_block(x1, moe_tensors, moe_shape, edges, weight_mode)
 
 
 # --------------------------------------------------------------------------------------

@@ -375,6 +375,48 @@ def test_moe_device_gather_equals_resident_without_host_round_trip(B, torch, M):
         assert st.host_syncs == 1 and st.streamed_bytes > 0
 
 
+@pytest.mark.parametrize("host_experts", [(), (1, 3, 4, 7)])
+def test_moe_layer_with_attention_matches_oracle(B, torch, host_experts):
+    """A decoder layer whose FFN is the MoE block (attention, then router + routed experts on x1): the residual stream
+    reaches the MoE half in fp32, the experts may sit on the host.  Two consecutive decode steps extend the caches."""
+    dshape = W.DENSE_SMALL
+    mshape = W.MoEShape(hidden=dshape.hidden, n_experts=8, ffn=64, top_k=2)
+    cfg, cap, pos = 94, 24, 9
+    Lw = W.dense_layer(cfg, 0, dshape)
+    Bk = W.moe_block(cfg, 0, mshape)
+    sl = W.q4_bytes(mshape.ffn, mshape.hidden)
+    attn_bytes = sum(W.q4_bytes(n, k) for r, n, k in dshape.tensor_shapes() if r in (W.ROLE_Q, W.ROLE_K, W.ROLE_V, W.ROLE_O))
+    ctx = make_ctx(B, attn_bytes + 3 * mshape.n_experts * (sl + 256) + MB, ring_slots=6, slot_bytes=sl, chunk_bytes=MB)
+    ids = {"attn_norm": ctx.register_f16(Lw[W.ROLE_ATTN_NORM], 0, W.ROLE_ATTN_NORM)}
+    for r, n in ((W.ROLE_Q, "wq"), (W.ROLE_K, "wk"), (W.ROLE_V, "wv"), (W.ROLE_O, "wo")):
+        ids[n] = ctx.register_q4(*Lw[r], layer=0, role=r)
+    ids["ffn_norm"] = ctx.register_f16(Bk[W.ROLE_FFN_NORM], 0, W.ROLE_FFN_NORM)
+    ids["router"] = ctx.register_f16(Bk[W.ROLE_ROUTER], 0, W.ROLE_ROUTER)
+    for r, n in ((W.ROLE_GATE, "w_gate"), (W.ROLE_UP, "w_up"), (W.ROLE_DOWN, "w_down")):
+        ids[n] = ctx.register_q4(*Bk[r], layer=0, role=r)
+    desc = B.layer_desc(hidden=dshape.hidden, ffn=mshape.ffn, n_q_heads=dshape.n_q_heads, n_kv_heads=dshape.n_kv_heads,
+                        head_dim=dshape.head_dim, kv_capacity=cap, rms_eps=dshape.rms_eps, rope_theta=dshape.rope_theta,
+                        n_experts=mshape.n_experts, top_k=mshape.top_k, **ids)
+    place = [(ids[n], -1, 1) for n in ("wq", "wk", "wv", "wo")]
+    place += [(ids[n], e, 0 if e in host_experts else 1) for n in ("w_gate", "w_up", "w_down") for e in range(mshape.n_experts)]
+    ctx.set_placement(place)
+    kc, vc = W.kv_cache(cfg, 0, dshape.n_kv_heads, cap, dshape.head_dim, pos)
+    kd, vd = H.to_dev(kc), H.to_dev(vc)
+    edges, wmode = ctx.numerics(B.ATS_MODE_DECODE)
+    at = H.oracle_dense_tensors(Lw)
+    mt = H.oracle_moe_tensors(Bk)
+    for s in range(2):
+        x = W.activations(cfg, 0, (1, dshape.hidden), step=s)
+        y = torch.empty((1, dshape.hidden), dtype=torch.float16, device="cuda")
+        ctx.layer_decode(desc, H.to_dev(x), y, kd, vd, pos + s, 1)
+        ctx.sync()
+        want, ids_ref, _, logits = O.moe_layer(x, at, dshape, mt, mshape, kc, vc, pos + s, edges, wmode)
+        assert O.min_rank_gap(logits, mshape.top_k) > 1e-4, "degenerate seed: near-tie among the routed experts"
+        H.assert_close(y.cpu().numpy(), want, what=f"attention + MoE layer, step {s}")
+        assert np.array_equal(ctx.debug_decode_buffer(desc, 1, 8, np.int32).reshape(1, -1)[:, :mshape.top_k], ids_ref)
+    ctx.close()
+
+
 def test_moe_small_ring_forces_waves(B, torch):
     shape = W.MOE_SMALL
     everything = set(range(shape.n_experts))
