@@ -1,8 +1,9 @@
 // Streaming decode GEMV for one token (sm_100a): the memory-bound hot kernel of the decode path.
 //
-// Structure: persistent CTAs (2 per SM) of 8 consumer warps + 1 producer warp.  The producer streams row tiles of the
-// packed weights (codes and scales, contiguous byte ranges) into a ring of shared-memory stages with 1-D bulk-async
-// copies (TMA) that complete on mbarriers; consumers never touch global memory for weights.  Every lane owns up to two
+// Structure: one persistent CTA per SM: 16 consumer warps in two groups of 8 + 1 producer warp.  The producer streams
+// row tiles of the packed weights (codes and scales, contiguous byte ranges) into a ring of 8 shared-memory stages with
+// 1-D bulk-async copies (TMA) that complete on mbarriers; tiles alternate between the groups; consumers never touch
+// global memory for weights.  Every lane owns up to two
 // quantization blocks (32 k each) of a k-part of the row and keeps the activation for them in registers for the whole
 // kernel, so a weight byte is read once from shared memory and an activation never again.
 //
@@ -14,7 +15,7 @@
 // precomputed per block.  Lane partials are reduced by warp shuffles, k-parts through shared memory, both in fixed order.
 //
 // Optional prologue: RMSNorm of the input row (fp16 or fp32) with an fp16 gain, rounded to fp16 (the operand edge of
-// the numerics contract), computed redundantly by every CTA while its first weight tiles are in flight.
+// the numerics contract), computed once per CTA by all 512 consumer threads while the first weight tiles are in flight.
 // All waits on mbarriers are bounded; on expiry the kernel raises a status word and returns.
 #include "ats_internal.h"
 
@@ -22,12 +23,15 @@ namespace ats {
 
 namespace {
 
-constexpr int kStages = 4;
-constexpr int kConsumerWarps = 8;
+constexpr int kStages = 8;
+constexpr int kGroups = 2;         // consumer groups per CTA, each with its own stream of tiles
+constexpr int kGroupWarps = 8;
+constexpr int kConsumerWarps = kGroups * kGroupWarps;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kRPW = 2;      // rows per consumer warp per tile
 constexpr int kJ = 2;        // quantization blocks per lane per row
-constexpr int kMaxIt = 48;   // tiles whose partial sums are buffered before a flush
+constexpr int kMaxDynSmem = 216 * 1024;  // ring + quantized activation row; 6 KB of static shared memory on top
+constexpr int kMaxIt = 48;   // tiles of a group whose partial sums are buffered before a flush
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
@@ -81,7 +85,9 @@ __device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {
   asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// named barriers: 1 and 2 = the two consumer groups (256 threads each), 3 = all consumers (512); 0 is __syncthreads
+__device__ __forceinline__ void group_sync(int grp) { asm volatile("bar.sync %0, 256;" ::"r"(grp + 1) : "memory"); }
+__device__ __forceinline__ void consumer_sync_all() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 
 __device__ __forceinline__ float silu_mul_f(float g, float u) { return g / (1.0f + expf(-g)) * u; }
 
@@ -92,49 +98,13 @@ __device__ __forceinline__ int f2i_magic(float x, float up) {
   return (int)__float_as_uint(fmaf(x, up, 12582912.0f)) - 0x4B400000;
 }
 
-// 32 fp16 activations (16 registers of half2, k ascending) -> three byte planes laid out to meet the masked code words.
+// Layout of a quantized activation block (28 words): three byte planes laid out to meet the masked code words.
 // Code word w of a block holds codes k = 8w..8w+7 at nibble positions (0,2,4,6,1,3,5,7); (word & 0x0F0F0F0F) therefore
 // carries k = 8w + {0,4,1,5} in its bytes and ((word >> 4) & 0x0F0F0F0F) carries k = 8w + {2,6,3,7}.
-// planes[p*8 + 2w + h] holds byte p of xi for those four k (h = 0 / 1).  mul = 2^-sh, corr = -8 * sum(xi) * mul.
-__device__ __forceinline__ void quantize_block(const uint32_t (&xh)[16], uint32_t (&planes)[24], float& mul, float& corr) {
-  uint32_t m = 0;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) m = __vmaxu2(m, xh[i] & 0x7C007C00u);
-  int E = (int)(max(m & 0xFFFFu, m >> 16) >> 10);
-  E = max(E, 1);
-  const int sh = 36 - E;  // |xi| < 2^22
-  const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
-  mul = __uint_as_float((uint32_t)(127 - sh) << 23);
-  int xi[32];
-  int sx = 0;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    __half2 h;
-    *reinterpret_cast<uint32_t*>(&h) = xh[i];
-    const float2 f = __half22float2(h);
-    xi[2 * i] = f2i_magic(f.x, up);
-    xi[2 * i + 1] = f2i_magic(f.y, up);
-    sx += xi[2 * i] + xi[2 * i + 1];
-  }
-  corr = -8.0f * (float)sx * mul;
-#pragma unroll
-  for (int w = 0; w < 4; ++w) {
-    const int* v = xi + 8 * w;
-    // a-side: k = 0,4,1,5 ; b-side: k = 2,6,3,7
-#pragma unroll
-    for (int p = 0; p < 3; ++p) {
-      const uint32_t sel_lo = 0x0040u + 0x0011u * p;  // bytes p of (x, y) -> result bytes 0,1
-      const uint32_t a01 = __byte_perm((uint32_t)v[0], (uint32_t)v[4], sel_lo);
-      const uint32_t a23 = __byte_perm((uint32_t)v[1], (uint32_t)v[5], sel_lo);
-      const uint32_t b01 = __byte_perm((uint32_t)v[2], (uint32_t)v[6], sel_lo);
-      const uint32_t b23 = __byte_perm((uint32_t)v[3], (uint32_t)v[7], sel_lo);
-      planes[p * 8 + 2 * w] = __byte_perm(a01, a23, 0x5410u);
-      planes[p * 8 + 2 * w + 1] = __byte_perm(b01, b23, 0x5410u);
-    }
-  }
-}
-
-// The same quantization done by four adjacent lanes, each holding one run of 8 consecutive elements (one code word's
+// planes[p*8 + 2w + h] holds byte p of xi for those four k (h = 0 / 1); words 24 and 25 hold mul = 2^-sh and
+// corr = -8 * sum(xi) * mul, with sh = 36 - E for the block's largest biased fp16 exponent E (|xi| < 2^22).
+//
+// The quantization is done by four adjacent lanes, each holding one run of 8 consecutive elements (one code word's
 // worth) of a 32-element block: exponent maximum and integer sum are shared by two butterfly shuffles.  Lane w of the
 // group writes plane words 2w, 2w+1 of every plane into blk[28] (24 plane words, then mul, corr).
 __device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32_t* blk) {
@@ -198,14 +168,20 @@ struct StreamParams {
 // bx / gx: index of this CTA among the gx CTAs that share the work described by p (a whole launch for the dense GEMV, one
 // (token, slot) job of a grouped-expert launch).  wait_first: the weight addresses themselves come from the preceding
 // kernel (expert ids), so nothing may be fetched before the grid dependency resolves.
+//
+// One CTA per SM: 16 consumer warps in two groups of 8 plus the producer warp.  The CTA's tiles alternate between the
+// groups (tile it belongs to group it % 2, stage it % 8), each group with its own partial-sum buffer and barrier, so
+// the tile loop is that of two independent 8-warp CTAs; what they share is the activation prologue: all 512 consumer
+// threads load, normalise and quantise the row ONCE per SM, a quarter of the instructions two CTAs per SM spend on it
+// (for K = 14336, where every CTA used to quantise the whole row in registers, an eighth).
 template <int PARTS, bool SW>
 __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool wait_first) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t full[kStages], empty[kStages];
-  __shared__ float part_s[kMaxIt * kConsumerWarps * kRPW];
+  __shared__ float part_s[kGroups][kMaxIt * kGroupWarps * kRPW];
   __shared__ float red_s[kConsumerWarps];
   __shared__ int fail_s;
-  constexpr int ROWS = kConsumerWarps / PARTS * kRPW;  // weight rows per tile
+  constexpr int ROWS = kGroupWarps / PARTS * kRPW;     // weight rows per tile
   constexpr int OUT_ROWS = SW ? ROWS / 2 : ROWS;       // output rows per tile
   const int K = p.K, nblk = K / 32;
   const int row_codes = K / 2, row_scales = K / 16;
@@ -216,7 +192,7 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
     fail_s = 0;
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&empty[s], kConsumerWarps);
+      mbar_init(&empty[s], kGroupWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -269,108 +245,96 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
   }
 
   // ------------------------------------------------------------------ consumers
-  const int tid = threadIdx.x;                        // 0..255
+  const int tid = threadIdx.x;                // 0..511
+  const int grp = warp / kGroupWarps;         // which of the two tile streams
+  const int wg = warp % kGroupWarps;          // warp within the group
+  const int tg = tid % (kGroupWarps * 32);    // thread within the group
   // The norm gains are parameters, not products of the preceding kernel: fetch them before waiting for it.  (Every CTA
   // reads the same few kilobytes, and such a broadcast read takes far longer than an ordinary L2 hit.)
-  uint4 graw[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-  if (PARTS <= 2 && p.gain) {
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int i0 = (tid + 256 * j) * 8;
-      if (i0 < K) graw[j] = __ldg(reinterpret_cast<const uint4*>(p.gain + i0));
-    }
-  }
+  uint4 graw = make_uint4(0, 0, 0, 0);
+  if (p.gain && tid * 8 < K) graw = __ldg(reinterpret_cast<const uint4*>(p.gain + tid * 8));
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the activation comes from the preceding kernel
-  const int part = warp % PARTS, rsub = warp / PARTS;
+  const int part = wg % PARTS, rsub = wg / PARTS;
   const int pblk = (nblk + PARTS - 1) / PARTS;
   const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
   uint32_t xr[kJ][24];
   float xm[kJ], xc[kJ];
-  if (PARTS <= 2) {
-    // K <= 4096.  Thread t owns the runs of 8 consecutive elements r = t + 256 j; four adjacent lanes hold one block.
-    // Optional RMSNorm (h = rn16(x * g / sqrt(mean(x^2) + eps))) and the block quantization both work on those
-    // registers; the quantized blocks go to shared memory once per CTA (28 words per block; the 112-byte pitch keeps
-    // the 128-bit reads conflict-free) and every lane then fetches the blocks of its k-part.
-    constexpr int kRuns = 2;
+  {
+    // Thread t owns the runs of 8 consecutive elements r = t + 512 j (one run when K <= 4096, up to four for K = 16384);
+    // four adjacent lanes hold one 32-element block.  The optional RMSNorm (h = rn16(x * g / sqrt(mean(x^2) + eps)),
+    // K <= 4096) and the block quantization work on those registers; the quantized blocks go to shared memory once
+    // per CTA (28 words per block; the 112-byte pitch keeps the 128-bit reads conflict-free) and every lane then
+    // fetches the blocks of its k-part.
     uint32_t* xq_s = reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes);
-    float xv[kRuns][8];
-    float ss = 0.f;
+    auto load_run = [&](const __half* src16, const float* src32, int i0, float (&xv)[8]) {
+      if (src32) {
+        const float4 a = *reinterpret_cast<const float4*>(src32 + i0);
+        const float4 b = *reinterpret_cast<const float4*>(src32 + i0 + 4);
+        xv[0] = a.x; xv[1] = a.y; xv[2] = a.z; xv[3] = a.w;
+        xv[4] = b.x; xv[5] = b.y; xv[6] = b.z; xv[7] = b.w;
+      } else {
+        const uint4 a = *reinterpret_cast<const uint4*>(src16 + i0);
+        const uint32_t w4[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
-    for (int j = 0; j < kRuns; ++j) {
-      const int i0 = (tid + 256 * j) * 8;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) xv[j][q] = 0.f;
-      if (i0 < K) {
-        if (p.gain && p.norm_in32) {
-          const float4 a = *reinterpret_cast<const float4*>(p.norm_in32 + i0);
-          const float4 b = *reinterpret_cast<const float4*>(p.norm_in32 + i0 + 4);
-          xv[j][0] = a.x; xv[j][1] = a.y; xv[j][2] = a.z; xv[j][3] = a.w;
-          xv[j][4] = b.x; xv[j][5] = b.y; xv[j][6] = b.z; xv[j][7] = b.w;
-        } else {
-          const uint4 a = *reinterpret_cast<const uint4*>((p.gain ? p.norm_in16 : p.x16) + i0);
-          const uint32_t w4[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            __half2 h2;
-            *reinterpret_cast<uint32_t*>(&h2) = w4[q];
-            const float2 f = __half22float2(h2);
-            xv[j][2 * q] = f.x;
-            xv[j][2 * q + 1] = f.y;
-          }
+        for (int q = 0; q < 4; ++q) {
+          __half2 h2;
+          *reinterpret_cast<uint32_t*>(&h2) = w4[q];
+          const float2 f = __half22float2(h2);
+          xv[2 * q] = f.x;
+          xv[2 * q + 1] = f.y;
         }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) ss = fmaf(xv[j][q], xv[j][q], ss);
       }
-    }
+    };
     if (p.gain) {
-      float gv[kRuns][8];
+      // norm prologue: K <= 4096, one run per thread
+      const int i0 = tid * 8;
+      const bool has = i0 < K;
+      float xv[8];
 #pragma unroll
-      for (int j = 0; j < kRuns; ++j) {
-        const int i0 = (tid + 256 * j) * 8;
-        if (i0 < K) {
-          const uint4 g4 = graw[j];
-          const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
+      for (int q = 0; q < 8; ++q) xv[q] = 0.f;
+      float ss = 0.f;
+      if (has) {
+        load_run(p.norm_in16, p.norm_in32, i0, xv);
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            __half2 h2;
-            *reinterpret_cast<uint32_t*>(&h2) = gw[q];
-            const float2 f = __half22float2(h2);
-            gv[j][2 * q] = f.x;
-            gv[j][2 * q + 1] = f.y;
-          }
-        }
+        for (int q = 0; q < 8; ++q) ss = fmaf(xv[q], xv[q], ss);
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
       if (lane == 0) red_s[warp] = ss;
-      consumer_sync();
+      consumer_sync_all();
       float tot = 0.f;
 #pragma unroll
       for (int w = 0; w < kConsumerWarps; ++w) tot += red_s[w];
       const float inv = 1.0f / sqrtf(tot / (float)K + p.eps);
+      if (has) {
+        const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
+        uint32_t o4[4];
 #pragma unroll
-      for (int j = 0; j < kRuns; ++j) {
-        const int i0 = (tid + 256 * j) * 8;
-        if (i0 < K) {
-          uint32_t o4[4];
+        for (int q = 0; q < 4; ++q) {
+          __half2 g2;
+          *reinterpret_cast<uint32_t*>(&g2) = gw[q];
+          const float2 gf = __half22float2(g2);
+          const __half2 h2 = __floats2half2_rn(xv[2 * q] * gf.x * inv, xv[2 * q + 1] * gf.y * inv);
+          o4[q] = *reinterpret_cast<const uint32_t*>(&h2);
+          const float2 f = __half22float2(h2);  // the operand is the fp16-rounded value
+          xv[2 * q] = f.x;
+          xv[2 * q + 1] = f.y;
+        }
+        if (p.h_out && bx == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+        quantize_run4(xv, tid & 3, xq_s + (size_t)(tid >> 2) * 28);
+      }
+    } else {
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const __half2 h2 = __floats2half2_rn(xv[j][2 * q] * gv[j][2 * q] * inv, xv[j][2 * q + 1] * gv[j][2 * q + 1] * inv);
-            o4[q] = *reinterpret_cast<const uint32_t*>(&h2);
-            const float2 f = __half22float2(h2);  // the operand is the fp16-rounded value
-            xv[j][2 * q] = f.x;
-            xv[j][2 * q + 1] = f.y;
-          }
-          if (p.h_out && bx == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+      for (int j = 0; j < 4; ++j) {
+        const int r = tid + 512 * j;  // run index; block r / 4, word r % 4.  All four lanes of a group are in range together.
+        if (r * 8 < K) {
+          float xv[8];
+          load_run(p.x16, nullptr, r * 8, xv);
+          quantize_run4(xv, r & 3, xq_s + (size_t)(r >> 2) * 28);
         }
       }
     }
-#pragma unroll
-    for (int j = 0; j < kRuns; ++j) {
-      const int r = tid + 256 * j;  // run index; block r / 4, word r % 4.  All four lanes of a group are in range together.
-      if (r * 8 < K) quantize_run4(xv[j], r & 3, xq_s + (size_t)(r >> 2) * 28);
-    }
-    consumer_sync();
+    consumer_sync_all();
 #pragma unroll
     for (int j = 0; j < kJ; ++j) {
       const int b = b0 + lane + 32 * j;
@@ -394,36 +358,17 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
         xc[j] = 0.f;
       }
     }
-  } else {
-#pragma unroll
-    for (int j = 0; j < kJ; ++j) {
-      const int b = b0 + lane + 32 * j;
-      if (b < b1) {
-        uint32_t xh[16];
-        const uint4* src = reinterpret_cast<const uint4*>(p.x16 + (size_t)b * 32);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint4 v = src[q];
-          xh[4 * q] = v.x;
-          xh[4 * q + 1] = v.y;
-          xh[4 * q + 2] = v.z;
-          xh[4 * q + 3] = v.w;
-        }
-        quantize_block(xh, xr[j], xm[j], xc[j]);
-      } else {
-#pragma unroll
-        for (int q = 0; q < 24; ++q) xr[j][q] = 0;
-        xm[j] = 0.f;
-        xc[j] = 0.f;
-      }
-    }
   }
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // this group's tiles: it = grp, grp + 2, ...; li counts them
+  const int n_li = n_it > grp ? (n_it - grp + kGroups - 1) / kGroups : 0;
+  float* my_part = part_s[grp];
   bool failed = false;
-  for (int it0 = 0; it0 < n_it; it0 += kMaxIt) {
-    const int it1 = min(n_it, it0 + kMaxIt);
-    for (int it = it0; it < it1; ++it) {
+  for (int li0 = 0; li0 < n_li; li0 += kMaxIt) {
+    const int li1 = min(n_li, li0 + kMaxIt);
+    for (int li = li0; li < li1; ++li) {
+      const int it = grp + kGroups * li;
       const int s = it % kStages;
       if (!mbar_wait(&full[s], (it / kStages) & 1)) {
         failed = true;
@@ -468,24 +413,24 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
         for (int r = 0; r < kRPW; ++r) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
       if (lane == 0) {
 #pragma unroll
-        for (int r = 0; r < kRPW; ++r) part_s[((it - it0) * ROWS + r * (ROWS / kRPW) + rsub) * PARTS + part] = acc[r];
+        for (int r = 0; r < kRPW; ++r) my_part[((li - li0) * ROWS + r * (ROWS / kRPW) + rsub) * PARTS + part] = acc[r];
       }
     }
     if (failed) fail_s = 1;
-    consumer_sync();
-    if (fail_s) {  // uniform over the consumers: nobody waits at a barrier for a warp that gave up
-      if (tid == 0) atomicExch(p.status, 1);
+    group_sync(grp);
+    if (fail_s) {  // a warp of either group gave up: nobody waits at a barrier for it
+      if (tg == 0) atomicExch(p.status, 1);
       return;
     }
     // flush: sum the k-parts (ascending) and run the epilogue
-    const int n_out = (it1 - it0) * OUT_ROWS;
-    for (int i = tid; i < n_out; i += 256) {
+    const int n_out = (li1 - li0) * OUT_ROWS;
+    for (int i = tg; i < n_out; i += kGroupWarps * 32) {
       const int itl = i / OUT_ROWS, j = i % OUT_ROWS;
-      const int tile = first + (it0 + itl) * gx;
+      const int tile = first + (grp + kGroups * (li0 + itl)) * gx;
       float v[2];
 #pragma unroll
       for (int h = 0; h < (SW ? 2 : 1); ++h) {
-        const float* ps = part_s + ((size_t)itl * ROWS + j + h * OUT_ROWS) * PARTS;
+        const float* ps = my_part + ((size_t)itl * ROWS + j + h * OUT_ROWS) * PARTS;
         float t = 0.f;
 #pragma unroll
         for (int q = 0; q < PARTS; ++q) t += ps[q];
@@ -509,12 +454,12 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
         }
       }
     }
-    consumer_sync();
+    group_sync(grp);
   }
 }
 
 template <int PARTS, bool SW>
-__global__ void __launch_bounds__(kThreads, 2) gemv_stream_kernel(const StreamParams p) {
+__global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamParams p) {
   gemv_stream_body<PARTS, SW>(p, (int)blockIdx.x, (int)gridDim.x, false);
 }
 
@@ -532,7 +477,7 @@ struct MoeSel {
   int ldx, ldy;
 };
 template <int PARTS, bool SW>
-__global__ void __launch_bounds__(kThreads, 2) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
+__global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
   StreamParams p = p0;
   const int job = blockIdx.y;
   int xrow, orow;
@@ -562,7 +507,7 @@ int parts_for(int K) { return K <= 2048 ? 1 : K <= 4096 ? 2 : K <= 8192 ? 4 : 8;
 bool gemv_stream_eligible(const GemvParams& p) {
   if (p.M != 1 || p.K % 256 != 0 || p.K > 16384) return false;
   const int parts = parts_for(p.K);
-  const int rows = kConsumerWarps / parts * kRPW;
+  const int rows = kGroupWarps / parts * kRPW;
   if (p.mode == GEMV_SWIGLU_F16) {
     if (p.n_seg != 2 || p.seg[0].n_rows != p.seg[1].n_rows || p.seg[0].n_rows % (rows / 2)) return false;
   } else {
@@ -575,7 +520,7 @@ bool gemv_stream_eligible(const GemvParams& p) {
 
 cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch) {
   const int parts = parts_for(g.K);
-  const int rows = kConsumerWarps / parts * kRPW;
+  const int rows = kGroupWarps / parts * kRPW;
   const bool sw = g.mode == GEMV_SWIGLU_F16;
   StreamParams p{};
   p.n_seg = g.n_seg;
@@ -605,8 +550,8 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   p.res16 = g.res16;
   p.status = status;
   const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (parts <= 2 ? (size_t)(g.K / 32) * 112 : 0);
-  const int grid = std::max(1, std::min(tiles, 2 * sm_count));
+  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * 112;
+  const int grid = std::max(1, std::min(tiles, sm_count));
   void (*kern)(const StreamParams) = nullptr;
   switch (parts) {
     case 1: kern = sw ? gemv_stream_kernel<1, true> : gemv_stream_kernel<1, false>; break;
@@ -617,10 +562,10 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   static uint64_t attr_done[8] = {};
   const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
     if (e != cudaSuccess) return e;
   }
-  if (smem > 100 * 1024) return cudaErrorInvalidValue;
+  if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreads);
@@ -637,7 +582,7 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
 
 bool moe_gemv_stream_eligible(const MoeGemvParams& p) {
   if (p.K % 256 != 0 || p.K > 16384) return false;
-  const int rows = kConsumerWarps / parts_for(p.K) * kRPW;
+  const int rows = kGroupWarps / parts_for(p.K) * kRPW;
   if (p.mode == GEMV_SWIGLU_F16) return p.n_rows % (rows / 2) == 0;
   return (p.mode == GEMV_OUT_F32 || p.mode == GEMV_OUT_F16) && p.n_rows % rows == 0;
 }
@@ -645,7 +590,7 @@ bool moe_gemv_stream_eligible(const MoeGemvParams& p) {
 cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, int* status, int sm_count, int pdl, cudaStream_t st,
                                    uint64_t* n_launch) {
   const int parts = parts_for(g.K);
-  const int rows = kConsumerWarps / parts * kRPW;
+  const int rows = kGroupWarps / parts * kRPW;
   const bool sw = g.mode == GEMV_SWIGLU_F16;
   const int n_jobs = jobs ? jobs->n : g.P;
   if (n_jobs <= 0) return cudaSuccess;
@@ -673,9 +618,9 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   MoeJobs none;
   none.n = 0;
   const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (parts <= 2 ? (size_t)(g.K / 32) * 112 : 0);
-  if (smem > 100 * 1024) return cudaErrorInvalidValue;
-  const int per_job = std::max(1, std::min(p.n_tiles, (2 * sm_count + n_jobs - 1) / n_jobs));
+  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * 112;
+  if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
+  const int per_job = std::max(1, std::min(p.n_tiles, sm_count / n_jobs));  // one wave: a CTA fills its SM
   void (*kern)(const StreamParams, const MoeSel, const MoeJobs) = nullptr;
   switch (parts) {
     case 1: kern = sw ? gemv_stream_moe_kernel<1, true> : gemv_stream_moe_kernel<1, false>; break;
@@ -686,7 +631,7 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   static uint64_t attr_done[8] = {};
   const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg{};
