@@ -7,12 +7,15 @@
 // quantization blocks (32 k each) of a k-part of the row and keeps the activation for them in registers for the whole
 // kernel, so a weight byte is read once from shared memory and an activation never again.
 //
-// Arithmetic: the activation block is re-expressed once per CTA as 23-bit block fixed point, x_k = xi_k * 2^-sh with
-// sh chosen from the block's largest exponent (exact for every element within 2^-11 of the block maximum, rounded at
-// 2^-23 of it otherwise, i.e. at the level of one fp32 rounding).  The three byte planes of xi are multiplied with the
-// masked 4-bit codes by dp4a: block dot products are exact integers; one fp32 multiply-add per block applies the
-// scale, and blocks are accumulated in fp32.  sum_k (u_k - 8) x_k = sum_k u_k x_k - 8 sum_k x_k with the second term
-// precomputed per block.  Lane partials are reduced by warp shuffles, k-parts through shared memory, both in fixed order.
+// Arithmetic: the activation block is re-expressed once per CTA as 16-bit block fixed point, x_k ~ xi_k * 2^-sh with
+// sh chosen from the block's largest exponent (exact for every element within 2^-4 of the block maximum, rounded at
+// 2^-16 of it otherwise: 32 times finer than fp16 resolves the maximum itself).  Pairs of xi meet pairs of masked 4-bit
+// codes in dp2a: block dot products are exact integers; one fp32 multiply-add per block applies the scale, and blocks
+// are accumulated in fp32.  sum_k (u_k - 8) x_k = sum_k u_k x_k - 8 sum_k x_k with the second term precomputed per
+// block.  All integer instructions issue at half rate on this part and the dot-product pipe is the one that fills, so
+// the instruction count per block (16 dp2a, 8 masks, 2 to combine) is what the format allows: the high nibbles are
+// used in place as 16 * code and their sum shifted back once per block.  Lane partials are reduced by warp shuffles,
+// k-parts through shared memory, both in fixed order.
 //
 // Optional prologue: RMSNorm of the input row (fp16 or fp32) with an fp16 gain, rounded to fp16 (the operand edge of
 // the numerics contract), computed once per CTA by all 512 consumer threads while the first weight tiles are in flight.
@@ -30,6 +33,7 @@ constexpr int kConsumerWarps = kGroups * kGroupWarps;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kRPW = 2;      // rows per consumer warp per tile
 constexpr int kJ = 2;        // quantization blocks per lane per row
+constexpr int kEarlyStages = 1;  // stages requested before the consumers have issued their activation loads
 constexpr int kMaxDynSmem = 216 * 1024;  // ring + quantized activation row; 6 KB of static shared memory on top
 constexpr int kMaxIt = 48;   // tiles of a group whose partial sums are buffered before a flush
 
@@ -75,14 +79,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
                : "memory");
 }
-__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {
+// d = c + a.lo16 * b.byte0 + a.hi16 * b.byte1 (dp2a_lo) or with bytes 2, 3 (dp2a_hi): signed halves, unsigned bytes
+__device__ __forceinline__ int dp2a_lo(uint32_t a, uint32_t b, int c) {
   int d;
-  asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  asm("dp2a.lo.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
-__device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {
+__device__ __forceinline__ int dp2a_hi(uint32_t a, uint32_t b, int c) {
   int d;
-  asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  asm("dp2a.hi.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
 // named barriers: 1 and 2 = the two consumer groups (256 threads each), 3 = all consumers (512); 0 is __syncthreads
@@ -98,15 +103,20 @@ __device__ __forceinline__ int f2i_magic(float x, float up) {
   return (int)__float_as_uint(fmaf(x, up, 12582912.0f)) - 0x4B400000;
 }
 
-// Layout of a quantized activation block (28 words): three byte planes laid out to meet the masked code words.
-// Code word w of a block holds codes k = 8w..8w+7 at nibble positions (0,2,4,6,1,3,5,7); (word & 0x0F0F0F0F) therefore
-// carries k = 8w + {0,4,1,5} in its bytes and ((word >> 4) & 0x0F0F0F0F) carries k = 8w + {2,6,3,7}.
-// planes[p*8 + 2w + h] holds byte p of xi for those four k (h = 0 / 1); words 24 and 25 hold mul = 2^-sh and
-// corr = -8 * sum(xi) * mul, with sh = 36 - E for the block's largest biased fp16 exponent E (|xi| < 2^22).
+// Layout of a quantized activation block (kXqWords words): the block's 32 activations as 16-bit block fixed point,
+// xi_k = rn(x_k * 2^sh) with sh = 29 - E for the block's largest biased fp16 exponent E, so |xi| <= 32752: exact for
+// every element within 2^-4 of the block maximum, rounded at 2^-16 of the maximum otherwise (32 times finer than
+// fp16's own resolution at the maximum).  Code word w of a block holds codes k = 8w..8w+7 at nibble positions
+// (0,2,4,6,1,3,5,7); (word & 0x0F0F0F0F) therefore carries k = 8w + {0,4,1,5} in its bytes and (word & 0xF0F0F0F0)
+// carries 16 times the codes of k = 8w + {2,6,3,7}.  Words 4w..4w+3 of the block hold the pairs (xi_{8w+0}, xi_{8w+4}),
+// (xi_{8w+1}, xi_{8w+5}), (xi_{8w+2}, xi_{8w+6}), (xi_{8w+3}, xi_{8w+7}) as two signed 16-bit halves (first in the
+// low half): the operands of dp2a.lo / dp2a.hi against the two masked words.  Words 16 and 17 hold mul = 2^-sh and
+// corr = -8 * sum(xi) * mul.
 //
 // The quantization is done by four adjacent lanes, each holding one run of 8 consecutive elements (one code word's
 // worth) of a 32-element block: exponent maximum and integer sum are shared by two butterfly shuffles.  Lane w of the
-// group writes plane words 2w, 2w+1 of every plane into blk[28] (24 plane words, then mul, corr).
+// group writes words 4w..4w+3.
+constexpr int kXqWords = 20;  // 18 used; the 80-byte pitch keeps the 128-bit reads of consecutive blocks conflict-free
 __device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32_t* blk) {
   uint32_t m = 0;
 #pragma unroll
@@ -115,7 +125,7 @@ __device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32
   m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
   // fp16 exponent field E = fp32 field - 112 (normals); subnormal fp16 values have fp32 fields <= 112 -> E = 1
   const int E = max((int)m - 112, 1);
-  const int sh = 36 - E;  // |xi| < 2^22
+  const int sh = 29 - E;  // the largest fp16 magnitude with field E, (2 - 2^-10) 2^(E-15), maps to 32752
   const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
   const float mul = __uint_as_float((uint32_t)(127 - sh) << 23);
   int xi[8];
@@ -127,16 +137,13 @@ __device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32
   }
   sx += __shfl_xor_sync(0xffffffffu, sx, 1);
   sx += __shfl_xor_sync(0xffffffffu, sx, 2);
-#pragma unroll
-  for (int p = 0; p < 3; ++p) {
-    const uint32_t sel_lo = 0x0040u + 0x0011u * p;
-    const uint32_t a01 = __byte_perm((uint32_t)xi[0], (uint32_t)xi[4], sel_lo);
-    const uint32_t a23 = __byte_perm((uint32_t)xi[1], (uint32_t)xi[5], sel_lo);
-    const uint32_t b01 = __byte_perm((uint32_t)xi[2], (uint32_t)xi[6], sel_lo);
-    const uint32_t b23 = __byte_perm((uint32_t)xi[3], (uint32_t)xi[7], sel_lo);
-    *reinterpret_cast<uint2*>(blk + p * 8 + 2 * w) = make_uint2(__byte_perm(a01, a23, 0x5410u), __byte_perm(b01, b23, 0x5410u));
-  }
-  if (w == 0) *reinterpret_cast<float2*>(blk + 24) = make_float2(mul, -8.0f * (float)sx * mul);
+  uint4 o;
+  o.x = __byte_perm((uint32_t)xi[0], (uint32_t)xi[4], 0x5410u);
+  o.y = __byte_perm((uint32_t)xi[1], (uint32_t)xi[5], 0x5410u);
+  o.z = __byte_perm((uint32_t)xi[2], (uint32_t)xi[6], 0x5410u);
+  o.w = __byte_perm((uint32_t)xi[3], (uint32_t)xi[7], 0x5410u);
+  *reinterpret_cast<uint4*>(blk + 4 * w) = o;
+  if (w == 0) *reinterpret_cast<float2*>(blk + 16) = make_float2(mul, -8.0f * (float)sx * mul);
 }
 
 struct StreamSeg {
@@ -177,7 +184,7 @@ struct StreamParams {
 template <int PARTS, bool SW>
 __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool wait_first) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ uint64_t full[kStages], empty[kStages];
+  __shared__ uint64_t full[kStages], empty[kStages], xbar;
   __shared__ float part_s[kGroups][kMaxIt * kGroupWarps * kRPW];
   __shared__ float red_s[kConsumerWarps];
   __shared__ int fail_s;
@@ -194,6 +201,7 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], kGroupWarps);
     }
+    mbar_init(&xbar, kConsumerWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -210,6 +218,12 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
         const int s = it % kStages;
         if (it >= kStages && !mbar_wait(&empty[s], ((it / kStages) - 1) & 1)) {
           atomicExch(p.status, 2);
+          break;
+        }
+        // Weight copies queued ahead of the consumers' activation loads delay them (the row is a cache hit that then
+        // waits behind megabytes of misses): one stage goes out at once, the rest after those loads have been issued.
+        if (it == kEarlyStages && !mbar_wait(&xbar, 0)) {
+          atomicExch(p.status, 3);
           break;
         }
         if (it == kStages) {
@@ -257,7 +271,7 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
   const int part = wg % PARTS, rsub = wg / PARTS;
   const int pblk = (nblk + PARTS - 1) / PARTS;
   const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
-  uint32_t xr[kJ][24];
+  uint32_t xr[kJ][16];
   float xm[kJ], xc[kJ];
   {
     // Thread t owns the runs of 8 consecutive elements r = t + 512 j (one run when K <= 4096, up to four for K = 16384);
@@ -293,8 +307,10 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
 #pragma unroll
       for (int q = 0; q < 8; ++q) xv[q] = 0.f;
       float ss = 0.f;
+      if (has) load_run(p.norm_in16, p.norm_in32, i0, xv);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&xbar);
       if (has) {
-        load_run(p.norm_in16, p.norm_in32, i0, xv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) ss = fmaf(xv[q], xv[q], ss);
       }
@@ -321,16 +337,32 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
           xv[2 * q + 1] = f.y;
         }
         if (p.h_out && bx == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-        quantize_run4(xv, tid & 3, xq_s + (size_t)(tid >> 2) * 28);
+        quantize_run4(xv, tid & 3, xq_s + (size_t)(tid >> 2) * kXqWords);
       }
     } else {
+      uint4 raw[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int r = tid + 512 * j;  // run index; block r / 4, word r % 4.  All four lanes of a group are in range together.
+        if (r * 8 < K) raw[j] = *reinterpret_cast<const uint4*>(p.x16 + r * 8);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&xbar);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int r = tid + 512 * j;
         if (r * 8 < K) {
           float xv[8];
-          load_run(p.x16, nullptr, r * 8, xv);
-          quantize_run4(xv, r & 3, xq_s + (size_t)(r >> 2) * 28);
+          const uint32_t w4[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            __half2 h2;
+            *reinterpret_cast<uint32_t*>(&h2) = w4[q];
+            const float2 f = __half22float2(h2);
+            xv[2 * q] = f.x;
+            xv[2 * q + 1] = f.y;
+          }
+          quantize_run4(xv, r & 3, xq_s + (size_t)(r >> 2) * kXqWords);
         }
       }
     }
@@ -339,21 +371,21 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
     for (int j = 0; j < kJ; ++j) {
       const int b = b0 + lane + 32 * j;
       if (b < b1) {
-        const uint4* src = reinterpret_cast<const uint4*>(xq_s + (size_t)b * 28);
+        const uint4* src = reinterpret_cast<const uint4*>(xq_s + (size_t)b * kXqWords);
 #pragma unroll
-        for (int q = 0; q < 6; ++q) {
+        for (int q = 0; q < 4; ++q) {
           const uint4 v = src[q];
           xr[j][4 * q] = v.x;
           xr[j][4 * q + 1] = v.y;
           xr[j][4 * q + 2] = v.z;
           xr[j][4 * q + 3] = v.w;
         }
-        const float2 mc = *reinterpret_cast<const float2*>(xq_s + (size_t)b * 28 + 24);
+        const float2 mc = *reinterpret_cast<const float2*>(xq_s + (size_t)b * kXqWords + 16);
         xm[j] = mc.x;
         xc[j] = mc.y;
       } else {
 #pragma unroll
-        for (int q = 0; q < 24; ++q) xr[j][q] = 0;
+        for (int q = 0; q < 16; ++q) xr[j][q] = 0;
         xm[j] = 0.f;
         xc[j] = 0.f;
       }
@@ -361,61 +393,76 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
   }
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // this group's tiles: it = grp, grp + 2, ...; li counts them
+  // this group's tiles: it = grp, grp + 2, ...; li counts them.  The cross-lane reduction of a tile's row sums is
+  // deferred into the next tile's iteration, where its shuffle latencies hide behind that tile's integer work.
   const int n_li = n_it > grp ? (n_it - grp + kGroups - 1) / kGroups : 0;
   float* my_part = part_s[grp];
   bool failed = false;
+  auto reduce_store = [&](float (&a)[kRPW], int slot) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+      for (int r = 0; r < kRPW; ++r) a[r] += __shfl_xor_sync(0xffffffffu, a[r], o);
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < kRPW; ++r) my_part[(slot * ROWS + r * (ROWS / kRPW) + rsub) * PARTS + part] = a[r];
+    }
+  };
   for (int li0 = 0; li0 < n_li; li0 += kMaxIt) {
     const int li1 = min(n_li, li0 + kMaxIt);
+    float prev[kRPW];
+    bool have_prev = false;
     for (int li = li0; li < li1; ++li) {
       const int it = grp + kGroups * li;
       const int s = it % kStages;
-      if (!mbar_wait(&full[s], (it / kStages) & 1)) {
+      if (!__all_sync(0xffffffffu, mbar_wait(&full[s], (it / kStages) & 1))) {
         failed = true;
         break;
       }
       const uint8_t* st = stages + (size_t)s * stage_bytes;
-      float acc[kRPW];
+      uint4 cw[kRPW][kJ];
+      float sc[kRPW][kJ];
 #pragma unroll
       for (int r = 0; r < kRPW; ++r) {
         const int row = r * (ROWS / kRPW) + rsub;  // stage row of this warp's r-th row
         const uint4* codes = reinterpret_cast<const uint4*>(st + (size_t)row * row_codes);
-        const __half* sc = reinterpret_cast<const __half*>(st + (size_t)ROWS * row_codes + (size_t)row * row_scales);
-        acc[r] = 0.f;
+        const __half* scp = reinterpret_cast<const __half*>(st + (size_t)ROWS * row_codes + (size_t)row * row_scales);
 #pragma unroll
         for (int j = 0; j < kJ; ++j) {
           const int b = b0 + lane + 32 * j;
-          if (b < b1) {
-            const uint4 q = codes[b];
-            const float scale = __half2float(sc[b]);
-            const uint32_t ws[4] = {q.x, q.y, q.z, q.w};
-            int d0 = 0, d1 = 0, d2 = 0;
+          const bool in = b < b1;
+          cw[r][j] = in ? codes[b] : make_uint4(0, 0, 0, 0);
+          sc[r][j] = in ? __half2float(scp[b]) : 0.f;
+        }
+      }
+      if (have_prev) reduce_store(prev, li - 1 - li0);
+      float acc[kRPW];
 #pragma unroll
-            for (int w = 0; w < 4; ++w) {
-              const uint32_t lo = ws[w] & 0x0F0F0F0Fu, hi = (ws[w] >> 4) & 0x0F0F0F0Fu;
-              d0 = dp4a_uu(lo, xr[j][2 * w], d0);
-              d0 = dp4a_uu(hi, xr[j][2 * w + 1], d0);
-              d1 = dp4a_uu(lo, xr[j][8 + 2 * w], d1);
-              d1 = dp4a_uu(hi, xr[j][8 + 2 * w + 1], d1);
-              d2 = dp4a_us(lo, xr[j][16 + 2 * w], d2);
-              d2 = dp4a_us(hi, xr[j][16 + 2 * w + 1], d2);
-            }
-            const float dot = fmaf((float)d2, 65536.f, (float)(d1 * 256 + d0));
-            acc[r] = fmaf(scale, fmaf(dot, xm[j], xc[j]), acc[r]);
+      for (int r = 0; r < kRPW; ++r) {
+        acc[r] = 0.f;
+#pragma unroll
+        for (int j = 0; j < kJ; ++j) {
+          const uint32_t ws[4] = {cw[r][j].x, cw[r][j].y, cw[r][j].z, cw[r][j].w};
+          int dl = 0, dh = 0;
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const uint32_t lo = ws[w] & 0x0F0F0F0Fu, hi = ws[w] & 0xF0F0F0F0u;  // hi carries 16 * code
+            dl = dp2a_lo(xr[j][4 * w], lo, dl);
+            dl = dp2a_hi(xr[j][4 * w + 1], lo, dl);
+            dh = dp2a_lo(xr[j][4 * w + 2], hi, dh);
+            dh = dp2a_hi(xr[j][4 * w + 3], hi, dh);
           }
+          const float dot = (float)(dl + (dh >> 4));  // dh is a multiple of 16; |dot| < 2^24: exact
+          acc[r] = fmaf(sc[r][j], fmaf(dot, xm[j], xc[j]), acc[r]);
         }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);  // this warp is done reading stage s
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-        for (int r = 0; r < kRPW; ++r) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
-      if (lane == 0) {
-#pragma unroll
-        for (int r = 0; r < kRPW; ++r) my_part[((li - li0) * ROWS + r * (ROWS / kRPW) + rsub) * PARTS + part] = acc[r];
-      }
+      for (int r = 0; r < kRPW; ++r) prev[r] = acc[r];
+      have_prev = true;
     }
+    if (have_prev && !failed) reduce_store(prev, li1 - 1 - li0);
     if (failed) fail_s = 1;
     group_sync(grp);
     if (fail_s) {  // a warp of either group gave up: nobody waits at a barrier for it
@@ -550,7 +597,7 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   p.res16 = g.res16;
   p.status = status;
   const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * 112;
+  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * (kXqWords * 4);
   const int grid = std::max(1, std::min(tiles, sm_count));
   void (*kern)(const StreamParams) = nullptr;
   switch (parts) {
@@ -618,7 +665,7 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   MoeJobs none;
   none.n = 0;
   const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * 112;
+  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * (kXqWords * 4);
   if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
   const int per_job = std::max(1, std::min(p.n_tiles, sm_count / n_jobs));  // one wave: a CTA fills its SM
   void (*kern)(const StreamParams, const MoeSel, const MoeJobs) = nullptr;

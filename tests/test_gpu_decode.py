@@ -182,9 +182,11 @@ def test_dense_layer_decode_matches_oracle(B, torch, shape_name, pos, cap):
     for got, ref in ((kg, kc), (vg, vc)):
         assert np.array_equal(np.delete(got, pos, axis=1), np.delete(ref, pos, axis=1))
         a, b = got[:, pos].astype(np.float64), ref[:, pos].astype(np.float64)
-        # one fp16 ulp where the value is not tiny; near zero the fp32 accumulation error (absolute) is what bounds it
+        # one fp16 ulp where the value is not tiny; near zero the absolute error of the projection bounds it: the
+        # activations enter the block dot products as 16-bit block fixed point (each rounded within 2^-17 of its block's
+        # maximum, about 1e-5 of the output's scale after the sum over k) and the blocks are accumulated in fp32
         ulp = np.spacing(np.abs(ref[:, pos]).astype(np.float16)).astype(np.float64)
-        assert np.all(np.abs(a - b) <= ulp + 2e-5 * np.abs(b).max())
+        assert np.all(np.abs(a - b) <= ulp + 1e-4 * np.abs(b).max())
     assert st.streamed_bytes == 0 and st.resident_bytes == H.dense_layer_bytes(shape)
 
 
