@@ -26,16 +26,46 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
 }
 
-// The work of one (split, kv head) job.  nthr = group * 32 * SUB threads take part, numbered tid = 0 .. nthr-1; they
-// synchronise with __syncthreads() when they are the whole CTA (CTA_SYNC) and with named barrier 1 otherwise.
+// The work of one (split, kv head) job, in two parts: staging the past cache rows (which do not depend on the new
+// token's projections) and everything after those projections exist.  nthr = group * 32 * SUB threads take part,
+// numbered tid = 0 .. nthr-1; they synchronise with __syncthreads() when they are the whole CTA (CTA_SYNC) and with
+// named barrier 4 otherwise.
+template <int D, int SUB>
+__device__ __forceinline__ void attn_decode_stage(const AttnDecodeParams& p, const int split, const int kvh, const int tid,
+                                                  const int nthr, uint8_t* dyn_s) {
+  constexpr int POS = 32 * SUB;
+  constexpr int CH = D * 2 / 16;
+  constexpr int KROW = D * 2 + 16;
+  constexpr int VROW = D * 2;
+  uint8_t* k_s = dyn_s;
+  uint8_t* v_s = dyn_s + (size_t)POS * KROW;
+  const int n_ctx = p.pos + 1;
+  const int tc0 = split * POS;
+  const int rows_here = min(POS, n_ctx - tc0);
+  const bool own = split == p.pos / POS;
+  const int r_new = p.pos - tc0;
+  for (int c = tid; c < rows_here * CH; c += nthr) {
+    const int row = c / CH, ch = c % CH;
+    if (!(own && row == r_new)) {
+      const size_t off = ((size_t)kvh * p.cap + tc0 + row) * D + ch * 8;
+      cp_async16(k_s + (size_t)row * KROW + ch * 16, p.kc + off);
+      cp_async16(v_s + (size_t)row * VROW + ch * 16, p.vc + off);
+    }
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  // value rows beyond the context are read by the PV loop with weight zero: they must hold finite numbers
+  for (int c = tid + rows_here * CH; c < POS * CH; c += nthr)
+    *reinterpret_cast<uint4*>(v_s + (size_t)(c / CH) * VROW + (c % CH) * 16) = make_uint4(0, 0, 0, 0);
+}
+
 template <int D, int SUB, bool CTA_SYNC>
-__device__ __forceinline__ void attn_decode_body(const AttnDecodeParams& p, const int split, const int kvh, const int n_splits,
-                                                 const int tid, const int nthr, uint8_t* dyn_s) {
+__device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, const int split, const int kvh, const int n_splits,
+                                                    const int tid, const int nthr, uint8_t* dyn_s) {
   auto job_sync = [&]() {
     if (CTA_SYNC)
       __syncthreads();
     else
-      asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+      asm volatile("bar.sync 4, %0;" ::"r"(nthr) : "memory");
   };
   constexpr int POS = 32 * SUB;        // positions per CTA
   constexpr int V = D / 32;            // output dims per lane
@@ -56,24 +86,8 @@ __device__ __forceinline__ void attn_decode_body(const AttnDecodeParams& p, cons
   const int half = D / 2, n_ctx = p.pos + 1;
   const int qd = p.n_q * D, kvd = p.n_kv * D;
   const int tc0 = split * POS;                     // first position of the CTA
-  const int rows_here = min(POS, n_ctx - tc0);     // >= 1
   const bool own = split == p.pos / POS;           // this CTA holds the new token's position
   const int r_new = p.pos - tc0;
-  // The cache rows of past tokens do not depend on the preceding kernel.
-  for (int c = tid; c < rows_here * CH; c += nthr) {
-    const int row = c / CH, ch = c % CH;
-    if (!(own && row == r_new)) {
-      const size_t off = ((size_t)kvh * p.cap + tc0 + row) * D + ch * 8;
-      cp_async16(k_s + (size_t)row * KROW + ch * 16, p.kc + off);
-      cp_async16(v_s + (size_t)row * VROW + ch * 16, p.vc + off);
-    }
-  }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-  // value rows beyond the context are read by the PV loop with weight zero: they must hold finite numbers
-  for (int c = tid + rows_here * CH; c < POS * CH; c += nthr)
-    *reinterpret_cast<uint4*>(v_s + (size_t)(c / CH) * VROW + (c % CH) * 16) = make_uint4(0, 0, 0, 0);
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v of the new token come from the preceding kernel
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // rotary embedding of the group's query heads into shared memory
   for (int idx = tid; idx < G * half; idx += nthr) {
     const int g2 = idx / half, i = idx % half;
@@ -240,6 +254,16 @@ __device__ __forceinline__ void attn_decode_body(const AttnDecodeParams& p, cons
   const float inv = 1.0f / l;
 #pragma unroll
   for (int q = 0; q < EPT; ++q) p.a16[(size_t)hq2 * D + j + 64 * q] = __float2half_rn(o[q] * inv);
+}
+
+// Stand-alone form: the cache rows of past tokens are requested before the grid dependency resolves.
+template <int D, int SUB, bool CTA_SYNC>
+__device__ __forceinline__ void attn_decode_body(const AttnDecodeParams& p, const int split, const int kvh, const int n_splits,
+                                                 const int tid, const int nthr, uint8_t* dyn_s) {
+  attn_decode_stage<D, SUB>(p, split, kvh, tid, nthr, dyn_s);
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v of the new token come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  attn_decode_compute<D, SUB, CTA_SYNC>(p, split, kvh, n_splits, tid, nthr, dyn_s);
 }
 
 }  // namespace ats

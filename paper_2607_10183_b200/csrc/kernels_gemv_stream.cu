@@ -1,508 +1,26 @@
-// Streaming decode GEMV for one token (sm_100a): the memory-bound hot kernel of the decode path.
-//
-// Structure: one persistent CTA per SM: 16 consumer warps in two groups of 8 + 1 producer warp.  The producer streams
-// row tiles of the packed weights (codes and scales, contiguous byte ranges) into a ring of 8 shared-memory stages with
-// 1-D bulk-async copies (TMA) that complete on mbarriers; tiles alternate between the groups; consumers never touch
-// global memory for weights.  Every lane owns up to two
-// quantization blocks (32 k each) of a k-part of the row and keeps the activation for them in registers for the whole
-// kernel, so a weight byte is read once from shared memory and an activation never again.
-//
-// Arithmetic: the activation block is re-expressed once per CTA as 16-bit block fixed point, x_k ~ xi_k * 2^-sh with
-// sh chosen from the block's largest exponent (exact for every element within 2^-4 of the block maximum, rounded at
-// 2^-16 of it otherwise: 32 times finer than fp16 resolves the maximum itself).  Pairs of xi meet pairs of masked 4-bit
-// codes in dp2a: block dot products are exact integers; one fp32 multiply-add per block applies the scale, and blocks
-// are accumulated in fp32.  sum_k (u_k - 8) x_k = sum_k u_k x_k - 8 sum_k x_k with the second term precomputed per
-// block.  All integer instructions issue at half rate on this part and the dot-product pipe is the one that fills, so
-// the instruction count per block (16 dp2a, 8 masks, 2 to combine) is what the format allows: the high nibbles are
-// used in place as 16 * code and their sum shifted back once per block.  Lane partials are reduced by warp shuffles,
-// k-parts through shared memory, both in fixed order.
-//
-// Optional prologue: RMSNorm of the input row (fp16 or fp32) with an fp16 gain, rounded to fp16 (the operand edge of
-// the numerics contract), computed once per CTA by all 512 consumer threads while the first weight tiles are in flight.
-// All waits on mbarriers are bounded; on expiry the kernel raises a status word and returns.
-#include "ats_internal.h"
+// Stand-alone launches of the streaming decode GEMV (sm_100a): the dense single-token GEMV and its grouped-expert form.
+// The device code of a phase (producer, consumers, arithmetic) is in gemv_stream_body.cuh.
+#include "gemv_stream_body.cuh"
 
 namespace ats {
 
 namespace {
 
-constexpr int kStages = 8;
-constexpr int kGroups = 2;         // consumer groups per CTA, each with its own stream of tiles
-constexpr int kGroupWarps = 8;
-constexpr int kConsumerWarps = kGroups * kGroupWarps;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kRPW = 2;      // rows per consumer warp per tile
-constexpr int kJ = 2;        // quantization blocks per lane per row
-constexpr int kEarlyStages = 1;  // stages requested before the consumers have issued their activation loads
-constexpr int kMaxDynSmem = 216 * 1024;  // ring + quantized activation row; 6 KB of static shared memory on top
-constexpr int kMaxIt = 48;   // tiles of a group whose partial sums are buffered before a flush
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after about a second of SM clocks (the caller then raises the status word and returns).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    for (int i = 0; i < 64; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > 2000000000ll) return false;
-  }
-}
-// Weights are read once per call: the copies carry an evict-first L2 policy so that a step's 100+ MB of weights do not
-// push the activations, the KV cache and the kernels' own instructions out of the L2.
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
-               : "memory");
-}
-// d = c + a.lo16 * b.byte0 + a.hi16 * b.byte1 (dp2a_lo) or with bytes 2, 3 (dp2a_hi): signed halves, unsigned bytes
-__device__ __forceinline__ int dp2a_lo(uint32_t a, uint32_t b, int c) {
-  int d;
-  asm("dp2a.lo.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ int dp2a_hi(uint32_t a, uint32_t b, int c) {
-  int d;
-  asm("dp2a.hi.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-// named barriers: 1 and 2 = the two consumer groups (256 threads each), 3 = all consumers (512); 0 is __syncthreads
-__device__ __forceinline__ void group_sync(int grp) { asm volatile("bar.sync %0, 256;" ::"r"(grp + 1) : "memory"); }
-__device__ __forceinline__ void consumer_sync_all() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
-
-__device__ __forceinline__ float silu_mul_f(float g, float u) { return g / (1.0f + expf(-g)) * u; }
-
-// rn(x * up) as an integer for |x * up| < 2^22 (up a power of two, so the product is exact): adding 1.5 * 2^23 leaves the
-// rounded integer in the low mantissa bits.  One FMA and one integer add instead of a conversion instruction, which
-// issues at a quarter of their rate.
-__device__ __forceinline__ int f2i_magic(float x, float up) {
-  return (int)__float_as_uint(fmaf(x, up, 12582912.0f)) - 0x4B400000;
-}
-
-// Layout of a quantized activation block (kXqWords words): the block's 32 activations as 16-bit block fixed point,
-// xi_k = rn(x_k * 2^sh) with sh = 29 - E for the block's largest biased fp16 exponent E, so |xi| <= 32752: exact for
-// every element within 2^-4 of the block maximum, rounded at 2^-16 of the maximum otherwise (32 times finer than
-// fp16's own resolution at the maximum).  Code word w of a block holds codes k = 8w..8w+7 at nibble positions
-// (0,2,4,6,1,3,5,7); (word & 0x0F0F0F0F) therefore carries k = 8w + {0,4,1,5} in its bytes and (word & 0xF0F0F0F0)
-// carries 16 times the codes of k = 8w + {2,6,3,7}.  Words 4w..4w+3 of the block hold the pairs (xi_{8w+0}, xi_{8w+4}),
-// (xi_{8w+1}, xi_{8w+5}), (xi_{8w+2}, xi_{8w+6}), (xi_{8w+3}, xi_{8w+7}) as two signed 16-bit halves (first in the
-// low half): the operands of dp2a.lo / dp2a.hi against the two masked words.  Words 16 and 17 hold mul = 2^-sh and
-// corr = -8 * sum(xi) * mul.
-//
-// The quantization is done by four adjacent lanes, each holding one run of 8 consecutive elements (one code word's
-// worth) of a 32-element block: exponent maximum and integer sum are shared by two butterfly shuffles.  Lane w of the
-// group writes words 4w..4w+3.
-constexpr int kXqWords = 20;  // 18 used; the 80-byte pitch keeps the 128-bit reads of consecutive blocks conflict-free
-__device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32_t* blk) {
-  uint32_t m = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) m = max(m, (__float_as_uint(x[i]) >> 23) & 0xFFu);  // fp32 exponent field of an fp16-valued number
-  m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
-  m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
-  // fp16 exponent field E = fp32 field - 112 (normals); subnormal fp16 values have fp32 fields <= 112 -> E = 1
-  const int E = max((int)m - 112, 1);
-  const int sh = 29 - E;  // the largest fp16 magnitude with field E, (2 - 2^-10) 2^(E-15), maps to 32752
-  const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
-  const float mul = __uint_as_float((uint32_t)(127 - sh) << 23);
-  int xi[8];
-  int sx = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    xi[i] = f2i_magic(x[i], up);
-    sx += xi[i];
-  }
-  sx += __shfl_xor_sync(0xffffffffu, sx, 1);
-  sx += __shfl_xor_sync(0xffffffffu, sx, 2);
-  uint4 o;
-  o.x = __byte_perm((uint32_t)xi[0], (uint32_t)xi[4], 0x5410u);
-  o.y = __byte_perm((uint32_t)xi[1], (uint32_t)xi[5], 0x5410u);
-  o.z = __byte_perm((uint32_t)xi[2], (uint32_t)xi[6], 0x5410u);
-  o.w = __byte_perm((uint32_t)xi[3], (uint32_t)xi[7], 0x5410u);
-  *reinterpret_cast<uint4*>(blk + 4 * w) = o;
-  if (w == 0) *reinterpret_cast<float2*>(blk + 16) = make_float2(mul, -8.0f * (float)sx * mul);
-}
-
-struct StreamSeg {
-  const uint8_t* base;
-  int n_rows;
-  int tile0;  // first tile index of the segment
-};
-
-struct StreamParams {
-  StreamSeg seg[3];
-  int n_seg;
-  int n_tiles;
-  int K;
-  int mode;
-  // activation source: x16 (already the operand), or a row to RMS-normalise first
-  const __half* x16;
-  const __half* norm_in16;
-  const float* norm_in32;
-  const __half* gain;
-  float eps;
-  __half* h_out;  // optional copy of the normalised operand (written by CTA 0)
-  float* y32;
-  __half* y16;
-  const float* res32;
-  const __half* res16;
-  int* status;
-};
-
-// bx / gx: index of this CTA among the gx CTAs that share the work described by p (a whole launch for the dense GEMV, one
-// (token, slot) job of a grouped-expert launch).  wait_first: the weight addresses themselves come from the preceding
-// kernel (expert ids), so nothing may be fetched before the grid dependency resolves.
-//
-// One CTA per SM: 16 consumer warps in two groups of 8 plus the producer warp.  The CTA's tiles alternate between the
-// groups (tile it belongs to group it % 2, stage it % 8), each group with its own partial-sum buffer and barrier, so
-// the tile loop is that of two independent 8-warp CTAs; what they share is the activation prologue: all 512 consumer
-// threads load, normalise and quantise the row ONCE per SM, a quarter of the instructions two CTAs per SM spend on it
-// (for K = 14336, where every CTA used to quantise the whole row in registers, an eighth).
+// A whole kernel as one phase: the ring starts empty, the grid dependency is resolved by griddepcontrol.
 template <int PARTS, bool SW>
 __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool wait_first) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ uint64_t full[kStages], empty[kStages], xbar;
-  __shared__ float part_s[kGroups][kMaxIt * kGroupWarps * kRPW];
-  __shared__ float red_s[kConsumerWarps];
-  __shared__ int fail_s;
-  constexpr int ROWS = kGroupWarps / PARTS * kRPW;     // weight rows per tile
-  constexpr int OUT_ROWS = SW ? ROWS / 2 : ROWS;       // output rows per tile
-  const int K = p.K, nblk = K / 32;
-  const int row_codes = K / 2, row_scales = K / 16;
-  const int stage_bytes = ROWS * (row_codes + row_scales);
-  uint8_t* stages = smem;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) {
-    fail_s = 0;
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&full[s], 1);
-      mbar_init(&empty[s], kGroupWarps);
-    }
-    mbar_init(&xbar, kConsumerWarps);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-  const int first = bx;
-  const int n_it = first < p.n_tiles ? (p.n_tiles - first + gx - 1) / gx : 0;
-
-  if (warp == kConsumerWarps) {
-    // ------------------------------------------------------------------ producer: weights do not depend on the
-    // preceding kernel, so their copies start before the grid dependency is resolved.
-    if (lane == 0) {
-      const uint64_t pol = l2_evict_first_policy();
-      if (wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
-      for (int it = 0; it < n_it; ++it) {
-        const int s = it % kStages;
-        if (it >= kStages && !mbar_wait(&empty[s], ((it / kStages) - 1) & 1)) {
-          atomicExch(p.status, 2);
-          break;
-        }
-        // Weight copies queued ahead of the consumers' activation loads delay them (the row is a cache hit that then
-        // waits behind megabytes of misses): one stage goes out at once, the rest after those loads have been issued.
-        if (it == kEarlyStages && !mbar_wait(&xbar, 0)) {
-          atomicExch(p.status, 3);
-          break;
-        }
-        if (it == kStages) {
-          // The first stages are in flight.  Dependents may only be released once this grid's own dependency is
-          // resolved, so that a dependent's prologue never overlaps anything older than this kernel.
-          asm volatile("griddepcontrol.wait;" ::: "memory");
-          asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-        }
-        const int tile = first + it * gx;
-        uint8_t* dst = stages + (size_t)s * stage_bytes;
-        mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
-        if (SW) {
-          // gate rows land in stage rows [0, ROWS/2), up rows in [ROWS/2, ROWS)
-          const size_t r0 = (size_t)tile * OUT_ROWS;
-          const uint8_t *g = p.seg[0].base, *u = p.seg[1].base;
-          const size_t n = (size_t)p.seg[0].n_rows;
-          bulk_g2s(dst, g + r0 * row_codes, OUT_ROWS * row_codes, &full[s], pol);
-          bulk_g2s(dst + OUT_ROWS * row_codes, u + r0 * row_codes, OUT_ROWS * row_codes, &full[s], pol);
-          uint8_t* sd = dst + ROWS * row_codes;
-          bulk_g2s(sd, g + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s], pol);
-          bulk_g2s(sd + OUT_ROWS * row_scales, u + n * row_codes + r0 * row_scales, OUT_ROWS * row_scales, &full[s], pol);
-        } else {
-          int sg = 0;
-          while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
-          const size_t r0 = (size_t)(tile - p.seg[sg].tile0) * ROWS;
-          const uint8_t* b = p.seg[sg].base;
-          bulk_g2s(dst, b + r0 * row_codes, ROWS * row_codes, &full[s], pol);
-          bulk_g2s(dst + ROWS * row_codes, b + (size_t)p.seg[sg].n_rows * row_codes + r0 * row_scales, ROWS * row_scales, &full[s], pol);
-        }
-      }
-    }
+  __shared__ StreamShared sh;
+  constexpr int ROWS = kGroupWarps / PARTS * kRPW;
+  const int stage_bytes = ROWS * (p.K / 2 + p.K / 16);
+  stream_init(sh);
+  const StreamRing ring{smem, stage_bytes, kStages, reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes), 0, 0};
+  if ((threadIdx.x >> 5) == kConsumerWarps) {
+    // weights do not depend on the preceding kernel, so their copies start before the grid dependency is resolved
+    if ((threadIdx.x & 31) == 0) stream_produce<PARTS, SW, true>(p, bx, gx, wait_first, sh, ring, l2_evict_first_policy());
     return;
   }
-
-  // ------------------------------------------------------------------ consumers
-  const int tid = threadIdx.x;                // 0..511
-  const int grp = warp / kGroupWarps;         // which of the two tile streams
-  const int wg = warp % kGroupWarps;          // warp within the group
-  const int tg = tid % (kGroupWarps * 32);    // thread within the group
-  // The norm gains are parameters, not products of the preceding kernel: fetch them before waiting for it.  (Every CTA
-  // reads the same few kilobytes, and such a broadcast read takes far longer than an ordinary L2 hit.)
-  uint4 graw = make_uint4(0, 0, 0, 0);
-  if (p.gain && tid * 8 < K) graw = __ldg(reinterpret_cast<const uint4*>(p.gain + tid * 8));
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // the activation comes from the preceding kernel
-  const int part = wg % PARTS, rsub = wg / PARTS;
-  const int pblk = (nblk + PARTS - 1) / PARTS;
-  const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
-  uint32_t xr[kJ][16];
-  float xm[kJ], xc[kJ];
-  {
-    // Thread t owns the runs of 8 consecutive elements r = t + 512 j (one run when K <= 4096, up to four for K = 16384);
-    // four adjacent lanes hold one 32-element block.  The optional RMSNorm (h = rn16(x * g / sqrt(mean(x^2) + eps)),
-    // K <= 4096) and the block quantization work on those registers; the quantized blocks go to shared memory once
-    // per CTA (28 words per block; the 112-byte pitch keeps the 128-bit reads conflict-free) and every lane then
-    // fetches the blocks of its k-part.
-    uint32_t* xq_s = reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes);
-    auto load_run = [&](const __half* src16, const float* src32, int i0, float (&xv)[8]) {
-      if (src32) {
-        const float4 a = *reinterpret_cast<const float4*>(src32 + i0);
-        const float4 b = *reinterpret_cast<const float4*>(src32 + i0 + 4);
-        xv[0] = a.x; xv[1] = a.y; xv[2] = a.z; xv[3] = a.w;
-        xv[4] = b.x; xv[5] = b.y; xv[6] = b.z; xv[7] = b.w;
-      } else {
-        const uint4 a = *reinterpret_cast<const uint4*>(src16 + i0);
-        const uint32_t w4[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          __half2 h2;
-          *reinterpret_cast<uint32_t*>(&h2) = w4[q];
-          const float2 f = __half22float2(h2);
-          xv[2 * q] = f.x;
-          xv[2 * q + 1] = f.y;
-        }
-      }
-    };
-    if (p.gain) {
-      // norm prologue: K <= 4096, one run per thread
-      const int i0 = tid * 8;
-      const bool has = i0 < K;
-      float xv[8];
-#pragma unroll
-      for (int q = 0; q < 8; ++q) xv[q] = 0.f;
-      float ss = 0.f;
-      if (has) load_run(p.norm_in16, p.norm_in32, i0, xv);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&xbar);
-      if (has) {
-#pragma unroll
-        for (int q = 0; q < 8; ++q) ss = fmaf(xv[q], xv[q], ss);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      if (lane == 0) red_s[warp] = ss;
-      consumer_sync_all();
-      float tot = 0.f;
-#pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) tot += red_s[w];
-      const float inv = 1.0f / sqrtf(tot / (float)K + p.eps);
-      if (has) {
-        const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
-        uint32_t o4[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          __half2 g2;
-          *reinterpret_cast<uint32_t*>(&g2) = gw[q];
-          const float2 gf = __half22float2(g2);
-          const __half2 h2 = __floats2half2_rn(xv[2 * q] * gf.x * inv, xv[2 * q + 1] * gf.y * inv);
-          o4[q] = *reinterpret_cast<const uint32_t*>(&h2);
-          const float2 f = __half22float2(h2);  // the operand is the fp16-rounded value
-          xv[2 * q] = f.x;
-          xv[2 * q + 1] = f.y;
-        }
-        if (p.h_out && bx == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-        quantize_run4(xv, tid & 3, xq_s + (size_t)(tid >> 2) * kXqWords);
-      }
-    } else {
-      uint4 raw[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int r = tid + 512 * j;  // run index; block r / 4, word r % 4.  All four lanes of a group are in range together.
-        if (r * 8 < K) raw[j] = *reinterpret_cast<const uint4*>(p.x16 + r * 8);
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&xbar);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int r = tid + 512 * j;
-        if (r * 8 < K) {
-          float xv[8];
-          const uint32_t w4[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            __half2 h2;
-            *reinterpret_cast<uint32_t*>(&h2) = w4[q];
-            const float2 f = __half22float2(h2);
-            xv[2 * q] = f.x;
-            xv[2 * q + 1] = f.y;
-          }
-          quantize_run4(xv, r & 3, xq_s + (size_t)(r >> 2) * kXqWords);
-        }
-      }
-    }
-    consumer_sync_all();
-#pragma unroll
-    for (int j = 0; j < kJ; ++j) {
-      const int b = b0 + lane + 32 * j;
-      if (b < b1) {
-        const uint4* src = reinterpret_cast<const uint4*>(xq_s + (size_t)b * kXqWords);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint4 v = src[q];
-          xr[j][4 * q] = v.x;
-          xr[j][4 * q + 1] = v.y;
-          xr[j][4 * q + 2] = v.z;
-          xr[j][4 * q + 3] = v.w;
-        }
-        const float2 mc = *reinterpret_cast<const float2*>(xq_s + (size_t)b * kXqWords + 16);
-        xm[j] = mc.x;
-        xc[j] = mc.y;
-      } else {
-#pragma unroll
-        for (int q = 0; q < 16; ++q) xr[j][q] = 0;
-        xm[j] = 0.f;
-        xc[j] = 0.f;
-      }
-    }
-  }
-
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // this group's tiles: it = grp, grp + 2, ...; li counts them.  The cross-lane reduction of a tile's row sums is
-  // deferred into the next tile's iteration, where its shuffle latencies hide behind that tile's integer work.
-  const int n_li = n_it > grp ? (n_it - grp + kGroups - 1) / kGroups : 0;
-  float* my_part = part_s[grp];
-  bool failed = false;
-  auto reduce_store = [&](float (&a)[kRPW], int slot) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-      for (int r = 0; r < kRPW; ++r) a[r] += __shfl_xor_sync(0xffffffffu, a[r], o);
-    if (lane == 0) {
-#pragma unroll
-      for (int r = 0; r < kRPW; ++r) my_part[(slot * ROWS + r * (ROWS / kRPW) + rsub) * PARTS + part] = a[r];
-    }
-  };
-  for (int li0 = 0; li0 < n_li; li0 += kMaxIt) {
-    const int li1 = min(n_li, li0 + kMaxIt);
-    float prev[kRPW];
-    bool have_prev = false;
-    for (int li = li0; li < li1; ++li) {
-      const int it = grp + kGroups * li;
-      const int s = it % kStages;
-      if (!__all_sync(0xffffffffu, mbar_wait(&full[s], (it / kStages) & 1))) {
-        failed = true;
-        break;
-      }
-      const uint8_t* st = stages + (size_t)s * stage_bytes;
-      uint4 cw[kRPW][kJ];
-      float sc[kRPW][kJ];
-#pragma unroll
-      for (int r = 0; r < kRPW; ++r) {
-        const int row = r * (ROWS / kRPW) + rsub;  // stage row of this warp's r-th row
-        const uint4* codes = reinterpret_cast<const uint4*>(st + (size_t)row * row_codes);
-        const __half* scp = reinterpret_cast<const __half*>(st + (size_t)ROWS * row_codes + (size_t)row * row_scales);
-#pragma unroll
-        for (int j = 0; j < kJ; ++j) {
-          const int b = b0 + lane + 32 * j;
-          const bool in = b < b1;
-          cw[r][j] = in ? codes[b] : make_uint4(0, 0, 0, 0);
-          sc[r][j] = in ? __half2float(scp[b]) : 0.f;
-        }
-      }
-      if (have_prev) reduce_store(prev, li - 1 - li0);
-      float acc[kRPW];
-#pragma unroll
-      for (int r = 0; r < kRPW; ++r) {
-        acc[r] = 0.f;
-#pragma unroll
-        for (int j = 0; j < kJ; ++j) {
-          const uint32_t ws[4] = {cw[r][j].x, cw[r][j].y, cw[r][j].z, cw[r][j].w};
-          int dl = 0, dh = 0;
-#pragma unroll
-          for (int w = 0; w < 4; ++w) {
-            const uint32_t lo = ws[w] & 0x0F0F0F0Fu, hi = ws[w] & 0xF0F0F0F0u;  // hi carries 16 * code
-            dl = dp2a_lo(xr[j][4 * w], lo, dl);
-            dl = dp2a_hi(xr[j][4 * w + 1], lo, dl);
-            dh = dp2a_lo(xr[j][4 * w + 2], hi, dh);
-            dh = dp2a_hi(xr[j][4 * w + 3], hi, dh);
-          }
-          const float dot = (float)(dl + (dh >> 4));  // dh is a multiple of 16; |dot| < 2^24: exact
-          acc[r] = fmaf(sc[r][j], fmaf(dot, xm[j], xc[j]), acc[r]);
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[s]);  // this warp is done reading stage s
-#pragma unroll
-      for (int r = 0; r < kRPW; ++r) prev[r] = acc[r];
-      have_prev = true;
-    }
-    if (have_prev && !failed) reduce_store(prev, li1 - 1 - li0);
-    if (failed) fail_s = 1;
-    group_sync(grp);
-    if (fail_s) {  // a warp of either group gave up: nobody waits at a barrier for it
-      if (tg == 0) atomicExch(p.status, 1);
-      return;
-    }
-    // flush: sum the k-parts (ascending) and run the epilogue
-    const int n_out = (li1 - li0) * OUT_ROWS;
-    for (int i = tg; i < n_out; i += kGroupWarps * 32) {
-      const int itl = i / OUT_ROWS, j = i % OUT_ROWS;
-      const int tile = first + (grp + kGroups * (li0 + itl)) * gx;
-      float v[2];
-#pragma unroll
-      for (int h = 0; h < (SW ? 2 : 1); ++h) {
-        const float* ps = my_part + ((size_t)itl * ROWS + j + h * OUT_ROWS) * PARTS;
-        float t = 0.f;
-#pragma unroll
-        for (int q = 0; q < PARTS; ++q) t += ps[q];
-        v[h] = t;
-      }
-      if (SW) {
-        p.y16[(size_t)tile * OUT_ROWS + j] = __float2half_rn(silu_mul_f(v[0], v[1]));
-      } else {
-        // output index: rows of the segments lie side by side
-        int sg = 0;
-        while (sg + 1 < p.n_seg && tile >= p.seg[sg + 1].tile0) ++sg;
-        int row = (tile - p.seg[sg].tile0) * ROWS + j;
-        for (int q = 0; q < sg; ++q) row += p.seg[q].n_rows;
-        switch (p.mode) {
-          case GEMV_OUT_F32: p.y32[row] = v[0]; break;
-          case GEMV_OUT_F16: p.y16[row] = __float2half_rn(v[0]); break;
-          case GEMV_RES16_OUT_F32: p.y32[row] = __half2float(p.res16[row]) + v[0]; break;
-          case GEMV_RES32_OUT_F16: p.y16[row] = __float2half_rn(p.res32[row] + v[0]); break;
-          case GEMV_RES16_OUT_F16: p.y16[row] = __float2half_rn(__half2float(p.res16[row]) + v[0]); break;
-          default: break;
-        }
-      }
-    }
-    group_sync(grp);
-  }
+  stream_consume<PARTS, SW>(p, bx, gx, sh, ring, [] { asm volatile("griddepcontrol.wait;" ::: "memory"); }, true);
 }
 
 template <int PARTS, bool SW>
@@ -547,57 +65,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const Stre
   gemv_stream_body<PARTS, SW>(p, (int)blockIdx.x, (int)gridDim.x, m.ids != nullptr);
 }
 
-int parts_for(int K) { return K <= 2048 ? 1 : K <= 4096 ? 2 : K <= 8192 ? 4 : 8; }
+int parts_for(int K) { return stream_parts_for(K); }
 
 }  // namespace
 
-bool gemv_stream_eligible(const GemvParams& p) {
-  if (p.M != 1 || p.K % 256 != 0 || p.K > 16384) return false;
-  const int parts = parts_for(p.K);
-  const int rows = kGroupWarps / parts * kRPW;
-  if (p.mode == GEMV_SWIGLU_F16) {
-    if (p.n_seg != 2 || p.seg[0].n_rows != p.seg[1].n_rows || p.seg[0].n_rows % (rows / 2)) return false;
-  } else {
-    for (int s = 0; s < p.n_seg; ++s)
-      if (p.seg[s].n_rows % rows) return false;
-  }
-  if (p.norm_gain && p.K > 4096) return false;  // the fused norm prologue covers hidden sizes up to 4096
-  return true;
-}
+bool gemv_stream_eligible(const GemvParams& p) { return stream_shape_ok(p); }
 
 cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch) {
   const int parts = parts_for(g.K);
-  const int rows = kGroupWarps / parts * kRPW;
   const bool sw = g.mode == GEMV_SWIGLU_F16;
-  StreamParams p{};
-  p.n_seg = g.n_seg;
-  int tiles = 0;
-  if (sw) {
-    p.seg[0] = StreamSeg{g.seg[0].base, g.seg[0].n_rows, 0};
-    p.seg[1] = StreamSeg{g.seg[1].base, g.seg[1].n_rows, 0};
-    tiles = g.seg[0].n_rows / (rows / 2);
-  } else {
-    for (int s = 0; s < g.n_seg; ++s) {
-      p.seg[s] = StreamSeg{g.seg[s].base, g.seg[s].n_rows, tiles};
-      tiles += g.seg[s].n_rows / rows;
-    }
-  }
-  p.n_tiles = tiles;
-  p.K = g.K;
-  p.mode = g.mode;
-  p.x16 = g.x;
-  p.norm_in16 = g.norm_x16;
-  p.norm_in32 = g.norm_x32;
-  p.gain = g.norm_gain;
-  p.eps = g.norm_eps;
-  p.h_out = g.norm_out;
-  p.y32 = g.y32;
-  p.y16 = g.y16;
-  p.res32 = g.res32;
-  p.res16 = g.res16;
-  p.status = status;
-  const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * (kXqWords * 4);
+  const StreamParams p = stream_params_from(g, status);
+  const int tiles = p.n_tiles;
+  const size_t stage_bytes = stream_stage_bytes(g.K);
+  const size_t smem = kStages * stage_bytes + stream_xq_bytes(g.K);
   const int grid = std::max(1, std::min(tiles, sm_count));
   void (*kern)(const StreamParams) = nullptr;
   switch (parts) {
