@@ -182,7 +182,7 @@ struct StreamShared {
   uint64_t xbar;  // consumers -> producer: the activation loads of the current phase have been issued
   float part_s[kGroups][kMaxIt * kGroupWarps * kRPW];
   float red_s[kConsumerWarps];
-  int fail_s;
+  int fail_g[kGroups];  // a warp of the group gave up a bounded wait (written and read by that group only)
 };
 
 // Where a phase's ring stages live and where its iterations sit in the CTA's global sequence: stage and barrier parity
@@ -198,7 +198,7 @@ struct StreamRing {
 
 __device__ __forceinline__ void stream_init(StreamShared& sh) {
   if (threadIdx.x == 0) {
-    sh.fail_s = 0;
+    for (int g = 0; g < kGroups; ++g) sh.fail_g[g] = 0;
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sh.full[s], 1);
       mbar_init(&sh.empty[s], kGroupWarps);
@@ -493,9 +493,9 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
       have_prev = true;
     }
     if (have_prev && !failed) reduce_store(prev, li1 - 1 - li0);
-    if (failed) sh.fail_s = 1;
+    if (failed) sh.fail_g[grp] = 1;
     group_sync(grp);
-    if (sh.fail_s) {  // a warp of either group gave up: nobody waits at a barrier for it
+    if (sh.fail_g[grp]) {  // a warp of this group gave up; every thread of the group reads the same flag and leaves here
       if (tg == 0) atomicExch(p.status, 1);
       return false;
     }
