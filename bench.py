@@ -335,6 +335,42 @@ def extra_moe(torch, B, W, peaks, quick):
             elif hybrid and st.streamed_bytes:
                 out[key]["pcie_gbs_over_call_time"] = st.streamed_bytes / n / dt / 1e9
         ctx.close()
+    # prefill of the same block: 512 tokens per call, every (token, slot) pair a row of a grouped GEMM over the experts
+    T = 128 if quick else 512
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, w_gate=0, w_up=0, w_down=0)
+    ws = B.workspace_bytes(probe, T) + (1 << 20)
+    for hybrid in (False, True):
+        ctx = B.Context(ws + 3 * shape.n_experts * (sl + 256) + 8 * (sl + 256) + (16 << 20), workspace_bytes=ws, ring_slots=8,
+                        slot_bytes=sl, chunk_bytes=sl)
+        ids = {"ffn_norm": ctx.register_f16(Bk[W.ROLE_FFN_NORM]), "router": ctx.register_f16(Bk[W.ROLE_ROUTER])}
+        for name, r in (("w_gate", W.ROLE_GATE), ("w_up", W.ROLE_UP), ("w_down", W.ROLE_DOWN)):
+            ids[name] = ctx.register_q4(*Bk[r], role=r)
+        desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, rms_eps=shape.rms_eps, **ids)
+        ctx.set_placement([(ids[n], e, B.ATS_HOST if (hybrid and e % 2) else B.ATS_GPU) for n in ("w_gate", "w_up", "w_down")
+                           for e in range(shape.n_experts)])
+        xs = [torch.from_numpy(W.activations(4, 0, (T, shape.hidden), step=s)).cuda() for s in range(4)]
+        y = torch.empty((T, shape.hidden), dtype=torch.float16, device="cuda")
+        n = 8 if quick else 32
+
+        def gop(k):
+            for i in range(k):
+                ctx.layer_prefill(desc, xs[i % 4], y, None, None, 0, T)
+        gop(4)
+        ctx.sync()
+        t0 = time.perf_counter()
+        gop(n)
+        ctx.sync()
+        dt = (time.perf_counter() - t0) / n
+        flop = 2.0 * T * shape.top_k * 3 * shape.hidden * shape.ffn
+        key = f"prefill_T{T}_{'hybrid' if hybrid else 'resident'}"
+        out[key] = {"ms_per_call": dt * 1e3, "tokens_per_s": T / dt, "expert_gemm_flop_per_call": flop,
+                    "expert_gemm_tflops_over_call_time": flop / dt / 1e12,
+                    "timing": "wall clock around back-to-back calls (each has one host synchronisation for the routing ids)"}
+        if hybrid:
+            # every odd expert that some token selected is read once per 128 of its rows, in place over PCIe
+            out[key]["host_expert_bytes_upper"] = 3 * sl * (shape.n_experts // 2)
+            out[key]["pcie_gbs_lower_bound_if_all_odd_experts_selected"] = 3 * sl * (shape.n_experts // 2) / dt / 1e9
+        ctx.close()
     return out
 
 

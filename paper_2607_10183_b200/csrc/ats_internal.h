@@ -255,6 +255,11 @@ cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_ro
                                        uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_attn_prefill(const __half* q_rot16, const __half* kc, const __half* vc, __half* a16, int T, int n_q,
                                 int n_kv, int d, int cap, int pos0, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
+// MoE prefill helpers (kernels_prefill.cu): rows gathered in expert order, and the gated sum back in token order
+cudaError_t launch_moe_gather_rows(const __half* h, const int* order, int k, __half* xs, int P, int H, cudaStream_t st,
+                                   uint64_t* n_launch, int pdl = 0);
+cudaError_t launch_moe_combine_sorted(const __half* res, const float* gates, const __half* d, const int* pos, __half* y, int T, int k,
+                                      int H, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch,
                             int pdl = 0);
 
@@ -276,6 +281,14 @@ struct GemmParams {
   const __half* res;
   __half* y2;
   int pdl;  // programmatic dependent launch allowed (see launch_dep)
+  // grouped form (MoE prefill): the T activation rows are sorted by expert; expert e owns rows grp_off[e] .. grp_off[e+1]-1
+  // and multiplies them with slice e of every segment (seg[i].base + e * grp_stride, or grp_tab[i][e] where a table is
+  // given: device or mapped host addresses).  No split-K, no residual.
+  const int* grp_off;       // DEVICE [n_groups + 1]; null = plain GEMM
+  int n_groups;
+  int grp_max_rows;         // the largest expert's row count (sizes the grid)
+  uint64_t grp_stride;
+  const uint8_t* const* grp_tab[3];
 };
 uint64_t gemm_scratch_bytes(int T, int n_total, int K);
 cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);

@@ -43,6 +43,7 @@ int32_t check_cuda(ats_ctx* c, cudaError_t e, const char* what) {
     if (_s != ATS_OK) return _s;   \
   } while (0)
 
+constexpr int kMaxPairs = 65536;  // (token, slot) pairs of one MoE call at most: ids, then the prefill's sort arrays, in ctx->ids_host
 constexpr uint64_t kWsReserved = 1024;  // status word + attention counters at the start of the workspace
 
 // Kernel timing: a pair of events around one launch on the compute stream.
@@ -355,6 +356,11 @@ struct LayerWs {
   __half* d16 = nullptr;
   void* gemm_scratch = nullptr;
   uint64_t gemm_scratch_bytes = 0;
+  // MoE prefill: rows in expert order
+  __half* xs16 = nullptr;
+  int* order = nullptr;
+  int* pos = nullptr;
+  int* grp_off = nullptr;
   uint64_t total = 0;
   bool ok = true;
 };
@@ -404,11 +410,25 @@ static LayerWs layout_prefill(const ats_layer_desc& L, uint32_t T, uint8_t* base
     scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)H, (int)qd));
   }
   w.h2_16 = (__half*)b.take(T * H * 2);
-  w.gu16 = (__half*)b.take((uint64_t)T * 2 * L.ffn * 2);
-  w.act16 = (__half*)b.take((uint64_t)T * L.ffn * 2);
-  w.d16 = (__half*)b.take(T * H * 2);
-  scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)(2 * L.ffn), (int)H));
-  scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)H, (int)L.ffn));
+  if (L.n_experts) {
+    // every (token, slot) pair is a row of the expert GEMMs
+    const uint64_t P = (uint64_t)T * L.top_k;
+    w.ids = (int32_t*)b.take(P * 4);
+    w.gates = (float*)b.take(P * 4);
+    w.order = (int*)b.take(P * 4);
+    w.pos = (int*)b.take(P * 4);
+    w.grp_off = (int*)b.take(((uint64_t)L.n_experts + 1) * 4);
+    w.xs16 = (__half*)b.take(P * H * 2);
+    w.gu16 = (__half*)b.take(P * 2 * L.ffn * 2);
+    w.act16 = (__half*)b.take(P * L.ffn * 2);
+    w.d16 = (__half*)b.take(P * H * 2);
+  } else {
+    w.gu16 = (__half*)b.take((uint64_t)T * 2 * L.ffn * 2);
+    w.act16 = (__half*)b.take((uint64_t)T * L.ffn * 2);
+    w.d16 = (__half*)b.take(T * H * 2);
+    scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)(2 * L.ffn), (int)H));
+    scratch = std::max(scratch, gemm_scratch_bytes((int)T, (int)H, (int)L.ffn));
+  }
   w.gemm_scratch = b.take(scratch);
   w.gemm_scratch_bytes = scratch;
   w.total = align_up(b.off);
@@ -687,7 +707,7 @@ int32_t ats_init(const ats_config* cfg, ats_ctx** out) {
   }
   ok &= cudaEventCreateWithFlags(&ctx->ids_event, cudaEventDisableTiming) == cudaSuccess;
   ok &= cudaEventCreateWithFlags(&ctx->sync_event, cudaEventDisableTiming) == cudaSuccess;
-  ok &= cudaHostAlloc((void**)&ctx->ids_host, 4096 * sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess;
+  ok &= cudaHostAlloc((void**)&ctx->ids_host, (3 * (size_t)kMaxPairs + 2048) * sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess;
   ok &= cudaHostAlloc((void**)&ctx->host_status, 64, cudaHostAllocDefault) == cudaSuccess;
   if (ws >= kWsReserved) {
     ctx->dev_status = (int*)ctx->ws;
@@ -1020,7 +1040,6 @@ static int32_t check_layer(ats_ctx* ctx, const ats_layer_desc* L, bool prefill) 
   ATS_TRY(check_f16(ctx, L->ffn_norm, L->hidden, 1, "ffn_norm"));
   const uint32_t E = L->n_experts ? L->n_experts : 1;
   if (L->n_experts) {
-    if (prefill) return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE prefill is not implemented");
     if (L->top_k == 0 || L->top_k > 32 || L->top_k > L->n_experts || L->n_experts > 1024)
       return fail(ctx, ATS_ERR_SHAPE, "top_k %u of %u experts unsupported", L->top_k, L->n_experts);
     ATS_TRY(check_f16(ctx, L->router, L->n_experts, L->hidden, "router"));
@@ -1034,7 +1053,7 @@ static int32_t check_layer(ats_ctx* ctx, const ats_layer_desc* L, bool prefill) 
 uint64_t ats_workspace_bytes(const ats_layer_desc* L, uint32_t max_tokens) {
   if (!L || max_tokens == 0) return 0;
   uint64_t need = layout_decode(*L, std::min<uint32_t>(max_tokens, 32), nullptr, ~0ull).total;
-  if (L->n_experts == 0) need = std::max(need, layout_prefill(*L, max_tokens, nullptr, ~0ull).total);
+  need = std::max(need, layout_prefill(*L, max_tokens, nullptr, ~0ull).total);
   // staging rows of ats_layer_decode_host (input and output), each padded to the arena alignment
   need += 2 * align_up((uint64_t)std::min<uint32_t>(max_tokens, 32) * L->hidden * 2);
   return need + kAlign;
@@ -1242,9 +1261,20 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     plan_dense(ctx, L->wv, &qkv[2]);
     plan_dense(ctx, L->wo, &wo);
   }
-  plan_dense(ctx, L->w_gate, &gu[0]);
-  plan_dense(ctx, L->w_up, &gu[1]);
-  plan_dense(ctx, L->w_down, &wd);
+  const bool moe = L->n_experts != 0;
+  if (moe) {
+    if ((uint64_t)T * L->top_k > (uint64_t)kMaxPairs)
+      return fail(ctx, ATS_ERR_SHAPE, "MoE prefill takes T * top_k <= %d pairs per call", kMaxPairs);
+    for (int id : {L->w_gate, L->w_up, L->w_down}) {
+      const Tensor& t = ctx->tensors[id];
+      if (!t.contiguous_dev && !t.slice_tab_dev)
+        return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE prefill with host-placed experts needs the pinned store mapped into the device");
+    }
+  } else {
+    plan_dense(ctx, L->w_gate, &gu[0]);
+    plan_dense(ctx, L->w_up, &gu[1]);
+    plan_dense(ctx, L->w_down, &wd);
+  }
   ATS_TRY(pump(ctx));
 
   const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
@@ -1277,6 +1307,81 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     resid = w.x1_16;
   }
   ATS_CUDA(launch_rmsnorm(resid, 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, w.h2_16, (int)T, H, L->rms_eps, ctx->cs, nl, pdl));
+  if (moe) {
+    // Routed FFN over T tokens: every (token, slot) pair becomes a row; rows are sorted by expert so that each expert's
+    // rows are one contiguous block of a grouped GEMM (one launch for all experts).  The sort runs on the host from the
+    // routing ids (one synchronisation per call); expert slices are read where they are: resident copies, or the pinned
+    // host store through its device mapping for host-placed experts (every slice is read once per 128 of its rows).
+    const int k = (int)L->top_k, E = (int)L->n_experts, P = (int)T * k, F = (int)L->ffn;
+    ATS_CUDA(launch_router_topk(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)T, H, E, k,
+                                (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, ctx->cs, nl, pdl));
+    ATS_TRY(fetch_ids(ctx, w.ids, P, E));
+    int32_t* order_h = ctx->ids_host + kMaxPairs;       // sorted position -> pair
+    int32_t* pos_h = ctx->ids_host + 2 * kMaxPairs;     // pair -> sorted position
+    int32_t* off_h = ctx->ids_host + 3 * kMaxPairs;     // expert -> first sorted position; [E] = P
+    std::vector<int> cnt(E + 1, 0);
+    for (int p2 = 0; p2 < P; ++p2) cnt[ctx->ids_host[p2] + 1]++;
+    int max_rows = 0;
+    for (int e = 0; e < E; ++e) {
+      max_rows = std::max(max_rows, cnt[e + 1]);
+      cnt[e + 1] += cnt[e];
+    }
+    for (int e = 0; e <= E; ++e) off_h[e] = cnt[e];
+    for (int p2 = 0; p2 < P; ++p2) {  // stable: pairs of an expert keep their (token, slot) order
+      const int r = cnt[ctx->ids_host[p2]]++;
+      order_h[r] = p2;
+      pos_h[p2] = r;
+    }
+    ATS_CUDA(cudaMemcpyAsync(w.order, order_h, (size_t)P * 4, cudaMemcpyHostToDevice, ctx->cs));
+    ATS_CUDA(cudaMemcpyAsync(w.pos, pos_h, (size_t)P * 4, cudaMemcpyHostToDevice, ctx->cs));
+    ATS_CUDA(cudaMemcpyAsync(w.grp_off, off_h, (size_t)(E + 1) * 4, cudaMemcpyHostToDevice, ctx->cs));
+    ATS_CUDA(launch_moe_gather_rows(w.h2_16, w.order, k, w.xs16, P, H, ctx->cs, nl, pdl));
+    const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
+    auto slice0 = [](const Tensor& t) -> const uint8_t* { return t.contiguous_dev ? t.slices[0].dev : nullptr; };
+    std::string err;
+    GemmParams m{};
+    m.T = P;
+    m.pdl = pdl;
+    m.status = ctx->dev_status;
+    m.grp_off = w.grp_off;
+    m.n_groups = E;
+    m.grp_max_rows = max_rows;
+    // gate | up side by side
+    m.n_seg = 2;
+    m.K = H;
+    m.seg[0] = GemvSeg{slice0(tg), F};
+    m.seg[1] = GemvSeg{slice0(tu), F};
+    m.grp_stride = tg.slice_stride;
+    m.grp_tab[0] = tg.contiguous_dev ? nullptr : tg.slice_tab_dev;
+    m.grp_tab[1] = tu.contiguous_dev ? nullptr : tu.slice_tab_dev;
+    if ((tg.contiguous_dev != tu.contiguous_dev) && (!tg.slice_tab_dev || !tu.slice_tab_dev))
+      return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE prefill: gate and up need the same kind of placement or mapped slice tables");
+    if (tg.contiguous_dev != tu.contiguous_dev) {  // mixed: use the tables for both
+      m.grp_tab[0] = tg.slice_tab_dev;
+      m.grp_tab[1] = tu.slice_tab_dev;
+    }
+    m.x = w.xs16;
+    m.ldx = H;
+    m.y = w.gu16;
+    m.ldy = 2 * F;
+    cudaError_t ce = launch_gemm(m, ctx->cs, nl, &err);
+    if (ce != cudaSuccess) return check_cuda(ctx, ce, err.empty() ? "launch_gemm (expert gate/up)" : err.c_str());
+    ATS_CUDA(launch_swiglu16(w.gu16, 2 * F, F, w.act16, P, ctx->cs, nl, pdl));
+    m.n_seg = 1;
+    m.K = F;
+    m.seg[0] = GemvSeg{slice0(td), H};
+    m.grp_stride = td.slice_stride;
+    m.grp_tab[0] = td.contiguous_dev ? nullptr : td.slice_tab_dev;
+    m.grp_tab[1] = nullptr;
+    m.x = w.act16;
+    m.ldx = F;
+    m.y = w.d16;
+    m.ldy = H;
+    ce = launch_gemm(m, ctx->cs, nl, &err);
+    if (ce != cudaSuccess) return check_cuda(ctx, ce, err.empty() ? "launch_gemm (expert down)" : err.c_str());
+    ATS_CUDA(launch_moe_combine_sorted(resid, w.gates, w.d16, w.pos, (__half*)x_out, (int)T, k, H, ctx->cs, nl, pdl));
+    return ATS_OK;
+  }
   g.x = w.h2_16;
   g.ldx = H;
   g.y = w.gu16;

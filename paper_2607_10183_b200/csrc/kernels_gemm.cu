@@ -62,6 +62,11 @@ struct GemmKParams {
   int* status;
   const __half* res;  // optional residual: y2 = rn16(res + y)
   __half* y2;
+  // grouped form (one weight slice per expert, blockIdx.z = expert; splits = 1): expert e multiplies the activation rows
+  // grp_off[e] .. grp_off[e+1]-1 (rows sorted by expert) with slice e of every segment and writes the same rows of y
+  const int* grp_off;                 // DEVICE [n_experts + 1], null = the plain form
+  unsigned long long grp_stride;      // bytes between the slices of consecutive experts (contiguous resident experts)
+  const uint8_t* const* grp_tab[3];   // per segment: DEVICE table of slice addresses (device or mapped host memory), or null
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -178,12 +183,24 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
   const int row0 = (tile - p.seg[sg].tile0) * p.bf;
   const int n_rows = p.seg[sg].n_rows;
   const int t0 = blockIdx.y * TTILE;
-  const int Tt = min(TTILE, p.T - t0);
+  // grouped form: the expert's rows and weight slice.  The row offsets were written by a copy that precedes this launch
+  // in the stream, so every thread waits for the grid dependency before reading them.
+  int T_ = p.T, rowoff = 0;
+  const uint8_t* segbase = p.seg[sg].base;
+  if (p.grp_off) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int e = blockIdx.z;
+    rowoff = p.grp_off[e];
+    T_ = p.grp_off[e + 1] - rowoff;
+    if (t0 >= T_) return;  // this expert has fewer rows than the grid's token blocks cover (no barrier, no tensor memory yet)
+    segbase = p.grp_tab[sg] ? p.grp_tab[sg][e] : segbase + (size_t)e * p.grp_stride;
+  }
+  const int Tt = min(TTILE, T_ - t0);
   const int nmma = min(p.bf, (n_rows - row0 + 15) / 16 * 16);  // MMA N: the features of this tile that hold real rows
   const int n_dq = (p.bf + 15) / 16;                           // dequantization warps with rows to fill (16 rows each)
   const int boxes = (Tt + BOXR - 1) / BOXR;                  // TMA boxes of 64 activation rows
   const int n_mb = (Tt + BM - 1) / BM;                       // 128-token blocks (MMA M) that hold real tokens
-  const int split = blockIdx.z;
+  const int split = p.grp_off ? 0 : blockIdx.z;
   const int ks0 = split * p.ksteps_per_split;
   const int nks = min(p.ksteps_per_split, p.total_ksteps - ks0);
   if (threadIdx.x == 0) {
@@ -225,7 +242,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
         uint8_t* bdst = smem + (size_t)s * kStageBytes + FT * A_BYTES;
         mbar_expect_tx(&full_b[s], tx);
         for (int b = 0; b < boxes; ++b)
-          tma_load_2d(bdst + (size_t)b * BOXR * BK * 2, &xmap, (ks0 + i) * BK, t0 + b * BOXR, &full_b[s]);
+          tma_load_2d(bdst + (size_t)b * BOXR * BK * 2, &xmap, (ks0 + i) * BK, rowoff + t0 + b * BOXR, &full_b[s]);
       }
     }
   } else if (warp == 1) {
@@ -281,8 +298,8 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
     const int grow = row0 + r;
     const bool valid = grow < n_rows;
     const int K = p.K, nblk = K / 32;
-    const uint8_t* crow = p.seg[sg].base + (size_t)(valid ? grow : 0) * (K / 2);
-    const __half* srow = reinterpret_cast<const __half*>(p.seg[sg].base + (size_t)n_rows * (K / 2)) + (size_t)(valid ? grow : 0) * nblk;
+    const uint8_t* crow = segbase + (size_t)(valid ? grow : 0) * (K / 2);
+    const __half* srow = reinterpret_cast<const __half*>(segbase + (size_t)n_rows * (K / 2)) + (size_t)(valid ? grow : 0) * nblk;
     // Packed weights are fetched kPD k-steps ahead into registers: a k-step lasts about a thousand cycles, less than
     // the latency of a first-touch DRAM read under load.  Scales come as one 16-byte load per row for four k-steps
     // (eight blocks) when the row's scale array is 16-byte aligned, else one fp16 at a time.
@@ -378,7 +395,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
       const int mb = (w2 >> 2) % MB;        // token block = accumulator
       const int ch = w2 / (MB * 4);         // which half of the feature columns
       const int t = t0 + mb * BM + q * 32 + lane;
-      const bool tvalid = t < p.T;
+      const bool tvalid = t < T_;
       const int colbase = p.seg[sg].col0 + row0;
       const bool vec = (p.ldy % 8 == 0) && (colbase % 8 == 0) &&
                        (((reinterpret_cast<uintptr_t>(p.y) | reinterpret_cast<uintptr_t>(p.res) | reinterpret_cast<uintptr_t>(p.y2)) & 15) == 0);
@@ -403,7 +420,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
                 const int r = 4 * j + (lane >> 3), cq = lane & 7;
                 const uint4 val = *reinterpret_cast<const uint4*>(stg + r * 144 + cq * 16);
                 const int tt = tbase + r;
-                if (tt < p.T) *reinterpret_cast<uint4*>(p.partial + ((size_t)split * p.T + tt) * p.ldy + colbase + c0 + cq * 4) = val;
+                if (tt < T_) *reinterpret_cast<uint4*>(p.partial + ((size_t)split * p.T + tt) * p.ldy + colbase + c0 + cq * 4) = val;
               }
               __syncwarp();
             } else if (tvalid) {
@@ -430,8 +447,8 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
                 const int r = 8 * j + (lane >> 2), cq = lane & 3;
                 const uint4 o4 = *reinterpret_cast<const uint4*>(stg + r * 80 + cq * 16);
                 const int tt = tbase + r;
-                if (tt < p.T) {
-                  const size_t off = (size_t)tt * p.ldy + colbase + c0 + cq * 8;
+                if (tt < T_) {
+                  const size_t off = (size_t)(rowoff + tt) * p.ldy + colbase + c0 + cq * 8;
                   *reinterpret_cast<uint4*>(p.y + off) = o4;
                   if (p.res) {
                     const uint4 r4 = *reinterpret_cast<const uint4*>(p.res + off);
@@ -449,14 +466,14 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(c
               }
               __syncwarp();
             } else if (tvalid) {
-              __half* dst = p.y + (size_t)t * p.ldy + colbase + c0;
+              __half* dst = p.y + (size_t)(rowoff + t) * p.ldy + colbase + c0;
 #pragma unroll
               for (int e = 0; e < 32; ++e)
                 if (e < nf) {
                   const __half h = __float2half_rn(__uint_as_float(v[e]));
                   dst[e] = h;
                   if (p.res) {
-                    const size_t off = (size_t)t * p.ldy + colbase + c0 + e;
+                    const size_t off = (size_t)(rowoff + t) * p.ldy + colbase + c0 + e;
                     p.y2[off] = __float2half_rn(__half2float(p.res[off]) + __half2float(h));
                   }
                 }
@@ -626,7 +643,12 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   int seg_rows[3] = {0, 0, 0};
   for (int i = 0; i < g.n_seg; ++i) seg_rows[i] = g.seg[i].n_rows;
   const int total_ksteps = (g.K + BK - 1) / BK;
-  const GemmPlan pl = choose_plan(seg_rows, g.n_seg, g.T, g.ldy, total_ksteps, sm_count, g.scratch ? g.scratch_bytes : 0);
+  GemmPlan pl = choose_plan(seg_rows, g.n_seg, g.T, g.ldy, total_ksteps, sm_count, g.scratch ? g.scratch_bytes : 0);
+  if (g.grp_off) {
+    // per-expert row counts are small next to the tile: 128-token tiles unless an expert holds several of them
+    if (g.res || g.n_groups <= 0 || g.grp_max_rows <= 0) return cudaErrorInvalidValue;
+    pl = GemmPlan{g.grp_max_rows > 256, 1, g.grp_max_rows > 256 ? 256 : 128};
+  }
   const bool wide = pl.wide;
   const int bf = pl.bf, tt = wide ? 256 : 128;
   GemmKParams p{};
@@ -638,7 +660,7 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
     tiles += (g.seg[i].n_rows + bf - 1) / bf;
     col += g.seg[i].n_rows;
   }
-  const int tchunks = (g.T + tt - 1) / tt;
+  const int tchunks = g.grp_off ? (g.grp_max_rows + tt - 1) / tt : (g.T + tt - 1) / tt;
   p.K = g.K;
   p.T = g.T;
   p.total_ksteps = total_ksteps;
@@ -650,6 +672,9 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   p.status = g.status;
   p.res = g.res;
   p.y2 = g.y2;
+  p.grp_off = g.grp_off;
+  p.grp_stride = g.grp_stride;
+  for (int i = 0; i < 3; ++i) p.grp_tab[i] = g.grp_tab[i];
   static uint64_t attr_done = 0;
   if (first_use_on_device(&attr_done)) {
     cudaError_t e1 = cudaFuncSetAttribute(gemm_q4_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -657,7 +682,7 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
     if (e1 != cudaSuccess) return e1;
     if (e2 != cudaSuccess) return e2;
   }
-  dim3 grid(tiles, tchunks, p.splits);
+  dim3 grid(tiles, tchunks, g.grp_off ? g.n_groups : p.splits);
   ++*n_launch;
   cudaError_t e;
   if (wide) {

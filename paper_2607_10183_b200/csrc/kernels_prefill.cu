@@ -321,4 +321,75 @@ cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int 
   return launch_dep(swiglu16_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, gu, ld, ffn, act, n8);
 }
 
+// MoE prefill: rows sorted by expert.  xs[r] = h[order[r] / k] (order[r] = the (token, slot) pair at sorted position r);
+// 16 bytes per thread.
+__global__ void moe_gather_rows_kernel(const __half* __restrict__ h, const int* __restrict__ order, int k, __half* __restrict__ xs,
+                                       uint64_t n8, int H) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // h comes from the preceding kernel, order from a preceding copy
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int per_row = H / 8;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t r = i / per_row, c = (i % per_row) * 8;
+    const int t = order[r] / k;
+    *reinterpret_cast<uint4*>(xs + r * H + c) = *reinterpret_cast<const uint4*>(h + (uint64_t)t * H + c);
+  }
+}
+
+cudaError_t launch_moe_gather_rows(const __half* h, const int* order, int k, __half* xs, int P, int H, cudaStream_t st,
+                                   uint64_t* n_launch, int pdl) {
+  const uint64_t n8 = (uint64_t)P * H / 8;  // H is a multiple of 32
+  const int grid = (int)std::min<uint64_t>((n8 + 255) / 256, 148 * 8);
+  ++*n_launch;
+  return launch_dep(moe_gather_rows_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, h, order, k, xs, n8, H);
+}
+
+// y[t] = rn16(res[t] + sum_j gates[t][j] * d[pos[t k + j]]) with the sum in slot order, fp32; pos[p] = sorted position
+// of pair p.  8 columns per thread.
+__global__ void moe_combine_sorted_kernel(const __half* __restrict__ res, const float* __restrict__ gates, const __half* __restrict__ d,
+                                          const int* __restrict__ pos, __half* __restrict__ y, uint64_t n8, int k, int H) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int per_row = H / 8;
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n8; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t t = i / per_row, c = (i % per_row) * 8;
+    float acc[8];
+    {
+      const uint4 rv = *reinterpret_cast<const uint4*>(res + t * H + c);
+      const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 f = __half22float2(bits_as_half2(rw[q]));
+        acc[2 * q] = f.x;
+        acc[2 * q + 1] = f.y;
+      }
+    }
+    for (int j = 0; j < k; ++j) {
+      const float gj = gates[t * k + j];
+      const uint4 dv = *reinterpret_cast<const uint4*>(d + (uint64_t)pos[t * k + j] * H + c);
+      const uint32_t dw[4] = {dv.x, dv.y, dv.z, dv.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 f = __half22float2(bits_as_half2(dw[q]));
+        acc[2 * q] = fmaf(gj, f.x, acc[2 * q]);
+        acc[2 * q + 1] = fmaf(gj, f.y, acc[2 * q + 1]);
+      }
+    }
+    uint32_t ow[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const __half2 r2 = __floats2half2_rn(acc[2 * q], acc[2 * q + 1]);
+      ow[q] = *reinterpret_cast<const uint32_t*>(&r2);
+    }
+    *reinterpret_cast<uint4*>(y + t * H + c) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+  }
+}
+
+cudaError_t launch_moe_combine_sorted(const __half* res, const float* gates, const __half* d, const int* pos, __half* y, int T, int k,
+                                      int H, cudaStream_t st, uint64_t* n_launch, int pdl) {
+  const uint64_t n8 = (uint64_t)T * H / 8;
+  const int grid = (int)std::min<uint64_t>((n8 + 255) / 256, 148 * 8);
+  ++*n_launch;
+  return launch_dep(moe_combine_sorted_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, res, gates, d, pos, y, n8, k, H);
+}
+
 }  // namespace ats

@@ -264,3 +264,105 @@ def test_prefill_layer_stage_by_stage_full_size(B, torch):
     H.assert_close(g["act"], O.rn16(O.silu(g["gu"][:, :ffn]) * g["gu"][:, ffn:]), what="swiglu")
     H.assert_close(g["d"], O.linear(g["act"], *t["w_down"], F16, round_out=True), what="w_down")
     assert np.array_equal(yg.astype(np.float64), O.rn16(g["x1"] + g["d"]))
+
+
+# ------------------------------------------------------------------------------------------------- MoE prefill
+def run_moe_prefill(B, torch, shape, cfg, T, host_experts):
+    """The routed FFN block over T tokens in one ats_layer_prefill call (no attention)."""
+    Bk = W.moe_block(cfg, 0, shape)
+    sl = W.q4_bytes(shape.ffn, shape.hidden)
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, w_gate=0, w_up=0, w_down=0)
+    ws = B.workspace_bytes(probe, T) + MB
+    ctx = B.Context(ws + 8 * (sl + 256) + 3 * shape.n_experts * (sl + 256) + MB, workspace_bytes=ws, ring_slots=8, slot_bytes=sl,
+                    chunk_bytes=MB)
+    desc, ids = H.register_moe_block(ctx, Bk)
+    ctx.set_placement([(ids[n], e, B.ATS_HOST if e in host_experts else B.ATS_GPU) for n in ("w_gate", "w_up", "w_down")
+                       for e in range(shape.n_experts)])
+    x = W.activations(cfg, 0, (T, shape.hidden))
+    y = torch.empty((T, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.reset_stats()
+    ctx.layer_prefill(desc, H.to_dev(x), y, None, None, 0, T)
+    ctx.sync()
+    out = (Bk, x, y.cpu().numpy(), ctx.stats(), ctx.numerics(B.ATS_MODE_PREFILL))
+    ctx.close()
+    return out
+
+
+@pytest.mark.parametrize("T", [1, 37, 150])
+def test_moe_prefill_block_matches_oracle_small(B, torch, T):
+    """Every token of the chunk against the oracle's routed FFN under the prefill contract (fp16 GEMM outputs, fp16-rounded
+    weights); 16 experts, top-4: expert row counts from 0 to well over one 128-row tile at T = 150 (ragged tails)."""
+    shape, cfg = W.MOE_SMALL, 97
+    Bk, x, y, st, (edges, wmode) = run_moe_prefill(B, torch, shape, cfg, T, set())
+    want, ids_ref, gates_ref, logits = O.moe_block(x, H.oracle_moe_tensors(Bk), shape, edges, wmode)
+    # a token whose k-th and (k+1)-th logits nearly tie may legitimately route differently in fp32: leave it out
+    clear = np.array([O.min_rank_gap(logits[t:t + 1], shape.top_k) > 1e-4 for t in range(T)])
+    assert clear.sum() >= T - 2
+    H.assert_close(y[clear], want[clear], what="moe prefill block")
+    assert st.host_syncs == 1 and st.streamed_bytes == 0
+    # host-placed experts are read in place through the mapped pinned store: same bits
+    odd = {e for e in range(shape.n_experts) if e % 2}
+    _, _, y_h, st_h, _ = run_moe_prefill(B, torch, shape, cfg, T, odd)
+    assert np.array_equal(y.view(np.uint16), y_h.view(np.uint16))
+    _, _, y_all, _, _ = run_moe_prefill(B, torch, shape, cfg, T, set(range(shape.n_experts)))
+    assert np.array_equal(y.view(np.uint16), y_all.view(np.uint16))
+
+
+def test_moe_prefill_block_full_size_sampled_tokens(B, torch):
+    """Config-4 shapes (hidden 2048, 128 experts x 768, top-8), 512 tokens: sampled tokens against the oracle, and the
+    single-token decode path on the same tokens (a different kernel family, same contract up to the fp16 edges)."""
+    shape, cfg, T = W.MOE_FULL, 4, 512
+    Bk, x, y, st, (edges, wmode) = run_moe_prefill(B, torch, shape, cfg, T, set())
+    assert np.all(np.isfinite(y.astype(np.float64)))
+    sample = [0, 1, 127, 128, 300, 511]
+    want, _, _, logits = O.moe_block(x[sample], H.oracle_moe_tensors(Bk), shape, edges, wmode)
+    assert O.min_rank_gap(logits, shape.top_k) > 1e-4
+    H.assert_close(y[sample], want, what="moe prefill block, sampled tokens")
+    odd = {e for e in range(shape.n_experts) if e % 2}
+    _, _, y_h, _, _ = run_moe_prefill(B, torch, shape, cfg, T, odd)
+    assert np.array_equal(y.view(np.uint16), y_h.view(np.uint16))
+
+
+@pytest.mark.parametrize("host_experts", [(), (1, 3, 4, 7)])
+def test_moe_layer_with_attention_prefill_matches_oracle(B, torch, host_experts):
+    """A decoder layer whose FFN is the MoE block, over a chunk of tokens: causal attention with cache append, then the
+    routed experts on x1 (fp16 residual stream, as in the dense prefill contract)."""
+    dshape = W.DENSE_SMALL
+    mshape = W.MoEShape(hidden=dshape.hidden, n_experts=8, ffn=64, top_k=2)
+    cfg, cap, pos0, T = 94, 64, 5, 41
+    Lw = W.dense_layer(cfg, 0, dshape)
+    Bk = W.moe_block(cfg, 0, mshape)
+    sl = W.q4_bytes(mshape.ffn, mshape.hidden)
+    attn_bytes = sum(W.q4_bytes(n, k) for r, n, k in dshape.tensor_shapes() if r in (W.ROLE_Q, W.ROLE_K, W.ROLE_V, W.ROLE_O))
+    probe = B.layer_desc(hidden=dshape.hidden, ffn=mshape.ffn, wq=0, n_q_heads=dshape.n_q_heads, n_kv_heads=dshape.n_kv_heads,
+                         head_dim=dshape.head_dim, kv_capacity=cap, n_experts=mshape.n_experts, top_k=mshape.top_k)
+    ws = B.workspace_bytes(probe, T) + MB
+    ctx = B.Context(ws + 6 * (sl + 256) + attn_bytes + 3 * mshape.n_experts * (sl + 256) + MB, workspace_bytes=ws, ring_slots=6,
+                    slot_bytes=sl, chunk_bytes=MB)
+    ids = {"attn_norm": ctx.register_f16(Lw[W.ROLE_ATTN_NORM], 0, W.ROLE_ATTN_NORM)}
+    for r, n in ((W.ROLE_Q, "wq"), (W.ROLE_K, "wk"), (W.ROLE_V, "wv"), (W.ROLE_O, "wo")):
+        ids[n] = ctx.register_q4(*Lw[r], layer=0, role=r)
+    ids["ffn_norm"] = ctx.register_f16(Bk[W.ROLE_FFN_NORM], 0, W.ROLE_FFN_NORM)
+    ids["router"] = ctx.register_f16(Bk[W.ROLE_ROUTER], 0, W.ROLE_ROUTER)
+    for r, n in ((W.ROLE_GATE, "w_gate"), (W.ROLE_UP, "w_up"), (W.ROLE_DOWN, "w_down")):
+        ids[n] = ctx.register_q4(*Bk[r], layer=0, role=r)
+    desc = B.layer_desc(hidden=dshape.hidden, ffn=mshape.ffn, n_q_heads=dshape.n_q_heads, n_kv_heads=dshape.n_kv_heads,
+                        head_dim=dshape.head_dim, kv_capacity=cap, rms_eps=dshape.rms_eps, rope_theta=dshape.rope_theta,
+                        n_experts=mshape.n_experts, top_k=mshape.top_k, **ids)
+    place = [(ids[n], -1, 1) for n in ("wq", "wk", "wv", "wo")]
+    place += [(ids[n], e, 0 if e in host_experts else 1) for n in ("w_gate", "w_up", "w_down") for e in range(mshape.n_experts)]
+    ctx.set_placement(place)
+    kc, vc = W.kv_cache(cfg, 0, dshape.n_kv_heads, cap, dshape.head_dim, pos0)
+    kd, vd = H.to_dev(kc), H.to_dev(vc)
+    edges, wmode = ctx.numerics(B.ATS_MODE_PREFILL)
+    x = W.activations(cfg, 0, (T, dshape.hidden))
+    y = torch.empty((T, dshape.hidden), dtype=torch.float16, device="cuda")
+    ctx.layer_prefill(desc, H.to_dev(x), y, kd, vd, pos0, T)
+    ctx.sync()
+    want, _, _, logits = O.moe_layer(x, H.oracle_dense_tensors(Lw), dshape, H.oracle_moe_tensors(Bk), mshape, kc, vc, pos0, edges, wmode)
+    clear = np.array([O.min_rank_gap(logits[t:t + 1], mshape.top_k) > 1e-4 for t in range(T)])
+    assert clear.sum() >= T - 2
+    H.assert_close(y.cpu().numpy()[clear], want[clear], what="attention + MoE layer, prefill")
+    kg = kd.cpu().numpy()
+    assert np.max(np.abs(kg[:, pos0:pos0 + T].astype(np.float64) - kc[:, pos0:pos0 + T].astype(np.float64))) <= 4e-3 * np.max(np.abs(kc))
+    ctx.close()
