@@ -340,7 +340,8 @@ def extra_moe(torch, B, W, peaks, quick):
     probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, w_gate=0, w_up=0, w_down=0)
     ws = B.workspace_bytes(probe, T) + (1 << 20)
     for hybrid in (False, True):
-        ctx = B.Context(ws + 3 * shape.n_experts * (sl + 256) + 8 * (sl + 256) + (16 << 20), workspace_bytes=ws, ring_slots=8,
+        wsx = ws + (3 * (shape.n_experts // 2) * (sl + 256) + (1 << 20) if hybrid else 0)  # room to stage the selected host experts
+        ctx = B.Context(wsx + 3 * shape.n_experts * (sl + 256) + 8 * (sl + 256) + (16 << 20), workspace_bytes=wsx, ring_slots=8,
                         slot_bytes=sl, chunk_bytes=sl)
         ids = {"ffn_norm": ctx.register_f16(Bk[W.ROLE_FFN_NORM]), "router": ctx.register_f16(Bk[W.ROLE_ROUTER])}
         for name, r in (("w_gate", W.ROLE_GATE), ("w_up", W.ROLE_UP), ("w_down", W.ROLE_DOWN)):
@@ -367,9 +368,10 @@ def extra_moe(torch, B, W, peaks, quick):
                     "expert_gemm_tflops_over_call_time": flop / dt / 1e12,
                     "timing": "wall clock around back-to-back calls (each has one host synchronisation for the routing ids)"}
         if hybrid:
-            # every odd expert that some token selected is read once per 128 of its rows, in place over PCIe
-            out[key]["host_expert_bytes_upper"] = 3 * sl * (shape.n_experts // 2)
-            out[key]["pcie_gbs_lower_bound_if_all_odd_experts_selected"] = 3 * sl * (shape.n_experts // 2) / dt / 1e9
+            # the selected odd experts' slices, gathered into the workspace by the copy kernel (one launch per call)
+            st = ctx.stats()
+            out[key]["host_bytes_moved_per_call"] = st.streamed_bytes / (n + 4)
+            out[key]["pcie_gbs_over_call_time"] = st.streamed_bytes / (n + 4) / dt / 1e9
         ctx.close()
     return out
 

@@ -205,7 +205,15 @@ int32_t ats_layer_decode_host(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/,
                               void* x_out /*HOST*/, void* k_cache /*DEVICE*/, void* v_cache /*DEVICE*/, uint32_t pos,
                               uint32_t M);
 /* Prefill: T tokens of one sequence at cache positions pos0 .. pos0+T-1 (pos0+T <= kv_capacity); projections run as
- * dequantize-fused tensor-core GEMMs.  Same buffers as decode with M = T.  Dense FFN only. */
+ * dequantize-fused tensor-core GEMMs.  Same buffers as decode with M = T.
+ * Layers with routed experts (the MoE prefill of Section 5's workloads): every (token, slot) pair becomes a row, rows
+ * are sorted by expert on the host from the routing ids (one synchronisation per call; T * top_k <= 65536) and each
+ * projection is ONE grouped GEMM launch in which every expert multiplies its own block of rows with its own slice;
+ * y = rn16(x1 + sum_j gate_j d_j) with the expert outputs d_j rounded to fp16 as every GEMM output of the prefill
+ * contract is.  Host-placed experts that some token selected are brought into the part of the workspace that lies beyond
+ * ats_workspace_bytes(desc, T) by one SM-driven copy launch (bulk-async copies from the mapped pinned store, the copy
+ * kernel of Section 4.2.1; counted in ats_stats.streamed_bytes, not in copies) when that part holds them; otherwise the
+ * GEMMs read those slices in place over PCIe, which is several times slower.  Same results either way. */
 int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, const void* x_in /*DEVICE*/,
                           void* x_out /*DEVICE*/, void* k_cache /*DEVICE*/, void* v_cache /*DEVICE*/, uint32_t pos0,
                           uint32_t T);

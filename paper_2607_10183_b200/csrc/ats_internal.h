@@ -44,6 +44,7 @@ struct Tensor {
   // expert-stacked tensors: device array of one address per slice, the resident copy or the slice's place in the pinned
   // host store as the device sees it (mapped memory); null for single-slice tensors
   const uint8_t** slice_tab_dev = nullptr;
+  const uint8_t* host_dev = nullptr;  // the pinned store as the device addresses it (null when it is not mapped)
 };
 
 struct RingSlot {
@@ -84,6 +85,7 @@ struct ats_ctx {
   uint32_t next_slot = 0;
   // pinned scratch for routing ids (host side of the one synchronisation on the MoE path)
   int32_t* ids_host = nullptr;
+  uint8_t* stage_host = nullptr;  // pinned scratch for per-call tables (MoE prefill: slice addresses, copy list)
   cudaEvent_t ids_event = nullptr;
   cudaEvent_t sync_event = nullptr;
   uint32_t fail_copies = 0;
@@ -260,6 +262,17 @@ cudaError_t launch_moe_gather_rows(const __half* h, const int* order, int k, __h
                                    uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_moe_combine_sorted(const __half* res, const float* gates, const __half* d, const int* pos, __half* y, int T, int k,
                                       int H, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
+// SM-driven gather of host-placed slices into device memory (kernels_prefill.cu): chunks of at most 32 KB, src in the
+// mapped pinned store, both addresses and sizes multiples of 16 bytes
+struct CopyChunk {
+  const uint8_t* src;
+  uint8_t* dst;
+  uint32_t bytes;
+  uint32_t pad;
+};
+constexpr uint32_t kCopyChunkBytes = 32 * 1024;
+cudaError_t launch_host_gather(const CopyChunk* list, int n, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch,
+                               int pdl = 0);
 cudaError_t launch_swiglu16(const __half* gu, int ld, int ffn, __half* act, int T, cudaStream_t st, uint64_t* n_launch,
                             int pdl = 0);
 

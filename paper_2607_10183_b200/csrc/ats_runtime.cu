@@ -44,6 +44,7 @@ int32_t check_cuda(ats_ctx* c, cudaError_t e, const char* what) {
   } while (0)
 
 constexpr int kMaxPairs = 65536;  // (token, slot) pairs of one MoE call at most: ids, then the prefill's sort arrays, in ctx->ids_host
+constexpr size_t kStageHostBytes = 1 << 20;  // pinned scratch for per-call tables
 constexpr uint64_t kWsReserved = 1024;  // status word + attention counters at the start of the workspace
 
 // Kernel timing: a pair of events around one launch on the compute stream.
@@ -473,6 +474,7 @@ static int32_t apply_placement(ats_ctx* ctx) {
     t.any_host = false;
     t.contiguous_dev = true;
     t.slice_tab_dev = nullptr;
+    t.host_dev = nullptr;
     if (t.slices.size() > 1) {
       off = align_up(off);
       t.slice_tab_dev = reinterpret_cast<const uint8_t**>(ctx->resident + off);
@@ -504,6 +506,7 @@ static int32_t apply_placement(ats_ctx* ctx) {
       t.slice_tab_dev = nullptr;  // the store is not mapped on this system: the ring path remains
       continue;
     }
+    t.host_dev = static_cast<const uint8_t*>(host_dev);
     std::vector<const uint8_t*> tab(t.slices.size());
     for (size_t e = 0; e < t.slices.size(); ++e)
       tab[e] = t.slices[e].where == ATS_GPU ? t.slices[e].dev : static_cast<const uint8_t*>(host_dev) + e * t.slice_stride;
@@ -709,6 +712,7 @@ int32_t ats_init(const ats_config* cfg, ats_ctx** out) {
   ok &= cudaEventCreateWithFlags(&ctx->sync_event, cudaEventDisableTiming) == cudaSuccess;
   ok &= cudaHostAlloc((void**)&ctx->ids_host, (3 * (size_t)kMaxPairs + 2048) * sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess;
   ok &= cudaHostAlloc((void**)&ctx->host_status, 64, cudaHostAllocDefault) == cudaSuccess;
+  ok &= cudaHostAlloc((void**)&ctx->stage_host, kStageHostBytes, cudaHostAllocDefault) == cudaSuccess;
   if (ws >= kWsReserved) {
     ctx->dev_status = (int*)ctx->ws;
     ok &= cudaMemsetAsync(ctx->ws, 0, kWsReserved, ctx->cs) == cudaSuccess;
@@ -738,6 +742,7 @@ int32_t ats_destroy(ats_ctx* ctx) {
   if (ctx->ids_event) cudaEventDestroy(ctx->ids_event);
   if (ctx->sync_event) cudaEventDestroy(ctx->sync_event);
   if (ctx->ids_host) cudaFreeHost(ctx->ids_host);
+  if (ctx->stage_host) cudaFreeHost(ctx->stage_host);
   if (ctx->host_status) cudaFreeHost(ctx->host_status);
   delete ctx;
   return ATS_OK;
@@ -1338,6 +1343,56 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     ATS_CUDA(launch_moe_gather_rows(w.h2_16, w.order, k, w.xs16, P, H, ctx->cs, nl, pdl));
     const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
     auto slice0 = [](const Tensor& t) -> const uint8_t* { return t.contiguous_dev ? t.slices[0].dev : nullptr; };
+    // Host-placed experts that some token selected: one SM-driven gather brings their slices into what the workspace has
+    // left beyond this layer's buffers, and per-call address tables point the GEMMs there.  Without that room (or
+    // without a mapped store) the GEMMs read the slices in place through the per-tensor tables (slower: 32-byte reads).
+    const uint8_t* const* call_tab[3] = {nullptr, nullptr, nullptr};
+    {
+      const Tensor* ts3[3] = {&tg, &tu, &td};
+      uint64_t need = 0;
+      int n_host = 0;
+      for (const Tensor* t : ts3)
+        if (!t->contiguous_dev && t->host_dev)
+          for (int e = 0; e < E; ++e)
+            if (off_h[e + 1] > off_h[e] && t->slices[e].where != ATS_GPU) {
+              need += t->slice_stride;
+              ++n_host;
+            }
+      const uint64_t tab_bytes = align_up(3ull * E * sizeof(uint8_t*));
+      const uint64_t n_chunks = n_host ? (need + kCopyChunkBytes - 1) / kCopyChunkBytes + n_host : 0;
+      const uint64_t list_bytes = align_up(n_chunks * sizeof(CopyChunk));
+      const uint64_t room = align_up(ctx->cfg.workspace_bytes) - w.total;
+      if (n_host && tab_bytes + list_bytes + need <= room && tab_bytes + list_bytes <= kStageHostBytes) {
+        uint8_t* dev_tab = ctx->ws + w.total;
+        uint8_t* dev_list = dev_tab + tab_bytes;
+        uint8_t* stage = dev_list + list_bytes;
+        const uint8_t** tab_h = reinterpret_cast<const uint8_t**>(ctx->stage_host);
+        CopyChunk* list_h = reinterpret_cast<CopyChunk*>(ctx->stage_host + tab_bytes);
+        int nc = 0;
+        uint64_t so = 0;
+        for (int i = 0; i < 3; ++i) {
+          const Tensor* t = ts3[i];
+          for (int e = 0; e < E; ++e) {
+            const Slice& sl = t->slices[e];
+            if (sl.where == ATS_GPU) {
+              tab_h[i * E + e] = sl.dev;
+            } else if (off_h[e + 1] > off_h[e] && t->host_dev) {
+              tab_h[i * E + e] = stage + so;
+              const uint8_t* src = t->host_dev + (uint64_t)e * t->slice_stride;
+              for (uint64_t o = 0; o < t->slice_stride; o += kCopyChunkBytes)
+                list_h[nc++] = CopyChunk{src + o, stage + so + o, (uint32_t)std::min<uint64_t>(kCopyChunkBytes, t->slice_stride - o), 0};
+              so += t->slice_stride;
+            } else {
+              tab_h[i * E + e] = t->host_dev ? t->host_dev + (uint64_t)e * t->slice_stride : nullptr;  // no rows: never read
+            }
+          }
+        }
+        ATS_CUDA(cudaMemcpyAsync(dev_tab, ctx->stage_host, tab_bytes + (size_t)nc * sizeof(CopyChunk), cudaMemcpyHostToDevice, ctx->cs));
+        ATS_CUDA(launch_host_gather(reinterpret_cast<const CopyChunk*>(dev_list), nc, ctx->dev_status, ctx->sm_count, ctx->cs, nl, pdl));
+        for (int i = 0; i < 3; ++i) call_tab[i] = reinterpret_cast<const uint8_t* const*>(dev_tab) + (size_t)i * E;
+        ctx->stats.streamed_bytes += need;
+      }
+    }
     std::string err;
     GemmParams m{};
     m.T = P;
@@ -1352,14 +1407,8 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     m.seg[0] = GemvSeg{slice0(tg), F};
     m.seg[1] = GemvSeg{slice0(tu), F};
     m.grp_stride = tg.slice_stride;
-    m.grp_tab[0] = tg.contiguous_dev ? nullptr : tg.slice_tab_dev;
-    m.grp_tab[1] = tu.contiguous_dev ? nullptr : tu.slice_tab_dev;
-    if ((tg.contiguous_dev != tu.contiguous_dev) && (!tg.slice_tab_dev || !tu.slice_tab_dev))
-      return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE prefill: gate and up need the same kind of placement or mapped slice tables");
-    if (tg.contiguous_dev != tu.contiguous_dev) {  // mixed: use the tables for both
-      m.grp_tab[0] = tg.slice_tab_dev;
-      m.grp_tab[1] = tu.slice_tab_dev;
-    }
+    m.grp_tab[0] = call_tab[0] ? call_tab[0] : tg.contiguous_dev ? nullptr : tg.slice_tab_dev;
+    m.grp_tab[1] = call_tab[1] ? call_tab[1] : tu.contiguous_dev ? nullptr : tu.slice_tab_dev;
     m.x = w.xs16;
     m.ldx = H;
     m.y = w.gu16;
@@ -1371,7 +1420,7 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     m.K = F;
     m.seg[0] = GemvSeg{slice0(td), H};
     m.grp_stride = td.slice_stride;
-    m.grp_tab[0] = td.contiguous_dev ? nullptr : td.slice_tab_dev;
+    m.grp_tab[0] = call_tab[2] ? call_tab[2] : td.contiguous_dev ? nullptr : td.slice_tab_dev;
     m.grp_tab[1] = nullptr;
     m.x = w.act16;
     m.ldx = F;

@@ -392,4 +392,77 @@ cudaError_t launch_moe_combine_sorted(const __half* res, const float* gates, con
   return launch_dep(moe_combine_sorted_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, res, gates, d, pos, y, n8, k, H);
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Copy kernel for host-placed expert slices (the SM-driven transfer path of Sections 4.1 / 4.2.1): every chunk of the
+// list is pulled from the mapped pinned store into shared memory with a bulk-async copy and pushed to its place in
+// device memory with another; one thread per CTA keeps four chunks in flight.  One launch moves all the slices a call
+// needs, so the per-copy cost of the DMA path (about a third of the time of a sub-megabyte copy) is not paid.
+namespace {
+constexpr int kCopyStages = 4;
+constexpr int kCopyChunk = 32 * 1024;
+__device__ __forceinline__ uint32_t cp_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool cp_mbar_wait(uint64_t* bar, uint32_t parity) {
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 64; ++i) {
+      uint32_t ok;
+      asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                   : "=r"(ok) : "r"(cp_smem_u32(bar)), "r"(parity) : "memory");
+      if (ok) return true;
+    }
+    if (clock64() - t0 > 4000000000ll) return false;  // about two seconds: the source is across PCIe
+  }
+}
+}  // namespace
+
+__global__ void __launch_bounds__(32, 1) host_gather_kernel(const CopyChunk* __restrict__ list, int n, int* status) {
+  extern __shared__ __align__(128) uint8_t cp_s[];
+  __shared__ uint64_t full[kCopyStages];
+  if (threadIdx.x != 0) return;
+  for (int s = 0; s < kCopyStages; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(cp_smem_u32(&full[s])));
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the list was written by a copy that precedes this launch
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int first = blockIdx.x, gx = gridDim.x;
+  const int n_my = first < n ? (n - first + gx - 1) / gx : 0;
+  auto issue_load = [&](int j) {
+    const int s = j % kCopyStages;
+    const CopyChunk c = list[first + j * gx];
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(cp_smem_u32(&full[s])), "r"(c.bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     cp_smem_u32(cp_s + (size_t)s * kCopyChunk)),
+                 "l"(c.src), "r"(c.bytes), "r"(cp_smem_u32(&full[s]))
+                 : "memory");
+  };
+  for (int j = 0; j < min(kCopyStages, n_my); ++j) issue_load(j);
+  for (int j = 0; j < n_my; ++j) {
+    const int s = j % kCopyStages;
+    if (!cp_mbar_wait(&full[s], (uint32_t)(j / kCopyStages) & 1u)) {
+      atomicExch(status, 5);
+      break;
+    }
+    const CopyChunk c = list[first + j * gx];
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(c.dst), "r"(cp_smem_u32(cp_s + (size_t)s * kCopyChunk)),
+                 "r"(c.bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    if (j + kCopyStages < n_my) {
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the store has read stage s: it may be refilled
+      issue_load(j + kCopyStages);
+    }
+  }
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+cudaError_t launch_host_gather(const CopyChunk* list, int n, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch, int pdl) {
+  if (n <= 0) return cudaSuccess;
+  static uint64_t attr_done = 0;
+  if (first_use_on_device(&attr_done)) {
+    cudaError_t e = cudaFuncSetAttribute(host_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCopyStages * kCopyChunk);
+    if (e != cudaSuccess) return e;
+  }
+  ++*n_launch;
+  return launch_dep(host_gather_kernel, dim3(std::min(n, sm_count)), dim3(32), (size_t)kCopyStages * kCopyChunk, st, pdl, 1, list, n, status);
+}
+
 }  // namespace ats

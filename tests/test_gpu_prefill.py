@@ -267,12 +267,12 @@ def test_prefill_layer_stage_by_stage_full_size(B, torch):
 
 
 # ------------------------------------------------------------------------------------------------- MoE prefill
-def run_moe_prefill(B, torch, shape, cfg, T, host_experts):
+def run_moe_prefill(B, torch, shape, cfg, T, host_experts, extra_ws=0):
     """The routed FFN block over T tokens in one ats_layer_prefill call (no attention)."""
     Bk = W.moe_block(cfg, 0, shape)
     sl = W.q4_bytes(shape.ffn, shape.hidden)
     probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, w_gate=0, w_up=0, w_down=0)
-    ws = B.workspace_bytes(probe, T) + MB
+    ws = B.workspace_bytes(probe, T) + MB + extra_ws  # room beyond the layer's buffers: where selected host experts are staged
     ctx = B.Context(ws + 8 * (sl + 256) + 3 * shape.n_experts * (sl + 256) + MB, workspace_bytes=ws, ring_slots=8, slot_bytes=sl,
                     chunk_bytes=MB)
     desc, ids = H.register_moe_block(ctx, Bk)
@@ -319,8 +319,12 @@ def test_moe_prefill_block_full_size_sampled_tokens(B, torch):
     assert O.min_rank_gap(logits, shape.top_k) > 1e-4
     H.assert_close(y[sample], want, what="moe prefill block, sampled tokens")
     odd = {e for e in range(shape.n_experts) if e % 2}
-    _, _, y_h, _, _ = run_moe_prefill(B, torch, shape, cfg, T, odd)
-    assert np.array_equal(y.view(np.uint16), y_h.view(np.uint16))
+    _, _, y_h, st_h, _ = run_moe_prefill(B, torch, shape, cfg, T, odd)  # no room to stage: slices read in place
+    assert np.array_equal(y.view(np.uint16), y_h.view(np.uint16)) and st_h.streamed_bytes == 0
+    sl = W.q4_bytes(shape.ffn, shape.hidden)
+    _, _, y_s, st_s, _ = run_moe_prefill(B, torch, shape, cfg, T, odd, extra_ws=3 * (shape.n_experts // 2) * (sl + 256) + MB)
+    assert np.array_equal(y.view(np.uint16), y_s.view(np.uint16))  # staged by the copy kernel
+    assert 0 < st_s.streamed_bytes <= 3 * (shape.n_experts // 2) * (sl + 256) and st_s.copies == 0
 
 
 @pytest.mark.parametrize("host_experts", [(), (1, 3, 4, 7)])
