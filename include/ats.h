@@ -66,7 +66,10 @@ enum {
                                      space), picking each slice's address from a per-tensor table on the device by the
                                      expert id (the zero-copy path of Sections 4.1 / 4.2.1).  Same arithmetic, same results;
                                      ats_stats.streamed_bytes / copies / host_syncs do not count these reads.  Calls with
-                                     more than one token keep the ring path (it moves every distinct expert once). */
+                                     more than one token: the distinct selected host-placed experts are gathered into the
+                                     part of the workspace beyond the call's own buffers by one launch of an SM-driven copy
+                                     kernel (each slice crosses PCIe once; counted in streamed_bytes, not in copies) when that
+                                     part holds them; otherwise they keep the ring path. */
   /* timing experiments only: do not launch a stage of ats_layer_decode (its outputs are then stale); bit 24 = QKV GEMV,
    * 25 = attention, 26 = O GEMV, 27 = gate/up GEMV, 28 = down GEMV */
   ATS_FLAG_DEBUG_SKIP_SHIFT = 24

@@ -536,7 +536,7 @@ static cudaError_t launch_moe_gemv_any(ats_ctx* ctx, const MoeGemvParams& p, con
 }
 
 static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_dev, const int32_t* ids_host,
-                             MoeGemvParams p) {
+                             MoeGemvParams p, const uint8_t* const* call_tab0 = nullptr, const uint8_t* const* call_tab1 = nullptr) {
   const Tensor& t0 = ctx->tensors[id0];
   const Tensor* t1 = id1 >= 0 ? &ctx->tensors[id1] : nullptr;
   p.n_rows = (int)t0.d.n_out;
@@ -544,7 +544,10 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
   p.stride = t0.slice_stride;
   p.ids = ids_dev;
   if (!ids_host) {
-    if (t0.contiguous_dev && (!t1 || t1->contiguous_dev)) {
+    if (call_tab0) {  // per-call tables: resident copies, or slices the copy kernel has gathered into the workspace
+      p.tab0 = call_tab0;
+      p.tab1 = call_tab1;
+    } else if (t0.contiguous_dev && (!t1 || t1->contiguous_dev)) {
       p.base0 = t0.slices[0].dev;
       p.base1 = t1 ? t1->slices[0].dev : nullptr;
     } else {  // device-initiated gather: addresses from the per-tensor tables
@@ -1190,12 +1193,72 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     if (moe_gemv_stream_eligible(probe1) && moe_gemv_stream_eligible(probe2)) implicit = true;
   }
   const int32_t* ids_host = nullptr;
+  const uint8_t* const* call_tab[3] = {nullptr, nullptr, nullptr};
   if (!implicit) {
     ATS_TRY(fetch_ids(ctx, w.ids, P, E));
     ids_host = ctx->ids_host;
-    const int tids[3] = {L->w_gate, L->w_up, L->w_down};
-    plan_moe(ctx, ids_host, P, tids, 2, 3);
-    ATS_TRY(pump(ctx));
+    // Several tokens under ATS_FLAG_MOE_DEVICE_GATHER: the distinct selected host-placed experts are gathered into the
+    // workspace beyond this call's buffers by one launch of the copy kernel (every slice crosses PCIe once, no per-copy
+    // cost), when that room exists and the streaming kernel takes the shapes; the stages then run as one launch each
+    // over per-call address tables.  Otherwise: the staging ring.
+    bool staged = false;
+    if ((ctx->cfg.flags & ATS_FLAG_MOE_DEVICE_GATHER) && tg.host_dev && tu.host_dev && td.host_dev) {
+      MoeGemvParams probe1{}, probe2{};
+      probe1.K = H; probe1.n_rows = (int)L->ffn; probe1.mode = GEMV_SWIGLU_F16;
+      probe2.K = (int)L->ffn; probe2.n_rows = H; probe2.mode = GEMV_OUT_F32;
+      const Tensor* ts3[3] = {&tg, &tu, &td};
+      std::vector<uint8_t> sel(E, 0);
+      for (int pr = 0; pr < P; ++pr) sel[ids_host[pr]] = 1;
+      uint64_t need = 0;
+      int n_host = 0;
+      for (const Tensor* t : ts3)
+        for (int e = 0; e < E; ++e)
+          if (sel[e] && t->slices[e].where != ATS_GPU) {
+            need += t->slice_stride;
+            ++n_host;
+          }
+      const uint64_t tab_bytes = align_up(3ull * E * sizeof(uint8_t*));
+      const uint64_t list_bytes = align_up(((need + kCopyChunkBytes - 1) / kCopyChunkBytes + n_host) * sizeof(CopyChunk));
+      const uint64_t room = align_up(ctx->cfg.workspace_bytes) - w.total;
+      if (moe_gemv_stream_eligible(probe1) && moe_gemv_stream_eligible(probe2) && tab_bytes + list_bytes + need <= room &&
+          tab_bytes + list_bytes <= kStageHostBytes) {
+        uint8_t* dev_tab = ctx->ws + w.total;
+        uint8_t* dev_list = dev_tab + tab_bytes;
+        uint8_t* stage = dev_list + list_bytes;
+        const uint8_t** tab_h = reinterpret_cast<const uint8_t**>(ctx->stage_host);
+        CopyChunk* list_h = reinterpret_cast<CopyChunk*>(ctx->stage_host + tab_bytes);
+        int nc = 0;
+        uint64_t so = 0;
+        for (int i = 0; i < 3; ++i) {
+          const Tensor* t = ts3[i];
+          for (int e = 0; e < E; ++e) {
+            const Slice& sl = t->slices[e];
+            if (sl.where == ATS_GPU) {
+              tab_h[i * E + e] = sl.dev;
+            } else if (sel[e]) {
+              tab_h[i * E + e] = stage + so;
+              const uint8_t* src = t->host_dev + (uint64_t)e * t->slice_stride;
+              for (uint64_t o = 0; o < t->slice_stride; o += kCopyChunkBytes)
+                list_h[nc++] = CopyChunk{src + o, stage + so + o, (uint32_t)std::min<uint64_t>(kCopyChunkBytes, t->slice_stride - o), 0};
+              so += t->slice_stride;
+            } else {
+              tab_h[i * E + e] = t->host_dev + (uint64_t)e * t->slice_stride;  // not selected: never read
+            }
+          }
+        }
+        ATS_CUDA(cudaMemcpyAsync(dev_tab, ctx->stage_host, tab_bytes + (size_t)nc * sizeof(CopyChunk), cudaMemcpyHostToDevice, ctx->cs));
+        ATS_CUDA(launch_host_gather(reinterpret_cast<const CopyChunk*>(dev_list), nc, ctx->dev_status, ctx->sm_count, ctx->cs, nl, pdl));
+        for (int i = 0; i < 3; ++i) call_tab[i] = reinterpret_cast<const uint8_t* const*>(dev_tab) + (size_t)i * E;
+        ctx->stats.streamed_bytes += need;
+        staged = true;
+        ids_host = nullptr;  // the stages take the ids on the device
+      }
+    }
+    if (!staged) {
+      const int tids[3] = {L->w_gate, L->w_up, L->w_down};
+      plan_moe(ctx, ids_host, P, tids, 2, 3);
+      ATS_TRY(pump(ctx));
+    }
   }
   MoeGemvParams s1{};
   s1.P = P;
@@ -1205,7 +1268,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   s1.y16 = w.act16;
   s1.ldy = (int)L->ffn;
   s1.mode = GEMV_SWIGLU_F16;
-  ATS_TRY(run_moe_stage(ctx, L->w_gate, L->w_up, w.ids, ids_host, s1));
+  ATS_TRY(run_moe_stage(ctx, L->w_gate, L->w_up, w.ids, ids_host, s1, call_tab[0], call_tab[1]));
   MoeGemvParams s2{};
   s2.P = P;
   s2.x_div = 1;
@@ -1214,7 +1277,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   s2.y32 = w.d32;
   s2.ldy = H;
   s2.mode = GEMV_OUT_F32;
-  ATS_TRY(run_moe_stage(ctx, L->w_down, -1, w.ids, ids_host, s2));
+  ATS_TRY(run_moe_stage(ctx, L->w_down, -1, w.ids, ids_host, s2, call_tab[2], nullptr));
   ATS_CUDA(launch_moe_combine(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, w.gates, w.d32, (__half*)x_out, (int)M, k, H,
                               ctx->cs, nl, pdl));
   return ATS_OK;

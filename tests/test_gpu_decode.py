@@ -311,10 +311,9 @@ def test_route_topk_bit_exact_with_ties(B, torch):
     ctx.close()
 
 
-def run_moe(B, torch, shape, cfg, M, host_experts, ring_slots=8, chunk=MB, flags=0):
+def run_moe(B, torch, shape, cfg, M, host_experts, ring_slots=8, chunk=MB, flags=0, ws=4 * MB):
     Bk = W.moe_block(cfg, 0, shape)
     sl = W.q4_bytes(shape.ffn, shape.hidden)
-    ws = 4 * MB
     ctx = make_ctx(B, 3 * shape.n_experts * (sl + 256) + MB, ws=ws, ring_slots=ring_slots, slot_bytes=sl, chunk_bytes=chunk, flags=flags)
     desc, ids = H.register_moe_block(ctx, Bk)
     ent = []
@@ -373,8 +372,14 @@ def test_moe_device_gather_equals_resident_without_host_round_trip(B, torch, M):
     if M == 1:  # the gather path: nothing through the ring, no ids on the host
         assert st.host_syncs == 0 and st.streamed_bytes == 0 and st.copies == 0
         assert st_all.host_syncs == 0 and st_all.streamed_bytes == 0
-    else:       # several tokens keep the ring path (every distinct expert moves once)
-        assert st.host_syncs == 1 and st.streamed_bytes > 0
+    else:       # several tokens, no room in the workspace: the ring path (every distinct expert moves once)
+        assert st.host_syncs == 1 and st.streamed_bytes > 0 and st.copies > 0
+        # with room beyond the call's buffers the copy kernel gathers the distinct selected experts in one launch
+        sl = W.q4_bytes(shape.ffn, shape.hidden)
+        _, _, y_st, st_st = run_moe(B, torch, shape, cfg, M, odd, flags=B.ATS_FLAG_MOE_DEVICE_GATHER, ws=4 * MB + 3 * 64 * (sl + 256))
+        assert np.array_equal(y_res.view(np.uint16), y_st.view(np.uint16))
+        # same distinct experts as the ring run moved (slices of this shape need no padding), no DMA copies
+        assert st_st.host_syncs == 1 and st_st.copies == 0 and st_st.streamed_bytes == st.streamed_bytes
 
 
 @pytest.mark.parametrize("host_experts", [(), (1, 3, 4, 7)])
