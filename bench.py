@@ -490,8 +490,89 @@ def extra_model_loop(torch, B, W, peaks, quick):
             "decode_frac_of_measured_hbm": weight_bytes / (dec_ms / gen * 1e-3) / 1e9 / peaks["hbm_gbs"], "logits_finite": finite}
 
 
+def extra_model_loop_moe(torch, B, W, peaks, quick):
+    """Whole-model loop on an MoE layer shape (hidden 2048, 32 query / 4 kv heads of 128, 128 experts x SwiGLU 768, top-8):
+    a stack of attention + routed-expert layers; a 512-token prompt prefilled in one chunk, then decode steps through every
+    layer.  Once with everything resident, once with the odd experts of every layer in pinned host memory (read in place by
+    the single-token decode kernels, gathered by the copy kernel for the prefill chunk)."""
+    mshape = W.MOE_FULL
+    Hd, nq, nkv, hd = mshape.hidden, 32, 4, 128
+    L = 2 if quick else 4
+    prompt, gen = (128 if quick else 512), (8 if quick else 32)
+    cap = prompt + gen
+    sl = W.q4_bytes(mshape.ffn, Hd)
+    attn_shapes = ((W.ROLE_Q, "wq", nq * hd, Hd), (W.ROLE_K, "wk", nkv * hd, Hd), (W.ROLE_V, "wv", nkv * hd, Hd), (W.ROLE_O, "wo", Hd, nq * hd))
+    attn_bytes = sum(W.q4_bytes(n, k) for _, _, n, k in attn_shapes)
+    probe = B.layer_desc(hidden=Hd, ffn=mshape.ffn, wq=0, n_q_heads=nq, n_kv_heads=nkv, head_dim=hd, kv_capacity=cap,
+                         n_experts=mshape.n_experts, top_k=mshape.top_k)
+    blocks = [W.moe_block(4, i, mshape) for i in range(2)]  # two distinct expert sets, registered L times
+    out = {"workload": f"{L} layers of attention + MoE FFN ({mshape.n_experts} experts, top-{mshape.top_k}): prompt {prompt} in one chunk, "
+                       f"then {gen} decode steps", "layers": L, "expert_bytes_per_layer": 3 * mshape.n_experts * sl}
+    for hybrid in (False, True):
+        stage = 3 * (mshape.n_experts // 2) * (sl + 256) + (1 << 20) if hybrid else 0
+        ws = max(B.workspace_bytes(probe, prompt), B.workspace_bytes(probe, 1)) + (1 << 20) + stage
+        arena = ws + 8 * (sl + 256) + L * (attn_bytes + 3 * mshape.n_experts * (sl + 256) + (1 << 20)) + (4 << 20)
+        ctx = B.Context(arena, workspace_bytes=ws, ring_slots=8, slot_bytes=sl, chunk_bytes=sl,
+                        flags=B.ATS_FLAG_MOE_DEVICE_GATHER if hybrid else 0)
+        descs, place = [], []
+        damp = np.float16(0.1)
+        for l in range(L):
+            Bk = blocks[l % 2]
+            ids = {"attn_norm": ctx.register_f16(Bk[W.ROLE_FFN_NORM] * damp, l, W.ROLE_ATTN_NORM)}
+            for r, name, n, k in attn_shapes:
+                ids[name] = ctx.register_q4(*W.q4_packed(7, l % 2, r, n, k), layer=l, role=r)
+                place.append((ids[name], -1, B.ATS_GPU))
+            ids["ffn_norm"] = ctx.register_f16(Bk[W.ROLE_FFN_NORM] * damp, l, W.ROLE_FFN_NORM)
+            ids["router"] = ctx.register_f16(Bk[W.ROLE_ROUTER], l, W.ROLE_ROUTER)
+            for r, name in ((W.ROLE_GATE, "w_gate"), (W.ROLE_UP, "w_up"), (W.ROLE_DOWN, "w_down")):
+                ids[name] = ctx.register_q4(*Bk[r], layer=l, role=r)
+                place += [(ids[name], e, B.ATS_HOST if (hybrid and e % 2) else B.ATS_GPU) for e in range(mshape.n_experts)]
+            descs.append(B.layer_desc(hidden=Hd, ffn=mshape.ffn, n_q_heads=nq, n_kv_heads=nkv, head_dim=hd, kv_capacity=cap,
+                                      rms_eps=mshape.rms_eps, rope_theta=10000.0, n_experts=mshape.n_experts, top_k=mshape.top_k, **ids))
+        ctx.set_placement(place)
+        caches = [(torch.zeros((nkv, cap, hd), dtype=torch.float16, device="cuda"), torch.zeros((nkv, cap, hd), dtype=torch.float16, device="cuda"))
+                  for _ in range(L)]
+        x0 = torch.from_numpy(W.activations(7, 0, (prompt, Hd)) * 0.25).cuda()
+        pa, pb = torch.empty_like(x0), torch.empty_like(x0)
+        d0 = torch.from_numpy(W.activations(7, 1, (1, Hd)) * 0.25).cuda()
+        da, db = torch.empty_like(d0), torch.empty_like(d0)
+
+        def prefill():
+            src, dst = x0, pa
+            for l in range(L):
+                ctx.layer_prefill(descs[l], src, dst, caches[l][0], caches[l][1], 0, prompt)
+                src, dst = dst, (pb if dst is pa else pa)
+            return src
+
+        def decode(n):
+            for s in range(n):
+                src, dst = d0, da
+                for l in range(L):
+                    ctx.layer_decode(descs[l], src, dst, caches[l][0], caches[l][1], prompt + s, 1)
+                    src, dst = dst, (db if dst is da else da)
+            return src
+        prefill()
+        decode(2)
+        ctx.sync()
+        ctx.reset_stats()
+        t0 = time.perf_counter()
+        last = prefill()
+        ctx.sync()
+        pre_s = time.perf_counter() - t0
+        st = ctx.stats()
+        dec_ms = event_time_ms(torch, ctx.compute, lambda: decode(gen))
+        finite = bool(torch.isfinite(last.float()).all().item()) and bool(torch.isfinite(da.float()).all().item())
+        key = "hybrid_odd_experts_on_host" if hybrid else "resident"
+        out[key] = {"prefill_ms": pre_s * 1e3, "prefill_tokens_per_s": prompt / pre_s, "prefill_host_bytes_moved": float(st.streamed_bytes),
+                    "prefill_pcie_gbs_over_wall_time": st.streamed_bytes / pre_s / 1e9,
+                    "decode_ms_per_token": dec_ms / gen, "decode_tokens_per_s": gen / (dec_ms * 1e-3), "outputs_finite": finite,
+                    "timing": "prefill: wall clock (one host synchronisation per layer for the routing ids); decode: CUDA events"}
+        ctx.close()
+    return out
+
+
 STACK_LAYERS = [0]
-EXTRAS = {"model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
+EXTRAS = {"model_loop_moe": extra_model_loop_moe, "model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
 
 
 def run_ours(args):
@@ -637,7 +718,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the figures of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--quick", action="store_true", help="smaller extras")
-    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop"],
+    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe"],
                     help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
     ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = 8, or 4 with --quick; 32 = the full configuration)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")
