@@ -104,6 +104,50 @@ def test_linear_gemv_matches_oracle(B, torch, N, K, M):
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))  # placement never changes the math
 
 
+def test_streaming_gemv_activation_extremes(B, torch):
+    """The single-token kernel carries each 32-element activation block as 16-bit fixed point scaled by the block's largest
+    exponent.  Blocks that stress that form: all zeros, fp16 subnormals only, one element at the top of the fp16 range
+    among tiny ones (the tiny ones fall below the block's resolution: their contribution is below the gate by
+    construction), alternating signs at full scale, and a one-hot (which must return the weight column exactly)."""
+    N, K = 512, 2048  # a shape the streaming kernel takes (K a multiple of 256, rows a multiple of 16)
+    packed, scales = W.q4_packed(95, 0, W.ROLE_Q, N, K)
+    scales = (scales.astype(np.float32) * 1e-3).astype(np.float16)  # keeps the full-scale cases inside fp16 on output
+    rng = np.random.default_rng(11)
+    cases = {}
+    cases["zeros"] = np.zeros(K, dtype=np.float16)
+    cases["subnormal"] = (rng.integers(-1023, 1024, size=K).astype(np.float64) * 2.0 ** -24).astype(np.float16)
+    x = (rng.standard_normal(K) * 1e-4).astype(np.float16)
+    x[::32] = np.float16(60000.0) * np.where(rng.random(K // 32) < 0.5, -1, 1).astype(np.float16)
+    cases["outlier_per_block"] = x
+    cases["full_scale_alternating"] = (np.float16(65504.0) * np.where(np.arange(K) % 2, -1, 1)).astype(np.float16)
+    x = np.zeros(K, dtype=np.float16)
+    x[777] = np.float16(1.0)
+    cases["one_hot"] = x
+    x = rng.standard_normal(K).astype(np.float16)
+    x[rng.random(K) < 0.5] = 0  # half the elements exactly zero, some blocks mostly empty
+    cases["sparse"] = x
+    ctx = make_ctx(B, W.q4_bytes(N, K))
+    tid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(tid, -1, B.ATS_GPU)])
+    for name, xv in cases.items():
+        y = torch.full((1, N), 7.0, dtype=torch.float16, device="cuda")
+        ctx.linear(tid, H.to_dev(xv[None, :]), y, 1)
+        ctx.sync()
+        got = y.cpu().numpy()
+        want = O.linear(xv[None, :].astype(np.float64), packed, scales, round_out=True)
+        assert np.all(np.isfinite(want.astype(np.float64))), name
+        if name == "zeros":
+            assert np.all(got == 0), name
+        elif name == "one_hot":
+            assert np.array_equal(got.view(np.uint16), np.asarray(want, dtype=np.float16).view(np.uint16)), name
+        elif name == "subnormal":
+            # outputs are far below fp16's normal range: compare absolutely, at the resolution of the fp16 output
+            assert np.max(np.abs(got.astype(np.float64) - want.astype(np.float64))) <= 2.0 ** -24, name
+        else:
+            H.assert_close(got, want, what=f"gemv, activations: {name}")
+    ctx.close()
+
+
 def test_linear_closed_forms_on_gpu(B, torch):
     """One-hot activations return a weight column exactly; all-ones with unit scales return integer row sums."""
     N, K = 40, 256
