@@ -246,6 +246,9 @@ size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx);
 cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch);
 cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
                                float* gates, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
+cudaError_t launch_router_topk_norm(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
+                                    float* gates, const void* norm_x, int norm_x_f32, const __half* norm_gain, float eps,
+                                    cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 // y16[m] = rn16(res[m] + sum_j gates[m][j] * d32[m*k + j])   (res fp16 or fp32)
 cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gates, const float* d32, __half* y16,
                                int M, int k, int H, cudaStream_t st, uint64_t* n_launch, int pdl = 0);

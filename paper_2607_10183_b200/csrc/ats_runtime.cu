@@ -1141,9 +1141,6 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     o.mode = GEMV_RES16_OUT_F32;
     if (!(skip & 4)) ATS_TRY(run_gemv_group(ctx, &wo, 1, o));
   }
-  if (L->n_experts != 0)  // the MoE path needs the normalised row in memory (router and grouped GEMV read it)
-    ATS_CUDA(launch_rmsnorm(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev,
-                            w.h2_16, (int)M, H, L->rms_eps, ctx->cs, nl, pdl));
   if (L->n_experts == 0) {
     GemvParams g{};
     g.M = (int)M;
@@ -1178,8 +1175,10 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   }
   // ---- MoE FFN
   const int k = (int)L->top_k, P = (int)M * k, E = (int)L->n_experts;
-  ATS_CUDA(launch_router_topk(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)M, H, E, k,
-                              (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, ctx->cs, nl, pdl));
+  // the FFN norm runs inside the router launch; the normalised rows land in h2_16 for the expert kernels
+  ATS_CUDA(launch_router_topk_norm(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)M, H, E, k,
+                                   (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, attn ? (const void*)w.x1_32 : x_in,
+                                   attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, L->rms_eps, ctx->cs, nl, pdl));
   const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
   bool implicit = tg.contiguous_dev && tu.contiguous_dev && td.contiguous_dev;
   if (!implicit && M == 1 && (ctx->cfg.flags & ATS_FLAG_MOE_DEVICE_GATHER) && tg.slice_tab_dev && tu.slice_tab_dev && td.slice_tab_dev) {

@@ -642,10 +642,15 @@ __device__ __forceinline__ void st_cluster_f32(const float* local_smem_ptr, uint
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
 }
 
+// Optional RMSNorm prologue (gain != null): the token's row is xn (fp16 or fp32), every CTA of the cluster sums its
+// squares itself (the whole row is a few kilobytes), normalises its own eighth, h = rn16(x * g / sqrt(mean(x^2) + eps)),
+// uses it and writes it to h_out for the expert kernels that follow.
 __global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(const __half* __restrict__ h,
                                                                                const __half* __restrict__ wr, int H, int E, int Epad,
                                                                                int k, int renorm, int32_t* __restrict__ ids,
-                                                                               float* __restrict__ gates) {
+                                                                               float* __restrict__ gates, const void* __restrict__ xn,
+                                                                               int xn_f32, const __half* __restrict__ gain, float eps,
+                                                                               __half* __restrict__ h_out) {
   extern __shared__ __align__(16) float smem[];
   const int Hc = H / kRouterCluster;          // rows of this CTA
   const int L = E / 8;                        // threads per row
@@ -659,7 +664,31 @@ __global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(c
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t rank = cluster_ctarank();
   const int row0 = (int)rank * Hc;
-  for (int i = threadIdx.x; i < Hc; i += kRouterClThreads) h_s[i] = __half2float(h[(size_t)m * H + row0 + i]);
+  if (gain) {
+    __shared__ float red[kRouterClThreads / 32];
+    const __half* x16 = static_cast<const __half*>(xn) + (size_t)m * H;
+    const float* x32 = static_cast<const float*>(xn) + (size_t)m * H;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < H; i += kRouterClThreads) {
+      const float v = xn_f32 ? x32[i] : __half2float(x16[i]);
+      ss = fmaf(v, v, ss);
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kRouterClThreads / 32; ++w) t += red[w];
+    const float inv = 1.0f / sqrtf(t / (float)H + eps);
+    for (int i = threadIdx.x; i < Hc; i += kRouterClThreads) {
+      const float v = xn_f32 ? x32[row0 + i] : __half2float(x16[row0 + i]);
+      const __half hv = __float2half_rn(v * __half2float(gain[row0 + i]) * inv);
+      h_s[i] = __half2float(hv);
+      h_out[(size_t)m * H + row0 + i] = hv;
+    }
+  } else {
+    for (int i = threadIdx.x; i < Hc; i += kRouterClThreads) h_s[i] = __half2float(h[(size_t)m * H + row0 + i]);
+  }
   __syncthreads();
   const int grp = threadIdx.x / L, e0 = (threadIdx.x % L) * 8;
   float acc[8];
@@ -703,6 +732,14 @@ __global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(c
 
 cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
                                float* gates, cudaStream_t st, uint64_t* n_launch, int pdl) {
+  return launch_router_topk_norm(h, wr, M, H, E, k, renorm, ids, gates, nullptr, 0, nullptr, 0.f, st, n_launch, pdl);
+}
+
+// With norm_gain: h = RMSNorm(norm_x; norm_gain) is computed first and written to h (which the kernels after the router
+// read); one launch where the cluster kernel takes the shape, else the stand-alone norm and then the router.
+cudaError_t launch_router_topk_norm(const __half* h, const __half* wr, int M, int H, int E, int k, int renorm, int32_t* ids,
+                                    float* gates, const void* norm_x, int norm_x_f32, const __half* norm_gain, float eps,
+                                    cudaStream_t st, uint64_t* n_launch, int pdl) {
   int Epad = 32;
   while (Epad < E) Epad <<= 1;
   if (E % 8 == 0 && H % (8 * kRouterCluster) == 0 && (((uintptr_t)wr | (uintptr_t)h) & 15) == 0) {
@@ -715,8 +752,12 @@ cudaError_t launch_router_topk(const __half* h, const __half* wr, int M, int H, 
       }
       ++*n_launch;
       return launch_dep(router_topk_cluster_kernel, dim3(kRouterCluster, M), dim3(kRouterClThreads), smem_cl, st, pdl, kRouterCluster,
-                        h, wr, H, E, Epad, k, renorm, ids, gates);
+                        h, wr, H, E, Epad, k, renorm, ids, gates, norm_x, norm_x_f32, norm_gain, eps, const_cast<__half*>(h));
     }
+  }
+  if (norm_gain) {
+    cudaError_t e = launch_rmsnorm(norm_x, norm_x_f32, norm_gain, const_cast<__half*>(h), M, H, eps, st, n_launch, pdl);
+    if (e != cudaSuccess) return e;
   }
   const size_t smem = ((size_t)H + kRouterThreads + Epad) * sizeof(float);
   if (smem > 48 * 1024) {
