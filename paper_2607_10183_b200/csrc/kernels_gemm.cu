@@ -166,7 +166,7 @@ __device__ __forceinline__ uint4 dequant8(uint32_t w, __half2 s2) {
 }
 
 template <int FT, int TT>
-__global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const GemmKParams p) {
+__global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const GemmKParams p) {
   using Cfg = TileCfg<FT, TT>;
   constexpr int BF = Cfg::BF, TTILE = TT, MB = TT / BM, kDequantWarps = Cfg::kDequantWarps, kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -691,8 +691,10 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
     e = launch_dep(gemm_q4_kernel<2, 256>, grid, dim3(Cfg::kThreads), (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, p);
   } else {
     using Cfg = TileCfg<1, 128>;
-    p.stages = Cfg::kStages;
-    e = launch_dep(gemm_q4_kernel<1, 128>, grid, dim3(Cfg::kThreads), (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, p);
+    // Grouped form: every CTA streams its own expert's weights once and has few real rows, so what counts is how many
+    // weight loads are in flight per SM: three stages let two CTAs share an SM (registers are capped for that).
+    p.stages = g.grp_off ? 3 : Cfg::kStages;
+    e = launch_dep(gemm_q4_kernel<1, 128>, grid, dim3(Cfg::kThreads), (size_t)p.stages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, p);
   }
   if (e != cudaSuccess) return e;
   if (p.splits > 1) {
