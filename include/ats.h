@@ -201,8 +201,8 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, cons
                          uint32_t M);
 /* The same decode step driven from HOST buffers, as a caller that holds activations on the host sees it: copies x_in
  * (HOST fp16 [M][hidden]; pinned memory makes the copy asynchronous) into the workspace, runs ats_layer_decode on the
- * compute stream, copies the result into x_out (HOST fp16 [M][hidden]) and waits for the stream, so x_out is valid on
- * return.  The caches stay on the DEVICE.  Needs 2 * M * hidden * 2 bytes of workspace beyond ats_layer_decode's
+ * compute stream, copies the result into x_out (HOST fp16 [M][hidden]; when x_out is pinned memory the layer's last kernel
+ * writes it there directly and no copy is made) and waits for the stream, so x_out is valid on return.  The caches stay on the DEVICE.  Needs 2 * M * hidden * 2 bytes of workspace beyond ats_layer_decode's
  * (ats_workspace_bytes includes them).  Errors as ats_layer_decode, plus ATS_ERR_CUDA from the copies or the wait. */
 int32_t ats_layer_decode_host(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, const void* x_in /*HOST*/,
                               void* x_out /*HOST*/, void* k_cache /*DEVICE*/, void* v_cache /*DEVICE*/, uint32_t pos,

@@ -85,6 +85,8 @@ struct ats_ctx {
   uint32_t next_slot = 0;
   // pinned scratch for routing ids (host side of the one synchronisation on the MoE path)
   int32_t* ids_host = nullptr;
+  const void* host_out_seen = nullptr;  // last x_out of ats_layer_decode_host and its device alias (null: not pinned)
+  void* host_out_alias = nullptr;
   uint8_t* stage_host = nullptr;  // pinned scratch for per-call tables (MoE prefill: slice addresses, copy list)
   cudaEvent_t ids_event = nullptr;
   cudaEvent_t sync_event = nullptr;

@@ -1297,9 +1297,25 @@ int32_t ats_layer_decode_host(ats_ctx* ctx, const ats_layer_desc* L, const void*
     return fail(ctx, ATS_ERR_NOMEM, "workspace too small: host-driven decode needs %llu bytes", (unsigned long long)need);
   uint8_t* xin_dev = ctx->ws + w.total;
   uint8_t* xout_dev = xin_dev + stage;
+  // A pinned output buffer is addressable by the device: the layer's last kernel then writes the row straight into it
+  // (a few kilobytes of posted writes over PCIe) and the device-to-host copy with its fixed cost of several
+  // microseconds is not needed.  The answer for a buffer is cached: the query costs about as much as a launch.
+  void* out_alias = nullptr;
+  if (x_out == ctx->host_out_seen) {
+    out_alias = ctx->host_out_alias;
+  } else {
+    cudaPointerAttributes pa{};
+    if (cudaPointerGetAttributes(&pa, x_out) == cudaSuccess && pa.type == cudaMemoryTypeHost && pa.devicePointer &&
+        (reinterpret_cast<uintptr_t>(pa.devicePointer) & 15) == 0)
+      out_alias = pa.devicePointer;
+    else
+      cudaGetLastError();
+    ctx->host_out_seen = x_out;
+    ctx->host_out_alias = out_alias;
+  }
   ATS_CUDA(cudaMemcpyAsync(xin_dev, x_in, row_bytes, cudaMemcpyHostToDevice, ctx->cs));
-  ATS_TRY(ats_layer_decode(ctx, L, xin_dev, xout_dev, k_cache, v_cache, pos, M));
-  ATS_CUDA(cudaMemcpyAsync(x_out, xout_dev, row_bytes, cudaMemcpyDeviceToHost, ctx->cs));
+  ATS_TRY(ats_layer_decode(ctx, L, xin_dev, out_alias ? out_alias : xout_dev, k_cache, v_cache, pos, M));
+  if (!out_alias) ATS_CUDA(cudaMemcpyAsync(x_out, xout_dev, row_bytes, cudaMemcpyDeviceToHost, ctx->cs));
   ATS_CUDA(cudaStreamSynchronize(ctx->cs));
   return ATS_OK;
 }

@@ -189,7 +189,13 @@ def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, fl
     ctx.reset_stats()
     for s in range(steps):
         x = W.activations(cfg, 0, (1, shape.hidden), step=s)
-        if host_io:
+        if host_io == "pageable":  # ordinary host memory: the result comes back by a copy
+            xh = np.ascontiguousarray(x)
+            yh = np.zeros((1, shape.hidden), dtype=np.float16)
+            ctx.layer_decode_host(desc, xh, yh, kd, vd, pos + s, 1)
+            ys.append(yh.copy())
+            continue
+        if host_io:  # pinned memory: the layer's last kernel writes the result into it directly
             xh = torch.from_numpy(x).pin_memory()
             yh = torch.zeros((1, shape.hidden), dtype=torch.float16).pin_memory()
             ctx.layer_decode_host(desc, xh, yh, kd, vd, pos + s, 1)  # returns with yh valid: no sync here
@@ -240,10 +246,11 @@ def test_host_driven_decode_equals_device_driven(B, torch):
     shape, cfg, pos, cap = W.DENSE_SMALL, 96, 20, 40
     for placement in (ALL_GPU, {**ALL_GPU, "wk": 0, "w_up": 0, "w_down": 0}):
         dev = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, steps=3)
-        host = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, steps=3, host_io=True)
-        for a, b in zip(dev[0], host[0]):
-            assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
-        assert np.array_equal(dev[1], host[1]) and np.array_equal(dev[2], host[2])
+        for mode in (True, "pageable"):
+            host = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, steps=3, host_io=mode)
+            for a, b in zip(dev[0], host[0]):
+                assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+            assert np.array_equal(dev[1], host[1]) and np.array_equal(dev[2], host[2])
 
 
 def test_placement_invariance_and_bookkeeping_small(B, torch):
