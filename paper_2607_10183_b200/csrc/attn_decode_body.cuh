@@ -1,4 +1,5 @@
-// Decode attention for one (split, kv head) job, shared by the stand-alone kernel and the fused decode-layer kernel.
+// Decode attention for one (split, kv head) job: the device code of the decode attention kernel, written so that a
+// subset of a CTA's threads can run it too (CTA_SYNC = false).
 #pragma once
 #include "ats_internal.h"
 

@@ -1,6 +1,6 @@
-// Streaming decode GEMV for one token (sm_100a): the memory-bound hot kernel of the decode path.  Device code shared by
-// the stand-alone GEMV kernels and the fused decode-layer kernel, which runs a layer's four GEMVs as phases of one launch
-// over one ring.
+// Streaming decode GEMV for one token (sm_100a): the memory-bound hot kernel of the decode path.  Device code of the dense
+// and the grouped-expert kernels, written as a producer function and a consumer function over an explicit ring state (a
+// kernel may run several such phases back to back over one ring; the kernels in this library run one).
 //
 // Structure: one persistent CTA per SM: 16 consumer warps in two groups of 8 + 1 producer warp.  The producer streams
 // row tiles of the packed weights (codes and scales, contiguous byte ranges) into a ring of 8 shared-memory stages with

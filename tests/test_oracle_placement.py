@@ -102,8 +102,8 @@ def test_units_round_sizes_up_and_budget_down():
 def test_32_layer_dense_stack_at_60_percent():
     """The 32-layer stack of the dense workload at a 60 % byte budget, sizes = values = bytes, c = 0.
     Independent cross-checks: the result fills the budget's 2246 MiB units exactly and equals the
-    textbook knapsack optimum; the resident/streamed byte split was also found by a separate
-    numpy probe during the survey of this build (2,326,265,856 resident / 1,599,602,688 streamed)."""
+    textbook knapsack optimum; the resident/streamed byte split (2,326,265,856 resident /
+    1,599,602,688 streamed) was also obtained by an independent numpy knapsack over the same sizes."""
     shape = W.DENSE_FULL
     nbytes = [W.q4_bytes(n, k) for _ in range(32) for (_, n, k) in shape.tensor_shapes()]
     total = sum(nbytes)
