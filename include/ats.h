@@ -274,6 +274,19 @@ int32_t ats_measure_h2d(ats_ctx* ctx, uint64_t bytes, uint32_t reps, double* out
  * injection; nothing faults on the device).  The failing call returns ATS_ERR_CUDA and the context is poisoned. */
 int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n);
 
+/* The two ends of a whole-model loop around the layer calls (Section 5's workloads run whole models).
+ * ats_embed: rows token_ids[m] of a Q4B32 table [vocab = n_out][hidden = k_in], dequantized to fp16 (scale * code rounded
+ * once, as ats_dequantize writes it): out DEVICE fp16 [M][k_in].  token_ids DEVICE int32 [M]; an id outside [0, n_out)
+ * gives a row of zeros and makes the next ats_sync fail.  A host-placed table is read in place through the mapped pinned
+ * store (a few rows per call), never streamed whole.
+ * ats_lm_head: logits = W_head * RMSNorm(x; norm_id gain, eps), x DEVICE fp16 [M][hidden], logits DEVICE fp16 [M][vocab];
+ * the normalised row is rounded to fp16 before the product (the contract's edge "h").  M = 1 runs as one launch of the
+ * streaming GEMV with the norm as its prologue (hidden <= 4096 and a shape that kernel takes); otherwise a norm launch
+ * into `scratch` (DEVICE fp16 [M][hidden], caller-provided, may be NULL only for the one-launch case) and ats_linear. */
+int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids /*DEVICE*/, uint32_t M, void* out /*DEVICE*/);
+int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, const void* x /*DEVICE*/, void* logits /*DEVICE*/,
+                    uint32_t M, void* scratch /*DEVICE*/);
+
 /* Debug/test hook: device address and byte size of an intermediate of the most recent ats_layer_decode call shape
  * (which = 0 h, 1 qkv (fp32 [q|k|v]), 2 q_rot (fp32), 3 a (fp16), 4 x1 (fp32), 5 h2 (fp16), 6 act (fp16), 7 d (fp32, MoE),
  * 8 ids (int32, MoE), 9 gates (fp32, MoE)).  The workspace is reused by every call; read it after ats_sync(). */

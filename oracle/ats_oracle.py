@@ -101,6 +101,19 @@ def linear(x: np.ndarray, packed: np.ndarray, scales: np.ndarray, weight_mode: i
 # --------------------------------------------------------------------------------------
 # a6: layer glue
 # --------------------------------------------------------------------------------------
+def embed(token_ids, packed: np.ndarray, scales: np.ndarray) -> np.ndarray:
+    """Embedding lookup in a block-quantized table [vocab][hidden]: row t is the dequantized row rounded
+    once to fp16 (the model's residual stream starts as fp16).  Returns fp16 [M, hidden]."""
+    w = dequantize(packed, scales, WEIGHT_F16)  # rn16(scale * code) per element
+    return np.asarray(w[np.asarray(token_ids, dtype=np.int64)], dtype=np.float16)
+
+
+def lm_head(x, gain: np.ndarray, eps: float, packed: np.ndarray, scales: np.ndarray, weight_mode: int = WEIGHT_EXACT) -> np.ndarray:
+    """Final RMSNorm (rounded to fp16: the contract's edge "h") and the vocabulary projection; logits fp16."""
+    h = rn16(rmsnorm(np.asarray(x, dtype=np.float64), gain, eps))
+    return linear(h, packed, scales, weight_mode, round_out=True)
+
+
 def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
     """h_i = x_i g_i / sqrt(mean_j x_j^2 + eps), per row."""
     x = np.asarray(x, dtype=np.float64)

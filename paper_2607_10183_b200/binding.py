@@ -28,7 +28,7 @@ EDGES = ("h", "q", "k", "v", "q_rot", "a", "o", "x1", "h2", "g", "u", "act", "d"
 
 EXPORTS = (
     "ats_init", "ats_destroy", "ats_last_error", "ats_register_tensor", "ats_tensor_slice_bytes", "ats_set_placement",
-    "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode", "ats_layer_decode_host",
+    "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode", "ats_layer_decode_host", "ats_embed", "ats_lm_head",
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
     "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
     "ats_host_unpack_q4",
@@ -82,6 +82,8 @@ def _load():
         "ats_moe_linear": (i32, [vp, i32, vp, vp, vp, u32, u32, u32]),
         "ats_layer_decode": (i32, [vp, P(ats_layer_desc), vp, vp, vp, vp, u32, u32]),
         "ats_layer_decode_host": (i32, [vp, P(ats_layer_desc), vp, vp, vp, vp, u32, u32]),
+        "ats_embed": (i32, [vp, i32, vp, u32, vp]),
+        "ats_lm_head": (i32, [vp, i32, i32, C.c_float, vp, vp, u32, vp]),
         "ats_layer_prefill": (i32, [vp, P(ats_layer_desc), vp, vp, vp, vp, u32, u32]),
         "ats_workspace_bytes": (u64, [P(ats_layer_desc), u32]),
         "ats_dequantize": (i32, [vp, i32, i32, vp, u32]),
@@ -235,6 +237,14 @@ class Context:
     def layer_decode_host(self, desc, x_in_host, x_out_host, k_cache, v_cache, pos, M=1):
         return self.check(lib.ats_layer_decode_host(self.h, C.byref(desc), _ptr(x_in_host), _ptr(x_out_host), _ptr(k_cache),
                                                     _ptr(v_cache), pos, M))
+
+    def embed(self, tid, token_ids, out, M):
+        """Rows token_ids[m] (device int32) of a Q4B32 table as fp16 rows of `out` (device)."""
+        return self.check(lib.ats_embed(self.h, tid, _ptr(token_ids), M, _ptr(out)))
+
+    def lm_head(self, norm_id, head_id, eps, x, logits, M=1, scratch=None):
+        """logits = W_head * RMSNorm(x); `scratch` (device fp16 [M][hidden]) is needed unless the one-launch form applies."""
+        return self.check(lib.ats_lm_head(self.h, norm_id, head_id, eps, _ptr(x), _ptr(logits), M, _ptr(scratch)))
 
     def layer_prefill(self, desc, x_in, x_out, k_cache, v_cache, pos0, T):
         return self.check(lib.ats_layer_prefill(self.h, C.byref(desc), _ptr(x_in), _ptr(x_out), _ptr(k_cache), _ptr(v_cache), pos0, T))

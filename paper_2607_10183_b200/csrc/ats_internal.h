@@ -228,6 +228,8 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& p, const MoeJobs* jobs /
 
 cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, cudaStream_t st,
                            uint64_t* n_launch);
+cudaError_t launch_embed_rows(const uint8_t* slice, int n_rows, int K, const int32_t* ids, int M, __half* out, int* status,
+                              cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
                            cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 // decode attention, fused with the rotary embedding and the KV append (kernels_decode.cu)

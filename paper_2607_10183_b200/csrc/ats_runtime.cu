@@ -909,6 +909,73 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M)
   return run_gemm_group(ctx, &op, 1, g);
 }
 
+static int32_t check_f16(ats_ctx* ctx, int32_t id, uint32_t n_out, uint32_t k_in, const char* name);
+
+int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids, uint32_t M, void* out) {
+  ATS_TRY(precheck(ctx, true));
+  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", id);
+  if (!token_ids || !out) return fail(ctx, ATS_ERR_INVALID, "null pointer");
+  if (M == 0) return ATS_OK;
+  const uint8_t* ptr = t->slices[0].dev;
+  if (t->slices[0].where != ATS_GPU) {
+    // a host-placed table: the rows are read where they are (a lookup touches a few kilobytes of a table of hundreds of
+    // megabytes)
+    if (!t->host_dev) {
+      void* alias = nullptr;
+      if (cudaHostGetDevicePointer(&alias, t->host, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ctx, ATS_ERR_UNSUPPORTED, "host-placed embedding table: the pinned store is not mapped into the device");
+      }
+      t->host_dev = static_cast<const uint8_t*>(alias);
+    }
+    ptr = t->host_dev;
+  }
+  const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
+  ATS_CUDA(launch_embed_rows(ptr, (int)t->d.n_out, (int)t->d.k_in, token_ids, (int)M, (__half*)out, ctx->dev_status, ctx->cs,
+                             &ctx->stats.kernel_launches, pdl));
+  return ATS_OK;
+}
+
+int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, const void* x, void* logits, uint32_t M, void* scratch) {
+  ATS_TRY(precheck(ctx, true));
+  Tensor* t = get_tensor(ctx, head_id, ATS_FMT_Q4B32);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", head_id);
+  ATS_TRY(check_f16(ctx, norm_id, t->d.k_in, 1, "final norm"));
+  if (!x || !logits) return fail(ctx, ATS_ERR_INVALID, "null pointer");
+  if (M == 0) return ATS_OK;
+  const __half* gain = (const __half*)ctx->tensors[norm_id].f16_dev;
+  const int K = (int)t->d.k_in, N = (int)t->d.n_out;
+  if (M == 1) {
+    GemvParams p{};
+    p.M = 1;
+    p.norm_x16 = (const __half*)x;
+    p.norm_gain = gain;
+    p.norm_eps = eps;
+    p.norm_out = (__half*)scratch;
+    p.x = (const __half*)scratch;  // used only when the norm runs as its own launch
+    p.ldx = K;
+    p.y16 = (__half*)logits;
+    p.ldy = N;
+    p.mode = GEMV_OUT_F16;
+    GemvParams probe = p;
+    probe.K = K;
+    probe.n_seg = 1;
+    probe.seg[0] = GemvSeg{nullptr, N};
+    if (!scratch && !gemv_stream_eligible(probe))
+      return fail(ctx, ATS_ERR_INVALID, "ats_lm_head needs `scratch` for this shape (the norm runs as a launch of its own)");
+    plan_begin(ctx);
+    Operand op;
+    plan_dense(ctx, head_id, &op);
+    ATS_TRY(pump(ctx));
+    return run_gemv_group(ctx, &op, 1, p);
+  }
+  if (!scratch) return fail(ctx, ATS_ERR_INVALID, "ats_lm_head with M > 1 needs `scratch`");
+  const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
+  ATS_CUDA(launch_rmsnorm(x, 0, gain, (__half*)scratch, (int)M, K, eps, ctx->cs, &ctx->stats.kernel_launches, pdl));
+  return ats_linear(ctx, head_id, scratch, logits, M);
+}
+
 int32_t ats_linear_static_scratch(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M) {
   ATS_TRY(precheck(ctx, true));
   Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);

@@ -78,6 +78,43 @@ __global__ void dequant_kernel(const uint8_t* __restrict__ slice, int n_rows, in
   }
 }
 
+// Embedding lookup: out[m] = rn16(scale * code) of row ids[m] of a Q4B32 table (the fp16 form ats_dequantize writes).
+// One thread per code word; ids outside [0, n_rows) give a row of zeros and raise the status word.
+__global__ void embed_rows_kernel(const uint8_t* __restrict__ slice, int n_rows, int K, const int32_t* __restrict__ ids, int M,
+                                  __half* __restrict__ out, int* __restrict__ status) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the ids may come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int wpr = K / 8;  // words per row
+  const uint32_t* codes = reinterpret_cast<const uint32_t*>(slice);
+  const __half* scales = reinterpret_cast<const __half*>(slice + (uint64_t)n_rows * K / 2);
+  for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < (uint64_t)M * wpr; i += (uint64_t)gridDim.x * blockDim.x) {
+    const int m = (int)(i / wpr), w = (int)(i % wpr);
+    const int row = ids[m];
+    uint4 o = make_uint4(0, 0, 0, 0);
+    if (row >= 0 && row < n_rows) {
+      __half2 c[4];
+      unpack8(codes[(uint64_t)row * wpr + w], c);
+      const __half2 s2 = __half2half2(scales[(uint64_t)row * (K / 32) + w / 4]);
+      __half2 r0 = __hmul2(c[0], s2), r1 = __hmul2(c[1], s2), r2 = __hmul2(c[2], s2), r3 = __hmul2(c[3], s2);
+      o.x = *reinterpret_cast<uint32_t*>(&r0);
+      o.y = *reinterpret_cast<uint32_t*>(&r1);
+      o.z = *reinterpret_cast<uint32_t*>(&r2);
+      o.w = *reinterpret_cast<uint32_t*>(&r3);
+    } else if (w == 0) {
+      atomicExch(status, 6);
+    }
+    reinterpret_cast<uint4*>(out)[i] = o;
+  }
+}
+
+cudaError_t launch_embed_rows(const uint8_t* slice, int n_rows, int K, const int32_t* ids, int M, __half* out, int* status,
+                              cudaStream_t st, uint64_t* n_launch, int pdl) {
+  const uint64_t words = (uint64_t)M * K / 8;
+  const int grid = (int)std::min<uint64_t>((words + 255) / 256, 148 * 8);
+  ++*n_launch;
+  return launch_dep(embed_rows_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, slice, n_rows, K, ids, M, out, status);
+}
+
 cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, cudaStream_t st,
                            uint64_t* n_launch) {
   const uint64_t words = (uint64_t)n_rows * K / 8;

@@ -148,6 +148,61 @@ def test_streaming_gemv_activation_extremes(B, torch):
     ctx.close()
 
 
+@pytest.mark.parametrize("where", ["gpu", "host"])
+def test_embed_rows_bit_exact(B, torch, where):
+    """Embedding lookup = the dequantized rows rounded once to fp16, bit for bit; a host-placed table is read in place."""
+    V, Hd = 1000, 512
+    packed, scales = W.q4_packed(95, 0, W.ROLE_Q, V, Hd)
+    ctx = make_ctx(B, W.q4_bytes(V, Hd), slot_bytes=W.q4_bytes(V, Hd))
+    tid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(tid, -1, B.ATS_GPU if where == "gpu" else B.ATS_HOST)])
+    ids = np.array([0, 999, 17, 17, 512, 3], dtype=np.int32)
+    out = torch.full((len(ids), Hd), 7.0, dtype=torch.float16, device="cuda")
+    ctx.reset_stats()
+    ctx.embed(tid, H.to_dev(ids), out, len(ids))
+    ctx.sync()
+    want = O.embed(ids, packed, scales)
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), want.view(np.uint16))
+    assert ctx.stats().streamed_bytes == 0  # never streamed whole
+    # an id outside the table: a row of zeros, and the next sync reports it
+    bad = np.array([5, V], dtype=np.int32)
+    out2 = torch.full((2, Hd), 7.0, dtype=torch.float16, device="cuda")
+    ctx.embed(tid, H.to_dev(bad), out2, 2)
+    with pytest.raises(B.AtsError):
+        ctx.sync()
+    assert np.all(out2.cpu().numpy()[1] == 0)
+    ctx.close()
+
+
+@pytest.mark.parametrize("V,Hd,M", [(4096, 1024, 1), (1000, 448, 1), (2048, 512, 5), (640, 256, 12)])
+def test_lm_head_matches_oracle(B, torch, V, Hd, M):
+    """Final norm + vocabulary projection: one launch of the streaming GEMV for a single row where its shapes allow, a norm
+    launch and the GEMV / GEMM otherwise."""
+    packed, scales = W.q4_packed(95, 1, W.ROLE_Q, V, Hd)
+    gain = W.activations(95, 3, (Hd,)).astype(np.float16)
+    x = W.activations(95, 0, (M, Hd))
+    eps = 1e-5
+    ctx = make_ctx(B, W.q4_bytes(V, Hd) + 64 * 1024, ws=16 * MB)
+    nid = ctx.register_f16(gain)
+    hid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(hid, -1, B.ATS_GPU)])
+    logits = torch.empty((M, V), dtype=torch.float16, device="cuda")
+    scratch = torch.empty((M, Hd), dtype=torch.float16, device="cuda")
+    ctx.lm_head(nid, hid, eps, H.to_dev(x), logits, M, scratch)
+    ctx.sync()
+    edges, wmode = ctx.numerics(B.ATS_MODE_PREFILL if M > 8 else B.ATS_MODE_DECODE)
+    want = O.lm_head(x, gain, eps, packed, scales, wmode)
+    H.assert_close(logits.cpu().numpy(), want, what=f"lm head {V}x{Hd} M={M}")
+    if (V, Hd, M) == (4096, 1024, 1):  # the one-launch form needs no scratch
+        logits2 = torch.empty_like(logits)
+        ctx.reset_stats()
+        ctx.lm_head(nid, hid, eps, H.to_dev(x), logits2, 1, None)
+        ctx.sync()
+        assert ctx.stats().kernel_launches == 1
+        assert np.array_equal(logits.cpu().numpy().view(np.uint16), logits2.cpu().numpy().view(np.uint16))
+    ctx.close()
+
+
 def test_linear_closed_forms_on_gpu(B, torch):
     """One-hot activations return a weight column exactly; all-ones with unit scales return integer row sums."""
     N, K = 40, 256

@@ -328,3 +328,39 @@ def test_moe_linear_matches_linear_per_slot():
     xs = W.activations(92, 1, (2, 2, shape.ffn))
     y2 = O.moe_linear(xs, ids, *t["w_down"], x_per_slot=True)
     assert np.array_equal(y2[1, 0], O.linear(xs[1, 0][None], t["w_down"][0][5], t["w_down"][1][5], round_out=True)[0])
+
+
+def test_embed_and_lm_head_closed_forms():
+    """embed: with a power-of-two scale the looked-up row is the integer codes times that scale, for every id incl. repeats;
+    a scale whose product needs rounding gives the fp16 nearest to the exact rational.  lm_head: with a unit gain and an
+    input of constant magnitude c the normalised row is sign(x) * c / sqrt(c^2 + eps), so the logits are that factor times
+    the signed row sums of the codes."""
+    from fractions import Fraction
+    rng = np.random.default_rng(3)
+    V, Hd = 12, 64
+    codes = rng.integers(-8, 8, size=(V, Hd)).astype(np.int64)
+    nib = np.where(codes < 0, codes + 16, codes).astype(np.uint8)
+    packed = (nib[:, 0::2] | (nib[:, 1::2] << 4)).astype(np.uint8)  # byte j: code 2j low nibble, 2j+1 high nibble
+    scales = np.full((V, Hd // 32), 0.25, dtype=np.float16)
+    ids = np.array([5, 0, 11, 5], dtype=np.int32)
+    got = O.embed(ids, packed, scales)
+    assert got.dtype == np.float16 and np.array_equal(got.astype(np.float64), codes[ids] * 0.25)
+    s = np.float16(0.3333)  # code * s is not an fp16 number in general
+    scales2 = np.full((V, Hd // 32), s, dtype=np.float16)
+    got2 = O.embed(ids, packed, scales2).astype(np.float64)
+    sf = Fraction(float(s))
+    for m, t in enumerate(ids):
+        for k in range(Hd):
+            exact = sf * int(codes[t, k])
+            cand = np.float16(float(exact))
+            assert got2[m, k] == float(cand)  # float(exact) is exact here (15 significant bits): one rounding to fp16
+    # lm_head
+    c = 0.5
+    eps = 1e-2
+    x = (c * np.where(rng.random(Hd) < 0.5, -1.0, 1.0)).astype(np.float16)[None, :]
+    gain = np.ones(Hd, dtype=np.float16)
+    ones = np.ones((V, Hd // 32), dtype=np.float16)
+    logits = O.lm_head(x, gain, eps, packed, ones)
+    h = np.float64(np.float16(c / np.sqrt(c * c + eps)))  # the normalised magnitude, rounded to fp16 as the contract says
+    want = (codes * np.sign(x.astype(np.float64))).sum(axis=1) * h
+    assert np.array_equal(np.asarray(logits, dtype=np.float64)[0], O.rn16(want))
