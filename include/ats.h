@@ -50,7 +50,11 @@ enum {
 };
 
 enum { ATS_HOST = 0, ATS_GPU = 1 };             /* placement b_i (Section 4.3.2) */
-enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1 };    /* F16: router weight [k_in][n_out], norm gain [n_out] */
+enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1, ATS_FMT_W16 = 2 };
+/* F16: small auxiliary tensors (router weight [k_in][n_out], norm gain [n_out]): always resident, no placement.
+ * W16: an unquantized fp16 weight matrix [n_out][k_in] (the paper runs one of its models with FP16 weights, Section 5.1):
+ * a dense tensor (n_experts = 1, k_in a multiple of 8) placed and streamed like a Q4B32 tensor (2 bytes per weight);
+ * ats_linear takes it; the layer calls, ats_moe_linear and ats_dequantize take Q4B32 tensors only. */
 enum { ATS_OUT_F32 = 0, ATS_OUT_F16 = 1 };      /* ats_dequantize output */
 enum { ATS_MODE_DECODE = 0, ATS_MODE_PREFILL = 1 };
 

@@ -98,6 +98,14 @@ def linear(x: np.ndarray, packed: np.ndarray, scales: np.ndarray, weight_mode: i
     return rn16(y) if round_out else y
 
 
+def linear_w16(x: np.ndarray, w16: np.ndarray, round_out: bool = False) -> np.ndarray:
+    """The per-tensor operator for an unquantized fp16 weight matrix [N][K] (the paper runs one of its models with
+    FP16 weights): y[m,n] = sum_k w[n,k] x[m,k] in fp64 over the fp16 values as they are."""
+    w = np.asarray(w16, dtype=np.float16).astype(np.float64)
+    y = np.asarray(x, dtype=np.float64) @ w.T
+    return rn16(y) if round_out else y
+
+
 # --------------------------------------------------------------------------------------
 # a6: layer glue
 # --------------------------------------------------------------------------------------

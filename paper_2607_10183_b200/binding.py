@@ -18,7 +18,7 @@ ATS_OK = 0
 ATS_ERR_INVALID, ATS_ERR_SHAPE, ATS_ERR_NOMEM, ATS_ERR_BUDGET = -1, -2, -3, -4
 ATS_ERR_STATE, ATS_ERR_CUDA, ATS_ERR_TIMEOUT, ATS_ERR_UNSUPPORTED = -5, -6, -7, -8
 ATS_HOST, ATS_GPU = 0, 1
-ATS_FMT_Q4B32, ATS_FMT_F16 = 0, 1
+ATS_FMT_Q4B32, ATS_FMT_F16, ATS_FMT_W16 = 0, 1, 2
 ATS_OUT_F32, ATS_OUT_F16 = 0, 1
 ATS_MODE_DECODE, ATS_MODE_PREFILL = 0, 1
 ATS_FLAG_POISON_SLOTS, ATS_FLAG_SKIP_SCALE_CHECK, ATS_FLAG_TIME_KERNELS, ATS_FLAG_NO_PDL, ATS_FLAG_MOE_DEVICE_GATHER = 1, 2, 4, 8, 16
@@ -184,6 +184,15 @@ class Context:
         d = ats_tensor_desc(ATS_FMT_Q4B32, E, n_out, k_in, layer, role, value, switch_cost)
         out = C.c_int32(-1)
         self.check(lib.ats_register_tensor(self.h, C.byref(d), packed.ctypes.data, scales.ctypes.data, C.byref(out)))
+        return out.value
+
+    def register_w16(self, w: np.ndarray, layer=0, role=0, value=-1, switch_cost=0) -> int:
+        """An unquantized fp16 weight matrix [n_out][k_in] (placed and streamed like a quantized tensor)."""
+        w = np.ascontiguousarray(w, dtype=np.float16)
+        n_out, k_in = w.shape
+        d = ats_tensor_desc(ATS_FMT_W16, 1, n_out, k_in, layer, role, value, switch_cost)
+        out = C.c_int32(-1)
+        self.check(lib.ats_register_tensor(self.h, C.byref(d), w.ctypes.data, None, C.byref(out)))
         return out.value
 
     def register_f16(self, data: np.ndarray, layer=0, role=0) -> int:

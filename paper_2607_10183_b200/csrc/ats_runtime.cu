@@ -97,6 +97,13 @@ static Tensor* get_tensor(ats_ctx* ctx, int32_t id, uint32_t fmt) {
   Tensor* t = &ctx->tensors[id];
   return t->d.fmt == fmt ? t : nullptr;
 }
+// tensors that take part in placement: block-quantized or fp16 weight matrices
+static bool placeable(const Tensor& t) { return t.d.fmt == ATS_FMT_Q4B32 || t.d.fmt == ATS_FMT_W16; }
+static Tensor* get_weight(ats_ctx* ctx, int32_t id) {
+  if (id < 0 || (size_t)id >= ctx->tensors.size()) return nullptr;
+  Tensor* t = &ctx->tensors[id];
+  return placeable(*t) ? t : nullptr;
+}
 
 // ------------------------------------------------------------------------------------ streaming ring
 // The per-call execution plan is the ordered list ctx->plan of slices to stream.  Copies are issued in plan order into
@@ -757,7 +764,7 @@ int32_t ats_register_tensor(ats_ctx* ctx, const ats_tensor_desc* d, const void* 
                             int32_t* out_id) {
   ATS_TRY(precheck(ctx, false));
   if (!d || !codes || !out_id) return fail(ctx, ATS_ERR_INVALID, "null argument");
-  if (d->fmt != ATS_FMT_Q4B32 && d->fmt != ATS_FMT_F16) return fail(ctx, ATS_ERR_INVALID, "unknown format %u", d->fmt);
+  if (d->fmt != ATS_FMT_Q4B32 && d->fmt != ATS_FMT_F16 && d->fmt != ATS_FMT_W16) return fail(ctx, ATS_ERR_INVALID, "unknown format %u", d->fmt);
   if (d->n_out == 0 || d->k_in == 0 || d->n_experts == 0) return fail(ctx, ATS_ERR_SHAPE, "zero dimension");
   if (d->switch_cost < 0) return fail(ctx, ATS_ERR_INVALID, "switch_cost must be >= 0");
   Tensor t;
@@ -770,6 +777,21 @@ int32_t ats_register_tensor(ats_ctx* ctx, const ats_tensor_desc* d, const void* 
       return fail(ctx, ATS_ERR_NOMEM, "pinned allocation of %llu bytes failed", (unsigned long long)t.host_bytes);
     }
     memcpy(t.host, codes, t.host_bytes);
+  } else if (d->fmt == ATS_FMT_W16) {
+    if (d->n_experts != 1) return fail(ctx, ATS_ERR_SHAPE, "W16 tensors are not stacked");
+    if (d->k_in % 8) return fail(ctx, ATS_ERR_SHAPE, "k_in = %u is not a multiple of 8", d->k_in);
+    t.codes_bytes = (uint64_t)d->n_out * d->k_in * 2;
+    t.slice_bytes = t.codes_bytes;
+    t.slice_stride = align_up(t.slice_bytes);
+    t.host_bytes = t.slice_stride;
+    if (cudaHostAlloc((void**)&t.host, t.host_bytes, cudaHostAllocDefault) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, ATS_ERR_NOMEM, "pinned allocation of %llu bytes failed", (unsigned long long)t.host_bytes);
+    }
+    memcpy(t.host, codes, t.slice_bytes);
+    if (t.slice_stride > t.slice_bytes) memset(t.host + t.slice_bytes, 0, t.slice_stride - t.slice_bytes);
+    t.slices.resize(1);
+    if (t.d.value < 0) t.d.value = (int64_t)t.slice_bytes;
   } else {
     if (d->k_in % kBlock) return fail(ctx, ATS_ERR_SHAPE, "k_in = %u is not a multiple of 32", d->k_in);
     if (!scales) return fail(ctx, ATS_ERR_INVALID, "null scales");
@@ -814,8 +836,8 @@ int32_t ats_set_placement(ats_ctx* ctx, const int32_t* ids, const int32_t* exper
   ATS_TRY(precheck(ctx, false));
   if (n && (!ids || !where)) return fail(ctx, ATS_ERR_INVALID, "null argument");
   for (uint32_t i = 0; i < n; ++i) {
-    Tensor* t = get_tensor(ctx, ids[i], ATS_FMT_Q4B32);
-    if (!t) return fail(ctx, ATS_ERR_INVALID, "entry %u: id %d is not a registered Q4B32 tensor", i, ids[i]);
+    Tensor* t = get_weight(ctx, ids[i]);
+    if (!t) return fail(ctx, ATS_ERR_INVALID, "entry %u: id %d is not a registered weight tensor", i, ids[i]);
     const int32_t e = experts ? experts[i] : -1;
     if (e < -1 || e >= (int32_t)t->slices.size()) return fail(ctx, ATS_ERR_INVALID, "entry %u: expert %d out of range", i, e);
     if (where[i] != ATS_HOST && where[i] != ATS_GPU) return fail(ctx, ATS_ERR_INVALID, "entry %u: placement %u", i, where[i]);
@@ -842,7 +864,7 @@ int32_t ats_plan_placement(ats_ctx* ctx, uint64_t budget_bytes, uint32_t granule
   std::vector<int> idx;
   for (size_t i = 0; i < ctx->tensors.size(); ++i) {
     const Tensor& t = ctx->tensors[i];
-    if (t.d.fmt != ATS_FMT_Q4B32) continue;
+    if (!placeable(t)) continue;
     const uint64_t bytes = t.slice_bytes * t.slices.size();
     s.push_back((int64_t)((bytes + G - 1) / G));
     r.push_back(t.d.value);
@@ -851,7 +873,7 @@ int32_t ats_plan_placement(ats_ctx* ctx, uint64_t budget_bytes, uint32_t granule
     idx.push_back((int)i);
   }
   if (out_where && n != idx.size())
-    return fail(ctx, ATS_ERR_INVALID, "out_where holds %u entries, %zu Q4B32 tensors are registered", n, idx.size());
+    return fail(ctx, ATS_ERR_INVALID, "out_where holds %u entries, %zu weight tensors are registered", n, idx.size());
   std::vector<uint8_t> b;
   static_placement(s, r, c, is_exp, (int64_t)(budget_bytes / G), &b);
   for (size_t j = 0; j < idx.size(); ++j)
@@ -877,14 +899,25 @@ int32_t ats_get_placement(const ats_ctx* ctx, int32_t id, int32_t expert, uint8_
 
 int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M) {
   ATS_TRY(precheck(ctx, true));
-  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
-  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", id);
+  Tensor* t = get_weight(ctx, id);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense weight tensor", id);
   if (!x || !y) return fail(ctx, ATS_ERR_INVALID, "null pointer");
   if (M == 0) return ATS_OK;
   plan_begin(ctx);
   Operand op;
   plan_dense(ctx, id, &op);
   ATS_TRY(pump(ctx));
+  if (t->d.fmt == ATS_FMT_W16) {
+    const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
+    ATS_TRY(acquire_ops(ctx, &op, 1));
+    if (M <= 8) {
+      ATS_CUDA(launch_gemv_w16((const __half*)op.ptr, (int)t->d.n_out, (int)t->d.k_in, (const __half*)x, (int)t->d.k_in, (__half*)y,
+                               (int)t->d.n_out, (int)M, ctx->cs, &ctx->stats.kernel_launches, pdl));
+    } else {
+      return fail(ctx, ATS_ERR_UNSUPPORTED, "W16 tensors take M <= 8 rows");
+    }
+    return release_ops(ctx, &op, 1);
+  }
   if (M <= 8) {
     GemvParams p{};
     p.M = (int)M;

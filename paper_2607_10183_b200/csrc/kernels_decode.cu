@@ -128,6 +128,86 @@ cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, i
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------- fp16-weight GEMV
+// y[m][n] = rn16(sum_k W[n][k] x[m][k]) for an unquantized fp16 matrix W [N][K], M <= 8 rows of x.  HBM-bound at 2 bytes per
+// weight: a warp owns two rows at a time, its lanes walk K in 16-byte pieces with eight weight loads in flight per thread
+// (streaming loads: every weight is used once); x comes through L1.  Products of fp16 values are exact in fp32; sums in
+// fp32, lanes combined by shuffles in fixed order.
+template <int M>
+__global__ void __launch_bounds__(256) gemv_w16_kernel(const __half* __restrict__ W, int N, int K, const __half* __restrict__ x, int ldx,
+                                                       __half* __restrict__ y, int ldy) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // x comes from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int lane = threadIdx.x & 31;
+  const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), n_warps = gridDim.x * (blockDim.x >> 5);
+  const int nch = K / 8;  // 16-byte pieces per row
+  auto dot8 = [](const uint4& a, const uint4& b, float acc) {
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float2 fa = __half22float2(u32_as_half2(aw[q])), fb = __half22float2(u32_as_half2(bw[q]));
+      acc = fmaf(fa.x, fb.x, acc);
+      acc = fmaf(fa.y, fb.y, acc);
+    }
+    return acc;
+  };
+  for (int rp = warp; 2 * rp < N; rp += n_warps) {
+    const int r0 = 2 * rp, r1 = min(r0 + 1, N - 1);
+    const uint4* w0 = reinterpret_cast<const uint4*>(W + (size_t)r0 * K);
+    const uint4* w1 = reinterpret_cast<const uint4*>(W + (size_t)r1 * K);
+    float acc[2][M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) acc[0][m] = acc[1][m] = 0.f;
+    for (int c0 = lane; c0 < nch; c0 += 128) {
+      uint4 a[4], b[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + 32 * u;
+        a[u] = c < nch ? __ldcs(w0 + c) : make_uint4(0, 0, 0, 0);
+        b[u] = c < nch ? __ldcs(w1 + c) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + 32 * u;
+        if (c < nch) {
+#pragma unroll
+          for (int m = 0; m < M; ++m) {
+            const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * ldx) + c);
+            acc[0][m] = dot8(a[u], xv, acc[0][m]);
+            acc[1][m] = dot8(b[u], xv, acc[1][m]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const float s0 = warp_sum(acc[0][m]), s1 = warp_sum(acc[1][m]);
+      if (lane == 0) {
+        y[(size_t)m * ldy + r0] = __float2half_rn(s0);
+        if (r0 + 1 < N) y[(size_t)m * ldy + r0 + 1] = __float2half_rn(s1);
+      }
+    }
+  }
+}
+
+cudaError_t launch_gemv_w16(const __half* W, int N, int K, const __half* x, int ldx, __half* y, int ldy, int M, cudaStream_t st,
+                            uint64_t* n_launch, int pdl) {
+  if (M < 1 || M > 8 || K % 8) return cudaErrorInvalidValue;
+  const int pairs = (N + 1) / 2;
+  const dim3 grid(std::max(1, std::min((pairs + 7) / 8, 148 * 8))), block(256);
+  ++*n_launch;
+  switch (M) {
+    case 1: return launch_dep(gemv_w16_kernel<1>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+    case 2: return launch_dep(gemv_w16_kernel<2>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+    case 3: return launch_dep(gemv_w16_kernel<3>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+    case 4: return launch_dep(gemv_w16_kernel<4>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+    case 5: return launch_dep(gemv_w16_kernel<5>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+    case 6: return launch_dep(gemv_w16_kernel<6>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+    case 7: return launch_dep(gemv_w16_kernel<7>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+    default: return launch_dep(gemv_w16_kernel<8>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+  }
+}
+
 // ------------------------------------------------------------------------------------------- GEMV core (a2, a5)
 constexpr int kGemvMaxWarps = 8;
 constexpr int kWR = 4;  // weight rows a CTA works on at once

@@ -203,6 +203,35 @@ def test_lm_head_matches_oracle(B, torch, V, Hd, M):
     ctx.close()
 
 
+@pytest.mark.parametrize("N,K,M", [(1, 8, 1), (7, 72, 3), (130, 1000, 8), (257, 4096, 1), (4096, 4096, 1), (64, 14336, 5)])
+def test_linear_w16_gemv_matches_oracle(B, torch, N, K, M):
+    """An unquantized fp16 weight matrix: resident and streamed through the ring give the same bits; both match the oracle."""
+    rng = np.random.default_rng(N * 131 + K)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float16)
+    x = W.activations(95, 0, (M, K))
+    want = O.linear_w16(x, w, round_out=True)
+    outs = []
+    nb = N * K * 2
+    slot = -(-nb // 256) * 256
+    for where in (B.ATS_GPU, B.ATS_HOST):
+        ctx = make_ctx(B, slot, slot_bytes=slot, chunk_bytes=64 * 1024)
+        tid = ctx.register_w16(w)
+        ctx.set_placement([(tid, -1, where)])
+        y = torch.full((M, N), 7.0, dtype=torch.float16, device="cuda")
+        ctx.reset_stats()
+        ctx.linear(tid, H.to_dev(x), y, M)
+        ctx.sync()
+        st = ctx.stats()
+        if where == B.ATS_HOST:
+            assert st.streamed_bytes == nb and st.copies == -(-nb // (64 * 1024))
+        else:
+            assert st.streamed_bytes == 0 and st.resident_bytes == nb
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want, what=f"w16 gemv {N}x{K} M={M}")
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+
+
 def test_linear_closed_forms_on_gpu(B, torch):
     """One-hot activations return a weight column exactly; all-ones with unit scales return integer row sums."""
     N, K = 40, 256

@@ -364,3 +364,24 @@ def test_embed_and_lm_head_closed_forms():
     h = np.float64(np.float16(c / np.sqrt(c * c + eps)))  # the normalised magnitude, rounded to fp16 as the contract says
     want = (codes * np.sign(x.astype(np.float64))).sum(axis=1) * h
     assert np.array_equal(np.asarray(logits, dtype=np.float64)[0], O.rn16(want))
+
+
+def test_linear_w16_exact_rational_and_special_cases():
+    """fp16 weights: against exact rational arithmetic on a small case; one-hot activations pick a column; a row of the
+    identity returns the activation; rounding of the standalone output happens once."""
+    from fractions import Fraction
+    rng = np.random.default_rng(9)
+    N, K, M = 5, 16, 3
+    w = rng.standard_normal((N, K)).astype(np.float16)
+    x = rng.standard_normal((M, K)).astype(np.float16)
+    got = O.linear_w16(x, w)
+    for m in range(M):
+        for n in range(N):
+            exact = sum(Fraction(float(w[n, k])) * Fraction(float(x[m, k])) for k in range(K))
+            assert abs(Fraction(float(got[m, n])) - exact) <= abs(exact) * Fraction(1, 2 ** 45) + Fraction(1, 2 ** 60)
+    e = np.zeros((1, K), dtype=np.float16)
+    e[0, 7] = 1
+    assert np.array_equal(O.linear_w16(e, w)[0], w[:, 7].astype(np.float64))
+    assert np.array_equal(O.linear_w16(x, np.eye(K, dtype=np.float16)), x.astype(np.float64))
+    y16 = O.linear_w16(x, w, round_out=True)
+    assert np.array_equal(y16, O.rn16(got))
