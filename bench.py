@@ -497,6 +497,48 @@ def extra_model_loop(torch, B, W, peaks, quick):
             "decode_frac_of_measured_hbm": weight_bytes / (dec_ms / gen * 1e-3) / 1e9 / peaks["hbm_gbs"], "logits_finite": finite}
 
 
+def extra_w16(torch, B, W, peaks, quick):
+    """Unquantized fp16 weight matrices (the format of the paper's FP16 model): the single-row GEMV against the HBM peak
+    (2 bytes per weight) and the TMA + tcgen05 GEMM, both operands by TMA, against the tensor peak."""
+    out = {"workload": "fp16 weights: GEMV (1 row) over rotated replicas, GEMM over 512 and 2048 rows"}
+    rng = np.random.default_rng(16)
+    for (N, K, reps) in ((4096, 4096, 16), (14336, 4096, 8)):
+        nb = N * K * 2
+        ctx = B.Context(reps * (nb + 4096) + (4 << 20), workspace_bytes=1 << 20)
+        w = (rng.standard_normal((N, K)) * 0.05).astype(np.float16)
+        ids = [ctx.register_w16(w) for _ in range(reps)]
+        ctx.set_placement([(t, -1, B.ATS_GPU) for t in ids])
+        x = torch.from_numpy(W.activations(16, 0, (1, K))).cuda()
+        y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+
+        def go(n):
+            for i in range(n):
+                ctx.linear(ids[i % reps], x, y, 1)
+        go(2 * reps)
+        ctx.sync()
+        n = (10 if quick else 40) * reps
+        us = event_time_ms(torch, ctx.compute, lambda: go(n)) * 1e3 / n
+        out[f"gemv_{N}x{K}"] = {"us_per_call": us, "gbs": nb / us / 1e3, "frac_of_measured_hbm": nb / us / 1e3 / peaks["hbm_gbs"]}
+        ctx.close()
+    for (N, K, T) in ((14336, 4096, 512), (14336, 4096, 2048)):
+        nb = N * K * 2
+        ws = 9 * T * N * 4 + (2 << 20)
+        ctx = B.Context(ws + nb + (4 << 20), workspace_bytes=ws)
+        tid = ctx.register_w16((rng.standard_normal((N, K)) * 0.05).astype(np.float16))
+        ctx.set_placement([(tid, -1, B.ATS_GPU)])
+        x = torch.from_numpy(W.activations(16, 1, (T, K))).cuda()
+        y = torch.empty((T, N), dtype=torch.float16, device="cuda")
+        for _ in range(3):
+            ctx.linear(tid, x, y, T)
+        ctx.sync()
+        n = 5 if quick else 20
+        ms = event_time_ms(torch, ctx.compute, lambda: [ctx.linear(tid, x, y, T) for _ in range(n)]) / n
+        tf = 2.0 * T * N * K / (ms * 1e-3) / 1e12
+        out[f"gemm_{N}x{K}_T{T}"] = {"us_per_call": ms * 1e3, "tflops": tf, "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"]}
+        ctx.close()
+    return out
+
+
 def extra_model_loop_moe(torch, B, W, peaks, quick):
     """Whole-model loop on an MoE layer shape (hidden 2048, 32 query / 4 kv heads of 128, 128 experts x SwiGLU 768, top-8):
     a stack of attention + routed-expert layers; a 512-token prompt prefilled in one chunk, then decode steps through every
@@ -579,7 +621,7 @@ def extra_model_loop_moe(torch, B, W, peaks, quick):
 
 
 STACK_LAYERS = [0]
-EXTRAS = {"model_loop_moe": extra_model_loop_moe, "model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
+EXTRAS = {"model_loop_moe": extra_model_loop_moe, "w16_formats": extra_w16, "model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
 
 
 def run_ours(args):
@@ -726,7 +768,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the figures of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--quick", action="store_true", help="smaller extras")
-    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe"],
+    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe", "w16_formats"],
                     help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
     ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = 8, or 4 with --quick; 32 = the full configuration)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")

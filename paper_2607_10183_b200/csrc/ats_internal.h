@@ -307,6 +307,7 @@ struct GemmParams {
   // grouped form (MoE prefill): the T activation rows are sorted by expert; expert e owns rows grp_off[e] .. grp_off[e+1]-1
   // and multiplies them with slice e of every segment (seg[i].base + e * grp_stride, or grp_tab[i][e] where a table is
   // given: device or mapped host addresses).  No split-K, no residual.
+  int w16;                  // seg[0].base is an unquantized fp16 matrix [n_rows][K] (one segment, no grouping)
   const int* grp_off;       // DEVICE [n_groups + 1]; null = plain GEMM
   int n_groups;
   int grp_max_rows;         // the largest expert's row count (sizes the grid)

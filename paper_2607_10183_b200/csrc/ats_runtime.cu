@@ -914,7 +914,26 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M)
       ATS_CUDA(launch_gemv_w16((const __half*)op.ptr, (int)t->d.n_out, (int)t->d.k_in, (const __half*)x, (int)t->d.k_in, (__half*)y,
                                (int)t->d.n_out, (int)M, ctx->cs, &ctx->stats.kernel_launches, pdl));
     } else {
-      return fail(ctx, ATS_ERR_UNSUPPORTED, "W16 tensors take M <= 8 rows");
+      GemmParams g{};
+      g.w16 = 1;
+      g.n_seg = 1;
+      g.seg[0] = GemvSeg{op.ptr, (int)t->d.n_out};
+      g.K = (int)t->d.k_in;
+      g.T = (int)M;
+      g.x = (const __half*)x;
+      g.ldx = (int)t->d.k_in;
+      g.y = (__half*)y;
+      g.ldy = (int)t->d.n_out;
+      g.status = ctx->dev_status;
+      g.pdl = pdl;
+      g.scratch_bytes = gemm_scratch_bytes((int)M, (int)t->d.n_out, (int)t->d.k_in);
+      if (g.scratch_bytes + kWsReserved > align_up(ctx->cfg.workspace_bytes))
+        return fail(ctx, ATS_ERR_NOMEM, "workspace too small for the GEMM: need %llu bytes",
+                    (unsigned long long)(g.scratch_bytes + kWsReserved));
+      g.scratch = ctx->ws + kWsReserved;
+      std::string err;
+      cudaError_t ce = launch_gemm(g, ctx->cs, &ctx->stats.kernel_launches, &err);
+      if (ce != cudaSuccess) return check_cuda(ctx, ce, err.empty() ? "launch_gemm (fp16 weights)" : err.c_str());
     }
     return release_ops(ctx, &op, 1);
   }

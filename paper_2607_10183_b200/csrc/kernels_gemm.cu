@@ -64,6 +64,7 @@ struct GemmKParams {
   __half* y2;
   // grouped form (one weight slice per expert, blockIdx.z = expert; splits = 1): expert e multiplies the activation rows
   // grp_off[e] .. grp_off[e+1]-1 (rows sorted by expert) with slice e of every segment and writes the same rows of y
+  int w16;  // the weights are an unquantized fp16 matrix (one segment): their tiles come by TMA, nothing is dequantized
   const int* grp_off;                 // DEVICE [n_experts + 1], null = the plain form
   unsigned long long grp_stride;      // bytes between the slices of consecutive experts (contiguous resident experts)
   const uint8_t* const* grp_tab[3];   // per segment: DEVICE table of slice addresses (device or mapped host memory), or null
@@ -166,7 +167,7 @@ __device__ __forceinline__ uint4 dequant8(uint32_t w, __half2 s2) {
 }
 
 template <int FT, int TT>
-__global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const GemmKParams p) {
+__global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap, const GemmKParams p) {
   using Cfg = TileCfg<FT, TT>;
   constexpr int BF = Cfg::BF, TTILE = TT, MB = TT / BM, kDequantWarps = Cfg::kDequantWarps, kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -232,7 +233,10 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) ge
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (activation tile)
     if (lane == 0) {
-      const uint32_t tx = (uint32_t)boxes * BOXR * BK * 2;
+      // fp16 weights: the weight tile of a stage is loaded like the activation tile (boxes of 64 rows x 64 k, rows past the
+      // matrix read as zeros) and counted on the same barrier
+      const int wboxes = p.w16 ? (nmma + BOXR - 1) / BOXR : 0;
+      const uint32_t tx = (uint32_t)(boxes + wboxes) * BOXR * BK * 2;
       for (int i = 0; i < nks; ++i) {
         const int s = i % S;
         if (i >= S && !mbar_wait(&empty[s], ((i / S) - 1) & 1)) {
@@ -243,6 +247,8 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) ge
         mbar_expect_tx(&full_b[s], tx);
         for (int b = 0; b < boxes; ++b)
           tma_load_2d(bdst + (size_t)b * BOXR * BK * 2, &xmap, (ks0 + i) * BK, rowoff + t0 + b * BOXR, &full_b[s]);
+        for (int b = 0; b < wboxes; ++b)
+          tma_load_2d(smem + (size_t)s * kStageBytes + (size_t)b * BOXR * BK * 2, &wmap, (ks0 + i) * BK, row0 + b * BOXR, &full_b[s]);
       }
     }
   } else if (warp == 1) {
@@ -258,7 +264,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) ge
       int s = 0;
       uint32_t par = 0;
       for (int i = 0; i < nks; ++i) {
-        if (!mbar_wait(&full_a[s], par) || !mbar_wait(&full_b[s], par)) {
+        if ((!p.w16 && !mbar_wait(&full_a[s], par)) || !mbar_wait(&full_b[s], par)) {
           fail_s = 1;
           ok = false;
           break;
@@ -324,7 +330,7 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) ge
       const uint32_t w = d == 0 ? v.x : d == 1 ? v.y : d == 2 ? v.z : v.w;
       return (w >> (16 * hb)) & 0xFFFFu;
     };
-    const int nks_dq = w2 < n_dq ? nks : 0;  // warps beyond the tile's width have no rows: they only take part in the epilogue
+    const int nks_dq = (w2 < n_dq && !p.w16) ? nks : 0;  // warps beyond the tile's width (and all of them with fp16 weights) have no rows to dequantize: they only take part in the epilogue
     if (vec_sc && nks_dq > 0) snext = fetch_scale8(ks0);
 #pragma unroll
     for (int d = 0; d < kPD; ++d) {
@@ -635,6 +641,21 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
     if (err) *err = "cuTensorMapEncodeTiled failed for the activation tile";
     return cudaErrorInvalidValue;
   }
+  CUtensorMap wmap = xmap;  // only read by the kernel when the weights are fp16
+  if (g.w16) {
+    if (g.n_seg != 1 || g.grp_off || ((uintptr_t)g.seg[0].base & 15) || (g.K % 8)) {
+      if (err) *err = "fp16 weights: one 16-byte aligned matrix with K a multiple of 8";
+      return cudaErrorInvalidValue;
+    }
+    const cuuint64_t wdims[2] = {(cuuint64_t)g.K, (cuuint64_t)g.seg[0].n_rows};
+    const cuuint64_t wstrides[1] = {(cuuint64_t)g.K * 2};
+    if (enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<uint8_t*>(g.seg[0].base), wdims, wstrides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+      if (err) *err = "cuTensorMapEncodeTiled failed for the weight tile";
+      return cudaErrorInvalidValue;
+    }
+  }
   int sm_count = 148;
   int dev = 0;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
@@ -672,6 +693,7 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   p.status = g.status;
   p.res = g.res;
   p.y2 = g.y2;
+  p.w16 = g.w16;
   p.grp_off = g.grp_off;
   p.grp_stride = g.grp_stride;
   for (int i = 0; i < 3; ++i) p.grp_tab[i] = g.grp_tab[i];
@@ -688,13 +710,13 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   if (wide) {
     using Cfg = TileCfg<2, 256>;
     p.stages = Cfg::kStages;
-    e = launch_dep(gemm_q4_kernel<2, 256>, grid, dim3(Cfg::kThreads), (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, p);
+    e = launch_dep(gemm_q4_kernel<2, 256>, grid, dim3(Cfg::kThreads), (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, wmap, p);
   } else {
     using Cfg = TileCfg<1, 128>;
     // Grouped form: every CTA streams its own expert's weights once and has few real rows, so what counts is how many
     // weight loads are in flight per SM: three stages let two CTAs share an SM (registers are capped for that).
     p.stages = g.grp_off ? 3 : Cfg::kStages;
-    e = launch_dep(gemm_q4_kernel<1, 128>, grid, dim3(Cfg::kThreads), (size_t)p.stages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, p);
+    e = launch_dep(gemm_q4_kernel<1, 128>, grid, dim3(Cfg::kThreads), (size_t)p.stages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, wmap, p);
   }
   if (e != cudaSuccess) return e;
   if (p.splits > 1) {

@@ -370,3 +370,28 @@ def test_moe_layer_with_attention_prefill_matches_oracle(B, torch, host_experts)
     kg = kd.cpu().numpy()
     assert np.max(np.abs(kg[:, pos0:pos0 + T].astype(np.float64) - kc[:, pos0:pos0 + T].astype(np.float64))) <= 4e-3 * np.max(np.abs(kc))
     ctx.close()
+
+
+@pytest.mark.parametrize("N,K,T", [(128, 64, 16), (136, 320, 127), (384, 1024, 129), (130, 96, 300), (1024, 4096, 512), (4096, 1024, 9)])
+def test_linear_w16_gemm_matches_oracle(B, torch, N, K, T):
+    """More than 8 rows against an unquantized fp16 weight matrix: the tcgen05 GEMM with the weight tile loaded by TMA
+    instead of dequantized; ragged N, K, T, split-K shapes; resident and streamed give the same bits."""
+    rng = np.random.default_rng(N * 7 + K * 3 + T)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float16)
+    x = W.activations(96, 0, (T, K))
+    want = O.linear_w16(x, w, round_out=True)
+    nb = N * K * 2
+    slot = -(-nb // 256) * 256
+    outs = []
+    for where in (B.ATS_GPU, B.ATS_HOST):
+        ws = 9 * T * N * 4 + 2 * MB
+        ctx = B.Context(ws + 2 * (slot + 256) + slot + MB, workspace_bytes=ws, ring_slots=2, slot_bytes=slot, chunk_bytes=MB)
+        tid = ctx.register_w16(w)
+        ctx.set_placement([(tid, -1, where)])
+        y = torch.full((T, N), 7.0, dtype=torch.float16, device="cuda")
+        ctx.linear(tid, H.to_dev(x), y, T)
+        ctx.sync()
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want, what=f"w16 gemm {N}x{K} T={T}")
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
