@@ -311,6 +311,11 @@ int32_t ats_host_solve_placement(const int64_t* s, const int64_t* r, const int64
                                  int64_t M, uint8_t* out_b, int64_t* out_objective);
 /* Interchange layout -> the library's internal slice layout (n_out*k_in/2 code bytes followed by n_out*k_in/32 fp16
  * scales) and back; out_* are HOST buffers of the same sizes as the inputs.  The round trip is the identity. */
+/* The row order of the MoE prefill's grouped GEMMs (host only): the stable sort of the P (token, slot) pairs by expert id.
+ * ids[p] in [0, E); order[r] = the pair at sorted position r; pos[p] = the sorted position of pair p; off[e] = first
+ * position of expert e, off[E] = P; *max_rows = the largest expert's row count.  ATS_ERR_INVALID for an id out of range. */
+int32_t ats_host_group_pairs(const int32_t* ids, uint32_t P, uint32_t E, int32_t* order, int32_t* pos, int32_t* off,
+                             int32_t* max_rows);
 int32_t ats_host_repack_q4(const void* codes, const void* scales, void* out_slice, uint32_t n_out, uint32_t k_in);
 int32_t ats_host_unpack_q4(const void* slice, void* out_codes, void* out_scales, uint32_t n_out, uint32_t k_in);
 

@@ -31,7 +31,7 @@ EXPORTS = (
     "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode", "ats_layer_decode_host", "ats_embed", "ats_lm_head",
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
     "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
-    "ats_host_unpack_q4",
+    "ats_host_unpack_q4", "ats_host_group_pairs",
 )
 
 
@@ -99,6 +99,7 @@ def _load():
         "ats_host_solve_placement": (i32, [vp, vp, vp, vp, u32, C.c_int64, vp, P(C.c_int64)]),
         "ats_host_repack_q4": (i32, [vp, vp, vp, u32, u32]),
         "ats_host_unpack_q4": (i32, [vp, vp, vp, u32, u32]),
+        "ats_host_group_pairs": (i32, [vp, u32, u32, vp, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -303,6 +304,18 @@ class Context:
 
 def workspace_bytes(desc: ats_layer_desc, max_tokens: int) -> int:
     return int(lib.ats_workspace_bytes(C.byref(desc), max_tokens))
+
+
+def host_group_pairs(ids, E):
+    """Stable sort of (token, slot) pairs by expert (host only).  Returns (order, pos, off, max_rows)."""
+    ids = np.ascontiguousarray(ids, dtype=np.int32).reshape(-1)
+    P = ids.size
+    order, pos, off = np.zeros(P, np.int32), np.zeros(P, np.int32), np.zeros(E + 1, np.int32)
+    mx = C.c_int32()
+    st = lib.ats_host_group_pairs(ids.ctypes.data, P, E, order.ctypes.data, pos.ctypes.data, off.ctypes.data, C.byref(mx))
+    if st != ATS_OK:
+        raise AtsError(st, "ats_host_group_pairs")
+    return order, pos, off, mx.value
 
 
 def host_solve_placement(s, r, c, M, is_expert=None):

@@ -1521,19 +1521,9 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     int32_t* order_h = ctx->ids_host + kMaxPairs;       // sorted position -> pair
     int32_t* pos_h = ctx->ids_host + 2 * kMaxPairs;     // pair -> sorted position
     int32_t* off_h = ctx->ids_host + 3 * kMaxPairs;     // expert -> first sorted position; [E] = P
-    std::vector<int> cnt(E + 1, 0);
-    for (int p2 = 0; p2 < P; ++p2) cnt[ctx->ids_host[p2] + 1]++;
     int max_rows = 0;
-    for (int e = 0; e < E; ++e) {
-      max_rows = std::max(max_rows, cnt[e + 1]);
-      cnt[e + 1] += cnt[e];
-    }
-    for (int e = 0; e <= E; ++e) off_h[e] = cnt[e];
-    for (int p2 = 0; p2 < P; ++p2) {  // stable: pairs of an expert keep their (token, slot) order
-      const int r = cnt[ctx->ids_host[p2]]++;
-      order_h[r] = p2;
-      pos_h[p2] = r;
-    }
+    if (ats_host_group_pairs(ctx->ids_host, (uint32_t)P, (uint32_t)E, order_h, pos_h, off_h, &max_rows) != ATS_OK)
+      return fail(ctx, ATS_ERR_INVALID, "routing ids out of range");
     ATS_CUDA(cudaMemcpyAsync(w.order, order_h, (size_t)P * 4, cudaMemcpyHostToDevice, ctx->cs));
     ATS_CUDA(cudaMemcpyAsync(w.pos, pos_h, (size_t)P * 4, cudaMemcpyHostToDevice, ctx->cs));
     ATS_CUDA(cudaMemcpyAsync(w.grp_off, off_h, (size_t)(E + 1) * 4, cudaMemcpyHostToDevice, ctx->cs));

@@ -168,6 +168,29 @@ int32_t ats_host_solve_placement(const int64_t* s, const int64_t* r, const int64
   return ATS_OK;
 }
 
+int32_t ats_host_group_pairs(const int32_t* ids, uint32_t P, uint32_t E, int32_t* order, int32_t* pos, int32_t* off,
+                             int32_t* max_rows) {
+  if (!ids || !order || !pos || !off || !max_rows || E == 0) return ATS_ERR_INVALID;
+  std::vector<int32_t> cnt((size_t)E + 1, 0);
+  for (uint32_t p = 0; p < P; ++p) {
+    if (ids[p] < 0 || (uint32_t)ids[p] >= E) return ATS_ERR_INVALID;
+    cnt[(size_t)ids[p] + 1]++;
+  }
+  int32_t mx = 0;
+  for (uint32_t e = 0; e < E; ++e) {
+    mx = std::max(mx, cnt[e + 1]);
+    cnt[e + 1] += cnt[e];
+  }
+  for (uint32_t e = 0; e <= E; ++e) off[e] = cnt[e];
+  for (uint32_t p = 0; p < P; ++p) {  // stable: pairs of an expert keep their (token, slot) order
+    const int32_t r = cnt[ids[p]]++;
+    order[r] = (int32_t)p;
+    pos[p] = r;
+  }
+  *max_rows = mx;
+  return ATS_OK;
+}
+
 int32_t ats_host_repack_q4(const void* codes, const void* scales, void* out_slice, uint32_t n_out, uint32_t k_in) {
   if (!codes || !scales || !out_slice) return ATS_ERR_INVALID;
   if (k_in % ats::kBlock || n_out == 0 || k_in == 0) return ATS_ERR_SHAPE;

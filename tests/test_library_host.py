@@ -4,6 +4,7 @@ import os
 import re
 
 import numpy as np
+import pytest
 
 from oracle import ats_oracle as O
 from paper_2607_10183_b200 import workloads as W
@@ -73,3 +74,23 @@ def test_repack_round_trip_is_identity():
     assert np.array_equal(p2, packed) and np.array_equal(s2.view(np.uint16), scales.view(np.uint16))
     assert not np.array_equal(sl[:packed.size].reshape(packed.shape), packed)  # the internal order differs
     assert B.ats_host_repack_q4(packed.ctypes.data, scales.ctypes.data, sl.ctypes.data, 37, 40) == B.ATS_ERR_SHAPE
+
+
+def test_group_pairs_is_the_stable_sort_by_expert():
+    """Row order of the MoE prefill: against numpy's stable argsort, incl. empty experts, one expert taking everything,
+    no pairs at all, and an id out of range."""
+    from paper_2607_10183_b200 import binding as B
+    rng = np.random.default_rng(4)
+    for P, E in ((0, 4), (1, 1), (37, 5), (4096, 128), (300, 1024)):
+        ids = rng.integers(0, E, size=P, dtype=np.int32)
+        if P == 37:
+            ids[:] = 3  # one expert takes every row
+        order, pos, off, mx = B.host_group_pairs(ids, E)
+        want = np.argsort(ids, kind="stable").astype(np.int32)
+        assert np.array_equal(order, want)
+        assert np.array_equal(pos[order], np.arange(P, dtype=np.int32))
+        cnt = np.bincount(ids, minlength=E)
+        assert np.array_equal(off, np.concatenate(([0], np.cumsum(cnt))).astype(np.int32))
+        assert mx == (cnt.max() if P else 0)
+    with pytest.raises(B.AtsError):
+        B.host_group_pairs(np.array([0, 7], dtype=np.int32), 7)
