@@ -134,12 +134,12 @@ int32_t ats_tensor_slice_bytes(const ats_ctx* ctx, int32_t id, uint64_t* out_byt
 int32_t ats_set_placement(ats_ctx* ctx, const int32_t* ids /*HOST*/, const int32_t* experts /*HOST*/,
                           const uint8_t* where /*HOST*/, uint32_t n);
 
-/* Algorithm 1 (static tensor placement): knapsack DP over the registered Q4B32 tensors in registration order with
+/* Algorithm 1 (static tensor placement): knapsack DP over the registered weight tensors (Q4B32 and W16) in registration order with
  * sizes s_i = ceil(bytes/granule), budget M = floor(budget_bytes/granule), values r_i and switch costs c_i;
  * for a model with expert tensors the expert / non-expert partition rule of Algorithm 1 applies (a stacked expert
  * tensor is one item).  granule_bytes = 0 selects 1 MiB (the paper quantizes at MB granularity).
- * Applies the result like ats_set_placement and writes one ATS_HOST/ATS_GPU byte per Q4B32 tensor (registration
- * order) to out_where[0..n) if non-null; n must then equal the number of Q4B32 tensors. */
+ * Applies the result like ats_set_placement and writes one ATS_HOST/ATS_GPU byte per weight tensor (registration
+ * order) to out_where[0..n) if non-null; n must then equal the number of weight tensors. */
 int32_t ats_plan_placement(ats_ctx* ctx, uint64_t budget_bytes, uint32_t granule_bytes, uint8_t* out_where /*HOST*/,
                            uint32_t n);
 int32_t ats_get_placement(const ats_ctx* ctx, int32_t id, int32_t expert, uint8_t* out_where /*HOST*/);

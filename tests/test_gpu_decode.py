@@ -232,6 +232,45 @@ def test_linear_w16_gemv_matches_oracle(B, torch, N, K, M):
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
 
 
+def test_plan_placement_over_mixed_formats(B, torch):
+    """Algorithm 1 sees quantized and fp16 weight tensors alike (sizes in granules, values = bytes): the library's vector
+    equals the oracle's on the same numbers, and the placed tensors compute the same bits as an all-resident run."""
+    rng = np.random.default_rng(21)
+    shapes = [("q4", 512, 1024), ("w16", 256, 512), ("q4", 1024, 512), ("w16", 512, 512), ("q4", 256, 256)]
+    G = 64 * 1024
+    data, nbytes = [], []
+    for kind, N, K in shapes:
+        if kind == "q4":
+            data.append(W.q4_packed(95, len(data), W.ROLE_Q, N, K))
+            nbytes.append(W.q4_bytes(N, K))
+        else:
+            data.append((rng.standard_normal((N, K)) * 0.05).astype(np.float16))
+            nbytes.append(N * K * 2)
+    budget = int(0.55 * sum(nbytes))
+    slot = max(-(-b // 256) * 256 for b in nbytes)
+    outs = {}
+    for mode in ("all", "plan"):
+        ctx = make_ctx(B, sum(nbytes) + 4096 * len(nbytes), ring_slots=2, slot_bytes=slot, chunk_bytes=64 * 1024)
+        ids = [ctx.register_q4(*d) if k[0] == "q4" else ctx.register_w16(d) for k, d in zip(shapes, data)]
+        if mode == "all":
+            ctx.set_placement([(t, -1, B.ATS_GPU) for t in ids])
+        else:
+            got = ctx.plan_placement(budget, len(ids), G)
+            want = O.static_placement(O.size_units(nbytes, G), nbytes, [0] * len(ids), O.budget_units(budget, G))
+            assert list(got) == list(want) and 0 < sum(got) < len(ids)
+        ys = []
+        for t, (kind, N, K) in zip(ids, shapes):
+            x = W.activations(95, 1, (1, K))
+            y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+            ctx.linear(t, H.to_dev(x), y, 1)
+            ctx.sync()
+            ys.append(y.cpu().numpy())
+        outs[mode] = ys
+        ctx.close()
+    for a, b in zip(outs["all"], outs["plan"]):
+        assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+
+
 def test_linear_closed_forms_on_gpu(B, torch):
     """One-hot activations return a weight column exactly; all-ones with unit scales return integer row sums."""
     N, K = 40, 256
