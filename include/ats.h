@@ -54,7 +54,11 @@ enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1, ATS_FMT_W16 = 2 };
 /* F16: small auxiliary tensors (router weight [k_in][n_out], norm gain [n_out]): always resident, no placement.
  * W16: an unquantized fp16 weight matrix [n_out][k_in] (the paper runs one of its models with FP16 weights, Section 5.1):
  * a dense tensor (n_experts = 1, k_in a multiple of 8) placed and streamed like a Q4B32 tensor (2 bytes per weight);
- * ats_linear takes it; the layer calls, ats_moe_linear and ats_dequantize take Q4B32 tensors only. */
+ * ats_linear and ats_lm_head take it, and so do ats_layer_decode / ats_layer_decode_host / ats_layer_prefill for a dense
+ * layer whose seven matrices are all W16 (mixed formats within a layer: ATS_ERR_INVALID; MoE layers: Q4B32 experts only;
+ * fp32 accumulation, the same roundings between operators as the quantized layer; the norm runs as a launch of its
+ * own and fused groups (QKV, gate|up) become one GEMV launch or one GEMM per matrix).  ats_moe_linear, ats_embed and
+ * ats_dequantize take Q4B32 tensors only. */
 enum { ATS_OUT_F32 = 0, ATS_OUT_F16 = 1 };      /* ats_dequantize output */
 enum { ATS_MODE_DECODE = 0, ATS_MODE_PREFILL = 1 };
 
@@ -286,7 +290,8 @@ int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n);
  * ats_lm_head: logits = W_head * RMSNorm(x; norm_id gain, eps), x DEVICE fp16 [M][hidden], logits DEVICE fp16 [M][vocab];
  * the normalised row is rounded to fp16 before the product (the contract's edge "h").  M = 1 runs as one launch of the
  * streaming GEMV with the norm as its prologue (hidden <= 4096 and a shape that kernel takes); otherwise a norm launch
- * into `scratch` (DEVICE fp16 [M][hidden], caller-provided, may be NULL only for the one-launch case) and ats_linear. */
+ * into `scratch` (DEVICE fp16 [M][hidden], caller-provided, may be NULL only for the one-launch case) and ats_linear.
+ * A W16 head always takes the second form (scratch required). */
 int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids /*DEVICE*/, uint32_t M, void* out /*DEVICE*/);
 int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, const void* x /*DEVICE*/, void* logits /*DEVICE*/,
                     uint32_t M, void* scratch /*DEVICE*/);

@@ -106,6 +106,14 @@ def linear_w16(x: np.ndarray, w16: np.ndarray, round_out: bool = False) -> np.nd
     return rn16(y) if round_out else y
 
 
+def apply_weight(x, w, weight_mode: int = WEIGHT_EXACT) -> np.ndarray:
+    """The per-tensor operator for a layer's weight given either as (packed, scales) (block-quantized) or as a
+    1-tuple (w16,) holding an unquantized fp16 matrix."""
+    if len(w) == 1:
+        return linear_w16(x, w[0])
+    return linear(x, w[0], w[1], weight_mode)
+
+
 # --------------------------------------------------------------------------------------
 # a6: layer glue
 # --------------------------------------------------------------------------------------
@@ -181,10 +189,10 @@ def silu(z):
 
 def swiglu_ffn(h2, w_gate, w_up, w_down, edges, weight_mode):
     """d = W_down (silu(W_gate h2) * (W_up h2)) with the contract's roundings."""
-    g = _edge(linear(h2, *w_gate, weight_mode), "g", edges)
-    u = _edge(linear(h2, *w_up, weight_mode), "u", edges)
+    g = _edge(apply_weight(h2, w_gate, weight_mode), "g", edges)
+    u = _edge(apply_weight(h2, w_up, weight_mode), "u", edges)
     act = _edge(silu(g) * u, "act", edges)
-    return _edge(linear(act, *w_down, weight_mode), "d", edges)
+    return _edge(apply_weight(act, w_down, weight_mode), "d", edges)
 
 
 def attention_block(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.ndarray, pos0: int,
@@ -201,9 +209,9 @@ def attention_block(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.nd
     T = x.shape[0]
     nq, nkv, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     h = _edge(rmsnorm(x, tensors["attn_norm"], shape.rms_eps), "h", edges)
-    q = _edge(linear(h, *tensors["wq"], weight_mode), "q", edges).reshape(T, nq, d)
-    k = _edge(linear(h, *tensors["wk"], weight_mode), "k", edges).reshape(T, nkv, d)
-    v = _edge(linear(h, *tensors["wv"], weight_mode), "v", edges).reshape(T, nkv, d)
+    q = _edge(apply_weight(h, tensors["wq"], weight_mode), "q", edges).reshape(T, nq, d)
+    k = _edge(apply_weight(h, tensors["wk"], weight_mode), "k", edges).reshape(T, nkv, d)
+    v = _edge(apply_weight(h, tensors["wv"], weight_mode), "v", edges).reshape(T, nkv, d)
     pos = (pos0 + np.arange(T, dtype=np.float64)).reshape(T, 1)
     q_rot = _edge(rope(q, pos, shape.rope_theta), "q_rot", edges)
     k_rot = rope(k, pos, shape.rope_theta)
@@ -214,7 +222,7 @@ def attention_block(x, tensors: dict, shape, k_cache: np.ndarray, v_cache: np.nd
     for t in range(T):
         a[t] = attention_one(q_rot[t], k_cache, v_cache, pos0 + t + 1).reshape(-1)
     a = _edge(a, "a", edges)
-    o = _edge(linear(a, *tensors["wo"], weight_mode), "o", edges)
+    o = _edge(apply_weight(a, tensors["wo"], weight_mode), "o", edges)
     return _edge(x + o, "x1", edges)
 
 

@@ -146,11 +146,12 @@ struct GemvParams {
   float norm_eps;
   __half* norm_out;
   int pdl;  // allow the launch to overlap the tail of the preceding kernel (programmatic dependent launch)
+  int w16;  // the segments are unquantized fp16 matrices [n_rows][K] (launch_gemv_w16; no norm prologue)
 };
 cudaError_t launch_gemv(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
-// fp16-weight GEMV (kernels_decode.cu): y16[m][n] = rn16(sum_k W[n][k] x[m][k]), M <= 8, K a multiple of 8
-cudaError_t launch_gemv_w16(const __half* W, int N, int K, const __half* x, int ldx, __half* y, int ldy, int M, cudaStream_t st,
-                            uint64_t* n_launch, int pdl = 0);
+// fp16-weight GEMV (kernels_decode.cu): the same segments, epilogue modes and fp32 accumulation as launch_gemv over
+// unquantized fp16 matrices; M <= 8, K a multiple of 8, x given (the norm prologue fields are ignored)
+cudaError_t launch_gemv_w16(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
 // the streaming single-token kernel (kernels_gemv_stream.cu): shapes it accepts, and its launcher
 bool gemv_stream_eligible(const GemvParams& p);
 cudaError_t launch_gemv_stream(const GemvParams& p, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch);

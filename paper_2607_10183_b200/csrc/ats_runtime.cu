@@ -79,7 +79,8 @@ static uint64_t gemv_work_bytes(const GemvParams& p) {
   const uint64_t K = (uint64_t)p.K, M = (uint64_t)p.M;
   const uint64_t out_rows = p.mode == GEMV_SWIGLU_F16 ? rows / 2 : rows;
   const uint64_t out_b = (p.mode == GEMV_OUT_F32 || p.mode == GEMV_RES16_OUT_F32) ? 4 : 2;
-  return rows * K / 2 + rows * (K / 32) * 2 + M * K * 2 + M * out_rows * out_b;
+  const uint64_t w_bytes = p.w16 ? rows * K * 2 : rows * K / 2 + rows * (K / 32) * 2;
+  return w_bytes + M * K * 2 + M * out_rows * out_b;
 }
 
 static int32_t precheck(ats_ctx* ctx, bool need_placement) {
@@ -242,7 +243,7 @@ static int count_streamed(const Operand* ops, int n) {
 // RMSNorm launch when a norm prologue was asked for).  Which kernel runs depends on shapes only, never on placement.
 static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
   p.pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
-  if (gemv_stream_eligible(p)) {
+  if (!p.w16 && gemv_stream_eligible(p)) {
     TimedLaunch tl(ctx, 0, gemv_work_bytes(p));
     ATS_CUDA(launch_gemv_stream(p, ctx->dev_status, ctx->sm_count, ctx->cs, &ctx->stats.kernel_launches));
     return ATS_OK;
@@ -255,7 +256,10 @@ static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
     p.norm_gain = nullptr;
   }
   TimedLaunch tl(ctx, 0, gemv_work_bytes(p));
-  ATS_CUDA(launch_gemv(p, ctx->cs, &ctx->stats.kernel_launches));
+  if (p.w16)
+    ATS_CUDA(launch_gemv_w16(p, ctx->cs, &ctx->stats.kernel_launches));
+  else
+    ATS_CUDA(launch_gemv(p, ctx->cs, &ctx->stats.kernel_launches));
   return ATS_OK;
 }
 
@@ -263,6 +267,7 @@ static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
 // the group at once the segments run one by one (same per-row arithmetic, so results do not depend on it).
 static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
   p.K = (int)ops[0].t->d.k_in;
+  p.w16 = ops[0].t->d.fmt == ATS_FMT_W16;  // a group shares one format (check_layer)
   if (count_streamed(ops, n) <= (int)ctx->cfg.ring_slots || n == 1) {
     ATS_TRY(acquire_ops(ctx, ops, n));
     p.n_seg = n;
@@ -292,8 +297,10 @@ static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
 static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
   p.K = (int)ops[0].t->d.k_in;
   p.status = ctx->dev_status;
+  p.w16 = ops[0].t->d.fmt == ATS_FMT_W16;  // a group shares one format (check_layer)
   std::string err;
-  if (count_streamed(ops, n) <= (int)ctx->cfg.ring_slots || n == 1) {
+  // fp16 weight tiles come through one tensor map per matrix: such a group always runs matrix by matrix
+  if ((count_streamed(ops, n) <= (int)ctx->cfg.ring_slots && !p.w16) || n == 1) {
     ATS_TRY(acquire_ops(ctx, ops, n));
     p.n_seg = n;
     uint64_t rows = 0;
@@ -907,36 +914,6 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M)
   Operand op;
   plan_dense(ctx, id, &op);
   ATS_TRY(pump(ctx));
-  if (t->d.fmt == ATS_FMT_W16) {
-    const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
-    ATS_TRY(acquire_ops(ctx, &op, 1));
-    if (M <= 8) {
-      ATS_CUDA(launch_gemv_w16((const __half*)op.ptr, (int)t->d.n_out, (int)t->d.k_in, (const __half*)x, (int)t->d.k_in, (__half*)y,
-                               (int)t->d.n_out, (int)M, ctx->cs, &ctx->stats.kernel_launches, pdl));
-    } else {
-      GemmParams g{};
-      g.w16 = 1;
-      g.n_seg = 1;
-      g.seg[0] = GemvSeg{op.ptr, (int)t->d.n_out};
-      g.K = (int)t->d.k_in;
-      g.T = (int)M;
-      g.x = (const __half*)x;
-      g.ldx = (int)t->d.k_in;
-      g.y = (__half*)y;
-      g.ldy = (int)t->d.n_out;
-      g.status = ctx->dev_status;
-      g.pdl = pdl;
-      g.scratch_bytes = gemm_scratch_bytes((int)M, (int)t->d.n_out, (int)t->d.k_in);
-      if (g.scratch_bytes + kWsReserved > align_up(ctx->cfg.workspace_bytes))
-        return fail(ctx, ATS_ERR_NOMEM, "workspace too small for the GEMM: need %llu bytes",
-                    (unsigned long long)(g.scratch_bytes + kWsReserved));
-      g.scratch = ctx->ws + kWsReserved;
-      std::string err;
-      cudaError_t ce = launch_gemm(g, ctx->cs, &ctx->stats.kernel_launches, &err);
-      if (ce != cudaSuccess) return check_cuda(ctx, ce, err.empty() ? "launch_gemm (fp16 weights)" : err.c_str());
-    }
-    return release_ops(ctx, &op, 1);
-  }
   if (M <= 8) {
     GemvParams p{};
     p.M = (int)M;
@@ -991,8 +968,8 @@ int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids, uint32_t M
 
 int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, const void* x, void* logits, uint32_t M, void* scratch) {
   ATS_TRY(precheck(ctx, true));
-  Tensor* t = get_tensor(ctx, head_id, ATS_FMT_Q4B32);
-  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", head_id);
+  Tensor* t = get_weight(ctx, head_id);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense weight tensor", head_id);
   ATS_TRY(check_f16(ctx, norm_id, t->d.k_in, 1, "final norm"));
   if (!x || !logits) return fail(ctx, ATS_ERR_INVALID, "null pointer");
   if (M == 0) return ATS_OK;
@@ -1014,7 +991,7 @@ int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, c
     probe.K = K;
     probe.n_seg = 1;
     probe.seg[0] = GemvSeg{nullptr, N};
-    if (!scratch && !gemv_stream_eligible(probe))
+    if (!scratch && (t->d.fmt == ATS_FMT_W16 || !gemv_stream_eligible(probe)))
       return fail(ctx, ATS_ERR_INVALID, "ats_lm_head needs `scratch` for this shape (the norm runs as a launch of its own)");
     plan_begin(ctx);
     Operand op;
@@ -1129,9 +1106,12 @@ int32_t ats_moe_linear(ats_ctx* ctx, int32_t id, const void* x, const int32_t* i
   return run_moe_stage(ctx, id, -1, ids_dev, ids_host, p);
 }
 
-static int32_t check_q4(ats_ctx* ctx, int32_t id, uint32_t n_out, uint32_t k_in, uint32_t n_experts, const char* name) {
-  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
-  if (!t) return fail(ctx, ATS_ERR_INVALID, "layer tensor %s (id %d) is not a registered Q4B32 tensor", name, id);
+// A layer's weight matrices share one format: Q4B32 (dense or stacked experts) or, for dense layers, fp16 (W16).
+static int32_t check_q4(ats_ctx* ctx, int32_t id, uint32_t fmt, uint32_t n_out, uint32_t k_in, uint32_t n_experts, const char* name) {
+  Tensor* t = get_tensor(ctx, id, fmt);
+  if (!t)
+    return fail(ctx, ATS_ERR_INVALID, "layer tensor %s (id %d) is not a registered %s tensor (a layer's weight matrices share one format)",
+                name, id, fmt == ATS_FMT_W16 ? "W16" : "Q4B32");
   if (t->d.n_out != n_out || t->d.k_in != k_in || t->slices.size() != n_experts)
     return fail(ctx, ATS_ERR_SHAPE, "layer tensor %s is [%zu][%u][%u], the layer needs [%u][%u][%u]", name, t->slices.size(),
                 t->d.n_out, t->d.k_in, n_experts, n_out, k_in);
@@ -1150,16 +1130,20 @@ static int32_t check_layer(ats_ctx* ctx, const ats_layer_desc* L, bool prefill) 
   if (!L) return fail(ctx, ATS_ERR_INVALID, "null layer descriptor");
   if (L->hidden == 0 || L->ffn == 0) return fail(ctx, ATS_ERR_SHAPE, "zero hidden/ffn size");
   if (L->hidden % 32 || L->ffn % 32) return fail(ctx, ATS_ERR_SHAPE, "hidden and ffn must be multiples of 32");
+  // the format of w_gate decides: every other matrix of the layer must have it too
+  uint32_t fmt = ATS_FMT_Q4B32;
+  if (Tensor* tg = get_weight(ctx, L->w_gate)) fmt = tg->d.fmt;
+  if (fmt == ATS_FMT_W16 && L->n_experts) return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE layers take Q4B32 expert tensors");
   if (L->wq >= 0) {
     if (L->head_dim != 64 && L->head_dim != 128) return fail(ctx, ATS_ERR_UNSUPPORTED, "head_dim %u (64 or 128)", L->head_dim);
     if (L->n_kv_heads == 0 || L->n_q_heads % L->n_kv_heads) return fail(ctx, ATS_ERR_SHAPE, "n_q_heads %% n_kv_heads != 0");
     if (L->n_q_heads / L->n_kv_heads > 8) return fail(ctx, ATS_ERR_UNSUPPORTED, "more than 8 query heads per kv head");
     const uint32_t qd = L->n_q_heads * L->head_dim, kvd = L->n_kv_heads * L->head_dim;
     ATS_TRY(check_f16(ctx, L->attn_norm, L->hidden, 1, "attn_norm"));
-    ATS_TRY(check_q4(ctx, L->wq, qd, L->hidden, 1, "wq"));
-    ATS_TRY(check_q4(ctx, L->wk, kvd, L->hidden, 1, "wk"));
-    ATS_TRY(check_q4(ctx, L->wv, kvd, L->hidden, 1, "wv"));
-    ATS_TRY(check_q4(ctx, L->wo, L->hidden, qd, 1, "wo"));
+    ATS_TRY(check_q4(ctx, L->wq, fmt, qd, L->hidden, 1, "wq"));
+    ATS_TRY(check_q4(ctx, L->wk, fmt, kvd, L->hidden, 1, "wk"));
+    ATS_TRY(check_q4(ctx, L->wv, fmt, kvd, L->hidden, 1, "wv"));
+    ATS_TRY(check_q4(ctx, L->wo, fmt, L->hidden, qd, 1, "wo"));
     if (L->kv_capacity == 0) return fail(ctx, ATS_ERR_SHAPE, "kv_capacity is 0");
     if (!prefill && (L->kv_capacity > 131072 || L->n_q_heads > 192))
       return fail(ctx, ATS_ERR_UNSUPPORTED, "decode attention supports kv_capacity <= 131072 and <= 192 query heads");
@@ -1171,9 +1155,9 @@ static int32_t check_layer(ats_ctx* ctx, const ats_layer_desc* L, bool prefill) 
       return fail(ctx, ATS_ERR_SHAPE, "top_k %u of %u experts unsupported", L->top_k, L->n_experts);
     ATS_TRY(check_f16(ctx, L->router, L->n_experts, L->hidden, "router"));
   }
-  ATS_TRY(check_q4(ctx, L->w_gate, L->ffn, L->hidden, E, "w_gate"));
-  ATS_TRY(check_q4(ctx, L->w_up, L->ffn, L->hidden, E, "w_up"));
-  ATS_TRY(check_q4(ctx, L->w_down, L->hidden, L->ffn, E, "w_down"));
+  ATS_TRY(check_q4(ctx, L->w_gate, fmt, L->ffn, L->hidden, E, "w_gate"));
+  ATS_TRY(check_q4(ctx, L->w_up, fmt, L->ffn, L->hidden, E, "w_up"));
+  ATS_TRY(check_q4(ctx, L->w_down, fmt, L->hidden, L->ffn, E, "w_down"));
   return ATS_OK;
 }
 

@@ -129,18 +129,48 @@ cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, i
 }
 
 // ------------------------------------------------------------------------------------------- fp16-weight GEMV
-// y[m][n] = rn16(sum_k W[n][k] x[m][k]) for an unquantized fp16 matrix W [N][K], M <= 8 rows of x.  HBM-bound at 2 bytes per
-// weight: a warp owns two rows at a time, its lanes walk K in 16-byte pieces with eight weight loads in flight per thread
-// (streaming loads: every weight is used once); x comes through L1.  Products of fp16 values are exact in fp32; sums in
-// fp32, lanes combined by shuffles in fixed order.
+// The per-tensor operator for unquantized fp16 matrices W [N][K], M <= 8 rows of x, with the epilogues of the quantized
+// GEMV (plain, + residual, SwiGLU of two matrices) and up to three matrices side by side (fused QKV).  HBM-bound at 2 bytes
+// per weight: a warp owns two weight rows at a time (two outputs; for SwiGLU the gate row and the up row of one output), its
+// lanes walk K in 16-byte pieces with eight weight loads in flight per thread (streaming loads: every weight is used once); x
+// comes through L1.  Products of fp16 values are exact in fp32; sums in fp32, lanes combined by shuffles in fixed order.
+struct W16Params {
+  const __half* w[3];
+  int n_rows[3];
+  int n_seg, K, mode;
+  const __half* x;
+  int ldx;
+  float* y32;
+  __half* y16;
+  int ldy;
+  const float* res32;
+  const __half* res16;
+  int ldres;
+  int ksplit;  // warps that share one pair of rows, each on its own part of K: 1, 2, 4 or 8
+};
 template <int M>
-__global__ void __launch_bounds__(256) gemv_w16_kernel(const __half* __restrict__ W, int N, int K, const __half* __restrict__ x, int ldx,
-                                                       __half* __restrict__ y, int ldy) {
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // x comes from the preceding kernel
+__global__ void __launch_bounds__(256) gemv_w16_kernel(const W16Params p) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const int lane = threadIdx.x & 31;
-  const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), n_warps = gridDim.x * (blockDim.x >> 5);
-  const int nch = K / 8;  // 16-byte pieces per row
+  bool waited = false;  // x and the residual come from the preceding kernel; the first weight loads need not wait for it
+  __shared__ float red_s[8][2][M];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int K = p.K, nch = K / 8;  // 16-byte pieces per row
+  const bool sw = p.mode == GEMV_SWIGLU_F16;
+  int n_rows = 0;  // weight rows side by side (SwiGLU: outputs, each fed by one gate row and one up row)
+  if (sw) n_rows = p.n_rows[0];
+  else n_rows = p.n_rows[0] + (p.n_seg > 1 ? p.n_rows[1] : 0) + (p.n_seg > 2 ? p.n_rows[2] : 0);
+  auto row_ptr = [&](int r) {  // constant indices only: a runtime index would move the parameters to local memory
+    const __half* base = p.w[0];
+    if (p.n_seg > 1 && r >= p.n_rows[0]) {
+      r -= p.n_rows[0];
+      base = p.w[1];
+      if (p.n_seg > 2 && r >= p.n_rows[1]) {
+        r -= p.n_rows[1];
+        base = p.w[2];
+      }
+    }
+    return reinterpret_cast<const uint4*>(base + (size_t)r * K);
+  };
   auto dot8 = [](const uint4& a, const uint4& b, float acc) {
     const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
@@ -151,60 +181,125 @@ __global__ void __launch_bounds__(256) gemv_w16_kernel(const __half* __restrict_
     }
     return acc;
   };
-  for (int rp = warp; 2 * rp < N; rp += n_warps) {
-    const int r0 = 2 * rp, r1 = min(r0 + 1, N - 1);
-    const uint4* w0 = reinterpret_cast<const uint4*>(W + (size_t)r0 * K);
-    const uint4* w1 = reinterpret_cast<const uint4*>(W + (size_t)r1 * K);
+  // A unit is two weight rows: two neighbouring output rows, or the gate and up rows of one SwiGLU output.  `ksplit`
+  // warps share a unit, each taking one contiguous part of K (few rows would otherwise leave every warp a long serial
+  // walk with one batch of loads in flight at a time); the CTA's 8 warps hold 8 / ksplit units.
+  const int n_units = sw ? n_rows : (n_rows + 1) / 2;
+  const int ks = p.ksplit, upc = 8 / ks;  // units per CTA and round
+  const int part = w % ks, slot = w / ks;
+  const int per = (((nch + ks - 1) / ks) + 31) & ~31;  // pieces per part (whole 512-byte lines)
+  const int c_lo = part * per, c_hi = min(nch, c_lo + per);
+  for (int u0 = blockIdx.x * upc; u0 < n_units; u0 += gridDim.x * upc) {
+    const int u = u0 + slot;
+    const bool live = u < n_units;
+    const int r0 = sw ? u : 2 * u, r1 = sw ? u : min(r0 + 1, n_rows - 1);
     float acc[2][M];
 #pragma unroll
     for (int m = 0; m < M; ++m) acc[0][m] = acc[1][m] = 0.f;
-    for (int c0 = lane; c0 < nch; c0 += 128) {
-      uint4 a[4], b[4];
+    if (live) {
+      const uint4* w0 = sw ? reinterpret_cast<const uint4*>(p.w[0] + (size_t)r0 * K) : row_ptr(r0);
+      const uint4* w1 = sw ? reinterpret_cast<const uint4*>(p.w[1] + (size_t)r0 * K) : row_ptr(r1);
+      for (int c0 = c_lo + lane; c0 < c_hi; c0 += 128) {
+        uint4 a[4], b[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int c = c0 + 32 * u;
-        a[u] = c < nch ? __ldcs(w0 + c) : make_uint4(0, 0, 0, 0);
-        b[u] = c < nch ? __ldcs(w1 + c) : make_uint4(0, 0, 0, 0);
-      }
+        for (int i = 0; i < 4; ++i) {
+          const int c = c0 + 32 * i;
+          a[i] = c < c_hi ? __ldcs(w0 + c) : make_uint4(0, 0, 0, 0);
+          b[i] = c < c_hi ? __ldcs(w1 + c) : make_uint4(0, 0, 0, 0);
+        }
+        if (!waited) {
+          asm volatile("griddepcontrol.wait;" ::: "memory");
+          waited = true;
+        }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int c = c0 + 32 * u;
-        if (c < nch) {
+        for (int i = 0; i < 4; ++i) {
+          const int c = c0 + 32 * i;
+          if (c < c_hi) {
 #pragma unroll
-          for (int m = 0; m < M; ++m) {
-            const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * ldx) + c);
-            acc[0][m] = dot8(a[u], xv, acc[0][m]);
-            acc[1][m] = dot8(b[u], xv, acc[1][m]);
+            for (int m = 0; m < M; ++m) {
+              const uint4 xv = __ldg(reinterpret_cast<const uint4*>(p.x + (size_t)m * p.ldx) + c);
+              acc[0][m] = dot8(a[i], xv, acc[0][m]);
+              acc[1][m] = dot8(b[i], xv, acc[1][m]);
+            }
           }
         }
       }
+    }
+    if (!waited) {  // no piece for this lane
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      waited = true;
     }
 #pragma unroll
     for (int m = 0; m < M; ++m) {
       const float s0 = warp_sum(acc[0][m]), s1 = warp_sum(acc[1][m]);
       if (lane == 0) {
-        y[(size_t)m * ldy + r0] = __float2half_rn(s0);
-        if (r0 + 1 < N) y[(size_t)m * ldy + r0 + 1] = __float2half_rn(s1);
+        red_s[w][0][m] = s0;
+        red_s[w][1][m] = s1;
       }
     }
+    __syncthreads();
+    // one thread per (unit, row of the pair, activation row) adds the parts in fixed order and writes the output
+    if (threadIdx.x < upc * 2 * M) {
+      const int m = threadIdx.x % M, h = (threadIdx.x / M) & 1, sl = threadIdx.x / (2 * M);
+      const int uu = u0 + sl;
+      float s = 0.f, s_up = 0.f;
+      for (int q = 0; q < ks; ++q) {
+        s += red_s[sl * ks + q][sw ? 0 : h][m];
+        if (sw) s_up += red_s[sl * ks + q][1][m];
+      }
+      const int r = sw ? uu : 2 * uu + h;
+      if (uu < n_units && r < n_rows && !(sw && h)) {
+        const size_t o = (size_t)m * p.ldy + r, ro = (size_t)m * p.ldres + r;
+        switch (p.mode) {
+          case GEMV_OUT_F32: p.y32[o] = s; break;
+          case GEMV_OUT_F16: p.y16[o] = __float2half_rn(s); break;
+          case GEMV_RES16_OUT_F32: p.y32[o] = __half2float(p.res16[ro]) + s; break;
+          case GEMV_RES32_OUT_F16: p.y16[o] = __float2half_rn(p.res32[ro] + s); break;
+          case GEMV_RES16_OUT_F16: p.y16[o] = __float2half_rn(__half2float(p.res16[ro]) + s); break;
+          case GEMV_SWIGLU_F16: p.y16[o] = __float2half_rn(silu_mul(s, s_up)); break;
+          default: break;
+        }
+      }
+    }
+    __syncthreads();
   }
+  if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-cudaError_t launch_gemv_w16(const __half* W, int N, int K, const __half* x, int ldx, __half* y, int ldy, int M, cudaStream_t st,
-                            uint64_t* n_launch, int pdl) {
-  if (M < 1 || M > 8 || K % 8) return cudaErrorInvalidValue;
-  const int pairs = (N + 1) / 2;
-  const dim3 grid(std::max(1, std::min((pairs + 7) / 8, 148 * 8))), block(256);
+cudaError_t launch_gemv_w16(const GemvParams& g, cudaStream_t st, uint64_t* n_launch) {
+  if (g.M < 1 || g.M > 8 || g.K % 8 || g.n_seg < 1 || g.n_seg > 3) return cudaErrorInvalidValue;
+  W16Params p{};
+  int n_out = 0;
+  for (int s = 0; s < g.n_seg; ++s) {
+    p.w[s] = reinterpret_cast<const __half*>(g.seg[s].base);
+    p.n_rows[s] = g.seg[s].n_rows;
+    n_out += g.seg[s].n_rows;
+  }
+  if (g.mode == GEMV_SWIGLU_F16) {
+    if (g.n_seg != 2 || g.seg[0].n_rows != g.seg[1].n_rows) return cudaErrorInvalidValue;
+    n_out = g.seg[0].n_rows;
+  }
+  p.n_seg = g.n_seg; p.K = g.K; p.mode = g.mode;
+  p.x = g.x; p.ldx = g.ldx; p.y32 = g.y32; p.y16 = g.y16; p.ldy = g.ldy;
+  p.res32 = g.res32; p.res16 = g.res16; p.ldres = g.ldres;
+  const int n_units = g.mode == GEMV_SWIGLU_F16 ? n_out : (n_out + 1) / 2;
+  // Split K while the units alone give fewer warps than the machine holds (4 CTAs of 8 warps per SM) and every part keeps
+  // at least one full pass of a warp (128 pieces of 16 bytes).  A function of the shapes only.
+  int ks = 1;
+  while (ks < 8 && (long)n_units * ks <= 148L * 32 && (g.K / 8) / (ks * 2) >= 128) ks *= 2;
+  p.ksplit = ks;
+  const int upc = 8 / ks;
+  const dim3 grid(std::max(1, std::min((n_units + upc - 1) / upc, 148 * 8))), block(256);
   ++*n_launch;
-  switch (M) {
-    case 1: return launch_dep(gemv_w16_kernel<1>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
-    case 2: return launch_dep(gemv_w16_kernel<2>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
-    case 3: return launch_dep(gemv_w16_kernel<3>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
-    case 4: return launch_dep(gemv_w16_kernel<4>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
-    case 5: return launch_dep(gemv_w16_kernel<5>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
-    case 6: return launch_dep(gemv_w16_kernel<6>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
-    case 7: return launch_dep(gemv_w16_kernel<7>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
-    default: return launch_dep(gemv_w16_kernel<8>, grid, block, 0, st, pdl, 1, W, N, K, x, ldx, y, ldy);
+  switch (g.M) {
+    case 1: return launch_dep(gemv_w16_kernel<1>, grid, block, 0, st, g.pdl, 1, p);
+    case 2: return launch_dep(gemv_w16_kernel<2>, grid, block, 0, st, g.pdl, 1, p);
+    case 3: return launch_dep(gemv_w16_kernel<3>, grid, block, 0, st, g.pdl, 1, p);
+    case 4: return launch_dep(gemv_w16_kernel<4>, grid, block, 0, st, g.pdl, 1, p);
+    case 5: return launch_dep(gemv_w16_kernel<5>, grid, block, 0, st, g.pdl, 1, p);
+    case 6: return launch_dep(gemv_w16_kernel<6>, grid, block, 0, st, g.pdl, 1, p);
+    case 7: return launch_dep(gemv_w16_kernel<7>, grid, block, 0, st, g.pdl, 1, p);
+    default: return launch_dep(gemv_w16_kernel<8>, grid, block, 0, st, g.pdl, 1, p);
   }
 }
 

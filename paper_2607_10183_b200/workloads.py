@@ -16,6 +16,8 @@ workload configurations instead:
   nibbles.  Drawing the *bytes* uniformly in [0, 255] gives exactly that
   distribution for every code, and is far cheaper than drawing codes one by one.
 * one fp16 scale per block of 32 consecutive k of a row, ``|N(0, 0.02)|``.
+* unquantized fp16 weight matrices (the FP16 model of Section 5.1) ``N(0, 0.09)`` rounded to fp16: the
+  standard deviation a dequantized weight of the recipe above has.
 * activations and KV-cache entries ``N(0, 1)`` rounded to fp16.
 * router weights ``N(0, 0.02)`` rounded to fp16.
 * RMSNorm gains zero-mean normal, rounded to fp16: std 0.25 in the dense layers, std 1 in the MoE
@@ -36,7 +38,7 @@ import numpy as np
 # roles (the tag that selects a random stream)
 ROLE_Q, ROLE_K, ROLE_V, ROLE_O, ROLE_GATE, ROLE_UP, ROLE_DOWN = 0, 1, 2, 3, 4, 5, 6
 ROLE_ROUTER, ROLE_ATTN_NORM, ROLE_FFN_NORM, ROLE_X, ROLE_KCACHE, ROLE_VCACHE = 7, 8, 9, 10, 11, 12
-PART_CODES, PART_SCALES = 0, 1
+PART_CODES, PART_SCALES, PART_W16 = 0, 1, 2
 
 BLOCK = 32  # weights per quantization block
 
@@ -139,6 +141,21 @@ def dense_layer(config: int, layer: int, shape: DenseShape = DENSE_FULL) -> dict
     out = {"shape": shape}
     for role, n_out, k_in in shape.tensor_shapes():
         out[role] = q4_packed(config, layer, role, n_out, k_in)
+    out[ROLE_ATTN_NORM] = norm_gain(config, layer, ROLE_ATTN_NORM, shape.hidden)
+    out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden)
+    return out
+
+
+def w16_matrix(config: int, layer: int, role: int, n_out: int, k_in: int) -> np.ndarray:
+    """An unquantized fp16 weight matrix ``[N][K]``."""
+    return stream(config, layer, role, PART_W16).normal(0.0, 0.09, size=(n_out, k_in)).astype(np.float16)
+
+
+def dense_layer_w16(config: int, layer: int, shape: DenseShape = DENSE_FULL) -> dict:
+    """A dense decoder layer whose seven matrices are unquantized fp16: ``{role: (w16,)}`` plus the norm gains."""
+    out = {"shape": shape}
+    for role, n_out, k_in in shape.tensor_shapes():
+        out[role] = (w16_matrix(config, layer, role, n_out, k_in),)
     out[ROLE_ATTN_NORM] = norm_gain(config, layer, ROLE_ATTN_NORM, shape.hidden)
     out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden)
     return out

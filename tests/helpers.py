@@ -55,16 +55,23 @@ def oracle_moe_tensors(B):
 
 
 def register_dense_layer(ctx, L, layer_idx, kv_capacity):
-    """Registers one dense layer's tensors in execution order; returns (layer descriptor, {role: id})."""
+    """Registers one dense layer's tensors in execution order; returns (layer descriptor, {role: id}).  A matrix given
+    as (packed, scales) is block-quantized, one given as (w16,) is an unquantized fp16 matrix."""
     from paper_2607_10183_b200 import binding as B
     shape = L["shape"]
     ids = {}
+
+    def reg(r):
+        if len(L[r]) == 1:
+            return ctx.register_w16(L[r][0], layer=layer_idx, role=r)
+        return ctx.register_q4(*L[r], layer=layer_idx, role=r)
+
     ids["attn_norm"] = ctx.register_f16(L[W.ROLE_ATTN_NORM], layer_idx, W.ROLE_ATTN_NORM)
     for r in (W.ROLE_Q, W.ROLE_K, W.ROLE_V, W.ROLE_O):
-        ids[ROLE_NAME[r]] = ctx.register_q4(*L[r], layer=layer_idx, role=r)
+        ids[ROLE_NAME[r]] = reg(r)
     ids["ffn_norm"] = ctx.register_f16(L[W.ROLE_FFN_NORM], layer_idx, W.ROLE_FFN_NORM)
     for r in (W.ROLE_GATE, W.ROLE_UP, W.ROLE_DOWN):
-        ids[ROLE_NAME[r]] = ctx.register_q4(*L[r], layer=layer_idx, role=r)
+        ids[ROLE_NAME[r]] = reg(r)
     desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
                         head_dim=shape.head_dim, kv_capacity=kv_capacity, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, **ids)
     return desc, ids

@@ -203,6 +203,29 @@ def test_lm_head_matches_oracle(B, torch, V, Hd, M):
     ctx.close()
 
 
+@pytest.mark.parametrize("M", [1, 4, 20])
+def test_lm_head_fp16_weights_matches_oracle(B, torch, M):
+    """The vocabulary projection as an unquantized fp16 matrix (the FP16 model's head): norm launch, then GEMV or GEMM."""
+    V, Hd, eps = 1000, 448, 1e-5
+    w = W.w16_matrix(95, 2, W.ROLE_Q, V, Hd)
+    gain = W.activations(95, 3, (Hd,)).astype(np.float16)
+    x = W.activations(95, 0, (M, Hd))
+    ctx = make_ctx(B, V * Hd * 2 + 64 * 1024, ws=16 * MB)
+    nid, hid = ctx.register_f16(gain), ctx.register_w16(w)
+    ctx.set_placement([(hid, -1, B.ATS_GPU)])
+    logits = torch.empty((M, V), dtype=torch.float16, device="cuda")
+    scratch = torch.empty((M, Hd), dtype=torch.float16, device="cuda")
+    ctx.lm_head(nid, hid, eps, H.to_dev(x), logits, M, scratch)
+    ctx.sync()
+    want = O.linear_w16(O.rn16(O.rmsnorm(x, gain, eps)), w, round_out=True)
+    H.assert_close(logits.cpu().numpy(), want, what=f"fp16 lm head M={M}")
+    if M == 1:  # this format has no one-launch form: without scratch the call is refused
+        with pytest.raises(B.AtsError) as e:
+            ctx.lm_head(nid, hid, eps, H.to_dev(x), logits, 1, None)
+        assert e.value.code == B.ATS_ERR_INVALID
+    ctx.close()
+
+
 @pytest.mark.parametrize("N,K,M", [(1, 8, 1), (7, 72, 3), (130, 1000, 8), (257, 4096, 1), (4096, 4096, 1), (64, 14336, 5)])
 def test_linear_w16_gemv_matches_oracle(B, torch, N, K, M):
     """An unquantized fp16 weight matrix: resident and streamed through the ring give the same bits; both match the oracle."""
@@ -361,6 +384,64 @@ def test_dense_layer_decode_matches_oracle(B, torch, shape_name, pos, cap):
         ulp = np.spacing(np.abs(ref[:, pos]).astype(np.float16)).astype(np.float64)
         assert np.all(np.abs(a - b) <= ulp + 1e-4 * np.abs(b).max())
     assert st.streamed_bytes == 0 and st.resident_bytes == H.dense_layer_bytes(shape)
+
+
+@pytest.mark.parametrize("M", [1, 3])
+def test_dense_layer_fp16_weights_decode_matches_oracle(B, torch, M):
+    """A dense layer whose seven matrices are unquantized fp16 (the FP16 model of Section 5.1): the decode step with
+    attention (M = 1) and the FFN-only step over M rows against the oracle; streaming four of the matrices through the
+    ring gives the same bits as the resident run; a layer that mixes formats is refused."""
+    shape, cfg, pos, cap = W.DENSE_SMALL, 94, 37, 64
+    L = W.dense_layer_w16(cfg, 0, shape)
+    by_name = {H.ROLE_NAME[r]: n * k * 2 for r, n, k in shape.tensor_shapes()}
+    nbytes, slot = sum(by_name.values()), max(by_name.values())
+    hybrid = dict(ALL_GPU, wq=0, wo=0, w_up=0, w_down=0)
+    x = W.activations(cfg, 0, (M, shape.hidden))
+    t = H.oracle_dense_tensors(L)
+    outs = []
+    for placement in (ALL_GPU, hybrid):
+        ctx = make_ctx(B, nbytes + 16 * 256 + 4 * shape.hidden * 2, ring_slots=2, slot_bytes=slot, chunk_bytes=64 * 1024)
+        desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+        ctx.set_placement([(ids[n], -1, w) for n, w in placement.items()])
+        edges, wmode = ctx.numerics(B.ATS_MODE_DECODE)
+        kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos)
+        kd, vd = H.to_dev(kc), H.to_dev(vc)
+        y = torch.empty((M, shape.hidden), dtype=torch.float16, device="cuda")
+        ctx.reset_stats()
+        if M == 1:
+            ctx.layer_decode(desc, H.to_dev(x), y, kd, vd, pos, 1)
+            want = O.dense_layer(x, t, shape, kc, vc, pos, edges, wmode)  # appends position `pos` to kc, vc
+            used = list(ALL_GPU)
+        else:  # FFN only: the same tensors without the attention half
+            ffn_ids = {n: ids[n] for n in ("ffn_norm", "w_gate", "w_up", "w_down")}
+            ffn_desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, rms_eps=shape.rms_eps, **ffn_ids)
+            ctx.layer_decode(ffn_desc, H.to_dev(x), y, None, None, 0, M)
+            h2 = O._edge(O.rmsnorm(x, t["ffn_norm"], shape.rms_eps), "h2", edges)
+            want = (x.astype(np.float64) + O.swiglu_ffn(h2, t["w_gate"], t["w_up"], t["w_down"], edges, wmode)).astype(np.float16)
+            used = ["w_gate", "w_up", "w_down"]
+        ctx.sync()
+        assert ctx.stats().streamed_bytes == sum(by_name[n] for n in used if placement[n] == 0)
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want, what=f"fp16-weight decode layer, M={M}")
+        if M == 1:
+            got_k = kd.cpu().numpy()
+            assert np.array_equal(np.delete(got_k, pos, axis=1), np.delete(kc, pos, axis=1))
+            a, b = got_k[:, pos].astype(np.float64), kc[:, pos].astype(np.float64)
+            assert np.all(np.abs(a - b) <= np.spacing(np.abs(kc[:, pos])).astype(np.float64) + 1e-4 * np.abs(b).max())
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+    # one quantized matrix among fp16 ones: a status, not a launch
+    mixed = dict(L)
+    mixed[W.ROLE_DOWN] = W.q4_packed(cfg, 0, W.ROLE_DOWN, shape.hidden, shape.ffn)
+    ctx = make_ctx(B, nbytes + MB)
+    desc, ids = H.register_dense_layer(ctx, mixed, 0, cap)
+    ctx.set_placement([(ids[n], -1, 1) for n in ALL_GPU])
+    y = torch.empty((1, shape.hidden), dtype=torch.float16, device="cuda")
+    kd = H.to_dev(W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos)[0])
+    with pytest.raises(B.AtsError) as e:
+        ctx.layer_decode(desc, H.to_dev(x[:1]), y, kd, kd.clone(), pos, 1)
+    assert e.value.code == B.ATS_ERR_INVALID
+    ctx.close()
 
 
 def test_host_driven_decode_equals_device_driven(B, torch):

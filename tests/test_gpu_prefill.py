@@ -395,3 +395,37 @@ def test_linear_w16_gemm_matches_oracle(B, torch, N, K, T):
         H.assert_close(outs[-1], want, what=f"w16 gemm {N}x{K} T={T}")
         ctx.close()
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+
+
+@pytest.mark.parametrize("pos0,T,cap", [(0, 9, 16), (5, 150, 160)])
+def test_dense_layer_fp16_weights_prefill_matches_oracle(B, torch, pos0, T, cap):
+    """The prefill chunk of a dense layer with unquantized fp16 matrices (one GEMM per matrix, the residual of the
+    O projection in its epilogue) against the oracle; streamed matrices give the same bits as resident ones."""
+    shape, cfg = W.DENSE_SMALL, 93
+    L = W.dense_layer_w16(cfg, 0, shape)
+    nbytes = sum(n * k * 2 for _, n, k in shape.tensor_shapes())
+    slot = max(n * k * 2 for _, n, k in shape.tensor_shapes())
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=cap)
+    ws = B.workspace_bytes(probe, T) + MB
+    x = W.activations(cfg, 0, (T, shape.hidden))
+    outs = []
+    for placement in (ALL_GPU, dict(ALL_GPU, wk=0, wo=0, w_gate=0, w_down=0)):
+        ctx = B.Context(ws + 2 * (slot + 256) + nbytes + MB, workspace_bytes=ws, ring_slots=2, slot_bytes=slot, chunk_bytes=MB)
+        desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+        ctx.set_placement([(ids[n], -1, w) for n, w in placement.items()])
+        edges, wmode = ctx.numerics(B.ATS_MODE_PREFILL)
+        kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos0)
+        kd, vd = H.to_dev(kc), H.to_dev(vc)
+        y = torch.empty((T, shape.hidden), dtype=torch.float16, device="cuda")
+        ctx.layer_prefill(desc, H.to_dev(x), y, kd, vd, pos0, T)
+        ctx.sync()
+        want = O.dense_layer(x, H.oracle_dense_tensors(L), shape, kc, vc, pos0, edges, wmode)
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want, what="fp16-weight prefill layer")
+        got_k = kd.cpu().numpy()
+        assert np.array_equal(got_k[:, :pos0], kc[:, :pos0]) and np.array_equal(got_k[:, pos0 + T:], kc[:, pos0 + T:])
+        a, b = got_k[:, pos0:pos0 + T].astype(np.float64), kc[:, pos0:pos0 + T].astype(np.float64)
+        assert np.max(np.abs(a - b)) <= 4e-3 * np.max(np.abs(b))
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
