@@ -448,3 +448,145 @@ def streamed_moe(ids: np.ndarray, expert_where, slice_bytes, chunk_bytes: int):
     nbytes = sum(int(slice_bytes[t]) for t, _ in order)
     copies = sum(-(-int(slice_bytes[t]) // chunk_bytes) for t, _ in order)
     return nbytes, copies, order
+
+
+# --------------------------------------------------------------------------------------
+# f2: dynamic transfer scheduling (Algorithm 2) and the re-scheduling gate (Algorithm 3)
+# --------------------------------------------------------------------------------------
+# Tensors are numbered 1..n in execution order as in Section 4.4; the Python lists are 0-based, so
+# tensor i is element i-1.  Backends are HOST (the paper's CPU) and GPU.  Readings the text leaves
+# open (each is listed with the design's other readings):
+#  * j = 0, "the start of the round", is a legal transfer start point with dp[0, CPU] = 0; seg(0, i)
+#    then covers tensors 1..i-1 and tensor 1 has no predecessor, hence no switch cost.  Without it
+#    the first host tensor of a round could never be promoted.
+#  * the switch cost at the boundary of a promoted tensor is the objective's c_i * 1{rb_{i-1} != rb_i}
+#    with rb_{i-1} = b_{i-1} (everything between the start point and i runs on its default backend):
+#    c_i is charged when b_{i-1} is the host.  (The listing prints the opposite indicator, which
+#    would charge a transfer between two GPU operators and none when the activation does cross.)
+#  * the start point j of a promoted tensor's transfer is a decision of the plan, as the listing's
+#    minimum over j says: the latency T of the problem formulation is evaluated with
+#    delta_i = max(w_i - seg(j_i, i), 0) for the chosen j_i.  A plan is admissible when every start
+#    point is the round start or a host tensor executed on the host, and nothing between j_i and i
+#    is promoted (those tensors run on their default backends: that is what seg adds up).
+NO_TRANSFER = -2  # start point of a tensor that is not promoted
+ROUND_START = -1  # the transfer starts when the round starts (j = 0 in the paper's numbering)
+
+
+def seg_window(j: int, i: int, b, t_gpu, t_host, c) -> float:
+    """seg(j, i) (Section 4.4.1): compute and activation-transfer time along the DEFAULT path strictly
+    between tensors j and i (1-based; j = 0 is the round start): sum over k = j+1 .. i-1 of t_k on
+    backend b_k, plus c_k where b_{k-1} != b_k."""
+    total = 0.0
+    for k in range(j + 1, i):
+        total += t_gpu[k - 1] if b[k - 1] == GPU else t_host[k - 1]
+        if k >= 2 and b[k - 2] != b[k - 1]:
+            total += c[k - 1]
+    return total
+
+
+def transfer_latency(rb, start, b, t_gpu, t_host, c, w) -> float:
+    """T(rb) of Section 4.4.1 for a plan: execution times on the runtime backends, switch costs
+    between neighbours on different runtime backends, and for every promoted tensor (b_i = HOST,
+    rb_i = GPU) the exposed part max(w_i - seg(j_i, i), 0) of its weight transfer, j_i = start[i]
+    (0-based tensor index, ROUND_START for the start of the round)."""
+    n = len(b)
+    total = 0.0
+    for i in range(1, n + 1):
+        total += t_gpu[i - 1] if rb[i - 1] == GPU else t_host[i - 1]
+        if i >= 2 and rb[i - 2] != rb[i - 1]:
+            total += c[i - 1]
+        if b[i - 1] == HOST and rb[i - 1] == GPU:
+            j = 0 if start[i - 1] == ROUND_START else start[i - 1] + 1
+            total += max(w[i - 1] - seg_window(j, i, b, t_gpu, t_host, c), 0.0)
+    return total
+
+
+def dynamic_transfer(b, t_gpu, t_host, c, w):
+    """Algorithm 2 (Dynamic Transfer Scheduling), in the listing's order: the seg table, then one pass
+    over the tensors with two states per tensor (the partial schedule ends on the host / on the GPU).
+    A GPU-resident tensor extends either state and can only end on the GPU; a host tensor either
+    stays (extends either state, ends on the host) or is promoted: the minimum over legal start
+    points j of dp[j, host] + max(w_i, seg[j, i]), plus the switch cost at i and t_i^g.
+
+    Ties keep the earlier candidate in the order the listing enumerates them (same-backend
+    predecessor before the other one, smaller j first, host before GPU at the end).
+    Returns (T*, rb, start) with rb[i] in {HOST, GPU} and start[i] as transfer_latency takes it.
+    """
+    n = len(b)
+    INF = float("inf")
+    seg = [[0.0] * (n + 2) for _ in range(n + 1)]
+    for j in range(0, n + 1):
+        for i in range(j + 1, n + 1):
+            seg[j][i] = seg_window(j, i, b, t_gpu, t_host, c)
+    # dp[i][s]: best latency of tensors 1..i with tensor i run on s; back[i][s] = (previous tensor, its state)
+    dp = [[INF, INF] for _ in range(n + 1)]
+    back = [[None, None] for _ in range(n + 1)]
+    dp[0][HOST] = 0.0
+    dp[0][GPU] = 0.0
+    for i in range(1, n + 1):
+        sw = c[i - 1] if i >= 2 else 0.0
+        if b[i - 1] == GPU:
+            cand = [(dp[i - 1][GPU], (i - 1, GPU)), (dp[i - 1][HOST] + sw, (i - 1, HOST))]
+            if i == 1:
+                cand = [(0.0, (0, GPU))]
+            best = min(cand, key=lambda t: t[0])
+            dp[i][GPU] = best[0] + t_gpu[i - 1]
+            back[i][GPU] = best[1]
+        else:
+            cand = [(dp[i - 1][HOST], (i - 1, HOST)), (dp[i - 1][GPU] + sw, (i - 1, GPU))]
+            if i == 1:
+                cand = [(0.0, (0, HOST))]
+            best = min(cand, key=lambda t: t[0])
+            dp[i][HOST] = best[0] + t_host[i - 1]
+            back[i][HOST] = best[1]
+            best_v, best_j = INF, None
+            for j in range(0, i):
+                if j >= 1 and b[j - 1] != HOST:
+                    continue
+                v = dp[j][HOST] + max(w[i - 1], seg[j][i])
+                if v < best_v:
+                    best_v, best_j = v, j
+            if best_j is not None:
+                at_i = c[i - 1] if (i >= 2 and b[i - 2] == HOST) else 0.0
+                dp[i][GPU] = best_v + at_i + t_gpu[i - 1]
+                back[i][GPU] = (best_j, HOST)
+    end = HOST if dp[n][HOST] <= dp[n][GPU] else GPU
+    t_star = dp[n][end]
+    rb = list(b)
+    start = [NO_TRANSFER] * n
+    i, s = n, end
+    while i >= 1:
+        pj, ps = back[i][s]
+        rb[i - 1] = s
+        if b[i - 1] == HOST and s == GPU:
+            start[i - 1] = ROUND_START if pj == 0 else pj - 1
+            # tensors strictly between the start point and i keep their default backends (rb = b already)
+        i, s = pj, ps
+    return t_star, rb, start
+
+
+def deviation(m_prev, m_cur) -> float:
+    """ComputeDeviation of Algorithm 3 (the paper names it without a formula): the largest relative
+    change of any measured quantity, |cur - prev| / prev; a quantity that was 0 and is not any more
+    counts as an unbounded change, one that stays 0 as none."""
+    d = 0.0
+    for p, q in zip(m_prev, m_cur):
+        if p == q:
+            continue
+        d = max(d, abs(q - p) / abs(p) if p != 0 else float("inf"))
+    return d
+
+
+def reschedule(b, rb_prev, m_prev, m_cur, eps: float, tau: float, t_now: float, t_last: float):
+    """Algorithm 3 (Load-aware Re-scheduling).  A measurement snapshot is the tuple (t_gpu, t_host, c, w)
+    of per-tensor lists.  Keeps the previous assignment while the deviation is below eps or less
+    than tau has passed since the last re-scheduling; otherwise runs Algorithm 2 on the current
+    snapshot, which becomes the reference, and the clock restarts.
+    Returns (rb, reference snapshot, time of last re-scheduling, replanned?)."""
+    flat = lambda m: [v for part in m for v in part]
+    d = deviation(flat(m_prev), flat(m_cur))
+    if d < eps or t_now - t_last < tau:
+        return list(rb_prev), m_prev, t_last, False
+    t_gpu, t_host, c, w = m_cur
+    _, rb, _ = dynamic_transfer(b, t_gpu, t_host, c, w)
+    return rb, m_cur, t_now, True
