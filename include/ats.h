@@ -324,6 +324,36 @@ int32_t ats_host_group_pairs(const int32_t* ids, uint32_t P, uint32_t E, int32_t
 int32_t ats_host_repack_q4(const void* codes, const void* scales, void* out_slice, uint32_t n_out, uint32_t k_in);
 int32_t ats_host_unpack_q4(const void* slice, void* out_codes, void* out_scales, uint32_t n_out, uint32_t k_in);
 
+/* Load-aware dynamic transfer (Section 4.4), host only.  A round runs tensors 0..n-1 in order; b[i] (ATS_HOST / ATS_GPU) is
+ * the default backend from static placement, t_gpu[i] / t_host[i] the current execution times of tensor i's operator on the
+ * GPU / on the host, c[i] the activation-transfer cost paid when tensors i-1 and i run on different backends (c[0] unused),
+ * w[i] the weight-transfer time of tensor i (for an expert operator in a decode round: of the activated experts only).  All
+ * times in one unit, finite and >= 0 (else ATS_ERR_INVALID).
+ *
+ * ats_host_dynamic_transfer: Algorithm 2.  Writes the runtime backend assignment to out_rb[0..n): resident tensors stay on
+ * the GPU; a host tensor stays or is promoted (out_rb[i] = ATS_GPU), in which case out_start[i] (optional array) is the
+ * tensor after which its weight transfer starts, ATS_ROUND_START for the start of the round; ATS_NO_TRANSFER elsewhere.
+ * *out_latency (optional) = the round latency T of Section 4.4.1 for that plan: execution times on the runtime backends +
+ * switch costs + for every promoted tensor the part of w[i] that the default-path work between its start point and i does
+ * not hide.  Between a start point and its promoted tensor nothing else is promoted.  O(n^2) time, O(n) space.
+ * ats_host_transfer_latency: T for a caller-given plan (ATS_ERR_INVALID if a resident tensor is moved off the GPU or a
+ * start index is not before its tensor; whether the start points are admissible is the caller's business).
+ * ats_host_deviation: ComputeDeviation of Algorithm 3, read as the largest relative change |cur - prev| / prev over the n
+ * measured quantities (a quantity leaving 0 counts as infinite, one staying 0 as none).
+ * ats_host_reschedule: Algorithm 3.  m_ref / m_cur are measurement snapshots [4n] = t_gpu | t_host | c | w.  If the
+ * deviation of m_cur from m_ref is below eps, or less than tau has passed since *t_last, nothing changes (the previous
+ * rb / start stay, *out_replanned = 0); otherwise Algorithm 2 runs on m_cur into rb / start (start optional), m_cur becomes
+ * the reference, *t_last = t_now and *out_replanned = 1; rebuilding the execution plan for the new assignment is the
+ * caller's step.  The paper uses eps = 0.15 and tau = 5 x the recent time per output token. */
+enum { ATS_ROUND_START = -1, ATS_NO_TRANSFER = -2 };
+int32_t ats_host_dynamic_transfer(const uint8_t* b, const double* t_gpu, const double* t_host, const double* c, const double* w,
+                                  uint32_t n, uint8_t* out_rb, int32_t* out_start, double* out_latency);
+int32_t ats_host_transfer_latency(const uint8_t* rb, const int32_t* start, const uint8_t* b, const double* t_gpu, const double* t_host,
+                                  const double* c, const double* w, uint32_t n, double* out_latency);
+double ats_host_deviation(const double* m_prev, const double* m_cur, uint32_t n);
+int32_t ats_host_reschedule(const uint8_t* b, uint32_t n, double* m_ref, const double* m_cur, double eps, double tau, double t_now,
+                            double* t_last, uint8_t* rb, int32_t* start, int32_t* out_replanned);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,7 +31,8 @@ EXPORTS = (
     "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode", "ats_layer_decode_host", "ats_embed", "ats_lm_head",
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
     "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
-    "ats_host_unpack_q4", "ats_host_group_pairs",
+    "ats_host_unpack_q4", "ats_host_group_pairs", "ats_host_dynamic_transfer", "ats_host_transfer_latency", "ats_host_deviation",
+    "ats_host_reschedule",
 )
 
 
@@ -100,6 +101,10 @@ def _load():
         "ats_host_repack_q4": (i32, [vp, vp, vp, u32, u32]),
         "ats_host_unpack_q4": (i32, [vp, vp, vp, u32, u32]),
         "ats_host_group_pairs": (i32, [vp, u32, u32, vp, vp, vp, vp]),
+        "ats_host_dynamic_transfer": (i32, [vp, vp, vp, vp, vp, u32, vp, vp, P(C.c_double)]),
+        "ats_host_transfer_latency": (i32, [vp, vp, vp, vp, vp, vp, vp, u32, P(C.c_double)]),
+        "ats_host_deviation": (C.c_double, [vp, vp, u32]),
+        "ats_host_reschedule": (i32, [vp, u32, vp, vp, C.c_double, C.c_double, C.c_double, P(C.c_double), vp, vp, P(C.c_int32)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -316,6 +321,58 @@ def host_group_pairs(ids, E):
     if st != ATS_OK:
         raise AtsError(st, "ats_host_group_pairs")
     return order, pos, off, mx.value
+
+
+ATS_ROUND_START, ATS_NO_TRANSFER = -1, -2
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def host_dynamic_transfer(b, t_gpu, t_host, c, w):
+    """Algorithm 2 on plain arrays (host only).  Returns (latency, rb uint8 array, start int32 array)."""
+    b = np.ascontiguousarray(b, dtype=np.uint8)
+    tg, th, cc, ww = _f64(t_gpu), _f64(t_host), _f64(c), _f64(w)
+    n = b.size
+    rb, start, lat = np.zeros(n, np.uint8), np.zeros(n, np.int32), C.c_double()
+    st = lib.ats_host_dynamic_transfer(b.ctypes.data, tg.ctypes.data, th.ctypes.data, cc.ctypes.data, ww.ctypes.data, n,
+                                       rb.ctypes.data, start.ctypes.data, C.byref(lat))
+    if st != ATS_OK:
+        raise AtsError(st, "ats_host_dynamic_transfer")
+    return lat.value, rb, start
+
+
+def host_transfer_latency(rb, start, b, t_gpu, t_host, c, w):
+    """The round latency T of Section 4.4.1 for a given plan (host only)."""
+    rb, b = np.ascontiguousarray(rb, dtype=np.uint8), np.ascontiguousarray(b, dtype=np.uint8)
+    start = np.ascontiguousarray(start, dtype=np.int32)
+    tg, th, cc, ww = _f64(t_gpu), _f64(t_host), _f64(c), _f64(w)
+    lat = C.c_double()
+    st = lib.ats_host_transfer_latency(rb.ctypes.data, start.ctypes.data, b.ctypes.data, tg.ctypes.data, th.ctypes.data,
+                                       cc.ctypes.data, ww.ctypes.data, b.size, C.byref(lat))
+    if st != ATS_OK:
+        raise AtsError(st, "ats_host_transfer_latency")
+    return lat.value
+
+
+def host_deviation(m_prev, m_cur):
+    a, b = _f64(m_prev).reshape(-1), _f64(m_cur).reshape(-1)
+    return float(lib.ats_host_deviation(a.ctypes.data, b.ctypes.data, a.size))
+
+
+def host_reschedule(b, m_ref, m_cur, eps, tau, t_now, t_last, rb, start=None):
+    """Algorithm 3 (host only).  m_ref (float64 [4n], updated in place), rb (uint8 [n]) and start (int32 [n], optional) are
+    the caller's state arrays.  Returns (t_last, replanned)."""
+    b = np.ascontiguousarray(b, dtype=np.uint8)
+    assert m_ref.dtype == np.float64 and m_ref.flags.c_contiguous and rb.dtype == np.uint8
+    cur = _f64(m_cur).reshape(-1)
+    tl, did = C.c_double(t_last), C.c_int32()
+    st = lib.ats_host_reschedule(b.ctypes.data, b.size, m_ref.ctypes.data, cur.ctypes.data, eps, tau, t_now, C.byref(tl),
+                                 rb.ctypes.data, None if start is None else start.ctypes.data, C.byref(did))
+    if st != ATS_OK:
+        raise AtsError(st, "ats_host_reschedule")
+    return tl.value, bool(did.value)
 
 
 def host_solve_placement(s, r, c, M, is_expert=None):
