@@ -583,6 +583,28 @@ def extra_w16(torch, B, W, peaks, quick):
     return out
 
 
+def extra_epd(torch, B, W, peaks, quick):
+    """Empirical performance density of the seven matrices of one dense layer (decode, one row): the measured operator time
+    resident and host-placed, per byte, and the residency benefit that Algorithm 1 takes as r_i."""
+    shape = W.DENSE_FULL
+    names = {W.ROLE_Q: "wq", W.ROLE_K: "wk", W.ROLE_V: "wv", W.ROLE_O: "wo", W.ROLE_GATE: "w_gate", W.ROLE_UP: "w_up", W.ROLE_DOWN: "w_down"}
+    Lw = W.dense_layer(2, 0, shape)
+    sizes = {r: W.q4_bytes(n, k) for r, n, k in shape.tensor_shapes()}
+    slot = max(sizes.values())
+    ring = 2 * (slot + 256)
+    ctx = B.Context(sum(sizes.values()) + ring + (8 << 20), workspace_bytes=1 << 20, ring_slots=2, slot_bytes=slot, chunk_bytes=4 << 20)
+    out = {"workload": "dense layer of config 2, one row per operator: time resident / host-placed (streamed through the ring), per tensor"}
+    for r, n, k in shape.tensor_shapes():
+        tid = ctx.register_q4(*Lw[r], layer=0, role=r)
+        x = torch.from_numpy(W.activations(2, 0, (1, k), role=r)).cuda()
+        y = torch.empty((1, n), dtype=torch.float16, device="cuda")
+        t_res, t_host = ctx.profile_tensor(tid, x, y, 1, iters=10 if quick else 50)
+        out[names[r]] = {"bytes": sizes[r], "t_resident_us": t_res, "t_host_us": t_host, "k_resident_ns_per_MB": t_res * 1e3 / (sizes[r] / 1e6),
+                         "k_host_ns_per_MB": t_host * 1e3 / (sizes[r] / 1e6), "r_us": t_host - t_res}
+    ctx.close()
+    return out
+
+
 def extra_model_loop_moe(torch, B, W, peaks, quick):
     """Whole-model loop on an MoE layer shape (hidden 2048, 32 query / 4 kv heads of 128, 128 experts x SwiGLU 768, top-8):
     a stack of attention + routed-expert layers; a 512-token prompt prefilled in one chunk, then decode steps through every
@@ -665,7 +687,7 @@ def extra_model_loop_moe(torch, B, W, peaks, quick):
 
 
 STACK_LAYERS = [0]
-EXTRAS = {"model_loop_moe": extra_model_loop_moe, "w16_formats": extra_w16, "model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
+EXTRAS = {"epd_profile": extra_epd, "model_loop_moe": extra_model_loop_moe, "w16_formats": extra_w16, "model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
 
 
 def run_ours(args):
@@ -812,7 +834,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the figures of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--quick", action="store_true", help="smaller extras")
-    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe", "w16_formats"],
+    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe", "w16_formats", "epd_profile"],
                     help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
     ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = 8, or 4 with --quick; 32 = the full configuration)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")

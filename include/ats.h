@@ -154,6 +154,21 @@ int32_t ats_get_placement(const ats_ctx* ctx, int32_t id, int32_t expert, uint8_
  * If the tensor is placed on the host it is streamed through the ring for this call. */
 int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /*DEVICE*/, uint32_t M);
 
+/* Empirical performance density (Section 4.3.1: k_i = t_i / s_i from measured operator times).  Times ats_linear on dense
+ * weight tensor `id` over M rows (x, y DEVICE scratch as ats_linear takes them), `iters` back-to-back calls after a warm-up,
+ * with CUDA events on the compute stream: once with the tensor resident (*t_resident_us, the paper's t^g) and once with it
+ * placed on the host and streamed through the ring (*t_host_us: the steady-state cost of leaving it off the GPU; this
+ * library has no CPU executor, so that is what stands where the paper has t^c).  The caller forms k = t / bytes and the
+ * residency benefit r_i = t_host - t_resident and hands it to Algorithm 1 through ats_set_tensor_value.
+ * The call replaces the placement while it measures (this tensor alone on the GPU / on the host, everything else on the
+ * host) and puts the previous one back before it returns; it synchronises.  ATS_ERR_BUDGET if the tensor fits neither the
+ * resident region nor a ring slot.  Stacked expert tensors: ATS_ERR_INVALID (profile the operator through ats_moe_linear).
+ * ats_set_tensor_value: replaces r_i (value < 0: the default, the tensor's byte size) and c_i of a registered weight tensor;
+ * the placement in force stays until the next ats_plan_placement. */
+int32_t ats_profile_tensor(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /*DEVICE*/, uint32_t M, uint32_t iters,
+                           double* t_resident_us /*HOST*/, double* t_host_us /*HOST*/);
+int32_t ats_set_tensor_value(ats_ctx* ctx, int32_t id, int64_t value, int64_t switch_cost);
+
 /* ats_linear for callers that must not allocate.  (The paper has no counterpart; this is a packaging variant.)
  * Some hosts of this library cannot hand it device memory beyond their tensors: code running inside a captured or
  * replayed region, plug-ins of an inference server whose memory pool is frozen after start-up, or a process that

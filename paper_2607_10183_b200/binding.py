@@ -32,7 +32,7 @@ EXPORTS = (
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
     "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
     "ats_host_unpack_q4", "ats_host_group_pairs", "ats_host_dynamic_transfer", "ats_host_transfer_latency", "ats_host_deviation",
-    "ats_host_reschedule",
+    "ats_host_reschedule", "ats_profile_tensor", "ats_set_tensor_value",
 )
 
 
@@ -101,6 +101,8 @@ def _load():
         "ats_host_repack_q4": (i32, [vp, vp, vp, u32, u32]),
         "ats_host_unpack_q4": (i32, [vp, vp, vp, u32, u32]),
         "ats_host_group_pairs": (i32, [vp, u32, u32, vp, vp, vp, vp]),
+        "ats_profile_tensor": (i32, [vp, i32, vp, vp, u32, u32, P(C.c_double), P(C.c_double)]),
+        "ats_set_tensor_value": (i32, [vp, i32, C.c_int64, C.c_int64]),
         "ats_host_dynamic_transfer": (i32, [vp, vp, vp, vp, vp, u32, vp, vp, P(C.c_double)]),
         "ats_host_transfer_latency": (i32, [vp, vp, vp, vp, vp, vp, vp, u32, P(C.c_double)]),
         "ats_host_deviation": (C.c_double, [vp, vp, u32]),
@@ -200,6 +202,15 @@ class Context:
         out = C.c_int32(-1)
         self.check(lib.ats_register_tensor(self.h, C.byref(d), w.ctypes.data, None, C.byref(out)))
         return out.value
+
+    def profile_tensor(self, tid, x, y, M, iters=20):
+        """Measured operator time of a dense weight tensor, resident and host-placed: (t_resident_us, t_host_us)."""
+        a, b = C.c_double(), C.c_double()
+        self.check(lib.ats_profile_tensor(self.h, tid, _ptr(x), _ptr(y), M, iters, C.byref(a), C.byref(b)))
+        return a.value, b.value
+
+    def set_tensor_value(self, tid, value, switch_cost=0):
+        self.check(lib.ats_set_tensor_value(self.h, tid, int(value), int(switch_cost)))
 
     def register_f16(self, data: np.ndarray, layer=0, role=0) -> int:
         data = np.ascontiguousarray(data, dtype=np.float16)

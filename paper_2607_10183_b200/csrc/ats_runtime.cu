@@ -938,6 +938,78 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M)
   return run_gemm_group(ctx, &op, 1, g);
 }
 
+// Empirical performance density (Section 4.3.1): the measured time of one tensor's operator with the tensor resident and
+// with the tensor placed on the host, from which the caller forms k_i = t_i / s_i and the residency benefit r_i.
+int32_t ats_profile_tensor(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M, uint32_t iters, double* t_resident_us,
+                           double* t_host_us) {
+  ATS_TRY(precheck(ctx, false));
+  Tensor* t = get_weight(ctx, id);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense weight tensor", id);
+  if (!x || !y || !t_resident_us || !t_host_us || M == 0 || iters == 0) return fail(ctx, ATS_ERR_INVALID, "null pointer or zero count");
+  // the placement in force is put back afterwards
+  std::vector<uint8_t> saved;
+  for (Tensor& u : ctx->tensors)
+    for (Slice& sl : u.slices) saved.push_back(sl.where);
+  const bool was_placed = ctx->placed;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  ATS_CUDA(cudaEventCreate(&e0));
+  cudaError_t ce = cudaEventCreate(&e1);
+  if (ce != cudaSuccess) {
+    cudaEventDestroy(e0);
+    return check_cuda(ctx, ce, "cudaEventCreate");
+  }
+  auto restore = [&]() -> int32_t {
+    size_t k = 0;
+    for (Tensor& u : ctx->tensors)
+      for (Slice& sl : u.slices) sl.where = saved[k++];
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    ctx->placed = false;
+    return was_placed ? apply_placement(ctx) : ATS_OK;
+  };
+  int32_t st = ATS_OK;
+  for (int mode = 0; mode < 2 && st == ATS_OK; ++mode) {
+    // this tensor alone decides: everything else sits on the host and is not touched
+    for (Tensor& u : ctx->tensors)
+      if (placeable(u))
+        for (Slice& sl : u.slices) sl.where = ATS_HOST;
+    t->slices[0].where = mode == 0 ? ATS_GPU : ATS_HOST;
+    ctx->placed = false;
+    st = apply_placement(ctx);
+    for (uint32_t i = 0; i < 2 && st == ATS_OK; ++i) st = ats_linear(ctx, id, x, y, M);  // warm-up
+    if (st != ATS_OK) break;
+    if ((ce = cudaEventRecord(e0, ctx->cs)) != cudaSuccess) break;
+    for (uint32_t i = 0; i < iters && st == ATS_OK; ++i) st = ats_linear(ctx, id, x, y, M);
+    if (st != ATS_OK) break;
+    if ((ce = cudaEventRecord(e1, ctx->cs)) != cudaSuccess) break;
+    if ((ce = cudaEventSynchronize(e1)) != cudaSuccess) break;
+    float ms = 0.f;
+    if ((ce = cudaEventElapsedTime(&ms, e0, e1)) != cudaSuccess) break;
+    *(mode == 0 ? t_resident_us : t_host_us) = (double)ms * 1e3 / iters;
+  }
+  if (ce != cudaSuccess) {
+    restore();
+    return check_cuda(ctx, ce, "ats_profile_tensor timing");
+  }
+  if (st != ATS_OK) {
+    const std::string why = ctx->err;
+    restore();
+    ctx->err = why;
+    return st;
+  }
+  return restore();
+}
+
+int32_t ats_set_tensor_value(ats_ctx* ctx, int32_t id, int64_t value, int64_t switch_cost) {
+  ATS_TRY(precheck(ctx, false));
+  Tensor* t = get_weight(ctx, id);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not a weight tensor", id);
+  if (switch_cost < 0) return fail(ctx, ATS_ERR_INVALID, "switch_cost must be >= 0");
+  t->d.value = value < 0 ? (int64_t)(t->slices.size() * t->slice_bytes) : value;
+  t->d.switch_cost = switch_cost;
+  return ATS_OK;
+}
+
 static int32_t check_f16(ats_ctx* ctx, int32_t id, uint32_t n_out, uint32_t k_in, const char* name);
 
 int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids, uint32_t M, void* out) {

@@ -294,6 +294,58 @@ def test_plan_placement_over_mixed_formats(B, torch):
         assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
 
 
+def test_profile_tensor_feeds_measured_values_into_algorithm_1(B, torch):
+    """Empirical performance density (Section 4.3.1): operator times measured resident and host-placed, turned into the
+    residency benefit r_i of each tensor and handed to Algorithm 1; the resulting placement is the oracle's on the same
+    integers.  The measuring call leaves the placement (or the unplaced state) and the results of later calls as they were."""
+    shapes = [(4096, 4096), (1024, 1024), (8192, 4096), (2048, 2048)]
+    data = [W.q4_packed(92, i, W.ROLE_Q, n, k) for i, (n, k) in enumerate(shapes)]
+    nbytes = [W.q4_bytes(n, k) for n, k in shapes]
+    slot = max(nbytes)
+    ctx = make_ctx(B, sum(nbytes) + 64 * 1024, ring_slots=2, slot_bytes=slot, chunk_bytes=4 * MB)
+    ids = [ctx.register_q4(*d) for d in data]
+    xs = [H.to_dev(W.activations(92, i, (1, k))) for i, (n, k) in enumerate(shapes)]
+    ys = [torch.empty((1, n), dtype=torch.float16, device="cuda") for n, k in shapes]
+    # before any placement: measuring works and leaves the context unplaced
+    t_res0, t_host0 = ctx.profile_tensor(ids[1], xs[1], ys[1], 1, iters=5)
+    assert t_res0 > 0 and t_host0 > 0
+    with pytest.raises(B.AtsError) as e:
+        ctx.linear(ids[1], xs[1], ys[1], 1)
+    assert e.value.code == B.ATS_ERR_STATE
+    place = [(ids[0], -1, B.ATS_GPU), (ids[1], -1, B.ATS_HOST), (ids[2], -1, B.ATS_HOST), (ids[3], -1, B.ATS_GPU)]
+    ctx.set_placement(place)
+    before = []
+    for t, x, y in zip(ids, xs, ys):
+        ctx.linear(t, x, y, 1)
+        ctx.sync()
+        before.append(y.cpu().numpy().copy())
+    t_res, t_host = zip(*[ctx.profile_tensor(t, x, y, 1, iters=10) for t, x, y in zip(ids, xs, ys)])
+    # a streamed tensor costs its PCIe time, far above its HBM time; more bytes cost more
+    for i in (0, 2, 3):
+        assert t_host[i] > 3 * t_res[i], (i, t_res, t_host)
+    assert t_host[2] > t_host[0] > t_host[3] > t_host[1]
+    # the placement in force is back, and so are the bits
+    assert [ctx.get_placement(t) for t in ids] == [w for _, _, w in place]
+    for t, x, y, ref in zip(ids, xs, ys, before):
+        y.zero_()
+        ctx.linear(t, x, y, 1)
+        ctx.sync()
+        assert np.array_equal(y.cpu().numpy().view(np.uint16), ref.view(np.uint16))
+    # r_i in nanoseconds saved per call by residency, c_i = 0; budget: 70 % of the bytes at 1 MiB granularity
+    r = [max(0, int(round(1e3 * (h - g)))) for g, h in zip(t_res, t_host)]
+    for t, v in zip(ids, r):
+        ctx.set_tensor_value(t, v, 0)
+    budget = int(0.7 * sum(nbytes))
+    got = ctx.plan_placement(budget, len(ids))
+    s_units = O.size_units(nbytes)
+    want = O.static_placement(s_units, r, [0] * len(ids), O.budget_units(budget))
+    assert list(got) == list(want)
+    # density k = t / s: what the tensors' times say per byte (the figure the paper sorts tensors by)
+    k_res = [g / b for g, b in zip(t_res, nbytes)]
+    assert all(v > 0 for v in k_res)
+    ctx.close()
+
+
 def test_linear_closed_forms_on_gpu(B, torch):
     """One-hot activations return a weight column exactly; all-ones with unit scales return integer row sums."""
     N, K = 40, 256
