@@ -80,11 +80,41 @@ def dequantize(packed: np.ndarray, scales: np.ndarray, weight_mode: int = WEIGHT
 
     ``WEIGHT_F16`` rounds that product once to fp16 (what a tensor-core operand holds).
     """
+    if np.asarray(scales).dtype == np.uint8:  # shared-exponent bytes: the microscaling 4-bit format
+        w = dequantize_mxfp4(packed, scales)
+        return rn16(w) if weight_mode == WEIGHT_F16 else w
     codes = unpack_codes(packed).astype(np.float64)
     s = np.asarray(scales, dtype=np.float16).astype(np.float64)
     assert codes.shape[-1] == s.shape[-1] * BLOCK, "one scale per 32 consecutive k"
     w = codes * np.repeat(s, BLOCK, axis=-1)
     return rn16(w) if weight_mode == WEIGHT_F16 else w
+
+
+def dequantize_mxfp4(packed: np.ndarray, scales_e8m0: np.ndarray) -> np.ndarray:
+    """MXFP4, the other 4-bit format the paper evaluates (Section 5.1): blocks of 32 elements along K, each element a
+    4-bit float (1 sign, 2 exponent, 1 mantissa bit; exponent bias 1), one shared power-of-two scale per block stored as
+    a biased 8-bit exponent.  Written from the definition of the microscaling formats:
+
+      element: s e1 e0 m  ->  (-1)^s * (m / 2            if e = 0   (subnormal)
+                                        2^(e-1) * (1 + m/2) otherwise), e = 2 e1 + e0
+      scale:   X = 2^(byte - 127), byte 255 = not a number (rejected)
+      w[n,k] = X[n, k // 32] * element[n,k]
+
+    Bytes are packed like the other 4-bit format: byte j of a row holds element 2j in bits 0..3 and element 2j+1 in
+    bits 4..7.  Every w is a small integer times a power of two, exact in fp64 (and in fp16 for |exponent| small)."""
+    p = np.asarray(packed, dtype=np.uint8)
+    nib = np.empty(p.shape[:-1] + (p.shape[-1] * 2,), dtype=np.uint8)
+    nib[..., 0::2] = p & 0x0F
+    nib[..., 1::2] = p >> 4
+    sign = np.where(nib & 8, -1.0, 1.0)
+    e = ((nib >> 1) & 3).astype(np.int64)
+    m = (nib & 1).astype(np.float64)
+    mag = np.where(e == 0, m / 2.0, np.ldexp(1.0 + m / 2.0, e - 1))
+    sb = np.asarray(scales_e8m0, dtype=np.uint8)
+    assert not np.any(sb == 255), "a block scale of 255 encodes NaN"
+    assert nib.shape[-1] == sb.shape[-1] * BLOCK, "one scale per 32 consecutive k"
+    scale = np.ldexp(1.0, sb.astype(np.int64) - 127)
+    return sign * mag * np.repeat(scale, BLOCK, axis=-1)
 
 
 # --------------------------------------------------------------------------------------

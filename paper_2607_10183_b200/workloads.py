@@ -16,6 +16,9 @@ workload configurations instead:
   nibbles.  Drawing the *bytes* uniformly in [0, 255] gives exactly that
   distribution for every code, and is far cheaper than drawing codes one by one.
 * one fp16 scale per block of 32 consecutive k of a row, ``|N(0, 0.02)|``.
+* the microscaling 4-bit format (MXFP4, Section 5.1): element bytes uniform in [0, 255] (every 4-bit float encoding
+  equally likely), one shared-exponent byte per block of 32 uniform in [119, 123] (block scales 2^-8 .. 2^-4, which
+  gives weights of standard deviation about 0.1 like the other formats).
 * unquantized fp16 weight matrices (the FP16 model of Section 5.1) ``N(0, 0.09)`` rounded to fp16: the
   standard deviation a dequantized weight of the recipe above has.
 * activations and KV-cache entries ``N(0, 1)`` rounded to fp16.
@@ -38,7 +41,7 @@ import numpy as np
 # roles (the tag that selects a random stream)
 ROLE_Q, ROLE_K, ROLE_V, ROLE_O, ROLE_GATE, ROLE_UP, ROLE_DOWN = 0, 1, 2, 3, 4, 5, 6
 ROLE_ROUTER, ROLE_ATTN_NORM, ROLE_FFN_NORM, ROLE_X, ROLE_KCACHE, ROLE_VCACHE = 7, 8, 9, 10, 11, 12
-PART_CODES, PART_SCALES, PART_W16 = 0, 1, 2
+PART_CODES, PART_SCALES, PART_W16, PART_MXSCALE = 0, 1, 2, 3
 
 BLOCK = 32  # weights per quantization block
 
@@ -72,6 +75,17 @@ def codes_to_packed(codes: np.ndarray) -> np.ndarray:
     assert c.shape[-1] % 2 == 0 and c.min() >= -8 and c.max() <= 7
     u = (c.astype(np.int16) & 0xF).astype(np.uint8)
     return (u[..., 0::2] | (u[..., 1::2] << 4)).astype(np.uint8)
+
+
+def mxfp4_packed(config: int, layer: int, role: int, n_out: int, k_in: int, n_experts: int = 1):
+    """A weight in the microscaling 4-bit format: ``(packed, scale_bytes)`` with ``packed`` uint8 ``[E][N][K/2]``
+    (two elements per byte, even k in the low nibble) and ``scale_bytes`` uint8 ``[E][N][K/32]`` (biased exponents)."""
+    assert k_in % BLOCK == 0
+    shape_c = (n_out, k_in // 2) if n_experts == 1 else (n_experts, n_out, k_in // 2)
+    shape_s = (n_out, k_in // BLOCK) if n_experts == 1 else (n_experts, n_out, k_in // BLOCK)
+    packed = stream(config, layer, role, PART_CODES).integers(0, 256, size=shape_c, dtype=np.uint8)
+    scale_bytes = stream(config, layer, role, PART_MXSCALE).integers(119, 124, size=shape_s, dtype=np.uint8)
+    return packed, scale_bytes
 
 
 def activations(config: int, layer: int, shape, step: int = 0, role: int = ROLE_X) -> np.ndarray:
@@ -156,6 +170,16 @@ def dense_layer_w16(config: int, layer: int, shape: DenseShape = DENSE_FULL) -> 
     out = {"shape": shape}
     for role, n_out, k_in in shape.tensor_shapes():
         out[role] = (w16_matrix(config, layer, role, n_out, k_in),)
+    out[ROLE_ATTN_NORM] = norm_gain(config, layer, ROLE_ATTN_NORM, shape.hidden)
+    out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden)
+    return out
+
+
+def dense_layer_mxfp4(config: int, layer: int, shape: DenseShape = DENSE_FULL) -> dict:
+    """A dense decoder layer whose seven matrices are in the microscaling 4-bit format: ``{role: (packed, scale_bytes)}``."""
+    out = {"shape": shape}
+    for role, n_out, k_in in shape.tensor_shapes():
+        out[role] = mxfp4_packed(config, layer, role, n_out, k_in)
     out[ROLE_ATTN_NORM] = norm_gain(config, layer, ROLE_ATTN_NORM, shape.hidden)
     out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden)
     return out

@@ -385,3 +385,80 @@ def test_linear_w16_exact_rational_and_special_cases():
     assert np.array_equal(O.linear_w16(x, np.eye(K, dtype=np.float16)), x.astype(np.float64))
     y16 = O.linear_w16(x, w, round_out=True)
     assert np.array_equal(y16, O.rn16(got))
+
+
+# ---------------------------------------------------------------- the microscaling 4-bit format (Section 5.1)
+def test_mxfp4_golden_elements_and_scales():
+    section = 0
+    for line in open(os.path.join(GOLD, "mxfp4_elements.txt")):
+        if line.startswith("# byte"):
+            section = 1
+        if line.startswith("#") or not line.strip():
+            continue
+        a, b = line.split()
+        if section == 0:
+            code = int(a, 2)
+            for pos in (0, 1):  # the element in the low and in the high nibble of a byte
+                packed = np.zeros((1, 16), dtype=np.uint8)
+                packed[0, 3] = code << (4 * pos)
+                w = O.dequantize(packed, np.array([[127]], dtype=np.uint8))[0]
+                assert w[6 + pos] == float(b) and np.signbit(w[6 + pos]) == b.startswith("-"), line
+                assert np.count_nonzero(w) == (1 if float(b) != 0 else 0)
+        else:
+            packed = np.full((1, 16), 0x22, dtype=np.uint8)  # every element 1.0
+            w = O.dequantize(packed, np.array([[int(a)]], dtype=np.uint8))[0]
+            assert np.all(w == float(b)), line
+
+
+def test_mxfp4_integer_form_block_indexing_and_scale_steps():
+    # twice the element is an integer: the magnitudes are 0 1 2 3 4 6 8 12 (an independent, all-integer statement)
+    twice = [0, 1, 2, 3, 4, 6, 8, 12]
+    rng = np.random.default_rng(31)
+    packed = rng.integers(0, 256, size=(5, 48), dtype=np.uint8)   # K = 96: three blocks per row
+    sb = rng.integers(100, 150, size=(5, 3), dtype=np.uint8)
+    w = O.dequantize(packed, sb)
+    for n in range(5):
+        for k in range(96):
+            nib = (int(packed[n, k // 2]) >> (4 * (k & 1))) & 15
+            want = Fraction((-1 if nib & 8 else 1) * twice[nib & 7], 2) * Fraction(2) ** (int(sb[n, k // 32]) - 127)
+            assert Fraction(float(w[n, k])) == want
+    # one step of the scale byte doubles every weight of its block and nothing else
+    sb2 = sb.copy()
+    sb2[2, 1] += 1
+    w2 = O.dequantize(packed, sb2)
+    assert np.array_equal(w2[2, 32:64], 2 * w[2, 32:64])
+    w2[2, 32:64] = w[2, 32:64]
+    assert np.array_equal(w2, w)
+    with pytest.raises(AssertionError):
+        O.dequantize(packed, np.full((5, 3), 255, dtype=np.uint8))
+    # the tensor-core operand mode rounds to fp16 like for the other format; for block exponents from -23 to 13 every weight
+    # already is an fp16 value (0.5 * 2^-23 is the smallest subnormal, 6 * 2^13 is below the largest finite), so it changes nothing
+    assert np.array_equal(O.dequantize(packed, sb, O.WEIGHT_F16), O.rn16(w))
+    for lo, hi in ((104, 141), (104, 105), (140, 141)):
+        sb3 = rng.integers(lo, hi, size=(5, 3), dtype=np.uint8)
+        w3 = O.dequantize(packed, sb3)
+        assert np.array_equal(O.dequantize(packed, sb3, O.WEIGHT_F16), w3) and np.all(np.isfinite(w3.astype(np.float16)))
+        assert np.array_equal(w3.astype(np.float16).astype(np.float64), w3)
+    assert not np.array_equal(O.rn16(O.dequantize(packed, np.full((5, 3), 103, dtype=np.uint8))), O.dequantize(packed, np.full((5, 3), 103, dtype=np.uint8)))
+
+
+def test_mxfp4_linear_exact_rational():
+    rng = np.random.default_rng(32)
+    N, K, M = 6, 64, 3
+    packed = rng.integers(0, 256, size=(N, K // 2), dtype=np.uint8)
+    sb = rng.integers(118, 132, size=(N, K // 32), dtype=np.uint8)
+    x = rng.standard_normal((M, K)).astype(np.float16)
+    y = O.linear(x, packed, sb)
+    twice = [0, 1, 2, 3, 4, 6, 8, 12]
+    for m in range(M):
+        for n in range(N):
+            exact = Fraction(0)
+            for k in range(K):
+                nib = (int(packed[n, k // 2]) >> (4 * (k & 1))) & 15
+                wv = Fraction((-1 if nib & 8 else 1) * twice[nib & 7], 2) * Fraction(2) ** (int(sb[n, k // 32]) - 127)
+                exact += wv * Fraction(float(x[m, k]))
+            assert abs(Fraction(float(y[m, n])) - exact) <= abs(exact) * Fraction(1, 2 ** 45) + Fraction(1, 2 ** 60)
+    # all elements 1.0 and unit scales: row sums of x
+    ones = np.full((2, K // 2), 0x22, dtype=np.uint8)
+    y1 = O.linear(x, ones, np.full((2, K // 32), 127, dtype=np.uint8))
+    assert np.allclose(y1[:, 0], x.astype(np.float64).sum(axis=1), rtol=0, atol=1e-12)
