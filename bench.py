@@ -583,6 +583,47 @@ def extra_w16(torch, B, W, peaks, quick):
     return out
 
 
+def extra_mxfp4(torch, B, W, peaks, quick):
+    """The microscaling 4-bit format: the single-row GEMV (generic kernel: fp32 accumulation of exact products) against
+    the HBM peak at the slice's bytes per weight, and the tcgen05 GEMM with in-kernel dequantization against the tensor peak."""
+    out = {"workload": "MXFP4 weights: GEMV (1 row) over rotated replicas, GEMM over 512 and 2048 rows"}
+    for (N, K, reps) in ((4096, 4096, 16), (14336, 4096, 8)):
+        nb = W.q4_bytes(N, K)
+        ctx = B.Context(reps * (nb + 4096) + (4 << 20), workspace_bytes=1 << 20)
+        packed, sb = W.mxfp4_packed(17, 0, W.ROLE_Q, N, K)
+        ids = [ctx.register_mxfp4(packed, sb) for _ in range(reps)]
+        ctx.set_placement([(t, -1, B.ATS_GPU) for t in ids])
+        x = torch.from_numpy(W.activations(17, 0, (1, K))).cuda()
+        y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+
+        def go(n):
+            for i in range(n):
+                ctx.linear(ids[i % reps], x, y, 1)
+        go(2 * reps)
+        ctx.sync()
+        n = (10 if quick else 40) * reps
+        us = event_time_ms(torch, ctx.compute, lambda: go(n)) * 1e3 / n
+        out[f"gemv_{N}x{K}"] = {"us_per_call": us, "gbs": nb / us / 1e3, "frac_of_measured_hbm": nb / us / 1e3 / peaks["hbm_gbs"]}
+        ctx.close()
+    for (N, K, T) in ((14336, 4096, 512), (14336, 4096, 2048)):
+        nb = W.q4_bytes(N, K)
+        ws = 9 * T * N * 4 + (2 << 20)
+        ctx = B.Context(ws + nb + (4 << 20), workspace_bytes=ws)
+        tid = ctx.register_mxfp4(*W.mxfp4_packed(17, 1, W.ROLE_Q, N, K))
+        ctx.set_placement([(tid, -1, B.ATS_GPU)])
+        x = torch.from_numpy(W.activations(17, 1, (T, K))).cuda()
+        y = torch.empty((T, N), dtype=torch.float16, device="cuda")
+        for _ in range(3):
+            ctx.linear(tid, x, y, T)
+        ctx.sync()
+        n = 5 if quick else 20
+        ms = event_time_ms(torch, ctx.compute, lambda: [ctx.linear(tid, x, y, T) for _ in range(n)]) / n
+        tf = 2.0 * T * N * K / (ms * 1e-3) / 1e12
+        out[f"gemm_{N}x{K}_T{T}"] = {"us_per_call": ms * 1e3, "tflops": tf, "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"]}
+        ctx.close()
+    return out
+
+
 def extra_epd(torch, B, W, peaks, quick):
     """Empirical performance density of the seven matrices of one dense layer (decode, one row): the measured operator time
     resident and host-placed, per byte, and the residency benefit that Algorithm 1 takes as r_i."""
@@ -687,7 +728,7 @@ def extra_model_loop_moe(torch, B, W, peaks, quick):
 
 
 STACK_LAYERS = [0]
-EXTRAS = {"epd_profile": extra_epd, "model_loop_moe": extra_model_loop_moe, "w16_formats": extra_w16, "model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
+EXTRAS = {"mxfp4_formats": extra_mxfp4, "epd_profile": extra_epd, "model_loop_moe": extra_model_loop_moe, "w16_formats": extra_w16, "model_loop": extra_model_loop, "cfg1_gemv": extra_gemv, "cfg3_prefill": extra_prefill, "cfg4_moe": extra_moe, "cfg5_stream": extra_stream}
 
 
 def run_ours(args):
@@ -834,7 +875,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the figures of the other configs")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--quick", action="store_true", help="smaller extras")
-    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe", "w16_formats", "epd_profile"],
+    ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe", "w16_formats", "epd_profile", "mxfp4_formats"],
                     help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
     ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = 8, or 4 with --quick; 32 = the full configuration)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")

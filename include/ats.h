@@ -50,7 +50,7 @@ enum {
 };
 
 enum { ATS_HOST = 0, ATS_GPU = 1 };             /* placement b_i (Section 4.3.2) */
-enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1, ATS_FMT_W16 = 2 };
+enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1, ATS_FMT_W16 = 2, ATS_FMT_MXFP4 = 3 };
 /* F16: small auxiliary tensors (router weight [k_in][n_out], norm gain [n_out]): always resident, no placement.
  * W16: an unquantized fp16 weight matrix [n_out][k_in] (the paper runs one of its models with FP16 weights, Section 5.1):
  * a dense tensor (n_experts = 1, k_in a multiple of 8) placed and streamed like a Q4B32 tensor (2 bytes per weight);
@@ -58,7 +58,16 @@ enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1, ATS_FMT_W16 = 2 };
  * layer whose seven matrices are all W16 (mixed formats within a layer: ATS_ERR_INVALID; MoE layers: Q4B32 experts only;
  * fp32 accumulation, the same roundings between operators as the quantized layer; the norm runs as a launch of its
  * own and fused groups (QKV, gate|up) become one GEMV launch or one GEMM per matrix).  ats_moe_linear, ats_embed and
- * ats_dequantize take Q4B32 tensors only. */
+ * ats_dequantize take 4-bit tensors only.
+ * MXFP4: the microscaling 4-bit format, the other 4-bit format the paper evaluates (Section 5.1).  Interchange layout:
+ * codes uint8 [E][n_out][k_in/2], byte j of a row = element 2j in bits 0..3 and element 2j+1 in bits 4..7, each element a
+ * 4-bit float (sign, 2 exponent bits with bias 1, 1 mantissa bit, exponent 0 subnormal: 0, 0.5, 1, 1.5, 2, 3, 4, 6 and
+ * their negatives); scales uint8 [E][n_out][k_in/32], one biased exponent per block of 32: 2^(byte - 127).  Byte 255
+ * (not a number): ATS_ERR_INVALID; exponents outside -23 .. 13 (bytes 104 .. 140): ATS_ERR_UNSUPPORTED, because every
+ * weight must be an fp16 value (it is the tensor-core operand).  Inside the library the tensor has the slice layout and
+ * size of a Q4B32 tensor (the scale kept as an fp16 power of two) and takes every call a Q4B32 tensor takes, dense or
+ * stacked; weights are exact in both the GEMV and the GEMM.  The single-token streaming kernels are integer-code
+ * kernels: MXFP4 tensors run on the generic GEMV kernels. */
 enum { ATS_OUT_F32 = 0, ATS_OUT_F16 = 1 };      /* ats_dequantize output */
 enum { ATS_MODE_DECODE = 0, ATS_MODE_PREFILL = 1 };
 
@@ -111,7 +120,7 @@ typedef struct {
   uint32_t fmt;        /* ATS_FMT_* */
   uint32_t n_experts;  /* 1 = dense tensor; > 1 = stacked expert tensor [E][n_out][k_in] */
   uint32_t n_out;      /* output features N */
-  uint32_t k_in;       /* input features K (Q4B32: multiple of 32) */
+  uint32_t k_in;       /* input features K (Q4B32, MXFP4: multiple of 32) */
   uint32_t layer;      /* informational */
   uint32_t role;       /* informational */
   int64_t value;       /* r_i, the benefit of residency; < 0 selects the default r_i = byte size */

@@ -18,7 +18,7 @@ ATS_OK = 0
 ATS_ERR_INVALID, ATS_ERR_SHAPE, ATS_ERR_NOMEM, ATS_ERR_BUDGET = -1, -2, -3, -4
 ATS_ERR_STATE, ATS_ERR_CUDA, ATS_ERR_TIMEOUT, ATS_ERR_UNSUPPORTED = -5, -6, -7, -8
 ATS_HOST, ATS_GPU = 0, 1
-ATS_FMT_Q4B32, ATS_FMT_F16, ATS_FMT_W16 = 0, 1, 2
+ATS_FMT_Q4B32, ATS_FMT_F16, ATS_FMT_W16, ATS_FMT_MXFP4 = 0, 1, 2, 3
 ATS_OUT_F32, ATS_OUT_F16 = 0, 1
 ATS_MODE_DECODE, ATS_MODE_PREFILL = 0, 1
 ATS_FLAG_POISON_SLOTS, ATS_FLAG_SKIP_SCALE_CHECK, ATS_FLAG_TIME_KERNELS, ATS_FLAG_NO_PDL, ATS_FLAG_MOE_DEVICE_GATHER = 1, 2, 4, 8, 16
@@ -185,6 +185,9 @@ class Context:
 
     # ---- registry / placement
     def register_q4(self, packed: np.ndarray, scales: np.ndarray, layer=0, role=0, value=-1, switch_cost=0) -> int:
+        """A 4-bit block tensor: fp16 scales select the integer-code format, uint8 scale bytes the microscaling format."""
+        if np.asarray(scales).dtype == np.uint8:
+            return self.register_mxfp4(packed, scales, layer, role, value, switch_cost)
         packed = np.ascontiguousarray(packed, dtype=np.uint8)
         scales = np.ascontiguousarray(scales, dtype=np.float16)
         E = packed.shape[0] if packed.ndim == 3 else 1
@@ -192,6 +195,17 @@ class Context:
         d = ats_tensor_desc(ATS_FMT_Q4B32, E, n_out, k_in, layer, role, value, switch_cost)
         out = C.c_int32(-1)
         self.check(lib.ats_register_tensor(self.h, C.byref(d), packed.ctypes.data, scales.ctypes.data, C.byref(out)))
+        return out.value
+
+    def register_mxfp4(self, packed: np.ndarray, scale_bytes: np.ndarray, layer=0, role=0, value=-1, switch_cost=0) -> int:
+        """Microscaling 4-bit floats [E][n_out][k_in/2] with one biased-exponent byte per block of 32."""
+        packed = np.ascontiguousarray(packed, dtype=np.uint8)
+        scale_bytes = np.ascontiguousarray(scale_bytes, dtype=np.uint8)
+        E = packed.shape[0] if packed.ndim == 3 else 1
+        n_out, k_in = packed.shape[-2], packed.shape[-1] * 2
+        d = ats_tensor_desc(ATS_FMT_MXFP4, E, n_out, k_in, layer, role, value, switch_cost)
+        out = C.c_int32(-1)
+        self.check(lib.ats_register_tensor(self.h, C.byref(d), packed.ctypes.data, scale_bytes.ctypes.data, C.byref(out)))
         return out.value
 
     def register_w16(self, w: np.ndarray, layer=0, role=0, value=-1, switch_cost=0) -> int:

@@ -147,6 +147,7 @@ struct GemvParams {
   __half* norm_out;
   int pdl;  // allow the launch to overlap the tail of the preceding kernel (programmatic dependent launch)
   int w16;  // the segments are unquantized fp16 matrices [n_rows][K] (launch_gemv_w16; no norm prologue)
+  int mx;   // the segments hold microscaling 4-bit floats (same slice layout, power-of-two fp16 block scales): generic kernel only
 };
 cudaError_t launch_gemv(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
 // fp16-weight GEMV (kernels_decode.cu): the same segments, epilogue modes and fp32 accumulation as launch_gemv over
@@ -222,6 +223,7 @@ struct MoeGemvParams {
   __half* y16;
   int ldy;
   int mode;  // GEMV_OUT_F32, GEMV_OUT_F16 or GEMV_SWIGLU_F16
+  int mx;    // microscaling 4-bit floats instead of integer codes (generic kernel only)
 };
 cudaError_t launch_moe_gemv(const MoeGemvParams& p, const MoeJobs* jobs /*null = implicit*/, cudaStream_t st,
                             uint64_t* n_launch);
@@ -230,10 +232,10 @@ bool moe_gemv_stream_eligible(const MoeGemvParams& p);
 cudaError_t launch_moe_gemv_stream(const MoeGemvParams& p, const MoeJobs* jobs /*null = implicit*/, int* status, int sm_count,
                                    int pdl, cudaStream_t st, uint64_t* n_launch);
 
-cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, cudaStream_t st,
+cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, int mx, cudaStream_t st,
                            uint64_t* n_launch);
 cudaError_t launch_embed_rows(const uint8_t* slice, int n_rows, int K, const int32_t* ids, int M, __half* out, int* status,
-                              cudaStream_t st, uint64_t* n_launch, int pdl = 0);
+                              int mx, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
                            cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 // decode attention, fused with the rotary embedding and the KV append (kernels_decode.cu)
@@ -309,6 +311,7 @@ struct GemmParams {
   // and multiplies them with slice e of every segment (seg[i].base + e * grp_stride, or grp_tab[i][e] where a table is
   // given: device or mapped host addresses).  No split-K, no residual.
   int w16;                  // seg[0].base is an unquantized fp16 matrix [n_rows][K] (one segment, no grouping)
+  int mx;                   // the slices hold microscaling 4-bit floats (same layout as the integer codes)
   const int* grp_off;       // DEVICE [n_groups + 1]; null = plain GEMM
   int n_groups;
   int grp_max_rows;         // the largest expert's row count (sizes the grid)
@@ -323,6 +326,8 @@ cudaError_t gemm_static_scratch(void** out);
 
 // host-side pieces
 void repack_q4(const uint8_t* codes_in, const uint16_t* scales_in, uint8_t* slice_out, uint64_t n_rows, uint64_t K);
+// the microscaling format into the same slice layout: elements keep their encoding, scale bytes become fp16 powers of two
+void repack_mxfp4(const uint8_t* codes_in, const uint8_t* scale_bytes_in, uint8_t* slice_out, uint64_t n_rows, uint64_t K);
 // Algorithm 1's dense solver; returns placement bytes (ATS_HOST/ATS_GPU) and the objective.
 void solve_knapsack_dp(const std::vector<int64_t>& s, const std::vector<int64_t>& r, const std::vector<int64_t>& c,
                        int64_t M, std::vector<uint8_t>* b, int64_t* objective);

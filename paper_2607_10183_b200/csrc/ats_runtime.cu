@@ -99,7 +99,14 @@ static Tensor* get_tensor(ats_ctx* ctx, int32_t id, uint32_t fmt) {
   return t->d.fmt == fmt ? t : nullptr;
 }
 // tensors that take part in placement: block-quantized or fp16 weight matrices
-static bool placeable(const Tensor& t) { return t.d.fmt == ATS_FMT_Q4B32 || t.d.fmt == ATS_FMT_W16; }
+static bool placeable(const Tensor& t) { return t.d.fmt == ATS_FMT_Q4B32 || t.d.fmt == ATS_FMT_W16 || t.d.fmt == ATS_FMT_MXFP4; }
+// the two 4-bit block formats share the slice layout and every kernel that reads it
+static bool four_bit(const Tensor& t) { return t.d.fmt == ATS_FMT_Q4B32 || t.d.fmt == ATS_FMT_MXFP4; }
+static Tensor* get_4bit(ats_ctx* ctx, int32_t id) {
+  if (id < 0 || (size_t)id >= ctx->tensors.size()) return nullptr;
+  Tensor* t = &ctx->tensors[id];
+  return four_bit(*t) ? t : nullptr;
+}
 static Tensor* get_weight(ats_ctx* ctx, int32_t id) {
   if (id < 0 || (size_t)id >= ctx->tensors.size()) return nullptr;
   Tensor* t = &ctx->tensors[id];
@@ -243,7 +250,7 @@ static int count_streamed(const Operand* ops, int n) {
 // RMSNorm launch when a norm prologue was asked for).  Which kernel runs depends on shapes only, never on placement.
 static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
   p.pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
-  if (!p.w16 && gemv_stream_eligible(p)) {
+  if (gemv_stream_eligible(p)) {
     TimedLaunch tl(ctx, 0, gemv_work_bytes(p));
     ATS_CUDA(launch_gemv_stream(p, ctx->dev_status, ctx->sm_count, ctx->cs, &ctx->stats.kernel_launches));
     return ATS_OK;
@@ -268,6 +275,7 @@ static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
 static int32_t run_gemv_group(ats_ctx* ctx, Operand* ops, int n, GemvParams p) {
   p.K = (int)ops[0].t->d.k_in;
   p.w16 = ops[0].t->d.fmt == ATS_FMT_W16;  // a group shares one format (check_layer)
+  p.mx = ops[0].t->d.fmt == ATS_FMT_MXFP4;
   if (count_streamed(ops, n) <= (int)ctx->cfg.ring_slots || n == 1) {
     ATS_TRY(acquire_ops(ctx, ops, n));
     p.n_seg = n;
@@ -298,6 +306,7 @@ static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
   p.K = (int)ops[0].t->d.k_in;
   p.status = ctx->dev_status;
   p.w16 = ops[0].t->d.fmt == ATS_FMT_W16;  // a group shares one format (check_layer)
+  p.mx = ops[0].t->d.fmt == ATS_FMT_MXFP4;
   std::string err;
   // fp16 weight tiles come through one tensor map per matrix: such a group always runs matrix by matrix
   if ((count_streamed(ops, n) <= (int)ctx->cfg.ring_slots && !p.w16) || n == 1) {
@@ -557,6 +566,7 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
   p.K = (int)t0.d.k_in;
   p.stride = t0.slice_stride;
   p.ids = ids_dev;
+  p.mx = t0.d.fmt == ATS_FMT_MXFP4;
   if (!ids_host) {
     if (call_tab0) {  // per-call tables: resident copies, or slices the copy kernel has gathered into the workspace
       p.tab0 = call_tab0;
@@ -771,7 +781,8 @@ int32_t ats_register_tensor(ats_ctx* ctx, const ats_tensor_desc* d, const void* 
                             int32_t* out_id) {
   ATS_TRY(precheck(ctx, false));
   if (!d || !codes || !out_id) return fail(ctx, ATS_ERR_INVALID, "null argument");
-  if (d->fmt != ATS_FMT_Q4B32 && d->fmt != ATS_FMT_F16 && d->fmt != ATS_FMT_W16) return fail(ctx, ATS_ERR_INVALID, "unknown format %u", d->fmt);
+  if (d->fmt != ATS_FMT_Q4B32 && d->fmt != ATS_FMT_F16 && d->fmt != ATS_FMT_W16 && d->fmt != ATS_FMT_MXFP4)
+    return fail(ctx, ATS_ERR_INVALID, "unknown format %u", d->fmt);
   if (d->n_out == 0 || d->k_in == 0 || d->n_experts == 0) return fail(ctx, ATS_ERR_SHAPE, "zero dimension");
   if (d->switch_cost < 0) return fail(ctx, ATS_ERR_INVALID, "switch_cost must be >= 0");
   Tensor t;
@@ -807,7 +818,19 @@ int32_t ats_register_tensor(ats_ctx* ctx, const ats_tensor_desc* d, const void* 
     t.slice_bytes = t.codes_bytes + N * (K / kBlock) * 2;
     t.slice_stride = align_up(t.slice_bytes);
     t.host_bytes = E * t.slice_stride;
-    if (!(ctx->cfg.flags & ATS_FLAG_SKIP_SCALE_CHECK)) {
+    const bool mx = d->fmt == ATS_FMT_MXFP4;
+    if (mx) {
+      // every weight must be an fp16 value (the tensor-core operand and the fp16 dequantized form): 0.5 * 2^e >= 2^-24
+      // and 6 * 2^e <= 65504 give e = byte - 127 in [-23, 13]; 255 encodes "not a number"
+      const uint8_t* s = (const uint8_t*)scales;
+      const uint64_t ns = E * N * (K / kBlock);
+      for (uint64_t i = 0; i < ns; ++i) {
+        if (s[i] == 255) return fail(ctx, ATS_ERR_INVALID, "block scale %llu is NaN (byte 255)", (unsigned long long)i);
+        if (s[i] < 104 || s[i] > 140)
+          return fail(ctx, ATS_ERR_UNSUPPORTED, "block scale %llu has exponent %d: supported range is -23 .. 13", (unsigned long long)i,
+                      (int)s[i] - 127);
+      }
+    } else if (!(ctx->cfg.flags & ATS_FLAG_SKIP_SCALE_CHECK)) {
       const uint16_t* s = (const uint16_t*)scales;
       const uint64_t ns = E * N * (K / kBlock);
       for (uint64_t i = 0; i < ns; ++i)
@@ -819,7 +842,10 @@ int32_t ats_register_tensor(ats_ctx* ctx, const ats_tensor_desc* d, const void* 
     }
     for (uint64_t e = 0; e < E; ++e) {
       uint8_t* dst = t.host + e * t.slice_stride;
-      repack_q4((const uint8_t*)codes + e * t.codes_bytes, (const uint16_t*)scales + e * N * (K / kBlock), dst, N, K);
+      if (mx)
+        repack_mxfp4((const uint8_t*)codes + e * t.codes_bytes, (const uint8_t*)scales + e * N * (K / kBlock), dst, N, K);
+      else
+        repack_q4((const uint8_t*)codes + e * t.codes_bytes, (const uint16_t*)scales + e * N * (K / kBlock), dst, N, K);
       if (t.slice_stride > t.slice_bytes) memset(dst + t.slice_bytes, 0, t.slice_stride - t.slice_bytes);
     }
     t.slices.resize(E);
@@ -1014,8 +1040,8 @@ static int32_t check_f16(ats_ctx* ctx, int32_t id, uint32_t n_out, uint32_t k_in
 
 int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids, uint32_t M, void* out) {
   ATS_TRY(precheck(ctx, true));
-  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
-  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", id);
+  Tensor* t = get_4bit(ctx, id);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense 4-bit tensor", id);
   if (!token_ids || !out) return fail(ctx, ATS_ERR_INVALID, "null pointer");
   if (M == 0) return ATS_OK;
   const uint8_t* ptr = t->slices[0].dev;
@@ -1033,7 +1059,7 @@ int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids, uint32_t M
     ptr = t->host_dev;
   }
   const int pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
-  ATS_CUDA(launch_embed_rows(ptr, (int)t->d.n_out, (int)t->d.k_in, token_ids, (int)M, (__half*)out, ctx->dev_status, ctx->cs,
+  ATS_CUDA(launch_embed_rows(ptr, (int)t->d.n_out, (int)t->d.k_in, token_ids, (int)M, (__half*)out, ctx->dev_status, t->d.fmt == ATS_FMT_MXFP4, ctx->cs,
                              &ctx->stats.kernel_launches, pdl));
   return ATS_OK;
 }
@@ -1117,8 +1143,8 @@ int32_t ats_linear_static_scratch(ats_ctx* ctx, int32_t id, const void* x, void*
 
 int32_t ats_dequantize(ats_ctx* ctx, int32_t id, int32_t expert, void* out_dev, uint32_t out_fmt) {
   ATS_TRY(precheck(ctx, true));
-  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
-  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not a Q4B32 tensor", id);
+  Tensor* t = get_4bit(ctx, id);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not a 4-bit tensor", id);
   if (expert < 0 || (size_t)expert >= t->slices.size()) return fail(ctx, ATS_ERR_INVALID, "expert %d out of range", expert);
   if (!out_dev || out_fmt > ATS_OUT_F16) return fail(ctx, ATS_ERR_INVALID, "bad output argument");
   plan_begin(ctx);
@@ -1129,7 +1155,7 @@ int32_t ats_dequantize(ats_ctx* ctx, int32_t id, int32_t expert, void* out_dev, 
     ATS_TRY(pump(ctx));
     ATS_TRY(acquire(ctx, f, &ptr));
   }
-  ATS_CUDA(launch_dequant(ptr, (int)t->d.n_out, (int)t->d.k_in, out_dev, out_fmt == ATS_OUT_F16, ctx->cs,
+  ATS_CUDA(launch_dequant(ptr, (int)t->d.n_out, (int)t->d.k_in, out_dev, out_fmt == ATS_OUT_F16, t->d.fmt == ATS_FMT_MXFP4, ctx->cs,
                           &ctx->stats.kernel_launches));
   if (f >= 0) ATS_TRY(release(ctx, f));
   return ATS_OK;
@@ -1152,8 +1178,8 @@ int32_t ats_route_topk(ats_ctx* ctx, int32_t router_id, const void* h, uint32_t 
 int32_t ats_moe_linear(ats_ctx* ctx, int32_t id, const void* x, const int32_t* ids_dev, void* y, uint32_t M, uint32_t k,
                        uint32_t x_per_slot) {
   ATS_TRY(precheck(ctx, true));
-  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
-  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not a Q4B32 tensor", id);
+  Tensor* t = get_4bit(ctx, id);
+  if (!t) return fail(ctx, ATS_ERR_INVALID, "id %d is not a 4-bit tensor", id);
   if (!x || !y || !ids_dev) return fail(ctx, ATS_ERR_INVALID, "null pointer");
   const uint32_t P = M * k;
   if (P == 0) return ATS_OK;
@@ -1183,7 +1209,7 @@ static int32_t check_q4(ats_ctx* ctx, int32_t id, uint32_t fmt, uint32_t n_out, 
   Tensor* t = get_tensor(ctx, id, fmt);
   if (!t)
     return fail(ctx, ATS_ERR_INVALID, "layer tensor %s (id %d) is not a registered %s tensor (a layer's weight matrices share one format)",
-                name, id, fmt == ATS_FMT_W16 ? "W16" : "Q4B32");
+                name, id, fmt == ATS_FMT_W16 ? "W16" : fmt == ATS_FMT_MXFP4 ? "MXFP4" : "Q4B32");
   if (t->d.n_out != n_out || t->d.k_in != k_in || t->slices.size() != n_experts)
     return fail(ctx, ATS_ERR_SHAPE, "layer tensor %s is [%zu][%u][%u], the layer needs [%u][%u][%u]", name, t->slices.size(),
                 t->d.n_out, t->d.k_in, n_experts, n_out, k_in);
@@ -1205,7 +1231,7 @@ static int32_t check_layer(ats_ctx* ctx, const ats_layer_desc* L, bool prefill) 
   // the format of w_gate decides: every other matrix of the layer must have it too
   uint32_t fmt = ATS_FMT_Q4B32;
   if (Tensor* tg = get_weight(ctx, L->w_gate)) fmt = tg->d.fmt;
-  if (fmt == ATS_FMT_W16 && L->n_experts) return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE layers take Q4B32 expert tensors");
+  if (fmt == ATS_FMT_W16 && L->n_experts) return fail(ctx, ATS_ERR_UNSUPPORTED, "MoE layers take 4-bit expert tensors");
   if (L->wq >= 0) {
     if (L->head_dim != 64 && L->head_dim != 128) return fail(ctx, ATS_ERR_UNSUPPORTED, "head_dim %u (64 or 128)", L->head_dim);
     if (L->n_kv_heads == 0 || L->n_q_heads % L->n_kv_heads) return fail(ctx, ATS_ERR_SHAPE, "n_q_heads %% n_kv_heads != 0");
@@ -1363,6 +1389,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     // read it again, and the ring path, which moves every distinct expert once, is the better one.
     MoeGemvParams probe1{}, probe2{};
     probe1.K = H; probe1.n_rows = (int)L->ffn; probe1.mode = GEMV_SWIGLU_F16;
+    probe1.mx = probe2.mx = tg.d.fmt == ATS_FMT_MXFP4;
     probe2.K = (int)L->ffn; probe2.n_rows = H; probe2.mode = GEMV_OUT_F32;
     if (moe_gemv_stream_eligible(probe1) && moe_gemv_stream_eligible(probe2)) implicit = true;
   }
@@ -1379,6 +1406,8 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     if ((ctx->cfg.flags & ATS_FLAG_MOE_DEVICE_GATHER) && tg.host_dev && tu.host_dev && td.host_dev) {
       MoeGemvParams probe1{}, probe2{};
       probe1.K = H; probe1.n_rows = (int)L->ffn; probe1.mode = GEMV_SWIGLU_F16;
+      probe1.mx = probe2.mx = tg.d.fmt == ATS_FMT_MXFP4;
+    probe1.mx = probe2.mx = tg.d.fmt == ATS_FMT_MXFP4;
       probe2.K = (int)L->ffn; probe2.n_rows = H; probe2.mode = GEMV_OUT_F32;
       const Tensor* ts3[3] = {&tg, &tu, &td};
       std::vector<uint8_t> sel(E, 0);
@@ -1644,6 +1673,7 @@ int32_t ats_layer_prefill(ats_ctx* ctx, const ats_layer_desc* L, const void* x_i
     m.grp_off = w.grp_off;
     m.n_groups = E;
     m.grp_max_rows = max_rows;
+    m.mx = tg.d.fmt == ATS_FMT_MXFP4;
     // gate | up side by side
     m.n_seg = 2;
     m.K = H;

@@ -32,6 +32,24 @@ __device__ __forceinline__ void unpack8(uint32_t w, __half2 (&c)[4]) {
   c[3] = __hfma2(u32_as_half2((w8 & 0x00F000F0u) | kMagic), k16th, kM72);
 }
 
+// The microscaling 4-bit float (1 sign, 2 exponent bits with bias 1, 1 mantissa bit; exponent 0 is subnormal) in the same
+// word layout.  The three magnitude bits placed at bits 11..9 of an fp16 (the two low exponent bits and the top mantissa
+// bit) read as the element times 2^-14, subnormal case included, since both formats treat exponent field 0 the same way;
+// one multiplication by 2^14 (exact) gives the element.  Pair j sits in nibbles j and j + 4.
+__device__ __forceinline__ void unpack8_mx(uint32_t w, __half2 (&c)[4]) {
+  const __half2 k2p14 = u32_as_half2(0x74007400u);  // 16384
+  const uint32_t kMag = 0x0E000E00u, kSgn = 0x80008000u;
+  c[0] = __hmul2(u32_as_half2(((w << 9) & kMag) | ((w << 12) & kSgn)), k2p14);
+  c[1] = __hmul2(u32_as_half2(((w << 5) & kMag) | ((w << 8) & kSgn)), k2p14);
+  c[2] = __hmul2(u32_as_half2(((w << 1) & kMag) | ((w << 4) & kSgn)), k2p14);
+  c[3] = __hmul2(u32_as_half2(((w >> 3) & kMag) | (w & kSgn)), k2p14);
+}
+// 8 exact fp16 element values of one word in either 4-bit format (mx: uniform over the launch)
+__device__ __forceinline__ void unpack8_any(uint32_t w, __half2 (&c)[4], int mx) {
+  if (mx) unpack8_mx(w, c);
+  else unpack8(w, c);
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -47,13 +65,13 @@ __device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.0f +
 
 // ------------------------------------------------------------------------------------------- dequantize (a1)
 template <bool F16>
-__global__ void dequant_kernel(const uint8_t* __restrict__ slice, int n_rows, int K, void* __restrict__ out) {
+__global__ void dequant_kernel(const uint8_t* __restrict__ slice, int n_rows, int K, void* __restrict__ out, int mx) {
   const uint64_t words = (uint64_t)n_rows * K / 8;
   const uint32_t* codes = reinterpret_cast<const uint32_t*>(slice);
   const __half* scales = reinterpret_cast<const __half*>(slice + (uint64_t)n_rows * K / 2);
   for (uint64_t w = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; w < words; w += (uint64_t)gridDim.x * blockDim.x) {
     __half2 c[4];
-    unpack8(codes[w], c);
+    unpack8_any(codes[w], c, mx);
     const __half s = scales[w / 4];  // 4 words per block of 32
     if (F16) {
       const __half2 s2 = __half2half2(s);
@@ -81,7 +99,7 @@ __global__ void dequant_kernel(const uint8_t* __restrict__ slice, int n_rows, in
 // Embedding lookup: out[m] = rn16(scale * code) of row ids[m] of a Q4B32 table (the fp16 form ats_dequantize writes).
 // One thread per code word; ids outside [0, n_rows) give a row of zeros and raise the status word.
 __global__ void embed_rows_kernel(const uint8_t* __restrict__ slice, int n_rows, int K, const int32_t* __restrict__ ids, int M,
-                                  __half* __restrict__ out, int* __restrict__ status) {
+                                  __half* __restrict__ out, int* __restrict__ status, int mx) {
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the ids may come from the preceding kernel
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int wpr = K / 8;  // words per row
@@ -93,7 +111,7 @@ __global__ void embed_rows_kernel(const uint8_t* __restrict__ slice, int n_rows,
     uint4 o = make_uint4(0, 0, 0, 0);
     if (row >= 0 && row < n_rows) {
       __half2 c[4];
-      unpack8(codes[(uint64_t)row * wpr + w], c);
+      unpack8_any(codes[(uint64_t)row * wpr + w], c, mx);
       const __half2 s2 = __half2half2(scales[(uint64_t)row * (K / 32) + w / 4]);
       __half2 r0 = __hmul2(c[0], s2), r1 = __hmul2(c[1], s2), r2 = __hmul2(c[2], s2), r3 = __hmul2(c[3], s2);
       o.x = *reinterpret_cast<uint32_t*>(&r0);
@@ -108,22 +126,22 @@ __global__ void embed_rows_kernel(const uint8_t* __restrict__ slice, int n_rows,
 }
 
 cudaError_t launch_embed_rows(const uint8_t* slice, int n_rows, int K, const int32_t* ids, int M, __half* out, int* status,
-                              cudaStream_t st, uint64_t* n_launch, int pdl) {
+                              int mx, cudaStream_t st, uint64_t* n_launch, int pdl) {
   const uint64_t words = (uint64_t)M * K / 8;
   const int grid = (int)std::min<uint64_t>((words + 255) / 256, 148 * 8);
   ++*n_launch;
-  return launch_dep(embed_rows_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, slice, n_rows, K, ids, M, out, status);
+  return launch_dep(embed_rows_kernel, dim3(grid), dim3(256), 0, st, pdl, 1, slice, n_rows, K, ids, M, out, status, mx);
 }
 
-cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, cudaStream_t st,
+cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, int mx, cudaStream_t st,
                            uint64_t* n_launch) {
   const uint64_t words = (uint64_t)n_rows * K / 8;
   const int block = 256;
   const int grid = (int)std::min<uint64_t>((words + block - 1) / block, 148 * 16);
   if (out_f16)
-    dequant_kernel<true><<<grid, block, 0, st>>>(slice, n_rows, K, out);
+    dequant_kernel<true><<<grid, block, 0, st>>>(slice, n_rows, K, out, mx);
   else
-    dequant_kernel<false><<<grid, block, 0, st>>>(slice, n_rows, K, out);
+    dequant_kernel<false><<<grid, block, 0, st>>>(slice, n_rows, K, out, mx);
   ++*n_launch;
   return cudaGetLastError();
 }
@@ -312,7 +330,7 @@ constexpr int kWR = 4;  // weight rows a CTA works on at once
 template <int M>
 __device__ __forceinline__ void gemv_accumulate(const uint4* const (&cptr)[kWR], const __half* const (&sptr)[kWR],
                                                 const bool (&valid)[kWR], const __half* __restrict__ x, int ldx, int nblk,
-                                                float (&acc)[kWR][M]) {
+                                                float (&acc)[kWR][M], int mx) {
   const int nthreads = blockDim.x;
   for (int blk = threadIdx.x; blk < nblk; blk += nthreads) {
     uint4 q[kWR];
@@ -323,7 +341,7 @@ __device__ __forceinline__ void gemv_accumulate(const uint4* const (&cptr)[kWR],
         q[i] = __ldg(cptr[i] + blk);
         s[i] = __half2float(sptr[i][blk]);
       } else {
-        q[i] = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);
+        q[i] = mx ? make_uint4(0, 0, 0, 0) : make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);
         s[i] = 0.f;
       }
     }
@@ -348,7 +366,7 @@ __device__ __forceinline__ void gemv_accumulate(const uint4* const (&cptr)[kWR],
       for (int i = 0; i < kWR; ++i) {
         const uint32_t word = j == 0 ? q[i].x : j == 1 ? q[i].y : j == 2 ? q[i].z : q[i].w;
         __half2 c[4];
-        unpack8(word, c);
+        unpack8_any(word, c, mx);
         float cf[8];
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
@@ -425,7 +443,7 @@ __global__ void __launch_bounds__(kGemvMaxWarps * 32) gemv_kernel(const GemvPara
   for (int i = 0; i < kWR; ++i)
 #pragma unroll
     for (int m = 0; m < M; ++m) acc[i][m] = 0.f;
-  gemv_accumulate<M>(cptr, sptr, valid, p.x, p.ldx, nblk, acc);
+  gemv_accumulate<M>(cptr, sptr, valid, p.x, p.ldx, nblk, acc, p.mx);
   gemv_reduce<M>(acc, red, tot);
 
   if (SW) {
@@ -533,7 +551,7 @@ __global__ void __launch_bounds__(kGemvMaxWarps * 32)
   float acc[kWR][1];
 #pragma unroll
   for (int i = 0; i < kWR; ++i) acc[i][0] = 0.f;
-  gemv_accumulate<1>(cptr, sptr, valid, p.x + (size_t)xrow * p.ldx, p.ldx, nblk, acc);
+  gemv_accumulate<1>(cptr, sptr, valid, p.x + (size_t)xrow * p.ldx, p.ldx, nblk, acc, p.mx);
   gemv_reduce<1>(acc, red, tot);
   if (SW) {
     if (threadIdx.x < kWR / 2) {

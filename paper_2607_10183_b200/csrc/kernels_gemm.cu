@@ -166,7 +166,26 @@ __device__ __forceinline__ uint4 dequant8(uint32_t w, __half2 s2) {
   return o;
 }
 
-template <int FT, int TT>
+// The same for a word of microscaling 4-bit floats: the magnitude bits land on bits 11..9 of each fp16 (= element * 2^-14,
+// exponent-0 subnormals included), 2^14 and the power-of-two block scale follow as two exact multiplications.
+__device__ __forceinline__ uint4 dequant8_mx(uint32_t w, __half2 s2) {
+  const __half2 k2p14 = u2h2(0x74007400u);
+  const uint32_t kMag = 0x0E000E00u, kSgn = 0x80008000u;
+  const __half2 c0 = __hmul2(__hmul2(u2h2(((w << 9) & kMag) | ((w << 12) & kSgn)), k2p14), s2);
+  const __half2 c1 = __hmul2(__hmul2(u2h2(((w << 5) & kMag) | ((w << 8) & kSgn)), k2p14), s2);
+  const __half2 c2 = __hmul2(__hmul2(u2h2(((w << 1) & kMag) | ((w << 4) & kSgn)), k2p14), s2);
+  const __half2 c3 = __hmul2(__hmul2(u2h2(((w >> 3) & kMag) | (w & kSgn)), k2p14), s2);
+  uint4 o;
+  o.x = *reinterpret_cast<const uint32_t*>(&c0);
+  o.y = *reinterpret_cast<const uint32_t*>(&c1);
+  o.z = *reinterpret_cast<const uint32_t*>(&c2);
+  o.w = *reinterpret_cast<const uint32_t*>(&c3);
+  return o;
+}
+
+// MX: the code words hold microscaling 4-bit floats (a compile-time switch: the branch inside the dequantization loop
+// costs the integer-code kernel 5 % when taken at run time).
+template <int FT, int TT, bool MX>
 __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap, const GemmKParams p) {
   using Cfg = TileCfg<FT, TT>;
   constexpr int BF = Cfg::BF, TTILE = TT, MB = TT / BM, kDequantWarps = Cfg::kDequantWarps, kStageBytes = Cfg::kStageBytes;
@@ -357,7 +376,12 @@ __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) ge
           if (!vec_sc) sbuf[d] = fetch_scale1(ks0 + i + kPD);
         }
         // the arithmetic needs no shared memory: do it before waiting for the stage to drain
-        const uint4 o0 = dequant8(c0.x, s0), o1 = dequant8(c0.y, s0), o2 = dequant8(c0.z, s0), o3 = dequant8(c0.w, s0);
+        uint4 o0, o1, o2, o3;
+        if constexpr (MX) {
+          o0 = dequant8_mx(c0.x, s0), o1 = dequant8_mx(c0.y, s0), o2 = dequant8_mx(c0.z, s0), o3 = dequant8_mx(c0.w, s0);
+        } else {
+          o0 = dequant8(c0.x, s0), o1 = dequant8(c0.y, s0), o2 = dequant8(c0.z, s0), o3 = dequant8(c0.w, s0);
+        }
         if (round > 0) {
           // one lane polls for the warp: hundreds of threads hammering the same mbarrier word slow its arrivals down
           int got = 1;
@@ -699,10 +723,14 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   for (int i = 0; i < 3; ++i) p.grp_tab[i] = g.grp_tab[i];
   static uint64_t attr_done = 0;
   if (first_use_on_device(&attr_done)) {
-    cudaError_t e1 = cudaFuncSetAttribute(gemm_q4_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    cudaError_t e2 = cudaFuncSetAttribute(gemm_q4_kernel<1, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e1 = cudaFuncSetAttribute(gemm_q4_kernel<2, 256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e2 = cudaFuncSetAttribute(gemm_q4_kernel<1, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e3 = cudaFuncSetAttribute(gemm_q4_kernel<2, 256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e4 = cudaFuncSetAttribute(gemm_q4_kernel<1, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e1 != cudaSuccess) return e1;
     if (e2 != cudaSuccess) return e2;
+    if (e3 != cudaSuccess) return e3;
+    if (e4 != cudaSuccess) return e4;
   }
   dim3 grid(tiles, tchunks, g.grp_off ? g.n_groups : p.splits);
   ++*n_launch;
@@ -710,13 +738,17 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   if (wide) {
     using Cfg = TileCfg<2, 256>;
     p.stages = Cfg::kStages;
-    e = launch_dep(gemm_q4_kernel<2, 256>, grid, dim3(Cfg::kThreads), (size_t)Cfg::kStages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, wmap, p);
+    const size_t smem = (size_t)Cfg::kStages * Cfg::kStageBytes + 1024;
+    e = g.mx ? launch_dep(gemm_q4_kernel<2, 256, true>, grid, dim3(Cfg::kThreads), smem, st, g.pdl, 1, xmap, wmap, p)
+             : launch_dep(gemm_q4_kernel<2, 256, false>, grid, dim3(Cfg::kThreads), smem, st, g.pdl, 1, xmap, wmap, p);
   } else {
     using Cfg = TileCfg<1, 128>;
     // Grouped form: every CTA streams its own expert's weights once and has few real rows, so what counts is how many
     // weight loads are in flight per SM: three stages let two CTAs share an SM (registers are capped for that).
     p.stages = g.grp_off ? 3 : Cfg::kStages;
-    e = launch_dep(gemm_q4_kernel<1, 128>, grid, dim3(Cfg::kThreads), (size_t)p.stages * Cfg::kStageBytes + 1024, st, g.pdl, 1, xmap, wmap, p);
+    const size_t smem = (size_t)p.stages * Cfg::kStageBytes + 1024;
+    e = g.mx ? launch_dep(gemm_q4_kernel<1, 128, true>, grid, dim3(Cfg::kThreads), smem, st, g.pdl, 1, xmap, wmap, p)
+             : launch_dep(gemm_q4_kernel<1, 128, false>, grid, dim3(Cfg::kThreads), smem, st, g.pdl, 1, xmap, wmap, p);
   }
   if (e != cudaSuccess) return e;
   if (p.splits > 1) {

@@ -69,7 +69,7 @@ int parts_for(int K) { return stream_parts_for(K); }
 
 }  // namespace
 
-bool gemv_stream_eligible(const GemvParams& p) { return stream_shape_ok(p); }
+bool gemv_stream_eligible(const GemvParams& p) { return !p.w16 && !p.mx && stream_shape_ok(p); }  // integer codes only
 
 cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch) {
   const int parts = parts_for(g.K);
@@ -108,6 +108,7 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
 }
 
 bool moe_gemv_stream_eligible(const MoeGemvParams& p) {
+  if (p.mx) return false;  // integer codes only
   if (p.K % 256 != 0 || p.K > 16384) return false;
   const int rows = kGroupWarps / parts_for(p.K) * kRPW;
   if (p.mode == GEMV_SWIGLU_F16) return p.n_rows % (rows / 2) == 0;

@@ -144,6 +144,28 @@ void repack_q4(const uint8_t* codes_in, const uint16_t* scales_in, uint8_t* slic
   for (uint64_t i = 0; i < ns; ++i) so[i] = scales_in[i];
 }
 
+// The microscaling 4-bit format into the same slice layout.  The element encodings are kept (no offset), in the same
+// nibble order; a scale byte b (2^(b - 127), accepted range 104..140) becomes the fp16 with that value: a normal number
+// for exponents >= -14, a subnormal (one mantissa bit) below.
+void repack_mxfp4(const uint8_t* codes_in, const uint8_t* scale_bytes_in, uint8_t* slice_out, uint64_t n_rows, uint64_t K) {
+  const uint64_t words = n_rows * K / 8;
+  uint32_t* out = reinterpret_cast<uint32_t*>(slice_out);
+  for (uint64_t w = 0; w < words; ++w) {
+    const uint8_t* p = codes_in + 4 * w;
+    const uint32_t v = (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24);
+    const uint32_t ev = v & 0x0F0F0F0Fu, od = (v >> 4) & 0x0F0F0F0Fu;
+    const uint32_t evp = (ev & 0xF) | ((ev >> 4) & 0xF0) | ((ev >> 8) & 0xF00) | ((ev >> 12) & 0xF000);
+    const uint32_t odp = (od & 0xF) | ((od >> 4) & 0xF0) | ((od >> 8) & 0xF00) | ((od >> 12) & 0xF000);
+    out[w] = evp | (odp << 16);
+  }
+  uint16_t* so = reinterpret_cast<uint16_t*>(slice_out + n_rows * K / 2);
+  const uint64_t ns = n_rows * (K / kBlock);
+  for (uint64_t i = 0; i < ns; ++i) {
+    const int e = (int)scale_bytes_in[i] - 127;
+    so[i] = e >= -14 ? (uint16_t)((e + 15) << 10) : (uint16_t)(1u << (e + 24));
+  }
+}
+
 }  // namespace ats
 
 extern "C" {

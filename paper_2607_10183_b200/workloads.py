@@ -196,6 +196,15 @@ def moe_block(config: int, layer: int, shape: MoEShape = MOE_FULL) -> dict:
     return out
 
 
+def moe_block_mxfp4(config: int, layer: int, shape: MoEShape = MOE_FULL) -> dict:
+    """An MoE FFN block whose stacked expert tensors are in the microscaling 4-bit format (router and gain as before)."""
+    out = moe_block(config, layer, shape)
+    out[ROLE_GATE] = mxfp4_packed(config, layer, ROLE_GATE, shape.ffn, shape.hidden, shape.n_experts)
+    out[ROLE_UP] = mxfp4_packed(config, layer, ROLE_UP, shape.ffn, shape.hidden, shape.n_experts)
+    out[ROLE_DOWN] = mxfp4_packed(config, layer, ROLE_DOWN, shape.hidden, shape.ffn, shape.n_experts)
+    return out
+
+
 def q4_bytes(n_out: int, k_in: int) -> int:
     """Bytes of one block-quantized matrix: 4-bit codes plus one fp16 scale per 32 weights."""
     return n_out * k_in // 2 + n_out * (k_in // BLOCK) * 2
