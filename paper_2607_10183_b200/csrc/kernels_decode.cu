@@ -304,7 +304,7 @@ cudaError_t launch_gemv_w16(const GemvParams& g, cudaStream_t st, uint64_t* n_la
   // Split K while the units alone give fewer warps than the machine holds (4 CTAs of 8 warps per SM) and every part keeps
   // at least one full pass of a warp (128 pieces of 16 bytes).  A function of the shapes only.
   int ks = 1;
-  while (ks < 8 && (long)n_units * ks <= 148L * 32 && (g.K / 8) / (ks * 2) >= 128) ks *= 2;
+  while (ks < 8 && (long)n_units * ks <= 2 * 148L * 32 && (g.K / 8) / (ks * 2) >= 128) ks *= 2;
   p.ksplit = ks;
   const int upc = 8 / ks;
   const dim3 grid(std::max(1, std::min((n_units + upc - 1) / upc, 148 * 8))), block(256);
@@ -681,12 +681,66 @@ __global__ void __launch_bounds__(256) rmsnorm16_vec_kernel(const __half* __rest
   }
 }
 
+// The same for fp32 rows (the residual stream between the two halves of a decode layer): eight elements per thread and
+// pass as two 16-byte loads, held in registers between the passes.
+__global__ void __launch_bounds__(256) rmsnorm32_vec_kernel(const float* __restrict__ x, const __half* __restrict__ gain,
+                                                            __half* __restrict__ out, int H, float eps) {
+  __shared__ float red[8];
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int n8 = H / 8;
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)blockIdx.x * H);
+  float4 xa[4], xb[4];
+  uint4 gv[4];
+  float ss = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = threadIdx.x + 256 * j;
+    xa[j] = xb[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    gv[j] = make_uint4(0, 0, 0, 0);
+    if (c < n8) {
+      xa[j] = xr[2 * c];
+      xb[j] = xr[2 * c + 1];
+      gv[j] = __ldg(reinterpret_cast<const uint4*>(gain) + c);
+    }
+    ss = fmaf(xa[j].x, xa[j].x, ss); ss = fmaf(xa[j].y, xa[j].y, ss); ss = fmaf(xa[j].z, xa[j].z, ss); ss = fmaf(xa[j].w, xa[j].w, ss);
+    ss = fmaf(xb[j].x, xb[j].x, ss); ss = fmaf(xb[j].y, xb[j].y, ss); ss = fmaf(xb[j].z, xb[j].z, ss); ss = fmaf(xb[j].w, xb[j].w, ss);
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) t += red[w];
+  const float inv = 1.0f / sqrtf(t / (float)H + eps);
+  uint4* orow = reinterpret_cast<uint4*>(out + (size_t)blockIdx.x * H);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = threadIdx.x + 256 * j;
+    if (c < n8) {
+      const float f[8] = {xa[j].x, xa[j].y, xa[j].z, xa[j].w, xb[j].x, xb[j].y, xb[j].z, xb[j].w};
+      const uint32_t g[4] = {gv[j].x, gv[j].y, gv[j].z, gv[j].w};
+      uint32_t o[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 gg = __half22float2(u32_as_half2(g[q]));
+        const __half2 h = __floats2half2_rn(f[2 * q] * gg.x * inv, f[2 * q + 1] * gg.y * inv);
+        o[q] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      orow[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+}
+
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
                            cudaStream_t st, uint64_t* n_launch, int pdl) {
   ++*n_launch;
   if (!x_is_f32 && H % 8 == 0 && H <= 8192 &&
       (((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(out)) & 15) == 0))
     return launch_dep(rmsnorm16_vec_kernel, dim3(M), dim3(256), 0, st, pdl, 1, (const __half*)x, gain, out, H, eps);
+  if (x_is_f32 && H % 8 == 0 && H <= 8192 &&
+      (((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(out)) & 15) == 0))
+    return launch_dep(rmsnorm32_vec_kernel, dim3(M), dim3(256), 0, st, pdl, 1, (const float*)x, gain, out, H, eps);
   if (x_is_f32) return launch_dep(rmsnorm_kernel<float>, dim3(M), dim3(256), 0, st, pdl, 1, (const float*)x, gain, out, H, eps);
   return launch_dep(rmsnorm_kernel<__half>, dim3(M), dim3(256), 0, st, pdl, 1, (const __half*)x, gain, out, H, eps);
 }
