@@ -315,7 +315,7 @@ int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n);
  * the normalised row is rounded to fp16 before the product (the contract's edge "h").  M = 1 runs as one launch of the
  * streaming GEMV with the norm as its prologue (hidden <= 4096 and a shape that kernel takes); otherwise a norm launch
  * into `scratch` (DEVICE fp16 [M][hidden], caller-provided, may be NULL only for the one-launch case) and ats_linear.
- * A W16 head always takes the second form (scratch required). */
+ * A W16 or MXFP4 head always takes the second form (scratch required). */
 int32_t ats_embed(ats_ctx* ctx, int32_t id, const int32_t* token_ids /*DEVICE*/, uint32_t M, void* out /*DEVICE*/);
 int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, const void* x /*DEVICE*/, void* logits /*DEVICE*/,
                     uint32_t M, void* scratch /*DEVICE*/);

@@ -1089,7 +1089,9 @@ int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, c
     probe.K = K;
     probe.n_seg = 1;
     probe.seg[0] = GemvSeg{nullptr, N};
-    if (!scratch && (t->d.fmt == ATS_FMT_W16 || !gemv_stream_eligible(probe)))
+    probe.w16 = t->d.fmt == ATS_FMT_W16;
+    probe.mx = t->d.fmt == ATS_FMT_MXFP4;
+    if (!scratch && !gemv_stream_eligible(probe))
       return fail(ctx, ATS_ERR_INVALID, "ats_lm_head needs `scratch` for this shape (the norm runs as a launch of its own)");
     plan_begin(ctx);
     Operand op;

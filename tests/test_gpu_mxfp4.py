@@ -260,3 +260,27 @@ def test_moe_block_prefill_matches_oracle(B, torch, T):
     assert clear.sum() >= T - 2
     H.assert_close(outs[0][clear], want[clear], what="mxfp4 moe prefill block")
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+
+
+@pytest.mark.parametrize("M", [1, 12])
+def test_lm_head_matches_oracle(B, torch, M):
+    """Final norm + vocabulary projection with an MXFP4 head: a norm launch, then the generic GEMV or the GEMM; without
+    scratch the call is refused (this format has no one-launch form)."""
+    V, Hd, eps = 1000, 448, 1e-5
+    packed, sb = W.mxfp4_packed(91, 3, W.ROLE_Q, V, Hd)
+    gain = W.activations(91, 3, (Hd,)).astype(np.float16)
+    x = W.activations(91, 4, (M, Hd))
+    ctx = ctx_for(B, W.q4_bytes(V, Hd) + 64 * 1024, ws=16 * MB)
+    nid, hid = ctx.register_f16(gain), ctx.register_mxfp4(packed, sb)
+    ctx.set_placement([(hid, -1, B.ATS_GPU)])
+    logits = torch.empty((M, V), dtype=torch.float16, device="cuda")
+    scratch = torch.empty((M, Hd), dtype=torch.float16, device="cuda")
+    ctx.lm_head(nid, hid, eps, H.to_dev(x), logits, M, scratch)
+    ctx.sync()
+    edges, wmode = ctx.numerics(B.ATS_MODE_PREFILL if M > 8 else B.ATS_MODE_DECODE)
+    H.assert_close(logits.cpu().numpy(), O.lm_head(x, gain, eps, packed, sb, wmode), what=f"mxfp4 lm head M={M}")
+    if M == 1:
+        with pytest.raises(B.AtsError) as e:
+            ctx.lm_head(nid, hid, eps, H.to_dev(x), logits, 1, None)
+        assert e.value.code == B.ATS_ERR_INVALID
+    ctx.close()
