@@ -240,9 +240,32 @@ def extra_gemv(torch, B, W, peaks, quick):
     alg = nb + K * 2 + N * 2
     back_to_back = alg * n / (ms * 1e-3) / 1e9
     kernel = st.timed_work[0] / (st.timed_ms[0] * 1e-3) / 1e9
-    return {"workload": "config 1: GEMV 4096x4096, batch 1, resident, 64 replicas rotated", "algorithmic_bytes": alg,
-            "us_per_call_back_to_back": ms * 1e3 / n, "gbs_back_to_back": back_to_back, "kernel_us": st.timed_ms[0] * 1e3 / st.timed_launches[0],
-            "gbs_kernel": kernel, "frac_of_measured_hbm": kernel / peaks["hbm_gbs"], "frac_of_nominal_8TBs": kernel / 8000.0}
+    out = {"workload": "config 1: GEMV 4096x4096, batch 1, resident, 64 replicas rotated", "algorithmic_bytes": alg,
+           "us_per_call_back_to_back": ms * 1e3 / n, "gbs_back_to_back": back_to_back, "kernel_us": st.timed_ms[0] * 1e3 / st.timed_launches[0],
+           "gbs_kernel": kernel, "frac_of_measured_hbm": kernel / peaks["hbm_gbs"], "frac_of_nominal_8TBs": kernel / 8000.0}
+    # several activation rows against one matrix (14336x4096, 4 replicas rotated): one row runs on the streaming kernel,
+    # two on the generic kernel, three to eight on the mma.sync kernel
+    N2, reps2 = 14336, 4
+    nb2 = W.q4_bytes(N2, K)
+    ctx = B.Context(reps2 * (nb2 + 256) + (4 << 20), workspace_bytes=1 << 20)
+    ids2 = [ctx.register_q4(*W.q4_packed(1, 1, W.ROLE_GATE, N2, K)) for _ in range(reps2)]
+    ctx.set_placement([(i, -1, B.ATS_GPU) for i in ids2])
+    rows = {}
+    for M in (1, 2, 4, 8):
+        xm = torch.from_numpy(W.activations(1, 1, (M, K))).cuda()
+        ym = torch.empty((M, N2), dtype=torch.float16, device="cuda")
+
+        def go2(k):
+            for i in range(k):
+                ctx.linear(ids2[i % reps2], xm, ym, M)
+        go2(2 * reps2)
+        ctx.sync()
+        k = reps2 * (10 if quick else 40)
+        us = event_time_ms(torch, ctx.compute, lambda: go2(k)) * 1e3 / k
+        rows[f"M{M}"] = {"us_per_call": us, "weight_gbs": nb2 / us / 1e3, "frac_of_measured_hbm": nb2 / us / 1e3 / peaks["hbm_gbs"]}
+    ctx.close()
+    out["rows_14336x4096"] = rows
+    return out
 
 
 def extra_prefill(torch, B, W, peaks, quick):

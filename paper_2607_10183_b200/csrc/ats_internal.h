@@ -153,6 +153,9 @@ cudaError_t launch_gemv(const GemvParams& p, cudaStream_t st, uint64_t* n_launch
 // fp16-weight GEMV (kernels_decode.cu): the same segments, epilogue modes and fp32 accumulation as launch_gemv over
 // unquantized fp16 matrices; M <= 8, K a multiple of 8, x given (the norm prologue fields are ignored)
 cudaError_t launch_gemv_w16(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
+// few-row GEMV of the 4-bit formats on mma.sync (kernels_gemv_mma.cu): same segments and epilogues as launch_gemv, x given
+bool gemv_mma_eligible(const GemvParams& p);
+cudaError_t launch_gemv_mma(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
 // the streaming single-token kernel (kernels_gemv_stream.cu): shapes it accepts, and its launcher
 bool gemv_stream_eligible(const GemvParams& p);
 cudaError_t launch_gemv_stream(const GemvParams& p, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch);

@@ -246,8 +246,9 @@ static int count_streamed(const Operand* ops, int n) {
   return c;
 }
 
-// One GEMV launch: the streaming kernel where the shapes allow it, else the generic kernel (preceded by a separate
-// RMSNorm launch when a norm prologue was asked for).  Which kernel runs depends on shapes only, never on placement.
+// One GEMV launch: the streaming kernel where the shapes allow it (one row of integer codes), else the fp16-weight kernel,
+// the mma.sync kernel (4-bit formats, three to eight rows) or the generic kernel, preceded by a separate RMSNorm launch
+// when a norm prologue was asked for.  Which kernel runs depends on format and shapes only, never on placement.
 static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
   p.pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
   if (gemv_stream_eligible(p)) {
@@ -265,6 +266,8 @@ static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
   TimedLaunch tl(ctx, 0, gemv_work_bytes(p));
   if (p.w16)
     ATS_CUDA(launch_gemv_w16(p, ctx->cs, &ctx->stats.kernel_launches));
+  else if (p.M >= 3 && gemv_mma_eligible(p))  // from three rows on the tensor-core form is the faster one (its cost does not grow with M)
+    ATS_CUDA(launch_gemv_mma(p, ctx->cs, &ctx->stats.kernel_launches));
   else
     ATS_CUDA(launch_gemv(p, ctx->cs, &ctx->stats.kernel_launches));
   return ATS_OK;
