@@ -4,22 +4,24 @@
 // The generic GEMV decodes every weight to fp32 and spends a fused multiply-add per weight and activation row: about five
 // thread instructions per weight, which is what bounds it (not HBM) for the microscaling format and for several rows.
 // Here a warp owns 16 weight rows; the weights of a 16 x 16 tile are the A operand, decoded straight into fp16 pairs in
-// the fragment layout (each thread decodes only the pair the layout gives it: two shifts and two logic operations for the
-// microscaling format, a shift, a logic operation and one fp16 subtraction for the integer codes), the M activation rows
+// the fragment layout (two shifts and two logic operations per pair for the microscaling format, one logic
+// operation and one fp16 operation for the integer codes), the M activation rows
 // are the eight columns of the B operand, and one instruction does the 16 x 16 x 8 products.  Products of fp16 values are
 // exact in fp32; the two k-steps of a 32-wide block accumulate in the instruction's fp32 accumulator, the block's scale
 // is applied in fp32 and blocks are summed in fp32, so weights stay exact as in the generic kernel.  The layout:
-//   A (16 x 16, row):  reg0 = (row g, k 2t..2t+1), reg1 = (row g+8, same k), reg2 = (row g, k 2t+8..2t+9), reg3 = (row g+8, ..)
-//   B (16 x 8, col):   reg0 = (k 2t..2t+1, column g), reg1 = (k 2t+8..2t+9, column g)
+//   A (16 x 16, row):  reg0 = (row g, kk 2t..2t+1), reg1 = (row g+8, same kk), reg2 = (row g, kk 2t+8..2t+9), reg3 = (row g+8, ..)
+//   B (16 x 8, col):   reg0 = (kk 2t..2t+1, column g), reg1 = (kk 2t+8..2t+9, column g)
 //   C (16 x 8):        c0 c1 = (row g, columns 2t 2t+1), c2 c3 = (row g+8, columns 2t 2t+1)        g = lane / 4, t = lane % 4
-// and a code word holds k = 0..7 of its row with the pair (2j, 2j+1) in nibbles j and j + 4, so thread t takes pair t of
-// word 2s (reg0/1) and of word 2s+1 (reg2/3) in k-step s.
+// The instruction sums over its sixteen kk whatever they stand for, so the k of a 32-wide block are dealt to the two
+// instructions in the order that suits the data: lane t takes k = 8t .. 8t+7 of the block, that is ONE code word per row
+// (word t of the block's four) and 16 contiguous bytes of x, with the word's pairs (2j, 2j+1), j = 0..3, as
+// (instruction j / 2, reg 0/1 or 2/3 by j % 2) on both operands.  All shifts of the decode are compile-time constants.
 //
 // A unit is 16 consecutive output rows (SwiGLU: 16 gate rows and the 16 up rows of the same outputs).  1, 2, 4 or 8 warps of
 // the CTA share a unit, each on its own part of K; partial tiles meet in shared memory and are added in fixed order.
-// Code loads are 16 bytes per thread and row; the four lanes that share a row pair load four consecutive blocks (64
-// contiguous bytes per row) and hand the words round by shuffle, four such loads per row in flight (sixteen blocks), the
-// first batch issued before the grid dependency resolves (weights do not depend on the preceding kernel).
+// Code loads are 4 bytes per thread, row and block (the quad's four words are the block's 16 contiguous bytes), sixteen
+// blocks in flight, the first batch issued before the grid dependency resolves (weights do not depend on the preceding
+// kernel).
 #include "ats_internal.h"
 
 namespace ats {
@@ -47,25 +49,29 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], 
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Pair t (nibbles t and t + 4) of a code word as two fp16 values.
-//   MX = false: offset-binary integer codes u = c + 8: the fp16 pair 1024 + u minus 1032.
+// The four pairs (k = 2j, 2j+1 in nibbles j and j + 4) of a code word as fp16 pairs.
+//   MX = false: offset-binary integer codes u = c + 8.  (w & 0x000F000F) | 0x6400.. is the fp16 pair 1024 + u, the
+//     0x00F000F0 pair is 1024 + 16 u: one subtraction or one multiply-add gives c exactly.
 //   MX = true: microscaling floats: magnitude bits onto bits 11..9 of each half, sign onto bit 15: element * 2^-14.
 template <bool MX>
-__device__ __forceinline__ uint32_t decode_pair(uint32_t w, int t) {
+__device__ __forceinline__ void decode_word(uint32_t w, uint32_t (&a)[4]) {
   if (MX) {
-    const uint32_t mag = __funnelshift_l(w, w, (9 - 4 * t) & 31) & 0x0E000E00u;
-    return (__funnelshift_l(w, w, (12 - 4 * t) & 31) & 0x80008000u) | mag;
+    const uint32_t kMag = 0x0E000E00u, kSgn = 0x80008000u;
+    a[0] = ((w << 9) & kMag) | ((w << 12) & kSgn);
+    a[1] = ((w << 5) & kMag) | ((w << 8) & kSgn);
+    a[2] = ((w << 1) & kMag) | ((w << 4) & kSgn);
+    a[3] = ((w >> 3) & kMag) | (w & kSgn);
   } else {
-    const uint32_t u = ((w >> (4 * t)) & 0x000F000Fu) | 0x64006400u;
-    __half2 h, k1032;
-    *reinterpret_cast<uint32_t*>(&h) = u;
-    *reinterpret_cast<uint32_t*>(&k1032) = 0x64086408u;
-    h = __hsub2(h, k1032);
-    return *reinterpret_cast<uint32_t*>(&h);
+    auto h2 = [](uint32_t v) { __half2 h; *reinterpret_cast<uint32_t*>(&h) = v; return h; };
+    auto u32 = [](__half2 h) { return *reinterpret_cast<uint32_t*>(&h); };
+    const uint32_t kMagic = 0x64006400u, w8 = w >> 8;
+    const __half2 k1032 = h2(0x64086408u), k16th = h2(0x2C002C00u), kM72 = h2(0xD480D480u);
+    a[0] = u32(__hsub2(h2((w & 0x000F000Fu) | kMagic), k1032));
+    a[1] = u32(__hfma2(h2((w & 0x00F000F0u) | kMagic), k16th, kM72));
+    a[2] = u32(__hsub2(h2((w8 & 0x000F000Fu) | kMagic), k1032));
+    a[3] = u32(__hfma2(h2((w8 & 0x00F000F0u) | kMagic), k16th, kM72));
   }
 }
-
-__device__ __forceinline__ uint32_t pick_word(const uint4& q, int j) { return j == 0 ? q.x : j == 1 ? q.y : j == 2 ? q.z : q.w; }
 
 // N (4, 8 or 16) consecutive block scales of a row as packed fp16 pairs: one or two vector loads where the address allows,
 // else scalar loads; blocks at or beyond b_hi read as zero.
@@ -101,7 +107,7 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const MmaGemvParams p) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   bool waited = false;  // x and the residual come from the preceding kernel; the first weight loads need not wait for it
   constexpr int NT = SW ? 2 : 1;   // weight tiles per unit
-  constexpr int NB = SW ? 1 : 2;   // 16-byte loads in flight per thread and row: a batch covers 4 * NB blocks
+  constexpr int NBK = SW ? 8 : 16;  // blocks in flight per thread and row
   __shared__ float red_s[8][NT][16][8];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -133,9 +139,8 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const MmaGemvParams p) {
   const int per = (((nblk + ks - 1) / ks) + 15) & ~15;  // blocks per part: whole batches, so that scale loads stay aligned
   const int b_lo = part * per, b_hi = min(nblk, b_lo + per);
   const uint32_t zero_word = MX ? 0u : 0x88888888u;  // eight zeros in either format
-  const __half* xrow = p.x + (size_t)min(g, M - 1) * p.ldx + 2 * t;
+  const __half* xrow = p.x + (size_t)min(g, M - 1) * p.ldx + 8 * t;
   const bool xlive = g < M;
-  const int quad = lane & ~3;
   for (int u0 = blockIdx.x * upc; u0 < n_units; u0 += gridDim.x * upc) {
     const int u = u0 + slot;
     float acc[NT][4];
@@ -154,57 +159,43 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const MmaGemvParams p) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) row_ptrs(live[h] ? r : 0, nt, cp[nt][h], sp[nt][h]);
       }
-      for (int b0 = b_lo; b0 < b_hi; b0 += 4 * NB) {
-        // The four lanes of a quad share their two rows: lane t loads blocks b0 + 4 i + t (64 contiguous bytes per row and
-        // quad), and each block's words travel to the other three lanes by shuffle when the block is consumed.
-        uint4 q[NB][NT][2];
-        uint32_t sc[NT][2][2 * NB];
+      for (int b0 = b_lo; b0 < b_hi; b0 += NBK) {
+        // Lane t of a quad loads word t of every block of its two rows (the quad's four words are the block's 16 contiguous
+        // bytes), NBK blocks in flight.
+        uint32_t q[NBK][NT][2];
+        uint32_t sc[NT][2][NBK / 2];
 #pragma unroll
-        for (int i = 0; i < NB; ++i) {
-          const int b = b0 + 4 * i + t;
+        for (int j = 0; j < NBK; ++j) {
+          const int b = b0 + j;
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int h = 0; h < 2; ++h)
-              q[i][nt][h] = (live[h] && b < b_hi) ? __ldcs(cp[nt][h] + b) : make_uint4(zero_word, zero_word, zero_word, zero_word);
+              q[j][nt][h] = (live[h] && b < b_hi) ? __ldg(reinterpret_cast<const uint32_t*>(cp[nt][h] + b) + t) : zero_word;
         }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-          for (int h = 0; h < 2; ++h) load_scales<4 * NB>(sp[nt][h], b0, b_hi, live[h], sc[nt][h]);
+          for (int h = 0; h < 2; ++h) load_scales<NBK>(sp[nt][h], b0, b_hi, live[h], sc[nt][h]);
         if (!waited) {
           asm volatile("griddepcontrol.wait;" ::: "memory");
           waited = true;
         }
 #pragma unroll
-        for (int j = 0; j < 4 * NB; ++j) {
+        for (int j = 0; j < NBK; ++j) {
           const int b = b0 + j;
           if (b >= b_hi) break;  // uniform over the warp
-          uint32_t xb[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) xb[e] = xlive ? __ldg(reinterpret_cast<const uint32_t*>(xrow + b * 32 + 8 * e)) : 0u;
-          const int src = quad | (j & 3);
+          // x[b * 32 + 8 t .. + 7]: the four pairs this lane's word multiplies, in instruction order
+          const uint4 xv = xlive ? __ldg(reinterpret_cast<const uint4*>(xrow + b * 32)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
-            uint32_t wd[2][4];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const uint4& v = q[j >> 2][nt][h];
-              wd[h][0] = __shfl_sync(0xffffffffu, v.x, src);
-              wd[h][1] = __shfl_sync(0xffffffffu, v.y, src);
-              wd[h][2] = __shfl_sync(0xffffffffu, v.z, src);
-              wd[h][3] = __shfl_sync(0xffffffffu, v.w, src);
-            }
+            uint32_t a0[4], a1[4];
+            decode_word<MX>(q[j][nt][0], a0);
+            decode_word<MX>(q[j][nt][1], a1);
             float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int s = 0; s < 2; ++s) {
-              uint32_t a[4];
-              a[0] = decode_pair<MX>(wd[0][2 * s], t);
-              a[1] = decode_pair<MX>(wd[1][2 * s], t);
-              a[2] = decode_pair<MX>(wd[0][2 * s + 1], t);
-              a[3] = decode_pair<MX>(wd[1][2 * s + 1], t);
-              mma16816(c, a, xb[2 * s], xb[2 * s + 1]);
-            }
+            const uint32_t f0[4] = {a0[0], a1[0], a0[1], a1[1]}, f1[4] = {a0[2], a1[2], a0[3], a1[3]};
+            mma16816(c, f0, xv.x, xv.y);
+            mma16816(c, f1, xv.z, xv.w);
             const float s0 = scale_of(sc[nt][0], j), s1 = scale_of(sc[nt][1], j);
             acc[nt][0] = fmaf(s0, c[0], acc[nt][0]);
             acc[nt][1] = fmaf(s0, c[1], acc[nt][1]);
@@ -257,7 +248,7 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const MmaGemvParams p) {
 
 bool gemv_mma_eligible(const GemvParams& g) {
   if (g.w16 || g.M < 1 || g.M > 8 || g.K % 32 || g.n_seg < 1 || g.n_seg > 3) return false;
-  if ((g.ldx & 1) || (reinterpret_cast<uintptr_t>(g.x) & 3)) return false;  // activation pairs are read as 32-bit words
+  if ((g.ldx & 7) || (reinterpret_cast<uintptr_t>(g.x) & 15)) return false;  // a lane reads its eight activations as 16 bytes
   if (g.mode == GEMV_SWIGLU_F16 && (g.n_seg != 2 || g.seg[0].n_rows != g.seg[1].n_rows)) return false;
   for (int s = 0; s < g.n_seg; ++s)
     if ((reinterpret_cast<uintptr_t>(g.seg[s].base) & 15) || (g.K / 2) % 16) return false;  // 16-byte code loads per block
