@@ -644,6 +644,40 @@ def extra_mxfp4(torch, B, W, peaks, quick):
         tf = 2.0 * T * N * K / (ms * 1e-3) / 1e12
         out[f"gemm_{N}x{K}_T{T}"] = {"us_per_call": ms * 1e3, "tflops": tf, "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"]}
         ctx.close()
+    # the whole dense layer of config 2 with MXFP4 matrices: one decode step at context 1024, four weight copies in rotation
+    shape = W.DENSE_FULL
+    names = {W.ROLE_Q: "wq", W.ROLE_K: "wk", W.ROLE_V: "wv", W.ROLE_O: "wo", W.ROLE_GATE: "w_gate", W.ROLE_UP: "w_up", W.ROLE_DOWN: "w_down"}
+    layer_bytes = sum(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
+    cap, reps = 1025, 4
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=cap)
+    ws = B.workspace_bytes(probe, 1) + (1 << 20)
+    ctx = B.Context(ws + reps * (layer_bytes + (1 << 20)) + (4 << 20), workspace_bytes=ws)
+    Lw = W.dense_layer_mxfp4(17, 0, shape)
+    descs, wids = [], []
+    for l in range(reps):
+        ids = {"attn_norm": ctx.register_f16(Lw[W.ROLE_ATTN_NORM], l, W.ROLE_ATTN_NORM), "ffn_norm": ctx.register_f16(Lw[W.ROLE_FFN_NORM], l, W.ROLE_FFN_NORM)}
+        for r in names:
+            ids[names[r]] = ctx.register_mxfp4(*Lw[r], layer=l, role=r)
+            wids.append(ids[names[r]])
+        descs.append(B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                                  head_dim=shape.head_dim, kv_capacity=cap, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, **ids))
+    ctx.set_placement([(t, -1, B.ATS_GPU) for t in wids])
+    kc, vc = W.kv_cache(17, 0, shape.n_kv_heads, cap, shape.head_dim, 1024)
+    kd, vd = torch.from_numpy(kc).cuda(), torch.from_numpy(vc).cuda()
+    x1 = torch.from_numpy(W.activations(17, 2, (1, shape.hidden))).cuda()
+    y1 = torch.empty_like(x1)
+
+    def dec(n):
+        for i in range(n):
+            ctx.layer_decode(descs[i % reps], x1, y1, kd, vd, 1024, 1)
+    dec(8)
+    ctx.sync()
+    n = 40 if quick else 400
+    us = event_time_ms(torch, ctx.compute, lambda: dec(n)) * 1e3 / n
+    out["layer_decode_ctx1024"] = {"us_per_layer": us, "weight_bytes": layer_bytes, "weight_gbs": layer_bytes / us / 1e3,
+                                   "frac_of_measured_hbm": layer_bytes / us / 1e3 / peaks["hbm_gbs"], "tokens_per_s": 1e6 / us}
+    ctx.close()
     return out
 
 

@@ -66,8 +66,8 @@ enum { ATS_FMT_Q4B32 = 0, ATS_FMT_F16 = 1, ATS_FMT_W16 = 2, ATS_FMT_MXFP4 = 3 };
  * (not a number): ATS_ERR_INVALID; exponents outside -23 .. 13 (bytes 104 .. 140): ATS_ERR_UNSUPPORTED, because every
  * weight must be an fp16 value (it is the tensor-core operand).  Inside the library the tensor has the slice layout and
  * size of a Q4B32 tensor (the scale kept as an fp16 power of two) and takes every call a Q4B32 tensor takes, dense or
- * stacked; weights are exact in both the GEMV and the GEMM.  The single-token streaming kernels are integer-code
- * kernels: MXFP4 tensors run on the generic GEMV kernels. */
+ * stacked; weights are exact in both the GEMV and the GEMM.  The single-token streaming kernels have a mode for this
+ * format (twice an element is an integer, looked up per nibble and fed to the same integer dot products). */
 enum { ATS_OUT_F32 = 0, ATS_OUT_F16 = 1 };      /* ats_dequantize output */
 enum { ATS_MODE_DECODE = 0, ATS_MODE_PREFILL = 1 };
 

@@ -119,7 +119,14 @@ __device__ __forceinline__ int f2i_magic(float x, float up) {
 // The quantization is done by four adjacent lanes, each holding one run of 8 consecutive elements (one code word's
 // worth) of a 32-element block: exponent maximum and integer sum are shared by two butterfly shuffles.  Lane w of the
 // group writes words 4w..4w+3.
+//
+// Microscaling 4-bit floats (MX): twice an element is an integer in [-12, 12]; the kernel looks the biased byte
+// 2 e + 16 up per nibble (see mx_bytes) and uses the same unsigned dot products: sum xi (2 e + 16) = 2 sum xi e + 16 sum xi,
+// so mul is halved and the correction stays -8 * sum(xi) * mul.  The lookup yields the bytes of a word's even k
+// (0,2,4,6) and odd k (1,3,5,7), so for this format words 4w..4w+3 hold the pairs (xi_0, xi_2), (xi_4, xi_6), (xi_1, xi_3),
+// (xi_5, xi_7) of the run.
 constexpr int kXqWords = 20;  // 18 used; the 80-byte pitch keeps the 128-bit reads of consecutive blocks conflict-free
+template <bool MX>
 __device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32_t* blk) {
   uint32_t m = 0;
 #pragma unroll
@@ -141,12 +148,33 @@ __device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32
   sx += __shfl_xor_sync(0xffffffffu, sx, 1);
   sx += __shfl_xor_sync(0xffffffffu, sx, 2);
   uint4 o;
-  o.x = __byte_perm((uint32_t)xi[0], (uint32_t)xi[4], 0x5410u);
-  o.y = __byte_perm((uint32_t)xi[1], (uint32_t)xi[5], 0x5410u);
-  o.z = __byte_perm((uint32_t)xi[2], (uint32_t)xi[6], 0x5410u);
-  o.w = __byte_perm((uint32_t)xi[3], (uint32_t)xi[7], 0x5410u);
+  if (MX) {
+    o.x = __byte_perm((uint32_t)xi[0], (uint32_t)xi[2], 0x5410u);
+    o.y = __byte_perm((uint32_t)xi[4], (uint32_t)xi[6], 0x5410u);
+    o.z = __byte_perm((uint32_t)xi[1], (uint32_t)xi[3], 0x5410u);
+    o.w = __byte_perm((uint32_t)xi[5], (uint32_t)xi[7], 0x5410u);
+  } else {
+    o.x = __byte_perm((uint32_t)xi[0], (uint32_t)xi[4], 0x5410u);
+    o.y = __byte_perm((uint32_t)xi[1], (uint32_t)xi[5], 0x5410u);
+    o.z = __byte_perm((uint32_t)xi[2], (uint32_t)xi[6], 0x5410u);
+    o.w = __byte_perm((uint32_t)xi[3], (uint32_t)xi[7], 0x5410u);
+  }
   *reinterpret_cast<uint4*>(blk + 4 * w) = o;
-  if (w == 0) *reinterpret_cast<float2*>(blk + 16) = make_float2(mul, -8.0f * (float)sx * mul);
+  if (w == 0) *reinterpret_cast<float2*>(blk + 16) = make_float2(MX ? 0.5f * mul : mul, -8.0f * (float)sx * mul);
+}
+
+// Four nibbles (the low 16 bits of sel: sign bit, three magnitude bits each) -> the bytes 2 e + 16 of their elements.
+// Twice the magnitudes are v = 0 1 2 3 4 6 8 12.  Two eight-byte tables for prmt: 16 - v, looked up with the sign bits
+// masked out, and 2 v, looked up with the sign bit left in the selector, where prmt returns the sign of the table byte
+// (0: every entry is positive) instead of the byte.  Their sum is 16 + v for a non-negative element and 16 - v for a
+// negative one; no byte exceeds 40, so one 32-bit addition adds the four bytes without carries.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));  // generic form: selector bit 3 = replicate the byte's sign
+  return d;
+}
+__device__ __forceinline__ uint32_t mx_bytes(uint32_t sel) {
+  return prmt(0x0D0E0F10u, 0x04080A0Cu, sel & 0x7777u) + prmt(0x06040200u, 0x18100C08u, sel);
 }
 
 struct StreamSeg {
@@ -278,7 +306,7 @@ __device__ __forceinline__ bool stream_produce(const StreamParams& p, const int 
 // group with its own partial-sum buffer and barrier, so the tile loop is that of two independent 8-warp CTAs; what they
 // share is the activation prologue: all 512 consumer threads load, normalise and quantise the row ONCE per SM.
 // Returns false after a bounded wait ran out (status word raised).
-template <int PARTS, bool SW, typename WaitFn>
+template <int PARTS, bool SW, bool MX, typename WaitFn>
 __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int bx, const int gx, StreamShared& sh,
                                                const StreamRing& ring, WaitFn wait_dep, const bool release_dependents) {
   constexpr int ROWS = kGroupWarps / PARTS * kRPW;     // weight rows per tile
@@ -366,7 +394,7 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
           xv[2 * q + 1] = f.y;
         }
         if (p.h_out && bx == 0) *reinterpret_cast<uint4*>(p.h_out + i0) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-        quantize_run4(xv, tid & 3, xq_s + (size_t)(tid >> 2) * kXqWords);
+        quantize_run4<MX>(xv, tid & 3, xq_s + (size_t)(tid >> 2) * kXqWords);
       }
     } else {
       uint4 raw[4];
@@ -391,7 +419,7 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
             xv[2 * q] = f.x;
             xv[2 * q + 1] = f.y;
           }
-          quantize_run4(xv, r & 3, xq_s + (size_t)(r >> 2) * kXqWords);
+          quantize_run4<MX>(xv, r & 3, xq_s + (size_t)(r >> 2) * kXqWords);
         }
       }
     }
@@ -476,13 +504,22 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
           int dl = 0, dh = 0;
 #pragma unroll
           for (int w = 0; w < 4; ++w) {
-            const uint32_t lo = ws[w] & 0x0F0F0F0Fu, hi = ws[w] & 0xF0F0F0F0u;  // hi carries 16 * code
-            dl = dp2a_lo(xr[j][4 * w], lo, dl);
-            dl = dp2a_hi(xr[j][4 * w + 1], lo, dl);
-            dh = dp2a_lo(xr[j][4 * w + 2], hi, dh);
-            dh = dp2a_hi(xr[j][4 * w + 3], hi, dh);
+            if (MX) {
+              const uint32_t ev = mx_bytes(ws[w]), od = mx_bytes(ws[w] >> 16);  // k = 0 2 4 6 and k = 1 3 5 7 of the word
+              dl = dp2a_lo(xr[j][4 * w], ev, dl);
+              dl = dp2a_hi(xr[j][4 * w + 1], ev, dl);
+              dh = dp2a_lo(xr[j][4 * w + 2], od, dh);
+              dh = dp2a_hi(xr[j][4 * w + 3], od, dh);
+            } else {
+              const uint32_t lo = ws[w] & 0x0F0F0F0Fu, hi = ws[w] & 0xF0F0F0F0u;  // hi carries 16 * code
+              dl = dp2a_lo(xr[j][4 * w], lo, dl);
+              dl = dp2a_hi(xr[j][4 * w + 1], lo, dl);
+              dh = dp2a_lo(xr[j][4 * w + 2], hi, dh);
+              dh = dp2a_hi(xr[j][4 * w + 3], hi, dh);
+            }
           }
-          const float dot = (float)(dl + (dh >> 4));  // dh is a multiple of 16; |dot| < 2^24: exact
+          // integer codes: dh is a multiple of 16; either way |dot| < 2^24: exact
+          const float dot = MX ? (float)(dl + dh) : (float)(dl + (dh >> 4));
           acc[r] = fmaf(sc[r][j], fmaf(dot, xm[j], xc[j]), acc[r]);
         }
       }

@@ -7,7 +7,7 @@ namespace ats {
 namespace {
 
 // A whole kernel as one phase: the ring starts empty, the grid dependency is resolved by griddepcontrol.
-template <int PARTS, bool SW>
+template <int PARTS, bool SW, bool MX>
 __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool wait_first) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ StreamShared sh;
@@ -20,12 +20,12 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
     if ((threadIdx.x & 31) == 0) stream_produce<PARTS, SW, true>(p, bx, gx, wait_first, sh, ring, l2_evict_first_policy());
     return;
   }
-  stream_consume<PARTS, SW>(p, bx, gx, sh, ring, [] { asm volatile("griddepcontrol.wait;" ::: "memory"); }, true);
+  stream_consume<PARTS, SW, MX>(p, bx, gx, sh, ring, [] { asm volatile("griddepcontrol.wait;" ::: "memory"); }, true);
 }
 
-template <int PARTS, bool SW>
+template <int PARTS, bool SW, bool MX>
 __global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamParams p) {
-  gemv_stream_body<PARTS, SW>(p, (int)blockIdx.x, (int)gridDim.x, false);
+  gemv_stream_body<PARTS, SW, MX>(p, (int)blockIdx.x, (int)gridDim.x, false);
 }
 
 // Grouped-expert variant: blockIdx.y selects the job (a (token, slot) pair), whose expert slices, activation row and
@@ -41,7 +41,7 @@ struct MoeSel {
   int x_div;
   int ldx, ldy;
 };
-template <int PARTS, bool SW>
+template <int PARTS, bool SW, bool MX>
 __global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
   StreamParams p = p0;
   const int job = blockIdx.y;
@@ -62,14 +62,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const Stre
   p.x16 = p0.x16 + (size_t)xrow * m.ldx;
   if (p0.y32) p.y32 = p0.y32 + (size_t)orow * m.ldy;
   if (p0.y16) p.y16 = p0.y16 + (size_t)orow * m.ldy;
-  gemv_stream_body<PARTS, SW>(p, (int)blockIdx.x, (int)gridDim.x, m.ids != nullptr);
+  gemv_stream_body<PARTS, SW, MX>(p, (int)blockIdx.x, (int)gridDim.x, m.ids != nullptr);
 }
 
 int parts_for(int K) { return stream_parts_for(K); }
 
 }  // namespace
 
-bool gemv_stream_eligible(const GemvParams& p) { return !p.w16 && !p.mx && stream_shape_ok(p); }  // integer codes only
+bool gemv_stream_eligible(const GemvParams& p) { return !p.w16 && stream_shape_ok(p); }  // the two 4-bit formats
 
 cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch) {
   const int parts = parts_for(g.K);
@@ -80,14 +80,23 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   const size_t smem = kStages * stage_bytes + stream_xq_bytes(g.K);
   const int grid = std::max(1, std::min(tiles, sm_count));
   void (*kern)(const StreamParams) = nullptr;
-  switch (parts) {
-    case 1: kern = sw ? gemv_stream_kernel<1, true> : gemv_stream_kernel<1, false>; break;
-    case 2: kern = sw ? gemv_stream_kernel<2, true> : gemv_stream_kernel<2, false>; break;
-    case 4: kern = sw ? gemv_stream_kernel<4, true> : gemv_stream_kernel<4, false>; break;
-    default: kern = sw ? gemv_stream_kernel<8, true> : gemv_stream_kernel<8, false>; break;
+  if (g.mx) {
+    switch (parts) {
+      case 1: kern = sw ? gemv_stream_kernel<1, true, true> : gemv_stream_kernel<1, false, true>; break;
+      case 2: kern = sw ? gemv_stream_kernel<2, true, true> : gemv_stream_kernel<2, false, true>; break;
+      case 4: kern = sw ? gemv_stream_kernel<4, true, true> : gemv_stream_kernel<4, false, true>; break;
+      default: kern = sw ? gemv_stream_kernel<8, true, true> : gemv_stream_kernel<8, false, true>; break;
+    }
+  } else {
+    switch (parts) {
+      case 1: kern = sw ? gemv_stream_kernel<1, true, false> : gemv_stream_kernel<1, false, false>; break;
+      case 2: kern = sw ? gemv_stream_kernel<2, true, false> : gemv_stream_kernel<2, false, false>; break;
+      case 4: kern = sw ? gemv_stream_kernel<4, true, false> : gemv_stream_kernel<4, false, false>; break;
+      default: kern = sw ? gemv_stream_kernel<8, true, false> : gemv_stream_kernel<8, false, false>; break;
+    }
   }
-  static uint64_t attr_done[8] = {};
-  const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
+  static uint64_t attr_done[16] = {};
+  const int ki = ((parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
     if (e != cudaSuccess) return e;
@@ -108,7 +117,6 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
 }
 
 bool moe_gemv_stream_eligible(const MoeGemvParams& p) {
-  if (p.mx) return false;  // integer codes only
   if (p.K % 256 != 0 || p.K > 16384) return false;
   const int rows = kGroupWarps / parts_for(p.K) * kRPW;
   if (p.mode == GEMV_SWIGLU_F16) return p.n_rows % (rows / 2) == 0;
@@ -150,14 +158,23 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
   const int per_job = std::max(1, std::min(p.n_tiles, sm_count / n_jobs));  // one wave: a CTA fills its SM
   void (*kern)(const StreamParams, const MoeSel, const MoeJobs) = nullptr;
-  switch (parts) {
-    case 1: kern = sw ? gemv_stream_moe_kernel<1, true> : gemv_stream_moe_kernel<1, false>; break;
-    case 2: kern = sw ? gemv_stream_moe_kernel<2, true> : gemv_stream_moe_kernel<2, false>; break;
-    case 4: kern = sw ? gemv_stream_moe_kernel<4, true> : gemv_stream_moe_kernel<4, false>; break;
-    default: kern = sw ? gemv_stream_moe_kernel<8, true> : gemv_stream_moe_kernel<8, false>; break;
+  if (g.mx) {
+    switch (parts) {
+      case 1: kern = sw ? gemv_stream_moe_kernel<1, true, true> : gemv_stream_moe_kernel<1, false, true>; break;
+      case 2: kern = sw ? gemv_stream_moe_kernel<2, true, true> : gemv_stream_moe_kernel<2, false, true>; break;
+      case 4: kern = sw ? gemv_stream_moe_kernel<4, true, true> : gemv_stream_moe_kernel<4, false, true>; break;
+      default: kern = sw ? gemv_stream_moe_kernel<8, true, true> : gemv_stream_moe_kernel<8, false, true>; break;
+    }
+  } else {
+    switch (parts) {
+      case 1: kern = sw ? gemv_stream_moe_kernel<1, true, false> : gemv_stream_moe_kernel<1, false, false>; break;
+      case 2: kern = sw ? gemv_stream_moe_kernel<2, true, false> : gemv_stream_moe_kernel<2, false, false>; break;
+      case 4: kern = sw ? gemv_stream_moe_kernel<4, true, false> : gemv_stream_moe_kernel<4, false, false>; break;
+      default: kern = sw ? gemv_stream_moe_kernel<8, true, false> : gemv_stream_moe_kernel<8, false, false>; break;
+    }
   }
-  static uint64_t attr_done[8] = {};
-  const int ki = (parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0);
+  static uint64_t attr_done[16] = {};
+  const int ki = ((parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
     if (e != cudaSuccess) return e;

@@ -284,3 +284,60 @@ def test_lm_head_matches_oracle(B, torch, M):
             ctx.lm_head(nid, hid, eps, H.to_dev(x), logits, 1, None)
         assert e.value.code == B.ATS_ERR_INVALID
     ctx.close()
+
+
+def test_dense_layer_decode_full_size_on_the_streaming_kernel(B, torch):
+    """Config-2 shapes with MXFP4 matrices: every GEMV of the step runs on the streaming single-token kernel (norm prologue,
+    fused QKV, residual epilogues, fused gate/up + SwiGLU) in its microscaling mode; output against the oracle, and the
+    same bits with the FFN matrices streamed from the host."""
+    shape, cfg, pos, cap = W.DENSE_FULL, 91, 300, 301
+    L = W.dense_layer_mxfp4(cfg, 0, shape)
+    t = H.oracle_dense_tensors(L)
+    by_name = {H.ROLE_NAME[r]: W.q4_bytes(n, k) for r, n, k in shape.tensor_shapes()}
+    slot = max(by_name.values())
+    x = W.activations(cfg, 0, (1, shape.hidden))
+    outs = []
+    for placement in (ALL_GPU, dict(ALL_GPU, w_gate=0, w_up=0, w_down=0)):
+        ctx = ctx_for(B, sum(by_name.values()) + 16 * 256 + 4 * shape.hidden * 2, slot=slot, chunk=4 * MB)
+        desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+        ctx.set_placement([(ids[n], -1, w) for n, w in placement.items()])
+        edges, wmode = ctx.numerics(B.ATS_MODE_DECODE)
+        kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos)
+        kd, vd = H.to_dev(kc), H.to_dev(vc)
+        y = torch.empty((1, shape.hidden), dtype=torch.float16, device="cuda")
+        ctx.reset_stats()
+        ctx.layer_decode(desc, H.to_dev(x), y, kd, vd, pos, 1)
+        ctx.sync()
+        assert ctx.stats().kernel_launches == 5  # four streaming GEMVs and the attention kernel: no separate norm launch
+        outs.append(y.cpu().numpy())
+        if placement is ALL_GPU:
+            want = O.dense_layer(x, t, shape, kc, vc, pos, edges, wmode)
+            H.assert_close(outs[-1], want, what="mxfp4 decode layer, full size")
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+
+
+@pytest.mark.parametrize("M", [1, 8])
+def test_moe_block_decode_full_size_on_the_streaming_kernel(B, torch, M):
+    """Config-4 shapes (hidden 2048, 128 experts x 768, top-8) with MXFP4 experts: the grouped-expert streaming kernel in its
+    microscaling mode, resident and with the odd experts on the host; ids bit-exact, output against the oracle."""
+    shape, cfg = W.MOE_FULL, 91
+    Bk = W.moe_block_mxfp4(cfg, 0, shape)
+    x = W.activations(cfg, 0, (M, shape.hidden))
+    want, ids_ref, gates_ref, logits = O.moe_block(x, H.oracle_moe_tensors(Bk), shape)
+    assert O.min_rank_gap(logits, shape.top_k) > 1e-4
+    outs = []
+    for host in (set(), {e for e in range(shape.n_experts) if e % 2}):
+        ctx = moe_ctx(B, shape, 32, ring_slots=16)
+        desc, ids = H.register_moe_block(ctx, Bk)
+        ctx.set_placement([(ids[n], e, B.ATS_HOST if e in host else B.ATS_GPU) for n in ("w_gate", "w_up", "w_down")
+                           for e in range(shape.n_experts)])
+        y = torch.empty((M, shape.hidden), dtype=torch.float16, device="cuda")
+        ctx.layer_decode(desc, H.to_dev(x), y, None, None, 0, M)
+        ctx.sync()
+        got_ids = ctx.debug_decode_buffer(desc, M, 8, np.int32).reshape(M, -1)[:, :shape.top_k]
+        assert np.array_equal(got_ids, ids_ref)
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want, what=f"mxfp4 moe block full size M={M}")
+        ctx.close()
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
