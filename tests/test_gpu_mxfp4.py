@@ -202,12 +202,12 @@ def test_dense_layer_prefill_matches_oracle(B, torch, pos0, T, cap):
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
 
 
-def moe_ctx(B, shape, T, ring_slots=8):
+def moe_ctx(B, shape, T, ring_slots=8, flags=0):
     sl = W.q4_bytes(shape.ffn, shape.hidden)
     probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, w_gate=0, w_up=0, w_down=0)
     ws = B.workspace_bytes(probe, T) + MB
     return B.Context(ws + ring_slots * (sl + 256) + 3 * shape.n_experts * (sl + 256) + MB, workspace_bytes=ws, ring_slots=ring_slots,
-                     slot_bytes=sl, chunk_bytes=MB)
+                     slot_bytes=sl, chunk_bytes=MB, flags=flags)
 
 
 @pytest.mark.parametrize("M", [1, 5])
@@ -327,8 +327,11 @@ def test_moe_block_decode_full_size_on_the_streaming_kernel(B, torch, M):
     want, ids_ref, gates_ref, logits = O.moe_block(x, H.oracle_moe_tensors(Bk), shape)
     assert O.min_rank_gap(logits, shape.top_k) > 1e-4
     outs = []
-    for host in (set(), {e for e in range(shape.n_experts) if e % 2}):
-        ctx = moe_ctx(B, shape, 32, ring_slots=16)
+    odd = {e for e in range(shape.n_experts) if e % 2}
+    # resident; odd experts on the host through the ring; the same read in place by the kernel (batch 1) / gathered by the
+    # copy kernel (batch 8) without the host round trip
+    for host, flags in ((set(), 0), (odd, 0), (odd, B.ATS_FLAG_MOE_DEVICE_GATHER)):
+        ctx = moe_ctx(B, shape, 32, ring_slots=16, flags=flags)
         desc, ids = H.register_moe_block(ctx, Bk)
         ctx.set_placement([(ids[n], e, B.ATS_HOST if e in host else B.ATS_GPU) for n in ("w_gate", "w_up", "w_down")
                            for e in range(shape.n_experts)])
@@ -339,5 +342,8 @@ def test_moe_block_decode_full_size_on_the_streaming_kernel(B, torch, M):
         assert np.array_equal(got_ids, ids_ref)
         outs.append(y.cpu().numpy())
         H.assert_close(outs[-1], want, what=f"mxfp4 moe block full size M={M}")
+        if flags and M == 1:
+            assert ctx.stats().host_syncs == 0
         ctx.close()
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+    assert np.array_equal(outs[0].view(np.uint16), outs[2].view(np.uint16))
