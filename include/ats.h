@@ -170,7 +170,8 @@ int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /
  * library has no CPU executor, so that is what stands where the paper has t^c).  The caller forms k = t / bytes and the
  * residency benefit r_i = t_host - t_resident and hands it to Algorithm 1 through ats_set_tensor_value.
  * The call replaces the placement while it measures (this tensor alone on the GPU / on the host, everything else on the
- * host) and puts the previous one back before it returns; it synchronises.  ATS_ERR_BUDGET if the tensor fits neither the
+ * host) and puts the previous one back before it returns; it synchronises, and its launches and copies count in the
+ * statistics like any other call's.  ATS_ERR_BUDGET if the tensor fits neither the
  * resident region nor a ring slot.  Stacked expert tensors: ATS_ERR_INVALID (profile the operator through ats_moe_linear).
  * ats_set_tensor_value: replaces r_i (value < 0: the default, the tensor's byte size) and c_i of a registered weight tensor;
  * the placement in force stays until the next ats_plan_placement. */

@@ -188,7 +188,7 @@ __device__ __forceinline__ uint4 dequant8_mx(uint32_t w, __half2 s2) {
 template <int FT, int TT, bool MX>
 __global__ void __launch_bounds__(TileCfg<FT, TT>::kThreads, FT == 1 ? 2 : 1) gemm_q4_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap, const GemmKParams p) {
   using Cfg = TileCfg<FT, TT>;
-  constexpr int BF = Cfg::BF, TTILE = TT, MB = TT / BM, kDequantWarps = Cfg::kDequantWarps, kStageBytes = Cfg::kStageBytes;
+  constexpr int BF = Cfg::BF, TTILE = TT, MB = TT / BM, kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_a[kMaxStages], full_b[kMaxStages], empty[kMaxStages], acc_full;
