@@ -77,6 +77,7 @@ enum {
   ATS_FLAG_SKIP_SCALE_CHECK = 2u, /* do not scan scales for Inf/NaN at registration */
   ATS_FLAG_TIME_KERNELS = 4u,     /* bracket every GEMV / grouped GEMV / GEMM launch with CUDA events (see ats_stats.timed_*) */
   ATS_FLAG_NO_PDL = 8u,           /* launch every kernel fully serialized (no programmatic dependent launch overlap) */
+  ATS_FLAG_NO_GEMM_PAIR = 32u,    /* do not run large GEMMs as pairs of CTAs on two SMs (tcgen05 cta_group::2): the single-CTA kernel only */
   ATS_FLAG_MOE_DEVICE_GATHER = 16u, /* single-token MoE stages with host-placed experts: no staging ring and no host round trip for the
                                      routing ids: the grouped-expert kernel reads the selected host-placed slices straight
                                      from the pinned host store over PCIe (the store is mapped into the device's address

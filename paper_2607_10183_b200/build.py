@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(HERE, "libats.so")
-SOURCES = ["ats_runtime.cu", "placement.cpp", "transfer_planner.cpp", "kernels_decode.cu", "kernels_gemv_stream.cu", "kernels_gemv_mma.cu", "kernels_prefill.cu", "kernels_gemm.cu"]
+SOURCES = ["ats_runtime.cu", "placement.cpp", "transfer_planner.cpp", "kernels_decode.cu", "kernels_gemv_stream.cu", "kernels_gemv_mma.cu", "kernels_prefill.cu", "kernels_gemm.cu", "kernels_gemm_pair.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
          "-Xcompiler", "-fPIC,-Wall,-Wno-unused-function", "--expt-relaxed-constexpr"]

@@ -323,6 +323,9 @@ struct GemmParams {
 };
 uint64_t gemm_scratch_bytes(int T, int n_total, int K);
 cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);
+// fp16-weight GEMM as a pair of CTAs (kernels_gemm_pair.cu): shapes it takes, and its launcher
+bool gemm_pair_eligible(const GemmParams& p);
+cudaError_t launch_gemm_pair(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);
 // fixed split-K scratch inside the library's device image (no allocation): capacity, and its address on the current device
 uint64_t gemm_static_scratch_capacity();
 cudaError_t gemm_static_scratch(void** out);

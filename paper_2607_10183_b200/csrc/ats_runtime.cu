@@ -344,7 +344,10 @@ static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
     cudaError_t e;
     {
       TimedLaunch tl(ctx, 2, 2ull * (uint64_t)p.T * rows * (uint64_t)p.K);
-      e = launch_gemm(p, ctx->cs, &ctx->stats.kernel_launches, &err);
+      if (!(ctx->cfg.flags & ATS_FLAG_NO_GEMM_PAIR) && gemm_pair_eligible(p))
+        e = launch_gemm_pair(p, ctx->cs, &ctx->stats.kernel_launches, &err);
+      else
+        e = launch_gemm(p, ctx->cs, &ctx->stats.kernel_launches, &err);
     }
     if (e != cudaSuccess) return check_cuda(ctx, e, err.empty() ? "launch_gemm" : err.c_str());
     return release_ops(ctx, ops, n);
@@ -359,7 +362,10 @@ static int32_t run_gemm_group(ats_ctx* ctx, Operand* ops, int n, GemmParams p) {
     cudaError_t e;
     {
       TimedLaunch tl(ctx, 2, 2ull * (uint64_t)q.T * (uint64_t)q.seg[0].n_rows * (uint64_t)q.K);
-      e = launch_gemm(q, ctx->cs, &ctx->stats.kernel_launches, &err);
+      if (!(ctx->cfg.flags & ATS_FLAG_NO_GEMM_PAIR) && gemm_pair_eligible(q))
+        e = launch_gemm_pair(q, ctx->cs, &ctx->stats.kernel_launches, &err);
+      else
+        e = launch_gemm(q, ctx->cs, &ctx->stats.kernel_launches, &err);
     }
     if (e != cudaSuccess) return check_cuda(ctx, e, err.empty() ? "launch_gemm" : err.c_str());
     ATS_TRY(release_ops(ctx, ops + i, 1));

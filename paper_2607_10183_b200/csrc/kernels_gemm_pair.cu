@@ -1,0 +1,327 @@
+// fp16-weight GEMM as a pair of CTAs on two SMs (tcgen05 cta_group::2): Y[T][N] = X[T][K] * W^T, W an unquantized fp16 matrix.
+//
+// A single CTA that computes 256 tokens x 256 features reads 96 bytes of operands per cycle from shared memory while
+// the tensor pipe is busy and refills 64 more: above the SM's 128.  As a pair, the instruction computes 256 tokens
+// (128 from each CTA's shared memory) x 256 features (128 weight rows from each CTA's shared memory), so every CTA
+// reads 64 bytes per cycle and refills 47.  Pair tile: 512 tokens (two 128-token blocks per CTA, one accumulator each,
+// all 512 tensor-memory columns of both SMs) x 256 features.
+//
+// Roles in each CTA: warp 0 = TMA producer (activations of its 256 tokens and its 128 weight rows, boxes of 64 rows x 64 k,
+// 128-byte swizzle), warp 1 = tensor-memory allocation (both CTAs, cta_group::2) and, in the leader (even rank) only,
+// MMA issue; warps 2..9 = epilogue (tcgen05.ld of the CTA's own accumulators, fp16 stores).
+// Barriers: the loads of BOTH CTAs complete on the leader's full barrier (loads carry cta_group::2 and name that barrier:
+// the own barrier's address with the peer bit cleared), for which the leader posts the byte count of both; the leader's
+// tcgen05.commit releases a stage in both CTAs (one commit per CTA: its own barrier, then the peer's through mapa).
+// Every mbarrier wait is bounded; a CTA that gives up raises the status word and skips its work, but every thread still
+// reaches the closing cluster barrier, so that no CTA leaves while its partner may still signal it.
+#include <cuda.h>
+
+#include "ats_internal.h"
+
+namespace ats {
+
+namespace {
+
+constexpr int BM = 128, BK = 64, BOXR = 64;
+constexpr int kTokPerCta = 256, kFeatPerCta = 128;           // per CTA: two token blocks, half of the pair's 256 features
+constexpr int kXBytes = kTokPerCta * BK * 2;                 // 32 KB
+constexpr int kWBytes = kFeatPerCta * BK * 2;                // 16 KB
+constexpr int kStageBytes = kXBytes + kWBytes;               // 48 KB
+constexpr int kStages = 4;
+constexpr int kThreads = 10 * 32;
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;               // clears the CTA-rank bit of a shared::cluster address
+
+struct PairParams {
+  int K, T, N;
+  int ksteps;
+  __half* y;
+  int ldy;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded spin (about a second of SM clocks)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_test_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_test_wait(bar, parity)) return true;
+    if (clock64() - t0 > 2000000000ll) return false;
+  }
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the load of one 64-row x 64-k box; its bytes complete on the pair leader's barrier
+__device__ __forceinline__ void tma_load_pair(void* dst, const CUtensorMap* map, int x, int y, uint64_t* own_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(own_bar) & kPeerBitMask)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;  // 128-byte swizzle
+  return d;
+}
+// kind::f16, fp16 x fp16 -> fp32, both operands K-major, M = 256 over the pair, N = 256
+__device__ __forceinline__ uint32_t umma_idesc_pair() { return (1u << 4) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24); }
+__device__ __forceinline__ void umma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives on the barrier at shared::cluster address `bar_addr` when the pair's MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, "
+      "%18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+        "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+        "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+    gemm_w16_pair_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap, const PairParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t full[kStages], empty[kStages], acc_full;
+  __shared__ uint32_t tmem_base_s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t rank = cluster_rank();     // 0 = leader
+  const int pair = blockIdx.x >> 1;          // feature tile of the pair
+  const int n0 = pair * 256 + (int)rank * kFeatPerCta;             // first weight row this CTA loads
+  const int t0 = blockIdx.y * 512 + (int)rank * kTokPerCta;        // first token of this CTA
+  const int nks = p.ksteps;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&full[s], 1);   // the leader's own arrive.expect_tx; the bytes of both CTAs' loads complete on it
+      mbar_init(&empty[s], 1);  // one commit from the leader's MMA thread
+    }
+    mbar_init(&acc_full, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // one warp of each CTA, same shared-memory offset and column count in both
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  cluster_sync_all();  // both CTAs' barriers are initialised and their tensor memory allocated before anyone signals the other
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_s;
+  if (warp == 0) asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations come from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  bool failed = false;
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < nks; ++i) {
+        const int s = i % kStages;
+        if (i >= kStages && !mbar_wait(&empty[s], ((i / kStages) - 1) & 1)) {
+          failed = true;
+          break;
+        }
+        uint8_t* st = smem + (size_t)s * kStageBytes;
+        if (rank == 0) mbar_expect_tx(&full[s], 2u * kStageBytes);
+        for (int b = 0; b < kTokPerCta / BOXR; ++b) tma_load_pair(st + kWBytes + (size_t)b * BOXR * BK * 2, &xmap, i * BK, t0 + b * BOXR, &full[s]);
+        for (int b = 0; b < kFeatPerCta / BOXR; ++b) tma_load_pair(st + (size_t)b * BOXR * BK * 2, &wmap, i * BK, n0 + b * BOXR, &full[s]);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = umma_idesc_pair();
+      const uint64_t desc0 = umma_desc(smem_u32(smem));
+      uint32_t empty_peer[kStages];
+#pragma unroll
+      for (int s = 0; s < kStages; ++s) empty_peer[s] = map_to_cta(smem_u32(&empty[s]), 1);
+      uint32_t accum = 0, par = 0;
+      int s = 0;
+      bool ok = true;
+      for (int i = 0; i < nks; ++i) {
+        if (!mbar_wait(&full[s], par)) {
+          ok = false;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t wdesc = desc0 + (uint64_t)((uint32_t)s * (uint32_t)(kStageBytes >> 4));  // weight rows: the B operand (N)
+        const uint64_t xdesc = wdesc + (uint64_t)(kWBytes >> 4);                                // activation rows: the A operand (M)
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk) {
+#pragma unroll
+          for (int mb = 0; mb < 2; ++mb)
+            umma_f16_pair(tmem_base + (uint32_t)(mb * 256), xdesc + (uint64_t)(mb * ((BM * BK * 2) >> 4) + 2 * kk), wdesc + (uint64_t)(2 * kk),
+                          idesc, kk > 0 ? 1u : accum);
+        }
+        accum = 1;
+        umma_commit_pair(smem_u32(&empty[s]));  // this CTA's producer may refill the stage ...
+        umma_commit_pair(empty_peer[s]);        // ... and so may the partner's
+        if (++s == kStages) {
+          s = 0;
+          par ^= 1;
+        }
+      }
+      if (ok) {
+        umma_commit_pair(smem_u32(&acc_full));
+        umma_commit_pair(map_to_cta(smem_u32(&acc_full), 1));
+      } else {
+        failed = true;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue: this CTA's 256 tokens x 256 features
+    const int w2 = warp - 2;           // 0..7
+    const int q = warp & 3;            // tensor-memory lane quarter this warp may read
+    const int half = w2 >> 2;          // which half of the 256 feature columns
+    int ready = 0;
+    if (nks > 0) {
+      if (lane == 0) ready = mbar_wait(&acc_full, 0) ? 1 : 0;
+      ready = __shfl_sync(0xffffffffu, ready, 0);
+    }
+    if (ready) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int nbase = pair * 256;
+#pragma unroll 1
+      for (int mb = 0; mb < 2; ++mb) {
+        const int t = t0 + mb * BM + q * 32 + lane;
+#pragma unroll 1
+        for (int c0 = half * 128; c0 < half * 128 + 128; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mb * 256 + c0), v);
+          if (t < p.T) {
+            __half* dst = p.y + (size_t)t * p.ldy + nbase + c0;
+            if (nbase + c0 + 32 <= p.N && (p.ldy % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0)) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 8) {
+                uint32_t o[4];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                  const __half2 hh = __floats2half2_rn(__uint_as_float(v[e + 2 * h]), __uint_as_float(v[e + 2 * h + 1]));
+                  o[h] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+                *reinterpret_cast<uint4*>(dst + e) = make_uint4(o[0], o[1], o[2], o[3]);
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (nbase + c0 + e < p.N) dst[e] = __float2half_rn(__uint_as_float(v[e]));
+            }
+          }
+        }
+      }
+    } else if (nks > 0) {
+      failed = true;
+    }
+  }
+  if (failed && p.status) atomicExch(p.status, 2);
+  // nobody leaves, frees tensor memory or lets its shared memory go while the partner may still read or signal it
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  cluster_sync_all();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+}  // namespace
+
+// Shapes the pair kernel takes: one fp16 matrix, no residual, no grouping, operands aligned for TMA, and enough tiles to
+// occupy three quarters of the SMs (it has no split-K: with fewer tiles the single-CTA kernel, which splits K, is faster;
+// measured cross-over: 112 CTAs even, 128 and more 8 to 17 % faster, 64 and fewer slower).
+bool gemm_pair_eligible(const GemmParams& g) {
+  if (!g.w16 || g.n_seg != 1 || g.grp_off || g.res || g.y2) return false;
+  if (g.T < 384 || g.K % 8 || g.ldx % 8 || g.K < BK) return false;
+  if ((reinterpret_cast<uintptr_t>(g.x) | reinterpret_cast<uintptr_t>(g.seg[0].base)) & 15) return false;
+  const long ctas = 2L * ((g.seg[0].n_rows + 255) / 256) * ((g.T + 511) / 512);
+  return ctas >= 112;
+}
+
+cudaError_t launch_gemm_pair(const GemmParams& g, cudaStream_t st, uint64_t* n_launch, std::string* err) {
+  if (!gemm_pair_eligible(g)) return cudaErrorInvalidValue;
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) {
+    if (err) *err = "cuTensorMapEncodeTiled is not available from the driver";
+    return cudaErrorNotSupported;
+  }
+  const int N = g.seg[0].n_rows;
+  CUtensorMap xmap, wmap;
+  const cuuint32_t box[2] = {BK, BOXR}, estr[2] = {1, 1};
+  const cuuint64_t xdims[2] = {(cuuint64_t)g.K, (cuuint64_t)g.T}, xstr[1] = {(cuuint64_t)g.ldx * 2};
+  const cuuint64_t wdims[2] = {(cuuint64_t)g.K, (cuuint64_t)N}, wstr[1] = {(cuuint64_t)g.K * 2};
+  if (enc(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half*>(g.x), xdims, xstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+      enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<uint8_t*>(g.seg[0].base), wdims, wstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+    if (err) *err = "cuTensorMapEncodeTiled failed";
+    return cudaErrorInvalidValue;
+  }
+  PairParams p{};
+  p.K = g.K;
+  p.T = g.T;
+  p.N = N;
+  p.ksteps = (g.K + BK - 1) / BK;
+  p.y = g.y;
+  p.ldy = g.ldy;
+  p.status = g.status;
+  const size_t smem = (size_t)kStages * kStageBytes + 1024;
+  static uint64_t attr_done = 0;
+  if (first_use_on_device(&attr_done)) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_w16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  const dim3 grid(2 * ((N + 255) / 256), (g.T + 511) / 512);
+  ++*n_launch;
+  return launch_dep(gemm_w16_pair_kernel, grid, dim3(kThreads), smem, st, g.pdl, 2, xmap, wmap, p);
+}
+
+}  // namespace ats

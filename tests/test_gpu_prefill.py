@@ -429,3 +429,28 @@ def test_dense_layer_fp16_weights_prefill_matches_oracle(B, torch, pos0, T, cap)
         assert np.max(np.abs(a - b)) <= 4e-3 * np.max(np.abs(b))
         ctx.close()
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+
+
+@pytest.mark.parametrize("N,K,T", [(14336, 256, 512), (14400, 200, 700), (7200, 4096, 1100)])
+def test_linear_w16_gemm_as_cta_pair_matches_oracle(B, torch, N, K, T):
+    """fp16-weight GEMMs with enough tiles run as pairs of CTAs on two SMs (tcgen05 cta_group::2: 512 tokens x 256 features
+    per pair, each CTA loading half of the weight rows).  Against the oracle, incl. ragged N, K and T (rows past the
+    matrix and k past K read as zeros, stores guarded), and against the single-CTA kernel selected by flag."""
+    rng = np.random.default_rng(N + K + T)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float16)
+    x = W.activations(96, 2, (T, K))
+    want = O.linear_w16(x, w, round_out=True)
+    outs = []
+    for flags in (0, B.ATS_FLAG_NO_GEMM_PAIR):
+        ws = 9 * T * N * 4 + 2 * MB
+        ctx = B.Context(ws + N * K * 2 + 4 * MB, workspace_bytes=ws, flags=flags)
+        tid = ctx.register_w16(w)
+        ctx.set_placement([(tid, -1, B.ATS_GPU)])
+        y = torch.full((T, N), 7.0, dtype=torch.float16, device="cuda")
+        ctx.linear(tid, H.to_dev(x), y, T)
+        ctx.sync()
+        outs.append(y.cpu().numpy())
+        H.assert_close(outs[-1], want, what=f"w16 gemm {N}x{K} T={T} flags={flags}")
+        ctx.close()
+    # same products, fp32 accumulation in both; the single-CTA kernel may split K, so not necessarily the same bits
+    H.assert_close(outs[0], outs[1].astype(np.float64), what="pair against single-CTA kernel")
