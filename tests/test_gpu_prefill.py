@@ -454,3 +454,30 @@ def test_linear_w16_gemm_as_cta_pair_matches_oracle(B, torch, N, K, T):
         ctx.close()
     # same products, fp32 accumulation in both; the single-CTA kernel may split K, so not necessarily the same bits
     H.assert_close(outs[0], outs[1].astype(np.float64), what="pair against single-CTA kernel")
+
+
+@pytest.mark.parametrize("fmt", ["q4", "mxfp4"])
+def test_linear_gemm_4bit_as_cta_pair_matches_oracle(B, torch, fmt):
+    """The dequantizing GEMM as a pair of CTAs (long reductions with at least 128 CTAs of tiles): every CTA dequantizes half
+    of the pair's 256 weight rows into its own shared memory, the leader issues the M = 256 instructions.  Sampled tokens
+    against the oracle (all features), the whole output against the single-CTA kernel selected by flag; ragged N and T."""
+    N, K, T = 4000, 8192, 2000
+    packed, scales = (W.q4_packed if fmt == "q4" else W.mxfp4_packed)(90, 0, W.ROLE_DOWN, N, K)
+    x = W.activations(90, 0, (T, K))
+    outs = []
+    for flags in (0, B.ATS_FLAG_NO_GEMM_PAIR):
+        ws = 9 * T * N * 4 + 2 * MB
+        ctx = B.Context(ws + W.q4_bytes(N, K) + 4 * MB, workspace_bytes=ws, flags=flags)
+        tid = ctx.register_q4(packed, scales)
+        ctx.set_placement([(tid, -1, B.ATS_GPU)])
+        edges, wmode = ctx.numerics(B.ATS_MODE_PREFILL)
+        y = torch.full((T, N), 7.0, dtype=torch.float16, device="cuda")
+        ctx.linear(tid, H.to_dev(x), y, T)
+        ctx.sync()
+        outs.append(y.cpu().numpy())
+        ctx.close()
+    rows = np.array([0, 1, 127, 128, 255, 256, 511, 512, 777, 1023, 1024, 1535, 1536, 1999])
+    want = O.linear(x[rows], packed, scales, wmode, round_out=True)
+    H.assert_close(outs[0][rows], want, what=f"{fmt} pair gemm, sampled tokens")
+    H.assert_close(outs[1][rows], want, what=f"{fmt} single-CTA gemm, sampled tokens")
+    H.assert_close(outs[0], outs[1].astype(np.float64), what="pair against single-CTA kernel")
