@@ -323,7 +323,10 @@ struct GemmParams {
 };
 uint64_t gemm_scratch_bytes(int T, int n_total, int K);
 cudaError_t launch_gemm(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);
-// fp16-weight GEMM as a pair of CTAs (kernels_gemm_pair.cu): shapes it takes, and its launcher
+// y = rn16(sum over splits of partial[s][T][ldy]) (+ optional residual into y2), splits in ascending order (kernels_gemm.cu)
+cudaError_t launch_gemm_splitk_reduce(const float* partial, __half* y, int T, int n_cols, int ldy, int splits, const __half* res, __half* y2,
+                                      int pdl, cudaStream_t st, uint64_t* n_launch);
+// GEMMs as pairs of CTAs (kernels_gemm_pair.cu): shapes they take, and their launcher
 bool gemm_pair_eligible(const GemmParams& p);
 cudaError_t launch_gemm_pair(const GemmParams& p, cudaStream_t st, uint64_t* n_launch, std::string* err);
 // fixed split-K scratch inside the library's device image (no allocation): capacity, and its address on the current device

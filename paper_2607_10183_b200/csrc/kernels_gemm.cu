@@ -761,6 +761,17 @@ cudaError_t launch_gemm(const GemmParams& g, cudaStream_t st, uint64_t* n_launch
   return e;
 }
 
+// The split-K sum as a launch of its own, for the other GEMM kernels of the library.
+cudaError_t launch_gemm_splitk_reduce(const float* partial, __half* y, int T, int n_cols, int ldy, int splits, const __half* res, __half* y2,
+                                      int pdl, cudaStream_t st, uint64_t* n_launch) {
+  int sm_count = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+  const size_t total = (size_t)T * n_cols;
+  const int blocks = (int)std::min<size_t>((total / 8 + 255) / 256 + 1, (size_t)sm_count * 8);
+  ++*n_launch;
+  return launch_dep(gemm_splitk_reduce_kernel, dim3(blocks), dim3(256), 0, st, pdl, 1, partial, y, T, n_cols, ldy, splits, res, y2);
+}
+
 // ---------------------------------------------------------------------------------------------------------------
 // Split-K scratch that needs no allocation: a fixed array in the library's own device image.
 // Every GPU that loads the library carries these 8 MiB from load until exit.

@@ -269,7 +269,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 // mbarrier.arrive.release.cluster instead, every arrival took about as long as a k-step and the kernel ran at 0.65 of the
 // single-CTA kernel's rate.  Per pair and k-step each CTA dequantizes half of what a single CTA would for the same
 // 512 x 256 outputs.  Measured against the single-CTA kernel: 6 to 12 % faster for long reductions (K >= 8192) from 128
-// CTAs on, within +-4 % otherwise, which is where the launcher uses it.
+// CTAs on (with few tiles: K split over blockIdx.z into fp32 partials that a second launch sums, 5 to 9 % faster from 1024
+// tokens on), within +-4 % otherwise, which is where the launcher uses it.
 struct PairSeg {
   const uint8_t* base;
   int n_rows;
@@ -286,6 +287,8 @@ struct PairQParams {
   const __half* res;  // optional residual: y2 = rn16(res + y)
   __half* y2;
   int* status;
+  int splits, ksteps_per_split;  // split-K over blockIdx.z: fp32 partials [splits][T][ldy], summed by a second launch
+  float* partial;
 };
 constexpr int kQStageBytes = kXBytes + kWBytes;  // weight half-tile first, then the activations (same layout as above)
 
@@ -344,7 +347,8 @@ __global__ void __launch_bounds__(kQThreads, 1) gemm_q4_pair_kernel(const __grid
   const int row0 = prow0 + (int)rank * kFeatPerCta;        // first weight row this CTA dequantizes
   const int n_rows = p.seg[sg].n_rows;
   const int t0 = blockIdx.y * 512 + (int)rank * kTokPerCta;
-  const int nks = p.ksteps;
+  const int ks0 = (int)blockIdx.z * p.ksteps_per_split;
+  const int nks = min(p.ksteps_per_split, p.ksteps - ks0);
   constexpr int kDqWarps = 16;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -376,7 +380,8 @@ __global__ void __launch_bounds__(kQThreads, 1) gemm_q4_pair_kernel(const __grid
         }
         uint8_t* st = smem + (size_t)s * kQStageBytes;
         if (rank == 0) mbar_expect_tx(&full[s], 2u * kXBytes);
-        for (int b = 0; b < kTokPerCta / BOXR; ++b) tma_load_pair(st + kWBytes + (size_t)b * BOXR * BK * 2, &xmap, i * BK, t0 + b * BOXR, &full[s]);
+        for (int b = 0; b < kTokPerCta / BOXR; ++b)
+          tma_load_pair(st + kWBytes + (size_t)b * BOXR * BK * 2, &xmap, (ks0 + i) * BK, t0 + b * BOXR, &full[s]);
       }
     }
   } else if (warp == 1) {
@@ -438,7 +443,7 @@ __global__ void __launch_bounds__(kQThreads, 1) gemm_q4_pair_kernel(const __grid
     uint2 qbuf[kPD];
     uint32_t sbuf[kPD];
     auto fetch = [&](int ks, uint2& q, uint32_t& sc) {
-      const int kb = ks * 2 + (qd >> 1);
+      const int kb = (ks0 + ks) * 2 + (qd >> 1);
       q = make_uint2(0, 0);
       sc = 0;
       if (valid && kb < nblk) {
@@ -512,6 +517,18 @@ __global__ void __launch_bounds__(kQThreads, 1) gemm_q4_pair_kernel(const __grid
           if (t >= p.T) continue;
           const int nf = min(32, n_rows - prow0 - c0);  // features of this chunk that exist
           if (nf <= 0) continue;
+          if (p.splits > 1) {  // fp32 partial of this K range; the sum over the splits runs as a second launch
+            float* pd = p.partial + ((size_t)blockIdx.z * p.T + t) * p.ldy + colbase + c0;
+            if (nf == 32 && (p.ldy % 4 == 0) && (colbase % 4 == 0)) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 4) *reinterpret_cast<uint4*>(pd + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (e < nf) pd[e] = __uint_as_float(v[e]);
+            }
+            continue;
+          }
           __half* dst = p.y + (size_t)t * p.ldy + colbase + c0;
           const __half* rs = p.res ? p.res + (size_t)t * p.ldy + colbase + c0 : nullptr;
           __half* d2 = p.y2 ? p.y2 + (size_t)t * p.ldy + colbase + c0 : nullptr;
@@ -583,6 +600,18 @@ static long pair_ctas(const GemmParams& g) {
   for (int i = 0; i < g.n_seg; ++i) pairs += (g.seg[i].n_rows + 255) / 256;
   return 2L * pairs * ((g.T + 511) / 512);
 }
+// Split-K factor of the dequantizing pair kernel: enough K ranges to bring the grid to about one CTA per SM, each at
+// least 16 k-steps long, as far as the scratch holds the fp32 partials.
+static int pair_splits(const GemmParams& g) {
+  const long ctas = pair_ctas(g);
+  if (g.w16 || ctas >= 112) return 1;
+  const int ksteps = (g.K + BK - 1) / BK;
+  int n_cols = 0;
+  for (int i = 0; i < g.n_seg; ++i) n_cols += g.seg[i].n_rows;
+  int s = 1;
+  while (s < 8 && ctas * s < 128 && ksteps / (s * 2) >= 16 && (uint64_t)(s * 2) * g.T * g.ldy * 4 <= (g.scratch ? g.scratch_bytes : 0)) s *= 2;
+  return s;
+}
 bool gemm_pair_eligible(const GemmParams& g) {
   if (g.grp_off || g.n_seg < 1 || g.n_seg > 3) return false;
   if (g.T < 384 || g.ldx % 8 || g.K < BK || (reinterpret_cast<uintptr_t>(g.x) & 15)) return false;
@@ -595,7 +624,9 @@ bool gemm_pair_eligible(const GemmParams& g) {
   for (int i = 0; i < g.n_seg; ++i)
     if (reinterpret_cast<uintptr_t>(g.seg[i].base) & 15) return false;
   if ((g.res != nullptr) != (g.y2 != nullptr)) return false;
-  return pair_ctas(g) >= 128;
+  const int splits = pair_splits(g);
+  if (splits > 1 && g.T < 1024) return false;  // split over K the pair gains 5-9 % from 1024 tokens on, nothing at 512
+  return pair_ctas(g) * splits >= 128;
 }
 
 cudaError_t launch_gemm_pair(const GemmParams& g, cudaStream_t st, uint64_t* n_launch, std::string* err) {
@@ -660,9 +691,18 @@ cudaError_t launch_gemm_pair(const GemmParams& g, cudaStream_t st, uint64_t* n_l
   p.res = g.res;
   p.y2 = g.y2;
   p.status = g.status;
-  const dim3 grid(2 * tiles, tchunks);
-  return g.mx ? launch_dep(gemm_q4_pair_kernel<true>, grid, dim3(kQThreads), smem, st, g.pdl, 2, xmap, p)
-              : launch_dep(gemm_q4_pair_kernel<false>, grid, dim3(kQThreads), smem, st, g.pdl, 2, xmap, p);
+  p.splits = pair_splits(g);
+  p.ksteps_per_split = (p.ksteps + p.splits - 1) / p.splits;
+  while (p.splits > 1 && (p.splits - 1) * p.ksteps_per_split >= p.ksteps) {  // no empty K range
+    --p.splits;
+    p.ksteps_per_split = (p.ksteps + p.splits - 1) / p.splits;
+  }
+  p.partial = (float*)g.scratch;
+  const dim3 grid(2 * tiles, tchunks, p.splits);
+  cudaError_t e = g.mx ? launch_dep(gemm_q4_pair_kernel<true>, grid, dim3(kQThreads), smem, st, g.pdl, 2, xmap, p)
+                       : launch_dep(gemm_q4_pair_kernel<false>, grid, dim3(kQThreads), smem, st, g.pdl, 2, xmap, p);
+  if (e != cudaSuccess || p.splits == 1) return e;
+  return launch_gemm_splitk_reduce(p.partial, g.y, g.T, col, g.ldy, p.splits, g.res, g.y2, g.pdl, st, n_launch);
 }
 
 }  // namespace ats

@@ -456,12 +456,12 @@ def test_linear_w16_gemm_as_cta_pair_matches_oracle(B, torch, N, K, T):
     H.assert_close(outs[0], outs[1].astype(np.float64), what="pair against single-CTA kernel")
 
 
-@pytest.mark.parametrize("fmt", ["q4", "mxfp4"])
-def test_linear_gemm_4bit_as_cta_pair_matches_oracle(B, torch, fmt):
-    """The dequantizing GEMM as a pair of CTAs (long reductions with at least 128 CTAs of tiles): every CTA dequantizes half
-    of the pair's 256 weight rows into its own shared memory, the leader issues the M = 256 instructions.  Sampled tokens
-    against the oracle (all features), the whole output against the single-CTA kernel selected by flag; ragged N and T."""
-    N, K, T = 4000, 8192, 2000
+@pytest.mark.parametrize("fmt,N,K,T", [("q4", 4000, 8192, 2000), ("mxfp4", 4000, 8192, 2000), ("q4", 4096, 14336, 1024), ("mxfp4", 3900, 14336, 1000)])
+def test_linear_gemm_4bit_as_cta_pair_matches_oracle(B, torch, fmt, N, K, T):
+    """The dequantizing GEMM as a pair of CTAs (long reductions): every CTA dequantizes half of the pair's 256 weight rows
+    into its own shared memory, the leader issues the M = 256 instructions; with few tiles K is split over blockIdx.z
+    and a second launch sums the fp32 partials (the 1024-token cases).  Sampled tokens against the oracle (all features), the
+    whole output against the single-CTA kernel selected by flag; ragged N and T."""
     packed, scales = (W.q4_packed if fmt == "q4" else W.mxfp4_packed)(90, 0, W.ROLE_DOWN, N, K)
     x = W.activations(90, 0, (T, K))
     outs = []
@@ -476,7 +476,7 @@ def test_linear_gemm_4bit_as_cta_pair_matches_oracle(B, torch, fmt):
         ctx.sync()
         outs.append(y.cpu().numpy())
         ctx.close()
-    rows = np.array([0, 1, 127, 128, 255, 256, 511, 512, 777, 1023, 1024, 1535, 1536, 1999])
+    rows = np.array([r for r in (0, 1, 127, 128, 255, 256, 499, 511, 512, 777, 1023, 1024, 1535, 1536, 1999) if r < T])
     want = O.linear(x[rows], packed, scales, wmode, round_out=True)
     H.assert_close(outs[0][rows], want, what=f"{fmt} pair gemm, sampled tokens")
     H.assert_close(outs[1][rows], want, what=f"{fmt} single-CTA gemm, sampled tokens")
