@@ -122,18 +122,93 @@ def oracle_layer_decode_step(cfg=2):
     return step
 
 
-def time_oracle(budget_s=15.0, max_reps=5):
-    step = oracle_layer_decode_step()
+def _timed(fn, budget_s, max_reps):
     t0 = time.time()
-    step()
+    fn()
     t1 = time.time() - t0
     reps = int(min(max_reps, max(1, round(budget_s / max(t1, 1e-3)))))
+    if reps == 1:
+        return t1, 1
     t0 = time.time()
     for _ in range(reps):
-        step()
-    dt = (time.time() - t0) / reps
+        fn()
+    return (time.time() - t0) / reps, reps
+
+
+def time_oracle(budget_s=15.0, max_reps=5):
+    dt, reps = _timed(oracle_layer_decode_step(), budget_s, max_reps)
     return {"value": 1.0 / dt, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
             "sample": f"{reps} decode steps of one dense layer (fp64 numpy oracle, {dt:.2f} s per step)"}
+
+
+def cpu_baseline_cfg1():
+    """Config 1 on the host cores: the oracle's GEMV of the 4096 x 4096 tensor, median of 3."""
+    from oracle import ats_oracle as O
+    from paper_2607_10183_b200 import workloads as W
+    packed, scales = W.q4_packed(1, 0, W.ROLE_Q, 4096, 4096)
+    x = W.activations(1, 0, (1, 4096))
+    ts = []
+    for _ in range(3):
+        t0 = time.time()
+        O.linear(x, packed, scales)
+        ts.append(time.time() - t0)
+    dt = statistics.median(ts)
+    alg = W.q4_bytes(4096, 4096) + 2 * 4096 * 2
+    return {"value": alg / dt / 1e9, "unit": "GB/s (algorithmic bytes)", "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"3 GEMVs 4096x4096 (dequantize + fp64 product), median {dt * 1e3:.0f} ms"}
+
+
+def cpu_baseline_cfg3():
+    """Config 3 on the host cores: the oracle's 512-token prefill of one dense layer, once."""
+    from oracle import ats_oracle as O
+    from paper_2607_10183_b200 import workloads as W
+    from tests import helpers as H
+    shape = W.DENSE_FULL
+    L = W.dense_layer(3, 0, shape)
+    x = W.activations(3, 0, (512, shape.hidden))
+    kc, vc = W.kv_cache(3, 0, shape.n_kv_heads, 512, shape.head_dim, 0)
+    t0 = time.time()
+    O.dense_layer(x, H.oracle_dense_tensors(L), shape, kc, vc, 0, frozenset(O.EDGES), O.WEIGHT_F16)
+    dt = time.time() - t0
+    return {"value": 512 / dt, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"one 512-token prefill of one dense layer, once ({dt:.1f} s)"}
+
+
+def cpu_baseline_cfg4():
+    """Config 4 on the host cores: the oracle's MoE block, batch 1 and 8."""
+    from oracle import ats_oracle as O
+    from paper_2607_10183_b200 import workloads as W
+    from tests import helpers as H
+    shape = W.MOE_FULL
+    t = H.oracle_moe_tensors(W.moe_block(4, 0, shape))
+    out = {"cores": oracle_threads(), "kind": "oracle", "unit": "tokens/s"}
+    for M in (1, 8):
+        x = W.activations(4, 0, (M, shape.hidden), step=0)
+        dt, reps = _timed(lambda: O.moe_block(x, t, shape), 4.0, 3)
+        out[f"M{M}"] = {"value": M / dt, "sample": f"{reps} MoE block calls of {M} token(s), {dt * 1e3:.0f} ms per call"}
+    return out
+
+
+def cpu_baseline_cfg5(n_layers=4):
+    """Config 5 on the host cores: one decode step at position 512 through `n_layers` of the 32 layers (a bounded sample;
+    the whole step is 32 layers), scaled to the full stack."""
+    from oracle import ats_oracle as O
+    from paper_2607_10183_b200 import workloads as W
+    from tests import helpers as H
+    shape = W.DENSE_FULL
+    edges = frozenset({"h", "a", "h2", "act"})
+    # the clock runs around the oracle calls only, not around the generation of their inputs
+    per_layer = []
+    x = W.activations(5, 0, (1, shape.hidden))
+    for l in range(n_layers):
+        L = W.dense_layer(5, l, shape)
+        kc, vc = W.kv_cache(5, l, shape.n_kv_heads, 513, shape.head_dim, 512)
+        t1 = time.time()
+        x = O.dense_layer(x, H.oracle_dense_tensors(L), shape, kc, vc, 512, edges, O.WEIGHT_EXACT)
+        per_layer.append(time.time() - t1)
+    dt = sum(per_layer) / n_layers * 32
+    return {"value": 1.0 / dt, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"{n_layers} of the 32 layers of one decode step at position 512 ({sum(per_layer):.1f} s), scaled to 32 layers"}
 
 
 def run_reference(args):
@@ -160,14 +235,15 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------------------------- our arm
-def build_dense_replicas(B, W, n_layers, cfg, kv_cap, ring_slots=0, slot_bytes=0, chunk_bytes=0, extra_ws=0, flags=0):
-    """A context holding n_layers distinct dense layers of the config-2 shape."""
+def build_dense_replicas(B, W, n_layers, cfg, kv_cap, ring_slots=0, slot_bytes=0, chunk_bytes=0, extra_ws=0, flags=0, resident_frac=1.0):
+    """A context holding n_layers distinct dense layers of the config-2 shape (resident_frac: the share of the weights the
+    arena leaves room for)."""
     shape = W.DENSE_FULL
     layer_bytes = sum(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
     probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
                          head_dim=shape.head_dim, kv_capacity=kv_cap)
     ws = max(B.workspace_bytes(probe, 1), extra_ws) + (1 << 20)
-    arena = ws + ring_slots * (slot_bytes + 256) + n_layers * (layer_bytes + 16 * 1024 + 4 * shape.hidden) + (1 << 20)
+    arena = ws + ring_slots * (slot_bytes + 256) + int(resident_frac * n_layers * layer_bytes) + n_layers * (16 * 1024 + 4 * shape.hidden) + (1 << 20)
     ctx = B.Context(arena, workspace_bytes=ws, ring_slots=ring_slots, slot_bytes=slot_bytes, chunk_bytes=chunk_bytes, flags=flags)
     names = {W.ROLE_Q: "wq", W.ROLE_K: "wk", W.ROLE_V: "wv", W.ROLE_O: "wo", W.ROLE_GATE: "w_gate", W.ROLE_UP: "w_up", W.ROLE_DOWN: "w_down"}
     descs, q4_ids = [], []
@@ -431,45 +507,111 @@ def extra_moe(torch, B, W, peaks, quick):
 
 
 def extra_stream(torch, B, W, peaks, quick, n_layers=None):
-    """Config 5: a stack of dense layers under a 60 % byte budget chosen by the library's placement DP (Algorithm 1);
-    the rest sits in pinned host memory and is streamed every decode step, overlapped with compute."""
+    """Config 5: the 32-layer dense stack (3.93 GB) under a 60 % byte budget chosen by the library's placement DP
+    (Algorithm 1); the other tensors sit in pinned host memory and are streamed through the ring on the transfer stream,
+    overlapped with compute: a 512-token prefill, then 128 decode steps at positions 512..639 (each step feeds a fresh
+    seeded row to layer 0).  Reported: decode ms per step and PCIe GB/s over steps 8..127, the hybrid prefill's PCIe
+    GB/s (one pass over the streamed bytes), and the round latency the paper's model T = sum t_i + sum max(w_i - seg, 0)
+    (Section 4.4.1, every host tensor promoted) predicts from measured t_i and w_i, beside the measured step."""
     shape = W.DENSE_FULL
-    L = n_layers or STACK_LAYERS[0] or (4 if quick else 8)
-    cap, pos0 = 640, 512
+    L = n_layers or STACK_LAYERS[0] or (4 if quick else 32)
+    cap, T, n_steps = 640, 512, (16 if quick else 128)
     slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
-    ctx, descs, q4_ids, layer_bytes = build_dense_replicas(B, W, L, 5, cap, ring_slots=8, slot_bytes=slot, chunk_bytes=8 << 20)
+    probe = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, kv_capacity=cap)
+    chunk = 8 << 20
+    ctx, descs, q4_ids, layer_bytes = build_dense_replicas(B, W, L, 5, cap, ring_slots=8, slot_bytes=slot, chunk_bytes=chunk,
+                                                           extra_ws=B.workspace_bytes(probe, T), resident_frac=0.62)
     total = L * layer_bytes
-    where = ctx.plan_placement(int(0.60 * total), len(q4_ids))
+    budget = (60 * total) // 100
+    where = ctx.plan_placement(budget, len(q4_ids))
     pcie = ctx.measure_h2d(8 * slot, 5)
     st0 = ctx.stats()
     caches = [(torch.zeros((shape.n_kv_heads, cap, shape.head_dim), dtype=torch.float16, device="cuda"),
                torch.zeros((shape.n_kv_heads, cap, shape.head_dim), dtype=torch.float16, device="cuda")) for _ in range(L)]
-    xa = torch.from_numpy(W.activations(5, 0, (1, shape.hidden))).cuda()
-    xb = torch.empty_like(xa)
+    # ---- hybrid prefill: one pass over the host-placed tensors
+    xp = torch.from_numpy(W.activations(5, 0, (T, shape.hidden), step=10_000)).cuda()
+    yp = torch.empty_like(xp)
 
-    def step(pos):
-        src, dst = xa, xb
+    def prefill():
+        a, b = xp, yp
         for l in range(L):
-            ctx.layer_decode(descs[l], src, dst, caches[l][0], caches[l][1], pos, 1)
-            src, dst = dst, src
-    for s in range(3):
-        step(pos0 + s)
+            ctx.layer_prefill(descs[l], a, b, caches[l][0], caches[l][1], 0, T)
+            a, b = b, a
+    prefill()
     ctx.sync()
     ctx.reset_stats()
-    n = 8 if quick else 24
     t0 = time.perf_counter()
-    for s in range(n):
-        step(pos0 + 3 + s)
+    prefill()
     ctx.sync()
-    dt = (time.perf_counter() - t0) / n
+    pre_s = time.perf_counter() - t0
+    pre_streamed = ctx.stats().streamed_bytes
+    # ---- decode steps
+    xs = [torch.from_numpy(W.activations(5, 0, (1, shape.hidden), step=s)).cuda() for s in range(n_steps)]
+    xa, xb = torch.empty_like(xs[0]), torch.empty_like(xs[0])
+
+    def step(s):
+        src, dst = xs[s], xa
+        for l in range(L):
+            ctx.layer_decode(descs[l], src, dst, caches[l][0], caches[l][1], T + s, 1)
+            src, dst = dst, (xb if dst is xa else xa)
+        return src
+    warm = min(8, n_steps // 2)
+    for s in range(warm):
+        step(s)
+    ctx.sync()
+    ctx.reset_stats()
+    t0 = time.perf_counter()
+    for s in range(warm, n_steps):
+        last = step(s)
+    ctx.sync()
+    dt = (time.perf_counter() - t0) / (n_steps - warm)
     st = ctx.stats()
-    streamed = st.streamed_bytes / n
+    streamed = st.streamed_bytes / (n_steps - warm)
+    finite = bool(torch.isfinite(last.float()).all().item())
     ctx.close()
-    return {"workload": f"config 5 shape: {L}-layer dense stack, 60 % byte budget via ats_plan_placement, decode steps at positions {pos0 + 3}+",
-            "layers": L, "total_weight_bytes": total, "resident_bytes": int(st0.resident_bytes), "resident_frac": st0.resident_bytes / total,
-            "gpu_tensors": int(where.sum()), "host_tensors": int(len(where) - where.sum()), "streamed_bytes_per_step": streamed,
-            "ms_per_step": dt * 1e3, "decode_tokens_per_s": 1.0 / dt, "pcie_gbs_streamed": streamed / dt / 1e9, "pcie_h2d_measured_gbs": pcie,
-            "frac_of_measured_pcie": streamed / dt / 1e9 / pcie, "fully_overlapped_at_80pct": bool(dt <= streamed / (0.8 * pcie * 1e9))}
+    del caches
+    torch.cuda.empty_cache()
+    # ---- the paper's overlap model with measured operator and transfer times (one layer's seven tensors, profiled alone)
+    modelled_ms, model_note = None, None
+    try:
+        sizes = {r: W.q4_bytes(n, k) for r, n, k in shape.tensor_shapes()}
+        pctx = B.Context(sum(sizes.values()) + 2 * (slot + 256) + (8 << 20), workspace_bytes=1 << 20, ring_slots=2, slot_bytes=slot, chunk_bytes=chunk)
+        Lw = W.dense_layer(5, 0, shape)
+        t_res, t_host = {}, {}
+        for r, n, k in shape.tensor_shapes():
+            tid = pctx.register_q4(*Lw[r], layer=0, role=r)
+            x1 = torch.from_numpy(W.activations(5, 0, (1, k), role=r)).cuda()
+            y1 = torch.empty((1, n), dtype=torch.float16, device="cuda")
+            t_res[r], t_host[r] = pctx.profile_tensor(tid, x1, y1, 1, iters=10 if quick else 30)
+        pctx.close()
+        roles = [r for r, _, _ in shape.tensor_shapes()] * L
+        b = np.asarray(where, dtype=np.uint8)
+        t_gpu = np.array([t_res[r] for r in roles])
+        w_us = np.array([t_host[r] for r in roles])  # steady-state time of the streamed operator = its transfer time
+        rb = np.ones(len(roles), dtype=np.uint8)
+        start, prev_host = np.full(len(roles), B.ATS_NO_TRANSFER, dtype=np.int32), B.ATS_ROUND_START
+        for i in range(len(roles)):
+            if b[i] == B.ATS_HOST:
+                start[i] = prev_host  # the transfer starts when the previous host-placed tensor has run
+                prev_host = i
+        modelled_ms = B.host_transfer_latency(rb, start, b, t_gpu, t_gpu, np.zeros(len(roles)), w_us) / 1e3
+        model_note = ("T = sum t_i + sum max(w_i - seg(j_i, i), 0) with every host-placed tensor promoted, j_i = the previous host-placed "
+                      "tensor, t_i = measured resident operator time, w_i = measured time of the operator when streamed (PCIe-bound), "
+                      "attention and norms not in the model; the runtime keeps up to 8 transfers queued ahead, the model only the next one")
+    except Exception as e:  # the model figure must not take the measurement down
+        model_note = f"{type(e).__name__}: {e}"
+    return {"workload": f"config 5: {L}-layer dense stack, 60 % byte budget via ats_plan_placement; {T}-token hybrid prefill, then "
+                        f"{n_steps} decode steps at positions {T}..{T + n_steps - 1} (timed: steps {warm}..{n_steps - 1})",
+            "layers": L, "total_weight_bytes": total, "budget_bytes": budget, "resident_bytes": int(st0.resident_bytes),
+            "resident_frac": st0.resident_bytes / total, "gpu_tensors": int(where.sum()), "host_tensors": int(len(where) - where.sum()),
+            "streamed_bytes_per_step": streamed, "ms_per_step": dt * 1e3, "decode_tokens_per_s": 1.0 / dt,
+            "pcie_gbs_streamed": streamed / dt / 1e9, "pcie_h2d_measured_gbs": pcie, "frac_of_measured_pcie": streamed / dt / 1e9 / pcie,
+            "fully_overlapped_at_80pct": bool(dt <= streamed / (0.8 * pcie * 1e9)),
+            "prefill": {"tokens": T, "ms": pre_s * 1e3, "tokens_per_s": T / pre_s, "streamed_bytes": float(pre_streamed),
+                        "pcie_gbs": pre_streamed / pre_s / 1e9, "frac_of_measured_pcie": pre_streamed / pre_s / 1e9 / pcie},
+            "modelled_ms": modelled_ms, "modelled_note": model_note, "outputs_finite": finite,
+            "timing": "wall clock around queued calls followed by ats_sync (the host never blocks inside a step)"}
 
 
 def extra_model_loop(torch, B, W, peaks, quick):
@@ -545,7 +687,8 @@ def extra_model_loop(torch, B, W, peaks, quick):
             "layers": L, "weight_bytes": weight_bytes, "prefill_ms": pre_ms, "prefill_tokens_per_s": prompt / (pre_ms * 1e-3),
             "decode_ms_per_token": dec_ms / gen, "decode_tokens_per_s": gen / (dec_ms * 1e-3),
             "decode_weight_gbs": weight_bytes / (dec_ms / gen * 1e-3) / 1e9,
-            "decode_frac_of_measured_hbm": weight_bytes / (dec_ms / gen * 1e-3) / 1e9 / peaks["hbm_gbs"], "logits_finite": finite}
+            "decode_frac_of_measured_hbm": weight_bytes / (dec_ms / gen * 1e-3) / 1e9 / peaks["hbm_gbs"], "logits_finite": finite,
+            "gains_damped": 0.1, "note": "timing only: the norm gains are scaled by 0.1 so that 32 random layers stay inside fp16"}
 
 
 def extra_w16(torch, B, W, peaks, quick):
@@ -804,6 +947,7 @@ def extra_model_loop_moe(torch, B, W, peaks, quick):
         dec_ms = event_time_ms(torch, ctx.compute, lambda: decode(gen))
         finite = bool(torch.isfinite(last.float()).all().item()) and bool(torch.isfinite(da.float()).all().item())
         key = "hybrid_odd_experts_on_host" if hybrid else "resident"
+        out["gains_damped"] = 0.1  # timing only: norm gains scaled by 0.1 so that the random stack stays inside fp16
         out[key] = {"prefill_ms": pre_s * 1e3, "prefill_tokens_per_s": prompt / pre_s, "prefill_host_bytes_moved": float(st.streamed_bytes),
                     "prefill_pcie_gbs_over_wall_time": st.streamed_bytes / pre_s / 1e9,
                     "decode_ms_per_token": dec_ms / gen, "decode_tokens_per_s": gen / (dec_ms * 1e-3), "outputs_finite": finite,
@@ -874,12 +1018,12 @@ def run_ours(args):
     # (programmatic dependent launch included) and nothing but them is inside the events.  Bracketing every launch
     # with its own event pair instead (ATS_FLAG_TIME_KERNELS) serialises the launches and adds ~3 us to each; that
     # figure is reported as `achieved_event_bracketed`.
-    skip_attn = 2 << 24
-    ctx.set_flags(skip_attn)
+    ctx.debug_skip_stages(2)  # the attention launch
     steps(args.warmup)
     barrier()
-    n_prof = min(args.steps, 5000)
+    n_prof = min(max(args.steps, 2000), 5000)  # at least 8000 launches, however few steps the headline was asked for
     gemv_only_ms = event_time_ms(torch, cs, lambda: steps(n_prof, args.warmup))
+    ctx.debug_skip_stages(0)
     ctx.set_flags(B.ATS_FLAG_TIME_KERNELS)
     ctx.reset_stats()
     steps(min(n_prof, 2000), args.warmup)
@@ -891,9 +1035,25 @@ def run_ours(args):
     avg_launch_us = gemv_only_ms * 1e3 / (4 * n_prof)
     achieved = bytes_per_launch / (avg_launch_us * 1e-6) / 1e9
     bracketed = gemv_bytes / (st.timed_ms[0] * 1e-3) / 1e9 if st.timed_ms[0] > 0 else None
+    step_bytes = layer_bytes + 2 * shape.n_kv_heads * cap * shape.head_dim * 2 + 4 * shape.hidden * 2
+    step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
+    try:
+        hbm_read = ctx.measure_hbm_read(min(R * layer_bytes, 1 << 30), 5)
+    except Exception:
+        hbm_read = None
     roofline = {"bound": "hbm", "kernel": "gemv_stream_kernel (4 launches per step: fused QKV, O, fused gate/up+SwiGLU, down)",
+                # the whole step first: all algorithmic bytes of the step (weights, KV cache, activations) over the step time
+                "step_achieved": step_gbs, "step_frac": step_gbs / peaks["hbm_gbs"],
+                # the dominant kernel family, timed live in a region that runs the same steps without the attention launch
+                # (the four GEMV launches back to back with their dependent-launch overlap, as in the step)
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"] + " HBM copy bandwidth",
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBs": achieved / 8000.0,
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "frac_is": "GEMV family: bytes per launch / average launch time in a timed region of the same steps with the attention "
+                           "launch left out (launches overlap as in the step); step_frac is the whole step, "
+                           "frac_event_bracketed every launch between its own pair of events (serialised)",
+                "frac_event_bracketed": (bracketed / peaks["hbm_gbs"]) if bracketed else None,
+                "frac_of_nominal_8TBs": achieved / 8000.0,
+                "hbm_read_probe_gbs": hbm_read, "frac_of_read_probe": (achieved / hbm_read) if hbm_read else None,
                 "bytes_per_launch": bytes_per_launch, "avg_launch_us": avg_launch_us, "launches_timed": 4 * n_prof,
                 "achieved_event_bracketed": bracketed, "traffic": args.traffic if args.traffic else 30.73e6,
                 "traffic_note": "ncu dram__bytes_read+write per launch, mean of the four launches of a step (123 MB / 4); equals the algorithmic bytes"}
@@ -905,6 +1065,8 @@ def run_ours(args):
         for s in range(start, start + n):
             r = s % R
             ctx.layer_decode_host(descs[r], x_host, y_host, caches[r][0], caches[r][1], pos, 1)
+    ctx.register_host_buffer(x_host)  # registered pinned buffers: no copy engine, completion word instead of a stream wait
+    ctx.register_host_buffer(y_host)
     e2e_steps(min(args.warmup, 50))
     barrier()
     n_e2e = min(args.steps, 5000)
@@ -915,7 +1077,8 @@ def run_ours(args):
     e2e_s = max_over_ranks(dist, e2e_s, "cuda")
     e2e = {"value": aggregate_throughput(world, n_e2e, e2e_s), "unit": "tokens/s", "h2d_bytes_per_step": int(x_host.numel() * 2),
            "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": n_e2e,
-           "d2h_via": "the layer's last kernel stores the result row into the pinned host buffer; the call returns after the stream has drained"}
+           "d2h_via": "registered pinned buffers: a kernel fetches the input row from the host buffer, the layer's last kernel stores the "
+                      "result row into the host buffer, the call returns when the device has written the completion word"}
     ctx.close()
     del ctx, caches
     torch.cuda.empty_cache()
@@ -923,14 +1086,23 @@ def run_ours(args):
     extra, cpu = {}, None
     if rank == 0:
         if not args.no_extra:
-            for name, fn in EXTRAS.items():
+            names = list(EXTRAS) if args.all_extras else ["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream"]
+            for name in names:
                 try:
-                    extra[name] = fn(torch, B, W, peaks, args.quick)
+                    extra[name] = EXTRAS[name](torch, B, W, peaks, args.quick)
                 except Exception as e:  # an extra must never take the headline line down
                     extra[name] = {"error": f"{type(e).__name__}: {e}"}
                 torch.cuda.empty_cache()
         if world == 1 and not args.no_cpu:
             cpu = time_oracle()
+            # the oracle beside every configuration's GPU figure (bounded samples; a reported baseline, not a target)
+            for name, fn in (("cfg1_gemv", cpu_baseline_cfg1), ("cfg3_prefill", cpu_baseline_cfg3), ("cfg4_moe", cpu_baseline_cfg4),
+                             ("cfg5_stream", cpu_baseline_cfg5)):
+                if isinstance(extra.get(name), dict) and "error" not in extra[name]:
+                    try:
+                        extra[name]["cpu_baseline"] = fn()
+                    except Exception as e:
+                        extra[name]["cpu_baseline"] = {"error": f"{type(e).__name__}: {e}"}
     sampler.stop()
     if dist is not None:
         dist.barrier()
@@ -945,7 +1117,7 @@ def run_ours(args):
                        "replicas_rotated": R, "weight_bytes_per_step": layer_bytes,
                        "l2_policy": f"steps rotate over {R} distinct layers ({R * layer_bytes / 1e6:.0f} MB of weights > 126 MB L2)",
                        "multi_gpu": "replicas only (no data-path collective)"},
-            "step_bytes_gbs": (layer_bytes + 2 * shape.n_kv_heads * cap * shape.head_dim * 2) / (ms / args.steps * 1e-3) / 1e9,
+            "step_bytes_gbs": step_gbs,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "extra": extra}
     print(json.dumps(line))
 
@@ -962,7 +1134,8 @@ def main():
     ap.add_argument("--quick", action="store_true", help="smaller extras")
     ap.add_argument("--only-extra", default=None, choices=["cfg1_gemv", "cfg3_prefill", "cfg4_moe", "cfg5_stream", "model_loop", "model_loop_moe", "w16_formats", "epd_profile", "mxfp4_formats"],
                     help="run just one of the other configs' measurements (quick size) and print it; used for profiling")
-    ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = 8, or 4 with --quick; 32 = the full configuration)")
+    ap.add_argument("--stack-layers", type=int, default=0, help="layers of the config-5 stack in the streaming extra (0 = the full 32, or 4 with --quick)")
+    ap.add_argument("--all-extras", action="store_true", help="also run the figures beyond the five configurations (other weight formats, whole-model loops, EPD profile)")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per GEMV launch to quote in roofline.traffic")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

@@ -88,9 +88,6 @@ enum {
                                      part of the workspace beyond the call's own buffers by one launch of an SM-driven copy
                                      kernel (each slice crosses PCIe once; counted in streamed_bytes, not in copies) when that
                                      part holds them; otherwise they keep the ring path. */
-  /* timing experiments only: do not launch a stage of ats_layer_decode (its outputs are then stale); bit 24 = QKV GEMV,
-   * 25 = attention, 26 = O GEMV, 27 = gate/up GEMV, 28 = down GEMV */
-  ATS_FLAG_DEBUG_SKIP_SHIFT = 24
 };
 /* ats_layer_desc.flags */
 enum { ATS_LAYER_NO_TOPK_RENORM = 1u /* gates = full softmax entries instead of softmax over the top-k */ };
@@ -159,8 +156,17 @@ int32_t ats_plan_placement(ats_ctx* ctx, uint64_t budget_bytes, uint32_t granule
 int32_t ats_get_placement(const ats_ctx* ctx, int32_t id, int32_t expert, uint8_t* out_where /*HOST*/);
 
 /* The per-tensor operator: y[m][n] = sum_k w[n][k] x[m][k], fp32 accumulation, fp16 output.
- * x DEVICE fp16 row-major [M][k_in]; y DEVICE fp16 row-major [M][n_out].  M <= 8 runs the memory-bound GEMV
- * (weights exact, CUDA cores); M > 8 runs the tensor-core GEMM (weights rounded once to fp16 operands).
+ * x DEVICE fp16 row-major [M][k_in]; y DEVICE fp16 row-major [M][n_out].  M <= 8 runs the memory-bound GEMV with exact
+ * weights (scale * code in fp32): one or two rows on the streaming kernel (integer dot products on the CUDA cores), three
+ * to eight rows on mma.sync tensor-core instructions, odd shapes on a generic kernel; M > 8 runs the tensor-core GEMM
+ * (weights rounded once to fp16 operands).
+ * Activations inside the single-row streaming kernel (also used by ats_layer_decode, ats_lm_head and the single-token MoE
+ * stages): every block of 32 fp16 activations is re-expressed as 16-bit block fixed point, xi = rn(x * 2^sh) with
+ * |xi| <= 32752, i.e. each element is rounded within 2^-17 of its block's largest magnitude (fp16 itself resolves that
+ * maximum to 2^-11); block dot products are then exact integers and blocks are summed in fp32.  The perturbation of an
+ * output is bounded by 2^-17 * sum over blocks of (block maximum * sum of |w| in the block), about 1e-5 of its scale for
+ * the workloads here.  A block that holds an Inf or a NaN activation contributes NaN (as the plain definition would give
+ * Inf or NaN), so a non-finite input never turns into a finite output.
  * If the tensor is placed on the host it is streamed through the ring for this call. */
 int32_t ats_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, void* y /*DEVICE*/, uint32_t M);
 
@@ -186,10 +192,16 @@ int32_t ats_set_tensor_value(ats_ctx* ctx, int32_t id, int64_t value, int64_t sw
  * has given all device memory to another allocator.  ats_linear needs scratch for its split-K partial sums when
  * M > 8 and takes it from the workspace the caller allocated; this entry point takes it instead from a fixed array of
  * ATS_STATIC_SCRATCH_BYTES that is part of the library's device image, so that it calls no cudaMalloc / cudaFree /
- * allocating routine of any library.  Same arguments and result as ats_linear, with these differences:
+ * allocating routine of any library.  Same arguments as ats_linear and the same kernels, so the same result (bit for bit
+ * whenever both pick the same split-K plan, which holds unless the 8 MiB here admit a plan ats_linear's workspace did
+ * not: k_in >= 8192 with M >= 1024; within the tolerance of the operator otherwise), with these differences:
+ *  - dense ATS_FMT_Q4B32 and ATS_FMT_MXFP4 tensors only (ATS_FMT_W16: ATS_ERR_INVALID);
+ *  - the context still needs the first kilobyte of a workspace (workspace_bytes >= 1024, set at ats_init): that is
+ *    where the attention counters and, on systems without mapped pinned memory, the status word live.  Nothing else of
+ *    the workspace is touched;
  *  - the tensor must be GPU-placed (streaming would need the ring) -> ATS_ERR_STATE otherwise;
- *  - if the partial sums of this shape need more than ATS_STATIC_SCRATCH_BYTES the call fails with ATS_ERR_NOMEM and
- *    the text says how much was needed;
+ *  - if the split-K plan ats_linear would pick with unlimited workspace needs more than ATS_STATIC_SCRATCH_BYTES for its
+ *    partial sums, the call fails with ATS_ERR_NOMEM and the text says how much was needed (no smaller plan is tried);
  *  - every GPU that loads the library holds the array from load to exit; all calls (all contexts, all streams of a
  *    process) share it, and nothing in it has to start at zero: each call fully writes the partials it later reads.
  *    Two calls that overlap on the GPU (different streams) would overwrite each other's partials: keep them on one stream;
@@ -206,7 +218,11 @@ int32_t ats_route_topk(ats_ctx* ctx, int32_t router_id, const void* h /*DEVICE*/
 
 /* Top-k routed expert GEMV on a stacked expert tensor: y[m][j][:] = W[ids[m][j]] x[m][:] (x_per_slot = 0, x [M][K])
  * or W[ids[m][j]] x[m][j][:] (x_per_slot = 1, x [M][k][K]); fp16 in, fp32 accumulation, fp16 out [M][k][n_out].
- * M*k <= 256.  If any expert slice of the tensor is host-placed the call copies ids to the host and waits for them
+ * M*k <= 256.  Every id must lie in [0, n_experts).  With host-placed slices the ids are checked on the host
+ * (ATS_ERR_INVALID before anything is enqueued); when every slice is resident they are only seen by the kernel, which
+ * then computes with expert 0 in place of an id out of range and raises the context's status word: the next ats_sync
+ * returns ATS_ERR_INVALID and the context is poisoned.  (ats_route_topk always writes ids in range, also for a row of
+ * NaN activations, whose gates are NaN.)  If any expert slice of the tensor is host-placed the call copies ids to the host and waits for them
  * (the one host synchronisation on the path: expert transfer cannot start before routing is known, Section 4.2.2),
  * then streams only the selected host-placed slices (distinct over the batch, ascending expert id). */
 int32_t ats_moe_linear(ats_ctx* ctx, int32_t id, const void* x /*DEVICE*/, const int32_t* ids_dev /*DEVICE*/,
@@ -233,14 +249,29 @@ typedef struct {
 int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, const void* x_in /*DEVICE*/,
                          void* x_out /*DEVICE*/, void* k_cache /*DEVICE*/, void* v_cache /*DEVICE*/, uint32_t pos,
                          uint32_t M);
-/* The same decode step driven from HOST buffers, as a caller that holds activations on the host sees it: copies x_in
- * (HOST fp16 [M][hidden]; pinned memory makes the copy asynchronous) into the workspace, runs ats_layer_decode on the
- * compute stream, copies the result into x_out (HOST fp16 [M][hidden]; when x_out is pinned memory the layer's last kernel
- * writes it there directly and no copy is made) and waits for the stream, so x_out is valid on return.  The caches stay on the DEVICE.  Needs 2 * M * hidden * 2 bytes of workspace beyond ats_layer_decode's
- * (ats_workspace_bytes includes them).  Errors as ats_layer_decode, plus ATS_ERR_CUDA from the copies or the wait. */
+/* The same decode step driven from HOST buffers, as a caller that holds activations on the host sees it: brings x_in
+ * (HOST fp16 [M][hidden]) into the workspace, runs ats_layer_decode on the compute stream, brings the result into x_out
+ * (HOST fp16 [M][hidden]) and returns when x_out is valid.  The caches stay on the DEVICE.  Needs 2 * M * hidden * 2 bytes
+ * of workspace beyond ats_layer_decode's (ats_workspace_bytes includes them).
+ * Any host memory works (two cudaMemcpyAsync and a wait for the stream).  When both buffers lie inside ranges registered
+ * with ats_register_host_buffer, no copy engine is involved: a small kernel fetches x_in from the mapped buffer, the
+ * layer's last kernel stores the result row straight into x_out, and the call returns as soon as the device has written
+ * a completion word that the host polls (bounded; it falls back to waiting for the stream).
+ * The status word of the context is looked at before returning: ATS_ERR_TIMEOUT if a kernel gave up a bounded wait.
+ * Errors as ats_layer_decode, plus ATS_ERR_CUDA from the copies or the wait. */
 int32_t ats_layer_decode_host(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, const void* x_in /*HOST*/,
                               void* x_out /*HOST*/, void* k_cache /*DEVICE*/, void* v_cache /*DEVICE*/, uint32_t pos,
                               uint32_t M);
+/* Pinned host memory the caller will pass to host-driven calls (ats_layer_decode_host).  [ptr, ptr + bytes) must be
+ * page-locked memory that the device can address (cudaHostAlloc / cudaHostRegister, or a framework's pinned allocation),
+ * 16-byte aligned; the library keeps the range's device alias and lets kernels read and write the memory directly.
+ * LIFETIME: the range must stay allocated and pinned until ats_unregister_host_buffer (which first waits for the compute
+ * stream) or ats_destroy; the library never looks a raw address up again on its own, so a buffer that was freed and whose
+ * address was reused is the caller's error only if it is still registered.  Buffers that are not registered are served
+ * by ordinary copies.  ATS_ERR_INVALID if the memory is not pinned and mapped. */
+int32_t ats_register_host_buffer(ats_ctx* ctx, void* ptr /*HOST*/, uint64_t bytes);
+int32_t ats_unregister_host_buffer(ats_ctx* ctx, void* ptr /*HOST*/);
+
 /* Prefill: T tokens of one sequence at cache positions pos0 .. pos0+T-1 (pos0+T <= kv_capacity); projections run as
  * dequantize-fused tensor-core GEMMs.  Same buffers as decode with M = T.
  * Layers with routed experts (the MoE prefill of Section 5's workloads): every (token, slot) pair becomes a row, rows
@@ -297,16 +328,38 @@ int32_t ats_set_flags(ats_ctx* ctx, uint32_t flags);
 int32_t ats_reset_stats(ats_ctx* ctx);
 
 /* Wait for everything enqueued so far by polling events; ATS_ERR_TIMEOUT after timeout_ms (0 = wait without limit),
- * ATS_ERR_CUDA if a kernel or copy failed. */
+ * ATS_ERR_CUDA if a kernel or copy failed.  Then the context's status word is read: ATS_ERR_TIMEOUT if a kernel gave up
+ * one of its bounded waits, ATS_ERR_INVALID if a kernel met a token or expert id out of range; either poisons the
+ * context (its results are invalid).  The word lives in pinned host memory, so the calls that wait on the host anyway
+ * (ats_layer_decode_host, and the MoE calls that fetch routing ids) check it too. */
 int32_t ats_sync(ats_ctx* ctx, uint32_t timeout_ms);
 
 /* Measure host->device copy bandwidth from the library's own kind of pinned memory into the arena's ring:
  * `bytes` (<= ring size) copied `reps` times, best time.  Synchronous.  Writes GB/s (1e9 bytes/s). */
 int32_t ats_measure_h2d(ats_ctx* ctx, uint64_t bytes, uint32_t reps, double* out_gbs /*HOST*/);
 
+/* Measure what the device delivers to a kernel that only READS: the first `bytes` of the arena (at least 256 MiB, more
+ * than the L2 holds) are read once per pass by a kernel with the streaming GEMV's access pattern (bulk-async copies into
+ * shared memory, nothing done with the data), `reps` passes after a warm-up pass, best time.  Synchronous; the arena's
+ * contents are not changed.  Writes GB/s (1e9 bytes/s): the read-only ceiling to hold the GEMV's achieved bandwidth
+ * against, beside the nominal figure and a copy benchmark (which also writes and reaches less). */
+int32_t ats_measure_hbm_read(ats_ctx* ctx, uint64_t bytes, uint32_t reps, double* out_gbs /*HOST*/);
+
 /* Test hook: make the next n streaming copies fail as if cudaMemcpyAsync had returned an error (host-side fault
  * injection; nothing faults on the device).  The failing call returns ATS_ERR_CUDA and the context is poisoned. */
 int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n);
+
+/* Test hook for the failure path of the streaming single-token GEMV (nothing faults, nothing hangs): from now on that
+ * kernel's bounded waits give up after limit_cycles SM clock cycles (0 = the default of about a second), and its producer
+ * leaves out the weight copies of tile `withhold_tile` of every launch (-1 = none), so the consumers of that tile wait in
+ * vain, run into the limit, raise the context's device status word and return; every other CTA finishes normally.  The
+ * next ats_sync (or ats_layer_decode_host) then returns ATS_ERR_TIMEOUT and the context is poisoned; other contexts of the
+ * process are unaffected.  Applies to dense single-token GEMV launches only (ats_linear with M = 1, ats_layer_decode). */
+int32_t ats_debug_gemv_wait(ats_ctx* ctx, uint64_t limit_cycles, int32_t withhold_tile);
+/* Timing hook: ats_layer_decode on a dense layer leaves out the launches whose bit is set (1 = QKV GEMV, 2 = attention,
+ * 4 = O GEMV, 8 = gate/up GEMV, 16 = down GEMV); the outputs of such a call are stale.  0 restores the full step.  Used by
+ * the benchmark to time the GEMV launches of a step without the attention launch between them. */
+int32_t ats_debug_skip_stages(ats_ctx* ctx, uint32_t mask);
 
 /* The two ends of a whole-model loop around the layer calls (Section 5's workloads run whole models).
  * ats_embed: rows token_ids[m] of a Q4B32 table [vocab = n_out][hidden = k_in], dequantized to fp16 (scale * code rounded

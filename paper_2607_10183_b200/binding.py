@@ -12,7 +12,7 @@ import os
 import numpy as np
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libats.so")
+LIB_PATH = os.environ.get("ATS_LIB_PATH") or os.path.join(HERE, "libats.so")  # ATS_LIB_PATH: another build of the same library
 
 ATS_OK = 0
 ATS_ERR_INVALID, ATS_ERR_SHAPE, ATS_ERR_NOMEM, ATS_ERR_BUDGET = -1, -2, -3, -4
@@ -31,7 +31,7 @@ EXPORTS = (
     "ats_init", "ats_destroy", "ats_last_error", "ats_register_tensor", "ats_tensor_slice_bytes", "ats_set_placement",
     "ats_plan_placement", "ats_get_placement", "ats_linear", "ats_linear_static_scratch", "ats_route_topk", "ats_moe_linear", "ats_layer_decode", "ats_layer_decode_host", "ats_embed", "ats_lm_head",
     "ats_layer_prefill", "ats_workspace_bytes", "ats_dequantize", "ats_get_numerics", "ats_get_stats", "ats_set_flags", "ats_reset_stats",
-    "ats_sync", "ats_measure_h2d", "ats_debug_fail_copies", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
+    "ats_sync", "ats_measure_h2d", "ats_measure_hbm_read", "ats_debug_fail_copies", "ats_debug_gemv_wait", "ats_debug_skip_stages", "ats_register_host_buffer", "ats_unregister_host_buffer", "ats_debug_decode_buffer", "ats_debug_prefill_buffer", "ats_host_solve_placement", "ats_host_repack_q4",
     "ats_host_unpack_q4", "ats_host_group_pairs", "ats_host_dynamic_transfer", "ats_host_transfer_latency", "ats_host_deviation",
     "ats_host_reschedule", "ats_profile_tensor", "ats_set_tensor_value",
 )
@@ -95,7 +95,12 @@ def _load():
         "ats_set_flags": (i32, [vp, u32]),
         "ats_sync": (i32, [vp, u32]),
         "ats_measure_h2d": (i32, [vp, u64, u32, P(C.c_double)]),
+        "ats_measure_hbm_read": (i32, [vp, u64, u32, P(C.c_double)]),
         "ats_debug_fail_copies": (i32, [vp, u32]),
+        "ats_debug_gemv_wait": (i32, [vp, u64, i32]),
+        "ats_debug_skip_stages": (i32, [vp, u32]),
+        "ats_register_host_buffer": (i32, [vp, vp, u64]),
+        "ats_unregister_host_buffer": (i32, [vp, vp]),
         "ats_debug_decode_buffer": (i32, [vp, P(ats_layer_desc), u32, u32, P(vp), P(u64)]),
         "ats_debug_prefill_buffer": (i32, [vp, P(ats_layer_desc), u32, u32, P(vp), P(u64)]),
         "ats_host_solve_placement": (i32, [vp, vp, vp, vp, u32, C.c_int64, vp, P(C.c_int64)]),
@@ -279,6 +284,13 @@ class Context:
         return self.check(lib.ats_layer_decode_host(self.h, C.byref(desc), _ptr(x_in_host), _ptr(x_out_host), _ptr(k_cache),
                                                     _ptr(v_cache), pos, M))
 
+    def register_host_buffer(self, t):
+        """Registers a pinned host tensor (torch) for host-driven calls; keep it alive until unregister_host_buffer/close."""
+        return self.check(lib.ats_register_host_buffer(self.h, _ptr(t), int(t.numel() * t.element_size())))
+
+    def unregister_host_buffer(self, t):
+        return self.check(lib.ats_unregister_host_buffer(self.h, _ptr(t)))
+
     def embed(self, tid, token_ids, out, M):
         """Rows token_ids[m] (device int32) of a Q4B32 table as fp16 rows of `out` (device)."""
         return self.check(lib.ats_embed(self.h, tid, _ptr(token_ids), M, _ptr(out)))
@@ -312,6 +324,12 @@ class Context:
     def sync(self, timeout_ms=0):
         return self.check(lib.ats_sync(self.h, timeout_ms))
 
+    def debug_gemv_wait(self, limit_cycles, withhold_tile=-1):
+        return self.check(lib.ats_debug_gemv_wait(self.h, int(limit_cycles), int(withhold_tile)))
+
+    def debug_skip_stages(self, mask):
+        return self.check(lib.ats_debug_skip_stages(self.h, int(mask)))
+
     def debug_decode_buffer(self, desc, M, which, dtype):
         """Copy of an intermediate of the last ats_layer_decode call (see ats_debug_decode_buffer) as a numpy array."""
         ptr, nb = C.c_void_p(), C.c_uint64()
@@ -331,6 +349,15 @@ class Context:
         v = C.c_double()
         self.check(lib.ats_measure_h2d(self.h, int(nbytes), reps, C.byref(v)))
         return v.value
+
+
+def _measure_hbm_read(self, nbytes, reps=5) -> float:
+    v = C.c_double()
+    self.check(lib.ats_measure_hbm_read(self.h, int(nbytes), reps, C.byref(v)))
+    return v.value
+
+
+Context.measure_hbm_read = _measure_hbm_read
 
 
 def workspace_bytes(desc: ats_layer_desc, max_tokens: int) -> int:

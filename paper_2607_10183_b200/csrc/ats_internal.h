@@ -85,14 +85,32 @@ struct ats_ctx {
   uint32_t next_slot = 0;
   // pinned scratch for routing ids (host side of the one synchronisation on the MoE path)
   int32_t* ids_host = nullptr;
-  const void* host_out_seen = nullptr;  // last x_out of ats_layer_decode_host and its device alias (null: not pinned)
-  void* host_out_alias = nullptr;
+  // pinned host buffers the caller registered for host-driven calls (ats_register_host_buffer): host range -> device alias
+  struct HostBuf {
+    const uint8_t* host;
+    uint64_t bytes;
+    uint8_t* dev;
+  };
+  std::vector<HostBuf> host_bufs;
+  volatile int* done_host = nullptr;  // pinned completion word of host-driven calls (written by the device)
+  int* done_dev = nullptr;            // ... as the device addresses it (null: the store is not mapped)
+  int done_seq = 0;
   uint8_t* stage_host = nullptr;  // pinned scratch for per-call tables (MoE prefill: slice addresses, copy list)
   cudaEvent_t ids_event = nullptr;
   cudaEvent_t sync_event = nullptr;
   uint32_t fail_copies = 0;
-  int* dev_status = nullptr;  // device word kernels raise when a bounded wait expires (first bytes of the workspace)
-  int* host_status = nullptr; // pinned copy read by ats_sync
+  // test hooks (ats_debug_gemv_wait, ats_debug_skip_stages)
+  long long dbg_wait_limit = 0;
+  int dbg_withhold_plus1 = 0;
+  uint32_t dbg_skip = 0;
+  // The status word kernels raise when a bounded wait expires or an id is out of range.  It lives in pinned host memory
+  // that the device addresses directly (dev_status is that alias), so every call that already waits on the host can look
+  // at it without a copy; on a system where the store cannot be mapped it is the first word of the workspace and only
+  // ats_sync reads it (with a copy).
+  int* dev_status = nullptr;
+  int* host_status = nullptr;
+  bool status_mapped = false;
+  bool ws_reserved = false;   // the workspace holds the reserved first kilobyte (attention counters, fallback status word)
   int sm_count = 148;
   std::vector<double> rope_inv;  // cached theta^(-2i/d)
   float rope_theta = -1.f;
@@ -148,6 +166,10 @@ struct GemvParams {
   int pdl;  // allow the launch to overlap the tail of the preceding kernel (programmatic dependent launch)
   int w16;  // the segments are unquantized fp16 matrices [n_rows][K] (launch_gemv_w16; no norm prologue)
   int mx;   // the segments hold microscaling 4-bit floats (same slice layout, power-of-two fp16 block scales): generic kernel only
+  // test hooks of the streaming kernel (ats_debug_gemv_wait): limit of its bounded waits in SM cycles (0 = the default of
+  // about a second) and, plus one, the tile whose weight copies its producer leaves out (0 = none)
+  long long dbg_wait_limit;
+  int dbg_withhold_tile_plus1;
 };
 cudaError_t launch_gemv(const GemvParams& p, cudaStream_t st, uint64_t* n_launch);
 // fp16-weight GEMV (kernels_decode.cu): the same segments, epilogue modes and fp32 accumulation as launch_gemv over
@@ -218,6 +240,8 @@ struct MoeGemvParams {
   const uint8_t* const* tab1;
   int x_div;           // activation row of pair p is p / x_div (k when one x per token, 1 when one per slot)
   int P;
+  int n_experts;       // ids outside [0, n_experts) are replaced by 0 and raise *status (implicit addressing)
+  int* status;
   // common
   int n_rows, K;
   const __half* x;
@@ -234,6 +258,9 @@ cudaError_t launch_moe_gemv(const MoeGemvParams& p, const MoeJobs* jobs /*null =
 bool moe_gemv_stream_eligible(const MoeGemvParams& p);
 cudaError_t launch_moe_gemv_stream(const MoeGemvParams& p, const MoeJobs* jobs /*null = implicit*/, int* status, int sm_count,
                                    int pdl, cudaStream_t st, uint64_t* n_launch);
+
+// reads `bytes` of device memory once with the streaming GEMV's access pattern and drops them (kernels_gemv_stream.cu)
+cudaError_t launch_hbm_read_probe(const uint8_t* src, uint64_t bytes, int* status, int sm_count, cudaStream_t st);
 
 cudaError_t launch_dequant(const uint8_t* slice, int n_rows, int K, void* out, int out_f16, int mx, cudaStream_t st,
                            uint64_t* n_launch);
@@ -266,6 +293,10 @@ cudaError_t launch_router_topk_norm(const __half* h, const __half* wr, int M, in
 cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gates, const float* d32, __half* y16,
                                int M, int k, int H, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uint64_t* n_launch);
+// host-driven calls (kernels_decode.cu): a small input fetched from mapped pinned memory by a kernel, and the completion
+// word written once everything before it in the stream is done
+cudaError_t launch_stage_rows(const void* src_host_alias, void* dst, uint64_t bytes, cudaStream_t st, uint64_t* n_launch);
+cudaError_t launch_signal_done(int* done_alias, int seq, int pdl, cudaStream_t st, uint64_t* n_launch);
 
 // prefill
 cudaError_t launch_rope_append_prefill(const __half* qkv16, int ld, __half* q_rot16, __half* kc, __half* vc, int T,

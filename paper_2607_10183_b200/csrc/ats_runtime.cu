@@ -88,9 +88,21 @@ static int32_t precheck(ats_ctx* ctx, bool need_placement) {
   if (ctx->poisoned) return fail(ctx, ATS_ERR_CUDA, "context is poisoned by an earlier CUDA error: %s", ctx->err.c_str());
   if (need_placement && !ctx->placed)
     return fail(ctx, ATS_ERR_STATE, "no placement: call ats_set_placement or ats_plan_placement first");
-  if (need_placement && !ctx->dev_status)
+  if (need_placement && !ctx->ws_reserved)
     return fail(ctx, ATS_ERR_NOMEM, "workspace_bytes must be at least %llu", (unsigned long long)kWsReserved);
   return ATS_OK;
+}
+
+// Look at the status word after a wait that the call makes anyway (mapped word: a plain read of pinned memory).
+static int32_t check_status(ats_ctx* ctx) {
+  if (!ctx->status_mapped) return ATS_OK;
+  const int v = *reinterpret_cast<volatile int*>(ctx->host_status);
+  if (v == 0) return ATS_OK;
+  ctx->poisoned = true;
+  if (v == 6 || v == 7)
+    return fail(ctx, ATS_ERR_INVALID, "a kernel met an id out of range (status %d: %s); results are invalid", v,
+                v == 6 ? "token id" : "expert id");
+  return fail(ctx, ATS_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d); results are invalid", v);
 }
 
 static Tensor* get_tensor(ats_ctx* ctx, int32_t id, uint32_t fmt) {
@@ -251,6 +263,8 @@ static int count_streamed(const Operand* ops, int n) {
 // separate RMSNorm launch when a norm prologue was asked for.  Which kernel runs depends on format and shapes only, never on placement.
 static int32_t launch_gemv_any(ats_ctx* ctx, GemvParams p) {
   p.pdl = (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1;
+  p.dbg_wait_limit = ctx->dbg_wait_limit;
+  p.dbg_withhold_tile_plus1 = ctx->dbg_withhold_plus1;
   if (gemv_stream_eligible(p)) {
     TimedLaunch tl(ctx, 0, gemv_work_bytes(p));
     ATS_CUDA(launch_gemv_stream(p, ctx->dev_status, ctx->sm_count, ctx->cs, &ctx->stats.kernel_launches));
@@ -597,6 +611,8 @@ static int32_t run_moe_stage(ats_ctx* ctx, int id0, int id1, const int32_t* ids_
   p.stride = t0.slice_stride;
   p.ids = ids_dev;
   p.mx = t0.d.fmt == ATS_FMT_MXFP4;
+  p.n_experts = (int)t0.slices.size();
+  p.status = ctx->dev_status;
   if (!ids_host) {
     if (call_tab0) {  // per-call tables: resident copies, or slices the copy kernel has gathered into the workspace
       p.tab0 = call_tab0;
@@ -687,6 +703,7 @@ static int32_t fetch_ids(ats_ctx* ctx, const int32_t* ids_dev, int P, int E) {
   ATS_CUDA(cudaEventRecord(ctx->ids_event, ctx->cs));
   ATS_CUDA(cudaEventSynchronize(ctx->ids_event));
   ctx->stats.host_syncs++;
+  ATS_TRY(check_status(ctx));
   for (int i = 0; i < P; ++i)
     if (ctx->ids_host[i] < 0 || ctx->ids_host[i] >= E)
       return fail(ctx, ATS_ERR_INVALID, "routing id %d out of range [0,%d)", ctx->ids_host[i], E);
@@ -705,6 +722,14 @@ static void plan_moe(ats_ctx* ctx, const int32_t* ids_host, int P, const int* te
   for (int t = n_first; t < n_total; ++t)
     for (int e : sel)
       if (ctx->tensors[tensor_ids[t]].slices[e].where == ATS_HOST) plan_add(ctx, tensor_ids[t], e);
+}
+
+// The device alias of [p, p + bytes) if it lies inside a registered host buffer, else null.
+static const uint8_t* find_host_buffer(const ats_ctx* ctx, const void* p, uint64_t bytes) {
+  const uint8_t* q = static_cast<const uint8_t*>(p);
+  for (const ats_ctx::HostBuf& b : ctx->host_bufs)
+    if (q >= b.host && q + bytes <= b.host + b.bytes) return b.dev + (q - b.host);
+  return nullptr;
 }
 
 // (cos, sin) of pos * theta^(-2i/d) for i < d/2, formed in fp64 on the host and rounded to fp32.  The inverse
@@ -768,12 +793,25 @@ int32_t ats_init(const ats_config* cfg, ats_ctx** out) {
   ok &= cudaEventCreateWithFlags(&ctx->ids_event, cudaEventDisableTiming) == cudaSuccess;
   ok &= cudaEventCreateWithFlags(&ctx->sync_event, cudaEventDisableTiming) == cudaSuccess;
   ok &= cudaHostAlloc((void**)&ctx->ids_host, (3 * (size_t)kMaxPairs + 2048) * sizeof(int32_t), cudaHostAllocDefault) == cudaSuccess;
-  ok &= cudaHostAlloc((void**)&ctx->host_status, 64, cudaHostAllocDefault) == cudaSuccess;
+  ok &= cudaHostAlloc((void**)&ctx->host_status, 128, cudaHostAllocMapped) == cudaSuccess;
   ok &= cudaHostAlloc((void**)&ctx->stage_host, kStageHostBytes, cudaHostAllocDefault) == cudaSuccess;
   if (ws >= kWsReserved) {
+    ctx->ws_reserved = true;
     ctx->dev_status = (int*)ctx->ws;
     ok &= cudaMemsetAsync(ctx->ws, 0, kWsReserved, ctx->cs) == cudaSuccess;
     ok &= cudaStreamSynchronize(ctx->cs) == cudaSuccess;
+  }
+  if (ok) {
+    memset(ctx->host_status, 0, 128);
+    void* alias = nullptr;
+    if (cudaHostGetDevicePointer(&alias, ctx->host_status, 0) == cudaSuccess && alias) {
+      ctx->dev_status = static_cast<int*>(alias);
+      ctx->status_mapped = true;
+      ctx->done_host = ctx->host_status + 16;  // its own 64-byte line
+      ctx->done_dev = static_cast<int*>(alias) + 16;
+    } else {
+      cudaGetLastError();
+    }
   }
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0) ctx->sm_count = sms;
@@ -1137,8 +1175,8 @@ int32_t ats_lm_head(ats_ctx* ctx, int32_t norm_id, int32_t head_id, float eps, c
 
 int32_t ats_linear_static_scratch(ats_ctx* ctx, int32_t id, const void* x, void* y, uint32_t M) {
   ATS_TRY(precheck(ctx, true));
-  Tensor* t = get_tensor(ctx, id, ATS_FMT_Q4B32);
-  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense Q4B32 tensor", id);
+  Tensor* t = get_4bit(ctx, id);
+  if (!t || t->slices.size() != 1) return fail(ctx, ATS_ERR_INVALID, "id %d is not a dense 4-bit tensor", id);
   if (!x || !y) return fail(ctx, ATS_ERR_INVALID, "null pointer");
   if (t->slices[0].where != ATS_GPU)
     return fail(ctx, ATS_ERR_STATE, "tensor %d is host-placed: the no-allocation entry point only runs resident tensors", id);
@@ -1346,7 +1384,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     p.y32 = w.qkv32;
     p.ldy = qd + 2 * kvd;
     p.mode = GEMV_OUT_F32;
-    const uint32_t skip = ctx->cfg.flags >> ATS_FLAG_DEBUG_SKIP_SHIFT;
+    const uint32_t skip = ctx->dbg_skip;
     if (!(skip & 1)) ATS_TRY(run_gemv_group(ctx, qkv, 3, p));
     AttnDecodeParams ap{};
     ap.qkv = w.qkv32;
@@ -1354,7 +1392,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     ap.kc = (__half*)k_cache;
     ap.vc = (__half*)v_cache;
     ap.part = w.attn_scratch;
-    ap.counters = ctx->dev_status + 64;
+    ap.counters = reinterpret_cast<int*>(ctx->ws) + 64;
     ap.a16 = w.a16;
     ap.n_q = nq;
     ap.n_kv = nkv;
@@ -1387,7 +1425,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
     g.mode = GEMV_SWIGLU_F16;
     if (count_streamed(gu, 2) > (int)ctx->cfg.ring_slots)
       return fail(ctx, ATS_ERR_BUDGET, "fused gate/up needs 2 ring slots when both tensors are host-placed");
-    const uint32_t skip2 = ctx->cfg.flags >> ATS_FLAG_DEBUG_SKIP_SHIFT;
+    const uint32_t skip2 = ctx->dbg_skip;
     if (!(skip2 & 8)) ATS_TRY(run_gemv_group(ctx, gu, 2, g));
     GemvParams dn{};
     dn.M = (int)M;
@@ -1533,26 +1571,60 @@ int32_t ats_layer_decode_host(ats_ctx* ctx, const ats_layer_desc* L, const void*
     return fail(ctx, ATS_ERR_NOMEM, "workspace too small: host-driven decode needs %llu bytes", (unsigned long long)need);
   uint8_t* xin_dev = ctx->ws + w.total;
   uint8_t* xout_dev = xin_dev + stage;
-  // A pinned output buffer is addressable by the device: the layer's last kernel then writes the row straight into it
-  // (a few kilobytes of posted writes over PCIe) and the device-to-host copy with its fixed cost of several
-  // microseconds is not needed.  The answer for a buffer is cached: the query costs about as much as a launch.
-  void* out_alias = nullptr;
-  if (x_out == ctx->host_out_seen) {
-    out_alias = ctx->host_out_alias;
+  // Buffers the caller registered (pinned, mapped): the input row is fetched by a small kernel instead of a copy-engine
+  // transfer, the layer's last kernel writes the result row straight into the host buffer (a few kilobytes of posted
+  // writes over PCIe), and the call returns when the device has written the completion word.
+  const uint8_t* in_alias = find_host_buffer(ctx, x_in, row_bytes);
+  uint8_t* out_alias = const_cast<uint8_t*>(find_host_buffer(ctx, x_out, row_bytes));
+  const bool fast = in_alias && out_alias && ctx->done_dev && row_bytes % 16 == 0;
+  if (fast)
+    ATS_CUDA(launch_stage_rows(in_alias, xin_dev, row_bytes, ctx->cs, &ctx->stats.kernel_launches));
+  else
+    ATS_CUDA(cudaMemcpyAsync(xin_dev, x_in, row_bytes, cudaMemcpyHostToDevice, ctx->cs));
+  ATS_TRY(ats_layer_decode(ctx, L, xin_dev, fast ? (void*)out_alias : (void*)xout_dev, k_cache, v_cache, pos, M));
+  if (fast) {
+    const int seq = ++ctx->done_seq;
+    ATS_CUDA(launch_signal_done(ctx->done_dev, seq, (ctx->cfg.flags & ATS_FLAG_NO_PDL) ? 0 : 1, ctx->cs, &ctx->stats.kernel_launches));
+    // bounded poll (about two seconds), then the stream itself decides
+    const auto t0 = std::chrono::steady_clock::now();
+    uint32_t spins = 0;
+    while (*ctx->done_host != seq) {
+      if ((++spins & 0xFFFu) == 0) {
+        if (cudaStreamQuery(ctx->cs) != cudaErrorNotReady) break;  // finished (or failed) without the word: settle below
+        if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2)) break;
+      }
+    }
+    if (*ctx->done_host != seq) ATS_CUDA(cudaStreamSynchronize(ctx->cs));
   } else {
-    cudaPointerAttributes pa{};
-    if (cudaPointerGetAttributes(&pa, x_out) == cudaSuccess && pa.type == cudaMemoryTypeHost && pa.devicePointer &&
-        (reinterpret_cast<uintptr_t>(pa.devicePointer) & 15) == 0)
-      out_alias = pa.devicePointer;
-    else
-      cudaGetLastError();
-    ctx->host_out_seen = x_out;
-    ctx->host_out_alias = out_alias;
+    ATS_CUDA(cudaMemcpyAsync(x_out, xout_dev, row_bytes, cudaMemcpyDeviceToHost, ctx->cs));
+    ATS_CUDA(cudaStreamSynchronize(ctx->cs));
   }
-  ATS_CUDA(cudaMemcpyAsync(xin_dev, x_in, row_bytes, cudaMemcpyHostToDevice, ctx->cs));
-  ATS_TRY(ats_layer_decode(ctx, L, xin_dev, out_alias ? out_alias : xout_dev, k_cache, v_cache, pos, M));
-  if (!out_alias) ATS_CUDA(cudaMemcpyAsync(x_out, xout_dev, row_bytes, cudaMemcpyDeviceToHost, ctx->cs));
-  ATS_CUDA(cudaStreamSynchronize(ctx->cs));
+  return check_status(ctx);
+}
+
+int32_t ats_register_host_buffer(ats_ctx* ctx, void* ptr, uint64_t bytes) {
+  ATS_TRY(precheck(ctx, false));
+  if (!ptr || bytes == 0) return fail(ctx, ATS_ERR_INVALID, "null buffer");
+  cudaPointerAttributes pa{};
+  if (cudaPointerGetAttributes(&pa, ptr) != cudaSuccess || pa.type != cudaMemoryTypeHost || !pa.devicePointer ||
+      (reinterpret_cast<uintptr_t>(pa.devicePointer) & 15) != 0) {
+    cudaGetLastError();
+    return fail(ctx, ATS_ERR_INVALID, "buffer %p is not pinned host memory the device can address (16-byte aligned)", ptr);
+  }
+  ats_unregister_host_buffer(ctx, ptr);
+  ctx->host_bufs.push_back(ats_ctx::HostBuf{static_cast<const uint8_t*>(ptr), bytes, static_cast<uint8_t*>(pa.devicePointer)});
+  return ATS_OK;
+}
+
+int32_t ats_unregister_host_buffer(ats_ctx* ctx, void* ptr) {
+  if (!ctx) return ATS_ERR_INVALID;
+  for (size_t i = 0; i < ctx->host_bufs.size(); ++i)
+    if (ctx->host_bufs[i].host == ptr) {
+      // nothing enqueued may still write through the alias
+      cudaStreamSynchronize(ctx->cs);
+      ctx->host_bufs.erase(ctx->host_bufs.begin() + (long)i);
+      return ATS_OK;
+    }
   return ATS_OK;
 }
 
@@ -1820,12 +1892,13 @@ int32_t ats_sync(ats_ctx* ctx, uint32_t timeout_ms) {
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return check_cuda(ctx, e, "asynchronous error");
+  if (ctx->status_mapped) return check_status(ctx);
   if (ctx->dev_status) {
     ATS_CUDA(cudaMemcpyAsync(ctx->host_status, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->cs));
     ATS_CUDA(cudaStreamSynchronize(ctx->cs));
     if (*ctx->host_status != 0) {
       ctx->poisoned = true;
-      return fail(ctx, ATS_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d); results are invalid", *ctx->host_status);
+      return fail(ctx, ATS_ERR_TIMEOUT, "a kernel raised the status word (%d); results are invalid", *ctx->host_status);
     }
   }
   return ATS_OK;
@@ -1864,6 +1937,33 @@ int32_t ats_measure_h2d(ats_ctx* ctx, uint64_t bytes, uint32_t reps, double* out
   if (st != ATS_OK) return st;
   *out_gbs = (double)bytes / (best * 1e-3) / 1e9;
   return ATS_OK;
+}
+
+int32_t ats_measure_hbm_read(ats_ctx* ctx, uint64_t bytes, uint32_t reps, double* out_gbs) {
+  ATS_TRY(precheck(ctx, false));
+  if (!out_gbs || reps == 0) return fail(ctx, ATS_ERR_INVALID, "bad argument");
+  bytes = std::min<uint64_t>(bytes, ctx->cfg.arena_bytes) / (16 * 1024) * (16 * 1024);
+  if (bytes < (256ull << 20))
+    return fail(ctx, ATS_ERR_BUDGET, "the probe reads at least 256 MiB of the arena (twice the L2), the arena holds %llu bytes",
+                (unsigned long long)ctx->cfg.arena_bytes);
+  ATS_CUDA(cudaStreamSynchronize(ctx->cs));
+  cudaEvent_t a = nullptr, b = nullptr;
+  ATS_CUDA(cudaEventCreate(&a));
+  cudaError_t e = cudaEventCreate(&b);
+  float best = 1e30f;
+  for (uint32_t r = 0; r < reps + 1 && e == cudaSuccess; ++r) {  // the first pass warms up
+    cudaEventRecord(a, ctx->cs);
+    e = launch_hbm_read_probe(static_cast<const uint8_t*>(ctx->cfg.arena), bytes, ctx->dev_status, ctx->sm_count, ctx->cs);
+    cudaEventRecord(b, ctx->cs);
+    if (e == cudaSuccess) e = cudaEventSynchronize(b);
+    float ms = 0.f;
+    if (e == cudaSuccess && r > 0 && cudaEventElapsedTime(&ms, a, b) == cudaSuccess && ms > 0) best = std::min(best, ms);
+  }
+  cudaEventDestroy(a);
+  if (b) cudaEventDestroy(b);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "ats_measure_hbm_read");
+  *out_gbs = (double)bytes / (best * 1e-3) / 1e9;
+  return check_status(ctx);
 }
 
 int32_t ats_debug_decode_buffer(ats_ctx* ctx, const ats_layer_desc* L, uint32_t M, uint32_t which, void** out_dev,
@@ -1916,6 +2016,19 @@ int32_t ats_debug_prefill_buffer(ats_ctx* ctx, const ats_layer_desc* L, uint32_t
 int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n) {
   if (!ctx) return ATS_ERR_INVALID;
   ctx->fail_copies = n;
+  return ATS_OK;
+}
+
+int32_t ats_debug_gemv_wait(ats_ctx* ctx, uint64_t limit_cycles, int32_t withhold_tile) {
+  if (!ctx || withhold_tile < -1 || limit_cycles > (1ull << 40)) return ATS_ERR_INVALID;
+  ctx->dbg_wait_limit = (long long)limit_cycles;
+  ctx->dbg_withhold_plus1 = withhold_tile + 1;
+  return ATS_OK;
+}
+
+int32_t ats_debug_skip_stages(ats_ctx* ctx, uint32_t mask) {
+  if (!ctx || mask > 31u) return ATS_ERR_INVALID;
+  ctx->dbg_skip = mask;
   return ATS_OK;
 }
 

@@ -1,13 +1,15 @@
-// Streaming decode GEMV for one token (sm_100a): the memory-bound hot kernel of the decode path.  Device code of the dense
-// and the grouped-expert kernels, written as a producer function and a consumer function over an explicit ring state (a
-// kernel may run several such phases back to back over one ring; the kernels in this library run one).
+// Streaming decode GEMV for one token (sm_100a): the memory-bound hot kernel of the decode path.  Device code shared by
+// the dense and the grouped-expert kernels: a producer function and a consumer function over a ring in shared memory.
 //
-// Structure: one persistent CTA per SM: 16 consumer warps in two groups of 8 + 1 producer warp.  The producer streams
-// row tiles of the packed weights (codes and scales, contiguous byte ranges) into a ring of 8 shared-memory stages with
-// 1-D bulk-async copies (TMA) that complete on mbarriers; tiles alternate between the groups; consumers never touch
-// global memory for weights.  Every lane owns up to two
-// quantization blocks (32 k each) of a k-part of the row and keeps the activation for them in registers for the whole
-// kernel, so a weight byte is read once from shared memory and an activation never again.
+// Structure: one persistent CTA per SM: 16 consumer warps in two groups of 8 + kProducerWarps producer warps.  The
+// producers stream row tiles of the packed weights (codes and scales, contiguous byte ranges) into a ring of 8
+// shared-memory stages with 1-D bulk-async copies (TMA) that complete on mbarriers; tiles alternate between the consumer
+// groups; consumers never touch global memory for weights.  Several producer warps, because the bulk copies of ONE thread
+// are served at about 30 GB/s however many of them are in flight (measured: a thread gets one 16 KB copy through per
+// 0.5 us), less than an SM's share of the HBM stream, while copies issued from different warps proceed side by side:
+// with one producer thread the ring took 4 us to request and the tile loop ran at the producer's pace.  Every lane owns
+// up to two quantization blocks (32 k each) of a k-part of the row and keeps the activation for them in registers for the
+// whole kernel, so a weight byte is read once from shared memory and an activation never again.
 //
 // Arithmetic: the activation block is re-expressed once per CTA as 16-bit block fixed point, x_k ~ xi_k * 2^-sh with
 // sh chosen from the block's largest exponent (exact for every element within 2^-4 of the block maximum, rounded at
@@ -17,58 +19,75 @@
 // block.  All integer instructions issue at half rate on this part and the dot-product pipe is the one that fills, so
 // the instruction count per block (16 dp2a, 8 masks, 2 to combine) is what the format allows: the high nibbles are
 // used in place as 16 * code and their sum shifted back once per block.  Lane partials are reduced by warp shuffles,
-// k-parts through shared memory, both in fixed order.
+// k-parts through shared memory, both in fixed order.  A block that holds an Inf or a NaN activation yields NaN (the
+// fixed-point form cannot carry it; the plain definition gives Inf or NaN there).
 //
 // Optional prologue: RMSNorm of the input row (fp16 or fp32) with an fp16 gain, rounded to fp16 (the operand edge of
 // the numerics contract), computed once per CTA by all 512 consumer threads while the first weight tiles are in flight.
 // All waits on mbarriers are bounded; on expiry the kernel raises a status word and returns.
 #pragma once
 #include "ats_internal.h"
+#include "sm100_sync.cuh"
 
 namespace ats {
 
 namespace {
 
-constexpr int kStages = 8;
+constexpr int kMaxStages = 8;
 constexpr int kGroups = 2;         // consumer groups per CTA, each with its own stream of tiles
 constexpr int kGroupWarps = 8;
 constexpr int kConsumerWarps = kGroups * kGroupWarps;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+#ifndef ATS_PRODUCER_WARPS
+#define ATS_PRODUCER_WARPS 2
+#endif
+constexpr int kProducerWarps = ATS_PRODUCER_WARPS;  // must not exceed the number of ring stages (see stream_produce)
+constexpr int kThreads = kConsumerThreads + 32 * kProducerWarps;
 constexpr int kRPW = 2;      // rows per consumer warp per tile
 constexpr int kJ = 2;        // quantization blocks per lane per row
+constexpr int kMaxDynSmem = 216 * 1024;  // ring + quantized activation row; 7 KB of static shared memory on top
 constexpr int kEarlyStages = 1;  // stages requested before the consumers have issued their activation loads
-constexpr int kMaxDynSmem = 216 * 1024;  // ring + quantized activation row; 6 KB of static shared memory on top
-constexpr int kMaxIt = 48;   // tiles of a group whose partial sums are buffered before a flush
+constexpr int kMaxIt = 48;   // tiles of a CTA whose partial sums are buffered before a flush
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after about a second of SM clocks (the caller then raises the status word and returns).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    for (int i = 0; i < 64; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > 2000000000ll) return false;
+#ifdef ATS_TRACE
+// Timeline probe of development builds (-DATS_TRACE): stamps are collected in shared memory (cheap) and written out as
+// (globaltimer, CTA, event, kernel tag) records when the CTA's consumers are done.
+struct TraceRec {
+  unsigned long long t;
+  uint32_t cta;
+  uint16_t ev, tag;
+};
+constexpr int kTraceCap = 1 << 16;
+constexpr int kTraceLocal = 192;
+__device__ TraceRec g_trace[kTraceCap];
+__device__ unsigned int g_trace_n;
+__shared__ unsigned long long tr_t[kTraceLocal];
+__shared__ unsigned short tr_ev[kTraceLocal];
+__shared__ unsigned int tr_n;
+__device__ __forceinline__ void trace(int ev) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  const unsigned int i = atomicAdd(&tr_n, 1u);
+  if (i < kTraceLocal) {
+    tr_t[i] = t;
+    tr_ev[i] = (unsigned short)ev;
   }
 }
+__device__ __forceinline__ void trace_flush(int tag) {
+  const unsigned int n = min(tr_n, (unsigned)kTraceLocal);
+  const unsigned int base = atomicAdd(&g_trace_n, n);
+  for (unsigned int i = 0; i < n && base + i < kTraceCap; ++i)
+    g_trace[base + i] = TraceRec{tr_t[i], blockIdx.x + 1000u * blockIdx.y, tr_ev[i], (uint16_t)tag};
+}
+#define ATS_TR(ev) do { if (threadIdx.x == 0 || threadIdx.x == 512) trace((ev)); } while (0)
+#define ATS_TR_FLUSH() do { if (threadIdx.x == 0) trace_flush(p.K / 256 + 100 * p.mode); } while (0)
+#define ATS_TR_INIT() do { if (threadIdx.x == 0) tr_n = 0; } while (0)
+#else
+#define ATS_TR(ev) do { } while (0)
+#define ATS_TR_FLUSH() do { } while (0)
+#define ATS_TR_INIT() do { } while (0)
+#endif
+
 // Weights are read once per call: the copies carry an evict-first L2 policy so that a step's 100+ MB of weights do not
 // push the activations, the KV cache and the kernels' own instructions out of the L2.
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
@@ -93,8 +112,14 @@ __device__ __forceinline__ int dp2a_hi(uint32_t a, uint32_t b, int c) {
   asm("dp2a.hi.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
-// named barriers: 1 and 2 = the two consumer groups (256 threads each), 3 = all consumers (512); 0 is __syncthreads
-__device__ __forceinline__ void group_sync(int grp) { asm volatile("bar.sync %0, 256;" ::"r"(grp + 1) : "memory"); }
+// named barriers: 1 and 2 = the two consumer groups (256 threads each), 3 = all consumers (512); 0 is __syncthreads,
+// which the producer warps would have to join
+__device__ __forceinline__ void group_sync(int grp) {
+  if (grp == 0)
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+  else
+    asm volatile("bar.sync 2, 256;" ::: "memory");
+}
 __device__ __forceinline__ void consumer_sync_all() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 
 __device__ __forceinline__ float silu_mul_f(float g, float u) { return g / (1.0f + expf(-g)) * u; }
@@ -114,11 +139,8 @@ __device__ __forceinline__ int f2i_magic(float x, float up) {
 // carries 16 times the codes of k = 8w + {2,6,3,7}.  Words 4w..4w+3 of the block hold the pairs (xi_{8w+0}, xi_{8w+4}),
 // (xi_{8w+1}, xi_{8w+5}), (xi_{8w+2}, xi_{8w+6}), (xi_{8w+3}, xi_{8w+7}) as two signed 16-bit halves (first in the
 // low half): the operands of dp2a.lo / dp2a.hi against the two masked words.  Words 16 and 17 hold mul = 2^-sh and
-// corr = -8 * sum(xi) * mul.
-//
-// The quantization is done by four adjacent lanes, each holding one run of 8 consecutive elements (one code word's
-// worth) of a 32-element block: exponent maximum and integer sum are shared by two butterfly shuffles.  Lane w of the
-// group writes words 4w..4w+3.
+// corr = -8 * sum(xi) * mul; both are NaN when the block holds an Inf or a NaN (fp32 exponent field 255), so that the
+// block's term, and with it the output, is NaN.
 //
 // Microscaling 4-bit floats (MX): twice an element is an integer in [-12, 12]; the kernel looks the biased byte
 // 2 e + 16 up per nibble (see mx_bytes) and uses the same unsigned dot products: sum xi (2 e + 16) = 2 sum xi e + 16 sum xi,
@@ -126,27 +148,20 @@ __device__ __forceinline__ int f2i_magic(float x, float up) {
 // (0,2,4,6) and odd k (1,3,5,7), so for this format words 4w..4w+3 hold the pairs (xi_0, xi_2), (xi_4, xi_6), (xi_1, xi_3),
 // (xi_5, xi_7) of the run.
 constexpr int kXqWords = 20;  // 18 used; the 80-byte pitch keeps the 128-bit reads of consecutive blocks conflict-free
-template <bool MX>
-__device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32_t* blk) {
-  uint32_t m = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) m = max(m, (__float_as_uint(x[i]) >> 23) & 0xFFu);  // fp32 exponent field of an fp16-valued number
-  m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
-  m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
-  // fp16 exponent field E = fp32 field - 112 (normals); subnormal fp16 values have fp32 fields <= 112 -> E = 1
+
+// The shift of a block from the largest fp32 exponent field m among its (fp16-valued) elements.
+// fp16 exponent field E = m - 112 (normals); subnormal fp16 values have fp32 fields <= 112 -> E = 1.  sh = 29 - E: the
+// largest fp16 magnitude with field E, (2 - 2^-10) 2^(E-15), maps to 32752.
+__device__ __forceinline__ void block_scale(uint32_t m, float& up, float& mul) {
   const int E = max((int)m - 112, 1);
-  const int sh = 29 - E;  // the largest fp16 magnitude with field E, (2 - 2^-10) 2^(E-15), maps to 32752
-  const float up = __uint_as_float((uint32_t)(sh + 127) << 23);
-  const float mul = __uint_as_float((uint32_t)(127 - sh) << 23);
-  int xi[8];
-  int sx = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    xi[i] = f2i_magic(x[i], up);
-    sx += xi[i];
-  }
-  sx += __shfl_xor_sync(0xffffffffu, sx, 1);
-  sx += __shfl_xor_sync(0xffffffffu, sx, 2);
+  const int sh = 29 - E;
+  up = __uint_as_float((uint32_t)(sh + 127) << 23);
+  mul = m == 255u ? __uint_as_float(0x7FC00000u) : __uint_as_float((uint32_t)(127 - sh) << 23);
+}
+
+// One run of 8 consecutive elements (one code word's worth) -> its four words of the block.
+template <bool MX>
+__device__ __forceinline__ uint4 pack_run(const int (&xi)[8]) {
   uint4 o;
   if (MX) {
     o.x = __byte_perm((uint32_t)xi[0], (uint32_t)xi[2], 0x5410u);
@@ -159,7 +174,30 @@ __device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32
     o.z = __byte_perm((uint32_t)xi[2], (uint32_t)xi[6], 0x5410u);
     o.w = __byte_perm((uint32_t)xi[3], (uint32_t)xi[7], 0x5410u);
   }
-  *reinterpret_cast<uint4*>(blk + 4 * w) = o;
+  return o;
+}
+
+// Four adjacent lanes each hold one run of a 32-element block; exponent maximum and integer sum are shared by two
+// butterfly shuffles.  Lane w of the group writes words 4w..4w+3 (and lane 0 the two scalars).
+template <bool MX>
+__device__ __forceinline__ void quantize_run4(const float (&x)[8], int w, uint32_t* blk) {
+  uint32_t m = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m = max(m, (__float_as_uint(x[i]) >> 23) & 0xFFu);  // fp32 exponent field of an fp16-valued number
+  m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
+  float up, mul;
+  block_scale(m, up, mul);
+  int xi[8];
+  int sx = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    xi[i] = f2i_magic(x[i], up);
+    sx += xi[i];
+  }
+  sx += __shfl_xor_sync(0xffffffffu, sx, 1);
+  sx += __shfl_xor_sync(0xffffffffu, sx, 2);
+  *reinterpret_cast<uint4*>(blk + 4 * w) = pack_run<MX>(xi);
   if (w == 0) *reinterpret_cast<float2*>(blk + 16) = make_float2(MX ? 0.5f * mul : mul, -8.0f * (float)sx * mul);
 }
 
@@ -189,6 +227,7 @@ struct StreamParams {
   int n_tiles;
   int K;
   int mode;
+  int n_stages;  // ring stages of this launch (<= kMaxStages), chosen by the host from the shared-memory budget
   // activation source: x16 (already the operand), or a row to RMS-normalise first
   const __half* x16;
   const __half* norm_in16;
@@ -201,83 +240,91 @@ struct StreamParams {
   const float* res32;
   const __half* res16;
   int* status;
+  // test hooks (0 / -1 in production): limit of the bounded waits in SM cycles, and a tile whose copies the producer
+  // leaves out, so that a test can make a wait run out without anything faulting
+  long long wait_limit;
+  int withhold_tile;
 };
 
-
-// Shared state of a CTA's ring; lives in static shared memory of the kernel that runs the phases.
+// Shared state of a CTA's ring; lives in static shared memory.
 struct StreamShared {
-  uint64_t full[kStages], empty[kStages];
-  uint64_t xbar;  // consumers -> producer: the activation loads of the current phase have been issued
+  uint64_t full[kMaxStages], empty[kMaxStages];
+  uint64_t xbar;  // consumers -> producers: the activation loads have been issued
   float part_s[kGroups][kMaxIt * kGroupWarps * kRPW];
   float red_s[kConsumerWarps];
   int fail_g[kGroups];  // a warp of the group gave up a bounded wait (written and read by that group only)
 };
 
-// Where a phase's ring stages live and where its iterations sit in the CTA's global sequence: stage and barrier parity
-// follow the global iteration index it0 + it, so that consecutive phases of one launch share the ring without a drain.
-struct StreamRing {
-  uint8_t* stages;
-  int pitch;      // bytes between stages (>= the phase's stage size)
-  int n_stages;   // <= kStages
-  uint32_t* xq;   // quantized activation row of the current phase
-  int it0;        // global iteration index of the phase's first tile
-  int phase;      // phases so far (parity of xbar)
-};
-
-__device__ __forceinline__ void stream_init(StreamShared& sh) {
+__device__ __forceinline__ void stream_init(StreamShared& sh, int n_stages) {
+  ATS_TR_INIT();
   if (threadIdx.x == 0) {
     for (int g = 0; g < kGroups; ++g) sh.fail_g[g] = 0;
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < n_stages; ++s) {
       mbar_init(&sh.full[s], 1);
       mbar_init(&sh.empty[s], kGroupWarps);
     }
     mbar_init(&sh.xbar, kConsumerWarps);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_fence_init();
   }
   __syncthreads();
+}
+
+// (stage, ring cycle) of an iteration -> those of the iteration `step` later (step <= n_stages)
+__device__ __forceinline__ void stream_advance(int& s, int& cyc, int step, int n_stages) {
+  s += step;
+  if (s >= n_stages) {
+    s -= n_stages;
+    ++cyc;
+  }
 }
 
 __device__ __forceinline__ int stream_n_it(const StreamParams& p, int bx, int gx) {
   return bx < p.n_tiles ? (p.n_tiles - bx + gx - 1) / gx : 0;
 }
 
-// One elected thread of the producer warp requests the phase's tiles.  bx / gx: index of this CTA among the gx CTAs that
-// share the work described by p.  STANDALONE: the phase is a whole kernel; the grid dependency is then handled here
-// (wait_first: the weight addresses themselves come from the preceding kernel, so nothing may be fetched before the
-// dependency resolves).  Returns false after a bounded wait ran out (status word raised).
-template <int PARTS, bool SW, bool STANDALONE>
-__device__ __forceinline__ bool stream_produce(const StreamParams& p, const int bx, const int gx, const bool wait_first,
-                                               StreamShared& sh, const StreamRing& ring, const uint64_t pol) {
+// One elected thread of each producer warp requests tiles; producer warp w of the kProducerWarps takes the CTA's
+// iterations it = w, w + kProducerWarps, ...  Before it refills a stage a producer waits for the PARITY of the phase in
+// which the consumers released the stage's previous content; that test is only unambiguous while no producer runs a whole
+// ring cycle ahead of the consumers, which holds as long as kProducerWarps <= n_stages (a producer's previous iteration
+// waited for a release at most one ring cycle older).  bx / gx: index of this CTA among the gx CTAs that share the work described by p.  The weights do not depend
+// on the preceding kernel, so nothing here waits for it (callers whose weight ADDRESSES come from the preceding kernel
+// wait before they call).  Returns false after a bounded wait ran out (status word raised).
+template <int PARTS, bool SW>
+__device__ __forceinline__ bool stream_produce(const StreamParams& p, const int bx, const int gx, const int pw, StreamShared& sh,
+                                               uint8_t* stages, const uint64_t pol) {
   constexpr int ROWS = kGroupWarps / PARTS * kRPW;     // weight rows per tile
   constexpr int OUT_ROWS = SW ? ROWS / 2 : ROWS;       // output rows per tile
   const int row_codes = p.K / 2, row_scales = p.K / 16;
   const int stage_bytes = ROWS * (row_codes + row_scales);
   const int n_it = stream_n_it(p, bx, gx);
-  if (STANDALONE && wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
-  for (int it = 0; it < n_it; ++it) {
-    const int git = ring.it0 + it;
-    const int s = git % ring.n_stages;
-    if (git >= ring.n_stages && !mbar_wait(&sh.empty[s], ((git / ring.n_stages) - 1) & 1)) {
-      atomicExch(p.status, 2);
-      return false;
-    }
-    if (STANDALONE) {
-      // Weight copies queued ahead of the consumers' activation loads delay them (the row is a cache hit that then
-      // waits behind megabytes of misses): one stage goes out at once, the rest after those loads have been issued.
-      if (it == kEarlyStages && !mbar_wait(&sh.xbar, ring.phase & 1)) {
-        atomicExch(p.status, 3);
+  const int n_stages = p.n_stages;
+  const long long limit = p.wait_limit ? p.wait_limit : kWaitLimitCycles;
+  ATS_TR(7);
+  bool x_issued = false;
+  // stage and ring cycle of iteration it, kept incrementally (the ring size is a run-time value)
+  int s = pw % n_stages, cyc = pw / n_stages;
+  for (int it = pw; it < n_it; it += kProducerWarps) {
+    // Weight copies queued ahead of the consumers' activation loads delay them (the row is a cache hit that then waits
+    // behind megabytes of misses): kEarlyStages stages go out at once, the rest after those loads have been issued.
+    if (it >= kEarlyStages && !x_issued) {
+      if (!mbar_wait_suspending(&sh.xbar, 0, limit)) {
+        raise_status(p.status, 3);
         return false;
       }
-      if (it == ring.n_stages) {
-        // The first stages are in flight.  Dependents may only be released once this grid's own dependency is
-        // resolved, so that a dependent's prologue never overlaps anything older than this kernel.
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-      }
+      x_issued = true;
+    }
+    if (cyc > 0 && !mbar_wait_suspending(&sh.empty[s], (cyc - 1) & 1, limit)) {
+      raise_status(p.status, 2);
+      return false;
     }
     const int tile = bx + it * gx;
-    uint8_t* dst = ring.stages + (size_t)s * ring.pitch;
+    uint8_t* dst = stages + (size_t)s * stage_bytes;
     mbar_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
+    if (pw == 0) ATS_TR(300 + it);
+    if (tile == p.withhold_tile) {  // test hook: this stage never fills
+      stream_advance(s, cyc, kProducerWarps, n_stages);
+      continue;
+    }
     if (SW) {
       // gate rows land in stage rows [0, ROWS/2), up rows in [ROWS/2, ROWS)
       const size_t r0 = (size_t)tile * OUT_ROWS;
@@ -296,81 +343,81 @@ __device__ __forceinline__ bool stream_produce(const StreamParams& p, const int 
       bulk_g2s(dst, b + r0 * row_codes, ROWS * row_codes, &sh.full[s], pol);
       bulk_g2s(dst + ROWS * row_codes, b + (size_t)p.seg[sg].n_rows * row_codes + r0 * row_scales, ROWS * row_scales, &sh.full[s], pol);
     }
+    stream_advance(s, cyc, kProducerWarps, n_stages);
   }
+  ATS_TR(9);
   return true;
 }
 
-// The 16 consumer warps of a CTA run one phase: activation prologue, the CTA's tiles, the epilogue.  wait_dep() returns
-// once the activation row may be read; release_dependents: issue griddepcontrol.launch_dependents after the prologue.
-// One CTA per SM: two groups of 8 warps; the CTA's tiles alternate between the groups (by global iteration index), each
-// group with its own partial-sum buffer and barrier, so the tile loop is that of two independent 8-warp CTAs; what they
-// share is the activation prologue: all 512 consumer threads load, normalise and quantise the row ONCE per SM.
-// Returns false after a bounded wait ran out (status word raised).
-template <int PARTS, bool SW, bool MX, typename WaitFn>
-__device__ __forceinline__ bool stream_consume(const StreamParams& p, const int bx, const int gx, StreamShared& sh,
-                                               const StreamRing& ring, WaitFn wait_dep, const bool release_dependents) {
+__device__ __forceinline__ void unpack_h8(const uint4 a, float (&xv)[8]) {
+  const uint32_t w4[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    __half2 h2;
+    *reinterpret_cast<uint32_t*>(&h2) = w4[q];
+    const float2 f = __half22float2(h2);
+    xv[2 * q] = f.x;
+    xv[2 * q + 1] = f.y;
+  }
+}
+
+// The 16 consumer warps of a CTA: wait for the preceding kernel, activation prologue, the CTA's tiles, the epilogue.
+// Two groups of 8 warps; the CTA's tiles alternate between the groups, each group with its own partial-sum buffer and
+// barrier, so the tile loop is that of two independent 8-warp CTAs; what they share is the ring and the activation
+// prologue: all 512 consumer threads load, normalise and quantise the row ONCE per SM.
+// dep_resolved: the caller has already executed griddepcontrol.wait.  The dependent launch is released after the prologue.  Returns false after a bounded wait ran out (status word raised).
+template <int PARTS, bool SW, bool MX>
+__device__ __forceinline__ bool stream_consume(const StreamParams& p, const int bx, const int gx, StreamShared& sh, const uint8_t* stages,
+                                               uint32_t* xq_s, const bool dep_resolved) {
   constexpr int ROWS = kGroupWarps / PARTS * kRPW;     // weight rows per tile
   constexpr int OUT_ROWS = SW ? ROWS / 2 : ROWS;       // output rows per tile
   const int K = p.K, nblk = K / 32;
   const int row_codes = K / 2, row_scales = K / 16;
+  const int stage_bytes = ROWS * (row_codes + row_scales);
   const int n_it = stream_n_it(p, bx, gx);
-  const int first = bx;
-  const int tid = threadIdx.x;                // 0..511
+  const int n_stages = p.n_stages;
+  const long long limit = p.wait_limit ? p.wait_limit : kWaitLimitCycles;
+  const int tid = threadIdx.x;  // 0..511
   const int lane = tid & 31, warp = tid >> 5;
   const int grp = warp / kGroupWarps;         // which of the two tile streams
   const int wg = warp % kGroupWarps;          // warp within the group
   const int tg = tid % (kGroupWarps * 32);    // thread within the group
-  // The norm gains are parameters, not products of the preceding kernel: fetch them before waiting for it.  (Every CTA
-  // reads the same few kilobytes, and such a broadcast read takes far longer than an ordinary L2 hit.)
-  uint4 graw = make_uint4(0, 0, 0, 0);
-  if (p.gain && tid * 8 < K) graw = __ldg(reinterpret_cast<const uint4*>(p.gain + tid * 8));
-  wait_dep();  // the activation comes from the preceding kernel or phase
   const int part = wg % PARTS, rsub = wg / PARTS;
   const int pblk = (nblk + PARTS - 1) / PARTS;
   const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
   uint32_t xr[kJ][16];
   float xm[kJ], xc[kJ];
+  ATS_TR(0);
   {
     // Thread t owns the runs of 8 consecutive elements r = t + 512 j (one run when K <= 4096, up to four for K = 16384);
     // four adjacent lanes hold one 32-element block.  The optional RMSNorm (h = rn16(x * g / sqrt(mean(x^2) + eps)),
     // K <= 4096) and the block quantization work on those registers; the quantized blocks go to shared memory once
-    // per CTA (28 words per block; the 112-byte pitch keeps the 128-bit reads conflict-free) and every lane then
-    // fetches the blocks of its k-part.
-    uint32_t* xq_s = ring.xq;
-    auto load_run = [&](const __half* src16, const float* src32, int i0, float (&xv)[8]) {
-      if (src32) {
-        const float4 a = *reinterpret_cast<const float4*>(src32 + i0);
-        const float4 b = *reinterpret_cast<const float4*>(src32 + i0 + 4);
-        xv[0] = a.x; xv[1] = a.y; xv[2] = a.z; xv[3] = a.w;
-        xv[4] = b.x; xv[5] = b.y; xv[6] = b.z; xv[7] = b.w;
-      } else {
-        const uint4 a = *reinterpret_cast<const uint4*>(src16 + i0);
-        const uint32_t w4[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          __half2 h2;
-          *reinterpret_cast<uint32_t*>(&h2) = w4[q];
-          const float2 f = __half22float2(h2);
-          xv[2 * q] = f.x;
-          xv[2 * q + 1] = f.y;
-        }
-      }
-    };
+    // per CTA and every lane then fetches the blocks of its k-part.
     if (p.gain) {
-      // norm prologue: K <= 4096, one run per thread
+      // The norm gains are parameters, not products of the preceding kernel: fetch them before waiting for it.
       const int i0 = tid * 8;
       const bool has = i0 < K;
+      const uint4 graw = has ? __ldg(reinterpret_cast<const uint4*>(p.gain + i0)) : make_uint4(0, 0, 0, 0);
+      if (!dep_resolved) asm volatile("griddepcontrol.wait;" ::: "memory");
       float xv[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) xv[q] = 0.f;
-      float ss = 0.f;
-      if (has) load_run(p.norm_in16, p.norm_in32, i0, xv);
+      if (has) {
+        if (p.norm_in32) {
+          const float4 a = *reinterpret_cast<const float4*>(p.norm_in32 + i0);
+          const float4 b = *reinterpret_cast<const float4*>(p.norm_in32 + i0 + 4);
+          xv[0] = a.x; xv[1] = a.y; xv[2] = a.z; xv[3] = a.w;
+          xv[4] = b.x; xv[5] = b.y; xv[6] = b.z; xv[7] = b.w;
+        } else {
+          unpack_h8(*reinterpret_cast<const uint4*>(p.norm_in16 + i0), xv);
+        }
+      }
+      ATS_TR(1);
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.xbar);
-      if (has) {
+      float ss = 0.f;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) ss = fmaf(xv[q], xv[q], ss);
-      }
+      for (int q = 0; q < 8; ++q) ss = fmaf(xv[q], xv[q], ss);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
       if (lane == 0) sh.red_s[warp] = ss;
@@ -397,32 +444,27 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
         quantize_run4<MX>(xv, tid & 3, xq_s + (size_t)(tid >> 2) * kXqWords);
       }
     } else {
+      if (!dep_resolved) asm volatile("griddepcontrol.wait;" ::: "memory");
       uint4 raw[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const int r = tid + 512 * j;  // run index; block r / 4, word r % 4.  All four lanes of a group are in range together.
+        const int r = tid + kConsumerThreads * j;  // run index; block r / 4, word r % 4.  All four lanes of a block are in range together.
         if (r * 8 < K) raw[j] = *reinterpret_cast<const uint4*>(p.x16 + r * 8);
       }
+      ATS_TR(1);
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.xbar);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const int r = tid + 512 * j;
+        const int r = tid + kConsumerThreads * j;
         if (r * 8 < K) {
           float xv[8];
-          const uint32_t w4[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            __half2 h2;
-            *reinterpret_cast<uint32_t*>(&h2) = w4[q];
-            const float2 f = __half22float2(h2);
-            xv[2 * q] = f.x;
-            xv[2 * q + 1] = f.y;
-          }
+          unpack_h8(raw[j], xv);
           quantize_run4<MX>(xv, r & 3, xq_s + (size_t)(r >> 2) * kXqWords);
         }
       }
     }
+    ATS_TR(2);
     consumer_sync_all();
 #pragma unroll
     for (int j = 0; j < kJ; ++j) {
@@ -448,14 +490,15 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
       }
     }
   }
+  ATS_TR(3);
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  if (release_dependents) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // this group's tiles: it = grp, grp + 2, ...; li counts them.  The cross-lane reduction of a tile's row sums is
   // deferred into the next tile's iteration, where its shuffle latencies hide behind that tile's integer work.
-  const int it_first = (grp + kGroups - ring.it0 % kGroups) % kGroups;  // tiles go to the groups by global index
-  const int n_li = n_it > it_first ? (n_it - it_first + kGroups - 1) / kGroups : 0;
+  const int n_li = n_it > grp ? (n_it - grp + kGroups - 1) / kGroups : 0;
   float* my_part = sh.part_s[grp];
   bool failed = false;
+  int s = grp % n_stages, cyc = grp / n_stages;  // stage and ring cycle of the group's next tile
   auto reduce_store = [&](float (&a)[kRPW], int slot) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1)
@@ -471,13 +514,14 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
     float prev[kRPW];
     bool have_prev = false;
     for (int li = li0; li < li1; ++li) {
-      const int git = ring.it0 + it_first + kGroups * li;
-      const int s = git % ring.n_stages;
-      if (!__all_sync(0xffffffffu, mbar_wait(&sh.full[s], (git / ring.n_stages) & 1))) {
+      const int it = grp + kGroups * li;
+      if (!__all_sync(0xffffffffu, mbar_wait_suspending(&sh.full[s], cyc & 1, limit))) {
         failed = true;
         break;
       }
-      const uint8_t* st = ring.stages + (size_t)s * ring.pitch;
+      if (li == 0) ATS_TR(4);
+      ATS_TR(100 + it);
+      const uint8_t* st = stages + (size_t)s * stage_bytes;
       uint4 cw[kRPW][kJ];
       float sc[kRPW][kJ];
 #pragma unroll
@@ -524,23 +568,26 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
         }
       }
       __syncwarp();
+      ATS_TR(200 + it);
       if (lane == 0) mbar_arrive(&sh.empty[s]);  // this warp is done reading stage s
+      stream_advance(s, cyc, kGroups, n_stages);
 #pragma unroll
       for (int r = 0; r < kRPW; ++r) prev[r] = acc[r];
       have_prev = true;
     }
     if (have_prev && !failed) reduce_store(prev, li1 - 1 - li0);
+    ATS_TR(5);
     if (failed) sh.fail_g[grp] = 1;
     group_sync(grp);
     if (sh.fail_g[grp]) {  // a warp of this group gave up; every thread of the group reads the same flag and leaves here
-      if (tg == 0) atomicExch(p.status, 1);
+      if (tg == 0) raise_status(p.status, 1);
       return false;
     }
     // flush: sum the k-parts (ascending) and run the epilogue
     const int n_out = (li1 - li0) * OUT_ROWS;
     for (int i = tg; i < n_out; i += kGroupWarps * 32) {
       const int itl = i / OUT_ROWS, j = i % OUT_ROWS;
-      const int tile = first + (it_first + kGroups * (li0 + itl)) * gx;
+      const int tile = bx + (grp + kGroups * (li0 + itl)) * gx;
       float v[2];
 #pragma unroll
       for (int h = 0; h < (SW ? 2 : 1); ++h) {
@@ -570,10 +617,12 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
     }
     group_sync(grp);
   }
+  ATS_TR(6);
+  ATS_TR_FLUSH();
   return true;
 }
 
-// ------------------------------------------------------------------ host side: shapes the phase takes, its parameters
+// ------------------------------------------------------------------ host side: shapes the kernel takes, its parameters
 inline int stream_parts_for(int K) { return K <= 2048 ? 1 : K <= 4096 ? 2 : K <= 8192 ? 4 : 8; }
 
 inline bool stream_shape_ok(const GemvParams& p) {
@@ -590,9 +639,13 @@ inline bool stream_shape_ok(const GemvParams& p) {
   return true;
 }
 
-// Bytes of one ring stage and of the quantized activation row for a phase of this shape.
+// Bytes of one ring stage and of the quantized activation row, and the number of stages that fit the SM.
 inline size_t stream_stage_bytes(int K) { return (size_t)(kGroupWarps / stream_parts_for(K) * kRPW) * (K / 2 + K / 16); }
 inline size_t stream_xq_bytes(int K) { return (size_t)(K / 32) * (kXqWords * 4); }
+inline int stream_n_stages(int K) {
+  const size_t n = ((size_t)kMaxDynSmem - stream_xq_bytes(K)) / stream_stage_bytes(K);
+  return (int)std::min<size_t>(n, kMaxStages);
+}
 
 inline StreamParams stream_params_from(const GemvParams& g, int* status) {
   const int rows = kGroupWarps / stream_parts_for(g.K) * kRPW;
@@ -613,6 +666,7 @@ inline StreamParams stream_params_from(const GemvParams& g, int* status) {
   p.n_tiles = tiles;
   p.K = g.K;
   p.mode = g.mode;
+  p.n_stages = stream_n_stages(g.K);
   p.x16 = g.x;
   p.norm_in16 = g.norm_x16;
   p.norm_in32 = g.norm_x32;
@@ -624,6 +678,8 @@ inline StreamParams stream_params_from(const GemvParams& g, int* status) {
   p.res32 = g.res32;
   p.res16 = g.res16;
   p.status = status;
+  p.wait_limit = 0;
+  p.withhold_tile = -1;
   return p;
 }
 

@@ -7,6 +7,7 @@
 // once: y += scale * sum.  No tensor cores, no atomics; reductions run in a fixed order so results are reproducible
 // run to run and independent of where the weight bytes live (resident region or staging slot).
 #include "ats_internal.h"
+#include "sm100_sync.cuh"
 #include "attn_decode_body.cuh"
 
 namespace ats {
@@ -119,7 +120,7 @@ __global__ void embed_rows_kernel(const uint8_t* __restrict__ slice, int n_rows,
       o.z = *reinterpret_cast<uint32_t*>(&r2);
       o.w = *reinterpret_cast<uint32_t*>(&r3);
     } else if (w == 0) {
-      atomicExch(status, 6);
+      raise_status(status, 6);
     }
     reinterpret_cast<uint4*>(out)[i] = o;
   }
@@ -530,7 +531,11 @@ __global__ void __launch_bounds__(kGemvMaxWarps * 32)
     xrow = jobs.xrow[job];
     out_row = jobs.orow[job];
   } else {
-    const int e = p.ids[job];
+    int e = p.ids[job];
+    if ((unsigned)e >= (unsigned)p.n_experts) {  // an id that names no expert: expert 0 stands in and the status word says so
+      if (threadIdx.x == 0 && blockIdx.x == 0) raise_status(p.status, 7);
+      e = 0;
+    }
     b0 = p.base0 + (size_t)e * p.stride;
     b1 = SW ? p.base1 + (size_t)e * p.stride : nullptr;
     xrow = job / p.x_div;
@@ -755,9 +760,11 @@ cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __ha
 // memory (16-byte async copies, issued before the grid dependency resolves) and every head's warps read them from
 // there, so the cache crosses the L2-to-SM fabric once instead of once per query head; that traffic, not DRAM, bounds
 // this kernel.  Warp (head, sub-block) owns 32 positions, one per lane.
-// Positions per CTA: 64, or 128 for contexts beyond 1024 so that the final merge still reads all splits of a head in
-// one round trip (16 splits) up to 2048 positions.
-int attn_decode_pos_per_cta(int n_ctx) { return n_ctx <= 1024 ? 64 : 128; }
+// Positions per CTA: 64 up to 2048 positions of context (a CTA of 256 threads and 46 KB of shared memory for a group of
+// four heads of 128: small enough to sit on an SM beside a CTA of the streaming GEMV, so that this kernel's cache rows are
+// staged while the QKV projection still runs and the O projection's weights while this kernel runs), 128 beyond that
+// (fewer partials for the final merge, which reads 16 splits per round trip).
+int attn_decode_pos_per_cta(int n_ctx) { return n_ctx <= 2048 ? 64 : 128; }
 int attn_decode_splits(int n_ctx) {
   const int pc = attn_decode_pos_per_cta(n_ctx);
   return (n_ctx + pc - 1) / pc;
@@ -767,7 +774,7 @@ size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) {
 }
 
 template <int D, int SUB>
-__global__ void __launch_bounds__(512) attn_decode_fused_kernel(const AttnDecodeParams p) {
+__global__ void __maxnreg__(72) attn_decode_fused_kernel(const AttnDecodeParams p) {
   extern __shared__ __align__(16) uint8_t dyn_s[];
   attn_decode_body<D, SUB, true>(p, (int)blockIdx.x, (int)blockIdx.y, (int)gridDim.x, (int)threadIdx.x, (int)blockDim.x, dyn_s);
 }
@@ -818,6 +825,14 @@ __device__ __forceinline__ void router_select(const float* logit, int m, int E, 
   float sel_v = 0.f;  // lane j (< k) keeps the j-th selected logit
   int sel_i = 0;
   float total = 0.f, top = 0.f;
+  // A NaN logit (a NaN activation or weight) compares false with everything: it takes part in the selection as -inf so
+  // that the ids always lie in [0, E) (they index weight slices downstream), and every gate of the token becomes NaN.
+  bool has_nan = false;
+  for (int j = 0; j < per; ++j) {
+    const float v = logit[lane + 32 * j];
+    has_nan |= (lane + 32 * j < E) && (v != v);
+  }
+  has_nan = __any_sync(0xffffffffu, has_nan);
   if (!renorm) {
     float mx = -INFINITY;
     for (int j = 0; j < per; ++j) mx = fmaxf(mx, logit[lane + 32 * j]);
@@ -835,7 +850,8 @@ __device__ __forceinline__ void router_select(const float* logit, int m, int E, 
     int bi = 0x7fffffff;
     for (int j = 0; j < per; ++j) {
       if (taken & (1u << j)) continue;
-      const float v = logit[lane + 32 * j];
+      const float vr = logit[lane + 32 * j];
+      const float v = vr == vr ? vr : -INFINITY;
       const int idx = lane + 32 * j;
       if (idx < E && (v > bv || (v == bv && idx < bi))) {
         bv = v;
@@ -866,6 +882,7 @@ __device__ __forceinline__ void router_select(const float* logit, int m, int E, 
   } else {
     gate = lane < k ? expf(sel_v - top) / total : 0.f;
   }
+  if (has_nan) gate = __int_as_float(0x7FC00000);
   if (lane < k) {
     ids[(size_t)m * k + lane] = sel_i;
     gates[(size_t)m * k + lane] = gate;
@@ -1073,6 +1090,31 @@ cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gat
   if (res_is_f32)
     return launch_dep(moe_combine_kernel<float>, grid, dim3(256), 0, st, pdl, 1, (const float*)res, gates, d32, y16, k, H);
   return launch_dep(moe_combine_kernel<__half>, grid, dim3(256), 0, st, pdl, 1, (const __half*)res, gates, d32, y16, k, H);
+}
+
+// ---------------------------------------------------------------- host-driven calls: input staging and completion word
+// A few kilobytes of activations fetched from mapped pinned host memory by the SMs (16-byte loads over PCIe) into the
+// workspace: for rows this small a kernel is quicker than a copy-engine transfer and the engine hand-over around it.
+__global__ void stage_rows_kernel(const uint4* __restrict__ src_host, uint4* __restrict__ dst, int n16) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += gridDim.x * blockDim.x) dst[i] = src_host[i];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+cudaError_t launch_stage_rows(const void* src_host_alias, void* dst, uint64_t bytes, cudaStream_t st, uint64_t* n_launch) {
+  const int n16 = (int)(bytes / 16);
+  const int grid = std::max(1, std::min((n16 + 255) / 256, 8));
+  ++*n_launch;
+  return launch_dep(stage_rows_kernel, dim3(grid), dim3(256), 0, st, 0, 1, (const uint4*)src_host_alias, (uint4*)dst, n16);
+}
+// Completion word of a host-driven call: written (to mapped pinned host memory) once everything before it in the stream
+// has completed and its writes are visible, so the host can poll the word instead of synchronising with the stream.
+__global__ void signal_done_kernel(int* done, int seq) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  *reinterpret_cast<volatile int*>(done) = seq;
+  __threadfence_system();
+}
+cudaError_t launch_signal_done(int* done_alias, int seq, int pdl, cudaStream_t st, uint64_t* n_launch) {
+  ++*n_launch;
+  return launch_dep(signal_done_kernel, dim3(1), dim3(1), 0, st, pdl, 1, done_alias, seq);
 }
 
 cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uint64_t* n_launch) {

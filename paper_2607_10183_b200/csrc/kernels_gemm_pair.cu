@@ -17,6 +17,7 @@
 #include <cuda.h>
 
 #include "ats_internal.h"
+#include "sm100_sync.cuh"
 
 namespace ats {
 
@@ -39,32 +40,6 @@ struct PairParams {
   int* status;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// bounded spin (about a second of SM clocks)
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  if (mbar_test_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_test_wait(bar, parity)) return true;
-    if (clock64() - t0 > 2000000000ll) return false;
-  }
-}
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -252,7 +227,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       failed = true;
     }
   }
-  if (failed && p.status) atomicExch(p.status, 2);
+  if (failed && p.status) raise_status(p.status, 2);
   // nobody leaves, frees tensor memory or lets its shared memory go while the partner may still read or signal it
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   cluster_sync_all();
@@ -570,7 +545,7 @@ __global__ void __launch_bounds__(kQThreads, 1) gemm_q4_pair_kernel(const __grid
       failed = true;
     }
   }
-  if (failed && p.status) atomicExch(p.status, 2);
+  if (failed && p.status) raise_status(p.status, 2);
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   cluster_sync_all();
   if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");

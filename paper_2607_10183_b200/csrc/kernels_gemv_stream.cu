@@ -6,25 +6,30 @@ namespace ats {
 
 namespace {
 
-// A whole kernel as one phase: the ring starts empty, the grid dependency is resolved by griddepcontrol.
+// Registers per thread: capped so that the decode attention kernel's CTAs (256 threads of up to 72 registers, 46 KB of
+// shared memory) fit an SM beside a CTA of this kernel.  They are launched as this kernel's dependents and stage their
+// cache rows while it streams, and the CTAs of the GEMV after them move in beside them in turn.
+constexpr int kStreamMaxRegs = 80;
+
+// One CTA: ring set-up, then the producer warp and the consumer warps go their ways.  dep_resolved: the caller has already
+// waited for the preceding kernel (its weight addresses come from that kernel's output).
 template <int PARTS, bool SW, bool MX>
-__device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool wait_first) {
+__device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool dep_resolved) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ StreamShared sh;
   constexpr int ROWS = kGroupWarps / PARTS * kRPW;
   const int stage_bytes = ROWS * (p.K / 2 + p.K / 16);
-  stream_init(sh);
-  const StreamRing ring{smem, stage_bytes, kStages, reinterpret_cast<uint32_t*>(smem + (size_t)kStages * stage_bytes), 0, 0};
-  if ((threadIdx.x >> 5) == kConsumerWarps) {
+  stream_init(sh, p.n_stages);
+  if ((threadIdx.x >> 5) >= kConsumerWarps) {
     // weights do not depend on the preceding kernel, so their copies start before the grid dependency is resolved
-    if ((threadIdx.x & 31) == 0) stream_produce<PARTS, SW, true>(p, bx, gx, wait_first, sh, ring, l2_evict_first_policy());
+    if ((threadIdx.x & 31) == 0) stream_produce<PARTS, SW>(p, bx, gx, (int)(threadIdx.x >> 5) - kConsumerWarps, sh, smem, l2_evict_first_policy());
     return;
   }
-  stream_consume<PARTS, SW, MX>(p, bx, gx, sh, ring, [] { asm volatile("griddepcontrol.wait;" ::: "memory"); }, true);
+  stream_consume<PARTS, SW, MX>(p, bx, gx, sh, smem, reinterpret_cast<uint32_t*>(smem + (size_t)p.n_stages * stage_bytes), dep_resolved);
 }
 
 template <int PARTS, bool SW, bool MX>
-__global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamParams p) {
+__global__ void __maxnreg__(kStreamMaxRegs) gemv_stream_kernel(const StreamParams p) {
   gemv_stream_body<PARTS, SW, MX>(p, (int)blockIdx.x, (int)gridDim.x, false);
 }
 
@@ -40,15 +45,20 @@ struct MoeSel {
   const uint8_t* const* tab1;
   int x_div;
   int ldx, ldy;
+  int n_experts;
 };
 template <int PARTS, bool SW, bool MX>
-__global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
+__global__ void __maxnreg__(kStreamMaxRegs) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
   StreamParams p = p0;
   const int job = blockIdx.y;
   int xrow, orow;
   if (m.ids) {
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // the ids come from the router kernel
-    const size_t e = (size_t)m.ids[job];
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the ids come from the router kernel (every thread waits: the consumers skip their own wait)
+    size_t e = (size_t)(unsigned)m.ids[job];
+    if (e >= (size_t)m.n_experts) {  // an id that names no expert: expert 0 stands in and the status word says so
+      if (threadIdx.x == 0 && blockIdx.x == 0) raise_status(p0.status, 7);
+      e = 0;
+    }
     p.seg[0].base = m.tab0 ? m.tab0[e] : m.base0 + e * m.stride;
     if (SW) p.seg[1].base = m.tab1 ? m.tab1[e] : m.base1 + e * m.stride;
     xrow = job / m.x_div;
@@ -67,6 +77,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const Stre
 
 int parts_for(int K) { return stream_parts_for(K); }
 
+// The kernels take nearly all of an SM's shared memory for the ring.
+cudaError_t set_stream_kernel_attributes(const void* kern) {
+  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+}
+
 }  // namespace
 
 bool gemv_stream_eligible(const GemvParams& p) { return !p.w16 && stream_shape_ok(p); }  // the two 4-bit formats
@@ -74,10 +89,12 @@ bool gemv_stream_eligible(const GemvParams& p) { return !p.w16 && stream_shape_o
 cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, cudaStream_t st, uint64_t* n_launch) {
   const int parts = parts_for(g.K);
   const bool sw = g.mode == GEMV_SWIGLU_F16;
-  const StreamParams p = stream_params_from(g, status);
+  StreamParams p = stream_params_from(g, status);
+  p.wait_limit = g.dbg_wait_limit;
+  p.withhold_tile = g.dbg_withhold_tile_plus1 - 1;
   const int tiles = p.n_tiles;
   const size_t stage_bytes = stream_stage_bytes(g.K);
-  const size_t smem = kStages * stage_bytes + stream_xq_bytes(g.K);
+  const size_t smem = p.n_stages * stage_bytes + stream_xq_bytes(g.K);
   const int grid = std::max(1, std::min(tiles, sm_count));
   void (*kern)(const StreamParams) = nullptr;
   if (g.mx) {
@@ -98,10 +115,10 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   static uint64_t attr_done[16] = {};
   const int ki = ((parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+    cudaError_t e = set_stream_kernel_attributes(reinterpret_cast<const void*>(kern));
     if (e != cudaSuccess) return e;
   }
-  if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
+  if (smem > kMaxDynSmem || p.n_stages < kProducerWarps) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreads);
@@ -137,10 +154,12 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   p.n_tiles = sw ? g.n_rows / (rows / 2) : g.n_rows / rows;
   p.K = g.K;
   p.mode = g.mode;
+  p.n_stages = stream_n_stages(g.K);
   p.x16 = g.x;
   p.y32 = g.y32;
   p.y16 = g.y16;
   p.status = status;
+  p.withhold_tile = -1;
   MoeSel m{};
   m.base0 = g.base0;
   m.base1 = g.base1;
@@ -151,11 +170,11 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   m.x_div = g.x_div;
   m.ldx = g.ldx;
   m.ldy = g.ldy;
+  m.n_experts = g.n_experts;
   MoeJobs none;
   none.n = 0;
-  const size_t stage_bytes = (size_t)rows * (g.K / 2 + g.K / 16);
-  const size_t smem = kStages * stage_bytes + (size_t)(g.K / 32) * (kXqWords * 4);
-  if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
+  const size_t smem = p.n_stages * stream_stage_bytes(g.K) + stream_xq_bytes(g.K);
+  if (smem > kMaxDynSmem || p.n_stages < kProducerWarps) return cudaErrorInvalidValue;
   const int per_job = std::max(1, std::min(p.n_tiles, sm_count / n_jobs));  // one wave: a CTA fills its SM
   void (*kern)(const StreamParams, const MoeSel, const MoeJobs) = nullptr;
   if (g.mx) {
@@ -176,7 +195,7 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   static uint64_t attr_done[16] = {};
   const int ki = ((parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+    cudaError_t e = set_stream_kernel_attributes(reinterpret_cast<const void*>(kern));
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg{};
@@ -193,4 +212,68 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   return cudaLaunchKernelEx(&cfg, kern, p, m, jobs ? *jobs : none);
 }
 
+// ------------------------------------------------------------------------------------------ read-only HBM probe
+// What this GPU delivers to a kernel that only reads, with the access pattern of the streaming GEMV (bulk-async copies of
+// 16 KB into shared memory, four issuing warps per SM, nothing done with the data): the third denominator next to the
+// nominal figure and the measured copy bandwidth (a copy also writes, and reaches less).
+namespace {
+constexpr int kProbeWarps = 4, kProbeDepth = 2, kProbeChunk = 16 * 1024;
+__global__ void __launch_bounds__(kProbeWarps * 32) hbm_read_probe_kernel(const uint8_t* __restrict__ src, unsigned long long n_chunks,
+                                                                          int* status) {
+  extern __shared__ __align__(128) uint8_t probe_s[];
+  __shared__ uint64_t bar[kProbeWarps * kProbeDepth];
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) != 0) return;
+  uint64_t* mybar = bar + warp * kProbeDepth;
+  uint8_t* mysm = probe_s + (size_t)warp * kProbeDepth * kProbeChunk;
+  for (int s = 0; s < kProbeDepth; ++s) mbar_init(&mybar[s], 1);
+  mbar_fence_init();
+  const unsigned long long issuers = (unsigned long long)gridDim.x * kProbeWarps;
+  const unsigned long long first = (unsigned long long)blockIdx.x * kProbeWarps + warp;
+  const long long per = (long long)((n_chunks + issuers - 1) / issuers);
+  const uint64_t pol = l2_evict_first_policy();
+  for (long long it = 0; it < per + kProbeDepth; ++it) {
+    const int s = (int)(it % kProbeDepth);
+    if (it >= kProbeDepth && !mbar_wait(&mybar[s], (uint32_t)(((it / kProbeDepth) - 1) & 1))) {
+      raise_status(status, 8);
+      return;
+    }
+    if (it < per) {
+      const unsigned long long chunk = first + (unsigned long long)it * issuers;
+      if (chunk < n_chunks) {
+        mbar_expect_tx(&mybar[s], kProbeChunk);
+        bulk_g2s(mysm + (size_t)s * kProbeChunk, src + chunk * kProbeChunk, kProbeChunk, &mybar[s], pol);
+      } else {
+        mbar_arrive(&mybar[s]);
+      }
+    }
+  }
+}
+}  // namespace
+
+cudaError_t launch_hbm_read_probe(const uint8_t* src, uint64_t bytes, int* status, int sm_count, cudaStream_t st) {
+  const size_t smem = (size_t)kProbeWarps * kProbeDepth * kProbeChunk;
+  static uint64_t attr_done = 0;
+  if (first_use_on_device(&attr_done)) {
+    cudaError_t e = cudaFuncSetAttribute(hbm_read_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  hbm_read_probe_kernel<<<sm_count, kProbeWarps * 32, smem, st>>>(src, bytes / kProbeChunk, status);
+  return cudaGetLastError();
+}
+
 }  // namespace ats
+
+#ifdef ATS_TRACE
+// Development builds only: read and clear the timeline probe (see gemv_stream_body.cuh).
+extern "C" int ats_trace_read(void* out_host, int cap_records) {
+  unsigned int n = 0;
+  if (cudaMemcpyFromSymbol(&n, ats::g_trace_n, sizeof n) != cudaSuccess) return -1;
+  if (n > (unsigned)ats::kTraceCap) n = ats::kTraceCap;
+  if ((int)n > cap_records) n = cap_records;
+  if (n && cudaMemcpyFromSymbol(out_host, ats::g_trace, (size_t)n * sizeof(ats::TraceRec)) != cudaSuccess) return -1;
+  unsigned int zero = 0;
+  cudaMemcpyToSymbol(ats::g_trace_n, &zero, sizeof zero);
+  return (int)n;
+}
+#endif

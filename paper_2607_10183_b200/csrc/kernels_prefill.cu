@@ -2,6 +2,7 @@
 // over the cache (tensor cores), fp16 residual add and SwiGLU.  Every intermediate of the prefill path is stored as fp16 (the
 // operands of the tensor-core GEMMs), so these kernels read and write fp16 and compute in fp32.
 #include "ats_internal.h"
+#include "sm100_sync.cuh"
 
 namespace ats {
 
@@ -400,26 +401,13 @@ cudaError_t launch_moe_combine_sorted(const __half* res, const float* gates, con
 namespace {
 constexpr int kCopyStages = 4;
 constexpr int kCopyChunk = 32 * 1024;
-__device__ __forceinline__ uint32_t cp_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ bool cp_mbar_wait(uint64_t* bar, uint32_t parity) {
-  const long long t0 = clock64();
-  for (;;) {
-    for (int i = 0; i < 64; ++i) {
-      uint32_t ok;
-      asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                   : "=r"(ok) : "r"(cp_smem_u32(bar)), "r"(parity) : "memory");
-      if (ok) return true;
-    }
-    if (clock64() - t0 > 4000000000ll) return false;  // about two seconds: the source is across PCIe
-  }
-}
 }  // namespace
 
 __global__ void __launch_bounds__(32, 1) host_gather_kernel(const CopyChunk* __restrict__ list, int n, int* status) {
   extern __shared__ __align__(128) uint8_t cp_s[];
   __shared__ uint64_t full[kCopyStages];
   if (threadIdx.x != 0) return;
-  for (int s = 0; s < kCopyStages; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(cp_smem_u32(&full[s])));
+  for (int s = 0; s < kCopyStages; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&full[s])));
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the list was written by a copy that precedes this launch
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -428,21 +416,21 @@ __global__ void __launch_bounds__(32, 1) host_gather_kernel(const CopyChunk* __r
   auto issue_load = [&](int j) {
     const int s = j % kCopyStages;
     const CopyChunk c = list[first + j * gx];
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(cp_smem_u32(&full[s])), "r"(c.bytes) : "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&full[s])), "r"(c.bytes) : "memory");
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     cp_smem_u32(cp_s + (size_t)s * kCopyChunk)),
-                 "l"(c.src), "r"(c.bytes), "r"(cp_smem_u32(&full[s]))
+                     smem_u32(cp_s + (size_t)s * kCopyChunk)),
+                 "l"(c.src), "r"(c.bytes), "r"(smem_u32(&full[s]))
                  : "memory");
   };
   for (int j = 0; j < min(kCopyStages, n_my); ++j) issue_load(j);
   for (int j = 0; j < n_my; ++j) {
     const int s = j % kCopyStages;
-    if (!cp_mbar_wait(&full[s], (uint32_t)(j / kCopyStages) & 1u)) {
-      atomicExch(status, 5);
+    if (!mbar_wait_suspending(&full[s], (uint32_t)(j / kCopyStages) & 1u, 2 * kWaitLimitCycles)  /* about two seconds: the source is across PCIe */) {
+      raise_status(status, 5);
       break;
     }
     const CopyChunk c = list[first + j * gx];
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(c.dst), "r"(cp_smem_u32(cp_s + (size_t)s * kCopyChunk)),
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(c.dst), "r"(smem_u32(cp_s + (size_t)s * kCopyChunk)),
                  "r"(c.bytes)
                  : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");

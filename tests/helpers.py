@@ -9,11 +9,12 @@ TOL = 2e-3  # max relative error of fp outputs (fp32 accumulation vs the fp64 or
 def assert_close(y, ref, tol=TOL, what="", elementwise=True):
     """Max relative error per output row, measured two ways: normwise max|y-r| / max|r| <= tol (always), and mixed
     elementwise |y-r| <= tol (|r| + rms(r)) (a pure elementwise relative error is meaningless next to the zero crossings
-    of a dot product).  Single operators are held to both.  The end-to-end output of a whole layer whose every
-    intermediate is stored as fp16 is held to the normwise gate only: a one-ulp difference in the rounding of an
-    intermediate (fp32 accumulation and fp64 land on different sides of a rounding boundary for ~1 % of the elements)
-    is propagated by eleven rounded stages, and the maximum of the elementwise ratio over two million outputs is a tail
-    statistic of those flips, not a property of any kernel; the stage-wise tests hold every kernel to both gates."""
+    of a dot product).  Single operators and every stage of a layer are held to both (elementwise=True).  The end-to-end
+    output of a full-size prefill layer (eleven fp16-rounded stages, two million outputs) is held to the normwise gate and
+    to the mixed gate with its violations counted and bounded (elementwise="counted"): a one-ulp difference in the
+    rounding of an intermediate (fp32 accumulation and fp64 land on different sides of a rounding boundary for ~1 % of the
+    elements) propagates through the later stages, and the maximum of the ratio over millions of outputs is a tail
+    statistic of those flips; the stage-wise tests hold every kernel to both gates on the inputs it consumed."""
     y = np.asarray(y, dtype=np.float64).reshape(-1, np.asarray(y).shape[-1])
     r = np.asarray(ref, dtype=np.float64).reshape(y.shape)
     assert np.all(np.isfinite(y)), f"{what}: non-finite output"
@@ -22,7 +23,15 @@ def assert_close(y, ref, tol=TOL, what="", elementwise=True):
     assert norm.max() <= tol, f"{what}: normwise error {norm.max():.3e} > {tol}"
     rms = np.sqrt(np.mean(r * r, axis=1, keepdims=True))
     ratio = err / (tol * (np.abs(r) + rms) + 1e-300)
-    if elementwise:
+    if elementwise == "counted":
+        # End-to-end output of a layer whose every intermediate is stored as fp16: the mixed gate still holds for all but
+        # the few elements downstream of an intermediate that fp32 and fp64 arithmetic rounded to different fp16
+        # neighbours.  Those are counted and bounded instead of being let through: at most one element in a thousand may
+        # exceed the gate, and none by more than a factor of two.
+        over = ratio > 1.0
+        assert over.mean() <= 1e-3, f"{what}: {over.mean():.2e} of the elements exceed the mixed elementwise gate"
+        assert ratio.max() <= 2.0, f"{what}: mixed elementwise ratio {ratio.max():.3f} > 2"
+    elif elementwise:
         assert ratio.max() <= 1.0, f"{what}: mixed elementwise ratio {ratio.max():.3f} > 1"
     return float(norm.max()), float(ratio.max())
 

@@ -371,9 +371,12 @@ def test_linear_closed_forms_on_gpu(B, torch):
 
 
 # ------------------------------------------------------------------------------------------------- dense layer decode
-def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, flags=0, steps=1, chunk=MB, host_io=False):
+def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, flags=0, steps=1, chunk=MB, host_io=False,
+                     debug=None):
     """Returns (list of y per step, final K cache, final V cache, stats) for one layer.  host_io: drive the step through
-    ats_layer_decode_host from pinned host buffers instead of device buffers."""
+    ats_layer_decode_host from host buffers instead of device buffers ("registered": pinned buffers registered with the
+    library, True: pinned but unregistered, "pageable": ordinary memory).  debug: a dict that receives the last step's
+    normalised operand h (fp16) and the fp32 [q | k | v] projections as the library computed them."""
     L = W.dense_layer(cfg, 0, shape)
     slot = max(W.q4_bytes(n, k) for _, n, k in shape.tensor_shapes())
     ctx = make_ctx(B, H.dense_layer_bytes(shape) + 16 * 256 + 4 * shape.hidden * 2, ring_slots=ring_slots, slot_bytes=slot,
@@ -393,16 +396,25 @@ def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, fl
             ctx.layer_decode_host(desc, xh, yh, kd, vd, pos + s, 1)
             ys.append(yh.copy())
             continue
-        if host_io:  # pinned memory: the layer's last kernel writes the result into it directly
+        if host_io:  # pinned memory; registered: no copy engine, the layer's last kernel writes the result into it
             xh = torch.from_numpy(x).pin_memory()
             yh = torch.zeros((1, shape.hidden), dtype=torch.float16).pin_memory()
+            if host_io == "registered":
+                ctx.register_host_buffer(xh)
+                ctx.register_host_buffer(yh)
             ctx.layer_decode_host(desc, xh, yh, kd, vd, pos + s, 1)  # returns with yh valid: no sync here
             ys.append(yh.numpy().copy())
+            if host_io == "registered":
+                ctx.unregister_host_buffer(xh)
+                ctx.unregister_host_buffer(yh)
             continue
         y = torch.empty((1, shape.hidden), dtype=torch.float16, device="cuda")
         ctx.layer_decode(desc, H.to_dev(x), y, kd, vd, pos + s, 1)
         ctx.sync()
         ys.append(y.cpu().numpy())
+        if debug is not None:
+            debug["h"] = ctx.debug_decode_buffer(desc, 1, 0, np.float16).copy()
+            debug["qkv"] = ctx.debug_decode_buffer(desc, 1, 1, np.float32).copy()
     st = ctx.stats()
     out = (ys, kd.cpu().numpy(), vd.cpu().numpy(), st, ctx.numerics(B.ATS_MODE_DECODE))
     ctx.close()
@@ -410,6 +422,21 @@ def run_dense_decode(B, torch, shape, cfg, pos, cap, placement, ring_slots=2, fl
 
 
 ALL_GPU = {n: 1 for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")}
+
+
+def fixed_point_gemv_bound(h, w):
+    """Largest error the single-token GEMV may make on y = w h given ITS OWN operand h (fp16 values) and the exact weights
+    w [N][K]: every activation is rounded to the 16-bit fixed-point grid of its block of 32, whose step is 2^(E - 29) for
+    the fp16 exponent field E of the block's largest magnitude (so each activation moves by at most half a step), block dot
+    products are exact, and one fp32 multiply-add per block plus the fp32 scale product accumulate the blocks."""
+    h = np.asarray(h, dtype=np.float64).reshape(-1)
+    n, k = w.shape
+    m = np.abs(h.reshape(-1, 32)).max(axis=1)
+    e_field = np.maximum(np.floor(np.log2(np.maximum(m, 2.0 ** -24))) + 15, 1)
+    half_step = 2.0 ** (e_field - 30)
+    quant = np.abs(w).reshape(n, -1, 32).sum(axis=2) @ half_step
+    fp32 = (k // 32 + 3) * 2.0 ** -24 * (np.abs(w) @ np.abs(h))
+    return quant + fp32
 
 
 # positions around the attention kernel's tiling: 64 or 128 positions per CTA (contexts up to / beyond 1024), the final
@@ -420,21 +447,37 @@ ALL_GPU = {n: 1 for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")}
 def test_dense_layer_decode_matches_oracle(B, torch, shape_name, pos, cap):
     shape = W.DENSE_SMALL if shape_name == "small" else W.DENSE_FULL
     cfg = 96 if shape_name == "small" else 2
-    ys, kg, vg, st, (edges, wmode) = run_dense_decode(B, torch, shape, cfg, pos, cap, ALL_GPU)
+    dbg = {}
+    ys, kg, vg, st, (edges, wmode) = run_dense_decode(B, torch, shape, cfg, pos, cap, ALL_GPU, debug=dbg)
     L = W.dense_layer(cfg, 0, shape)
     kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos)
     x = W.activations(cfg, 0, (1, shape.hidden), step=0)
     want = O.dense_layer(x, H.oracle_dense_tensors(L), shape, kc, vc, pos, edges, wmode)
     H.assert_close(ys[0], want, what="decode layer output")
-    # cache rows written at `pos`: fp16 values within one ulp of the oracle's, everything else untouched
-    for got, ref in ((kg, kc), (vg, vc)):
+    # The projections and the cache rows, held to a bound derived from the inputs instead of a fitted constant: the exact
+    # product of the exact weights with the operand h the library itself formed (so that a flipped fp16 rounding of h
+    # does not enter), against the library's fp32 [q | k | v]; then the rows written at `pos`: the fp16 rounding of the
+    # rotated key / the value, so one fp16 ulp on top of the projection's bound (a rotation mixes two elements with
+    # |cos|, |sin| <= 1, and the fp32 rotation itself adds a relative 2^-22).  Everything else in the caches is untouched.
+    h_gpu = dbg["h"].astype(np.float64).reshape(-1)
+    qd, kvd, d = shape.n_q_heads * shape.head_dim, shape.n_kv_heads * shape.head_dim, shape.head_dim
+    qkv_gpu = dbg["qkv"].astype(np.float64).reshape(-1)
+    proj, bound = {}, {}
+    for name, role, lo, n in (("q", W.ROLE_Q, 0, qd), ("k", W.ROLE_K, qd, kvd), ("v", W.ROLE_V, qd + kvd, kvd)):
+        w = O.dequantize(*L[role])
+        proj[name], bound[name] = w @ h_gpu, fixed_point_gemv_bound(h_gpu, w)
+        err = np.abs(qkv_gpu[lo:lo + n] - proj[name])
+        assert np.all(err <= bound[name]), (name, float((err / bound[name]).max()))
+        # how tight the bound is on this data: errors of random sign stay well inside the worst case
+        assert err.max() <= 0.5 * bound[name].max()
+    k_rot = O.rope(proj["k"].reshape(shape.n_kv_heads, d), pos, shape.rope_theta)
+    bk = bound["k"].reshape(shape.n_kv_heads, d)
+    bk_rot = bk + np.roll(bk, d // 2, axis=1) + 2.0 ** -21 * np.abs(k_rot)
+    for got, ref, ref_new, b in ((kg, kc, k_rot, bk_rot), (vg, vc, proj["v"].reshape(shape.n_kv_heads, d), bound["v"].reshape(shape.n_kv_heads, d))):
         assert np.array_equal(np.delete(got, pos, axis=1), np.delete(ref, pos, axis=1))
-        a, b = got[:, pos].astype(np.float64), ref[:, pos].astype(np.float64)
-        # one fp16 ulp where the value is not tiny; near zero the absolute error of the projection bounds it: the
-        # activations enter the block dot products as 16-bit block fixed point (each rounded within 2^-17 of its block's
-        # maximum, about 1e-5 of the output's scale after the sum over k) and the blocks are accumulated in fp32
-        ulp = np.spacing(np.abs(ref[:, pos]).astype(np.float16)).astype(np.float64)
-        assert np.all(np.abs(a - b) <= ulp + 1e-4 * np.abs(b).max())
+        a = got[:, pos].astype(np.float64)
+        ulp = np.spacing(np.abs(ref_new).astype(np.float16)).astype(np.float64)
+        assert np.all(np.abs(a - ref_new) <= ulp + b)
     assert st.streamed_bytes == 0 and st.resident_bytes == H.dense_layer_bytes(shape)
 
 
@@ -479,7 +522,8 @@ def test_dense_layer_fp16_weights_decode_matches_oracle(B, torch, M):
             got_k = kd.cpu().numpy()
             assert np.array_equal(np.delete(got_k, pos, axis=1), np.delete(kc, pos, axis=1))
             a, b = got_k[:, pos].astype(np.float64), kc[:, pos].astype(np.float64)
-            assert np.all(np.abs(a - b) <= np.spacing(np.abs(kc[:, pos])).astype(np.float64) + 1e-4 * np.abs(b).max())
+            # fp16-weight GEMV: exact products summed in fp32, no fixed-point operand
+            assert np.all(np.abs(a - b) <= np.spacing(np.abs(kc[:, pos])).astype(np.float64) + 2e-5 * np.abs(b).max())
         ctx.close()
     assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
     # one quantized matrix among fp16 ones: a status, not a launch
@@ -502,7 +546,7 @@ def test_host_driven_decode_equals_device_driven(B, torch):
     shape, cfg, pos, cap = W.DENSE_SMALL, 96, 20, 40
     for placement in (ALL_GPU, {**ALL_GPU, "wk": 0, "w_up": 0, "w_down": 0}):
         dev = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, steps=3)
-        for mode in (True, "pageable"):
+        for mode in ("registered", True, "pageable"):
             host = run_dense_decode(B, torch, shape, cfg, pos, cap, placement, steps=3, host_io=mode)
             for a, b in zip(dev[0], host[0]):
                 assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
@@ -579,6 +623,9 @@ def test_stack_under_planned_budget_full_size(B, torch):
     res, _, st_res = run(None)
     hyb, where, st = run(0.60)
     assert 0 < int(where.sum()) < len(where)
+    budget = int(0.60 * n_layers * layer_bytes)
+    want_where = O.static_placement(O.size_units(nbytes * n_layers), nbytes * n_layers, [0] * (7 * n_layers), O.budget_units(budget))
+    assert list(where) == list(want_where)  # Algorithm 1 on the same records (value = byte size, no switch cost)
     for a, b in zip(res, hyb):
         assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
     assert st_res.streamed_bytes == 0
@@ -809,3 +856,120 @@ def test_errors_are_statuses_and_context_stays_usable(B, torch):
         ctx.set_placement([(tid, -1, 1)])
     assert e.value.code == B.ATS_ERR_BUDGET
     ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------- failure paths
+def test_gemv_non_finite_activation_gives_non_finite_output(B, torch):
+    """An Inf or a NaN among the activations must not turn into a finite output: the streaming kernel's fixed-point operand
+    cannot carry it, so the block's term becomes NaN (the plain definition gives Inf or NaN in every row here, since every
+    output sums over every k)."""
+    N, K = 64, 512
+    packed, scales = W.q4_packed(93, 0, W.ROLE_Q, N, K)
+    ctx = make_ctx(B, W.q4_bytes(N, K) + 512)
+    tid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(tid, -1, B.ATS_GPU)])
+    y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+    for bad_k, bad in ((5, np.inf), (300, -np.inf), (77, np.nan)):
+        x = W.activations(93, 0, (1, K))
+        x[0, bad_k] = bad
+        with np.errstate(invalid="ignore", over="ignore"):
+            want = O.linear(x, packed, scales)
+        assert not np.isfinite(want).any()
+        ctx.linear(tid, H.to_dev(x), y, 1)
+        ctx.sync()
+        assert not np.isfinite(y.cpu().numpy().astype(np.float32)).any(), (bad_k, bad)
+    # finite again afterwards
+    x = W.activations(93, 0, (1, K))
+    ctx.linear(tid, H.to_dev(x), y, 1)
+    ctx.sync()
+    H.assert_close(y.cpu().numpy(), O.linear(x, packed, scales), what="gemv after non-finite inputs")
+    ctx.close()
+
+
+def test_router_ids_stay_in_range_for_a_nan_row(B, torch):
+    """A row of NaN activations gives NaN logits, which compare false with everything: the ids must still name experts
+    (they index weight slices downstream) and the row's gates are NaN; the other rows are unaffected."""
+    rng = np.random.default_rng(12)
+    Hd, E, k, M = 128, 48, 6, 3
+    Wr = rng.normal(0, 0.02, size=(Hd, E)).astype(np.float16)
+    h = rng.normal(size=(M, Hd)).astype(np.float16)
+    h[1, :] = np.nan
+    ctx = make_ctx(B, 64 * 1024)
+    rid = ctx.register_f16(Wr)
+    ctx.set_placement([])
+    ids = torch.full((M, k), -7, dtype=torch.int32, device="cuda")
+    gates = torch.zeros((M, k), dtype=torch.float32, device="cuda")
+    ctx.route_topk(rid, H.to_dev(h), M, k, ids, gates)
+    ctx.sync()
+    got_ids, got_gates = ids.cpu().numpy(), gates.cpu().numpy()
+    assert got_ids.min() >= 0 and got_ids.max() < E
+    assert len(set(got_ids[1].tolist())) == k and np.isnan(got_gates[1]).all()
+    ids_ref, gates_ref, _ = O.route_topk(h[[0, 2]], Wr, k)
+    assert np.array_equal(got_ids[[0, 2]], ids_ref) and np.allclose(got_gates[[0, 2]], gates_ref, atol=1e-6)
+    ctx.close()
+
+
+def test_moe_linear_rejects_ids_out_of_range(B, torch):
+    """ids are caller data.  Host-placed slices: checked on the host before anything runs.  All slices resident: only the
+    kernel sees them; it computes with expert 0 in place of the bad id (no wild address) and raises the status word, so
+    the next ats_sync reports ATS_ERR_INVALID."""
+    shape = W.MOE_SMALL
+    Bk = W.moe_block(95, 0, shape)
+    sl = W.q4_bytes(shape.ffn, shape.hidden)
+    x = W.activations(95, 0, (1, shape.hidden))
+    for where, code_at in ((B.ATS_HOST, "call"), (B.ATS_GPU, "sync")):
+        ctx = make_ctx(B, shape.n_experts * (sl + 256) + 64 * 1024, ring_slots=4, slot_bytes=sl, chunk_bytes=sl)
+        tid = ctx.register_q4(*Bk[W.ROLE_GATE])
+        ctx.set_placement([(tid, -1, where)])
+        ids = torch.tensor([[1, shape.n_experts + 5, 2, -3]], dtype=torch.int32, device="cuda")
+        y = torch.zeros((1, 4, shape.ffn), dtype=torch.float16, device="cuda")
+        with pytest.raises(B.AtsError) as e:
+            ctx.moe_linear(tid, H.to_dev(x), ids, y, 1, 4)
+            assert code_at == "sync"
+            ctx.sync()
+        assert e.value.code == B.ATS_ERR_INVALID
+        if code_at == "sync":
+            # the slots with valid ids were computed; the bad ones ran on expert 0
+            got = y.cpu().numpy()
+            want = O.moe_linear(x, np.array([[1, 0, 2, 0]]), *Bk[W.ROLE_GATE])
+            H.assert_close(got.reshape(4, -1), want.reshape(4, -1), what="moe_linear with clamped ids")
+        ctx.close()
+
+
+def test_bounded_wait_expiry_is_reported_and_leaves_other_contexts_usable(B, torch):
+    """The failure path of the streaming GEMV, made to run without anything faulting or hanging: the test hook shortens
+    the kernel's wait limit to about two milliseconds and makes the producer leave out the copies of tile 0, so the
+    consumers of that tile wait in vain, give up, raise the status word and return; the other CTAs finish their rows.
+    ats_sync then returns ATS_ERR_TIMEOUT and the context refuses further work; a fresh context computes correctly."""
+    N, K = 64, 256  # four tiles of 16 rows, one per CTA
+    packed, scales = W.q4_packed(93, 1, W.ROLE_Q, N, K)
+    x = W.activations(93, 1, (1, K))
+    want = O.linear(x, packed, scales)
+    ctx = make_ctx(B, W.q4_bytes(N, K) + 512)
+    tid = ctx.register_q4(packed, scales)
+    ctx.set_placement([(tid, -1, B.ATS_GPU)])
+    y = torch.zeros((1, N), dtype=torch.float16, device="cuda")
+    ctx.linear(tid, H.to_dev(x), y, 1)
+    ctx.sync()
+    H.assert_close(y.cpu().numpy(), want, what="gemv before the injected expiry")
+    ctx.debug_gemv_wait(4_000_000, withhold_tile=0)
+    y.zero_()
+    ctx.linear(tid, H.to_dev(x), y, 1)
+    with pytest.raises(B.AtsError) as e:
+        ctx.sync(timeout_ms=5000)
+    assert e.value.code == B.ATS_ERR_TIMEOUT and "bounded wait" in str(e.value)
+    got = y.cpu().numpy()
+    assert not got[0, :16].any()  # tile 0 never arrived: its rows were not written
+    H.assert_close(got[:, 16:], want[:, 16:], what="rows of the tiles that did arrive")
+    with pytest.raises(B.AtsError) as e:
+        ctx.linear(tid, H.to_dev(x), y, 1)
+    assert e.value.code == B.ATS_ERR_CUDA  # poisoned
+    ctx.close()
+    ctx2 = make_ctx(B, W.q4_bytes(N, K) + 512)
+    t2 = ctx2.register_q4(packed, scales)
+    ctx2.set_placement([(t2, -1, B.ATS_GPU)])
+    y2 = torch.zeros((1, N), dtype=torch.float16, device="cuda")
+    ctx2.linear(t2, H.to_dev(x), y2, 1)
+    ctx2.sync()
+    H.assert_close(y2.cpu().numpy(), want, what="gemv on a fresh context after the expiry")
+    ctx2.close()

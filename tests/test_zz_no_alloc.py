@@ -6,7 +6,9 @@ The file name sorts last on purpose: a run that stops at the first failure has t
 import numpy as np
 import pytest
 
+from oracle import ats_oracle as O
 from paper_2607_10183_b200 import workloads as W
+from tests import helpers as H
 
 pytestmark = pytest.mark.gpu
 MB = 1 << 20
@@ -29,8 +31,19 @@ def test_static_scratch_linear_equals_linear_twice_in_a_row():
             want = torch.empty((T, N), dtype=torch.float16, device="cuda")
             got = torch.full((T, N), 3.0, dtype=torch.float16, device="cuda")
             ctx.linear(tid, x, want, T)
+            if call == 1:
+                # nothing may be allocated by the call: the device's free memory and torch's own pool stay as they are
+                # (the first call on a device has already resolved the array's address)
+                ctx.sync()
+                free0, alloc0, resv0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
             ctx.linear_static_scratch(tid, x, got, T)
             ctx.sync()
+            if call == 1:
+                assert torch.cuda.mem_get_info()[0] == free0
+                assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == resv0
+            # against the oracle as well (fp16 operands: the GEMM's weight mode), not only against the other entry point
+            H.assert_close(got.cpu().numpy(), O.linear(W.activations(77, call, (T, K)), packed, scales, O.WEIGHT_F16, round_out=True),
+                           what=f"static-scratch linear {N}x{K} T={T} vs oracle")
             # same kernels, same split choice, same summation order: the outputs are identical, which is well inside
             # the 2e-3 relative tolerance the other GEMM tests use
             a, b = got.cpu().numpy().astype(np.float64), want.cpu().numpy().astype(np.float64)
@@ -46,6 +59,7 @@ def test_static_scratch_linear_equals_linear_twice_in_a_row():
         ctx.linear_static_scratch(tid, x1, y2, 3)
         ctx.sync()
         assert np.array_equal(y1.cpu().numpy().view(np.uint16), y2.cpu().numpy().view(np.uint16))
+        H.assert_close(y2.cpu().numpy(), O.linear(W.activations(77, 5, (3, K)), packed, scales), what="static-scratch linear, 3 rows vs oracle")
         ctx.close()
 
 
@@ -69,4 +83,10 @@ def test_static_scratch_rejects_what_it_cannot_hold_and_host_placed_tensors():
     with pytest.raises(B.AtsError) as e:
         ctx.linear_static_scratch(tid, x, y, 16)
     assert e.value.code == B.ATS_ERR_STATE
+    # fp16 weight matrices are not taken by this entry point (the header says so)
+    wid = ctx.register_w16(np.zeros((64, 64), dtype=np.float16))
+    ctx.set_placement([(tid, -1, B.ATS_GPU), (wid, -1, B.ATS_GPU)])
+    with pytest.raises(B.AtsError) as e:
+        ctx.linear_static_scratch(wid, x, y, 16)
+    assert e.value.code == B.ATS_ERR_INVALID
     ctx.close()
