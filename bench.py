@@ -413,8 +413,10 @@ def extra_moe(torch, B, W, peaks, quick):
     Bk = W.moe_block(4, 0, shape)
     sl = W.q4_bytes(shape.ffn, shape.hidden)
     out = {"workload": "config 4: MoE block decode; hybrid = odd experts host-placed", "expert_slice_bytes": sl}
-    for hybrid in (False, True, "gather"):
-        # the gather runs get room in the workspace for the distinct host-placed experts of a call (the copy kernel's target)
+    for hybrid in (False, "ring", "gather"):
+        # "ring": the staging ring forced (ATS_FLAG_MOE_RING_ONLY); "gather": the library's default for host-placed experts
+        # (in-kernel reads of the mapped store at batch 1, the copy kernel into the workspace at batch 8), whose context gets
+        # room in the workspace for the distinct host-placed experts of a call
         ws = (8 << 20) + (3 * 64 * (sl + 256) if hybrid == "gather" else 0)
         ctx = B.Context(3 * shape.n_experts * (sl + 256) + 64 * (sl + 256) + (8 << 20) + ws, workspace_bytes=ws, ring_slots=64,
                         slot_bytes=sl, chunk_bytes=sl)
@@ -424,9 +426,8 @@ def extra_moe(torch, B, W, peaks, quick):
         desc = B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, n_experts=shape.n_experts, top_k=shape.top_k, rms_eps=shape.rms_eps, **ids)
         ctx.set_placement([(ids[n], e, B.ATS_HOST if (hybrid and e % 2) else B.ATS_GPU) for n in ("w_gate", "w_up", "w_down")
                            for e in range(shape.n_experts)])
-        if hybrid == "gather":
-            ctx.set_flags(B.ATS_FLAG_MOE_DEVICE_GATHER)  # host-placed experts read in place over PCIe, ids stay on the device
-        elif hybrid:
+        if hybrid == "ring":
+            ctx.set_flags(B.ATS_FLAG_MOE_RING_ONLY)
             out["pcie_h2d_measured_gbs"] = ctx.measure_h2d(64 * sl, 10)
         for M in (1, 8):
             xs = [torch.from_numpy(W.activations(4, 0, (M, shape.hidden), step=s)).cuda() for s in range(16)]
@@ -444,7 +445,7 @@ def extra_moe(torch, B, W, peaks, quick):
             ctx.sync()
             dt = (time.perf_counter() - t0) / n
             st = ctx.stats()
-            key = f"{'hybrid_device_gather' if hybrid == 'gather' else 'hybrid' if hybrid else 'resident'}_M{M}"
+            key = f"{'hybrid' if hybrid == 'gather' else 'hybrid_ring_only' if hybrid else 'resident'}_M{M}"
             out[key] = {"us_per_call": dt * 1e6, "tokens_per_s": M / dt, "streamed_bytes_per_call": st.streamed_bytes / n,
                         "launches_per_call": st.kernel_launches / n, "timing": "wall clock around back-to-back calls (host included)"}
             if not hybrid:
@@ -456,7 +457,7 @@ def extra_moe(torch, B, W, peaks, quick):
                 out[key]["expert_bytes_per_call_upper"] = moe_bytes
             if hybrid == "gather":
                 # the same inputs select the same experts as in the ring run: its byte count applies
-                moved = out[f"hybrid_M{M}"]["streamed_bytes_per_call"]
+                moved = out[f"hybrid_ring_only_M{M}"]["streamed_bytes_per_call"]
                 out[key]["host_bytes_read_per_call"] = moved
                 out[key]["pcie_gbs_over_call_time"] = moved / dt / 1e9
                 if M == 1:  # no host synchronisation inside a call: device time of a queue of calls
@@ -897,7 +898,7 @@ def extra_model_loop_moe(torch, B, W, peaks, quick):
         ws = max(B.workspace_bytes(probe, prompt), B.workspace_bytes(probe, 1)) + (1 << 20) + stage
         arena = ws + 8 * (sl + 256) + L * (attn_bytes + 3 * mshape.n_experts * (sl + 256) + (1 << 20)) + (4 << 20)
         ctx = B.Context(arena, workspace_bytes=ws, ring_slots=8, slot_bytes=sl, chunk_bytes=sl,
-                        flags=B.ATS_FLAG_MOE_DEVICE_GATHER if hybrid else 0)
+                        flags=0)
         descs, place = [], []
         damp = np.float16(0.1)
         for l in range(L):

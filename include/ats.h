@@ -78,16 +78,20 @@ enum {
   ATS_FLAG_TIME_KERNELS = 4u,     /* bracket every GEMV / grouped GEMV / GEMM launch with CUDA events (see ats_stats.timed_*) */
   ATS_FLAG_NO_PDL = 8u,           /* launch every kernel fully serialized (no programmatic dependent launch overlap) */
   ATS_FLAG_NO_GEMM_PAIR = 32u,    /* do not run large GEMMs as pairs of CTAs on two SMs (tcgen05 cta_group::2): the single-CTA kernel only */
-  ATS_FLAG_MOE_DEVICE_GATHER = 16u, /* single-token MoE stages with host-placed experts: no staging ring and no host round trip for the
-                                     routing ids: the grouped-expert kernel reads the selected host-placed slices straight
-                                     from the pinned host store over PCIe (the store is mapped into the device's address
-                                     space), picking each slice's address from a per-tensor table on the device by the
-                                     expert id (the zero-copy path of Sections 4.1 / 4.2.1).  Same arithmetic, same results;
-                                     ats_stats.streamed_bytes / copies / host_syncs do not count these reads.  Calls with
-                                     more than one token: the distinct selected host-placed experts are gathered into the
-                                     part of the workspace beyond the call's own buffers by one launch of an SM-driven copy
-                                     kernel (each slice crosses PCIe once; counted in streamed_bytes, not in copies) when that
-                                     part holds them; otherwise they keep the ring path. */
+  ATS_FLAG_MOE_RING_ONLY = 16u,   /* Decode-step MoE stages with host-placed experts always take the staging ring (ids to
+                                     the host, one cudaMemcpyAsync per chunk of every selected host-placed slice on the
+                                     transfer stream, counted in ats_stats.streamed_bytes / copies / host_syncs).
+                                     Without this flag the library uses the zero-copy path of Sections 4.1 / 4.2.1 where it
+                                     can (the pinned host store is mapped into the device's address space and every stacked
+                                     tensor has a device table of slice addresses, resident copy or place in the store):
+                                     one token: the grouped-expert kernels pick each selected slice's address by the expert
+                                     id on the device and stream a host-placed slice over PCIe straight into their
+                                     shared-memory ring: no ids on the host, no staging slot, no event (these reads are not
+                                     counted in streamed_bytes / copies / host_syncs); several tokens: the ids go to the
+                                     host, and the distinct selected host-placed experts are gathered into the part of the
+                                     workspace beyond the call's own buffers by one launch of an SM-driven copy kernel (each
+                                     slice crosses PCIe once; counted in streamed_bytes, not in copies) when that part holds
+                                     them; otherwise the ring.  Same arithmetic and the same results on every path. */
 };
 /* ats_layer_desc.flags */
 enum { ATS_LAYER_NO_TOPK_RENORM = 1u /* gates = full softmax entries instead of softmax over the top-k */ };

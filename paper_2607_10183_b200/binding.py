@@ -21,7 +21,7 @@ ATS_HOST, ATS_GPU = 0, 1
 ATS_FMT_Q4B32, ATS_FMT_F16, ATS_FMT_W16, ATS_FMT_MXFP4 = 0, 1, 2, 3
 ATS_OUT_F32, ATS_OUT_F16 = 0, 1
 ATS_MODE_DECODE, ATS_MODE_PREFILL = 0, 1
-ATS_FLAG_POISON_SLOTS, ATS_FLAG_SKIP_SCALE_CHECK, ATS_FLAG_TIME_KERNELS, ATS_FLAG_NO_PDL, ATS_FLAG_MOE_DEVICE_GATHER = 1, 2, 4, 8, 16
+ATS_FLAG_POISON_SLOTS, ATS_FLAG_SKIP_SCALE_CHECK, ATS_FLAG_TIME_KERNELS, ATS_FLAG_NO_PDL, ATS_FLAG_MOE_RING_ONLY = 1, 2, 4, 8, 16
 ATS_FLAG_NO_GEMM_PAIR = 32
 ATS_LAYER_NO_TOPK_RENORM = 1
 ATS_STATS_LIST = 512

@@ -1452,7 +1452,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
                                    attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, L->rms_eps, ctx->cs, nl, pdl));
   const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
   bool implicit = tg.contiguous_dev && tu.contiguous_dev && td.contiguous_dev;
-  if (!implicit && M == 1 && (ctx->cfg.flags & ATS_FLAG_MOE_DEVICE_GATHER) && tg.slice_tab_dev && tu.slice_tab_dev && td.slice_tab_dev) {
+  if (!implicit && M == 1 && !(ctx->cfg.flags & ATS_FLAG_MOE_RING_ONLY) && tg.slice_tab_dev && tu.slice_tab_dev && td.slice_tab_dev) {
     // the kernels find every selected slice themselves, in device memory or in the mapped host store: no ids on the
     // host, no ring (shapes the streaming kernel does not take keep the ring path).  One token only: its k experts are
     // distinct, so every host-placed slice crosses PCIe once; with several tokens, pairs that share an expert would each
@@ -1468,12 +1468,12 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   if (!implicit) {
     ATS_TRY(fetch_ids(ctx, w.ids, P, E));
     ids_host = ctx->ids_host;
-    // Several tokens under ATS_FLAG_MOE_DEVICE_GATHER: the distinct selected host-placed experts are gathered into the
+    // Several tokens (unless ATS_FLAG_MOE_RING_ONLY): the distinct selected host-placed experts are gathered into the
     // workspace beyond this call's buffers by one launch of the copy kernel (every slice crosses PCIe once, no per-copy
     // cost), when that room exists and the streaming kernel takes the shapes; the stages then run as one launch each
     // over per-call address tables.  Otherwise: the staging ring.
     bool staged = false;
-    if ((ctx->cfg.flags & ATS_FLAG_MOE_DEVICE_GATHER) && tg.host_dev && tu.host_dev && td.host_dev) {
+    if (!(ctx->cfg.flags & ATS_FLAG_MOE_RING_ONLY) && tg.host_dev && tu.host_dev && td.host_dev) {
       MoeGemvParams probe1{}, probe2{};
       probe1.K = H; probe1.n_rows = (int)L->ffn; probe1.mode = GEMV_SWIGLU_F16;
       probe1.mx = probe2.mx = tg.d.fmt == ATS_FMT_MXFP4;

@@ -514,7 +514,7 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
     float prev[kRPW];
     bool have_prev = false;
     for (int li = li0; li < li1; ++li) {
-      const int it = grp + kGroups * li;
+      [[maybe_unused]] const int it = grp + kGroups * li;
       if (!__all_sync(0xffffffffu, mbar_wait_suspending(&sh.full[s], cyc & 1, limit))) {
         failed = true;
         break;
@@ -536,6 +536,19 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
           cw[r][j] = in ? codes[b] : make_uint4(0, 0, 0, 0);
           sc[r][j] = in ? __half2float(scp[b]) : 0.f;
         }
+      }
+      // The stage is released as soon as its words are in registers, not after the arithmetic on them: a stage that is
+      // held while it is being computed on is a stage that is not in flight, and the ring is what keeps HBM busy.  The
+      // fold below makes the release wait for every load (an instruction issues only when its operands have arrived).
+      {
+        uint32_t fold = 0;
+#pragma unroll
+        for (int r = 0; r < kRPW; ++r)
+#pragma unroll
+          for (int j = 0; j < kJ; ++j) fold ^= cw[r][j].x ^ cw[r][j].y ^ cw[r][j].z ^ cw[r][j].w ^ __float_as_uint(sc[r][j]);
+        asm volatile("" ::"r"(fold) : "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.empty[s]);
       }
       if (have_prev) reduce_store(prev, li - 1 - li0);
       float acc[kRPW];
@@ -567,9 +580,7 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
           acc[r] = fmaf(sc[r][j], fmaf(dot, xm[j], xc[j]), acc[r]);
         }
       }
-      __syncwarp();
       ATS_TR(200 + it);
-      if (lane == 0) mbar_arrive(&sh.empty[s]);  // this warp is done reading stage s
       stream_advance(s, cyc, kGroups, n_stages);
 #pragma unroll
       for (int r = 0; r < kRPW; ++r) prev[r] = acc[r];

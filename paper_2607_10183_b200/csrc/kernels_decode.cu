@@ -760,11 +760,11 @@ cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __ha
 // memory (16-byte async copies, issued before the grid dependency resolves) and every head's warps read them from
 // there, so the cache crosses the L2-to-SM fabric once instead of once per query head; that traffic, not DRAM, bounds
 // this kernel.  Warp (head, sub-block) owns 32 positions, one per lane.
-// Positions per CTA: 64 up to 2048 positions of context (a CTA of 256 threads and 46 KB of shared memory for a group of
-// four heads of 128: small enough to sit on an SM beside a CTA of the streaming GEMV, so that this kernel's cache rows are
-// staged while the QKV projection still runs and the O projection's weights while this kernel runs), 128 beyond that
-// (fewer partials for the final merge, which reads 16 splits per round trip).
-int attn_decode_pos_per_cta(int n_ctx) { return n_ctx <= 2048 ? 64 : 128; }
+// Positions per CTA: 64, or 128 for contexts beyond 1024 so that the final merge still reads all splits of a head in
+// one round trip (16 splits) up to 2048 positions.  (64 positions up to 2048, with both kernels' registers capped so that
+// a CTA of this kernel fits an SM beside a CTA of the streaming GEMV, was measured and lost: the GEMV slows down by 0.5 us
+// per launch at 80 registers and this kernel by 2.9 us with 17 splits to merge, and nothing is gained back.)
+int attn_decode_pos_per_cta(int n_ctx) { return n_ctx <= 1024 ? 64 : 128; }
 int attn_decode_splits(int n_ctx) {
   const int pc = attn_decode_pos_per_cta(n_ctx);
   return (n_ctx + pc - 1) / pc;
@@ -774,7 +774,7 @@ size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) {
 }
 
 template <int D, int SUB>
-__global__ void __maxnreg__(72) attn_decode_fused_kernel(const AttnDecodeParams p) {
+__global__ void __launch_bounds__(512) attn_decode_fused_kernel(const AttnDecodeParams p) {
   extern __shared__ __align__(16) uint8_t dyn_s[];
   attn_decode_body<D, SUB, true>(p, (int)blockIdx.x, (int)blockIdx.y, (int)gridDim.x, (int)threadIdx.x, (int)blockDim.x, dyn_s);
 }
@@ -996,16 +996,27 @@ __global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(c
 #pragma unroll
   for (int q = 0; q < 8; ++q) acc[q] = 0.f;
   if (grp < R) {
-#pragma unroll 4
-    for (int i = grp; i < Hc; i += R) {
-      const uint4 w = __ldg(reinterpret_cast<const uint4*>(wr + (size_t)(row0 + i) * E + e0));
-      const float x = h_s[i];
-      const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+    // The rows of a thread are fetched in batches of 16 loads that are all issued before the first is used: the
+    // matrix is read once at memory latency (a token's 512 KB are 64 KB per CTA, one batch per thread), not once per row.
+    constexpr int kBatch = 16;
+    for (int i0 = grp; i0 < Hc; i0 += R * kBatch) {
+      uint4 w[kBatch];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float2 f = __half22float2(u32_as_half2(ws[q]));
-        acc[2 * q] = fmaf(x, f.x, acc[2 * q]);
-        acc[2 * q + 1] = fmaf(x, f.y, acc[2 * q + 1]);
+      for (int b = 0; b < kBatch; ++b) {
+        const int i = i0 + b * R;
+        w[b] = i < Hc ? __ldg(reinterpret_cast<const uint4*>(wr + (size_t)(row0 + i) * E + e0)) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) {
+        const int i = i0 + b * R;
+        const float x = i < Hc ? h_s[i] : 0.f;
+        const uint32_t ws[4] = {w[b].x, w[b].y, w[b].z, w[b].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float2 f = __half22float2(u32_as_half2(ws[q]));
+          acc[2 * q] = fmaf(x, f.x, acc[2 * q]);
+          acc[2 * q + 1] = fmaf(x, f.y, acc[2 * q + 1]);
+        }
       }
     }
 #pragma unroll

@@ -6,11 +6,6 @@ namespace ats {
 
 namespace {
 
-// Registers per thread: capped so that the decode attention kernel's CTAs (256 threads of up to 72 registers, 46 KB of
-// shared memory) fit an SM beside a CTA of this kernel.  They are launched as this kernel's dependents and stage their
-// cache rows while it streams, and the CTAs of the GEMV after them move in beside them in turn.
-constexpr int kStreamMaxRegs = 80;
-
 // One CTA: ring set-up, then the producer warp and the consumer warps go their ways.  dep_resolved: the caller has already
 // waited for the preceding kernel (its weight addresses come from that kernel's output).
 template <int PARTS, bool SW, bool MX>
@@ -29,7 +24,7 @@ __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const in
 }
 
 template <int PARTS, bool SW, bool MX>
-__global__ void __maxnreg__(kStreamMaxRegs) gemv_stream_kernel(const StreamParams p) {
+__global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamParams p) {
   gemv_stream_body<PARTS, SW, MX>(p, (int)blockIdx.x, (int)gridDim.x, false);
 }
 
@@ -48,7 +43,7 @@ struct MoeSel {
   int n_experts;
 };
 template <int PARTS, bool SW, bool MX>
-__global__ void __maxnreg__(kStreamMaxRegs) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
+__global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
   StreamParams p = p0;
   const int job = blockIdx.y;
   int xrow, orow;

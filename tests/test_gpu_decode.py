@@ -693,7 +693,7 @@ def test_moe_block_matches_oracle_and_streams_only_selected_experts(B, torch, sh
     odd = {e for e in range(shape.n_experts) if e % 2}
     chunk = 256 * 1024
     Bk, x, y_res, st_res = run_moe(B, torch, shape, cfg, M, set())
-    _, _, y_hyb, st_hyb = run_moe(B, torch, shape, cfg, M, odd, chunk=chunk, flags=B.ATS_FLAG_POISON_SLOTS)
+    _, _, y_hyb, st_hyb = run_moe(B, torch, shape, cfg, M, odd, chunk=chunk, flags=B.ATS_FLAG_POISON_SLOTS | B.ATS_FLAG_MOE_RING_ONLY)
     t = H.oracle_moe_tensors(Bk)
     want, ids_ref, gates_ref, logits = O.moe_block(x, t, shape)
     assert O.min_rank_gap(logits, shape.top_k) > 1e-4, "degenerate seed: near-tie among the routed experts"
@@ -712,16 +712,16 @@ def test_moe_block_matches_oracle_and_streams_only_selected_experts(B, torch, sh
 
 @pytest.mark.parametrize("M", [1, 8])
 def test_moe_device_gather_equals_resident_without_host_round_trip(B, torch, M):
-    """ATS_FLAG_MOE_DEVICE_GATHER: the grouped-expert kernels read the selected host-placed experts straight from the mapped
-    pinned store, addressed through the per-tensor slice table by the ids on the device.  Same bits as the all-resident
+    """The default path for host-placed experts (no ATS_FLAG_MOE_RING_ONLY): the grouped-expert kernels read the selected
+    host-placed experts straight from the mapped pinned store, addressed through the per-tensor slice table by the ids on the device.  Same bits as the all-resident
     run, no host synchronisation, nothing through the staging ring."""
     shape, cfg = W.MOE_FULL, 4
     odd = {e for e in range(shape.n_experts) if e % 2}
     _, _, y_res, _ = run_moe(B, torch, shape, cfg, M, set())
-    _, _, y_dg, st = run_moe(B, torch, shape, cfg, M, odd, flags=B.ATS_FLAG_MOE_DEVICE_GATHER)
+    _, _, y_dg, st = run_moe(B, torch, shape, cfg, M, odd)
     assert np.array_equal(y_res.view(np.uint16), y_dg.view(np.uint16))
     # every expert on the host
-    _, _, y_all, st_all = run_moe(B, torch, shape, cfg, M, set(range(shape.n_experts)), flags=B.ATS_FLAG_MOE_DEVICE_GATHER)
+    _, _, y_all, st_all = run_moe(B, torch, shape, cfg, M, set(range(shape.n_experts)))
     assert np.array_equal(y_res.view(np.uint16), y_all.view(np.uint16))
     if M == 1:  # the gather path: nothing through the ring, no ids on the host
         assert st.host_syncs == 0 and st.streamed_bytes == 0 and st.copies == 0
@@ -730,7 +730,7 @@ def test_moe_device_gather_equals_resident_without_host_round_trip(B, torch, M):
         assert st.host_syncs == 1 and st.streamed_bytes > 0 and st.copies > 0
         # with room beyond the call's buffers the copy kernel gathers the distinct selected experts in one launch
         sl = W.q4_bytes(shape.ffn, shape.hidden)
-        _, _, y_st, st_st = run_moe(B, torch, shape, cfg, M, odd, flags=B.ATS_FLAG_MOE_DEVICE_GATHER, ws=4 * MB + 3 * 64 * (sl + 256))
+        _, _, y_st, st_st = run_moe(B, torch, shape, cfg, M, odd, ws=4 * MB + 3 * 64 * (sl + 256))
         assert np.array_equal(y_res.view(np.uint16), y_st.view(np.uint16))
         # same distinct experts as the ring run moved (slices of this shape need no padding), no DMA copies
         assert st_st.host_syncs == 1 and st_st.copies == 0 and st_st.streamed_bytes == st.streamed_bytes
@@ -783,7 +783,7 @@ def test_moe_small_ring_forces_waves(B, torch):
     everything = set(range(shape.n_experts))
     Bk, x, y_res, _ = run_moe(B, torch, shape, 97, 5, set())
     for slots in (2, 3, 5):
-        _, _, y, st = run_moe(B, torch, shape, 97, 5, everything, ring_slots=slots, flags=B.ATS_FLAG_POISON_SLOTS)
+        _, _, y, st = run_moe(B, torch, shape, 97, 5, everything, ring_slots=slots, flags=B.ATS_FLAG_POISON_SLOTS | B.ATS_FLAG_MOE_RING_ONLY)
         assert np.array_equal(y.view(np.uint16), y_res.view(np.uint16)), slots
         assert st.ring_reuses > 0
 
