@@ -258,9 +258,9 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, cons
  * (HOST fp16 [M][hidden]) and returns when x_out is valid.  The caches stay on the DEVICE.  Needs 2 * M * hidden * 2 bytes
  * of workspace beyond ats_layer_decode's (ats_workspace_bytes includes them).
  * Any host memory works (two cudaMemcpyAsync and a wait for the stream).  When both buffers lie inside ranges registered
- * with ats_register_host_buffer, no copy engine is involved: a small kernel fetches x_in from the mapped buffer, the
- * layer's last kernel stores the result row straight into x_out, and the call returns as soon as the device has written
- * a completion word that the host polls (bounded; it falls back to waiting for the stream).
+ * with ats_register_host_buffer, only x_in is copied: the layer's last kernel stores the result row straight into x_out,
+ * and the call returns as soon as the device has written a completion word that the host polls (bounded; it falls back
+ * to waiting for the stream).
  * The status word of the context is looked at before returning: ATS_ERR_TIMEOUT if a kernel gave up a bounded wait.
  * Errors as ats_layer_decode, plus ATS_ERR_CUDA from the copies or the wait. */
 int32_t ats_layer_decode_host(ats_ctx* ctx, const ats_layer_desc* desc /*HOST*/, const void* x_in /*HOST*/,

@@ -269,15 +269,17 @@ cudaError_t launch_embed_rows(const uint8_t* slice, int n_rows, int K, const int
 cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __half* out, int M, int H, float eps,
                            cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 // decode attention, fused with the rotary embedding and the KV append (kernels_decode.cu)
+constexpr int kAttnMaxCounters = 192;  // arrival counters of the decode attention in the workspace's reserved head
 struct AttnDecodeParams {
   const float* qkv;   // [q | k | v] fp32 of the new token
   float* q_rot_out;   // optional copy of the rotated query (debug / tests)
   __half* kc;
   __half* vc;
   float* part;        // [n_q][splits][d + 2] scratch
-  int* counters;      // [n_kv] zero between launches
+  int* counters;      // [n_kv * hsplit] zero between launches
   __half* a16;        // [n_q * d]
   int n_q, n_kv, group, cap, pos;
+  int hsplit;         // CTAs that share a kv head's query heads (set by the launcher)
   float scale;
   float cs[128];      // (cos, sin) of pos * theta^(-2i/d), i < d/2
 };
@@ -293,9 +295,7 @@ cudaError_t launch_router_topk_norm(const __half* h, const __half* wr, int M, in
 cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gates, const float* d32, __half* y16,
                                int M, int k, int H, cudaStream_t st, uint64_t* n_launch, int pdl = 0);
 cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uint64_t* n_launch);
-// host-driven calls (kernels_decode.cu): a small input fetched from mapped pinned memory by a kernel, and the completion
-// word written once everything before it in the stream is done
-cudaError_t launch_stage_rows(const void* src_host_alias, void* dst, uint64_t bytes, cudaStream_t st, uint64_t* n_launch);
+// host-driven calls (kernels_decode.cu): the completion word written once everything before it in the stream is done
 cudaError_t launch_signal_done(int* done_alias, int seq, int pdl, cudaStream_t st, uint64_t* n_launch);
 
 // prefill

@@ -7,6 +7,32 @@ namespace ats {
 
 constexpr int kAttnMaxGroup = 8;  // query heads per kv head at most
 
+#ifdef ATS_TRACE_ATTN
+// Timeline probe of development builds: (globaltimer, CTA, event) records of thread 0 of every CTA.
+struct AttnTraceRec {
+  unsigned long long t;
+  unsigned int cta, ev;
+};
+__device__ AttnTraceRec g_attn_trace[1 << 15];
+__device__ unsigned int g_attn_trace_n;
+__shared__ unsigned long long s_attn_tr[8];
+__device__ __forceinline__ void attn_trace(int ev) {
+  if (threadIdx.x != 0) return;
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  s_attn_tr[ev] = t;
+  if (ev == 6 || ev == 7) {  // flush: 6 is every CTA's last stamp unless it merges (then 7 follows and re-flushes that one)
+    const int first = ev == 6 ? 0 : 7, n = ev == 6 ? 7 : 1;
+    const unsigned int i = atomicAdd(&g_attn_trace_n, (unsigned)n);
+    for (int k = 0; k < n; ++k)
+      if (i + k < (1u << 15)) g_attn_trace[i + k] = AttnTraceRec{s_attn_tr[first + k], blockIdx.x + 100u * blockIdx.y, (unsigned)(first + k)};
+  }
+}
+#define ATS_ATR(ev) attn_trace(ev)
+#else
+#define ATS_ATR(ev) do { } while (0)
+#endif
+
 __device__ __forceinline__ __half2 ad_half2(uint32_t v) {
   __half2 h;
   *reinterpret_cast<uint32_t*>(&h) = v;
@@ -27,7 +53,9 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
 }
 
-// The work of one (split, kv head) job, in two parts: staging the past cache rows (which do not depend on the new
+// Job (split, kv head, head part): the group's query heads are divided over `hsplit` CTAs (each stages the same cache rows
+// and attends with group / hsplit heads), so that short contexts still fill the SMs.  jy = kv head * hsplit + part.
+// The work of one job, in two parts: staging the past cache rows (which do not depend on the new
 // token's projections) and everything after those projections exist.  nthr = group * 32 * SUB threads take part,
 // numbered tid = 0 .. nthr-1; they synchronise with __syncthreads() when they are the whole CTA (CTA_SYNC) and with
 // named barrier 4 otherwise.
@@ -60,7 +88,7 @@ __device__ __forceinline__ void attn_decode_stage(const AttnDecodeParams& p, con
 }
 
 template <int D, int SUB, bool CTA_SYNC>
-__device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, const int split, const int kvh, const int n_splits,
+__device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, const int split, const int jy, const int n_splits,
                                                     const int tid, const int nthr, uint8_t* dyn_s) {
   auto job_sync = [&]() {
     if (CTA_SYNC)
@@ -81,7 +109,10 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
   __shared__ float w_m[MAXW], w_l[MAXW];
   __shared__ float w_acc[MAXW][D];
   __shared__ int is_last;
-  const int G = p.group;  // nthr = G * POS
+  const int G = p.group / p.hsplit;  // query heads of this CTA; nthr = G * POS
+  const int kvh = jy / p.hsplit;
+  const int hbase = kvh * p.group + (jy % p.hsplit) * G;  // first of them
+  const bool writer = jy % p.hsplit == 0;                 // one CTA per kv head appends to the caches
   const int lane = tid & 31, warp = tid >> 5;
   const int g = warp / SUB, sub = warp % SUB;
   const int half = D / 2, n_ctx = p.pos + 1;
@@ -92,7 +123,7 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
   // rotary embedding of the group's query heads into shared memory
   for (int idx = tid; idx < G * half; idx += nthr) {
     const int g2 = idx / half, i = idx % half;
-    const int hq2 = kvh * G + g2;
+    const int hq2 = hbase + g2;
     const float* q = p.qkv + (size_t)hq2 * D;
     const float a = q[i], b = q[i + half];
     const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
@@ -115,18 +146,22 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
       __half* srow = reinterpret_cast<__half*>(k_s + (size_t)r_new * KROW);
       srow[i] = ka;
       srow[i + half] = kb;
-      __half* dst = p.kc + ((size_t)kvh * p.cap + p.pos) * D;
-      dst[i] = ka;
-      dst[i + half] = kb;
+      if (writer) {
+        __half* dst = p.kc + ((size_t)kvh * p.cap + p.pos) * D;
+        dst[i] = ka;
+        dst[i + half] = kb;
+      }
     }
     for (int i = tid; i < D; i += nthr) {
       const __half vv = __float2half_rn(p.qkv[qd + kvd + (size_t)kvh * D + i]);
       reinterpret_cast<__half*>(v_s + (size_t)r_new * VROW)[i] = vv;
-      p.vc[((size_t)kvh * p.cap + p.pos) * D + i] = vv;
+      if (writer) p.vc[((size_t)kvh * p.cap + p.pos) * D + i] = vv;
     }
   }
+  ATS_ATR(2);
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   job_sync();
+  ATS_ATR(3);
   const int t0 = tc0 + sub * 32;
   const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
   const bool ok = lane < n_here;
@@ -182,10 +217,11 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
   }
 #pragma unroll
   for (int v = 0; v < V; ++v) w_acc[warp][lane * V + v] = acc[v];
+  ATS_ATR(4);
   job_sync();
   // merge each head's warps (ascending) into this split's partial: 64 threads per head
   const int g2 = tid / 64, j = tid % 64;
-  const int hq2 = kvh * G + g2;
+  const int hq2 = hbase + g2;
   if (g2 < G) {
     float* part = p.part + ((size_t)hq2 * n_splits + split) * (D + 2);
     float mx = -INFINITY;
@@ -209,17 +245,21 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
       part[D + 1] = l;
     }
   }
-  // the last CTA of this kv head merges the splits of its query heads
-  __threadfence();
+  // The last CTA of this job row merges the splits of its query heads.  The barrier orders every thread's partial
+  // before thread 0's fence, and the fence is cumulative: one thread's fence on each side of the counter publishes the
+  // CTA's partials and, in the last CTA, makes the others' visible to the loads below (which bypass L1).
+  ATS_ATR(5);
   job_sync();
   if (tid == 0) {
-    const int prev = atomicAdd(p.counters + kvh, 1);
+    __threadfence();
+    const int prev = atomicAdd(p.counters + jy, 1);
     is_last = prev == n_splits - 1;
-    if (is_last) p.counters[kvh] = 0;  // ready for the next launch
+    if (is_last) p.counters[jy] = 0;  // ready for the next launch
+    __threadfence();
   }
   job_sync();
+  ATS_ATR(6);
   if (!is_last || g2 >= G) return;
-  __threadfence();
   const float* base = p.part + (size_t)hq2 * n_splits * (D + 2);
   float mx = -INFINITY, l = 0.f, o[EPT];
 #pragma unroll
@@ -255,16 +295,19 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
   const float inv = 1.0f / l;
 #pragma unroll
   for (int q = 0; q < EPT; ++q) p.a16[(size_t)hq2 * D + j + 64 * q] = __float2half_rn(o[q] * inv);
+  ATS_ATR(7);
 }
 
 // Stand-alone form: the cache rows of past tokens are requested before the grid dependency resolves.
 template <int D, int SUB, bool CTA_SYNC>
-__device__ __forceinline__ void attn_decode_body(const AttnDecodeParams& p, const int split, const int kvh, const int n_splits,
+__device__ __forceinline__ void attn_decode_body(const AttnDecodeParams& p, const int split, const int jy, const int n_splits,
                                                  const int tid, const int nthr, uint8_t* dyn_s) {
-  attn_decode_stage<D, SUB>(p, split, kvh, tid, nthr, dyn_s);
+  ATS_ATR(0);
+  attn_decode_stage<D, SUB>(p, split, jy / p.hsplit, tid, nthr, dyn_s);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v of the new token come from the preceding kernel
+  ATS_ATR(1);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  attn_decode_compute<D, SUB, CTA_SYNC>(p, split, kvh, n_splits, tid, nthr, dyn_s);
+  attn_decode_compute<D, SUB, CTA_SYNC>(p, split, jy, n_splits, tid, nthr, dyn_s);
 }
 
 }  // namespace ats

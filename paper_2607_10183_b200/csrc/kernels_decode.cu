@@ -784,10 +784,15 @@ cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStr
   int pc = attn_decode_pos_per_cta(p.pos + 1);
   if (p.group * pc > 512) pc = 64;  // large groups: 64 positions keep the CTA within 512 threads
   const int splits = (p.pos + 1 + pc - 1) / pc;
+  // Short contexts give fewer jobs than SMs: the query heads of a group are then divided over 2 or 4 CTAs (each stages
+  // the same cache rows out of L2), which shortens the score and value loops of every CTA in proportion.
+  int hsplit = 1;
+  while (p.group % (2 * hsplit) == 0 && splits * p.n_kv * 2 * hsplit <= 148 && p.n_kv * 2 * hsplit <= kAttnMaxCounters) hsplit *= 2;
+  p.hsplit = hsplit;
   p.scale = 1.0f / sqrtf((float)d);
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(splits, p.n_kv);
-  cfg.blockDim = dim3(p.group * pc);
+  cfg.gridDim = dim3(splits, p.n_kv * hsplit);
+  cfg.blockDim = dim3(p.group / hsplit * pc);
   cfg.dynamicSmemBytes = (size_t)pc * (d * 4 + 16);
   static uint64_t attr_done = 0;
   if (first_use_on_device(&attr_done)) {
@@ -1103,19 +1108,7 @@ cudaError_t launch_moe_combine(const void* res, int res_is_f32, const float* gat
   return launch_dep(moe_combine_kernel<__half>, grid, dim3(256), 0, st, pdl, 1, (const __half*)res, gates, d32, y16, k, H);
 }
 
-// ---------------------------------------------------------------- host-driven calls: input staging and completion word
-// A few kilobytes of activations fetched from mapped pinned host memory by the SMs (16-byte loads over PCIe) into the
-// workspace: for rows this small a kernel is quicker than a copy-engine transfer and the engine hand-over around it.
-__global__ void stage_rows_kernel(const uint4* __restrict__ src_host, uint4* __restrict__ dst, int n16) {
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += gridDim.x * blockDim.x) dst[i] = src_host[i];
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-cudaError_t launch_stage_rows(const void* src_host_alias, void* dst, uint64_t bytes, cudaStream_t st, uint64_t* n_launch) {
-  const int n16 = (int)(bytes / 16);
-  const int grid = std::max(1, std::min((n16 + 255) / 256, 8));
-  ++*n_launch;
-  return launch_dep(stage_rows_kernel, dim3(grid), dim3(256), 0, st, 0, 1, (const uint4*)src_host_alias, (uint4*)dst, n16);
-}
+// ---------------------------------------------------------------- host-driven calls: completion word
 // Completion word of a host-driven call: written (to mapped pinned host memory) once everything before it in the stream
 // has completed and its writes are visible, so the host can poll the word instead of synchronising with the stream.
 __global__ void signal_done_kernel(int* done, int seq) {
@@ -1134,3 +1127,16 @@ cudaError_t launch_fill(void* p, uint64_t bytes, uint8_t v, cudaStream_t st, uin
 }
 
 }  // namespace ats
+
+#ifdef ATS_TRACE_ATTN
+extern "C" int ats_attn_trace_read(void* out_host, int cap_records) {
+  unsigned int n = 0;
+  if (cudaMemcpyFromSymbol(&n, ats::g_attn_trace_n, sizeof n) != cudaSuccess) return -1;
+  if (n > (1u << 15)) n = 1u << 15;
+  if ((int)n > cap_records) n = cap_records;
+  if (n && cudaMemcpyFromSymbol(out_host, ats::g_attn_trace, (size_t)n * sizeof(ats::AttnTraceRec)) != cudaSuccess) return -1;
+  unsigned int zero = 0;
+  cudaMemcpyToSymbol(ats::g_attn_trace_n, &zero, sizeof zero);
+  return (int)n;
+}
+#endif
