@@ -6,6 +6,16 @@
 namespace ats {
 
 constexpr int kAttnMaxGroup = 8;  // query heads per kv head at most
+constexpr int kAttnMaxWarps = 16;  // warps of a job at most (heads of the CTA * sub-blocks)
+constexpr int kAttnMaxD = 128;
+
+// Static shared memory of a job (head dimensions up to kAttnMaxD use the front of each row).
+struct AttnShared {
+  __align__(16) float q_s[kAttnMaxGroup][kAttnMaxD];  // rotated query heads
+  float w_acc[kAttnMaxWarps][kAttnMaxD];              // per-warp unnormalised outputs
+  float w_m[kAttnMaxWarps], w_l[kAttnMaxWarps];       // per-warp score maximum and sum of exponentials
+  int is_last;
+};
 
 #ifdef ATS_TRACE_ATTN
 // Timeline probe of development builds: (globaltimer, CTA, event) records of thread 0 of every CTA.
@@ -89,7 +99,7 @@ __device__ __forceinline__ void attn_decode_stage(const AttnDecodeParams& p, con
 
 template <int D, int SUB, bool CTA_SYNC>
 __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, const int split, const int jy, const int n_splits,
-                                                    const int tid, const int nthr, uint8_t* dyn_s) {
+                                                    const int tid, const int nthr, uint8_t* dyn_s, AttnShared& as) {
   auto job_sync = [&]() {
     if (CTA_SYNC)
       __syncthreads();
@@ -102,13 +112,13 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
   constexpr int KROW = D * 2 + 16;     // key row pitch in shared memory: the 16-byte pad makes lane-per-row reads conflict-free
   constexpr int VROW = D * 2;
   constexpr int EPT = D / 64;          // output elements per thread in the merges (64 threads per head)
-  constexpr int MAXW = 16;             // warps per CTA at most (group * SUB)
   uint8_t* k_s = dyn_s;                              // [POS][KROW]
   uint8_t* v_s = dyn_s + (size_t)POS * KROW;    // [POS][VROW]
-  __shared__ __align__(16) float q_s[kAttnMaxGroup][D];
-  __shared__ float w_m[MAXW], w_l[MAXW];
-  __shared__ float w_acc[MAXW][D];
-  __shared__ int is_last;
+  float (&q_s)[kAttnMaxGroup][kAttnMaxD] = as.q_s;
+  float (&w_acc)[kAttnMaxWarps][kAttnMaxD] = as.w_acc;
+  float (&w_m)[kAttnMaxWarps] = as.w_m;
+  float (&w_l)[kAttnMaxWarps] = as.w_l;
+  int& is_last = as.is_last;
   const int G = p.group / p.hsplit;  // query heads of this CTA; nthr = G * POS
   const int kvh = jy / p.hsplit;
   const int hbase = kvh * p.group + (jy % p.hsplit) * G;  // first of them
@@ -301,13 +311,13 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
 // Stand-alone form: the cache rows of past tokens are requested before the grid dependency resolves.
 template <int D, int SUB, bool CTA_SYNC>
 __device__ __forceinline__ void attn_decode_body(const AttnDecodeParams& p, const int split, const int jy, const int n_splits,
-                                                 const int tid, const int nthr, uint8_t* dyn_s) {
+                                                 const int tid, const int nthr, uint8_t* dyn_s, AttnShared& as) {
   ATS_ATR(0);
   attn_decode_stage<D, SUB>(p, split, jy / p.hsplit, tid, nthr, dyn_s);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // q, k, v of the new token come from the preceding kernel
   ATS_ATR(1);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  attn_decode_compute<D, SUB, CTA_SYNC>(p, split, jy, n_splits, tid, nthr, dyn_s);
+  attn_decode_compute<D, SUB, CTA_SYNC>(p, split, jy, n_splits, tid, nthr, dyn_s, as);
 }
 
 }  // namespace ats

@@ -776,7 +776,8 @@ size_t attn_decode_scratch_floats(int n_q, int d, int n_ctx) {
 template <int D, int SUB>
 __global__ void __launch_bounds__(512) attn_decode_fused_kernel(const AttnDecodeParams p) {
   extern __shared__ __align__(16) uint8_t dyn_s[];
-  attn_decode_body<D, SUB, true>(p, (int)blockIdx.x, (int)blockIdx.y, (int)gridDim.x, (int)threadIdx.x, (int)blockDim.x, dyn_s);
+  __shared__ AttnShared as;
+  attn_decode_body<D, SUB, true>(p, (int)blockIdx.x, (int)blockIdx.y, (int)gridDim.x, (int)threadIdx.x, (int)blockDim.x, dyn_s, as);
 }
 
 cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch) {

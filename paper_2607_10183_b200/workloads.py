@@ -150,13 +150,13 @@ MOE_SMALL = MoEShape(hidden=128, n_experts=16, ffn=96, top_k=4)
 MOE_FULL = MoEShape()
 
 
-def dense_layer(config: int, layer: int, shape: DenseShape = DENSE_FULL) -> dict:
-    """All tensors of one dense decoder layer: ``{role: (packed, scales)}`` plus the two norm gains."""
+def dense_layer(config: int, layer: int, shape: DenseShape = DENSE_FULL, gain_std: float = DENSE_GAIN_STD) -> dict:
+    """All tensors of one dense decoder layer: ``{role: (packed, scales)}`` plus the two norm gains ~N(0, gain_std)."""
     out = {"shape": shape}
     for role, n_out, k_in in shape.tensor_shapes():
         out[role] = q4_packed(config, layer, role, n_out, k_in)
-    out[ROLE_ATTN_NORM] = norm_gain(config, layer, ROLE_ATTN_NORM, shape.hidden)
-    out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden)
+    out[ROLE_ATTN_NORM] = norm_gain(config, layer, ROLE_ATTN_NORM, shape.hidden, gain_std)
+    out[ROLE_FFN_NORM] = norm_gain(config, layer, ROLE_FFN_NORM, shape.hidden, gain_std)
     return out
 
 

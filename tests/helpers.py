@@ -36,6 +36,17 @@ def assert_close(y, ref, tol=TOL, what="", elementwise=True):
     return float(norm.max()), float(ratio.max())
 
 
+def error_measures(y, ref, tol=TOL):
+    """The two figures assert_close gates (largest normwise error over the rows, largest mixed elementwise ratio), only
+    measured: for results a test reports without holding them to a bound."""
+    y = np.asarray(y, dtype=np.float64).reshape(-1, np.asarray(y).shape[-1])
+    r = np.asarray(ref, dtype=np.float64).reshape(y.shape)
+    err = np.abs(y - r)
+    norm = err.max(axis=1) / np.maximum(np.abs(r).max(axis=1), 1e-30)
+    rms = np.sqrt(np.mean(r * r, axis=1, keepdims=True))
+    return float(norm.max()), float((err / (tol * (np.abs(r) + rms) + 1e-300)).max())
+
+
 def bits_equal_mod_zero_sign(a, b):
     """Bitwise equality after mapping -0 to +0."""
     a = np.asarray(a)

@@ -481,6 +481,72 @@ def test_dense_layer_decode_matches_oracle(B, torch, shape_name, pos, cap):
     assert st.streamed_bytes == 0 and st.resident_bytes == H.dense_layer_bytes(shape)
 
 
+@pytest.mark.parametrize("gain_std", [W.DENSE_GAIN_STD, 1.0])
+def test_decode_layer_stage_by_stage_full_size(B, torch, gain_std):
+    """Config 2 (one token at position 1024 through the full-size layer), every kernel on its own: each stage's output is
+    compared with the oracle's definition of that stage applied to the inputs the stage actually consumed (read back from
+    the library's workspace), under both error gates; the GEMV stages also under the bound derived from their operand.
+    Once with the norm gains the other full-size tests use and once with gains ~N(0, 1); the end-to-end error of the layer
+    is reported, not gated, in this test."""
+    shape, cfg, pos, cap = W.DENSE_FULL, 2, 1024, 1025
+    L = W.dense_layer(cfg, 0, shape, gain_std)
+    t = H.oracle_dense_tensors(L)
+    ws = B.workspace_bytes(B.layer_desc(hidden=shape.hidden, ffn=shape.ffn, wq=0, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                                        head_dim=shape.head_dim, kv_capacity=cap), 1) + MB
+    ctx = B.Context(ws + H.dense_layer_bytes(shape) + 32 * 256 + 8 * shape.hidden + MB, workspace_bytes=ws)
+    desc, ids = H.register_dense_layer(ctx, L, 0, cap)
+    ctx.set_placement([(ids[n], -1, B.ATS_GPU) for n in ALL_GPU])
+    kc, vc = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, pos)
+    kd, vd = H.to_dev(kc), H.to_dev(vc)
+    x = W.activations(cfg, 0, (1, shape.hidden), step=0)
+    y = torch.empty((1, shape.hidden), dtype=torch.float16, device="cuda")
+    ctx.layer_decode(desc, H.to_dev(x), y, kd, vd, pos, 1)
+    ctx.sync()
+    g = {n: ctx.debug_decode_buffer(desc, 1, i, dt).astype(np.float64).reshape(1, -1)
+         for i, (n, dt) in enumerate((("h", np.float16), ("qkv", np.float32), ("q_rot", np.float32), ("a", np.float16), ("x1", np.float32),
+                                      ("h2", np.float16), ("act", np.float16)))}
+    yg, kg, vg = y.cpu().numpy(), kd.cpu().numpy(), vd.cpu().numpy()
+    edges, wmode = ctx.numerics(B.ATS_MODE_DECODE)
+    ctx.close()
+    nq, nkv, d, ffn, hid = shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn, shape.hidden
+    qd, kvd = nq * d, nkv * d
+    x64 = x.astype(np.float64)
+
+    def gemv_stage(got, operand, name, what):
+        """A single-token GEMV stage against the exact product with ITS operand: both gates and the derived bound."""
+        w = O.dequantize(*t[name])
+        ref = (w @ operand.reshape(-1)).reshape(1, -1)
+        H.assert_close(got, ref, what=what)
+        assert np.all(np.abs(got - ref).reshape(-1) <= fixed_point_gemv_bound(operand, w)), what
+        return ref
+
+    H.assert_close(g["h"], O.rn16(O.rmsnorm(x64, t["attn_norm"], shape.rms_eps)), what="h")
+    for name, lo, hi in (("wq", 0, qd), ("wk", qd, qd + kvd), ("wv", qd + kvd, qd + 2 * kvd)):
+        gemv_stage(g["qkv"][:, lo:hi], g["h"], name, name)
+    H.assert_close(g["q_rot"], O.rope(g["qkv"][:, :qd].reshape(1, nq, d), np.array([[float(pos)]]), shape.rope_theta).reshape(1, -1), what="q_rot")
+    # the row appended at `pos`: the fp16 rounding of the rotated key / of the value the library itself computed
+    k_new = O.rope(g["qkv"][:, qd:qd + kvd].reshape(1, nkv, d), np.array([[float(pos)]]), shape.rope_theta).reshape(nkv, d)
+    ulp = lambda r: np.spacing(np.abs(r).astype(np.float16)).astype(np.float64)
+    assert np.all(np.abs(kg[:, pos].astype(np.float64) - k_new) <= ulp(k_new))  # fp32 rotation vs fp64: at most the neighbouring fp16
+    assert np.array_equal(vg[:, pos], g["qkv"][:, qd + kvd:].reshape(nkv, d).astype(np.float32).astype(np.float16))
+    assert np.array_equal(np.delete(kg, pos, axis=1), np.delete(kc, pos, axis=1)) and np.array_equal(np.delete(vg, pos, axis=1), np.delete(vc, pos, axis=1))
+    a = O.attention_one(g["q_rot"].reshape(nq, d), kg, vg, pos + 1).reshape(1, -1)
+    H.assert_close(g["a"], O.rn16(a), what="attention")
+    o = gemv_stage(g["x1"] - x64, g["a"], "wo", "wo (x1 - x)")
+    H.assert_close(g["x1"], x64 + o, what="x1")
+    H.assert_close(g["h2"], O.rn16(O.rmsnorm(g["x1"], t["ffn_norm"], shape.rms_eps)), what="h2")
+    gate = O.dequantize(*t["w_gate"]) @ g["h2"].reshape(-1)
+    up = O.dequantize(*t["w_up"]) @ g["h2"].reshape(-1)
+    H.assert_close(g["act"], O.rn16(O.silu(gate) * up).reshape(1, -1), what="swiglu(gate, up)")
+    dn = O.dequantize(*t["w_down"]) @ g["act"].reshape(-1)
+    H.assert_close(yg, O.rn16(g["x1"] + dn.reshape(1, -1)), what="x1 + w_down act")
+    kc2, vc2 = kc.copy(), vc.copy()
+    want = O.dense_layer(x, t, shape, kc2, vc2, pos, edges, wmode)
+    end_to_end = H.error_measures(yg, want)
+    assert np.all(np.isfinite(yg.astype(np.float64)))
+    print(f"decode layer, gains ~N(0, {gain_std}): end-to-end normwise error {end_to_end[0]:.2e}, mixed elementwise ratio {end_to_end[1]:.2f}")
+
+
 @pytest.mark.parametrize("M", [1, 3])
 def test_dense_layer_fp16_weights_decode_matches_oracle(B, torch, M):
     """A dense layer whose seven matrices are unquantized fp16 (the FP16 model of Section 5.1): the decode step with

@@ -224,11 +224,14 @@ def make_stack_ctx(B, shape, cap, T, n_layers):
     return B.Context(arena, workspace_bytes=ws)
 
 
-def test_prefill_layer_stage_by_stage_full_size(B, torch):
+@pytest.mark.parametrize("gain_std", [W.DENSE_GAIN_STD, 1.0])
+def test_prefill_layer_stage_by_stage_full_size(B, torch, gain_std):
     """Config 3 (512 tokens through the full-size layer), every kernel on its own: each stage's output is compared with the
-    oracle's definition of that stage applied to the inputs the stage actually consumed, under both error gates."""
+    oracle's definition of that stage applied to the inputs the stage actually consumed, under both error gates.  Once with
+    the norm gains the other full-size tests use and once with gains ~N(0, 1), which make every intermediate four times
+    larger; the end-to-end error of the layer is reported, not gated, in this test."""
     shape, cfg, T, cap = W.DENSE_FULL, 3, 512, 512
-    L = W.dense_layer(cfg, 0, shape)
+    L = W.dense_layer(cfg, 0, shape, gain_std)
     t = H.oracle_dense_tensors(L)
     ctx = prefill_ctx(B, shape, cap, T, ALL_GPU)
     desc, ids = H.register_dense_layer(ctx, L, 0, cap)
@@ -242,6 +245,7 @@ def test_prefill_layer_stage_by_stage_full_size(B, torch):
     g = {n: ctx.debug_prefill_buffer(desc, T, i).astype(np.float64)
          for i, n in enumerate(("h", "qkv", "q_rot", "a", "o", "x1", "h2", "gu", "act", "d"))}
     yg, kg, vg = y.cpu().numpy(), kd.cpu().numpy(), vd.cpu().numpy()
+    e_pre, w_pre = ctx.numerics(B.ATS_MODE_PREFILL)
     ctx.close()
     nq, nkv, d, ffn = shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn
     qd, kvd = nq * d, nkv * d
@@ -264,6 +268,11 @@ def test_prefill_layer_stage_by_stage_full_size(B, torch):
     H.assert_close(g["act"], O.rn16(O.silu(g["gu"][:, :ffn]) * g["gu"][:, ffn:]), what="swiglu")
     H.assert_close(g["d"], O.linear(g["act"], *t["w_down"], F16, round_out=True), what="w_down")
     assert np.array_equal(yg.astype(np.float64), O.rn16(g["x1"] + g["d"]))
+    kc2, vc2 = W.kv_cache(cfg, 0, shape.n_kv_heads, cap, shape.head_dim, 0)
+    want = O.dense_layer(x, t, shape, kc2, vc2, 0, e_pre, w_pre)
+    end_to_end = H.error_measures(yg, want)
+    assert np.all(np.isfinite(yg.astype(np.float64)))
+    print(f"prefill layer, gains ~N(0, {gain_std}): end-to-end normwise error {end_to_end[0]:.2e}, mixed elementwise ratio {end_to_end[1]:.2f}")
 
 
 # ------------------------------------------------------------------------------------------------- MoE prefill
