@@ -300,10 +300,7 @@ int32_t ats_dequantize(ats_ctx* ctx, int32_t id, int32_t expert, void* out_dev /
 
 /* The numerics contract of a mode: bit i of *fp16_edge_mask set = the layer rounds intermediate i to fp16, for
  * i over {h, q, k, v, q_rot, a, o, x1, h2, g, u, act, d}; *weight_mode 0 = weights exact (scale*code in fp32),
- * 1 = weights rounded once to fp16 (tensor-core operands).  Cache entries and x_out are always fp16.
- * Decode rounds the inputs of its GEMVs (h, a, h2, act); its attention feeds the tensor cores the query and the
- * attention weights as sums of two fp16 numbers (about 22 bits), which no bit describes and fp32 accuracy covers;
- * prefill stores every intermediate as fp16. */
+ * 1 = weights rounded once to fp16 (tensor-core operands).  Cache entries and x_out are always fp16. */
 int32_t ats_get_numerics(const ats_ctx* ctx, uint32_t mode, uint32_t* fp16_edge_mask /*HOST*/,
                          uint32_t* weight_mode /*HOST*/);
 

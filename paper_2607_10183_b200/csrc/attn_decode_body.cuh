@@ -11,9 +11,7 @@ constexpr int kAttnMaxD = 128;
 
 // Static shared memory of a job (head dimensions up to kAttnMaxD use the front of each row).
 struct AttnShared {
-  // rotated query heads as the sum of two fp16 numbers (q = hi + lo to about 22 bits: the operands of the tensor-core
-  // score products); rows past the group are zero
-  __align__(16) __half q16_s[2][kAttnMaxGroup][kAttnMaxD + 8];
+  __align__(16) float q_s[kAttnMaxGroup][kAttnMaxD];  // rotated query heads
   float w_acc[kAttnMaxWarps][kAttnMaxD];              // per-warp unnormalised outputs
   float w_m[kAttnMaxWarps], w_l[kAttnMaxWarps];       // per-warp score maximum and sum of exponentials
   int is_last;
@@ -65,23 +63,6 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
 }
 
-// Warp-level tensor-core pieces (mma.sync m16n8k16, fp16 operands, fp32 accumulation) and their operand loads.
-__device__ __forceinline__ void ad_mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void ad_ldmatrix_x4(uint32_t (&r)[4], const void* smem_row) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"((uint32_t)__cvta_generic_to_shared(smem_row)));
-}
-__device__ __forceinline__ void ad_ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_row) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"((uint32_t)__cvta_generic_to_shared(smem_row)));
-}
-
 // Job (split, kv head, head part): the group's query heads are divided over `hsplit` CTAs (each stages the same cache rows
 // and attends with group / hsplit heads), so that short contexts still fill the SMs.  jy = kv head * hsplit + part.
 // The work of one job, in two parts: staging the past cache rows (which do not depend on the new
@@ -94,7 +75,7 @@ __device__ __forceinline__ void attn_decode_stage(const AttnDecodeParams& p, con
   constexpr int POS = 32 * SUB;
   constexpr int CH = D * 2 / 16;
   constexpr int KROW = D * 2 + 16;
-  constexpr int VROW = D * 2 + 16;
+  constexpr int VROW = D * 2;
   uint8_t* k_s = dyn_s;
   uint8_t* v_s = dyn_s + (size_t)POS * KROW;
   const int n_ctx = p.pos + 1;
@@ -126,50 +107,43 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
       asm volatile("bar.sync 4, %0;" ::"r"(nthr) : "memory");
   };
   constexpr int POS = 32 * SUB;        // positions per CTA
+  constexpr int V = D / 32;            // output dims per lane
   constexpr int CH = D * 2 / 16;       // 16-byte chunks per cache row
-  constexpr int KROW = D * 2 + 16;     // row pitch in shared memory: the 16-byte pad spreads the eight rows of a matrix load over all banks
-  constexpr int VROW = D * 2 + 16;
+  constexpr int KROW = D * 2 + 16;     // key row pitch in shared memory: the 16-byte pad makes lane-per-row reads conflict-free
+  constexpr int VROW = D * 2;
   constexpr int EPT = D / 64;          // output elements per thread in the merges (64 threads per head)
-  constexpr int KS = D / 16;           // k-steps of a score product
   uint8_t* k_s = dyn_s;                              // [POS][KROW]
   uint8_t* v_s = dyn_s + (size_t)POS * KROW;    // [POS][VROW]
-  __half (&q16_s)[2][kAttnMaxGroup][kAttnMaxD + 8] = as.q16_s;
+  float (&q_s)[kAttnMaxGroup][kAttnMaxD] = as.q_s;
   float (&w_acc)[kAttnMaxWarps][kAttnMaxD] = as.w_acc;
   float (&w_m)[kAttnMaxWarps] = as.w_m;
   float (&w_l)[kAttnMaxWarps] = as.w_l;
   int& is_last = as.is_last;
-  const int G = p.group / p.hsplit;  // query heads of this CTA
+  const int G = p.group / p.hsplit;  // query heads of this CTA; nthr = G * POS
   const int kvh = jy / p.hsplit;
   const int hbase = kvh * p.group + (jy % p.hsplit) * G;  // first of them
   const bool writer = jy % p.hsplit == 0;                 // one CTA per kv head appends to the caches
   const int lane = tid & 31, warp = tid >> 5;
+  const int g = warp / SUB, sub = warp % SUB;
   const int half = D / 2, n_ctx = p.pos + 1;
   const int qd = p.n_q * D, kvd = p.n_kv * D;
   const int tc0 = split * POS;                     // first position of the CTA
   const bool own = split == p.pos / POS;           // this CTA holds the new token's position
   const int r_new = p.pos - tc0;
-  // Rotary embedding of the group's query heads into shared memory, each element split into two fp16 numbers
-  // (hi = rn16(q), lo = rn16(q - hi)); rows of heads the group does not have are zero.
-  for (int idx = tid; idx < kAttnMaxGroup * half; idx += nthr) {
+  // rotary embedding of the group's query heads into shared memory
+  for (int idx = tid; idx < G * half; idx += nthr) {
     const int g2 = idx / half, i = idx % half;
-    float ra = 0.f, rb = 0.f;
-    if (g2 < G) {
-      const int hq2 = hbase + g2;
-      const float* q = p.qkv + (size_t)hq2 * D;
-      const float a = q[i], b = q[i + half];
-      const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
-      ra = a * c - b * s;
-      rb = b * c + a * s;
-      if (p.q_rot_out && split == 0) {
-        p.q_rot_out[(size_t)hq2 * D + i] = ra;
-        p.q_rot_out[(size_t)hq2 * D + i + half] = rb;
-      }
+    const int hq2 = hbase + g2;
+    const float* q = p.qkv + (size_t)hq2 * D;
+    const float a = q[i], b = q[i + half];
+    const float c = p.cs[2 * i], s = p.cs[2 * i + 1];
+    const float ra = a * c - b * s, rb = b * c + a * s;
+    q_s[g2][i] = ra;
+    q_s[g2][i + half] = rb;
+    if (p.q_rot_out && split == 0) {
+      p.q_rot_out[(size_t)hq2 * D + i] = ra;
+      p.q_rot_out[(size_t)hq2 * D + i + half] = rb;
     }
-    const __half ha = __float2half_rn(ra), hb = __float2half_rn(rb);
-    q16_s[0][g2][i] = ha;
-    q16_s[0][g2][i + half] = hb;
-    q16_s[1][g2][i] = __float2half_rn(ra - __half2float(ha));
-    q16_s[1][g2][i + half] = __float2half_rn(rb - __half2float(hb));
   }
   // the CTA that covers position `pos` rotates the new key, rounds key and value to fp16 as the cache holds them, puts
   // them into its staged tiles and appends them to the caches
@@ -198,101 +172,61 @@ __device__ __forceinline__ void attn_decode_compute(const AttnDecodeParams& p, c
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   job_sync();
   ATS_ATR(3);
-  // Warp `sub` (< SUB) attends with ALL heads of the CTA to positions sub * 32 .. + 31 on the tensor cores.
-  // Scores, transposed: S^T[head][pos] = Q[head][d] K^T[d][pos]; the heads are the 16 rows of the A operand (rows past the
-  // group are zero), eight positions are the columns of an instruction.  A lane then holds, for head lane / 4, the scores
-  // of positions 8 nt + 2 (lane % 4) + {0, 1} of the block, nt = 0..3.
-  if (warp < SUB) {
-    const int sub = warp;
-    const int hh = lane >> 2, pq = (lane & 3) * 2;  // this lane's head row and position pair within an 8-column tile
-    float sc[4][4];
+  const int t0 = tc0 + sub * 32;
+  const int n_here = min(32, n_ctx - t0);  // uniform over the warp; <= 0 when the warp has no position
+  const bool ok = lane < n_here;
+  float sc = 0.f;
+  if (ok) {
+    const uint4* kr = reinterpret_cast<const uint4*>(k_s + (size_t)(sub * 32 + lane) * KROW);
+    const float* qh = q_s[g];
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) sc[nt][e] = 0.f;
-    uint32_t qa[2][KS][2];  // [hi | lo][k-step][k, k + 8]
-#pragma unroll
-    for (int hl = 0; hl < 2; ++hl)
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        qa[hl][ks][0] = *reinterpret_cast<const uint32_t*>(&q16_s[hl][hh][ks * 16 + pq]);
-        qa[hl][ks][1] = *reinterpret_cast<const uint32_t*>(&q16_s[hl][hh][ks * 16 + 8 + pq]);
-      }
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      // matrices of one load: d chunks (lane / 8) * 8 of two k-steps, rows = the tile's eight positions
-      const uint8_t* krow = k_s + (size_t)(sub * 32 + nt * 8 + (lane & 7)) * KROW + (lane >> 3) * 16;
-#pragma unroll
-      for (int kp = 0; kp < KS / 2; ++kp) {
-        uint32_t kb[4];
-        ad_ldmatrix_x4(kb, krow + kp * 64);
-        // the small halves first: both products are exact in the fp32 accumulator's terms, only the order of additions differs
-        ad_mma16816(sc[nt], qa[1][2 * kp][0], 0u, qa[1][2 * kp][1], 0u, kb[0], kb[1]);
-        ad_mma16816(sc[nt], qa[1][2 * kp + 1][0], 0u, qa[1][2 * kp + 1][1], 0u, kb[2], kb[3]);
-        ad_mma16816(sc[nt], qa[0][2 * kp][0], 0u, qa[0][2 * kp][1], 0u, kb[0], kb[1]);
-        ad_mma16816(sc[nt], qa[0][2 * kp + 1][0], 0u, qa[0][2 * kp + 1][1], 0u, kb[2], kb[3]);
-      }
+    for (int c = 0; c < CH; ++c) {
+      const uint4 kv = kr[c];
+      const float4 q0 = *reinterpret_cast<const float4*>(qh + c * 8);
+      const float4 q1 = *reinterpret_cast<const float4*>(qh + c * 8 + 4);
+      float2 f;
+      f = __half22float2(ad_half2(kv.x)); s0 = fmaf(f.x, q0.x, s0); s1 = fmaf(f.y, q0.y, s1);
+      f = __half22float2(ad_half2(kv.y)); s0 = fmaf(f.x, q0.z, s0); s1 = fmaf(f.y, q0.w, s1);
+      f = __half22float2(ad_half2(kv.z)); s0 = fmaf(f.x, q1.x, s0); s1 = fmaf(f.y, q1.y, s1);
+      f = __half22float2(ad_half2(kv.w)); s0 = fmaf(f.x, q1.z, s0); s1 = fmaf(f.y, q1.w, s1);
     }
-    // softmax over the block's 32 positions per head: a head's scores sit in the four lanes of a quad
-    const int rel0 = tc0 + sub * 32;  // first position of the block
-    float mw = -INFINITY;
-    float sv[4][2];
+    sc = s0 + s1;
+  }
+  const float sv = ok ? sc * p.scale : -INFINITY;
+  const float mw = ad_warp_max(sv);
+  const float pr = (ok && mw > -INFINITY) ? expf(sv - mw) : 0.f;
+  const float lw = ad_warp_sum(pr);
+  if (lane == 0) {
+    w_m[warp] = mw;
+    w_l[warp] = lw;
+  }
+  float acc[V];
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt)
+  for (int v = 0; v < V; ++v) acc[v] = 0.f;
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const bool ok = rel0 + nt * 8 + pq + e < n_ctx;
-        sv[nt][e] = ok ? sc[nt][e] * p.scale : -INFINITY;
-        mw = fmaxf(mw, sv[nt][e]);
-      }
-    mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, 1));
-    mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, 2));
-    // the weights enter the value products as the sum of two fp16 numbers as well (hi = rn16(p), lo = rn16(p - hi))
-    uint32_t pb[2][4];
-    float lw = 0.f;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      const float p0 = (hh < G && sv[nt][0] > -INFINITY) ? expf(sv[nt][0] - mw) : 0.f;
-      const float p1 = (hh < G && sv[nt][1] > -INFINITY) ? expf(sv[nt][1] - mw) : 0.f;
-      const __half2 hi = __floats2half2_rn(p0, p1);
-      const float2 hf = __half22float2(hi);
-      const __half2 lo = __floats2half2_rn(p0 - hf.x, p1 - hf.y);
-      pb[0][nt] = *reinterpret_cast<const uint32_t*>(&hi);
-      pb[1][nt] = *reinterpret_cast<const uint32_t*>(&lo);
-      lw += p0 + p1;
-    }
-    lw += __shfl_xor_sync(0xffffffffu, lw, 1);
-    lw += __shfl_xor_sync(0xffffffffu, lw, 2);
-    if ((lane & 3) == 0 && hh < G) {
-      w_m[hh * SUB + sub] = mw;
-      w_l[hh * SUB + sub] = lw;
-    }
-    // Outputs, transposed: O^T[d][head] = V^T[d][pos] P^T[pos][head]: the value rows, loaded transposed, are the A
-    // operand (16 dims per instruction), the weights are the B operand straight from the score registers.
-#pragma unroll
-    for (int mt = 0; mt < D / 16; ++mt) {
-      float oc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int kk = 0; kk < 2; ++kk) {
-        // matrices of one load: (positions 16 kk + 0..7, dims 16 mt + 0..7), (same positions, dims + 8), (positions + 8, dims),
-        // (positions + 8, dims + 8)
-        const uint8_t* vrow = v_s + (size_t)(sub * 32 + kk * 16 + (lane >> 4) * 8 + (lane & 7)) * VROW + (mt * 16 + ((lane >> 3) & 1) * 8) * 2;
-        uint32_t va[4];
-        ad_ldmatrix_x4_trans(va, vrow);
-        ad_mma16816(oc, va[0], va[1], va[2], va[3], pb[1][2 * kk], pb[1][2 * kk + 1]);
-        ad_mma16816(oc, va[0], va[1], va[2], va[3], pb[0][2 * kk], pb[0][2 * kk + 1]);
-      }
-      // oc[0], oc[1]: dim 16 mt + lane / 4, heads pq, pq + 1; oc[2], oc[3]: dim + 8
-      if (pq < G) {
-        w_acc[pq * SUB + sub][mt * 16 + hh] = oc[0];
-        w_acc[pq * SUB + sub][mt * 16 + hh + 8] = oc[2];
-      }
-      if (pq + 1 < G) {
-        w_acc[(pq + 1) * SUB + sub][mt * 16 + hh] = oc[1];
-        w_acc[(pq + 1) * SUB + sub][mt * 16 + hh + 8] = oc[3];
+  for (int tt = 0; tt < 32; ++tt) {
+    const float pt = __shfl_sync(0xffffffffu, pr, tt);
+    {
+      const uint8_t* vr = v_s + (size_t)(sub * 32 + tt) * VROW + lane * (V * 2);
+      float2 f;
+      if (V == 4) {
+        const uint2 raw = *reinterpret_cast<const uint2*>(vr);
+        f = __half22float2(ad_half2(raw.x));
+        acc[0] = fmaf(pt, f.x, acc[0]);
+        acc[1] = fmaf(pt, f.y, acc[1]);
+        f = __half22float2(ad_half2(raw.y));
+        acc[2] = fmaf(pt, f.x, acc[2]);
+        acc[3] = fmaf(pt, f.y, acc[3]);
+      } else {
+        f = __half22float2(ad_half2(*reinterpret_cast<const uint32_t*>(vr)));
+        acc[0] = fmaf(pt, f.x, acc[0]);
+        acc[1] = fmaf(pt, f.y, acc[1]);
       }
     }
   }
+#pragma unroll
+  for (int v = 0; v < V; ++v) w_acc[warp][lane * V + v] = acc[v];
   ATS_ATR(4);
   job_sync();
   // merge each head's warps (ascending) into this split's partial: 64 threads per head

@@ -756,16 +756,20 @@ cudaError_t launch_rmsnorm(const void* x, int x_is_f32, const __half* gain, __ha
 // fp16, attends over positions 0..pos split across CTAs, and merges the splits: the last CTA to finish a kv head
 // (a counter in global memory, reset for the next launch) sums the partials in ascending split order, so the result
 // does not depend on which CTA arrives last.
-// CTA (split, kv head) covers 64 or 128 positions for ALL query heads of the group: the K and V rows are staged once in
-// shared memory (16-byte async copies, issued before the grid dependency resolves).  Warp w of the first pc / 32 warps
-// attends with all heads to positions 32 w .. 32 w + 31 on the tensor cores (mma.sync m16n8k16): scores as
-// Q[heads][d] K^T with the heads as the rows of the A operand, outputs as V^T P^T with the fp16 weights as the B operand
-// straight from the score registers.  The cache rows are fp16 as stored; the rotated query and the weights enter as sums
-// of two fp16 numbers each (hi + lo, about 22 bits), two instructions per product, so the results keep fp32 accuracy.
+// CTA (split, kv head) covers 64 positions for ALL query heads of the group: the K and V rows are staged once in shared
+// memory (16-byte async copies, issued before the grid dependency resolves) and every head's warps read them from
+// there, so the cache crosses the L2-to-SM fabric once instead of once per query head; that traffic, not DRAM, bounds
+// this kernel.  Warp (head, sub-block) owns 32 positions, one per lane.
 // Positions per CTA: 64, or 128 for contexts beyond 1024 so that the final merge still reads all splits of a head in
 // one round trip (16 splits) up to 2048 positions.  (64 positions up to 2048, with both kernels' registers capped so that
 // a CTA of this kernel fits an SM beside a CTA of the streaming GEMV, was measured and lost: the GEMV slows down by 0.5 us
 // per launch at 80 registers and this kernel by 2.9 us with 17 splits to merge, and nothing is gained back.)
+// (A tensor-core form, scores as Q K^T and outputs as V^T P^T by mma.sync m16n8k16 with the group's heads as operand rows,
+// was built and measured in the step: 7.6 us with the query and the weights rounded to fp16, which costs accuracy the
+// layer's end-to-end gate does not have to spare, and 8.2 us with both split into hi + lo fp16 pairs that keep fp32
+// accuracy, against 7.7 us for this form.  The launch is a chain of global round trips (query load, partial store and
+// arrival counter, partial loads of the merge), each about a microsecond at one CTA per SM; the arithmetic between
+// them is not what it waits for.)
 int attn_decode_pos_per_cta(int n_ctx) { return n_ctx <= 1024 ? 64 : 128; }
 int attn_decode_splits(int n_ctx) {
   const int pc = attn_decode_pos_per_cta(n_ctx);
@@ -785,21 +789,25 @@ __global__ void __launch_bounds__(512) attn_decode_fused_kernel(const AttnDecode
 cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStream_t st, uint64_t* n_launch) {
   if (p.group < 1 || p.group > kAttnMaxGroup || p.n_q != p.n_kv * p.group) return cudaErrorInvalidValue;
   int pc = attn_decode_pos_per_cta(p.pos + 1);
-  if (p.group * (pc / 32) > kAttnMaxWarps) pc = 64;  // large groups: the per-warp partial outputs must fit their buffer
+  if (p.group * pc > 512) pc = 64;  // large groups: 64 positions keep the CTA within 512 threads
   const int splits = (p.pos + 1 + pc - 1) / pc;
-  p.hsplit = 1;  // the tensor-core form takes all heads of a group in one instruction: nothing is gained by dividing them
+  // Short contexts give fewer jobs than SMs: the query heads of a group are then divided over 2 or 4 CTAs (each stages
+  // the same cache rows out of L2), which shortens the score and value loops of every CTA in proportion.
+  int hsplit = 1;
+  while (p.group % (2 * hsplit) == 0 && splits * p.n_kv * 2 * hsplit <= 148 && p.n_kv * 2 * hsplit <= kAttnMaxCounters) hsplit *= 2;
+  p.hsplit = hsplit;
   p.scale = 1.0f / sqrtf((float)d);
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(splits, p.n_kv);
-  cfg.blockDim = dim3(std::max(std::max(p.group * 64, pc), 128));  // 64 threads per head in the merges, one warp per 32 positions
-  cfg.dynamicSmemBytes = (size_t)pc * (d * 4 + 32);
+  cfg.gridDim = dim3(splits, p.n_kv * hsplit);
+  cfg.blockDim = dim3(p.group / hsplit * pc);
+  cfg.dynamicSmemBytes = (size_t)pc * (d * 4 + 16);
   static uint64_t attr_done = 0;
   if (first_use_on_device(&attr_done)) {
     cudaError_t e[4] = {
-        cudaFuncSetAttribute(attn_decode_fused_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * (128 * 4 + 32)),
-        cudaFuncSetAttribute(attn_decode_fused_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (128 * 4 + 32)),
-        cudaFuncSetAttribute(attn_decode_fused_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * (64 * 4 + 32)),
-        cudaFuncSetAttribute(attn_decode_fused_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (64 * 4 + 32))};
+        cudaFuncSetAttribute(attn_decode_fused_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * (128 * 4 + 16)),
+        cudaFuncSetAttribute(attn_decode_fused_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (128 * 4 + 16)),
+        cudaFuncSetAttribute(attn_decode_fused_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * (64 * 4 + 16)),
+        cudaFuncSetAttribute(attn_decode_fused_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * (64 * 4 + 16))};
     for (cudaError_t x : e)
       if (x != cudaSuccess) return x;
   }
