@@ -360,9 +360,11 @@ int32_t ats_debug_fail_copies(ats_ctx* ctx, uint32_t n);
  * next ats_sync (or ats_layer_decode_host) then returns ATS_ERR_TIMEOUT and the context is poisoned; other contexts of the
  * process are unaffected.  Applies to dense single-token GEMV launches only (ats_linear with M = 1, ats_layer_decode). */
 int32_t ats_debug_gemv_wait(ats_ctx* ctx, uint64_t limit_cycles, int32_t withhold_tile);
-/* Timing hook: ats_layer_decode on a dense layer leaves out the launches whose bit is set (1 = QKV GEMV, 2 = attention,
- * 4 = O GEMV, 8 = gate/up GEMV, 16 = down GEMV); the outputs of such a call are stale.  0 restores the full step.  Used by
- * the benchmark to time the GEMV launches of a step without the attention launch between them. */
+/* Timing hook: ats_layer_decode leaves out the launches whose bit is set (dense layers: 1 = QKV GEMV, 2 = attention,
+ * 4 = O GEMV, 8 = gate/up GEMV, 16 = down GEMV; routed-expert FFN with every expert resident: 32 = router, 64 = experts'
+ * gate/up stage, 128 = experts' down stage, 256 = gated sum; the skipped router leaves the ids of an earlier call in
+ * place, so run one full call first); the outputs of such a call are stale.  0 restores the full step.  Used by the
+ * benchmark to time the GEMV launches of a step without the attention launch between them. */
 int32_t ats_debug_skip_stages(ats_ctx* ctx, uint32_t mask);
 
 /* The two ends of a whole-model loop around the layer calls (Section 5's workloads run whole models).

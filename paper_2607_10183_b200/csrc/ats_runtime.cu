@@ -1449,9 +1449,11 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   // ---- MoE FFN
   const int k = (int)L->top_k, P = (int)M * k, E = (int)L->n_experts;
   // the FFN norm runs inside the router launch; the normalised rows land in h2_16 for the expert kernels
-  ATS_CUDA(launch_router_topk_norm(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)M, H, E, k,
-                                   (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, attn ? (const void*)w.x1_32 : x_in,
-                                   attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, L->rms_eps, ctx->cs, nl, pdl));
+  const uint32_t mskip = ctx->dbg_skip;  // timing hook: 32 router, 64 gate/up stage, 128 down stage, 256 combine
+  if (!(mskip & 32))
+    ATS_CUDA(launch_router_topk_norm(w.h2_16, (const __half*)ctx->tensors[L->router].f16_dev, (int)M, H, E, k,
+                                     (L->flags & ATS_LAYER_NO_TOPK_RENORM) ? 0 : 1, w.ids, w.gates, attn ? (const void*)w.x1_32 : x_in,
+                                     attn ? 1 : 0, (const __half*)ctx->tensors[L->ffn_norm].f16_dev, L->rms_eps, ctx->cs, nl, pdl));
   const Tensor &tg = ctx->tensors[L->w_gate], &tu = ctx->tensors[L->w_up], &td = ctx->tensors[L->w_down];
   bool implicit = tg.contiguous_dev && tu.contiguous_dev && td.contiguous_dev;
   if (!implicit && M == 1 && !(ctx->cfg.flags & ATS_FLAG_MOE_RING_ONLY) && tg.slice_tab_dev && tu.slice_tab_dev && td.slice_tab_dev) {
@@ -1543,7 +1545,7 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   s1.y16 = w.act16;
   s1.ldy = (int)L->ffn;
   s1.mode = GEMV_SWIGLU_F16;
-  ATS_TRY(run_moe_stage(ctx, L->w_gate, L->w_up, w.ids, ids_host, s1, call_tab[0], call_tab[1]));
+  if (!(mskip & 64)) ATS_TRY(run_moe_stage(ctx, L->w_gate, L->w_up, w.ids, ids_host, s1, call_tab[0], call_tab[1]));
   MoeGemvParams s2{};
   s2.P = P;
   s2.x_div = 1;
@@ -1552,8 +1554,9 @@ int32_t ats_layer_decode(ats_ctx* ctx, const ats_layer_desc* L, const void* x_in
   s2.y32 = w.d32;
   s2.ldy = H;
   s2.mode = GEMV_OUT_F32;
-  ATS_TRY(run_moe_stage(ctx, L->w_down, -1, w.ids, ids_host, s2, call_tab[2], nullptr));
-  ATS_CUDA(launch_moe_combine(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, w.gates, w.d32, (__half*)x_out, (int)M, k, H,
+  if (!(mskip & 128)) ATS_TRY(run_moe_stage(ctx, L->w_down, -1, w.ids, ids_host, s2, call_tab[2], nullptr));
+  if (!(mskip & 256))
+    ATS_CUDA(launch_moe_combine(attn ? (const void*)w.x1_32 : x_in, attn ? 1 : 0, w.gates, w.d32, (__half*)x_out, (int)M, k, H,
                               ctx->cs, nl, pdl));
   return ATS_OK;
 }
@@ -2031,7 +2034,7 @@ int32_t ats_debug_gemv_wait(ats_ctx* ctx, uint64_t limit_cycles, int32_t withhol
 }
 
 int32_t ats_debug_skip_stages(ats_ctx* ctx, uint32_t mask) {
-  if (!ctx || mask > 31u) return ATS_ERR_INVALID;
+  if (!ctx || mask > 511u) return ATS_ERR_INVALID;
   ctx->dbg_skip = mask;
   return ATS_OK;
 }

@@ -901,6 +901,64 @@ __device__ __forceinline__ void router_select(const float* logit, int m, int E, 
   }
 }
 
+// The same selection for up to 256 experts by counting, all threads of the CTA at once: the rank of a logit is the number
+// of logits that come before it in the order (larger value first, equal values: lower index first; NaN as -inf), so the
+// expert of rank r < k is the r-th selection of router_select; warp 0 then forms the gates with router_select's own
+// arithmetic.  sel_v / sel_i: k entries of shared memory.  Called by every thread of the CTA.
+__device__ __forceinline__ void router_select_counting(const float* logit, int m, int E, int Epad, int k, int renorm,
+                                                       int32_t* __restrict__ ids, float* __restrict__ gates, float* sel_v, int* sel_i) {
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    const float vr = logit[e];
+    const float v = vr == vr ? vr : -INFINITY;
+    int rank = 0;
+    for (int j = 0; j < E; j += 4) {  // E is a multiple of 8 here
+      const float4 o = *reinterpret_cast<const float4*>(logit + j);
+      const float o0 = o.x == o.x ? o.x : -INFINITY, o1 = o.y == o.y ? o.y : -INFINITY;
+      const float o2 = o.z == o.z ? o.z : -INFINITY, o3 = o.w == o.w ? o.w : -INFINITY;
+      rank += (o0 > v || (o0 == v && j < e)) + (o1 > v || (o1 == v && j + 1 < e)) + (o2 > v || (o2 == v && j + 2 < e)) +
+              (o3 > v || (o3 == v && j + 3 < e));
+    }
+    if (rank < k) {
+      sel_v[rank] = v;
+      sel_i[rank] = e;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  const int lane = threadIdx.x;
+  const int per = Epad / 32;
+  bool has_nan = false;
+  for (int j = 0; j < per; ++j) {
+    const float v = logit[lane + 32 * j];
+    has_nan |= (lane + 32 * j < E) && (v != v);
+  }
+  has_nan = __any_sync(0xffffffffu, has_nan);
+  const float my_v = lane < k ? sel_v[lane] : 0.f;
+  float gate;
+  if (renorm) {
+    const float mx = __shfl_sync(0xffffffffu, my_v, 0);
+    const float ex = lane < k ? expf(my_v - mx) : 0.f;
+    const float s = warp_sum(ex);
+    gate = ex / s;
+  } else {
+    float mx = -INFINITY;
+    for (int j = 0; j < per; ++j) mx = fmaxf(mx, logit[lane + 32 * j]);
+    mx = warp_max(mx);
+    float t = 0.f;
+    for (int j = 0; j < per; ++j) {
+      const float v = logit[lane + 32 * j];
+      t += v > -INFINITY ? expf(v - mx) : 0.f;
+    }
+    const float total = warp_sum(t);
+    gate = lane < k ? expf(my_v - mx) / total : 0.f;
+  }
+  if (has_nan) gate = __int_as_float(0x7FC00000);
+  if (lane < k) {
+    ids[(size_t)m * k + lane] = sel_i[lane];
+    gates[(size_t)m * k + lane] = gate;
+  }
+}
+
 constexpr int kRouterThreads = 1024;
 
 __global__ void __launch_bounds__(kRouterThreads) router_topk_kernel(const __half* __restrict__ h, const __half* __restrict__ wr,
@@ -973,17 +1031,37 @@ __global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(c
   float* cl = part + (size_t)R * E;           // [kRouterCluster][Epad]   (used in CTA 0)
   float* logit = cl + (size_t)kRouterCluster * Epad;  // [Epad]
   const int m = blockIdx.y;
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // inputs come from the preceding kernel
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t rank = cluster_ctarank();
   const int row0 = (int)rank * Hc;
+  const int grp = threadIdx.x / L, e0 = (threadIdx.x % L) * 8;
+  // The rows of a thread are fetched in batches of 16 loads that are all issued before the first is used: the matrix is
+  // read once at memory latency (a token's 512 KB are 64 KB per CTA, one batch per thread), not once per row.  The
+  // router matrix does not depend on the preceding kernel: the first batch is requested before waiting for it.
+  constexpr int kBatch = 16;
+  uint4 w[kBatch];
+#pragma unroll
+  for (int b = 0; b < kBatch; ++b) {
+    const int i = grp + b * R;
+    w[b] = (grp < R && i < Hc) ? __ldg(reinterpret_cast<const uint4*>(wr + (size_t)(row0 + i) * E + e0)) : make_uint4(0, 0, 0, 0);
+  }
+  // the norm gains of this CTA's rows are parameters too (up to 8 per thread: hidden sizes up to 16384)
+  float gain_pre[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const int i = (int)threadIdx.x + q * kRouterClThreads;
+    gain_pre[q] = (gain && i < Hc) ? __half2float(gain[row0 + i]) : 0.f;
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the token's row comes from the preceding kernel
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (gain) {
+    // every CTA sums the squares of the whole row (a few kilobytes) and normalises its own eighth; the row is read once
     __shared__ float red[kRouterClThreads / 32];
     const __half* x16 = static_cast<const __half*>(xn) + (size_t)m * H;
     const float* x32 = static_cast<const float*>(xn) + (size_t)m * H;
     float ss = 0.f;
     for (int i = threadIdx.x; i < H; i += kRouterClThreads) {
       const float v = xn_f32 ? x32[i] : __half2float(x16[i]);
+      if (i >= row0 && i < row0 + Hc) h_s[i - row0] = v;  // kept for the second pass
       ss = fmaf(v, v, ss);
     }
     ss = warp_sum(ss);
@@ -991,32 +1069,32 @@ __global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(c
     __syncthreads();
     float t = 0.f;
 #pragma unroll
-    for (int w = 0; w < kRouterClThreads / 32; ++w) t += red[w];
+    for (int w2 = 0; w2 < kRouterClThreads / 32; ++w2) t += red[w2];
     const float inv = 1.0f / sqrtf(t / (float)H + eps);
-    for (int i = threadIdx.x; i < Hc; i += kRouterClThreads) {
-      const float v = xn_f32 ? x32[row0 + i] : __half2float(x16[row0 + i]);
-      const __half hv = __float2half_rn(v * __half2float(gain[row0 + i]) * inv);
-      h_s[i] = __half2float(hv);
-      h_out[(size_t)m * H + row0 + i] = hv;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int i = (int)threadIdx.x + q * kRouterClThreads;
+      if (i < Hc) {
+        const __half hv = __float2half_rn(h_s[i] * gain_pre[q] * inv);
+        h_s[i] = __half2float(hv);
+        h_out[(size_t)m * H + row0 + i] = hv;
+      }
     }
   } else {
     for (int i = threadIdx.x; i < Hc; i += kRouterClThreads) h_s[i] = __half2float(h[(size_t)m * H + row0 + i]);
   }
   __syncthreads();
-  const int grp = threadIdx.x / L, e0 = (threadIdx.x % L) * 8;
   float acc[8];
 #pragma unroll
   for (int q = 0; q < 8; ++q) acc[q] = 0.f;
   if (grp < R) {
-    // The rows of a thread are fetched in batches of 16 loads that are all issued before the first is used: the
-    // matrix is read once at memory latency (a token's 512 KB are 64 KB per CTA, one batch per thread), not once per row.
-    constexpr int kBatch = 16;
     for (int i0 = grp; i0 < Hc; i0 += R * kBatch) {
-      uint4 w[kBatch];
+      if (i0 != grp) {
 #pragma unroll
-      for (int b = 0; b < kBatch; ++b) {
-        const int i = i0 + b * R;
-        w[b] = i < Hc ? __ldg(reinterpret_cast<const uint4*>(wr + (size_t)(row0 + i) * E + e0)) : make_uint4(0, 0, 0, 0);
+        for (int b = 0; b < kBatch; ++b) {
+          const int i = i0 + b * R;
+          w[b] = i < Hc ? __ldg(reinterpret_cast<const uint4*>(wr + (size_t)(row0 + i) * E + e0)) : make_uint4(0, 0, 0, 0);
+        }
       }
 #pragma unroll
       for (int b = 0; b < kBatch; ++b) {
@@ -1050,6 +1128,12 @@ __global__ void __launch_bounds__(kRouterClThreads) router_topk_cluster_kernel(c
     logit[e] = e < E ? t : -INFINITY;
   }
   __syncthreads();
+  if (E <= 256) {
+    __shared__ float sel_v[32];
+    __shared__ int sel_i[32];
+    router_select_counting(logit, m, E, Epad, k, renorm, ids, gates, sel_v, sel_i);
+    return;
+  }
   if (threadIdx.x >= 32) return;
   router_select(logit, m, E, Epad, k, renorm, ids, gates);
 }
@@ -1066,7 +1150,7 @@ cudaError_t launch_router_topk_norm(const __half* h, const __half* wr, int M, in
                                     cudaStream_t st, uint64_t* n_launch, int pdl) {
   int Epad = 32;
   while (Epad < E) Epad <<= 1;
-  if (E % 8 == 0 && H % (8 * kRouterCluster) == 0 && (((uintptr_t)wr | (uintptr_t)h) & 15) == 0) {
+  if (E % 8 == 0 && H % (8 * kRouterCluster) == 0 && H <= 8 * kRouterClThreads * kRouterCluster && (((uintptr_t)wr | (uintptr_t)h) & 15) == 0) {
     const int L = E / 8, R = kRouterClThreads / L;
     const size_t smem_cl = ((size_t)H / kRouterCluster + (size_t)R * E + (size_t)(kRouterCluster + 1) * Epad) * sizeof(float);
     if (smem_cl <= 160 * 1024) {
