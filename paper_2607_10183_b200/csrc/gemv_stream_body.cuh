@@ -47,7 +47,13 @@ constexpr int kRPW = 2;      // rows per consumer warp per tile
 constexpr int kJ = 2;        // quantization blocks per lane per row
 constexpr int kMaxDynSmem = 216 * 1024;  // ring + quantized activation row; 7 KB of static shared memory on top
 constexpr int kEarlyStages = 1;  // stages requested before the consumers have issued their activation loads
-constexpr int kMaxIt = 48;   // tiles of a CTA whose partial sums are buffered before a flush
+constexpr int kMaxIt = 48;   // tiles of a CTA whose partial sums are buffered before a flush (at kRPW rows per warp)
+// Short rows (K <= 1024: at most one quantization block per lane): a tile of the default geometry is a few kilobytes and
+// the per-copy cost of the producers, not the memory, sets the pace.  Such shapes take twice the rows per tile, one block
+// per lane, and four producer warps.
+constexpr int kRPWShort = 4, kJShort = 1, kProducerWarpsShort = 4;
+constexpr int kShortK = 1024;
+constexpr int kThreadsShort = kConsumerThreads + 32 * kProducerWarpsShort;
 
 #ifdef ATS_TRACE
 // Timeline probe of development builds (-DATS_TRACE): stamps are collected in shared memory (cheap) and written out as
@@ -285,14 +291,14 @@ __device__ __forceinline__ int stream_n_it(const StreamParams& p, int bx, int gx
 // One elected thread of each producer warp requests tiles; producer warp w of the kProducerWarps takes the CTA's
 // iterations it = w, w + kProducerWarps, ...  Before it refills a stage a producer waits for the PARITY of the phase in
 // which the consumers released the stage's previous content; that test is only unambiguous while no producer runs a whole
-// ring cycle ahead of the consumers, which holds as long as kProducerWarps <= n_stages (a producer's previous iteration
+// ring cycle ahead of the consumers, which holds as long as the number of producer warps (PW) <= n_stages (a producer's previous iteration
 // waited for a release at most one ring cycle older).  bx / gx: index of this CTA among the gx CTAs that share the work described by p.  The weights do not depend
 // on the preceding kernel, so nothing here waits for it (callers whose weight ADDRESSES come from the preceding kernel
 // wait before they call).  Returns false after a bounded wait ran out (status word raised).
-template <int PARTS, bool SW>
+template <int PARTS, bool SW, int RPW = kRPW, int PW = kProducerWarps>
 __device__ __forceinline__ bool stream_produce(const StreamParams& p, const int bx, const int gx, const int pw, StreamShared& sh,
                                                uint8_t* stages, const uint64_t pol) {
-  constexpr int ROWS = kGroupWarps / PARTS * kRPW;     // weight rows per tile
+  constexpr int ROWS = kGroupWarps / PARTS * RPW;     // weight rows per tile
   constexpr int OUT_ROWS = SW ? ROWS / 2 : ROWS;       // output rows per tile
   const int row_codes = p.K / 2, row_scales = p.K / 16;
   const int stage_bytes = ROWS * (row_codes + row_scales);
@@ -303,7 +309,7 @@ __device__ __forceinline__ bool stream_produce(const StreamParams& p, const int 
   bool x_issued = false;
   // stage and ring cycle of iteration it, kept incrementally (the ring size is a run-time value)
   int s = pw % n_stages, cyc = pw / n_stages;
-  for (int it = pw; it < n_it; it += kProducerWarps) {
+  for (int it = pw; it < n_it; it += PW) {
     // Weight copies queued ahead of the consumers' activation loads delay them (the row is a cache hit that then waits
     // behind megabytes of misses): kEarlyStages stages go out at once, the rest after those loads have been issued.
     if (it >= kEarlyStages && !x_issued) {
@@ -322,7 +328,7 @@ __device__ __forceinline__ bool stream_produce(const StreamParams& p, const int 
     mbar_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
     if (pw == 0) ATS_TR(300 + it);
     if (tile == p.withhold_tile) {  // test hook: this stage never fills
-      stream_advance(s, cyc, kProducerWarps, n_stages);
+      stream_advance(s, cyc, PW, n_stages);
       continue;
     }
     if (SW) {
@@ -343,7 +349,7 @@ __device__ __forceinline__ bool stream_produce(const StreamParams& p, const int 
       bulk_g2s(dst, b + r0 * row_codes, ROWS * row_codes, &sh.full[s], pol);
       bulk_g2s(dst + ROWS * row_codes, b + (size_t)p.seg[sg].n_rows * row_codes + r0 * row_scales, ROWS * row_scales, &sh.full[s], pol);
     }
-    stream_advance(s, cyc, kProducerWarps, n_stages);
+    stream_advance(s, cyc, PW, n_stages);
   }
   ATS_TR(9);
   return true;
@@ -366,10 +372,11 @@ __device__ __forceinline__ void unpack_h8(const uint4 a, float (&xv)[8]) {
 // barrier, so the tile loop is that of two independent 8-warp CTAs; what they share is the ring and the activation
 // prologue: all 512 consumer threads load, normalise and quantise the row ONCE per SM.
 // dep_resolved: the caller has already executed griddepcontrol.wait.  The dependent launch is released after the prologue.  Returns false after a bounded wait ran out (status word raised).
-template <int PARTS, bool SW, bool MX>
+template <int PARTS, bool SW, bool MX, int RPW = kRPW, int J = kJ>
 __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int bx, const int gx, StreamShared& sh, const uint8_t* stages,
                                                uint32_t* xq_s, const bool dep_resolved) {
-  constexpr int ROWS = kGroupWarps / PARTS * kRPW;     // weight rows per tile
+  constexpr int ROWS = kGroupWarps / PARTS * RPW;     // weight rows per tile
+  constexpr int MAXIT = kMaxIt * kRPW / RPW;           // tiles whose partial sums fit the buffer
   constexpr int OUT_ROWS = SW ? ROWS / 2 : ROWS;       // output rows per tile
   const int K = p.K, nblk = K / 32;
   const int row_codes = K / 2, row_scales = K / 16;
@@ -385,8 +392,8 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
   const int part = wg % PARTS, rsub = wg / PARTS;
   const int pblk = (nblk + PARTS - 1) / PARTS;
   const int b0 = part * pblk, b1 = min(nblk, b0 + pblk);
-  uint32_t xr[kJ][16];
-  float xm[kJ], xc[kJ];
+  uint32_t xr[J][16];
+  float xm[J], xc[J];
   ATS_TR(0);
   {
     // Thread t owns the runs of 8 consecutive elements r = t + 512 j (one run when K <= 4096, up to four for K = 16384);
@@ -467,7 +474,7 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
     ATS_TR(2);
     consumer_sync_all();
 #pragma unroll
-    for (int j = 0; j < kJ; ++j) {
+    for (int j = 0; j < J; ++j) {
       const int b = b0 + lane + 32 * j;
       if (b < b1) {
         const uint4* src = reinterpret_cast<const uint4*>(xq_s + (size_t)b * kXqWords);
@@ -499,19 +506,19 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
   float* my_part = sh.part_s[grp];
   bool failed = false;
   int s = grp % n_stages, cyc = grp / n_stages;  // stage and ring cycle of the group's next tile
-  auto reduce_store = [&](float (&a)[kRPW], int slot) {
+  auto reduce_store = [&](float (&a)[RPW], int slot) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-      for (int r = 0; r < kRPW; ++r) a[r] += __shfl_xor_sync(0xffffffffu, a[r], o);
+      for (int r = 0; r < RPW; ++r) a[r] += __shfl_xor_sync(0xffffffffu, a[r], o);
     if (lane == 0) {
 #pragma unroll
-      for (int r = 0; r < kRPW; ++r) my_part[(slot * ROWS + r * (ROWS / kRPW) + rsub) * PARTS + part] = a[r];
+      for (int r = 0; r < RPW; ++r) my_part[(slot * ROWS + r * (ROWS / RPW) + rsub) * PARTS + part] = a[r];
     }
   };
-  for (int li0 = 0; li0 < n_li; li0 += kMaxIt) {
-    const int li1 = min(n_li, li0 + kMaxIt);
-    float prev[kRPW];
+  for (int li0 = 0; li0 < n_li; li0 += MAXIT) {
+    const int li1 = min(n_li, li0 + MAXIT);
+    float prev[RPW];
     bool have_prev = false;
     for (int li = li0; li < li1; ++li) {
       [[maybe_unused]] const int it = grp + kGroups * li;
@@ -522,15 +529,15 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
       if (li == 0) ATS_TR(4);
       ATS_TR(100 + it);
       const uint8_t* st = stages + (size_t)s * stage_bytes;
-      uint4 cw[kRPW][kJ];
-      float sc[kRPW][kJ];
+      uint4 cw[RPW][J];
+      float sc[RPW][J];
 #pragma unroll
-      for (int r = 0; r < kRPW; ++r) {
-        const int row = r * (ROWS / kRPW) + rsub;  // stage row of this warp's r-th row
+      for (int r = 0; r < RPW; ++r) {
+        const int row = r * (ROWS / RPW) + rsub;  // stage row of this warp's r-th row
         const uint4* codes = reinterpret_cast<const uint4*>(st + (size_t)row * row_codes);
         const __half* scp = reinterpret_cast<const __half*>(st + (size_t)ROWS * row_codes + (size_t)row * row_scales);
 #pragma unroll
-        for (int j = 0; j < kJ; ++j) {
+        for (int j = 0; j < J; ++j) {
           const int b = b0 + lane + 32 * j;
           const bool in = b < b1;
           cw[r][j] = in ? codes[b] : make_uint4(0, 0, 0, 0);
@@ -543,20 +550,20 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
       {
         uint32_t fold = 0;
 #pragma unroll
-        for (int r = 0; r < kRPW; ++r)
+        for (int r = 0; r < RPW; ++r)
 #pragma unroll
-          for (int j = 0; j < kJ; ++j) fold ^= cw[r][j].x ^ cw[r][j].y ^ cw[r][j].z ^ cw[r][j].w ^ __float_as_uint(sc[r][j]);
+          for (int j = 0; j < J; ++j) fold ^= cw[r][j].x ^ cw[r][j].y ^ cw[r][j].z ^ cw[r][j].w ^ __float_as_uint(sc[r][j]);
         asm volatile("" ::"r"(fold) : "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.empty[s]);
       }
       if (have_prev) reduce_store(prev, li - 1 - li0);
-      float acc[kRPW];
+      float acc[RPW];
 #pragma unroll
-      for (int r = 0; r < kRPW; ++r) {
+      for (int r = 0; r < RPW; ++r) {
         acc[r] = 0.f;
 #pragma unroll
-        for (int j = 0; j < kJ; ++j) {
+        for (int j = 0; j < J; ++j) {
           const uint32_t ws[4] = {cw[r][j].x, cw[r][j].y, cw[r][j].z, cw[r][j].w};
           int dl = 0, dh = 0;
 #pragma unroll
@@ -583,7 +590,7 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
       ATS_TR(200 + it);
       stream_advance(s, cyc, kGroups, n_stages);
 #pragma unroll
-      for (int r = 0; r < kRPW; ++r) prev[r] = acc[r];
+      for (int r = 0; r < RPW; ++r) prev[r] = acc[r];
       have_prev = true;
     }
     if (have_prev && !failed) reduce_store(prev, li1 - 1 - li0);
@@ -635,11 +642,14 @@ __device__ __forceinline__ bool stream_consume(const StreamParams& p, const int 
 
 // ------------------------------------------------------------------ host side: shapes the kernel takes, its parameters
 inline int stream_parts_for(int K) { return K <= 2048 ? 1 : K <= 4096 ? 2 : K <= 8192 ? 4 : 8; }
+inline bool stream_short(int K) { return K <= kShortK; }                       // the wide-tile geometry applies
+inline int stream_rpw_for(int K) { return stream_short(K) ? kRPWShort : kRPW; }
+inline int stream_producers_for(int K) { return stream_short(K) ? kProducerWarpsShort : kProducerWarps; }
 
 inline bool stream_shape_ok(const GemvParams& p) {
   if (p.M != 1 || p.K % 256 != 0 || p.K > 16384) return false;
   const int parts = stream_parts_for(p.K);
-  const int rows = kGroupWarps / parts * kRPW;
+  const int rows = kGroupWarps / parts * stream_rpw_for(p.K);
   if (p.mode == GEMV_SWIGLU_F16) {
     if (p.n_seg != 2 || p.seg[0].n_rows != p.seg[1].n_rows || p.seg[0].n_rows % (rows / 2)) return false;
   } else {
@@ -651,7 +661,7 @@ inline bool stream_shape_ok(const GemvParams& p) {
 }
 
 // Bytes of one ring stage and of the quantized activation row, and the number of stages that fit the SM.
-inline size_t stream_stage_bytes(int K) { return (size_t)(kGroupWarps / stream_parts_for(K) * kRPW) * (K / 2 + K / 16); }
+inline size_t stream_stage_bytes(int K) { return (size_t)(kGroupWarps / stream_parts_for(K) * stream_rpw_for(K)) * (K / 2 + K / 16); }
 inline size_t stream_xq_bytes(int K) { return (size_t)(K / 32) * (kXqWords * 4); }
 inline int stream_n_stages(int K) {
   const size_t n = ((size_t)kMaxDynSmem - stream_xq_bytes(K)) / stream_stage_bytes(K);
@@ -659,7 +669,7 @@ inline int stream_n_stages(int K) {
 }
 
 inline StreamParams stream_params_from(const GemvParams& g, int* status) {
-  const int rows = kGroupWarps / stream_parts_for(g.K) * kRPW;
+  const int rows = kGroupWarps / stream_parts_for(g.K) * stream_rpw_for(g.K);
   const bool sw = g.mode == GEMV_SWIGLU_F16;
   StreamParams p{};
   p.n_seg = g.n_seg;

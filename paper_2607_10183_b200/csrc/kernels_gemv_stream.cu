@@ -8,24 +8,28 @@ namespace {
 
 // One CTA: ring set-up, then the producer warp and the consumer warps go their ways.  dep_resolved: the caller has already
 // waited for the preceding kernel (its weight addresses come from that kernel's output).
-template <int PARTS, bool SW, bool MX>
+// SHORT: the wide-tile geometry of short rows (K <= 1024; one k-part): four rows per warp, one block per lane, four
+// producer warps.
+template <int PARTS, bool SW, bool MX, bool SHORT>
 __device__ __forceinline__ void gemv_stream_body(const StreamParams& p, const int bx, const int gx, const bool dep_resolved) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ StreamShared sh;
-  constexpr int ROWS = kGroupWarps / PARTS * kRPW;
+  constexpr int RPW = SHORT ? kRPWShort : kRPW, J = SHORT ? kJShort : kJ, PW = SHORT ? kProducerWarpsShort : kProducerWarps;
+  constexpr int ROWS = kGroupWarps / PARTS * RPW;
   const int stage_bytes = ROWS * (p.K / 2 + p.K / 16);
   stream_init(sh, p.n_stages);
   if ((threadIdx.x >> 5) >= kConsumerWarps) {
     // weights do not depend on the preceding kernel, so their copies start before the grid dependency is resolved
-    if ((threadIdx.x & 31) == 0) stream_produce<PARTS, SW>(p, bx, gx, (int)(threadIdx.x >> 5) - kConsumerWarps, sh, smem, l2_evict_first_policy());
+    if ((threadIdx.x & 31) == 0)
+      stream_produce<PARTS, SW, RPW, PW>(p, bx, gx, (int)(threadIdx.x >> 5) - kConsumerWarps, sh, smem, l2_evict_first_policy());
     return;
   }
-  stream_consume<PARTS, SW, MX>(p, bx, gx, sh, smem, reinterpret_cast<uint32_t*>(smem + (size_t)p.n_stages * stage_bytes), dep_resolved);
+  stream_consume<PARTS, SW, MX, RPW, J>(p, bx, gx, sh, smem, reinterpret_cast<uint32_t*>(smem + (size_t)p.n_stages * stage_bytes), dep_resolved);
 }
 
-template <int PARTS, bool SW, bool MX>
-__global__ void __launch_bounds__(kThreads, 1) gemv_stream_kernel(const StreamParams p) {
-  gemv_stream_body<PARTS, SW, MX>(p, (int)blockIdx.x, (int)gridDim.x, false);
+template <int PARTS, bool SW, bool MX, bool SHORT = false>
+__global__ void __launch_bounds__(SHORT ? kThreadsShort : kThreads, 1) gemv_stream_kernel(const StreamParams p) {
+  gemv_stream_body<PARTS, SW, MX, SHORT>(p, (int)blockIdx.x, (int)gridDim.x, false);
 }
 
 // Grouped-expert variant: blockIdx.y selects the job (a (token, slot) pair), whose expert slices, activation row and
@@ -42,8 +46,8 @@ struct MoeSel {
   int ldx, ldy;
   int n_experts;
 };
-template <int PARTS, bool SW, bool MX>
-__global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
+template <int PARTS, bool SW, bool MX, bool SHORT = false>
+__global__ void __launch_bounds__(SHORT ? kThreadsShort : kThreads, 1) gemv_stream_moe_kernel(const StreamParams p0, const MoeSel m, const MoeJobs jobs) {
   StreamParams p = p0;
   const int job = blockIdx.y;
   int xrow, orow;
@@ -67,7 +71,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_stream_moe_kernel(const Stre
   p.x16 = p0.x16 + (size_t)xrow * m.ldx;
   if (p0.y32) p.y32 = p0.y32 + (size_t)orow * m.ldy;
   if (p0.y16) p.y16 = p0.y16 + (size_t)orow * m.ldy;
-  gemv_stream_body<PARTS, SW, MX>(p, (int)blockIdx.x, (int)gridDim.x, m.ids != nullptr);
+  gemv_stream_body<PARTS, SW, MX, SHORT>(p, (int)blockIdx.x, (int)gridDim.x, m.ids != nullptr);
 }
 
 int parts_for(int K) { return stream_parts_for(K); }
@@ -92,7 +96,12 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
   const size_t smem = p.n_stages * stage_bytes + stream_xq_bytes(g.K);
   const int grid = std::max(1, std::min(tiles, sm_count));
   void (*kern)(const StreamParams) = nullptr;
-  if (g.mx) {
+  const bool shrt = stream_short(g.K);
+  const int producers = stream_producers_for(g.K);
+  if (shrt) {
+    if (g.mx) kern = sw ? gemv_stream_kernel<1, true, true, true> : gemv_stream_kernel<1, false, true, true>;
+    else kern = sw ? gemv_stream_kernel<1, true, false, true> : gemv_stream_kernel<1, false, false, true>;
+  } else if (g.mx) {
     switch (parts) {
       case 1: kern = sw ? gemv_stream_kernel<1, true, true> : gemv_stream_kernel<1, false, true>; break;
       case 2: kern = sw ? gemv_stream_kernel<2, true, true> : gemv_stream_kernel<2, false, true>; break;
@@ -107,16 +116,16 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
       default: kern = sw ? gemv_stream_kernel<8, true, false> : gemv_stream_kernel<8, false, false>; break;
     }
   }
-  static uint64_t attr_done[16] = {};
-  const int ki = ((parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
+  static uint64_t attr_done[20] = {};
+  const int ki = ((shrt ? 4 : parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
     cudaError_t e = set_stream_kernel_attributes(reinterpret_cast<const void*>(kern));
     if (e != cudaSuccess) return e;
   }
-  if (smem > kMaxDynSmem || p.n_stages < kProducerWarps) return cudaErrorInvalidValue;
+  if (smem > kMaxDynSmem || p.n_stages < producers) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(shrt ? kThreadsShort : kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -130,7 +139,7 @@ cudaError_t launch_gemv_stream(const GemvParams& g, int* status, int sm_count, c
 
 bool moe_gemv_stream_eligible(const MoeGemvParams& p) {
   if (p.K % 256 != 0 || p.K > 16384) return false;
-  const int rows = kGroupWarps / parts_for(p.K) * kRPW;
+  const int rows = kGroupWarps / parts_for(p.K) * stream_rpw_for(p.K);
   if (p.mode == GEMV_SWIGLU_F16) return p.n_rows % (rows / 2) == 0;
   return (p.mode == GEMV_OUT_F32 || p.mode == GEMV_OUT_F16) && p.n_rows % rows == 0;
 }
@@ -138,8 +147,9 @@ bool moe_gemv_stream_eligible(const MoeGemvParams& p) {
 cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, int* status, int sm_count, int pdl, cudaStream_t st,
                                    uint64_t* n_launch) {
   const int parts = parts_for(g.K);
-  const int rows = kGroupWarps / parts * kRPW;
+  const int rows = kGroupWarps / parts * stream_rpw_for(g.K);
   const bool sw = g.mode == GEMV_SWIGLU_F16;
+  const bool shrt = stream_short(g.K);
   const int n_jobs = jobs ? jobs->n : g.P;
   if (n_jobs <= 0) return cudaSuccess;
   StreamParams p{};
@@ -169,10 +179,13 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
   MoeJobs none;
   none.n = 0;
   const size_t smem = p.n_stages * stream_stage_bytes(g.K) + stream_xq_bytes(g.K);
-  if (smem > kMaxDynSmem || p.n_stages < kProducerWarps) return cudaErrorInvalidValue;
+  if (smem > kMaxDynSmem || p.n_stages < stream_producers_for(g.K)) return cudaErrorInvalidValue;
   const int per_job = std::max(1, std::min(p.n_tiles, sm_count / n_jobs));  // one wave: a CTA fills its SM
   void (*kern)(const StreamParams, const MoeSel, const MoeJobs) = nullptr;
-  if (g.mx) {
+  if (shrt) {
+    if (g.mx) kern = sw ? gemv_stream_moe_kernel<1, true, true, true> : gemv_stream_moe_kernel<1, false, true, true>;
+    else kern = sw ? gemv_stream_moe_kernel<1, true, false, true> : gemv_stream_moe_kernel<1, false, false, true>;
+  } else if (g.mx) {
     switch (parts) {
       case 1: kern = sw ? gemv_stream_moe_kernel<1, true, true> : gemv_stream_moe_kernel<1, false, true>; break;
       case 2: kern = sw ? gemv_stream_moe_kernel<2, true, true> : gemv_stream_moe_kernel<2, false, true>; break;
@@ -187,15 +200,15 @@ cudaError_t launch_moe_gemv_stream(const MoeGemvParams& g, const MoeJobs* jobs, 
       default: kern = sw ? gemv_stream_moe_kernel<8, true, false> : gemv_stream_moe_kernel<8, false, false>; break;
     }
   }
-  static uint64_t attr_done[16] = {};
-  const int ki = ((parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
+  static uint64_t attr_done[20] = {};
+  const int ki = ((shrt ? 4 : parts == 1 ? 0 : parts == 2 ? 1 : parts == 4 ? 2 : 3) * 2 + (sw ? 1 : 0)) * 2 + (g.mx ? 1 : 0);
   if (first_use_on_device(&attr_done[ki])) {
     cudaError_t e = set_stream_kernel_attributes(reinterpret_cast<const void*>(kern));
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(per_job, n_jobs);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(shrt ? kThreadsShort : kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];

@@ -78,8 +78,10 @@ def test_dequant_random_tensor_and_expert_slices(B, torch):
 
 
 # ------------------------------------------------------------------------------------------------- a2 GEMV
+# (64, 256), (2048, 768), (96, 1024): single rows of at most 1024 elements take the streaming kernel's wide tiles (32 rows,
+# four producer warps); (2048, 768) is the down projection of a config-4 expert
 @pytest.mark.parametrize("N,K,M", [(1, 32, 1), (3, 64, 2), (17, 96, 3), (130, 1056, 8), (257, 4096, 1), (64, 14336, 5),
-                                   (4096, 4096, 1)])
+                                   (4096, 4096, 1), (64, 256, 1), (2048, 768, 1), (96, 1024, 1)])
 def test_linear_gemv_matches_oracle(B, torch, N, K, M):
     cfg = 1 if (N, K, M) == (4096, 4096, 1) else 95
     packed, scales = W.q4_packed(cfg, 0, W.ROLE_Q, N, K)
@@ -1007,7 +1009,7 @@ def test_bounded_wait_expiry_is_reported_and_leaves_other_contexts_usable(B, tor
     the kernel's wait limit to about two milliseconds and makes the producer leave out the copies of tile 0, so the
     consumers of that tile wait in vain, give up, raise the status word and return; the other CTAs finish their rows.
     ats_sync then returns ATS_ERR_TIMEOUT and the context refuses further work; a fresh context computes correctly."""
-    N, K = 64, 256  # four tiles of 16 rows, one per CTA
+    N, K = 64, 2048  # four tiles of 16 rows (rows longer than 1024 take 16-row tiles), one per CTA
     packed, scales = W.q4_packed(93, 1, W.ROLE_Q, N, K)
     x = W.activations(93, 1, (1, K))
     want = O.linear(x, packed, scales)

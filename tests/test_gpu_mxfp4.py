@@ -65,7 +65,7 @@ def test_dequant_every_element_pair_times_every_accepted_scale(B, torch):
     ctx.close()
 
 
-@pytest.mark.parametrize("N,K,M", [(8, 32, 1), (37, 96, 3), (130, 1024, 8), (4096, 4096, 1), (256, 14336, 2), (300, 4096, 20), (1024, 1024, 129)])
+@pytest.mark.parametrize("N,K,M", [(8, 32, 1), (37, 96, 3), (130, 1024, 8), (4096, 4096, 1), (256, 14336, 2), (300, 4096, 20), (1024, 1024, 129), (2048, 768, 1), (64, 256, 1)])
 def test_linear_matches_oracle_gemv_and_gemm(B, torch, N, K, M):
     """Up to 8 rows: the generic GEMV (fp32 accumulation of exact products); more: the tcgen05 GEMM with the weight tile
     dequantized in the kernel (weights exact in fp16).  Streamed through the ring = resident, bit for bit."""
