@@ -711,9 +711,13 @@ def test_gate_up_both_streamed_needs_two_slots(B, torch):
 
 
 # ------------------------------------------------------------------------------------------------- a4 routing, a5 MoE
-def test_route_topk_bit_exact_with_ties(B, torch):
+# (hidden, experts, k): the cluster kernel with the selection by counting ranks (up to 256 experts, incl. exactly 256), the
+# cluster kernel with the warp argmax (more experts), the one-CTA kernel (shapes the cluster form does not take), and the
+# largest router the library accepts
+@pytest.mark.parametrize("Hd,E,k", [(128, 48, 6), (128, 256, 8), (128, 264, 8), (100, 50, 6), (256, 1024, 32)])
+def test_route_topk_bit_exact_with_ties(B, torch, Hd, E, k):
     rng = np.random.default_rng(11)
-    Hd, E, k, M = 128, 48, 6, 9
+    M = 9
     Wr = rng.normal(0, 0.02, size=(Hd, E)).astype(np.float16)
     Wr[:, 9] = Wr[:, 2]
     Wr[:, 40] = Wr[:, 2]  # exact ties: equal columns give bitwise equal logits in any summation order
@@ -721,7 +725,7 @@ def test_route_topk_bit_exact_with_ties(B, torch):
     h[0] = (Wr[:, 2].astype(np.float32) * 50).astype(np.float16)  # token 0 ranks the tied experts first
     ids_ref, gates_ref, logits = O.route_topk(h, Wr, k)
     assert ids_ref[0, :3].tolist() == [2, 9, 40]
-    ctx = make_ctx(B, 64 * 1024)
+    ctx = make_ctx(B, MB)
     rid = ctx.register_f16(Wr)
     ctx.set_placement([])
     ids = torch.empty((M, k), dtype=torch.int32, device="cuda")
@@ -927,6 +931,52 @@ def test_errors_are_statuses_and_context_stays_usable(B, torch):
 
 
 # ------------------------------------------------------------------------------------------------- failure paths
+def test_empty_calls_and_longest_rows(B, torch):
+    """Degenerate and maximal sizes: calls over zero rows / tokens succeed and write nothing; the longest row the streaming
+    kernel takes (16384 elements) and the next longer one (which the generic kernel takes) both match the oracle."""
+    N, K = 64, 256
+    packed, scales = W.q4_packed(94, 0, W.ROLE_Q, N, K)
+    ctx = make_ctx(B, 4 * MB)
+    tid = ctx.register_q4(packed, scales)
+    rid = ctx.register_f16(np.zeros((K, 8), dtype=np.float16))
+    ctx.set_placement([(tid, -1, B.ATS_GPU)])
+    x = torch.zeros((1, K), dtype=torch.float16, device="cuda")
+    y = torch.full((1, N), 7.0, dtype=torch.float16, device="cuda")
+    ids = torch.full((1, 2), -5, dtype=torch.int32, device="cuda")
+    gates = torch.full((1, 2), 3.0, dtype=torch.float32, device="cuda")
+    ctx.linear(tid, x, y, 0)
+    ctx.route_topk(rid, x, 0, 2, ids, gates)
+    ctx.sync()
+    assert (y.cpu().numpy() == 7.0).all() and (ids.cpu().numpy() == -5).all() and (gates.cpu().numpy() == 3.0).all()
+    ctx.close()
+    shape = W.DENSE_SMALL
+    L = W.dense_layer(96, 0, shape)
+    ctx = make_ctx(B, H.dense_layer_bytes(shape) + 64 * 1024, ws=8 * MB)
+    desc, lids = H.register_dense_layer(ctx, L, 0, 16)
+    ctx.set_placement([(lids[n], -1, B.ATS_GPU) for n in ALL_GPU])
+    kd = torch.zeros((shape.n_kv_heads, 16, shape.head_dim), dtype=torch.float16, device="cuda")
+    vd = torch.zeros_like(kd)
+    xa = torch.zeros((1, shape.hidden), dtype=torch.float16, device="cuda")
+    ya = torch.full((1, shape.hidden), 7.0, dtype=torch.float16, device="cuda")
+    ctx.layer_decode(desc, xa, ya, kd, vd, 0, 0)
+    ctx.layer_prefill(desc, xa, ya, kd, vd, 0, 0)
+    ctx.sync()
+    assert (ya.cpu().numpy() == 7.0).all() and not kd.cpu().numpy().any() and not vd.cpu().numpy().any()
+    ctx.close()
+    for K2 in (16384, 16384 + 256):
+        N2 = 32
+        p2, s2 = W.q4_packed(94, 1, W.ROLE_Q, N2, K2)
+        x2 = W.activations(94, 1, (1, K2))
+        ctx = make_ctx(B, W.q4_bytes(N2, K2) + 64 * 1024)
+        t2 = ctx.register_q4(p2, s2)
+        ctx.set_placement([(t2, -1, B.ATS_GPU)])
+        y2 = torch.empty((1, N2), dtype=torch.float16, device="cuda")
+        ctx.linear(t2, H.to_dev(x2), y2, 1)
+        ctx.sync()
+        H.assert_close(y2.cpu().numpy(), O.linear(x2, p2, s2, round_out=True), what=f"gemv over rows of {K2} elements")
+        ctx.close()
+
+
 def test_gemv_non_finite_activation_gives_non_finite_output(B, torch):
     """An Inf or a NaN among the activations must not turn into a finite output: the streaming kernel's fixed-point operand
     cannot carry it, so the block's term becomes NaN (the plain definition gives Inf or NaN in every row here, since every
