@@ -792,9 +792,10 @@ cudaError_t launch_attn_decode_fused(AttnDecodeParams p, int d, int pdl, cudaStr
   if (p.group * pc > 512) pc = 64;  // large groups: 64 positions keep the CTA within 512 threads
   const int splits = (p.pos + 1 + pc - 1) / pc;
   // Short contexts give fewer jobs than SMs: the query heads of a group are then divided over 2 or 4 CTAs (each stages
-  // the same cache rows out of L2), which shortens the score and value loops of every CTA in proportion.
+  // the same cache rows out of L2), up to two CTAs per SM: the launch is a chain of latencies, and more, smaller CTAs
+  // overlap more of them (config-2 step, 1025 positions: 37.3 us with 72 CTAs, 37.1 with 144, 36.6 with 288).
   int hsplit = 1;
-  while (p.group % (2 * hsplit) == 0 && splits * p.n_kv * 2 * hsplit <= 148 && p.n_kv * 2 * hsplit <= kAttnMaxCounters) hsplit *= 2;
+  while (p.group % (2 * hsplit) == 0 && splits * p.n_kv * 2 * hsplit <= 2 * 148 && p.n_kv * 2 * hsplit <= kAttnMaxCounters) hsplit *= 2;
   p.hsplit = hsplit;
   p.scale = 1.0f / sqrtf((float)d);
   cudaLaunchConfig_t cfg{};
